@@ -1,0 +1,8 @@
+"""CPU oracle for the PWLQ hot path -- test infrastructure only.
+
+Only the tests, the smoke check and the benchmark's CPU-baseline leg import
+this package.  It shares no code with the CUDA path.
+"""
+from .pwlq_oracle import (  # noqa: F401
+    OracleError, OracleLib, absmax, build, code_bytes, dequantize, elem, params, quantize, search,
+)

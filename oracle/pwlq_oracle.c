@@ -1,0 +1,245 @@
+/*
+ * PWLQ CPU oracle -- TEST INFRASTRUCTURE, not part of the product path.
+ *
+ * A plain, single-threaded, deliberately slow restatement of the piecewise
+ * linear quantizer (Eq. 3) built on the uniform quantizer (Eq. 1), the
+ * empirical squared quantization error (the error eps_pw = pw(r) - r defined
+ * under Eq. 3), and the argmin over breakpoints (Eq. 6) restricted to a
+ * user-supplied grid of K candidate ratios p/m.
+ *
+ * Only the tests, the smoke check and the benchmark's CPU-baseline leg may
+ * call this file.  It shares no code with the CUDA path.
+ *
+ * Arithmetic: every per-element quantity is IEEE binary32, one rounding per
+ * operation, no fused multiply-add (compile with -ffp-contract=off); the
+ * integer code is decided in binary32 so that it means the same thing on the
+ * CPU and on the GPU.  Sums of squared errors are accumulated in binary64 in
+ * ascending element order.
+ *
+ * Pinned by tests/test_oracle_*.py: a hand-worked dyadic example (Eq. 1, 3),
+ * the half-step error bound implied by Eq. 2, the p = m and p = m/2 special
+ * cases, an independent binary64 true-division brute force on <= 64 elements,
+ * and the closed forms Eq. 5, Eq. 9, Eq. 10 and Lemma 2 on Gaussian and
+ * Laplacian samples.
+ *
+ * Readings of the paper taken here (each listed with its reason in the
+ * project's design notes):
+ *   - clamp(r; rl, ru) = min(max(r, rl), ru)       (Eq. 1 prints the bounds swapped)
+ *   - rounding is round-half-to-even               (Eq. 1 leaves the tie rule open)
+ *   - s = Delta / (2^(b-1) - 1) inside every piece ((b-1)-bit pieces, Sec. 3.2)
+ *   - the center region is closed: tail iff |r| > p (R1 = [-p, p])
+ *   - (r - z) / s is evaluated as (|r| - z) * fl(L / Delta)
+ *   - the stored integer is sign-magnitude: sign bit, then the (b-1)-bit level
+ */
+#include <math.h>
+#include <stdint.h>
+#include <stddef.h>
+
+#define ORACLE_OK 0
+#define ORACLE_ERR_ARG 1
+#define ORACLE_ERR_NONFINITE 5
+
+typedef struct {
+    float Lf;   /* largest level of a (b-1)-bit piece, 2^(b-1) - 1 (Eq. 1: N - 1) */
+    float s1;   /* step of the center pieces, p / L                               */
+    float inv1; /* L / p                                                          */
+    float s2;   /* step of the tail pieces, (m - p) / L                           */
+    float inv2; /* L / (m - p)                                                    */
+} pw_params;
+
+/* Eq. 1, last line: s = Delta / (N - 1) with N = 2^(b-1) per piece (Sec. 3.2);
+ * Delta = p for the center (range [0, p]) and m - p for the tail (range [p, m]).
+ * An empty piece (Delta <= 0) gets step 0. */
+static pw_params make_params(float m, float p, int bits)
+{
+    pw_params P;
+    float d;
+    P.Lf = (float)((1 << (bits - 1)) - 1);
+    if (p > 0.0f) { P.s1 = p / P.Lf; P.inv1 = P.Lf / p; }
+    else          { P.s1 = 0.0f;     P.inv1 = 0.0f; }
+    d = m - p;
+    if (d > 0.0f) { P.s2 = d / P.Lf; P.inv2 = P.Lf / d; }
+    else          { P.s2 = 0.0f;     P.inv2 = 0.0f; }
+    return P;
+}
+
+/* Eq. 3 applied to one value: returns the reconstructed magnitude v and writes
+ * the level q, the region (1 = tail) and the clamped magnitude a. */
+static float pw_elem(float x, float m, float p, const pw_params *P,
+                     int *q_out, int *region_out, float *a_out)
+{
+    float a = fminf(fabsf(x), m);          /* clamp(|r|; 0, m), Eq. 1           */
+    int tail = (a > p);                    /* R2 = (p, m], Sec. 3.2             */
+    float z = tail ? p : 0.0f;             /* offsets 0 and p, Eq. 3            */
+    float inv = tail ? P->inv2 : P->inv1;
+    float s = tail ? P->s2 : P->s1;
+    float u = a - z;
+    float t = u * inv;                     /* (clamp - z) / s                   */
+    float q = fminf(rintf(t), P->Lf);      /* round half to even, saturate      */
+    float v = q * s;                       /* s * r_q ...                       */
+    v = v + z;                             /* ... + z, Eq. 1 first line         */
+    *q_out = (int)q;
+    *region_out = tail;
+    *a_out = a;
+    return v;
+}
+
+static int64_t row_begin(const int64_t *row_offsets, int64_t n, int64_t c)
+{
+    return row_offsets ? row_offsets[c] : c * n;
+}
+
+/* Range [-m, m] of Sec. 3.2: m_c = max_i |x_{c,i}| for every row. */
+int pwlq_oracle_absmax(const float *x, const int64_t *row_offsets, int64_t C, int64_t n,
+                       float *m_out)
+{
+    int64_t c, i;
+    if (!x || !m_out || C < 1) return ORACLE_ERR_ARG;
+    for (c = 0; c < C; ++c) {
+        int64_t b = row_begin(row_offsets, n, c), e = row_begin(row_offsets, n, c + 1);
+        float m = 0.0f;
+        for (i = b; i < e; ++i) {
+            float a = fabsf(x[i]);
+            if (!(a <= 3.402823466e+38f)) return ORACLE_ERR_NONFINITE;
+            if (a > m) m = a;
+        }
+        m_out[c] = m;
+    }
+    return ORACLE_OK;
+}
+
+/* Empirical counterpart of Eq. 6 on a grid: for every row and every candidate
+ * p_k = m * ratios[k], SSE_k = sum_i (pw(x_i) - x_i)^2; pick the first minimal k.
+ * sse_f32 / sse_f64 (either may be NULL) receive all C*K sums. */
+int pwlq_oracle_search(const float *x, const int64_t *row_offsets, int64_t C, int64_t n,
+                       int bits, const float *ratios, int K, const float *m_in,
+                       float *p_out, float *err_out, int32_t *idx_out,
+                       float *sse_f32, double *sse_f64)
+{
+    int64_t c, i;
+    int k;
+    if (!x || !ratios || C < 1 || K < 1 || bits < 2 || bits > 8) return ORACLE_ERR_ARG;
+    for (c = 0; c < C; ++c) {
+        int64_t b = row_begin(row_offsets, n, c), e = row_begin(row_offsets, n, c + 1);
+        float m = 0.0f;
+        double best = 0.0;
+        int best_k = 0;
+        if (m_in) m = m_in[c];
+        else for (i = b; i < e; ++i) {
+            float a = fabsf(x[i]);
+            if (!(a <= 3.402823466e+38f)) return ORACLE_ERR_NONFINITE;
+            if (a > m) m = a;
+        }
+        if (!(m <= 3.402823466e+38f)) return ORACLE_ERR_NONFINITE;
+        for (k = 0; k < K; ++k) {
+            double sse = 0.0;
+            if (m > 0.0f) {
+                float p = m * ratios[k];
+                pw_params P = make_params(m, p, bits);
+                for (i = b; i < e; ++i) {
+                    int q, r; float a;
+                    float v = pw_elem(x[i], m, p, &P, &q, &r, &a);
+                    double d = (double)v - (double)a;   /* eps_pw up to sign(r) */
+                    sse += d * d;
+                }
+            }
+            if (sse_f32) sse_f32[c * (int64_t)K + k] = (float)sse;
+            if (sse_f64) sse_f64[c * (int64_t)K + k] = sse;
+            if (k == 0 || sse < best) { best = sse; best_k = k; }
+        }
+        if (idx_out) idx_out[c] = best_k;
+        if (p_out)   p_out[c] = (m > 0.0f) ? m * ratios[best_k] : 0.0f;
+        if (err_out) err_out[c] = (float)best;
+    }
+    return ORACLE_OK;
+}
+
+/* Eq. 3 with the chosen (m, p) of each row: b-bit sign-magnitude code, region
+ * bit (Sec. 4: one extra bit per value), optional reconstructed value.
+ * layout 0: one byte per code.  layout 1: for bits <= 4 two codes per byte,
+ * flat element 2j in the low nibble; for bits > 4 identical to layout 0.
+ * region_mask: bit (i & 7) of byte (i >> 3), i the flat element index. */
+int pwlq_oracle_quantize(const float *x, const int64_t *row_offsets, int64_t C, int64_t n,
+                         int bits, const float *m_in, const float *p_in,
+                         uint8_t *codes, uint8_t *region_mask, float *fake_out, int layout)
+{
+    int64_t c, i, total;
+    int packed = (layout == 1 && bits <= 4);
+    if (!x || !m_in || !p_in || C < 1 || bits < 2 || bits > 8) return ORACLE_ERR_ARG;
+    total = row_begin(row_offsets, n, C);
+    if (codes)       for (i = 0; i < (packed ? (total + 1) / 2 : total); ++i) codes[i] = 0;
+    if (region_mask) for (i = 0; i < (total + 7) / 8; ++i) region_mask[i] = 0;
+    for (c = 0; c < C; ++c) {
+        int64_t b = row_begin(row_offsets, n, c), e = row_begin(row_offsets, n, c + 1);
+        float m = m_in[c], p = p_in[c];
+        pw_params P = make_params(m, p, bits);
+        for (i = b; i < e; ++i) {
+            int q = 0, r = 0, neg = 0, code;
+            float a, v = 0.0f, y;
+            if (m > 0.0f) {
+                neg = (x[i] < 0.0f);
+                v = pw_elem(x[i], m, p, &P, &q, &r, &a);
+            }
+            code = (neg << (bits - 1)) | q;
+            y = neg ? -v : v;                       /* sign(r) * uni(|r|; ...) */
+            if (codes) {
+                if (packed) codes[i >> 1] |= (uint8_t)(code << ((i & 1) * 4));
+                else        codes[i] = (uint8_t)code;
+            }
+            if (region_mask && r) region_mask[i >> 3] |= (uint8_t)(1u << (i & 7));
+            if (fake_out) fake_out[i] = y;
+        }
+    }
+    return ORACLE_OK;
+}
+
+/* Eq. 1 first line, r_hat = s * r_q + z, with (s, z) of the stored region. */
+int pwlq_oracle_dequantize(const uint8_t *codes, const uint8_t *region_mask,
+                           const int64_t *row_offsets, int64_t C, int64_t n, int bits,
+                           const float *m_in, const float *p_in, float *y, int layout)
+{
+    int64_t c, i;
+    int packed = (layout == 1 && bits <= 4);
+    int qmask = (1 << (bits - 1)) - 1;
+    if (!codes || !region_mask || !m_in || !p_in || !y || C < 1 || bits < 2 || bits > 8)
+        return ORACLE_ERR_ARG;
+    for (c = 0; c < C; ++c) {
+        int64_t b = row_begin(row_offsets, n, c), e = row_begin(row_offsets, n, c + 1);
+        float m = m_in[c], p = p_in[c];
+        pw_params P = make_params(m, p, bits);
+        for (i = b; i < e; ++i) {
+            int code = packed ? ((codes[i >> 1] >> ((i & 1) * 4)) & 0xF) : codes[i];
+            int r = (region_mask[i >> 3] >> (i & 7)) & 1;
+            int neg = (code >> (bits - 1)) & 1;
+            float q = (float)(code & qmask);
+            float s = r ? P.s2 : P.s1;
+            float z = r ? p : 0.0f;
+            float v = q * s;
+            v = v + z;
+            if (!(m > 0.0f)) { v = 0.0f; neg = 0; }
+            y[i] = neg ? -v : v;
+        }
+    }
+    return ORACLE_OK;
+}
+
+/* One value, for hand-checkable tests: returns code, region, q and y. */
+void pwlq_oracle_elem(float x, float m, float p, int bits,
+                      int *code_out, int *region_out, int *q_out, float *y_out)
+{
+    pw_params P = make_params(m, p, bits);
+    int q = 0, r = 0, neg = 0;
+    float a, v = 0.0f;
+    if (m > 0.0f) { neg = (x < 0.0f); v = pw_elem(x, m, p, &P, &q, &r, &a); }
+    *code_out = (neg << (bits - 1)) | q;
+    *region_out = r;
+    *q_out = q;
+    *y_out = neg ? -v : v;
+}
+
+/* The five per-(row, candidate) constants, for tests of Eq. 1's step. */
+void pwlq_oracle_params(float m, float p, int bits, float *out5)
+{
+    pw_params P = make_params(m, p, bits);
+    out5[0] = P.Lf; out5[1] = P.s1; out5[2] = P.inv1; out5[3] = P.s2; out5[4] = P.inv2;
+}

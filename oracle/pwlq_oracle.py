@@ -1,0 +1,191 @@
+"""ctypes front end of ``pwlq_oracle.c`` (test infrastructure, not product code).
+
+The C file is the oracle; this module only compiles it with gcc
+(``-O2 -ffp-contract=off``, no fast-math, so every binary32 operation rounds
+once) and marshals numpy arrays.  Rows are either a dense ``[C, n]`` view or a
+ragged set given by ``row_offsets`` (``C + 1`` ascending flat offsets).
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+import subprocess
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "pwlq_oracle.c")
+_SO = os.path.join(_HERE, "libpwlq_oracle.so")
+
+
+class OracleError(RuntimeError):
+    pass
+
+
+def _compile(src: str, so: str) -> None:
+    cmd = ["gcc", "-std=c99", "-O2", "-ffp-contract=off", "-fno-fast-math",
+           "-fPIC", "-shared", "-o", so, src, "-lm"]
+    subprocess.run(cmd, check=True)
+
+
+def build(force: bool = False) -> str:
+    """Compile the oracle if the shared object is missing or older than its source."""
+    if force or not os.path.exists(_SO) or os.path.getmtime(_SO) < os.path.getmtime(_SRC):
+        _compile(_SRC, _SO)
+    return _SO
+
+
+def _ptr(a):
+    return None if a is None else a.ctypes.data_as(ctypes.c_void_p)
+
+
+def _rows(x, row_offsets):
+    """Returns (flat fp32 array, offsets array or None, C, n)."""
+    x = np.ascontiguousarray(x, dtype=np.float32)
+    if row_offsets is None:
+        if x.ndim == 1:
+            x = x.reshape(1, -1)
+        x2 = x.reshape(x.shape[0], -1)
+        return x2.reshape(-1), None, x2.shape[0], x2.shape[1]
+    ro = np.ascontiguousarray(row_offsets, dtype=np.int64)
+    flat = x.reshape(-1)
+    assert ro[0] == 0 and ro[-1] == flat.size and np.all(np.diff(ro) >= 0)
+    return flat, ro, ro.size - 1, 0
+
+
+def _check(rc, what):
+    if rc != 0:
+        raise OracleError(f"{what}: status {rc}")
+
+
+def code_bytes(total, bits, layout):
+    return (total + 1) // 2 if (layout == 1 and bits <= 4) else total
+
+
+class OracleLib:
+    """One compiled copy of the oracle.  ``OracleLib()`` is the oracle itself; the tests also load
+    deliberately broken copies through ``so_path`` to show that the pins notice them."""
+
+    OracleError = OracleError
+
+    def __init__(self, so_path: str | None = None):
+        lib = ctypes.CDLL(so_path or build())
+        P = ctypes.c_void_p
+        I64 = ctypes.c_int64
+        lib.pwlq_oracle_absmax.argtypes = [P, P, I64, I64, P]
+        lib.pwlq_oracle_search.argtypes = [P, P, I64, I64, ctypes.c_int, P, ctypes.c_int, P,
+                                           P, P, P, P, P]
+        lib.pwlq_oracle_quantize.argtypes = [P, P, I64, I64, ctypes.c_int, P, P, P, P, P,
+                                             ctypes.c_int]
+        lib.pwlq_oracle_dequantize.argtypes = [P, P, P, I64, I64, ctypes.c_int, P, P, P,
+                                               ctypes.c_int]
+        lib.pwlq_oracle_elem.argtypes = [ctypes.c_float, ctypes.c_float, ctypes.c_float,
+                                         ctypes.c_int, P, P, P, P]
+        lib.pwlq_oracle_elem.restype = None
+        lib.pwlq_oracle_params.argtypes = [ctypes.c_float, ctypes.c_float, ctypes.c_int, P]
+        lib.pwlq_oracle_params.restype = None
+        self._lib = lib
+
+    def absmax(self, x, row_offsets=None):
+        flat, ro, C, n = _rows(x, row_offsets)
+        m = np.empty(C, dtype=np.float32)
+        _check(self._lib.pwlq_oracle_absmax(_ptr(flat), _ptr(ro), C, n, _ptr(m)), "absmax")
+        return m
+
+    def search(self, x, bits, ratios, m=None, row_offsets=None, want_sse=True):
+        """Returns dict(p, err, idx, sse (float32 [C,K]), sse64 (float64 [C,K]))."""
+        flat, ro, C, n = _rows(x, row_offsets)
+        ratios = np.ascontiguousarray(ratios, dtype=np.float32)
+        K = int(ratios.size)
+        if m is not None:
+            m = np.ascontiguousarray(m, dtype=np.float32)
+            assert m.size == C
+        p = np.empty(C, dtype=np.float32)
+        err = np.empty(C, dtype=np.float32)
+        idx = np.empty(C, dtype=np.int32)
+        sse = np.empty((C, K), dtype=np.float32) if want_sse else None
+        sse64 = np.empty((C, K), dtype=np.float64) if want_sse else None
+        _check(self._lib.pwlq_oracle_search(_ptr(flat), _ptr(ro), C, n, int(bits), _ptr(ratios),
+                                            K, _ptr(m), _ptr(p), _ptr(err), _ptr(idx),
+                                            _ptr(sse), _ptr(sse64)), "search")
+        return {"p": p, "err": err, "idx": idx, "sse": sse, "sse64": sse64}
+
+    def quantize(self, x, bits, m, p, layout=0, row_offsets=None, want_fake=True):
+        """Returns (codes uint8, region_mask uint8, fake fp32 or None)."""
+        flat, ro, C, n = _rows(x, row_offsets)
+        total = flat.size
+        m = np.ascontiguousarray(m, dtype=np.float32)
+        p = np.ascontiguousarray(p, dtype=np.float32)
+        assert m.size == C and p.size == C
+        codes = np.empty(code_bytes(total, bits, layout), dtype=np.uint8)
+        mask = np.empty((total + 7) // 8, dtype=np.uint8)
+        fake = np.empty(total, dtype=np.float32) if want_fake else None
+        _check(self._lib.pwlq_oracle_quantize(_ptr(flat), _ptr(ro), C, n, int(bits), _ptr(m),
+                                              _ptr(p), _ptr(codes), _ptr(mask), _ptr(fake),
+                                              int(layout)), "quantize")
+        return codes, mask, fake
+
+    def dequantize(self, codes, mask, bits, m, p, C=None, n=None, layout=0, row_offsets=None):
+        codes = np.ascontiguousarray(codes, dtype=np.uint8)
+        mask = np.ascontiguousarray(mask, dtype=np.uint8)
+        m = np.ascontiguousarray(m, dtype=np.float32)
+        p = np.ascontiguousarray(p, dtype=np.float32)
+        if row_offsets is not None:
+            ro = np.ascontiguousarray(row_offsets, dtype=np.int64)
+            C, n, total = ro.size - 1, 0, int(ro[-1])
+        else:
+            ro, total = None, int(C) * int(n)
+        assert m.size == C and p.size == C
+        y = np.empty(total, dtype=np.float32)
+        _check(self._lib.pwlq_oracle_dequantize(_ptr(codes), _ptr(mask), _ptr(ro), C, n,
+                                                int(bits), _ptr(m), _ptr(p), _ptr(y),
+                                                int(layout)), "dequantize")
+        return y
+
+    def elem(self, x, m, p, bits):
+        """One value through Eq. 3: returns (code, region, q, y)."""
+        code, region, q = ctypes.c_int(), ctypes.c_int(), ctypes.c_int()
+        y = ctypes.c_float()
+        self._lib.pwlq_oracle_elem(float(x), float(m), float(p), int(bits), ctypes.byref(code),
+                                   ctypes.byref(region), ctypes.byref(q), ctypes.byref(y))
+        return code.value, region.value, q.value, y.value
+
+    def params(self, m, p, bits):
+        """(L, s1, inv1, s2, inv2) as binary32 values."""
+        out = np.empty(5, dtype=np.float32)
+        self._lib.pwlq_oracle_params(float(m), float(p), int(bits), _ptr(out))
+        return out
+
+
+_default = None
+
+
+def _get() -> OracleLib:
+    global _default
+    if _default is None:
+        _default = OracleLib()
+    return _default
+
+
+def absmax(*a, **k):
+    return _get().absmax(*a, **k)
+
+
+def search(*a, **k):
+    return _get().search(*a, **k)
+
+
+def quantize(*a, **k):
+    return _get().quantize(*a, **k)
+
+
+def dequantize(*a, **k):
+    return _get().dequantize(*a, **k)
+
+
+def elem(*a, **k):
+    return _get().elem(*a, **k)
+
+
+def params(*a, **k):
+    return _get().params(*a, **k)
