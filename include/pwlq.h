@@ -1,0 +1,148 @@
+/*
+ * pwlq.h -- C ABI of the PWLQ hot path for NVIDIA B200 (sm_100a).
+ *
+ * The library implements the data-parallel part of post-training piecewise
+ * linear quantization (arXiv 2002.00104): the range m of every row (Sec. 3.2),
+ * an empirical breakpoint search that evaluates the b-bit piecewise quantizer
+ * pw(r; b, m, p) of Eq. 3 for K candidate breakpoints p and keeps the one with
+ * the smallest squared error (the grid counterpart of Eq. 6), the quantizer
+ * itself (integer code + region bit, Sec. 4) and its inverse (Eq. 1, first line).
+ *
+ * Rows.  A tensor is viewed as C rows ("channels": per-output-channel weights,
+ * or one row for a per-layer tensor, Sec. 5).  The dense calls take a row-major
+ * [C, n] array; the *_ragged calls take rows of different lengths stored back
+ * to back, described by row_offsets[C + 1] (ascending flat element offsets,
+ * row_offsets[0] = 0, row_offsets[C] = total).  Flat index i = position in
+ * that storage.
+ *
+ * Arithmetic.  All values are IEEE binary32.  With L = 2^(bits-1) - 1, for a row
+ * with range m and breakpoint p:
+ *     s1 = p / L, inv1 = L / p, d = m - p, s2 = d / L, inv2 = L / d
+ *     (a piece whose range is not positive gets s = inv = 0),
+ *     a = min(|x|, m); tail = a > p; (z, s, inv) = tail ? (p, s2, inv2) : (0, s1, inv1);
+ *     q = min(rint((a - z) * inv), L)   (round half to even);  v = (q * s) + z,
+ * one rounding per operation, no fused multiply-add.  code = (x < 0) << (bits-1) | q,
+ * region = tail, y = (x < 0) ? -v : v.  Rows with m == 0 give code 0, region 0, y = +0.
+ * Quantize and dequantize follow this sequence exactly; the search may fuse
+ * operations (its sums agree with the sequence above to about 1e-6 relative).
+ *
+ * Pointers.  Unless a parameter says "host", every pointer is a DEVICE pointer
+ * owned by the caller, valid on the device that is current at the call; fp32 and
+ * int32 arrays need 4-byte alignment, int64 and workspace 8 / 256 bytes.  The
+ * library keeps no state between calls and allocates no memory (the *_host
+ * call included: it works in caller-provided device scratch).
+ *
+ * Execution.  Every call only enqueues work on `stream` (a cudaStream_t passed
+ * as void*, NULL = default stream) and returns; results are valid after the
+ * stream is synchronised.  Argument errors are reported by the return value
+ * with nothing enqueued.  Conditions found on the device (a non-finite range)
+ * are OR-ed into a 32-bit status word as bit (1 << code): the first 4 bytes of
+ * the search workspace, cleared by the call itself.
+ */
+#ifndef PWLQ_H_
+#define PWLQ_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+enum {
+    PWLQ_OK = 0,
+    PWLQ_ERR_INVALID_ARG = 1, /* null pointer, bits outside [2,8], C/n/K < 1, misaligned pointer */
+    PWLQ_ERR_UNSUPPORTED = 2, /* K or a size above the documented limit                       */
+    PWLQ_ERR_WORKSPACE = 3,   /* workspace missing or smaller than the *_workspace_bytes value  */
+    PWLQ_ERR_CUDA = 4,        /* a CUDA runtime call failed (launch configuration, stream, ...) */
+    PWLQ_ERR_NONFINITE = 5,   /* device status, bit 1 << 5: a row's range is Inf or NaN          */
+    PWLQ_ERR_TIMEOUT = 6      /* device status, bit 1 << 6: a bounded wait expired               */
+};
+
+enum {
+    PWLQ_CODES_U8 = 0,    /* one byte per value: low `bits` bits = sign << (bits-1) | q          */
+    PWLQ_CODES_PACKED = 1 /* bits <= 4: two values per byte, flat element 2j in the low nibble,
+                             (total+1)/2 bytes; bits > 4: same as PWLQ_CODES_U8                  */
+};
+
+#define PWLQ_MAX_K 4096 /* largest number of candidate breakpoints per search */
+
+/* Range of Sec. 3.2: m_out[c] = max_i |x[c, i]| (0 for an empty or all-zero row).  Exact
+ * (order-free integer maximum of the magnitude bits).  x: [C, n].  m_out: [C]. */
+int pwlq_absmax(const float* x, int64_t C, int64_t n, float* m_out, void* stream);
+/* Same for ragged rows.  total = row_offsets[C] (known to the host). */
+int pwlq_absmax_ragged(const float* x, const int64_t* row_offsets, int64_t C, int64_t total,
+                       float* m_out, void* stream);
+
+/* Bytes of device workspace pwlq_search needs for C rows of at most n values and K candidates
+ * (for the ragged call pass n = the longest row).  Returns 0 for invalid arguments. */
+size_t pwlq_search_workspace_bytes(int64_t C, int64_t n, int K);
+
+/* Breakpoint search, the grid form of Eq. 6 on the empirical error of Eq. 3.  For every row c
+ * and candidate k: p_k = m[c] * ratios[k] (one multiply), SSE[c,k] = sum_i (v_i - a_i)^2 over the
+ * row; idx_out[c] = smallest k attaining the minimum, p_out[c] = p_idx, err_out[c] = SSE[c,idx].
+ *   bits      b of the b-bit scheme, 2..8 (Sec. 3.2 requires b >= 2)
+ *   ratios    [K] candidate p/m in (0, 1], ascending; K in [1, PWLQ_MAX_K]
+ *   m         [C] ranges, or NULL: computed by the call (as pwlq_absmax) into the workspace
+ *   p_out, err_out, idx_out   [C] each; err_out may be NULL
+ *   sse_all   [C*K] row-major, or NULL
+ *   workspace at least pwlq_search_workspace_bytes(...), 256-byte aligned; its first 4 bytes
+ *             receive the device status (0, or 1 << PWLQ_ERR_NONFINITE) after the stream has run
+ * Rows with m == 0: idx 0, p 0, err 0.  Rows with a non-finite m: idx 0, p = err = 0, status set.
+ * Sums are formed in a fixed order: results are bit-reproducible from run to run. */
+int pwlq_search(const float* x, int64_t C, int64_t n, int bits, const float* ratios, int K,
+                const float* m, float* p_out, float* err_out, int32_t* idx_out, float* sse_all,
+                void* workspace, size_t workspace_bytes, void* stream);
+/* Same for ragged rows; max_n = longest row, total = row_offsets[C] (both known to the host). */
+int pwlq_search_ragged(const float* x, const int64_t* row_offsets, int64_t C, int64_t total,
+                       int64_t max_n, int bits, const float* ratios, int K, const float* m,
+                       float* p_out, float* err_out, int32_t* idx_out, float* sse_all,
+                       void* workspace, size_t workspace_bytes, void* stream);
+
+/* Quantizer of Eq. 3 with the chosen (m[c], p[c]) of each row, 0 < p <= m.
+ *   codes        PWLQ_CODES_U8: total bytes; PWLQ_CODES_PACKED and bits <= 4: (total+1)/2 bytes
+ *   region_mask  (total+7)/8 bytes; value i is bit (i & 7) of byte (i >> 3); 1 = tail region
+ *                (the one extra bit per value of Sec. 4); unused bits of the last byte are 0
+ *   fake_out     [total] reconstructed values y, or NULL
+ * Every output byte is written (no pre-clearing needed). */
+int pwlq_quantize(const float* x, int64_t C, int64_t n, int bits, const float* m, const float* p,
+                  uint8_t* codes, uint8_t* region_mask, float* fake_out, int code_layout,
+                  void* stream);
+int pwlq_quantize_ragged(const float* x, const int64_t* row_offsets, int64_t C, int64_t total,
+                         int bits, const float* m, const float* p, uint8_t* codes,
+                         uint8_t* region_mask, float* fake_out, int code_layout, void* stream);
+
+/* Inverse map, Eq. 1 first line: y = +-(q * s_region + z_region), z in {0, p} (Eq. 3, Sec. 4).
+ * Bit-identical to the fake_out of pwlq_quantize for the same (m, p). */
+int pwlq_dequantize(const uint8_t* codes, const uint8_t* region_mask, int64_t C, int64_t n,
+                    int bits, const float* m, const float* p, float* y, int code_layout,
+                    void* stream);
+int pwlq_dequantize_ragged(const uint8_t* codes, const uint8_t* region_mask,
+                           const int64_t* row_offsets, int64_t C, int64_t total, int bits,
+                           const float* m, const float* p, float* y, int code_layout,
+                           void* stream);
+
+/* Whole path from HOST buffers: copies x (and row_offsets, ratios) to the device, runs abs-max,
+ * search, quantize and dequantize there, and copies m, p, err, idx, codes and region_mask back.
+ * All *_host pointers are host memory (pinned memory makes the copies asynchronous); NULL
+ * row_offsets_host means dense [C, n] with n = total / C.  dev_scratch is device memory of at
+ * least pwlq_encode_host_scratch_bytes(...) bytes, 256-byte aligned.  The call returns after
+ * enqueueing; the host outputs are valid once `stream` is synchronised.  The dequantized tensor
+ * stays in dev_scratch (offset reported through y_dev_out when non-NULL). */
+size_t pwlq_encode_host_scratch_bytes(int64_t C, int64_t total, int64_t max_n, int K);
+int pwlq_encode_host(const float* x_host, const int64_t* row_offsets_host, int64_t C,
+                     int64_t total, int64_t max_n, int bits, const float* ratios_host, int K,
+                     float* m_host, float* p_host, float* err_host, int32_t* idx_host,
+                     uint8_t* codes_host, uint8_t* region_mask_host, int code_layout,
+                     void* dev_scratch, size_t dev_scratch_bytes, float** y_dev_out,
+                     void* stream);
+
+/* Text for a status value (static storage). */
+const char* pwlq_status_string(int status);
+/* Library version, "major.minor". */
+const char* pwlq_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* PWLQ_H_ */

@@ -1,0 +1,259 @@
+// C ABI of the PWLQ library: argument checks and kernel launches, nothing else.
+#include "../../include/pwlq.h"
+#include "pwlq_kernels.h"
+
+namespace {
+
+inline bool misaligned(const void* p, size_t a) {
+    return (reinterpret_cast<uintptr_t>(p) & (a - 1)) != 0;
+}
+inline cudaStream_t as_stream(void* s) { return static_cast<cudaStream_t>(s); }
+inline int from_cuda(cudaError_t e) { return e == cudaSuccess ? PWLQ_OK : PWLQ_ERR_CUDA; }
+inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+
+// Largest flat size: the streaming kernels index 8 values per thread with a 32-bit grid.
+constexpr int64_t kMaxTotal = (int64_t)1 << 40;
+
+int check_rows(int64_t C, int64_t n_or_total) {
+    if (C < 1 || n_or_total < 1) return PWLQ_ERR_INVALID_ARG;
+    if (C > ((int64_t)1 << 31) - 1) return PWLQ_ERR_UNSUPPORTED;
+    return PWLQ_OK;
+}
+
+int absmax_impl(const float* x, const int64_t* ro, int64_t C, int64_t n, int64_t total,
+                float* m_out, void* stream) {
+    if (!x || !m_out || misaligned(x, 4) || misaligned(m_out, 4) || misaligned(ro, 8))
+        return PWLQ_ERR_INVALID_ARG;
+    if (total > kMaxTotal) return PWLQ_ERR_UNSUPPORTED;
+    return from_cuda(pwlq::launch_absmax(x, ro, C, n, total, m_out, as_stream(stream)));
+}
+
+int search_impl(const float* x, const int64_t* ro, int64_t C, int64_t n, int64_t total,
+                int64_t max_n, int bits, const float* ratios, int K, const float* m, float* p_out,
+                float* err_out, int32_t* idx_out, float* sse_all, void* ws, size_t ws_bytes,
+                void* stream) {
+    if (!x || !ratios || !p_out || !idx_out || bits < 2 || bits > 8 || K < 1 || max_n < 1)
+        return PWLQ_ERR_INVALID_ARG;
+    if (misaligned(x, 4) || misaligned(ratios, 4) || misaligned(m, 4) || misaligned(p_out, 4) ||
+        misaligned(err_out, 4) || misaligned(idx_out, 4) || misaligned(sse_all, 4) ||
+        misaligned(ro, 8))
+        return PWLQ_ERR_INVALID_ARG;
+    if (K > PWLQ_MAX_K || total > kMaxTotal) return PWLQ_ERR_UNSUPPORTED;
+    const pwlq::SearchPlan plan = pwlq::plan_search(C, max_n, K);
+    if (C * plan.tiles > ((int64_t)1 << 31) - 1) return PWLQ_ERR_UNSUPPORTED;
+    if (!ws || ws_bytes < plan.bytes) return PWLQ_ERR_WORKSPACE;
+    if (misaligned(ws, 256)) return PWLQ_ERR_INVALID_ARG;
+    return from_cuda(pwlq::launch_search(x, ro, C, n, total, bits, ratios, K, m, p_out, err_out,
+                                         idx_out, sse_all, ws, plan, as_stream(stream)));
+}
+
+int quantize_impl(const float* x, const int64_t* ro, int64_t C, int64_t n, int64_t total,
+                  int bits, const float* m, const float* p, uint8_t* codes, uint8_t* mask,
+                  float* fake, int layout, void* stream) {
+    if (!x || !m || !p || !codes || !mask || bits < 2 || bits > 8 ||
+        (layout != PWLQ_CODES_U8 && layout != PWLQ_CODES_PACKED))
+        return PWLQ_ERR_INVALID_ARG;
+    if (misaligned(x, 4) || misaligned(m, 4) || misaligned(p, 4) || misaligned(fake, 4) ||
+        misaligned(ro, 8))
+        return PWLQ_ERR_INVALID_ARG;
+    if (total > kMaxTotal) return PWLQ_ERR_UNSUPPORTED;
+    return from_cuda(pwlq::launch_quantize(x, ro, C, n, total, bits, m, p, codes, mask, fake,
+                                           layout, as_stream(stream)));
+}
+
+int dequantize_impl(const uint8_t* codes, const uint8_t* mask, const int64_t* ro, int64_t C,
+                    int64_t n, int64_t total, int bits, const float* m, const float* p, float* y,
+                    int layout, void* stream) {
+    if (!codes || !mask || !m || !p || !y || bits < 2 || bits > 8 ||
+        (layout != PWLQ_CODES_U8 && layout != PWLQ_CODES_PACKED))
+        return PWLQ_ERR_INVALID_ARG;
+    if (misaligned(m, 4) || misaligned(p, 4) || misaligned(y, 4) || misaligned(ro, 8))
+        return PWLQ_ERR_INVALID_ARG;
+    if (total > kMaxTotal) return PWLQ_ERR_UNSUPPORTED;
+    return from_cuda(pwlq::launch_dequantize(codes, mask, ro, C, n, total, bits, m, p, y, layout,
+                                             as_stream(stream)));
+}
+
+inline size_t code_bytes(int64_t total, int bits, int layout) {
+    return (layout == PWLQ_CODES_PACKED && bits <= 4) ? (size_t)((total + 1) / 2) : (size_t)total;
+}
+
+// Layout of the device scratch of pwlq_encode_host (every block 256-byte aligned).
+struct HostPlan {
+    size_t x, ro, ratios, m, p, err, idx, codes, mask, y, ws, bytes;
+    pwlq::SearchPlan sp;
+};
+HostPlan plan_host(int64_t C, int64_t total, int64_t max_n, int K) {
+    HostPlan h;
+    size_t o = 0;
+    auto take = [&](size_t bytes) { size_t r = o; o = align_up(o + bytes, 256); return r; };
+    h.x = take(sizeof(float) * (size_t)total);
+    h.ro = take(sizeof(int64_t) * (size_t)(C + 1));
+    h.ratios = take(sizeof(float) * (size_t)K);
+    h.m = take(sizeof(float) * (size_t)C);
+    h.p = take(sizeof(float) * (size_t)C);
+    h.err = take(sizeof(float) * (size_t)C);
+    h.idx = take(sizeof(int32_t) * (size_t)C);
+    h.codes = take((size_t)total);
+    h.mask = take((size_t)((total + 7) / 8));
+    h.y = take(sizeof(float) * (size_t)total);
+    h.sp = pwlq::plan_search(C, max_n, K);
+    h.ws = take(h.sp.bytes);
+    h.bytes = o;
+    return h;
+}
+
+}  // namespace
+
+extern "C" {
+
+int pwlq_absmax(const float* x, int64_t C, int64_t n, float* m_out, void* stream) {
+    if (int rc = check_rows(C, n)) return rc;
+    return absmax_impl(x, nullptr, C, n, C * n, m_out, stream);
+}
+
+int pwlq_absmax_ragged(const float* x, const int64_t* row_offsets, int64_t C, int64_t total,
+                       float* m_out, void* stream) {
+    if (int rc = check_rows(C, total)) return rc;
+    if (!row_offsets) return PWLQ_ERR_INVALID_ARG;
+    return absmax_impl(x, row_offsets, C, 0, total, m_out, stream);
+}
+
+size_t pwlq_search_workspace_bytes(int64_t C, int64_t n, int K) {
+    if (C < 1 || n < 1 || K < 1 || K > PWLQ_MAX_K) return 0;
+    return pwlq::plan_search(C, n, K).bytes;
+}
+
+int pwlq_search(const float* x, int64_t C, int64_t n, int bits, const float* ratios, int K,
+                const float* m, float* p_out, float* err_out, int32_t* idx_out, float* sse_all,
+                void* workspace, size_t workspace_bytes, void* stream) {
+    if (int rc = check_rows(C, n)) return rc;
+    return search_impl(x, nullptr, C, n, C * n, n, bits, ratios, K, m, p_out, err_out, idx_out,
+                       sse_all, workspace, workspace_bytes, stream);
+}
+
+int pwlq_search_ragged(const float* x, const int64_t* row_offsets, int64_t C, int64_t total,
+                       int64_t max_n, int bits, const float* ratios, int K, const float* m,
+                       float* p_out, float* err_out, int32_t* idx_out, float* sse_all,
+                       void* workspace, size_t workspace_bytes, void* stream) {
+    if (int rc = check_rows(C, total)) return rc;
+    if (!row_offsets || max_n > total) return PWLQ_ERR_INVALID_ARG;
+    return search_impl(x, row_offsets, C, 0, total, max_n, bits, ratios, K, m, p_out, err_out,
+                       idx_out, sse_all, workspace, workspace_bytes, stream);
+}
+
+int pwlq_quantize(const float* x, int64_t C, int64_t n, int bits, const float* m, const float* p,
+                  uint8_t* codes, uint8_t* region_mask, float* fake_out, int code_layout,
+                  void* stream) {
+    if (int rc = check_rows(C, n)) return rc;
+    return quantize_impl(x, nullptr, C, n, C * n, bits, m, p, codes, region_mask, fake_out,
+                         code_layout, stream);
+}
+
+int pwlq_quantize_ragged(const float* x, const int64_t* row_offsets, int64_t C, int64_t total,
+                         int bits, const float* m, const float* p, uint8_t* codes,
+                         uint8_t* region_mask, float* fake_out, int code_layout, void* stream) {
+    if (int rc = check_rows(C, total)) return rc;
+    if (!row_offsets) return PWLQ_ERR_INVALID_ARG;
+    return quantize_impl(x, row_offsets, C, 0, total, bits, m, p, codes, region_mask, fake_out,
+                         code_layout, stream);
+}
+
+int pwlq_dequantize(const uint8_t* codes, const uint8_t* region_mask, int64_t C, int64_t n,
+                    int bits, const float* m, const float* p, float* y, int code_layout,
+                    void* stream) {
+    if (int rc = check_rows(C, n)) return rc;
+    return dequantize_impl(codes, region_mask, nullptr, C, n, C * n, bits, m, p, y, code_layout,
+                           stream);
+}
+
+int pwlq_dequantize_ragged(const uint8_t* codes, const uint8_t* region_mask,
+                           const int64_t* row_offsets, int64_t C, int64_t total, int bits,
+                           const float* m, const float* p, float* y, int code_layout,
+                           void* stream) {
+    if (int rc = check_rows(C, total)) return rc;
+    if (!row_offsets) return PWLQ_ERR_INVALID_ARG;
+    return dequantize_impl(codes, region_mask, row_offsets, C, 0, total, bits, m, p, y,
+                           code_layout, stream);
+}
+
+size_t pwlq_encode_host_scratch_bytes(int64_t C, int64_t total, int64_t max_n, int K) {
+    if (C < 1 || total < 1 || max_n < 1 || K < 1 || K > PWLQ_MAX_K) return 0;
+    return plan_host(C, total, max_n, K).bytes;
+}
+
+int pwlq_encode_host(const float* x_host, const int64_t* row_offsets_host, int64_t C,
+                     int64_t total, int64_t max_n, int bits, const float* ratios_host, int K,
+                     float* m_host, float* p_host, float* err_host, int32_t* idx_host,
+                     uint8_t* codes_host, uint8_t* region_mask_host, int code_layout,
+                     void* dev_scratch, size_t dev_scratch_bytes, float** y_dev_out,
+                     void* stream) {
+    if (int rc = check_rows(C, total)) return rc;
+    if (!x_host || !ratios_host || !m_host || !p_host || !idx_host || !codes_host ||
+        !region_mask_host || bits < 2 || bits > 8 || K < 1 || max_n < 1 || max_n > total ||
+        (code_layout != PWLQ_CODES_U8 && code_layout != PWLQ_CODES_PACKED))
+        return PWLQ_ERR_INVALID_ARG;
+    if (K > PWLQ_MAX_K || total > kMaxTotal) return PWLQ_ERR_UNSUPPORTED;
+    int64_t n = 0;
+    if (!row_offsets_host) {
+        if (total % C != 0 || max_n != total / C) return PWLQ_ERR_INVALID_ARG;
+        n = total / C;
+    }
+    const HostPlan h = plan_host(C, total, max_n, K);
+    if (!dev_scratch || dev_scratch_bytes < h.bytes) return PWLQ_ERR_WORKSPACE;
+    if (misaligned(dev_scratch, 256)) return PWLQ_ERR_INVALID_ARG;
+    unsigned char* d = static_cast<unsigned char*>(dev_scratch);
+    cudaStream_t st = as_stream(stream);
+    float* dx = reinterpret_cast<float*>(d + h.x);
+    int64_t* dro = row_offsets_host ? reinterpret_cast<int64_t*>(d + h.ro) : nullptr;
+    float* dr = reinterpret_cast<float*>(d + h.ratios);
+    float* dm = reinterpret_cast<float*>(d + h.m);
+    float* dp = reinterpret_cast<float*>(d + h.p);
+    float* de = reinterpret_cast<float*>(d + h.err);
+    int32_t* di = reinterpret_cast<int32_t*>(d + h.idx);
+    uint8_t* dc = d + h.codes;
+    uint8_t* dk = d + h.mask;
+    float* dy = reinterpret_cast<float*>(d + h.y);
+    const size_t cb = code_bytes(total, bits, code_layout), mb = (size_t)((total + 7) / 8);
+
+    cudaError_t e;
+#define PWLQ_TRY(call) do { e = (call); if (e != cudaSuccess) return PWLQ_ERR_CUDA; } while (0)
+    PWLQ_TRY(cudaMemcpyAsync(dx, x_host, sizeof(float) * (size_t)total, cudaMemcpyHostToDevice, st));
+    if (dro)
+        PWLQ_TRY(cudaMemcpyAsync(dro, row_offsets_host, sizeof(int64_t) * (size_t)(C + 1),
+                                 cudaMemcpyHostToDevice, st));
+    PWLQ_TRY(cudaMemcpyAsync(dr, ratios_host, sizeof(float) * (size_t)K, cudaMemcpyHostToDevice, st));
+    PWLQ_TRY(pwlq::launch_absmax(dx, dro, C, n, total, dm, st));
+    PWLQ_TRY(pwlq::launch_search(dx, dro, C, n, total, bits, dr, K, dm, dp, de, di, nullptr,
+                                 d + h.ws, h.sp, st));
+    PWLQ_TRY(pwlq::launch_quantize(dx, dro, C, n, total, bits, dm, dp, dc, dk, nullptr,
+                                   code_layout, st));
+    PWLQ_TRY(pwlq::launch_dequantize(dc, dk, dro, C, n, total, bits, dm, dp, dy, code_layout, st));
+    PWLQ_TRY(cudaMemcpyAsync(m_host, dm, sizeof(float) * (size_t)C, cudaMemcpyDeviceToHost, st));
+    PWLQ_TRY(cudaMemcpyAsync(p_host, dp, sizeof(float) * (size_t)C, cudaMemcpyDeviceToHost, st));
+    if (err_host)
+        PWLQ_TRY(cudaMemcpyAsync(err_host, de, sizeof(float) * (size_t)C, cudaMemcpyDeviceToHost, st));
+    PWLQ_TRY(cudaMemcpyAsync(idx_host, di, sizeof(int32_t) * (size_t)C, cudaMemcpyDeviceToHost, st));
+    PWLQ_TRY(cudaMemcpyAsync(codes_host, dc, cb, cudaMemcpyDeviceToHost, st));
+    PWLQ_TRY(cudaMemcpyAsync(region_mask_host, dk, mb, cudaMemcpyDeviceToHost, st));
+#undef PWLQ_TRY
+    if (y_dev_out) *y_dev_out = dy;
+    return PWLQ_OK;
+}
+
+const char* pwlq_status_string(int status) {
+    switch (status) {
+        case PWLQ_OK: return "ok";
+        case PWLQ_ERR_INVALID_ARG: return "invalid argument";
+        case PWLQ_ERR_UNSUPPORTED: return "size or K above the supported limit";
+        case PWLQ_ERR_WORKSPACE: return "workspace missing or too small";
+        case PWLQ_ERR_CUDA: return "CUDA runtime error";
+        case PWLQ_ERR_NONFINITE: return "a row's range is not finite";
+        case PWLQ_ERR_TIMEOUT: return "a bounded device wait expired";
+        default: return "unknown status";
+    }
+}
+
+const char* pwlq_version(void) { return "0.1"; }
+
+}  // extern "C"

@@ -1,0 +1,75 @@
+// Device helpers shared by the PWLQ kernels (sm_100a).
+//
+// The element arithmetic restates Eq. 1 and Eq. 3 of arXiv 2002.00104 in IEEE binary32 with one
+// rounding per operation; the explicit __f*_rn intrinsics are never contracted into FMAs.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace pwlq {
+
+constexpr int kWarp = 32;
+constexpr int kStatusNonFinite = 1 << 5;   // device status bit: 1 << PWLQ_ERR_NONFINITE
+
+struct PieceParams {
+    float p;     // breakpoint (offset z of the tail pieces, Eq. 3)
+    float s1;    // step of the center pieces, p / L        (Eq. 1: s = Delta / (N - 1))
+    float inv1;  // L / p
+    float s2;    // step of the tail pieces, (m - p) / L
+    float inv2;  // L / (m - p)
+};
+
+// Per-(row, candidate) constants.  A piece with a non-positive range gets step 0.
+__device__ __forceinline__ PieceParams make_params(float m, float p, float Lf) {
+    PieceParams P;
+    P.p = p;
+    if (p > 0.0f) { P.s1 = __fdiv_rn(p, Lf); P.inv1 = __fdiv_rn(Lf, p); }
+    else          { P.s1 = 0.0f;             P.inv1 = 0.0f; }
+    const float d = __fsub_rn(m, p);
+    if (d > 0.0f) { P.s2 = __fdiv_rn(d, Lf); P.inv2 = __fdiv_rn(Lf, d); }
+    else          { P.s2 = 0.0f;             P.inv2 = 0.0f; }
+    return P;
+}
+
+// Eq. 3 for one magnitude a = min(|x|, m): level q, region, reconstructed magnitude v.
+__device__ __forceinline__ void quantize_mag(float a, const PieceParams& P, float Lf,
+                                             int& q_out, int& tail_out, float& v_out) {
+    const bool tail = a > P.p;                       // R2 = (p, m]
+    const float z = tail ? P.p : 0.0f;
+    const float inv = tail ? P.inv2 : P.inv1;
+    const float s = tail ? P.s2 : P.s1;
+    const float u = __fsub_rn(a, z);
+    const float t = __fmul_rn(u, inv);
+    const float q = fminf(rintf(t), Lf);             // round half to even, saturate
+    float v = __fmul_rn(q, s);
+    v = __fadd_rn(v, z);
+    q_out = (int)q;
+    tail_out = tail ? 1 : 0;
+    v_out = v;
+}
+
+// Row lookup: dense rows have length n, ragged rows are given by ascending offsets.
+struct Rows {
+    const int64_t* offsets;  // [C + 1] or nullptr (dense)
+    int64_t C;
+    int64_t n;               // dense row length (unused when ragged)
+
+    __device__ __forceinline__ int64_t begin(int64_t c) const {
+        return offsets ? offsets[c] : c * n;
+    }
+    // Row that contains flat index i (0 <= i < total); empty rows are skipped.
+    __device__ __forceinline__ int64_t row_of(int64_t i) const {
+        if (!offsets) return i / n;
+        int64_t lo = 0, hi = C;                      // offsets[lo] <= i < offsets[hi]
+        while (hi - lo > 1) {
+            const int64_t mid = (lo + hi) >> 1;
+            if (offsets[mid] <= i) lo = mid; else hi = mid;
+        }
+        return lo;
+    }
+};
+
+__device__ __forceinline__ uint32_t abs_bits(float x) { return __float_as_uint(x) & 0x7fffffffu; }
+
+}  // namespace pwlq

@@ -1,0 +1,40 @@
+// Host-side launchers of the PWLQ kernels (internal to the library).
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stddef.h>
+#include <stdint.h>
+
+namespace pwlq {
+
+// Values of one row that a search CTA stages in shared memory at a time; longer rows are cut
+// into tiles whose partial sums are combined in a fixed order by a second kernel.
+constexpr int kSearchTile = 8192;
+
+cudaError_t launch_absmax(const float* x, const int64_t* row_offsets, int64_t C, int64_t n,
+                          int64_t total, float* m_out, cudaStream_t stream);
+
+struct SearchPlan {
+    int64_t tiles;         // tiles per row (by the longest row)
+    size_t off_m;          // workspace offset of the internally computed ranges [C] floats
+    size_t off_partials;   // workspace offset of the partial sums [C * tiles * K] doubles (tiles > 1)
+    size_t bytes;          // total workspace bytes
+};
+SearchPlan plan_search(int64_t C, int64_t max_n, int K);
+
+cudaError_t launch_search(const float* x, const int64_t* row_offsets, int64_t C, int64_t n,
+                          int64_t total, int bits, const float* ratios, int K, const float* m,
+                          float* p_out, float* err_out, int32_t* idx_out, float* sse_all,
+                          void* workspace, const SearchPlan& plan, cudaStream_t stream);
+
+cudaError_t launch_quantize(const float* x, const int64_t* row_offsets, int64_t C, int64_t n,
+                            int64_t total, int bits, const float* m, const float* p,
+                            uint8_t* codes, uint8_t* mask, float* fake, int layout,
+                            cudaStream_t stream);
+
+cudaError_t launch_dequantize(const uint8_t* codes, const uint8_t* mask,
+                              const int64_t* row_offsets, int64_t C, int64_t n, int64_t total,
+                              int bits, const float* m, const float* p, float* y, int layout,
+                              cudaStream_t stream);
+
+}  // namespace pwlq

@@ -1,0 +1,239 @@
+"""Thin Python binding of ``libpwlq.so`` (argument marshalling only).
+
+Every step of the path runs in the library's CUDA kernels; PyTorch is used for
+device memory and streams.  The functions mirror the C entry points declared in
+``include/pwlq.h`` and take CUDA tensors (or, for ``encode_host``, pinned host
+tensors).  There is no CPU fallback: if the shared library has not been built,
+or a tensor is not on a CUDA device, the call raises.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import Optional
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_LIB_PATH = os.path.join(_HERE, "libpwlq.so")
+_lib = None
+
+OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_WORKSPACE, ERR_CUDA, ERR_NONFINITE, ERR_TIMEOUT = range(7)
+CODES_U8, CODES_PACKED = 0, 1
+MAX_K = 4096
+
+_P, _I64, _INT, _SZ = ctypes.c_void_p, ctypes.c_int64, ctypes.c_int, ctypes.c_size_t
+_SIGNATURES = {
+    "pwlq_absmax": (_INT, [_P, _I64, _I64, _P, _P]),
+    "pwlq_absmax_ragged": (_INT, [_P, _P, _I64, _I64, _P, _P]),
+    "pwlq_search_workspace_bytes": (_SZ, [_I64, _I64, _INT]),
+    "pwlq_search": (_INT, [_P, _I64, _I64, _INT, _P, _INT, _P, _P, _P, _P, _P, _P, _SZ, _P]),
+    "pwlq_search_ragged": (_INT, [_P, _P, _I64, _I64, _I64, _INT, _P, _INT, _P, _P, _P, _P, _P, _P,
+                                  _SZ, _P]),
+    "pwlq_quantize": (_INT, [_P, _I64, _I64, _INT, _P, _P, _P, _P, _P, _INT, _P]),
+    "pwlq_quantize_ragged": (_INT, [_P, _P, _I64, _I64, _INT, _P, _P, _P, _P, _P, _INT, _P]),
+    "pwlq_dequantize": (_INT, [_P, _P, _I64, _I64, _INT, _P, _P, _P, _INT, _P]),
+    "pwlq_dequantize_ragged": (_INT, [_P, _P, _P, _I64, _I64, _INT, _P, _P, _P, _INT, _P]),
+    "pwlq_encode_host_scratch_bytes": (_SZ, [_I64, _I64, _I64, _INT]),
+    "pwlq_encode_host": (_INT, [_P, _P, _I64, _I64, _I64, _INT, _P, _INT, _P, _P, _P, _P, _P, _P,
+                                _INT, _P, _SZ, _P, _P]),
+    "pwlq_status_string": (ctypes.c_char_p, [_INT]),
+    "pwlq_version": (ctypes.c_char_p, []),
+}
+
+
+class PwlqError(RuntimeError):
+    def __init__(self, status: int, what: str):
+        self.status = status
+        super().__init__(f"{what}: {status_string(status)} (status {status})")
+
+
+def load_library(path: Optional[str] = None) -> ctypes.CDLL:
+    """Loads the C-ABI library; raises if it has not been built (no fallback exists)."""
+    global _lib
+    if _lib is None or path is not None:
+        path = path or _LIB_PATH
+        if not os.path.exists(path):
+            raise RuntimeError(
+                f"{path} is missing: build it with `python -m paper_2002_00104_b200.build` "
+                "(nvcc, sm_100a); this package has no CPU or PyTorch fallback")
+        lib = ctypes.CDLL(path)
+        for name, (res, args) in _SIGNATURES.items():
+            fn = getattr(lib, name)
+            fn.restype, fn.argtypes = res, args
+        _lib = lib
+    return _lib
+
+
+def exported_symbols():
+    return sorted(_SIGNATURES)
+
+
+def status_string(status: int) -> str:
+    return load_library().pwlq_status_string(int(status)).decode()
+
+
+def version() -> str:
+    return load_library().pwlq_version().decode()
+
+
+def _dev(t: Optional[torch.Tensor], dtype, what: str):
+    if t is None:
+        return None
+    if not (t.is_cuda and t.dtype == dtype and t.is_contiguous()):
+        raise ValueError(f"{what} must be a contiguous CUDA tensor of {dtype}")
+    return t.data_ptr()
+
+
+def _stream(stream) -> int:
+    s = stream if stream is not None else torch.cuda.current_stream()
+    return s.cuda_stream
+
+
+def _check(rc: int, what: str):
+    if rc != OK:
+        raise PwlqError(rc, what)
+
+
+def _shape(x: torch.Tensor, row_offsets):
+    """(C, n, total) of a dense [C, ...] tensor, or (C, None, total) for ragged rows."""
+    if row_offsets is None:
+        if x.dim() < 2:
+            raise ValueError("dense input must be [C, n] (use x[None] for a single row)")
+        C = x.shape[0]
+        return C, x.numel() // C, x.numel()
+    return row_offsets.numel() - 1, None, x.numel()
+
+
+def code_bytes(total: int, bits: int, layout: int) -> int:
+    return (total + 1) // 2 if (layout == CODES_PACKED and bits <= 4) else total
+
+
+def absmax(x, row_offsets=None, out=None, stream=None):
+    lib = load_library()
+    C, n, total = _shape(x, row_offsets)
+    m = out if out is not None else torch.empty(C, dtype=torch.float32, device=x.device)
+    if row_offsets is None:
+        rc = lib.pwlq_absmax(_dev(x, torch.float32, "x"), C, n, _dev(m, torch.float32, "out"),
+                             _stream(stream))
+    else:
+        rc = lib.pwlq_absmax_ragged(_dev(x, torch.float32, "x"),
+                                    _dev(row_offsets, torch.int64, "row_offsets"), C, total,
+                                    _dev(m, torch.float32, "out"), _stream(stream))
+    _check(rc, "pwlq_absmax")
+    return m
+
+
+def search_workspace_bytes(C: int, max_n: int, K: int) -> int:
+    return int(load_library().pwlq_search_workspace_bytes(C, max_n, K))
+
+
+def search(x, bits, ratios, m=None, row_offsets=None, max_n=None, want_sse=False,
+           workspace=None, out=None, stream=None):
+    """Returns dict(p, err, idx, sse or None, workspace).  ``workspace[:4]`` holds the status."""
+    lib = load_library()
+    C, n, total = _shape(x, row_offsets)
+    K = ratios.numel()
+    longest = n if row_offsets is None else int(max_n)
+    need = search_workspace_bytes(C, longest, K)
+    if workspace is None:
+        workspace = torch.empty(max(need, 256), dtype=torch.uint8, device=x.device)
+    if out is None:
+        out = {"p": torch.empty(C, dtype=torch.float32, device=x.device),
+               "err": torch.empty(C, dtype=torch.float32, device=x.device),
+               "idx": torch.empty(C, dtype=torch.int32, device=x.device),
+               "sse": torch.empty((C, K), dtype=torch.float32, device=x.device) if want_sse else None}
+    args_tail = (int(bits), _dev(ratios, torch.float32, "ratios"), K, _dev(m, torch.float32, "m"),
+                 _dev(out["p"], torch.float32, "p"), _dev(out["err"], torch.float32, "err"),
+                 _dev(out["idx"], torch.int32, "idx"), _dev(out.get("sse"), torch.float32, "sse"),
+                 _dev(workspace, torch.uint8, "workspace"), workspace.numel(), _stream(stream))
+    if row_offsets is None:
+        rc = lib.pwlq_search(_dev(x, torch.float32, "x"), C, n, *args_tail)
+    else:
+        rc = lib.pwlq_search_ragged(_dev(x, torch.float32, "x"),
+                                    _dev(row_offsets, torch.int64, "row_offsets"), C, total,
+                                    longest, *args_tail)
+    _check(rc, "pwlq_search")
+    out = dict(out)
+    out["workspace"] = workspace
+    return out
+
+
+def search_status(workspace) -> int:
+    """Device status bits of the last search that used this workspace (synchronises)."""
+    return int(workspace[:4].view(torch.int32).item())
+
+
+def quantize(x, bits, m, p, layout=CODES_U8, row_offsets=None, want_fake=False, out=None,
+             stream=None):
+    """Returns (codes uint8, region_mask uint8, fake fp32 or None)."""
+    lib = load_library()
+    C, n, total = _shape(x, row_offsets)
+    if out is None:
+        codes = torch.empty(code_bytes(total, bits, layout), dtype=torch.uint8, device=x.device)
+        mask = torch.empty((total + 7) // 8, dtype=torch.uint8, device=x.device)
+        fake = torch.empty(total, dtype=torch.float32, device=x.device) if want_fake else None
+    else:
+        codes, mask, fake = out
+    tail = (int(bits), _dev(m, torch.float32, "m"), _dev(p, torch.float32, "p"),
+            _dev(codes, torch.uint8, "codes"), _dev(mask, torch.uint8, "mask"),
+            _dev(fake, torch.float32, "fake"), int(layout), _stream(stream))
+    if row_offsets is None:
+        rc = lib.pwlq_quantize(_dev(x, torch.float32, "x"), C, n, *tail)
+    else:
+        rc = lib.pwlq_quantize_ragged(_dev(x, torch.float32, "x"),
+                                      _dev(row_offsets, torch.int64, "row_offsets"), C, total, *tail)
+    _check(rc, "pwlq_quantize")
+    return codes, mask, fake
+
+
+def dequantize(codes, mask, bits, m, p, C=None, n=None, layout=CODES_U8, row_offsets=None,
+               out=None, stream=None):
+    lib = load_library()
+    if row_offsets is None:
+        total = int(C) * int(n)
+    else:
+        C = row_offsets.numel() - 1
+        total = int(out.numel()) if out is not None else int(row_offsets[-1].item())
+    y = out if out is not None else torch.empty(total, dtype=torch.float32, device=codes.device)
+    tail = (int(bits), _dev(m, torch.float32, "m"), _dev(p, torch.float32, "p"),
+            _dev(y, torch.float32, "y"), int(layout), _stream(stream))
+    if row_offsets is None:
+        rc = lib.pwlq_dequantize(_dev(codes, torch.uint8, "codes"), _dev(mask, torch.uint8, "mask"),
+                                 int(C), int(n), *tail)
+    else:
+        rc = lib.pwlq_dequantize_ragged(_dev(codes, torch.uint8, "codes"),
+                                        _dev(mask, torch.uint8, "mask"),
+                                        _dev(row_offsets, torch.int64, "row_offsets"), C, total,
+                                        *tail)
+    _check(rc, "pwlq_dequantize")
+    return y
+
+
+def encode_host_scratch_bytes(C: int, total: int, max_n: int, K: int) -> int:
+    return int(load_library().pwlq_encode_host_scratch_bytes(C, total, max_n, K))
+
+
+def _host(t: Optional[torch.Tensor], dtype, what: str):
+    if t is None:
+        return None
+    if t.is_cuda or t.dtype != dtype or not t.is_contiguous():
+        raise ValueError(f"{what} must be a contiguous host tensor of {dtype}")
+    return t.data_ptr()
+
+
+def encode_host(x_host, row_offsets_host, C, max_n, bits, ratios_host, out_host, layout,
+                dev_scratch, stream=None):
+    """Whole path from (pinned) host tensors; ``out_host`` = dict(m, p, err, idx, codes, mask) of
+    host tensors that receive the results once the stream is synchronised."""
+    lib = load_library()
+    total = x_host.numel()
+    rc = lib.pwlq_encode_host(
+        _host(x_host, torch.float32, "x_host"), _host(row_offsets_host, torch.int64, "row_offsets"),
+        int(C), total, int(max_n), int(bits), _host(ratios_host, torch.float32, "ratios"),
+        ratios_host.numel(), _host(out_host["m"], torch.float32, "m"),
+        _host(out_host["p"], torch.float32, "p"), _host(out_host.get("err"), torch.float32, "err"),
+        _host(out_host["idx"], torch.int32, "idx"), _host(out_host["codes"], torch.uint8, "codes"),
+        _host(out_host["mask"], torch.uint8, "mask"), int(layout),
+        _dev(dev_scratch, torch.uint8, "dev_scratch"), dev_scratch.numel(), None, _stream(stream))
+    _check(rc, "pwlq_encode_host")

@@ -1,0 +1,224 @@
+"""GPU parity: the CUDA path (through the C ABI) against the CPU oracle, element by element."""
+import numpy as np
+import pytest
+import torch
+
+from gpu_util import check_search, dev
+from paper_2002_00104_b200 import workloads as W
+
+pytestmark = [pytest.mark.gpu,
+              pytest.mark.skipif(not torch.cuda.is_available(), reason="needs a CUDA device")]
+
+
+@pytest.fixture(scope="module")
+def pwlq():
+    from paper_2002_00104_b200 import pwlq as _p
+    _p.load_library()
+    return _p
+
+
+def np_(t):
+    return None if t is None else t.cpu().numpy()
+
+
+def run_search(pwlq, x, bits, ratios, row_offsets=None, max_n=None, m=None):
+    out = pwlq.search(dev(x), bits, dev(ratios), m=None if m is None else dev(m),
+                      row_offsets=None if row_offsets is None else dev(row_offsets),
+                      max_n=max_n, want_sse=True)
+    torch.cuda.synchronize()
+    return {k: np_(out[k]) for k in ("p", "err", "idx", "sse")}, pwlq.search_status(out["workspace"])
+
+
+# ------------------------------------------------------------------------------------ abs-max
+@pytest.mark.parametrize("C,n", [(1, 1), (3, 9), (5, 147), (64, 64), (7, 4607), (2, 100003), (1, 1 << 20)])
+def test_absmax_dense(pwlq, oracle, C, n):
+    rng = np.random.default_rng(C * 1000 + n)
+    x = rng.laplace(0, 0.02, (C, n)).astype(np.float32)
+    x[0, 0] = -x.max() * 3 if n > 1 else x[0, 0]
+    m = np_(pwlq.absmax(dev(x)))
+    assert np.array_equal(m, oracle.absmax(x))
+
+
+def test_absmax_ragged_and_unaligned(pwlq, oracle):
+    w = W.small_mixed(seed=11)
+    m = np_(pwlq.absmax(dev(w.x), row_offsets=dev(w.row_offsets)))
+    assert np.array_equal(m, oracle.absmax(w.x, w.row_offsets))
+    # base pointer 4 bytes off a 16-byte boundary: vector loads must not be used
+    buf = dev(np.concatenate([[0.0], w.x]).astype(np.float32))
+    m2 = np_(pwlq.absmax(buf[1:], row_offsets=dev(w.row_offsets)))
+    assert np.array_equal(m2, m)
+    z = np.zeros((4, 33), dtype=np.float32)
+    z[2, 5] = -0.0
+    assert np.array_equal(np_(pwlq.absmax(dev(z))), np.zeros(4, np.float32))
+
+
+# ------------------------------------------------------------------------- quantize / dequantize
+def canary(nbytes, dtype=torch.uint8):
+    """Output buffer with a guard band on both sides."""
+    pad = 64
+    buf = torch.full((nbytes + 2 * pad,), 0xA5, dtype=torch.uint8, device="cuda")
+    return buf, buf[pad:pad + nbytes]
+
+
+def guards_intact(buf, nbytes):
+    b = buf.cpu().numpy()
+    return np.all(b[:64] == 0xA5) and np.all(b[64 + nbytes:] == 0xA5)
+
+
+@pytest.mark.parametrize("bits", [2, 3, 4, 5, 6, 8])
+@pytest.mark.parametrize("layout", [0, 1])
+def test_quantize_dequantize_ragged_bit_exact(pwlq, oracle, bits, layout):
+    w = W.small_mixed(seed=20 + bits, bits=bits)
+    ratios = W.ratio_grid(16)
+    ora = oracle.search(w.x, bits, ratios, row_offsets=w.row_offsets)
+    m = oracle.absmax(w.x, w.row_offsets)
+    p = ora["p"]
+    oc, om, of = oracle.quantize(w.x, bits, m, p, layout=layout, row_offsets=w.row_offsets)
+    total = w.total
+    cbuf, codes = canary(pwlq.code_bytes(total, bits, layout))
+    mbuf, mask = canary((total + 7) // 8)
+    fbuf, fake8 = canary(total * 4)
+    fake = fake8.view(torch.float32)
+    pwlq.quantize(dev(w.x), bits, dev(m), dev(p), layout=layout, row_offsets=dev(w.row_offsets),
+                  out=(codes, mask, fake))
+    torch.cuda.synchronize()
+    assert np.array_equal(np_(codes), oc)
+    assert np.array_equal(np_(mask), om)
+    assert np_(fake).tobytes() == of.tobytes()
+    assert guards_intact(cbuf, codes.numel()) and guards_intact(mbuf, mask.numel())
+    assert guards_intact(fbuf, total * 4)
+    ybuf, y8 = canary(total * 4)
+    y = y8.view(torch.float32)
+    pwlq.dequantize(codes, mask, bits, dev(m), dev(p), layout=layout,
+                    row_offsets=dev(w.row_offsets), out=y)
+    torch.cuda.synchronize()
+    assert np_(y).tobytes() == of.tobytes()
+    assert guards_intact(ybuf, total * 4)
+
+
+@pytest.mark.parametrize("C,n,bits,layout", [(1, 1, 4, 1), (3, 9, 3, 1), (5, 147, 4, 1), (4, 4607, 8, 0),
+                                             (2, 100003, 4, 1), (64, 64, 6, 1), (16, 4096, 3, 1)])
+def test_quantize_dequantize_dense_bit_exact(pwlq, oracle, C, n, bits, layout):
+    rng = np.random.default_rng(C + n + bits)
+    x = (rng.standard_normal((C, n)) * 0.05).astype(np.float32)
+    if n > 4:
+        x[0, :3] = [0.0, -0.0, -1e-30]
+    m = oracle.absmax(x)
+    p = (m * rng.uniform(0.05, 1.0, C).astype(np.float32)).astype(np.float32)
+    if C > 1:
+        p[-1] = m[-1]                                # p = m: empty tail
+    oc, om, of = oracle.quantize(x, bits, m, p, layout=layout)
+    codes, mask, fake = pwlq.quantize(dev(x), bits, dev(m), dev(p), layout=layout, want_fake=True)
+    y = pwlq.dequantize(codes, mask, bits, dev(m), dev(p), C=C, n=n, layout=layout)
+    torch.cuda.synchronize()
+    assert np.array_equal(np_(codes), oc) and np.array_equal(np_(mask), om)
+    assert np_(fake).tobytes() == of.tobytes() and np_(y).tobytes() == of.tobytes()
+    assert np.array_equal(np_(y), oracle.dequantize(oc, om, bits, m, p, C=C, n=n, layout=layout))
+
+
+def test_quantize_worked_example(pwlq):
+    from conftest import read_golden
+    g = read_golden("worked_example_b3.txt")
+    x = np.array([float(v) for v in g["x"]], dtype=np.float32)[None]
+    m = np.array([12.0], np.float32)
+    for k, p in enumerate(float(v) for v in g["p"]):
+        codes, mask, fake = pwlq.quantize(dev(x), 3, dev(m), dev(np.array([p], np.float32)),
+                                          want_fake=True)
+        assert np_(codes).tolist() == [int(v) for v in g[f"code.{k}"]]
+        bits_ = np.unpackbits(np_(mask), bitorder="little")[:16]
+        assert bits_.tolist() == [int(v) for v in g[f"region.{k}"]]
+        assert np_(fake).tobytes() == np.array([float(v) for v in g[f"y.{k}"]], np.float32).tobytes()
+    out, _ = run_search(pwlq, x, 3, np.array([float(v) for v in g["ratios"]], np.float32))
+    assert out["idx"].tolist() == [1] and out["p"].tolist() == [6.0]
+    assert out["sse"][0].tolist() == [float(g[f"sse.{k}"][0]) for k in range(4)]
+
+
+def test_zero_rows_quantize_to_zero(pwlq, oracle):
+    x = np.zeros((3, 40), dtype=np.float32)
+    x[1] = np.linspace(-1, 1, 40)
+    m = oracle.absmax(x)
+    p = np.array([0.0, 0.25, 0.0], np.float32)
+    oc, om, of = oracle.quantize(x, 4, m, p, layout=1)
+    codes, mask, fake = pwlq.quantize(dev(x), 4, dev(m), dev(p), layout=1, want_fake=True)
+    assert np.array_equal(np_(codes), oc) and np.array_equal(np_(mask), om)
+    assert np_(fake).tobytes() == of.tobytes()
+
+
+# ------------------------------------------------------------------------------------- search
+@pytest.mark.parametrize("bits,K", [(4, 64), (3, 100), (4, 256), (8, 256), (2, 33), (6, 1024), (4, 1)])
+def test_search_ragged_small(pwlq, oracle, bits, K):
+    w = W.small_mixed(seed=bits * 7 + K, bits=bits, K=K)
+    ratios = W.ratio_grid(K)
+    ora = oracle.search(w.x, bits, ratios, row_offsets=w.row_offsets)
+    gpu, status = run_search(pwlq, w.x, bits, ratios, row_offsets=w.row_offsets,
+                             max_n=int(np.diff(w.row_offsets).max()))
+    assert status == 0
+    m = oracle.absmax(w.x, w.row_offsets)
+    check_search(gpu, ora, ratios, m, np.diff(w.row_offsets))
+
+
+@pytest.mark.parametrize("C,n,bits,K", [(1, 36864, 4, 100), (3, 20001, 4, 64), (2, 8192, 3, 256),
+                                        (5, 8193, 4, 40), (40, 147, 4, 256), (300, 9, 3, 256)])
+def test_search_dense_tiles_and_tails(pwlq, oracle, C, n, bits, K):
+    rng = np.random.default_rng(C * 31 + n)
+    x = rng.laplace(0, 0.02, (C, n)).astype(np.float32)
+    ratios = W.ratio_grid(K)
+    ora = oracle.search(x, bits, ratios)
+    gpu, status = run_search(pwlq, x, bits, ratios)
+    assert status == 0
+    check_search(gpu, ora, ratios, oracle.absmax(x), n)
+
+
+def test_search_with_given_range_and_unsorted_grid(pwlq, oracle):
+    rng = np.random.default_rng(77)
+    x = rng.standard_normal((6, 700)).astype(np.float32)
+    m = (oracle.absmax(x) * np.float32(1.25)).astype(np.float32)      # caller-chosen wider range
+    ratios = np.array([0.5, 0.2, 0.2, 0.9, 0.35, 1.0, 0.05], dtype=np.float32)
+    ora = oracle.search(x, 4, ratios, m=m)
+    gpu, _ = run_search(pwlq, x, 4, ratios, m=m)
+    check_search(gpu, ora, ratios, m, 700)
+
+
+def test_search_ties_take_lowest_index(pwlq):
+    x = np.array([[2.5, -2.5, 2.5, 2.5], [0.0, 0.0, 0.0, 0.0]], dtype=np.float32)
+    gpu, status = run_search(pwlq, x, 4, W.ratio_grid(10))
+    assert gpu["idx"].tolist() == [0, 0] and gpu["err"].tolist() == [0.0, 0.0]
+    assert gpu["p"].tolist() == [np.float32(2.5) * W.ratio_grid(10)[0], 0.0] and status == 0
+    rng = np.random.default_rng(5)
+    x = rng.laplace(0, 1, (1, 300)).astype(np.float32)
+    ratios = np.array([0.5, 0.2, 0.2, 0.9, 0.2], dtype=np.float32)
+    gpu, _ = run_search(pwlq, x, 4, ratios)
+    assert gpu["idx"].tolist() == [1]
+    assert gpu["sse"][0, 1] == gpu["sse"][0, 2] == gpu["sse"][0, 4]
+
+
+def test_search_reports_nonfinite_range(pwlq):
+    x = np.ones((3, 50), dtype=np.float32)
+    x[1, 7] = np.inf
+    gpu, status = run_search(pwlq, x, 4, W.ratio_grid(8))
+    assert status == 1 << pwlq.ERR_NONFINITE
+    assert gpu["idx"].tolist() == [0, 0, 0] and gpu["p"][1] == 0.0
+
+
+def test_search_is_reproducible(pwlq):
+    w = W.small_mixed(seed=1, K=256)
+    ratios = W.ratio_grid(256)
+    a, _ = run_search(pwlq, w.x, 4, ratios, row_offsets=w.row_offsets, max_n=9001)
+    b, _ = run_search(pwlq, w.x, 4, ratios, row_offsets=w.row_offsets, max_n=9001)
+    assert all(a[k].tobytes() == b[k].tobytes() for k in a)
+
+
+# ---------------------------------------------------------------------- argument errors (host)
+def test_argument_errors_launch_nothing(pwlq):
+    x = dev(np.ones((2, 8), np.float32))
+    r = dev(W.ratio_grid(4))
+    with pytest.raises(pwlq.PwlqError) as e:
+        pwlq.search(x, 1, r)
+    assert e.value.status == pwlq.ERR_INVALID_ARG
+    with pytest.raises(pwlq.PwlqError) as e:
+        pwlq.search(x, 4, r, workspace=torch.empty(256, dtype=torch.uint8, device="cuda"))
+    assert e.value.status == pwlq.ERR_WORKSPACE
+    with pytest.raises(pwlq.PwlqError) as e:
+        pwlq.search(x, 4, dev(W.ratio_grid(pwlq.MAX_K + 1)))
+    assert e.value.status == pwlq.ERR_UNSUPPORTED
+    torch.cuda.synchronize()
