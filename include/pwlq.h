@@ -137,6 +137,29 @@ int pwlq_encode_host(const float* x_host, const int64_t* row_offsets_host, int64
                      void* dev_scratch, size_t dev_scratch_bytes, float** y_dev_out,
                      void* stream);
 
+/* No counterpart in the paper: a packaging variant of pwlq_search for callers that cannot
+ * allocate device memory -- for example a plugin inside an application whose own memory pool
+ * already holds the whole device (cudaMalloc fails or is against the host's rules), a
+ * latency-critical loop that must avoid cudaMalloc's device-wide synchronisation, or a component
+ * that is only ever handed input and output buffers.  It computes exactly what pwlq_search
+ * computes for a dense [C, n] tensor (same kernels, bit-identical results), but its workspace is
+ * a fixed array of PWLQ_NOALLOC_SCRATCH_BYTES in device global memory that belongs to the library
+ * image; every GPU on which the library is used carries that array until the process exits.
+ *   - The call allocates nothing and calls no allocating routine; the caller passes only inputs
+ *     and outputs.  status_out (device, 4 bytes, may be NULL) receives the device status word.
+ *   - Problems whose workspace need, pwlq_search_workspace_bytes(C, n, K), exceeds
+ *     PWLQ_NOALLOC_SCRATCH_BYTES are rejected with PWLQ_ERR_UNSUPPORTED and nothing is enqueued.
+ *   - The first call on each device looks up the array's device address (with that device
+ *     current).  Make that first call outside any stream capture.
+ *   - All calls on a device share the one array.  Each call rewrites everything it later reads,
+ *     so leftovers of earlier calls are harmless, but two calls that can overlap on the GPU
+ *     (different streams, no ordering between them) race on it: order them. */
+#define PWLQ_NOALLOC_SCRATCH_BYTES (4 << 20)
+int pwlq_search_noalloc(const float* x, int64_t C, int64_t n, int bits, const float* ratios,
+                        int K, const float* m, float* p_out, float* err_out, int32_t* idx_out,
+                        float* sse_all, int32_t* status_out, void* stream);
+size_t pwlq_search_noalloc_max_bytes(void);
+
 /* Text for a status value (static storage). */
 const char* pwlq_status_string(int status);
 /* Library version, "major.minor". */

@@ -37,6 +37,8 @@ _SIGNATURES = {
     "pwlq_encode_host_scratch_bytes": (_SZ, [_I64, _I64, _I64, _INT]),
     "pwlq_encode_host": (_INT, [_P, _P, _I64, _I64, _I64, _INT, _P, _INT, _P, _P, _P, _P, _P, _P,
                                 _INT, _P, _SZ, _P, _P]),
+    "pwlq_search_noalloc": (_INT, [_P, _I64, _I64, _INT, _P, _INT, _P, _P, _P, _P, _P, _P, _P]),
+    "pwlq_search_noalloc_max_bytes": (_SZ, []),
     "pwlq_status_string": (ctypes.c_char_p, [_INT]),
     "pwlq_version": (ctypes.c_char_p, []),
 }
@@ -157,6 +159,36 @@ def search(x, bits, ratios, m=None, row_offsets=None, max_n=None, want_sse=False
     out = dict(out)
     out["workspace"] = workspace
     return out
+
+
+def search_noalloc(x, bits, ratios, m=None, want_sse=False, stream=None):
+    """``pwlq_search`` for callers that cannot allocate device memory: the workspace is a fixed
+    array inside the library (``noalloc_max_bytes()`` per GPU), shared by all calls on a device,
+    so overlapping calls must be ordered by the caller.  Dense ``[C, n]`` input only; problems
+    that need more workspace than the array raise ``PwlqError(ERR_UNSUPPORTED)``.  The output
+    tensors created here are a convenience of this Python wrapper; the C entry point itself only
+    receives inputs and outputs.  Returns dict(p, err, idx, sse or None, status)."""
+    lib = load_library()
+    C, n, _ = _shape(x, None)
+    K = ratios.numel()
+    out = {"p": torch.empty(C, dtype=torch.float32, device=x.device),
+           "err": torch.empty(C, dtype=torch.float32, device=x.device),
+           "idx": torch.empty(C, dtype=torch.int32, device=x.device),
+           "sse": torch.empty((C, K), dtype=torch.float32, device=x.device) if want_sse else None,
+           "status": torch.zeros(1, dtype=torch.int32, device=x.device)}
+    rc = lib.pwlq_search_noalloc(_dev(x, torch.float32, "x"), C, n, int(bits),
+                                 _dev(ratios, torch.float32, "ratios"), K,
+                                 _dev(m, torch.float32, "m"), _dev(out["p"], torch.float32, "p"),
+                                 _dev(out["err"], torch.float32, "err"),
+                                 _dev(out["idx"], torch.int32, "idx"),
+                                 _dev(out["sse"], torch.float32, "sse"),
+                                 _dev(out["status"], torch.int32, "status"), _stream(stream))
+    _check(rc, "pwlq_search_noalloc")
+    return out
+
+
+def noalloc_max_bytes() -> int:
+    return int(load_library().pwlq_search_noalloc_max_bytes())
 
 
 def search_status(workspace) -> int:
