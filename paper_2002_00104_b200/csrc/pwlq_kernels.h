@@ -15,6 +15,7 @@ cudaError_t launch_absmax(const float* x, const int64_t* row_offsets, int64_t C,
                           int64_t total, float* m_out, cudaStream_t stream);
 
 struct SearchPlan {
+    int64_t max_n;         // longest row
     int64_t tiles;         // tiles per row (by the longest row)
     size_t off_m;          // workspace offset of the internally computed ranges [C] floats
     size_t off_partials;   // workspace offset of the partial sums [C * tiles * K] doubles (tiles > 1)

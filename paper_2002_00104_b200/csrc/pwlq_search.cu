@@ -1,12 +1,29 @@
 // Breakpoint search: for every row and each of K candidate breakpoints p_k = m * ratio_k,
 // SSE_k = sum_i (pw(x_i; b, m, p_k) - x_i)^2 with the quantizer of Eq. 3, then the first minimal
-// k (grid form of Eq. 6).
+// k (grid form of Eq. 6).  Bound by the FP32 pipe: n * K evaluations per row, 4 bytes of HBM
+// traffic per value.
 //
-// One CTA per (row, tile of at most kSearchTile values).  The tile's magnitudes are staged once
-// in shared memory; every lane owns one candidate and walks the tile with 128-bit shared-memory
-// broadcasts, so HBM is read once per value and no per-candidate cross-lane reduction exists.
-// Sums run in binary32 over at most 256 terms per accumulator and are then carried in binary64,
-// always in the same order.
+// One CTA per (row, tile of at most kSearchTile values).
+//   1. The tile's magnitudes a = min(|x|, m) are bucketed by the candidate interval they fall in
+//      (j(a) = number of candidates with p_k < a) and counting-sorted into shared memory, with a
+//      deterministic placement (per-warp histograms + in-warp ranks), so that for candidate k the
+//      center values (a <= p_k) are exactly the first B_k entries and the tail values the rest.
+//   2. Every lane owns one candidate; a warp owns 32 consecutive candidates and walks the sorted
+//      tile with 128-bit shared-memory broadcasts.  Entries below the warp's lowest boundary run a
+//      select-free center loop, entries above its highest boundary a select-free tail loop, both
+//      on packed fp32x2 FMAs (two values per instruction); only the entries between the two
+//      boundaries need the per-lane region select.  No per-candidate cross-lane reduction exists.
+//   3. Sums run in binary32 over at most 256 terms per accumulator, are then carried in binary64,
+//      always in the same order: results are bit-reproducible.
+// Grids that are not ascending skip the sort and evaluate the region select for every (value,
+// candidate); grids with more than kSortMaxK candidates take a kernel that only does that.
+//
+// Fused arithmetic (per value and candidate; r, q, e in binary32):
+//     r = fma(u, inv, 1.5 * 2^23); q = r - 1.5 * 2^23      round-half-even of u * inv
+//     e = fma(q, -s, u)                                      u = a - z;  e = -(v - a) up to rounding
+// which differs from the operation-by-operation sequence of Eq. 1 only in rounding; the relative
+// effect on a sum is about 3 L 2^-23 / sqrt(n).  Rows shorter than L^2 / 2 therefore use the
+// unfused reconstruction v = (q * s) + z, e = v - a instead.
 #include "pwlq_common.cuh"
 #include "pwlq_kernels.h"
 
@@ -14,7 +31,9 @@ namespace pwlq {
 
 constexpr int kSThreads = 256;
 constexpr int kSWarps = kSThreads / 32;
-constexpr int kChunkVec = 256;   // float4 vectors per binary32 accumulation run
+constexpr int kChunkVec = 256;     // float4 vectors per binary32 accumulation run
+constexpr int kSortMaxK = 1024;    // largest K handled by the sorted kernel
+constexpr float kMagic = 12582912.0f;   // 1.5 * 2^23: adding it rounds to the nearest integer
 
 struct SearchArgs {
     const float* x;
@@ -23,6 +42,7 @@ struct SearchArgs {
     const float* ratios;
     int K;
     int bits;
+    int cap;            // tile capacity in values (multiple of 4, <= kSearchTile)
     int64_t tiles;
     double* partials;
     float* p_out;
@@ -32,6 +52,35 @@ struct SearchArgs {
     int* status;
 };
 
+// ---------------------------------------------------------------------------- packed fp32x2
+typedef unsigned long long u64;
+__device__ __forceinline__ u64 pack2(float lo, float hi) {
+    u64 r; asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi)); return r;
+}
+__device__ __forceinline__ void unpack2(u64 v, float& lo, float& hi) {
+    asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+}
+__device__ __forceinline__ u64 fma2(u64 a, u64 b, u64 c) {
+    u64 d; asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c)); return d;
+}
+__device__ __forceinline__ u64 add2(u64 a, u64 b) {
+    u64 d; asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b)); return d;
+}
+// Unfused reconstruction error of a pair of values: e = ((q * s) + z) - a, one rounding per
+// operation.  Done with scalar intrinsics: the assembler contracts a packed mul.rn.f32x2 followed
+// by add.rn.f32x2 into one packed FMA (observed on the device: the pair loses the product's
+// rounding, also when the product is written as fma(q, s, -0)), which the scalar forms never do.
+template <bool WITH_Z>
+__device__ __forceinline__ u64 exact_err2(u64 q, float s, float z, u64 a) {
+    float q0, q1, a0, a1;
+    unpack2(q, q0, q1);
+    unpack2(a, a0, a1);
+    float v0 = __fmul_rn(q0, s), v1 = __fmul_rn(q1, s);
+    if (WITH_Z) { v0 = __fadd_rn(v0, z); v1 = __fadd_rn(v1, z); }
+    return pack2(__fsub_rn(v0, a0), __fsub_rn(v1, a1));
+}
+
+// ------------------------------------------------------------------------------ reductions
 // First minimal (value, index) over K sums held in shared memory; result valid in thread 0.
 __device__ __forceinline__ void block_argmin(const double* sse, int K, double* red_val,
                                              int* red_idx, double& best_out, int& idx_out) {
@@ -85,80 +134,12 @@ __device__ __forceinline__ void write_row_result(const SearchArgs& a, int64_t ro
     if (a.err_out) a.err_out[row] = (float)best;
 }
 
-// Squared error of one magnitude under one candidate, operation by operation as in Eq. 1 / Eq. 3.
-__device__ __forceinline__ float sq_err_acc(float a, const PieceParams& P, float acc) {
-    const bool tail = a > P.p;
-    const float z = tail ? P.p : 0.0f;
-    const float inv = tail ? P.inv2 : P.inv1;
-    const float s = tail ? P.s2 : P.s1;
-    const float u = __fsub_rn(a, z);
-    const float t = __fmul_rn(u, inv);
-    const float q = rintf(t);                       // t <= L (1 + 2^-22): saturation cannot trigger
-    float v = __fmul_rn(q, s);
-    v = __fadd_rn(v, z);
-    const float e = __fsub_rn(v, a);
-    return __fmaf_rn(e, e, acc);
-}
-
-__global__ void __launch_bounds__(kSThreads)
-search_kernel(SearchArgs a) {
-    extern __shared__ __align__(16) unsigned char smem_raw[];
-    const int64_t row = blockIdx.x / a.tiles;
-    const int64_t tile = blockIdx.x - row * a.tiles;
-    const int64_t beg = a.rows.begin(row), end = a.rows.begin(row + 1);
-    const int64_t t_beg = beg + tile * kSearchTile;
-    if (t_beg >= end && tile > 0) return;            // this row has fewer tiles than the longest
-    const int cnt = (int)min((int64_t)kSearchTile, end - t_beg);
-    const float m = a.m[row];
-    const bool finite = __float_as_uint(m) < 0x7f800000u;
-    if (!finite || !(m > 0.0f) || cnt <= 0) {
-        if (!finite && threadIdx.x == 0 && tile == 0) atomicOr(a.status, kStatusNonFinite);
-        if (a.tiles == 1) write_degenerate_row(a, row);
-        return;                                      // tiles > 1: the combine kernel handles it
-    }
-
+// Sums the element slices of every candidate, then either stores the tile's partial sums or
+// finishes the row (all sums, argmin).  part: [E][K] binary64 in shared memory.
+__device__ __forceinline__ void finish_tile(const SearchArgs& a, int64_t row, int64_t tile,
+                                            float m, double* part, int E, double* red_val,
+                                            int* red_idx) {
     const int K = a.K;
-    const int G = (K + 31) / 32;                     // candidate groups of one warp
-    const int E = (G >= kSWarps) ? 1 : (kSWarps / G);  // element slices per group
-    const int cnt4 = (cnt + 3) >> 2;
-
-    float* tile_s = reinterpret_cast<float*>(smem_raw);                       // [cnt4 * 4]
-    double* part = reinterpret_cast<double*>(smem_raw + (size_t)((kSearchTile * 4 + 15) & ~15));
-    __shared__ double red_val[kSWarps];
-    __shared__ int red_idx[kSWarps];
-
-    for (int i = threadIdx.x; i < cnt4 * 4; i += kSThreads)
-        tile_s[i] = (i < cnt) ? fminf(fabsf(a.x[t_beg + i]), m) : 0.0f;   // zero padding: error 0
-    __syncthreads();
-
-    const float Lf = (float)((1 << (a.bits - 1)) - 1);
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    const float4* tile4 = reinterpret_cast<const float4*>(tile_s);
-    for (int item = warp; item < G * E; item += kSWarps) {
-        const int g = item % G, e = item / G;
-        const int k = g * 32 + lane;
-        const int lo = (int)((int64_t)cnt4 * e / E), hi = (int)((int64_t)cnt4 * (e + 1) / E);
-        if (k < K) {
-            const PieceParams P = make_params(m, __fmul_rn(m, a.ratios[k]), Lf);
-            double dacc = 0.0;
-            for (int base = lo; base < hi; base += kChunkVec) {
-                const int stop = min(base + kChunkVec, hi);
-                float a0 = 0.0f, a1 = 0.0f, a2 = 0.0f, a3 = 0.0f;
-#pragma unroll 2
-                for (int j = base; j < stop; ++j) {
-                    const float4 v = tile4[j];
-                    a0 = sq_err_acc(v.x, P, a0);
-                    a1 = sq_err_acc(v.y, P, a1);
-                    a2 = sq_err_acc(v.z, P, a2);
-                    a3 = sq_err_acc(v.w, P, a3);
-                }
-                dacc += ((double)a0 + (double)a1) + ((double)a2 + (double)a3);
-            }
-            part[e * K + k] = dacc;
-        }
-    }
-    __syncthreads();
-
     for (int k = threadIdx.x; k < K; k += kSThreads) {
         double tot = part[k];
         for (int e = 1; e < E; ++e) tot += part[e * K + k];
@@ -176,6 +157,366 @@ search_kernel(SearchArgs a) {
     if (threadIdx.x == 0) write_row_result(a, row, m, best, idx);
 }
 
+// ------------------------------------------------------------------- per-value evaluations
+// Region select for one (value, candidate); EXACT_V chooses the unfused reconstruction.
+template <bool EXACT_V>
+__device__ __forceinline__ float sq_err_select(float a, const PieceParams& P, float acc) {
+    const bool tail = a > P.p;
+    const float z = tail ? P.p : 0.0f;
+    const float inv = tail ? P.inv2 : P.inv1;
+    const float s = tail ? P.s2 : P.s1;
+    const float u = __fsub_rn(a, z);
+    if (EXACT_V) {
+        const float t = __fmul_rn(u, inv);
+        const float q = __fsub_rn(__fadd_rn(t, kMagic), kMagic);   // rint(t), 0 <= t < 2^22
+        float v = __fmul_rn(q, s);
+        v = __fadd_rn(v, z);
+        const float e = __fsub_rn(v, a);
+        return __fmaf_rn(e, e, acc);
+    } else {
+        const float q = __fsub_rn(__fmaf_rn(u, inv, kMagic), kMagic);
+        const float e = __fmaf_rn(q, -s, u);
+        return __fmaf_rn(e, e, acc);
+    }
+}
+
+struct Acc {
+    u64 v0, v1;            // packed accumulators of the select-free loops
+    float s0, s1, s2, s3;  // scalar accumulators of the select loop
+    double d;              // binary64 carry
+    __device__ __forceinline__ void clear() { v0 = v1 = 0ull; s0 = s1 = s2 = s3 = 0.0f; }
+    __device__ __forceinline__ void flush() {
+        float a, b, c, e;
+        unpack2(v0, a, b);
+        unpack2(v1, c, e);
+        d += ((double)a + (double)b) + ((double)c + (double)e);
+        d += ((double)s0 + (double)s1) + ((double)s2 + (double)s3);
+        clear();
+    }
+};
+
+// Candidate constants as fp32x2 pairs for the packed loops.
+struct Pairs {
+    u64 inv1, ns1, inv2, ns2, np, magic, nmagic;
+};
+
+template <bool EXACT_V>
+__device__ __forceinline__ void center_vec(const ulonglong2 v, const Pairs& c,
+                                           const PieceParams& P, Acc& A) {
+    const u64 r0 = fma2(v.x, c.inv1, c.magic), r1 = fma2(v.y, c.inv1, c.magic);
+    const u64 q0 = add2(r0, c.nmagic), q1 = add2(r1, c.nmagic);
+    u64 e0, e1;
+    if (EXACT_V) {
+        e0 = exact_err2<false>(q0, P.s1, 0.0f, v.x);
+        e1 = exact_err2<false>(q1, P.s1, 0.0f, v.y);
+    } else {
+        e0 = fma2(q0, c.ns1, v.x);
+        e1 = fma2(q1, c.ns1, v.y);
+    }
+    A.v0 = fma2(e0, e0, A.v0);
+    A.v1 = fma2(e1, e1, A.v1);
+}
+
+template <bool EXACT_V>
+__device__ __forceinline__ void tail_vec(const ulonglong2 v, const Pairs& c,
+                                         const PieceParams& P, Acc& A) {
+    const u64 u0 = add2(v.x, c.np), u1 = add2(v.y, c.np);
+    const u64 r0 = fma2(u0, c.inv2, c.magic), r1 = fma2(u1, c.inv2, c.magic);
+    const u64 q0 = add2(r0, c.nmagic), q1 = add2(r1, c.nmagic);
+    u64 e0, e1;
+    if (EXACT_V) {
+        e0 = exact_err2<true>(q0, P.s2, P.p, v.x);
+        e1 = exact_err2<true>(q1, P.s2, P.p, v.y);
+    } else {
+        e0 = fma2(q0, c.ns2, u0);
+        e1 = fma2(q1, c.ns2, u1);
+    }
+    A.v0 = fma2(e0, e0, A.v0);
+    A.v1 = fma2(e1, e1, A.v1);
+}
+
+template <bool EXACT_V>
+__device__ __forceinline__ void select_vec(const float4 v, const PieceParams& P, Acc& A) {
+    A.s0 = sq_err_select<EXACT_V>(v.x, P, A.s0);
+    A.s1 = sq_err_select<EXACT_V>(v.y, P, A.s1);
+    A.s2 = sq_err_select<EXACT_V>(v.z, P, A.s2);
+    A.s3 = sq_err_select<EXACT_V>(v.w, P, A.s3);
+}
+
+// Walks float4 vectors [lo, hi) of the tile in runs of kChunkVec with one of the three bodies.
+// MODE 0: center, 1: tail, 2: select.
+template <int MODE, bool EXACT_V>
+__device__ __forceinline__ void walk(const float* tile_s, int lo, int hi, const Pairs& c,
+                                     const PieceParams& P, Acc& A) {
+    const ulonglong2* t2 = reinterpret_cast<const ulonglong2*>(tile_s);
+    const float4* t4 = reinterpret_cast<const float4*>(tile_s);
+    for (int base = lo; base < hi; base += kChunkVec) {
+        const int stop = min(base + kChunkVec, hi);
+        if (MODE == 2) {
+#pragma unroll 2
+            for (int j = base; j < stop; ++j) select_vec<EXACT_V>(t4[j], P, A);
+        } else {
+#pragma unroll 4
+            for (int j = base; j < stop; ++j) {
+                if (MODE == 0) center_vec<EXACT_V>(t2[j], c, P, A);
+                else tail_vec<EXACT_V>(t2[j], c, P, A);
+            }
+        }
+        A.flush();
+    }
+}
+
+__host__ __device__ inline int slices_for(int K) {
+    const int G = (K + 31) / 32;
+    return (G >= kSWarps) ? 1 : (kSWarps / G);
+}
+
+// Region select for every (value, candidate) of an unsorted tile (zero-padded to whole vectors).
+__device__ __forceinline__ void eval_unsorted(const SearchArgs& a, const float* tile_s,
+                                              double* part, int cnt4, float m, int E) {
+    const int K = a.K;
+    const int G = (K + 31) / 32;
+    const float Lf = (float)((1 << (a.bits - 1)) - 1);
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const Pairs unused = {};
+    for (int item = warp; item < G * E; item += kSWarps) {
+        const int g = item % G, e = item / G;
+        const int k = g * 32 + lane;
+        const int lo = (int)((int64_t)cnt4 * e / E), hi = (int)((int64_t)cnt4 * (e + 1) / E);
+        if (k < K) {
+            const PieceParams P = make_params(m, __fmul_rn(m, a.ratios[k]), Lf);
+            Acc A;
+            A.clear();
+            A.d = 0.0;
+            walk<2, true>(tile_s, lo, hi, unused, P, A);
+            part[e * K + k] = A.d;
+        }
+    }
+}
+
+__device__ __forceinline__ bool row_setup(const SearchArgs& a, int64_t& row, int64_t& tile,
+                                          int64_t& t_beg, int& cnt, float& m) {
+    row = blockIdx.x / a.tiles;
+    tile = blockIdx.x - row * a.tiles;
+    const int64_t beg = a.rows.begin(row), end = a.rows.begin(row + 1);
+    t_beg = beg + tile * (int64_t)a.cap;
+    if (t_beg >= end && tile > 0) return false;      // this row has fewer tiles than the longest
+    cnt = (int)min((int64_t)a.cap, end - t_beg);
+    m = a.m[row];
+    const bool finite = __float_as_uint(m) < 0x7f800000u;
+    if (!finite || !(m > 0.0f) || cnt <= 0) {
+        if (!finite && threadIdx.x == 0 && tile == 0) atomicOr(a.status, kStatusNonFinite);
+        if (a.tiles == 1) write_degenerate_row(a, row);
+        return false;                                // tiles > 1: the combine kernel handles it
+    }
+    return true;
+}
+
+// ------------------------------------------------------------------------- sorted kernel
+// Shared memory: sorted tile | bucket ids | candidate breakpoints | bucket starts | per-warp
+// histograms | per-slice sums.
+struct SortedSmem {
+    float* tile;        // [cap + 4]
+    uint16_t* jbuf;     // [cap]
+    float* ps;          // [K]
+    int* start;         // [K + 2]
+    uint16_t* hist;     // [kSWarps][K + 2]
+    double* part;       // [E][K]
+};
+__host__ __device__ inline size_t sorted_smem_layout(int cap, int K, int E, size_t off[6]) {
+    size_t o = 0;
+    auto take = [&](size_t bytes) { size_t r = o; o = (o + bytes + 15) & ~(size_t)15; return r; };
+    off[0] = take(sizeof(float) * (size_t)(cap + 4));
+    off[1] = take(sizeof(uint16_t) * (size_t)cap);
+    off[2] = take(sizeof(float) * (size_t)K);
+    off[3] = take(sizeof(int) * (size_t)(K + 2));
+    off[4] = take(sizeof(uint16_t) * (size_t)kSWarps * (size_t)(K + 2));
+    off[5] = take(sizeof(double) * (size_t)E * (size_t)K);
+    return o;
+}
+
+template <bool EXACT_V>
+__device__ __forceinline__ void eval_sorted(const SearchArgs& a, const SortedSmem& S, float m,
+                                            int n4, int pad, int E) {
+    const int K = a.K;
+    const int G = (K + 31) / 32;
+    const float Lf = (float)((1 << (a.bits - 1)) - 1);
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    for (int item = warp; item < G * E; item += kSWarps) {
+        const int g = item % G, e = item / G;
+        const int k0 = g * 32, k1 = min(k0 + 31, K - 1);
+        const int k = min(k0 + lane, K - 1);
+        const int lo = (int)((int64_t)n4 * e / E), hi = (int)((int64_t)n4 * (e + 1) / E);
+        // entries [0, B_k) of the sorted tile are the center values of candidate k
+        const int c_hi = (pad + S.start[k0 + 1]) >> 2;        // whole vectors below every boundary
+        const int t_lo = (pad + S.start[k1 + 1] + 3) >> 2;    // whole vectors above every boundary
+        const PieceParams P = make_params(m, S.ps[k], Lf);
+        Pairs c;
+        c.inv1 = pack2(P.inv1, P.inv1); c.ns1 = pack2(-P.s1, -P.s1);
+        c.inv2 = pack2(P.inv2, P.inv2); c.ns2 = pack2(-P.s2, -P.s2);
+        c.np = pack2(-P.p, -P.p);
+        c.magic = pack2(kMagic, kMagic); c.nmagic = pack2(-kMagic, -kMagic);
+        Acc A;
+        A.clear();
+        A.d = 0.0;
+        walk<0, EXACT_V>(S.tile, lo, min(hi, c_hi), c, P, A);
+        walk<2, EXACT_V>(S.tile, max(lo, c_hi), min(hi, t_lo), c, P, A);
+        walk<1, EXACT_V>(S.tile, max(lo, t_lo), hi, c, P, A);
+        if (k0 + lane < K) S.part[e * K + k0 + lane] = A.d;
+    }
+}
+
+__global__ void __launch_bounds__(kSThreads)
+search_sorted_kernel(SearchArgs a) {
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    __shared__ double red_val[kSWarps];
+    __shared__ int red_idx[kSWarps];
+    __shared__ int warp_sums[kSWarps];
+    int64_t row, tile, t_beg;
+    int cnt;
+    float m;
+    if (!row_setup(a, row, tile, t_beg, cnt, m)) return;
+
+    const int K = a.K;
+    const int E = slices_for(K);
+    size_t off[6];
+    sorted_smem_layout(a.cap, K, E, off);
+    SortedSmem S;
+    S.tile = reinterpret_cast<float*>(smem_raw + off[0]);
+    S.jbuf = reinterpret_cast<uint16_t*>(smem_raw + off[1]);
+    S.ps = reinterpret_cast<float*>(smem_raw + off[2]);
+    S.start = reinterpret_cast<int*>(smem_raw + off[3]);
+    S.hist = reinterpret_cast<uint16_t*>(smem_raw + off[4]);
+    S.part = reinterpret_cast<double*>(smem_raw + off[5]);
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const unsigned full = 0xffffffffu;
+    const int HS = K + 2;                           // histogram stride; bucket K + 1 = "no value"
+
+    for (int k = threadIdx.x; k < K; k += kSThreads) S.ps[k] = __fmul_rn(m, a.ratios[k]);
+    for (int i = threadIdx.x; i < kSWarps * HS; i += kSThreads) S.hist[i] = 0;
+    __syncthreads();
+    int unordered = 0;
+    for (int k = threadIdx.x + 1; k < K; k += kSThreads) unordered |= (S.ps[k] < S.ps[k - 1]);
+    if (__syncthreads_or(unordered)) {
+        // the grid is not ascending: no sorted structure to exploit
+        const int cnt4 = (cnt + 3) >> 2;
+        for (int i = threadIdx.x; i < cnt4 * 4; i += kSThreads)
+            S.tile[i] = (i < cnt) ? fminf(fabsf(a.x[t_beg + i]), m) : 0.0f;
+        __syncthreads();
+        eval_unsorted(a, S.tile, S.part, cnt4, m, E);
+        __syncthreads();
+        finish_tile(a, row, tile, m, S.part, E, red_val, red_idx);
+        return;
+    }
+
+    // ---- pass 1: bucket of every value, per-warp histograms (each warp owns a contiguous segment)
+    const int seg = (((cnt + kSWarps - 1) / kSWarps) + 31) & ~31;
+    const int w_beg = min(warp * seg, cnt), w_end = min(w_beg + seg, cnt);
+    uint16_t* myhist = S.hist + warp * HS;
+    for (int base = w_beg; base < w_end; base += 32) {
+        const int i = base + lane;
+        int j = K + 1;
+        if (i < w_end) {
+            const float av = fminf(fabsf(a.x[t_beg + i]), m);
+            int lo = 0, hi = K;                      // j = number of candidates with p_k < a
+            while (lo < hi) {
+                const int mid = (lo + hi) >> 1;
+                if (S.ps[mid] < av) lo = mid + 1; else hi = mid;
+            }
+            j = lo;
+            S.jbuf[i] = (uint16_t)j;
+        }
+        const unsigned peers = __match_any_sync(full, j);
+        if (j <= K && lane == __ffs(peers) - 1) myhist[j] = (uint16_t)(myhist[j] + __popc(peers));
+        __syncwarp();
+    }
+    __syncthreads();
+
+    // ---- exclusive scan over buckets (and over warps inside a bucket)
+    {
+        const int per = (K + 1 + kSThreads - 1) / kSThreads;
+        const int j0 = min(threadIdx.x * per, K + 1), j1 = min(j0 + per, K + 1);
+        int local = 0;
+        for (int j = j0; j < j1; ++j)
+            for (int w = 0; w < kSWarps; ++w) local += S.hist[w * HS + j];
+        int incl = local;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const int t = __shfl_up_sync(full, incl, o);
+            if (lane >= o) incl += t;
+        }
+        if (lane == 31) warp_sums[warp] = incl;
+        __syncthreads();
+        int run = incl - local;
+        for (int w = 0; w < warp; ++w) run += warp_sums[w];
+        for (int j = j0; j < j1; ++j) {
+            S.start[j] = run;
+            for (int w = 0; w < kSWarps; ++w) {
+                const int c = S.hist[w * HS + j];
+                S.hist[w * HS + j] = (uint16_t)run;
+                run += c;
+            }
+        }
+        if (threadIdx.x == 0) S.start[K + 1] = cnt;
+    }
+    const int pad = (4 - (cnt & 3)) & 3;            // zeros in front: error 0 under every candidate
+    if (threadIdx.x < pad) S.tile[threadIdx.x] = 0.0f;
+    __syncthreads();
+
+    // ---- pass 2: stable placement (segment order, then lane order inside a group of 32)
+    for (int base = w_beg; base < w_end; base += 32) {
+        const int i = base + lane;
+        int j = K + 1;
+        float av = 0.0f;
+        if (i < w_end) {
+            j = S.jbuf[i];
+            av = fminf(fabsf(a.x[t_beg + i]), m);
+        }
+        const unsigned peers = __match_any_sync(full, j);
+        int pos = 0;
+        if (j <= K) pos = myhist[j] + __popc(peers & ((1u << lane) - 1u));
+        __syncwarp();
+        if (j <= K) {
+            S.tile[pad + pos] = av;
+            if (lane == __ffs(peers) - 1) myhist[j] = (uint16_t)(myhist[j] + __popc(peers));
+        }
+        __syncwarp();
+    }
+    __syncthreads();
+
+    // ---- evaluation
+    const int n4 = (pad + cnt) >> 2;
+    const int64_t n_row = a.rows.begin(row + 1) - a.rows.begin(row);
+    const int64_t L = (1 << (a.bits - 1)) - 1;
+    if (2 * n_row >= L * L) eval_sorted<false>(a, S, m, n4, pad, E);
+    else                    eval_sorted<true>(a, S, m, n4, pad, E);
+    __syncthreads();
+    finish_tile(a, row, tile, m, S.part, E, red_val, red_idx);
+}
+
+// ------------------------------------------------------------------------ generic kernel
+// More than kSortMaxK candidates: region select for every (value, candidate).
+__global__ void __launch_bounds__(kSThreads)
+search_generic_kernel(SearchArgs a) {
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    __shared__ double red_val[kSWarps];
+    __shared__ int red_idx[kSWarps];
+    int64_t row, tile, t_beg;
+    int cnt;
+    float m;
+    if (!row_setup(a, row, tile, t_beg, cnt, m)) return;
+    const int E = slices_for(a.K);
+    const int cnt4 = (cnt + 3) >> 2;
+    float* tile_s = reinterpret_cast<float*>(smem_raw);
+    double* part = reinterpret_cast<double*>(smem_raw + (((size_t)a.cap * 4 + 15) & ~(size_t)15));
+    for (int i = threadIdx.x; i < cnt4 * 4; i += kSThreads)
+        tile_s[i] = (i < cnt) ? fminf(fabsf(a.x[t_beg + i]), m) : 0.0f;   // zero padding: error 0
+    __syncthreads();
+    eval_unsorted(a, tile_s, part, cnt4, m, E);
+    __syncthreads();
+    finish_tile(a, row, tile, m, part, E, red_val, red_idx);
+}
+
 // Combines the tiles of long rows in ascending tile order and takes the argmin.
 __global__ void __launch_bounds__(kSThreads)
 search_combine_kernel(SearchArgs a) {
@@ -188,7 +529,7 @@ search_combine_kernel(SearchArgs a) {
     const float m = a.m[row];
     const bool finite = __float_as_uint(m) < 0x7f800000u;
     if (!finite || !(m > 0.0f) || n_row <= 0) { write_degenerate_row(a, row); return; }
-    const int64_t nt = (n_row + kSearchTile - 1) / kSearchTile;
+    const int64_t nt = (n_row + a.cap - 1) / a.cap;
     const int K = a.K;
     for (int k = threadIdx.x; k < K; k += kSThreads) {
         const double* src = a.partials + (size_t)row * a.tiles * K + k;
@@ -203,10 +544,12 @@ search_combine_kernel(SearchArgs a) {
     if (threadIdx.x == 0) write_row_result(a, row, m, best, idx);
 }
 
+// ------------------------------------------------------------------------------- host side
 static inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
 SearchPlan plan_search(int64_t C, int64_t max_n, int K) {
     SearchPlan p;
+    p.max_n = max_n;
     p.tiles = (max_n + kSearchTile - 1) / kSearchTile;
     if (p.tiles < 1) p.tiles = 1;
     p.off_m = 256;
@@ -215,12 +558,6 @@ SearchPlan plan_search(int64_t C, int64_t max_n, int K) {
     if (p.tiles > 1) p.bytes += sizeof(double) * (size_t)C * (size_t)p.tiles * (size_t)K;
     p.bytes = align_up(p.bytes, 256);
     return p;
-}
-
-static size_t search_smem_bytes(int K) {
-    const int G = (K + 31) / 32;
-    const int E = (G >= kSWarps) ? 1 : (kSWarps / G);
-    return (size_t)((kSearchTile * 4 + 15) & ~15) + sizeof(double) * (size_t)E * (size_t)K;
 }
 
 cudaError_t launch_search(const float* x, const int64_t* row_offsets, int64_t C, int64_t n,
@@ -244,6 +581,7 @@ cudaError_t launch_search(const float* x, const int64_t* row_offsets, int64_t C,
     a.K = K;
     a.bits = bits;
     a.tiles = plan.tiles;
+    a.cap = (plan.tiles > 1) ? kSearchTile : (int)((plan.max_n + 3) / 4 * 4);
     a.partials = reinterpret_cast<double*>(ws + plan.off_partials);
     a.p_out = p_out;
     a.err_out = err_out;
@@ -251,14 +589,27 @@ cudaError_t launch_search(const float* x, const int64_t* row_offsets, int64_t C,
     a.sse_all = sse_all;
     a.status = reinterpret_cast<int*>(ws);
 
-    const size_t smem = search_smem_bytes(K);
-    if (smem > 48 * 1024) {          // above the default limit: opt in (idempotent, per device)
-        e = cudaFuncSetAttribute(search_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                 (int)smem);
-        if (e != cudaSuccess) return e;
+    const int E = slices_for(K);
+    const unsigned grid = (unsigned)(C * plan.tiles);
+    if (K <= kSortMaxK) {
+        size_t off[6];
+        const size_t smem = sorted_smem_layout(a.cap, K, E, off);
+        if (smem > 48 * 1024) {      // above the default limit: opt in (idempotent, per device)
+            e = cudaFuncSetAttribute(search_sorted_kernel,
+                                     cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+            if (e != cudaSuccess) return e;
+        }
+        search_sorted_kernel<<<grid, kSThreads, smem, stream>>>(a);
+    } else {
+        const size_t smem = (((size_t)a.cap * 4 + 15) & ~(size_t)15) +
+                            sizeof(double) * (size_t)E * (size_t)K;
+        if (smem > 48 * 1024) {
+            e = cudaFuncSetAttribute(search_generic_kernel,
+                                     cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+            if (e != cudaSuccess) return e;
+        }
+        search_generic_kernel<<<grid, kSThreads, smem, stream>>>(a);
     }
-    const int64_t grid = C * plan.tiles;
-    search_kernel<<<(unsigned)grid, kSThreads, smem, stream>>>(a);
     e = cudaGetLastError();
     if (e != cudaSuccess) return e;
     if (plan.tiles > 1) {
