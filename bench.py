@@ -50,6 +50,18 @@ WORKLOADS = {
 }
 
 
+def make_workload(args, seed):
+    """The named workload; --bits / --K / --rows / --cols override its defaults (sweeps)."""
+    kw = {} if seed is None else {"seed": seed}
+    if args.workload == "laplace4096":
+        if args.rows: kw["rows"] = args.rows
+        if args.cols: kw["cols"] = args.cols
+    w = WORKLOADS[args.workload](**kw)
+    if args.bits: w.bits = args.bits
+    if args.K: w.K = args.K
+    return w
+
+
 def measured_peaks():
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(path):
@@ -146,7 +158,7 @@ def time_oracle(w: W.Workload, spans, threads: int):
 def run_reference(args, rank, world):
     if rank != 0:
         return
-    w = WORKLOADS[args.workload]()
+    w = make_workload(args, None)
     cores = os.cpu_count() or 1
     # size the per-step sample from a short calibration so that the run ends within minutes
     spans, _ = oracle_sample(w, 2e8)
@@ -187,7 +199,7 @@ def run_ours(args, rank, world, local_rank):
         dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
     pwlq.load_library()
 
-    w = WORKLOADS[args.workload](**({} if world == 1 else {"seed": 1000 + 17 * rank}))
+    w = make_workload(args, None if world == 1 else 1000 + 17 * rank)
     ratios_np = W.ratio_grid(w.K)
     max_n = int(np.diff(w.row_offsets).max())
     dense_n = w.uniform_n()
@@ -360,6 +372,10 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="resnet50", choices=sorted(WORKLOADS))
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--bits", type=int, default=0, help="override the workload's bit-width")
+    ap.add_argument("--K", type=int, default=0, help="override the number of candidates")
+    ap.add_argument("--rows", type=int, default=0, help="laplace4096 only: number of rows")
+    ap.add_argument("--cols", type=int, default=0, help="laplace4096 only: row length")
     args = ap.parse_args()
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))

@@ -24,12 +24,15 @@
 // which differs from the operation-by-operation sequence of Eq. 1 only in rounding; the relative
 // effect on a sum is about 3 L 2^-23 / sqrt(n).  Rows shorter than L^2 / 2 therefore use the
 // unfused reconstruction v = (q * s) + z, e = v - a instead.
+#include <algorithm>
+#include <cstdint>
+
 #include "pwlq_common.cuh"
 #include "pwlq_kernels.h"
 
 namespace pwlq {
 
-constexpr int kSThreads = 256;
+constexpr int kSThreads = 256;            // largest CTA; short rows run with fewer warps
 constexpr int kSWarps = kSThreads / 32;
 constexpr int kChunkVec = 256;     // float4 vectors per binary32 accumulation run
 constexpr int kSortMaxK = 1024;    // largest K handled by the sorted kernel
@@ -43,7 +46,9 @@ struct SearchArgs {
     int K;
     int bits;
     int cap;            // tile capacity in values (multiple of 4, <= kSearchTile)
-    int64_t tiles;
+    int64_t n_min, n_max;   // this launch handles the rows with n_min <= length <= n_max
+    int64_t grid_tiles;     // blockIdx.x = row * grid_tiles + tile
+    int64_t tiles;          // tiles per row in the partial-sum layout
     double* partials;
     float* p_out;
     float* err_out;
@@ -140,7 +145,7 @@ __device__ __forceinline__ void finish_tile(const SearchArgs& a, int64_t row, in
                                             float m, double* part, int E, double* red_val,
                                             int* red_idx) {
     const int K = a.K;
-    for (int k = threadIdx.x; k < K; k += kSThreads) {
+    for (int k = threadIdx.x; k < K; k += blockDim.x) {
         double tot = part[k];
         for (int e = 1; e < E; ++e) tot += part[e * K + k];
         if (a.tiles > 1) {
@@ -243,32 +248,34 @@ __device__ __forceinline__ void select_vec(const float4 v, const PieceParams& P,
     A.s3 = sq_err_select<EXACT_V>(v.w, P, A.s3);
 }
 
-// Walks float4 vectors [lo, hi) of the tile in runs of kChunkVec with one of the three bodies.
+// Walks float4 vectors first, first + step, ... (< hi) of the tile with one of the three bodies.
+// A binary32 accumulation run is closed after kChunkVec vectors; the last, shorter run stays open
+// for the caller to close (an accumulator therefore never sums more than 3 * kChunkVec terms).
 // MODE 0: center, 1: tail, 2: select.
 template <int MODE, bool EXACT_V>
-__device__ __forceinline__ void walk(const float* tile_s, int lo, int hi, const Pairs& c,
-                                     const PieceParams& P, Acc& A) {
+__device__ __forceinline__ void walk(const float* tile_s, int first, int hi, int step,
+                                     const Pairs& c, const PieceParams& P, Acc& A) {
     const ulonglong2* t2 = reinterpret_cast<const ulonglong2*>(tile_s);
     const float4* t4 = reinterpret_cast<const float4*>(tile_s);
-    for (int base = lo; base < hi; base += kChunkVec) {
-        const int stop = min(base + kChunkVec, hi);
+    for (int base = first; base < hi; base += kChunkVec * step) {
+        const int stop = min(base + kChunkVec * step, hi);
         if (MODE == 2) {
 #pragma unroll 2
-            for (int j = base; j < stop; ++j) select_vec<EXACT_V>(t4[j], P, A);
+            for (int j = base; j < stop; j += step) select_vec<EXACT_V>(t4[j], P, A);
         } else {
 #pragma unroll 4
-            for (int j = base; j < stop; ++j) {
+            for (int j = base; j < stop; j += step) {
                 if (MODE == 0) center_vec<EXACT_V>(t2[j], c, P, A);
                 else tail_vec<EXACT_V>(t2[j], c, P, A);
             }
         }
-        A.flush();
+        if (stop < hi) A.flush();
     }
 }
 
-__host__ __device__ inline int slices_for(int K) {
+__host__ __device__ inline int slices_for(int K, int warps) {
     const int G = (K + 31) / 32;
-    return (G >= kSWarps) ? 1 : (kSWarps / G);
+    return (G >= warps) ? 1 : (warps / G);
 }
 
 // Region select for every (value, candidate) of an unsorted tile (zero-padded to whole vectors).
@@ -279,7 +286,7 @@ __device__ __forceinline__ void eval_unsorted(const SearchArgs& a, const float* 
     const float Lf = (float)((1 << (a.bits - 1)) - 1);
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const Pairs unused = {};
-    for (int item = warp; item < G * E; item += kSWarps) {
+    for (int item = warp; item < G * E; item += (int)(blockDim.x >> 5)) {
         const int g = item % G, e = item / G;
         const int k = g * 32 + lane;
         const int lo = (int)((int64_t)cnt4 * e / E), hi = (int)((int64_t)cnt4 * (e + 1) / E);
@@ -288,7 +295,8 @@ __device__ __forceinline__ void eval_unsorted(const SearchArgs& a, const float* 
             Acc A;
             A.clear();
             A.d = 0.0;
-            walk<2, true>(tile_s, lo, hi, unused, P, A);
+            walk<2, true>(tile_s, lo, hi, 1, unused, P, A);
+            A.flush();
             part[e * K + k] = A.d;
         }
     }
@@ -296,9 +304,10 @@ __device__ __forceinline__ void eval_unsorted(const SearchArgs& a, const float* 
 
 __device__ __forceinline__ bool row_setup(const SearchArgs& a, int64_t& row, int64_t& tile,
                                           int64_t& t_beg, int& cnt, float& m) {
-    row = blockIdx.x / a.tiles;
-    tile = blockIdx.x - row * a.tiles;
+    row = blockIdx.x / a.grid_tiles;
+    tile = blockIdx.x - row * a.grid_tiles;
     const int64_t beg = a.rows.begin(row), end = a.rows.begin(row + 1);
+    if (end - beg < a.n_min || end - beg > a.n_max) return false;   // another launch's row
     t_beg = beg + tile * (int64_t)a.cap;
     if (t_beg >= end && tile > 0) return false;      // this row has fewer tiles than the longest
     cnt = (int)min((int64_t)a.cap, end - t_beg);
@@ -313,56 +322,114 @@ __device__ __forceinline__ bool row_setup(const SearchArgs& a, int64_t& row, int
 }
 
 // ------------------------------------------------------------------------- sorted kernel
-// Shared memory: sorted tile | bucket ids | candidate breakpoints | bucket starts | per-warp
-// histograms | per-slice sums.
+// A warp works on kCW consecutive candidates at a time; its 32 / kCW lane groups ("phases") take
+// every (32 / kCW)-th vector of the tile.  Fewer candidates per warp means fewer entries between
+// the lowest and the highest boundary, i.e. less work in the select loop.
+// Short tiles use wider groups: per work item there is a fixed cost (fetching the item, loading
+// the constants, closing the sums) that a handful of vectors per lane cannot amortise.
+constexpr int kCwLongTile = 8, kCwMidTile = 16, kCwShortTile = 32;
+constexpr int kLongTileMin = 3072, kMidTileMin = 768;     // values per tile
+__host__ __device__ inline int group_width(int cnt) {
+    return cnt >= kLongTileMin ? kCwLongTile : (cnt >= kMidTileMin ? kCwMidTile : kCwShortTile);
+}
+
+// Element slices per candidate group: enough (group, slice) work items to keep eight warps
+// busy.  Sized for the narrowest group so that one shared-memory layout serves every width.
+__host__ __device__ inline int slices_sorted(int K, int cw, int warps) {
+    const int G = (K + cw - 1) / cw;
+    const int E = (4 * warps + G - 1) / G;
+    return E < 1 ? 1 : (E > 8 ? 8 : E);
+}
+__host__ __device__ inline int max_slices_sorted(int K) {
+    return slices_sorted(K, kCwShortTile, kSWarps);    // fewest groups, most warps: most slices
+}
+
+// Shared memory: sorted tile | bucket ids | candidate breakpoints | candidate constants | bucket
+// starts | per-warp histograms | per-slice sums.
 struct SortedSmem {
     float* tile;        // [cap + 4]
-    uint16_t* jbuf;     // [cap]
+    uint32_t* jr;       // [cap]  bucket | rank << 11
     float* ps;          // [K]
+    float4* pa;         // [K]  (inv1, -s1, inv2, -s2)
     int* start;         // [K + 2]
     uint16_t* hist;     // [kSWarps][K + 2]
     double* part;       // [E][K]
 };
-__host__ __device__ inline size_t sorted_smem_layout(int cap, int K, int E, size_t off[6]) {
+__host__ __device__ inline size_t sorted_smem_layout(int cap, int K, int E, size_t off[7]) {
     size_t o = 0;
     auto take = [&](size_t bytes) { size_t r = o; o = (o + bytes + 15) & ~(size_t)15; return r; };
     off[0] = take(sizeof(float) * (size_t)(cap + 4));
-    off[1] = take(sizeof(uint16_t) * (size_t)cap);
+    off[1] = take(sizeof(uint32_t) * (size_t)cap);
     off[2] = take(sizeof(float) * (size_t)K);
-    off[3] = take(sizeof(int) * (size_t)(K + 2));
-    off[4] = take(sizeof(uint16_t) * (size_t)kSWarps * (size_t)(K + 2));
-    off[5] = take(sizeof(double) * (size_t)E * (size_t)K);
+    off[3] = take(sizeof(float4) * (size_t)K);
+    off[4] = take(sizeof(int) * (size_t)(K + 2));
+    off[5] = take(sizeof(uint16_t) * (size_t)kSWarps * (size_t)(K + 2));
+    off[6] = take(sizeof(double) * (size_t)E * (size_t)K);
     return o;
 }
 
-template <bool EXACT_V>
-__device__ __forceinline__ void eval_sorted(const SearchArgs& a, const SortedSmem& S, float m,
-                                            int n4, int pad, int E) {
+// j(a) = number of candidates with p_k < a, for ascending ps[0..K).  A linear-grid guess is
+// verified and corrected by up to three neighbour steps; grids far from linear fall back to a
+// binary search between the bounds found so far.  Exact for every ascending grid.
+__device__ __forceinline__ int bucket_of(const float* ps, int K, float a, float p_first,
+                                         float hint_scale) {
+    int j = min((int)ceilf(fmaxf((a - p_first) * hint_scale, 0.0f)), K);
+    int lo = 0, hi = K;                               // the answer lies in [lo, hi]
+#pragma unroll
+    for (int t = 0; t < 3; ++t) {
+        if (j > 0 && !(ps[j - 1] < a)) { hi = min(hi, j - 1); --j; }
+        else if (j < K && ps[j] < a)   { lo = max(lo, j + 1); ++j; }
+        else return j;
+    }
+    while (lo < hi) {
+        const int mid = (lo + hi) >> 1;
+        if (ps[mid] < a) lo = mid + 1; else hi = mid;
+    }
+    return lo;
+}
+
+template <int kCW, bool EXACT_V>
+__device__ __forceinline__ void eval_sorted(const SearchArgs& a, const SortedSmem& S, int n4,
+                                            int pad, int E, int* next_item) {
+    constexpr int kPhases = 32 / kCW;
     const int K = a.K;
-    const int G = (K + 31) / 32;
-    const float Lf = (float)((1 << (a.bits - 1)) - 1);
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    for (int item = warp; item < G * E; item += kSWarps) {
-        const int g = item % G, e = item / G;
-        const int k0 = g * 32, k1 = min(k0 + 31, K - 1);
-        const int k = min(k0 + lane, K - 1);
+    const int G = (K + kCW - 1) / kCW;
+    const int lane = threadIdx.x & 31;
+    const int ci = lane % kCW, ph = lane / kCW;
+    const unsigned full = 0xffffffffu;
+    for (;;) {
+        // work items are handed out in order (low candidates first: for bell-shaped data their
+        // boundaries lie in the dense part of the tile, so they carry the longest select loops)
+        int item = 0;
+        if (lane == 0) item = atomicAdd(next_item, 1);
+        item = __shfl_sync(full, item, 0);
+        if (item >= G * E) break;
+        const int g = item / E, e = item - g * E;
+        const int k0 = g * kCW, k1 = min(k0 + kCW - 1, K - 1);
+        const int k = min(k0 + ci, K - 1);
         const int lo = (int)((int64_t)n4 * e / E), hi = (int)((int64_t)n4 * (e + 1) / E);
         // entries [0, B_k) of the sorted tile are the center values of candidate k
-        const int c_hi = (pad + S.start[k0 + 1]) >> 2;        // whole vectors below every boundary
-        const int t_lo = (pad + S.start[k1 + 1] + 3) >> 2;    // whole vectors above every boundary
-        const PieceParams P = make_params(m, S.ps[k], Lf);
+        const int c_hi = min(hi, (pad + S.start[k0 + 1]) >> 2);      // vectors below every boundary
+        const int t_lo = max(lo, (pad + S.start[k1 + 1] + 3) >> 2);  // vectors above every boundary
+        const float4 pa = S.pa[k];
+        PieceParams P;
+        P.p = S.ps[k]; P.inv1 = pa.x; P.s1 = -pa.y; P.inv2 = pa.z; P.s2 = -pa.w;
         Pairs c;
-        c.inv1 = pack2(P.inv1, P.inv1); c.ns1 = pack2(-P.s1, -P.s1);
-        c.inv2 = pack2(P.inv2, P.inv2); c.ns2 = pack2(-P.s2, -P.s2);
+        c.inv1 = pack2(pa.x, pa.x); c.ns1 = pack2(pa.y, pa.y);
+        c.inv2 = pack2(pa.z, pa.z); c.ns2 = pack2(pa.w, pa.w);
         c.np = pack2(-P.p, -P.p);
         c.magic = pack2(kMagic, kMagic); c.nmagic = pack2(-kMagic, -kMagic);
         Acc A;
         A.clear();
         A.d = 0.0;
-        walk<0, EXACT_V>(S.tile, lo, min(hi, c_hi), c, P, A);
-        walk<2, EXACT_V>(S.tile, max(lo, c_hi), min(hi, t_lo), c, P, A);
-        walk<1, EXACT_V>(S.tile, max(lo, t_lo), hi, c, P, A);
-        if (k0 + lane < K) S.part[e * K + k0 + lane] = A.d;
+        walk<0, EXACT_V>(S.tile, lo + ph, c_hi, kPhases, c, P, A);
+        walk<2, EXACT_V>(S.tile, max(lo, c_hi) + ph, min(hi, t_lo), kPhases, c, P, A);
+        walk<1, EXACT_V>(S.tile, t_lo + ph, hi, kPhases, c, P, A);
+        A.flush();
+        double d = A.d;                               // phases combined in a fixed order
+#pragma unroll
+        for (int o = kCW; o < 32; o <<= 1) d += __shfl_xor_sync(full, d, o);
+        if (ph == 0 && k0 + ci < K) S.part[e * K + k0 + ci] = d;
     }
 }
 
@@ -372,73 +439,106 @@ search_sorted_kernel(SearchArgs a) {
     __shared__ double red_val[kSWarps];
     __shared__ int red_idx[kSWarps];
     __shared__ int warp_sums[kSWarps];
+    __shared__ int next_item;
     int64_t row, tile, t_beg;
     int cnt;
     float m;
     if (!row_setup(a, row, tile, t_beg, cnt, m)) return;
 
     const int K = a.K;
-    const int E = slices_for(K);
-    size_t off[6];
-    sorted_smem_layout(a.cap, K, E, off);
+    const int nwarps = (int)(blockDim.x >> 5), nthreads = (int)blockDim.x;
+    const int cw = group_width(cnt);
+    const int E = min(slices_sorted(K, cw, nwarps), max(1, cnt / 512));   // a slice is worth >= 128 vectors
+    size_t off[7];
+    sorted_smem_layout(a.cap, K, max_slices_sorted(K), off);
     SortedSmem S;
     S.tile = reinterpret_cast<float*>(smem_raw + off[0]);
-    S.jbuf = reinterpret_cast<uint16_t*>(smem_raw + off[1]);
+    S.jr = reinterpret_cast<uint32_t*>(smem_raw + off[1]);
     S.ps = reinterpret_cast<float*>(smem_raw + off[2]);
-    S.start = reinterpret_cast<int*>(smem_raw + off[3]);
-    S.hist = reinterpret_cast<uint16_t*>(smem_raw + off[4]);
-    S.part = reinterpret_cast<double*>(smem_raw + off[5]);
+    S.pa = reinterpret_cast<float4*>(smem_raw + off[3]);
+    S.start = reinterpret_cast<int*>(smem_raw + off[4]);
+    S.hist = reinterpret_cast<uint16_t*>(smem_raw + off[5]);
+    S.part = reinterpret_cast<double*>(smem_raw + off[6]);
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const unsigned full = 0xffffffffu;
     const int HS = K + 2;                           // histogram stride; bucket K + 1 = "no value"
 
-    for (int k = threadIdx.x; k < K; k += kSThreads) S.ps[k] = __fmul_rn(m, a.ratios[k]);
-    for (int i = threadIdx.x; i < kSWarps * HS; i += kSThreads) S.hist[i] = 0;
+    const float Lf = (float)((1 << (a.bits - 1)) - 1);
+    for (int k = threadIdx.x; k < K; k += nthreads) {
+        const PieceParams P = make_params(m, __fmul_rn(m, a.ratios[k]), Lf);
+        S.ps[k] = P.p;
+        S.pa[k] = make_float4(P.inv1, -P.s1, P.inv2, -P.s2);
+    }
+    for (int i = threadIdx.x; i < nwarps * HS; i += nthreads) S.hist[i] = 0;
+    if (threadIdx.x == 0) next_item = 0;
     __syncthreads();
     int unordered = 0;
-    for (int k = threadIdx.x + 1; k < K; k += kSThreads) unordered |= (S.ps[k] < S.ps[k - 1]);
+    for (int k = threadIdx.x + 1; k < K; k += nthreads) unordered |= (S.ps[k] < S.ps[k - 1]);
     if (__syncthreads_or(unordered)) {
         // the grid is not ascending: no sorted structure to exploit
         const int cnt4 = (cnt + 3) >> 2;
-        for (int i = threadIdx.x; i < cnt4 * 4; i += kSThreads)
+        for (int i = threadIdx.x; i < cnt4 * 4; i += nthreads)
             S.tile[i] = (i < cnt) ? fminf(fabsf(a.x[t_beg + i]), m) : 0.0f;
         __syncthreads();
-        eval_unsorted(a, S.tile, S.part, cnt4, m, E);
+        const int Eu = slices_for(K, nwarps);         // never more slices than the sorted layout
+        eval_unsorted(a, S.tile, S.part, cnt4, m, Eu);
         __syncthreads();
-        finish_tile(a, row, tile, m, S.part, E, red_val, red_idx);
+        finish_tile(a, row, tile, m, S.part, Eu, red_val, red_idx);
         return;
     }
 
-    // ---- pass 1: bucket of every value, per-warp histograms (each warp owns a contiguous segment)
-    const int seg = (((cnt + kSWarps - 1) / kSWarps) + 31) & ~31;
+    // ---- pass 1: bucket j and rank of every value (each warp owns a contiguous segment, which
+    // it walks four groups of 32 at a time so that the four lookups overlap); jr = j | rank << 11,
+    // rank = number of earlier values of this warp's segment in the same bucket
+    const int seg = (((cnt + nwarps - 1) / nwarps) + 31) & ~31;
     const int w_beg = min(warp * seg, cnt), w_end = min(w_beg + seg, cnt);
     uint16_t* myhist = S.hist + warp * HS;
-    for (int base = w_beg; base < w_end; base += 32) {
-        const int i = base + lane;
-        int j = K + 1;
-        if (i < w_end) {
-            const float av = fminf(fabsf(a.x[t_beg + i]), m);
-            int lo = 0, hi = K;                      // j = number of candidates with p_k < a
-            while (lo < hi) {
-                const int mid = (lo + hi) >> 1;
-                if (S.ps[mid] < av) lo = mid + 1; else hi = mid;
-            }
-            j = lo;
-            S.jbuf[i] = (uint16_t)j;
+    const float p_first = S.ps[0];
+    const float span = S.ps[K - 1] - p_first;
+    const float hint_scale = span > 0.0f ? (float)(K - 1) / span : 0.0f;
+    float nxt[4];                                   // values of the next iteration, already in flight
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+        const int i = w_beg + u * 32 + lane;
+        nxt[u] = (i < w_end) ? __ldg(a.x + t_beg + i) : 0.0f;
+    }
+    for (int base = w_beg; base < w_end; base += 128) {
+        float av[4];
+        int jv[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            av[u] = fminf(fabsf(nxt[u]), m);
+            const int i = base + 128 + u * 32 + lane;
+            nxt[u] = (i < w_end) ? __ldg(a.x + t_beg + i) : 0.0f;
         }
-        const unsigned peers = __match_any_sync(full, j);
-        if (j <= K && lane == __ffs(peers) - 1) myhist[j] = (uint16_t)(myhist[j] + __popc(peers));
-        __syncwarp();
+#pragma unroll
+        for (int u = 0; u < 4; ++u)
+            jv[u] = (base + u * 32 + lane < w_end) ? bucket_of(S.ps, K, av[u], p_first, hint_scale)
+                                                   : K + 1;
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            const int i = base + u * 32 + lane;
+            const int j = jv[u];
+            const unsigned peers = __match_any_sync(full, j);
+            int before = 0;
+            if (j <= K) before = myhist[j];
+            __syncwarp();
+            if (j <= K) {
+                if (lane == __ffs(peers) - 1) myhist[j] = (uint16_t)(before + __popc(peers));
+                S.jr[i] = (uint32_t)j | ((uint32_t)(before + __popc(peers & ((1u << lane) - 1u))) << 11);
+            }
+            __syncwarp();
+        }
     }
     __syncthreads();
 
     // ---- exclusive scan over buckets (and over warps inside a bucket)
     {
-        const int per = (K + 1 + kSThreads - 1) / kSThreads;
+        const int per = (K + 1 + nthreads - 1) / nthreads;
         const int j0 = min(threadIdx.x * per, K + 1), j1 = min(j0 + per, K + 1);
         int local = 0;
         for (int j = j0; j < j1; ++j)
-            for (int w = 0; w < kSWarps; ++w) local += S.hist[w * HS + j];
+            for (int w = 0; w < nwarps; ++w) local += S.hist[w * HS + j];
         int incl = local;
 #pragma unroll
         for (int o = 1; o < 32; o <<= 1) {
@@ -451,7 +551,7 @@ search_sorted_kernel(SearchArgs a) {
         for (int w = 0; w < warp; ++w) run += warp_sums[w];
         for (int j = j0; j < j1; ++j) {
             S.start[j] = run;
-            for (int w = 0; w < kSWarps; ++w) {
+            for (int w = 0; w < nwarps; ++w) {
                 const int c = S.hist[w * HS + j];
                 S.hist[w * HS + j] = (uint16_t)run;
                 run += c;
@@ -463,24 +563,16 @@ search_sorted_kernel(SearchArgs a) {
     if (threadIdx.x < pad) S.tile[threadIdx.x] = 0.0f;
     __syncthreads();
 
-    // ---- pass 2: stable placement (segment order, then lane order inside a group of 32)
-    for (int base = w_beg; base < w_end; base += 32) {
-        const int i = base + lane;
-        int j = K + 1;
-        float av = 0.0f;
-        if (i < w_end) {
-            j = S.jbuf[i];
-            av = fminf(fabsf(a.x[t_beg + i]), m);
+    // ---- pass 2: stable placement (bucket, then warp segment, then order inside the segment)
+    for (int base = w_beg; base < w_end; base += 128) {
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            const int i = base + u * 32 + lane;
+            if (i < w_end) {
+                const uint32_t jr = S.jr[i];
+                S.tile[pad + myhist[jr & 0x7ffu] + (jr >> 11)] = fminf(fabsf(a.x[t_beg + i]), m);
+            }
         }
-        const unsigned peers = __match_any_sync(full, j);
-        int pos = 0;
-        if (j <= K) pos = myhist[j] + __popc(peers & ((1u << lane) - 1u));
-        __syncwarp();
-        if (j <= K) {
-            S.tile[pad + pos] = av;
-            if (lane == __ffs(peers) - 1) myhist[j] = (uint16_t)(myhist[j] + __popc(peers));
-        }
-        __syncwarp();
     }
     __syncthreads();
 
@@ -488,8 +580,17 @@ search_sorted_kernel(SearchArgs a) {
     const int n4 = (pad + cnt) >> 2;
     const int64_t n_row = a.rows.begin(row + 1) - a.rows.begin(row);
     const int64_t L = (1 << (a.bits - 1)) - 1;
-    if (2 * n_row >= L * L) eval_sorted<false>(a, S, m, n4, pad, E);
-    else                    eval_sorted<true>(a, S, m, n4, pad, E);
+    const bool fused = 2 * n_row >= L * L;
+    if (cw == kCwLongTile) {
+        if (fused) eval_sorted<kCwLongTile, false>(a, S, n4, pad, E, &next_item);
+        else       eval_sorted<kCwLongTile, true>(a, S, n4, pad, E, &next_item);
+    } else if (cw == kCwMidTile) {
+        if (fused) eval_sorted<kCwMidTile, false>(a, S, n4, pad, E, &next_item);
+        else       eval_sorted<kCwMidTile, true>(a, S, n4, pad, E, &next_item);
+    } else {
+        if (fused) eval_sorted<kCwShortTile, false>(a, S, n4, pad, E, &next_item);
+        else       eval_sorted<kCwShortTile, true>(a, S, n4, pad, E, &next_item);
+    }
     __syncthreads();
     finish_tile(a, row, tile, m, S.part, E, red_val, red_idx);
 }
@@ -505,7 +606,7 @@ search_generic_kernel(SearchArgs a) {
     int cnt;
     float m;
     if (!row_setup(a, row, tile, t_beg, cnt, m)) return;
-    const int E = slices_for(a.K);
+    const int E = slices_for(a.K, kSWarps);
     const int cnt4 = (cnt + 3) >> 2;
     float* tile_s = reinterpret_cast<float*>(smem_raw);
     double* part = reinterpret_cast<double*>(smem_raw + (((size_t)a.cap * 4 + 15) & ~(size_t)15));
@@ -589,18 +690,41 @@ cudaError_t launch_search(const float* x, const int64_t* row_offsets, int64_t C,
     a.sse_all = sse_all;
     a.status = reinterpret_cast<int*>(ws);
 
-    const int E = slices_for(K);
-    const unsigned grid = (unsigned)(C * plan.tiles);
     if (K <= kSortMaxK) {
-        size_t off[6];
-        const size_t smem = sorted_smem_layout(a.cap, K, E, off);
-        if (smem > 48 * 1024) {      // above the default limit: opt in (idempotent, per device)
+        // Rows are served by CTAs sized to their length: the per-row latency of the sort and of
+        // the final argmin is hidden by the number of rows in flight, and short rows fit many
+        // more small CTAs per SM.  One launch per class; a CTA whose row belongs to another
+        // class exits at once.  A dense tensor has one class.
+        struct RowClass { int64_t n_min, n_max; int threads; };
+        const RowClass classes[3] = {{0, 256, 64}, {257, 1152, 128}, {1153, INT64_MAX, 256}};
+        size_t off[7];
+        const size_t smem_max = sorted_smem_layout(a.cap, K, max_slices_sorted(K), off);
+        if (smem_max > 48 * 1024) {  // above the default limit: opt in (idempotent, per device)
             e = cudaFuncSetAttribute(search_sorted_kernel,
-                                     cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+                                     cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_max);
             if (e != cudaSuccess) return e;
         }
-        search_sorted_kernel<<<grid, kSThreads, smem, stream>>>(a);
+        const int full_cap = a.cap;
+        for (const RowClass& rc : classes) {
+            if (plan.max_n < rc.n_min) continue;
+            if (!row_offsets && n > rc.n_max) continue;           // dense: every row has length n
+            const bool longest = rc.n_max == INT64_MAX;
+            a.n_min = rc.n_min;
+            a.n_max = rc.n_max;
+            a.grid_tiles = longest ? plan.tiles : 1;
+            a.cap = longest ? full_cap
+                            : (int)((std::min<int64_t>(plan.max_n, rc.n_max) + 3) / 4 * 4);
+            const size_t smem = sorted_smem_layout(a.cap, K, max_slices_sorted(K), off);
+            search_sorted_kernel<<<(unsigned)(C * a.grid_tiles), rc.threads, smem, stream>>>(a);
+            e = cudaGetLastError();
+            if (e != cudaSuccess) return e;
+        }
+        a.cap = full_cap;
     } else {
+        const int E = slices_for(K, kSWarps);
+        a.n_min = 0;
+        a.n_max = INT64_MAX;
+        a.grid_tiles = plan.tiles;
         const size_t smem = (((size_t)a.cap * 4 + 15) & ~(size_t)15) +
                             sizeof(double) * (size_t)E * (size_t)K;
         if (smem > 48 * 1024) {
@@ -608,7 +732,7 @@ cudaError_t launch_search(const float* x, const int64_t* row_offsets, int64_t C,
                                      cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
             if (e != cudaSuccess) return e;
         }
-        search_generic_kernel<<<grid, kSThreads, smem, stream>>>(a);
+        search_generic_kernel<<<(unsigned)(C * plan.tiles), kSThreads, smem, stream>>>(a);
     }
     e = cudaGetLastError();
     if (e != cudaSuccess) return e;
