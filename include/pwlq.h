@@ -160,6 +160,13 @@ int pwlq_search_noalloc(const float* x, int64_t C, int64_t n, int bits, const fl
                         float* sse_all, int32_t* status_out, void* stream);
 size_t pwlq_search_noalloc_max_bytes(void);
 
+/* The streaming kernels (abs-max, quantize) receive their inputs through asynchronous bulk copies
+ * whose completion they await with a bounded number of polls; a wait that runs out makes the
+ * kernel stop early and sets a flag on the device.  This call reads the flags (it synchronises
+ * with the device) and returns 0, or 1 << PWLQ_ERR_TIMEOUT if any wait has expired since the
+ * library was loaded, in which case the outputs of that call are not valid. */
+int pwlq_device_status(void);
+
 /* Text for a status value (static storage). */
 const char* pwlq_status_string(int status);
 /* Library version, "major.minor". */

@@ -40,7 +40,8 @@ int search_impl(const float* x, const int64_t* ro, int64_t C, int64_t n, int64_t
         return PWLQ_ERR_INVALID_ARG;
     if (K > PWLQ_MAX_K || total > kMaxTotal) return PWLQ_ERR_UNSUPPORTED;
     const pwlq::SearchPlan plan = pwlq::plan_search(C, max_n, K);
-    if (C * plan.tiles > ((int64_t)1 << 31) - 1) return PWLQ_ERR_UNSUPPORTED;
+    if (C * plan.tiles > ((int64_t)1 << 31) - 1 || C * ((K + 31) / 32) > ((int64_t)1 << 31) - 1)
+        return PWLQ_ERR_UNSUPPORTED;
     if (!ws || ws_bytes < plan.bytes) return PWLQ_ERR_WORKSPACE;
     if (misaligned(ws, 256)) return PWLQ_ERR_INVALID_ARG;
     return from_cuda(pwlq::launch_search(x, ro, C, n, total, bits, ratios, K, m, p_out, err_out,
@@ -239,6 +240,11 @@ int pwlq_encode_host(const float* x_host, const int64_t* row_offsets_host, int64
 #undef PWLQ_TRY
     if (y_dev_out) *y_dev_out = dy;
     return PWLQ_OK;
+}
+
+int pwlq_device_status(void) {
+    const int expired = pwlq::absmax_timeout_flag() | pwlq::quantize_timeout_flag();
+    return expired ? (1 << PWLQ_ERR_TIMEOUT) : 0;
 }
 
 const char* pwlq_status_string(int status) {

@@ -41,10 +41,13 @@ __device__ __forceinline__ void quantize_mag(float a, const PieceParams& P, floa
     const float s = tail ? P.s2 : P.s1;
     const float u = __fsub_rn(a, z);
     const float t = __fmul_rn(u, inv);
-    const float q = fminf(rintf(t), Lf);             // round half to even, saturate
+    // t + 1.5 * 2^23 rounds t (0 <= t < 2^22) to the nearest integer, ties to even, exactly like
+    // rintf; the integer then sits in the low mantissa bits of r
+    const float r = __fadd_rn(t, 12582912.0f);
+    const float q = fminf(__fsub_rn(r, 12582912.0f), Lf);     // saturate
     float v = __fmul_rn(q, s);
     v = __fadd_rn(v, z);
-    q_out = (int)q;
+    q_out = min(__float_as_int(r) - 0x4B400000, (int)Lf);
     tail_out = tail ? 1 : 0;
     v_out = v;
 }
@@ -71,5 +74,57 @@ struct Rows {
 };
 
 __device__ __forceinline__ uint32_t abs_bits(float x) { return __float_as_uint(x) & 0x7fffffffu; }
+
+// Row that contains flat index i, found by one warp together (every lane passes the same i and
+// gets the same answer): a 32-ary search, three dependent rounds of loads for up to 32768 rows
+// instead of fifteen.
+__device__ __forceinline__ int64_t warp_row_of(const Rows& rows, int64_t i) {
+    if (!rows.offsets) return i / rows.n;
+    const int lane = threadIdx.x & 31;
+    int64_t lo = 0, hi = rows.C;                     // offsets[lo] <= i < offsets[hi]
+    while (hi - lo > 1) {
+        const int64_t step = (hi - lo + 31) / 32;
+        const int64_t q = lo + (int64_t)(lane + 1) * step;
+        const bool le = (q < hi) && (rows.offsets[q] <= i);     // true for a prefix of the lanes
+        const int cnt = __popc(__ballot_sync(0xffffffffu, le));
+        const int64_t new_lo = lo + (int64_t)cnt * step;
+        hi = min(hi, new_lo + step);
+        lo = new_lo;
+    }
+    return lo;
+}
+
+// The rows that overlap one CTA's span of the flat storage, staged in shared memory so that the
+// per-thread row lookups never touch global memory.  R = table capacity; values that lie beyond
+// the last staged row (spans made of very many tiny or empty rows) use the global search.
+template <int R>
+struct RowTable {
+    int64_t off[R + 1];       // off[r] = first flat index of row row0 + r (INT64_MAX past the end)
+    int64_t row0;
+
+    // All threads of the CTA call this (two barriers); afterwards thread r still holds off[r] of
+    // the rows r = threadIdx.x, threadIdx.x + blockDim.x, ... it loaded.
+    __device__ __forceinline__ void load(const Rows& rows, int64_t span_beg) {
+        if (threadIdx.x < 32) {
+            const int64_t r0 = warp_row_of(rows, span_beg);
+            if (threadIdx.x == 0) row0 = r0;
+        }
+        __syncthreads();
+        const int64_t r0 = row0;
+        for (int r = threadIdx.x; r <= R; r += blockDim.x)
+            off[r] = (r0 + r <= rows.C) ? rows.begin(r0 + r) : INT64_MAX;
+        __syncthreads();
+    }
+    // Local index of the staged row containing i, or -1 when i lies beyond the staged rows.
+    __device__ __forceinline__ int find(int64_t i) const {
+        if (i >= off[R]) return -1;
+        int lo = 0, hi = R;                           // off[lo] <= i < off[hi]
+        while (hi - lo > 1) {
+            const int mid = (lo + hi) >> 1;
+            if (off[mid] <= i) lo = mid; else hi = mid;
+        }
+        return lo;
+    }
+};
 
 }  // namespace pwlq

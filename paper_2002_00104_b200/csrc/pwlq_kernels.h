@@ -19,6 +19,7 @@ struct SearchPlan {
     int64_t tiles;         // tiles per row (by the longest row)
     size_t off_m;          // workspace offset of the internally computed ranges [C] floats
     size_t off_partials;   // workspace offset of the partial sums [C * tiles * K] doubles (tiles > 1)
+    size_t off_sums;       // workspace offset of the combined sums [C * K] doubles (tiles > 1)
     size_t bytes;          // total workspace bytes
 };
 SearchPlan plan_search(int64_t C, int64_t max_n, int K);
@@ -37,5 +38,10 @@ cudaError_t launch_dequantize(const uint8_t* codes, const uint8_t* mask,
                               const int64_t* row_offsets, int64_t C, int64_t n, int64_t total,
                               int bits, const float* m, const float* p, float* y, int layout,
                               cudaStream_t stream);
+
+// 1 when a bounded wait of the kernel family expired since the library was loaded (reads a
+// device flag: synchronises with the device).
+int absmax_timeout_flag();
+int quantize_timeout_flag();
 
 }  // namespace pwlq

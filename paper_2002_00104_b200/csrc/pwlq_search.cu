@@ -618,30 +618,57 @@ search_generic_kernel(SearchArgs a) {
     finish_tile(a, row, tile, m, part, E, red_val, red_idx);
 }
 
-// Combines the tiles of long rows in ascending tile order and takes the argmin.
+// Long rows, step 1: sums the tiles' partial sums of 32 candidates of one row.  The tiles are cut
+// into eight consecutive segments, one per warp, each summed in ascending tile order; the eight
+// segment sums are then added in ascending order.  Fixed order, hence reproducible.
 __global__ void __launch_bounds__(kSThreads)
-search_combine_kernel(SearchArgs a) {
-    extern __shared__ __align__(16) unsigned char smem_raw[];
-    double* sse = reinterpret_cast<double*>(smem_raw);
+search_combine_kernel(SearchArgs a, double* __restrict__ sums) {
+    __shared__ double seg[kSWarps][32];
+    const int chunks = (a.K + 31) / 32;
+    const int64_t row = blockIdx.x / chunks;
+    const int chunk = (int)(blockIdx.x - row * chunks);
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int k = chunk * 32 + lane;
+    const int64_t n_row = a.rows.begin(row + 1) - a.rows.begin(row);
+    const float m = a.m[row];
+    const bool finite = __float_as_uint(m) < 0x7f800000u;
+    const bool degenerate = !finite || !(m > 0.0f) || n_row <= 0;
+    const int64_t nt = degenerate ? 0 : (n_row + a.cap - 1) / a.cap;
+    const int64_t t0 = nt * warp / kSWarps, t1 = nt * (warp + 1) / kSWarps;
+    double tot = 0.0;
+    if (k < a.K) {
+        const double* src = a.partials + (size_t)row * a.tiles * a.K + k;
+        for (int64_t t = t0; t < t1; ++t) tot += src[(size_t)t * a.K];
+    }
+    seg[warp][lane] = tot;
+    __syncthreads();
+    if (warp == 0 && k < a.K) {
+        double v = seg[0][lane];
+        for (int w = 1; w < kSWarps; ++w) v += seg[w][lane];
+        sums[row * a.K + k] = v;
+        if (a.sse_all) a.sse_all[row * a.K + k] = (float)v;
+    }
+}
+
+// Long rows, step 2: first minimal candidate of every row.
+__global__ void __launch_bounds__(kSThreads)
+search_argmin_kernel(SearchArgs a, const double* __restrict__ sums) {
     __shared__ double red_val[kSWarps];
     __shared__ int red_idx[kSWarps];
     const int64_t row = blockIdx.x;
     const int64_t n_row = a.rows.begin(row + 1) - a.rows.begin(row);
     const float m = a.m[row];
     const bool finite = __float_as_uint(m) < 0x7f800000u;
-    if (!finite || !(m > 0.0f) || n_row <= 0) { write_degenerate_row(a, row); return; }
-    const int64_t nt = (n_row + a.cap - 1) / a.cap;
-    const int K = a.K;
-    for (int k = threadIdx.x; k < K; k += kSThreads) {
-        const double* src = a.partials + (size_t)row * a.tiles * K + k;
-        double tot = 0.0;
-        for (int64_t t = 0; t < nt; ++t) tot += src[(size_t)t * K];
-        sse[k] = tot;
-        if (a.sse_all) a.sse_all[row * K + k] = (float)tot;
+    if (!finite || !(m > 0.0f) || n_row <= 0) {
+        if (threadIdx.x == 0) {
+            a.idx_out[row] = 0;
+            a.p_out[row] = 0.0f;
+            if (a.err_out) a.err_out[row] = 0.0f;
+        }
+        return;
     }
-    __syncthreads();
     double best; int idx;
-    block_argmin(sse, K, red_val, red_idx, best, idx);
+    block_argmin(sums + row * a.K, a.K, red_val, red_idx, best, idx);
     if (threadIdx.x == 0) write_row_result(a, row, m, best, idx);
 }
 
@@ -655,8 +682,13 @@ SearchPlan plan_search(int64_t C, int64_t max_n, int K) {
     if (p.tiles < 1) p.tiles = 1;
     p.off_m = 256;
     p.off_partials = align_up(p.off_m + sizeof(float) * (size_t)C, 256);
+    p.off_sums = p.off_partials;
     p.bytes = p.off_partials;
-    if (p.tiles > 1) p.bytes += sizeof(double) * (size_t)C * (size_t)p.tiles * (size_t)K;
+    if (p.tiles > 1) {
+        p.off_sums = align_up(p.off_partials +
+                              sizeof(double) * (size_t)C * (size_t)p.tiles * (size_t)K, 256);
+        p.bytes = p.off_sums + sizeof(double) * (size_t)C * (size_t)K;
+    }
     p.bytes = align_up(p.bytes, 256);
     return p;
 }
@@ -737,7 +769,12 @@ cudaError_t launch_search(const float* x, const int64_t* row_offsets, int64_t C,
     e = cudaGetLastError();
     if (e != cudaSuccess) return e;
     if (plan.tiles > 1) {
-        search_combine_kernel<<<(unsigned)C, kSThreads, sizeof(double) * (size_t)K, stream>>>(a);
+        double* sums = reinterpret_cast<double*>(ws + plan.off_sums);
+        const int64_t chunks = (K + 31) / 32;
+        search_combine_kernel<<<(unsigned)(C * chunks), kSThreads, 0, stream>>>(a, sums);
+        e = cudaGetLastError();
+        if (e != cudaSuccess) return e;
+        search_argmin_kernel<<<(unsigned)C, kSThreads, 0, stream>>>(a, sums);
         e = cudaGetLastError();
     }
     return e;

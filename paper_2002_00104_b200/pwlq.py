@@ -39,6 +39,7 @@ _SIGNATURES = {
                                 _INT, _P, _SZ, _P, _P]),
     "pwlq_search_noalloc": (_INT, [_P, _I64, _I64, _INT, _P, _INT, _P, _P, _P, _P, _P, _P, _P]),
     "pwlq_search_noalloc_max_bytes": (_SZ, []),
+    "pwlq_device_status": (_INT, []),
     "pwlq_status_string": (ctypes.c_char_p, [_INT]),
     "pwlq_version": (ctypes.c_char_p, []),
 }
@@ -69,6 +70,11 @@ def load_library(path: Optional[str] = None) -> ctypes.CDLL:
 
 def exported_symbols():
     return sorted(_SIGNATURES)
+
+
+def device_status() -> int:
+    """0, or 1 << ERR_TIMEOUT if a bounded device wait has expired (synchronises)."""
+    return int(load_library().pwlq_device_status())
 
 
 def status_string(status: int) -> str:

@@ -222,3 +222,8 @@ def test_argument_errors_launch_nothing(pwlq):
         pwlq.search(x, 4, dev(W.ratio_grid(pwlq.MAX_K + 1)))
     assert e.value.status == pwlq.ERR_UNSUPPORTED
     torch.cuda.synchronize()
+
+
+def test_no_bounded_wait_expired(pwlq):
+    """Runs after the parity tests of this file: none of their kernels gave up on a wait."""
+    assert pwlq.device_status() == 0
