@@ -1,0 +1,132 @@
+"""Parity at the full benchmark sizes, in the launch configuration bench.py times (ragged rows,
+ranges passed in, packed codes).  Where the oracle cannot do everything in seconds, it checks a
+stratified sample of rows (or of candidates) one by one, and properties that hold at any size
+cover the rest: exact ranges, p = m * ratio[idx], err = SSE[idx] = min SSE, and codes / region
+bits / reconstructed values of every single value against the oracle's quantizer."""
+import numpy as np
+import pytest
+import torch
+
+from gpu_util import check_search, dev
+from paper_2002_00104_b200 import workloads as W
+
+pytestmark = [pytest.mark.gpu,
+              pytest.mark.skipif(not torch.cuda.is_available(), reason="needs a CUDA device")]
+
+
+@pytest.fixture(scope="module")
+def pwlq():
+    from paper_2002_00104_b200 import pwlq as _p
+    _p.load_library()
+    return _p
+
+
+def run_path(pwlq, w, bits=None, K=None, want_sse=True):
+    bits = bits or w.bits
+    K = K or w.K
+    ratios = W.ratio_grid(K)
+    x = dev(w.x)
+    n = w.uniform_n()
+    if n is not None:
+        x, ro = x.view(w.C, n), None
+    else:
+        ro = dev(w.row_offsets)
+    max_n = int(np.diff(w.row_offsets).max())
+    m = pwlq.absmax(x, row_offsets=ro)
+    s = pwlq.search(x, bits, dev(ratios), m=m, row_offsets=ro, max_n=max_n, want_sse=want_sse)
+    codes, mask, _ = pwlq.quantize(x, bits, m, s["p"], layout=pwlq.CODES_PACKED, row_offsets=ro)
+    y = pwlq.dequantize(codes, mask, bits, m, s["p"], C=w.C, n=n, layout=pwlq.CODES_PACKED,
+                        row_offsets=ro)
+    torch.cuda.synchronize()
+    assert pwlq.search_status(s["workspace"]) == 0 and pwlq.device_status() == 0
+    out = {k: s[k].cpu().numpy() for k in ("p", "err", "idx")}
+    out["sse"] = s["sse"].cpu().numpy() if want_sse else None
+    out.update(m=m.cpu().numpy(), codes=codes.cpu().numpy(), mask=mask.cpu().numpy(),
+               y=y.cpu().numpy(), ratios=ratios, bits=bits, K=K)
+    return out
+
+
+def check_all_rows(oracle, w, g):
+    """Checks that need no per-candidate oracle work: every row, every value."""
+    m = oracle.absmax(w.x, w.row_offsets)
+    assert np.array_equal(g["m"], m)
+    want_p = (m * g["ratios"][g["idx"]]).astype(np.float32)
+    want_p[m == 0] = 0
+    assert np.array_equal(g["p"], want_p)
+    if g["sse"] is not None:
+        rows = np.arange(w.C)
+        mins = g["sse"].min(axis=1)
+        assert np.array_equal(g["sse"][rows, g["idx"]], mins)          # the minimum ...
+        assert np.array_equal(g["idx"], np.argmin(g["sse"], axis=1)) or \
+            np.all(g["sse"][rows, np.argmin(g["sse"], axis=1)] == mins)
+        assert np.allclose(g["err"], mins, rtol=2e-7, atol=0)          # ... is what err reports
+    oc, om, of = oracle.quantize(w.x, g["bits"], m, g["p"], layout=1, row_offsets=w.row_offsets)
+    assert np.array_equal(g["codes"], oc)
+    assert np.array_equal(g["mask"], om)
+    assert g["y"].tobytes() == of.tobytes()
+    return m
+
+
+def check_sampled_rows(oracle, w, g, rows, m):
+    lens = np.diff(w.row_offsets)
+    xs = np.concatenate([w.x[w.row_offsets[c]:w.row_offsets[c + 1]] for c in rows])
+    ro = np.concatenate([[0], np.cumsum(lens[rows])]).astype(np.int64)
+    ora = oracle.search(xs, g["bits"], g["ratios"], m=m[rows], row_offsets=ro)
+    sub = {k: g[k][rows] for k in ("p", "err", "idx", "sse")}
+    return check_search(sub, ora, g["ratios"], m[rows], lens[rows])
+
+
+def stratified_rows(w, per_length, every):
+    """Every `every`-th row plus the first `per_length` rows of each distinct length."""
+    lens = np.diff(w.row_offsets)
+    rows = set(range(0, w.C, every))
+    for n in np.unique(lens):
+        rows.update(np.nonzero(lens == n)[0][:per_length].tolist())
+    return np.array(sorted(rows))
+
+
+def test_single_conv_full(pwlq, oracle):
+    w = W.single_conv()
+    g = run_path(pwlq, w)
+    m = check_all_rows(oracle, w, g)
+    assert check_sampled_rows(oracle, w, g, np.array([0]), m) == 0
+
+
+def test_resnet50_full(pwlq, oracle):
+    w = W.resnet50()
+    g = run_path(pwlq, w)
+    m = check_all_rows(oracle, w, g)
+    differ = check_sampled_rows(oracle, w, g, stratified_rows(w, 3, 60), m)
+    assert differ <= 2          # near-ties only (check_search has already vetted each of them)
+
+
+def test_mobilenetv2_full(pwlq, oracle):
+    w = W.mobilenetv2()
+    g = run_path(pwlq, w)
+    m = check_all_rows(oracle, w, g)
+    check_sampled_rows(oracle, w, g, stratified_rows(w, 4, 25), m)
+
+
+def test_relu_activation_full(pwlq, oracle):
+    w = W.relu_activation()
+    g = run_path(pwlq, w)
+    m = check_all_rows(oracle, w, g)
+    idx = int(g["idx"][0])
+    ks = sorted({0, 1, 7, 100, 511, 1023, max(idx - 1, 0), idx, min(idx + 1, w.K - 1)})
+    ora = oracle.search(w.x, w.bits, g["ratios"][ks], m=m)
+    sse_o = ora["sse64"][0]
+    got = g["sse"][0, ks].astype(np.float64)
+    tol = 1e-5 * sse_o + w.total * (2.0 ** -23 * m[0]) ** 2 + 2.0 ** -23 * sse_o
+    assert np.all(np.abs(got - sse_o) <= tol), (got, sse_o)
+    # the chosen candidate beats its neighbours in the oracle's own sums (up to a near-tie)
+    best = sse_o[ks.index(idx)]
+    assert np.all(sse_o >= best * (1 - 1e-5))
+
+
+@pytest.mark.parametrize("bits", [3, 4, 6, 8])
+@pytest.mark.parametrize("K", [64, 256, 1024])
+def test_laplace_matrix_sweep(pwlq, oracle, bits, K):
+    w = W.laplace_matrix()
+    g = run_path(pwlq, w, bits=bits, K=K)
+    m = check_all_rows(oracle, w, g)
+    check_sampled_rows(oracle, w, g, np.arange(5, w.C, 512), m)
