@@ -307,6 +307,12 @@ def run_ours(args, rank, world, local_rank):
     else:
         stage_tot = stage_ms.sum(axis=0).tolist()
 
+    # kernels of this library per step: abs-max, one search launch per row-length class present
+    # (plus the two combine launches when a row exceeds one tile), quantize, dequantize
+    lens = np.diff(w.row_offsets)
+    classes = sum(bool(np.any((lens >= lo) & (lens <= hi)))
+                  for lo, hi in ((0, 256), (257, 1152), (1153, 1 << 62))) if w.K <= 1024 else 1
+    per_step = 1 + classes + (2 if max_n > 8192 else 0) + 2
     if rank == 0:
         peaks, peak_kind = measured_peaks()
         ec = w.elem_cand
@@ -345,7 +351,8 @@ def run_ours(args, rank, world, local_rank):
             "e2e": {"value": world * ec * e2e_steps / (e2e_ms * 1e-3) / 1e9, "unit": UNIT,
                     "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                     "ms_per_step": e2e_ms / e2e_steps, "matches_resident_path": same},
-            "gpu_launches": 4 * args.steps + 4 * (e2e_steps + 2) + 4 * max(3, args.warmup),
+            "gpu_launches": per_step * (args.steps + e2e_steps + 2 + max(3, args.warmup)),
+            "kernels_per_step": per_step,
             "clocks": clocks, "device_status": status,
         }
         for k in ("absmax", "quantize", "dequantize"):
@@ -367,7 +374,7 @@ def run_ours(args, rank, world, local_rank):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--steps", type=int, default=30)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="resnet50", choices=sorted(WORKLOADS))

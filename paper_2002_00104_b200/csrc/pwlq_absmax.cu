@@ -3,11 +3,11 @@
 // HBM-bound streaming reduction, 4 bytes read per value.  The flat storage is cut into spans of
 // kAbsSpan values that persistent CTAs walk; the spans arrive in a ring of shared-memory slots
 // filled by bulk asynchronous copies, three spans ahead.
-// A thread folds the magnitude bit patterns with an integer maximum (exact and order-free).  The
-// rows that overlap the span are staged in shared memory together with one maximum per row;
-// threads merge into those with shared-memory atomics (once per row they touch, after a warp
-// shuffle when the whole warp sits in one row), and the CTA issues one global atomicMax per row
-// of its span.
+// Magnitude bit patterns are folded with an integer maximum (exact and order-free).  A span that
+// lies inside one row is folded into per-thread registers that live on from span to span (one
+// atomic per warp when the row ends); a span that holds several rows is cut into one slice per
+// warp, and the warp walks the rows overlapping its slice (offsets staged in shared memory) with
+// a strided read, a shuffle reduction and one atomicMax per piece.
 #include "pwlq_common.cuh"
 #include "pwlq_kernels.h"
 #include "pwlq_pipeline.cuh"
@@ -17,15 +17,13 @@ namespace pwlq {
 constexpr int kAbsThreads = 256;
 constexpr int kAbsUnroll = 4;
 constexpr int kAbsSpan = kAbsThreads * 4 * kAbsUnroll;  // values per span
-constexpr int kAbsRows = 1024;                           // staged rows per span
 constexpr int kAbsStages = 3;                            // spans in flight per CTA
 
 static __device__ int g_absmax_timeout;                  // set when a bounded wait expired
 
 struct AbsSmem {
     BulkRing<kAbsStages, kAbsSpan * 4> ring;
-    RowTable<kAbsRows> T;
-    uint32_t s_max[kAbsRows];
+    SpanTable<false> T;
 };
 
 // Bytes of span `span` if it can be fetched by a bulk copy (aligned base, whole 16-byte units).
@@ -42,80 +40,65 @@ absmax_kernel(const float* __restrict__ x, Rows rows, int64_t total, uint32_t* _
     AbsSmem& S = *reinterpret_cast<AbsSmem*>(smem_raw);
     __shared__ int s_abort;
     const int64_t nspans = (total + kAbsSpan - 1) / kAbsSpan;
-    const bool ragged = rows.offsets != nullptr;
+    // this CTA's consecutive spans
+    const int64_t s0 = nspans * blockIdx.x / gridDim.x, s1 = nspans * (blockIdx.x + 1) / gridDim.x;
+    const bool use_table = rows.offsets != nullptr || rows.n < kAbsSpan;   // several rows per span
     if (threadIdx.x == 0) s_abort = 0;
     S.ring.init();
-    for (int it = 0; it < kAbsStages; ++it) {
-        const int64_t span = blockIdx.x + (int64_t)it * gridDim.x;
-        if (span < nspans)
-            S.ring.issue(it, x + span * kAbsSpan, abs_bulk_bytes(span, total, vec_ok));
+    for (int it = 0; it < kAbsStages; ++it)
+        if (s0 + it < s1)
+            S.ring.issue(it, x + (s0 + it) * kAbsSpan, abs_bulk_bytes(s0 + it, total, vec_ok));
+
+    int64_t row0 = 0;                                  // first staged row of the current span
+    RowFetch nf;
+    if (use_table && s0 < s1) {
+        row0 = warp_row_of(rows, s0 * kAbsSpan);       // every warp finds the same row
+        S.T.fetch(rows, nullptr, nullptr, row0, nf);
+        S.T.commit(nf, 0, 0.0f);
+        __syncthreads();
     }
 
-    // The row a thread is accumulating; it survives from span to span, so a long row costs one
-    // atomic per warp for the whole kernel.  loc >= 0: the row has a slot in S.s_max.
-    int loc = -1;
-    int64_t grow = -1, row_beg = 0, row_end = 0;
+    // The long row the CTA is inside of (the same for all of its threads) and this thread's
+    // maximum over it; both survive from span to span, so a long row costs one atomic per warp
+    // for the whole kernel.
+    int64_t grow = -1;
     uint32_t mx = 0;
-    auto flush = [&]() {
-        if (mx == 0) return;
-        if (loc >= 0) atomicMax(&S.s_max[loc], mx);
-        else if (grow >= 0) atomicMax(m_bits + grow, mx);
+    auto flush_merged = [&]() {                        // every lane of the warp calls this
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) mx = max(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+        if ((threadIdx.x & 31) == 0 && mx != 0 && grow >= 0) atomicMax(m_bits + grow, mx);
         mx = 0;
     };
 
-    // Same, after merging inside the warp when all of its lanes carry the same long row (every
-    // lane of the warp must call this).
-    auto flush_merged = [&]() {
-        const unsigned full = 0xffffffffu;
-        const int64_t g0 = __shfl_sync(full, grow, 0);
-        if (__all_sync(full, grow == g0 && loc < 0)) {
-#pragma unroll
-            for (int o = 16; o > 0; o >>= 1) mx = max(mx, __shfl_xor_sync(full, mx, o));
-            if ((threadIdx.x & 31) != 0) mx = 0;
-        }
-        flush();
-    };
-
-    int64_t it = 0;
-    for (int64_t span = blockIdx.x; span < nspans; span += gridDim.x, ++it) {
+    for (int64_t span = s0; span < s1; ++span) {
+        const int64_t it = span - s0;
         const int64_t span_beg = span * kAbsSpan;
         const int64_t span_end = min(span_beg + kAbsSpan, total);
-        // Does the span lie inside one row?  Dense: arithmetic.  Ragged: after staging the rows.
+        // Does the span lie inside one row?
         bool single;
-        int64_t first_row = 0;
-        if (ragged) {
-            S.T.load(rows, span_beg);                 // two barriers
-            first_row = S.T.row0;
+        int64_t first_row;
+        if (use_table) {
+            first_row = row0;
             single = S.T.off[1] >= span_end;
         } else {
             first_row = span_beg / rows.n;
             single = (first_row + 1) * rows.n >= span_end;
         }
-        if (!single) {                                 // several rows: merge through shared memory
+        // the next span starts in the row in which this one ends: request its table now
+        int64_t next_row0 = 0;
+        const bool has_next = use_table && span + 1 < s1;
+        if (has_next) {
+            const int l = S.T.find(span_end);
+            next_row0 = (l >= 0) ? row0 + l : rows.row_of(span_end);
+            S.T.fetch(rows, nullptr, nullptr, next_row0, nf);
+        }
+        if (!single) {                                 // several rows: nothing is carried across
             flush_merged();
-            loc = -1; grow = -1; row_beg = row_end = 0;
-            for (int r = threadIdx.x; r < kAbsRows; r += kAbsThreads) S.s_max[r] = 0;
-            __syncthreads();
+            grow = -1;
         } else if (grow != first_row) {                // a new long row begins
             flush_merged();
-            loc = -1;
             grow = first_row;
-            row_beg = rows.begin(grow);
-            row_end = rows.begin(grow + 1);
         }
-        auto enter = [&](int64_t i) {                  // only reached when the span has several rows
-            flush();
-            if (ragged) {
-                const int l = S.T.find(i);
-                if (l >= 0) { loc = l; grow = S.T.row0 + l; row_beg = S.T.off[l]; row_end = S.T.off[l + 1]; }
-                else { loc = -1; grow = rows.row_of(i); row_beg = rows.begin(grow); row_end = rows.begin(grow + 1); }
-            } else {
-                grow = i / rows.n;
-                row_beg = grow * rows.n;
-                row_end = row_beg + rows.n;
-                loc = (grow - first_row < kAbsRows) ? (int)(grow - first_row) : -1;
-            }
-        };
 
         float* xs = reinterpret_cast<float*>(S.ring.slot(it));
         if (abs_bulk_bytes(span, total, vec_ok) != 0) {
@@ -125,42 +108,59 @@ absmax_kernel(const float* __restrict__ x, Rows rows, int64_t total, uint32_t* _
                 xs[i] = x[span_beg + i];
             __syncthreads();
         }
+        if (single) {
+            // the whole span belongs to the carried row: registers only
 #pragma unroll
-        for (int j = 0; j < kAbsUnroll; ++j) {
-            const int li = (j * kAbsThreads + threadIdx.x) * 4;
-            const int64_t i = span_beg + li;
-            if (i < total) {
-                const float4 v = *reinterpret_cast<const float4*>(xs + li);
-                const float e[4] = {v.x, v.y, v.z, v.w};
-                if (i >= row_beg && i + 4 <= row_end) {    // still inside the current row
-                    mx = max(max(mx, abs_bits(e[0])),
-                             max(abs_bits(e[1]), max(abs_bits(e[2]), abs_bits(e[3]))));
+            for (int j = 0; j < kAbsUnroll; ++j) {
+                const int li = (j * kAbsThreads + threadIdx.x) * 4;
+                if (span_beg + li + 4 <= span_end) {
+                    const float4 v = *reinterpret_cast<const float4*>(xs + li);
+                    mx = max(max(mx, abs_bits(v.x)),
+                             max(abs_bits(v.y), max(abs_bits(v.z), abs_bits(v.w))));
                 } else {
-#pragma unroll
-                    for (int t = 0; t < 4; ++t) {
-                        if (i + t < total) {
-                            if (!(i + t >= row_beg && i + t < row_end)) enter(i + t);
-                            mx = max(mx, abs_bits(e[t]));
-                        }
-                    }
+                    for (int t = 0; t < 4; ++t)
+                        if (span_beg + li + t < span_end) mx = max(mx, abs_bits(xs[li + t]));
                 }
             }
+        } else {
+            // several rows: every warp takes a contiguous slice of the span and walks the rows
+            // that overlap it; per (slice, row) piece a strided read, a shuffle reduction and one
+            // atomic.  No per-value row lookup, no divergence.
+            const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+            constexpr int kSlice = kAbsSpan / (kAbsThreads / 32);
+            const int64_t sl_beg = span_beg + (int64_t)warp * kSlice;
+            const int64_t sl_end = min(sl_beg + kSlice, span_end);
+            int64_t pos = sl_beg;
+            int l = (pos < sl_end && use_table) ? S.T.find(pos) : -1;
+            while (pos < sl_end) {
+                int64_t r_glob, r_end;
+                if (l >= 0 && l < kTableRows) {            // staged row
+                    r_glob = row0 + l;
+                    r_end = S.T.off[l + 1];
+                    ++l;
+                } else {                                   // long dense rows, or beyond the staged rows
+                    r_glob = rows.row_of(pos);
+                    r_end = rows.begin(r_glob + 1);
+                }
+                const int64_t e = min(r_end, sl_end);
+                uint32_t v = 0;
+                for (int64_t i = pos + lane; i < e; i += 32) v = max(v, abs_bits(xs[i - span_beg]));
+#pragma unroll
+                for (int o = 16; o > 0; o >>= 1) v = max(v, __shfl_xor_sync(0xffffffffu, v, o));
+                if (lane == 0 && v != 0) atomicMax(m_bits + r_glob, v);
+                pos = e;
+            }
         }
-        if (!single) {
-            flush();
-            loc = -1; grow = -1; row_beg = row_end = 0;
-            __syncthreads();
-            for (int r = threadIdx.x; r < kAbsRows; r += kAbsThreads)
-                if (S.s_max[r] != 0) atomicMax(m_bits + first_row + r, S.s_max[r]);
-        }
-        __syncthreads();                              // slot, table and maxima are free again
+        __syncthreads();                              // slot and table are no longer read
         if (s_abort) {                                 // a wait ran out: report and leave
             if (threadIdx.x == 0) atomicExch(&g_absmax_timeout, 1);
             return;
         }
-        const int64_t ahead = span + (int64_t)kAbsStages * gridDim.x;
-        if (ahead < nspans)
-            S.ring.issue(it + kAbsStages, x + ahead * kAbsSpan, abs_bulk_bytes(ahead, total, vec_ok));
+        if (has_next) { S.T.commit(nf, 0, 0.0f); row0 = next_row0; }
+        if (span + kAbsStages < s1)
+            S.ring.issue(it + kAbsStages, x + (span + kAbsStages) * kAbsSpan,
+                         abs_bulk_bytes(span + kAbsStages, total, vec_ok));
+        if (use_table) __syncthreads();               // the next table is published
     }
     flush_merged();                                   // what is still carried at the end
 }

@@ -95,7 +95,83 @@ __device__ __forceinline__ int64_t warp_row_of(const Rows& rows, int64_t i) {
 }
 
 // The rows that overlap one CTA's span of the flat storage, staged in shared memory so that the
-// per-thread row lookups never touch global memory.  R = table capacity; values that lie beyond
+// per-thread row lookups never touch global memory.  A persistent CTA walks consecutive spans, so
+// the first row of the next span is the row in which the current span ends: the next table's
+// offsets (and ranges / breakpoints) are requested into registers before the current span is
+// processed and written to shared memory after it, which keeps every global round trip off the
+// critical path.  Values that lie beyond the last staged row (spans made of very many tiny or
+// empty rows) use the global search.
+constexpr int kTableRows = 512;
+constexpr int kTableThreads = 256;        // CTA size the fetch / commit pattern is written for
+
+struct RowFetch {                          // what one thread holds of the next table
+    int64_t off[3];                        // rows tid, tid + 256, and (thread 0) the end entry
+    float m[2], p[2];
+};
+
+template <bool PARAMS>
+struct SpanTable {
+    int64_t off[kTableRows + 1];  // off[r] = first flat index of row row0 + r (INT64_MAX past the end)
+    float m[PARAMS ? kTableRows : 1];
+    PieceParams P[PARAMS ? kTableRows : 1];
+
+    // Local index of the staged row containing i, or -1 when i lies beyond the staged rows.
+    // Rows inside one span are mostly equally long (one layer), so a proportional guess is tried
+    // first and corrected by a few neighbour steps; irregular tables fall back to bisection.
+    __device__ __forceinline__ int find(int64_t i) const {
+        const int64_t last = off[kTableRows];
+        if (i >= last) return -1;
+        int lo = 0, hi = kTableRows;                  // off[lo] <= i < off[hi]
+        if (last != INT64_MAX) {
+            const float scale = (float)kTableRows / (float)(last - off[0]);
+            int g = min(max((int)((float)(i - off[0]) * scale), 0), kTableRows - 1);
+#pragma unroll
+            for (int t = 0; t < 4; ++t) {
+                if (off[g] > i) { hi = g; g = max(g - 1, 0); }
+                else if (off[g + 1] <= i) { lo = g + 1; g = min(g + 1, kTableRows - 1); }
+                else return g;
+            }
+        }
+        while (hi - lo > 1) {
+            const int mid = (lo + hi) >> 1;
+            if (off[mid] <= i) lo = mid; else hi = mid;
+        }
+        return lo;
+    }
+    // Requests the table that starts at row r0 (no barrier; the values stay in registers).
+    __device__ __forceinline__ void fetch(const Rows& rows, const float* __restrict__ m_arr,
+                                          const float* __restrict__ p_arr, int64_t r0,
+                                          RowFetch& f) const {
+#pragma unroll
+        for (int u = 0; u < 2; ++u) {
+            const int64_t row = r0 + threadIdx.x + u * kTableThreads;
+            f.off[u] = (row <= rows.C) ? rows.begin(row) : INT64_MAX;
+            f.m[u] = f.p[u] = 0.0f;
+            if (PARAMS && row < rows.C) { f.m[u] = __ldg(m_arr + row); f.p[u] = __ldg(p_arr + row); }
+        }
+        f.off[2] = (threadIdx.x == 0 && r0 + kTableRows <= rows.C) ? rows.begin(r0 + kTableRows)
+                                                                   : INT64_MAX;
+    }
+    // Writes what fetch() requested; call between the barrier that retires the previous table and
+    // the barrier that publishes this one.  Constants are computed for rows that start before
+    // span_end only.
+    __device__ __forceinline__ void commit(const RowFetch& f, int64_t span_end, float Lf) {
+#pragma unroll
+        for (int u = 0; u < 2; ++u) {
+            const int r = threadIdx.x + u * kTableThreads;
+            off[r] = f.off[u];
+            if (PARAMS && f.off[u] < span_end) {
+                m[r] = f.m[u];
+                P[r] = make_params(f.m[u], f.p[u], Lf);
+            }
+        }
+        if (threadIdx.x == 0) off[kTableRows] = f.off[2];
+    }
+};
+
+// Stand-alone variant used by the quantize / dequantize kernels (their spans are not consecutive):
+// the rows that overlap one CTA's span, staged in shared memory so that the per-thread row lookups
+// never touch global memory.  R = table capacity; values that lie beyond
 // the last staged row (spans made of very many tiny or empty rows) use the global search.
 template <int R>
 struct RowTable {
