@@ -81,7 +81,7 @@ absmax_kernel(const float* __restrict__ x, Rows rows, int64_t total, uint32_t* _
             first_row = row0;
             single = S.T.off[1] >= span_end;
         } else {
-            first_row = span_beg / rows.n;
+            first_row = rows.dense_row(span_beg);
             single = (first_row + 1) * rows.n >= span_end;
         }
         // the next span starts in the row in which this one ends: request its table now
@@ -176,7 +176,7 @@ cudaError_t launch_absmax(const float* x, const int64_t* row_offsets, int64_t C,
     cudaError_t e = cudaMemsetAsync(m_out, 0, sizeof(float) * (size_t)C, stream);
     if (e != cudaSuccess) return e;
     if (total == 0) return cudaSuccess;
-    Rows rows{row_offsets, C, n};
+    Rows rows{row_offsets, C, n, n > 0 ? 1.0 / (double)n : 0.0};
     const int64_t nspans = (total + kAbsSpan - 1) / kAbsSpan;
     static int cached[64] = {0};                       // CTAs that fit the device at once
     int dev = 0;

@@ -57,13 +57,22 @@ struct Rows {
     const int64_t* offsets;  // [C + 1] or nullptr (dense)
     int64_t C;
     int64_t n;               // dense row length (unused when ragged)
+    double inv_n;            // 1 / n (dense), so that i / n costs a multiply and a correction
+
+    // i / n for dense rows without a 64-bit integer division (exact for i < 2^52).
+    __device__ __forceinline__ int64_t dense_row(int64_t i) const {
+        int64_t r = (int64_t)((double)i * inv_n);
+        if (r * n > i) --r;
+        else if ((r + 1) * n <= i) ++r;
+        return r;
+    }
 
     __device__ __forceinline__ int64_t begin(int64_t c) const {
         return offsets ? offsets[c] : c * n;
     }
     // Row that contains flat index i (0 <= i < total); empty rows are skipped.
     __device__ __forceinline__ int64_t row_of(int64_t i) const {
-        if (!offsets) return i / n;
+        if (!offsets) return dense_row(i);
         int64_t lo = 0, hi = C;                      // offsets[lo] <= i < offsets[hi]
         while (hi - lo > 1) {
             const int64_t mid = (lo + hi) >> 1;
@@ -79,7 +88,7 @@ __device__ __forceinline__ uint32_t abs_bits(float x) { return __float_as_uint(x
 // gets the same answer): a 32-ary search, three dependent rounds of loads for up to 32768 rows
 // instead of fifteen.
 __device__ __forceinline__ int64_t warp_row_of(const Rows& rows, int64_t i) {
-    if (!rows.offsets) return i / rows.n;
+    if (!rows.offsets) return rows.dense_row(i);
     const int lane = threadIdx.x & 31;
     int64_t lo = 0, hi = rows.C;                     // offsets[lo] <= i < offsets[hi]
     while (hi - lo > 1) {

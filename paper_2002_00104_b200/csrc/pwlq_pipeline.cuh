@@ -23,18 +23,21 @@ __device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, unsigned bytes) {
     asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;"
                  ::"r"(smem_addr(bar)), "r"(bytes) : "memory");
 }
+// One poll may park the thread for up to kSuspendNs (a hint to the hardware), so that waiting
+// threads do not compete for issue slots with the warps that already have their data.
+constexpr unsigned kSuspendNs = 2000;
 __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, unsigned parity) {
     unsigned ok;
     asm volatile(
         "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
         "selp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(ok) : "r"(smem_addr(bar)), "r"(parity) : "memory");
+        : "=r"(ok) : "r"(smem_addr(bar)), "r"(parity), "r"(kSuspendNs) : "memory");
     return ok != 0;
 }
-// Bounded wait: false after kMaxSpins unsuccessful polls (each poll already blocks for a
-// hardware-defined time slice), i.e. after far longer than any copy can take.
-constexpr int kMaxSpins = 1 << 20;
+// Bounded wait: false after kMaxSpins unsuccessful polls, i.e. after about half a second, far
+// longer than any copy can take.
+constexpr int kMaxSpins = 1 << 18;
 __device__ __forceinline__ bool mbar_wait(uint64_t* bar, unsigned parity) {
     for (int i = 0; i < kMaxSpins; ++i)
         if (mbar_try_wait(bar, parity)) return true;

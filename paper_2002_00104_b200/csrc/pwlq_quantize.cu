@@ -59,7 +59,7 @@ struct RowState {
                                          const float* __restrict__ p_arr, float Lf, int64_t i) {
         if (i >= beg && i < end) return;
         if (!rows.offsets) {                       // dense: arithmetic, constants from L1 / L2
-            const int64_t row = i / rows.n;
+            const int64_t row = rows.dense_row(i);
             beg = row * rows.n;
             end = beg + rows.n;
             m = __ldg(m_arr + row);
@@ -108,6 +108,9 @@ quantize_kernel(const float* __restrict__ x, Rows rows, int64_t total, int bits,
     QuantSmem& S = Q.rows;
     __shared__ int s_abort;
     const float Lf = (float)((1 << (bits - 1)) - 1);
+    const int Li = (1 << (bits - 1)) - 1;
+    const uint32_t sign_unit = 1u << (bits - 1);      // value of the sign bit inside a code
+    const int sign_shift = 32 - bits;                 // moves bit 31 onto the code's sign bit
     const int64_t nspans = (total + kQSpan - 1) / kQSpan;
     if (threadIdx.x == 0) s_abort = 0;
     Q.ring.init();
@@ -149,29 +152,56 @@ quantize_kernel(const float* __restrict__ x, Rows rows, int64_t total, int bits,
                 // all eight values in one row: the sequence of quantize_mag with the per-row
                 // tests hoisted, the level taken from the mantissa of t + 1.5 * 2^23, and the sign
                 // flag (x < 0, false for -0.0) read off the sign bit of x + 0.0
+                // Codes are packed and region bits gathered on the fly (no per-value branch).
                 const float m = rs.m;
                 const PieceParams P = rs.P;
-                const bool live = m > 0.0f;
-                const int Li = (1 << (bits - 1)) - 1;
+                uint32_t w0 = 0, w1 = 0, mb = 0;       // packed codes (w1: upper four, byte layout)
+                if (m > 0.0f) {
 #pragma unroll
-                for (int t = 0; t < 8; ++t) {
-                    const float xi = xv[t];
-                    const float a = fminf(fabsf(xi), m);
-                    const bool tail = a > P.p;
-                    const float z = tail ? P.p : 0.0f;
-                    const float inv = tail ? P.inv2 : P.inv1;
-                    const float r = __fadd_rn(__fmul_rn(__fsub_rn(a, z), inv), 12582912.0f);
-                    const uint32_t q = (uint32_t)min(__float_as_int(r) - 0x4B400000, Li);
-                    const uint32_t sb = __float_as_uint(__fadd_rn(xi, 0.0f)) >> 31;
-                    code[t] = live ? (q | (sb << (bits - 1))) : 0u;
-                    if (tail && live) mbyte |= 1u << t;
-                    if (WANT_FAKE) {
-                        const float s = tail ? P.s2 : P.s1;
-                        const float qf = fminf(__fsub_rn(r, 12582912.0f), Lf);
-                        const float v = __fadd_rn(__fmul_rn(qf, s), z);
-                        yv[t] = live ? __uint_as_float(__float_as_uint(v) | (sb << 31)) : 0.0f;
+                    for (int t = 0; t < 8; ++t) {
+                        const float xi = xv[t];
+                        const float a = fminf(fabsf(xi), m);
+                        const bool tail = a > P.p;
+                        const float z = tail ? P.p : 0.0f;
+                        const float inv = tail ? P.inv2 : P.inv1;
+                        const float r = __fadd_rn(__fmul_rn(__fsub_rn(a, z), inv), 12582912.0f);
+                        const uint32_t q = (uint32_t)min(__float_as_int(r) - 0x4B400000, Li);
+                        const uint32_t xs0 = __float_as_uint(__fadd_rn(xi, 0.0f));   // sign bit = (x < 0)
+                        const uint32_t code = ((xs0 >> sign_shift) & sign_unit) | q;
+                        if (PACKED) w0 += code << (4 * t);
+                        else if (t < 4) w0 += code << (8 * t);
+                        else w1 += code << (8 * (t - 4));
+                        mb += tail ? (1u << t) : 0u;
+                        if (WANT_FAKE) {
+                            const float s = tail ? P.s2 : P.s1;
+                            const float qf = fminf(__fsub_rn(r, 12582912.0f), Lf);
+                            const float v = __fadd_rn(__fmul_rn(qf, s), z);
+                            yv[t] = __uint_as_float(__float_as_uint(v) | (xs0 & 0x80000000u));
+                        }
+                    }
+                } else if (WANT_FAKE) {
+#pragma unroll
+                    for (int t = 0; t < 8; ++t) yv[t] = 0.0f;
+                }
+                mask[i0 >> 3] = (uint8_t)mb;
+                if (PACKED) {
+                    uint8_t* dst = codes + (i0 >> 1);
+                    if (vec_codes) *reinterpret_cast<uint32_t*>(dst) = w0;
+                    else for (int b = 0; b < 4; ++b) dst[b] = (uint8_t)(w0 >> (8 * b));
+                } else {
+                    uint8_t* dst = codes + i0;
+                    if (vec_codes) *reinterpret_cast<uint2*>(dst) = make_uint2(w0, w1);
+                    else for (int b = 0; b < 8; ++b) dst[b] = (uint8_t)((b < 4 ? w0 : w1) >> (8 * (b & 3)));
+                }
+                if (WANT_FAKE) {
+                    if (vec_fake) {
+                        __stcs(reinterpret_cast<float4*>(fake + i0), make_float4(yv[0], yv[1], yv[2], yv[3]));
+                        __stcs(reinterpret_cast<float4*>(fake + i0 + 4), make_float4(yv[4], yv[5], yv[6], yv[7]));
+                    } else {
+                        for (int t = 0; t < 8; ++t) fake[i0 + t] = yv[t];
                     }
                 }
+                continue;
             } else {
 #pragma unroll
                 for (int t = 0; t < 8; ++t) {
@@ -286,6 +316,7 @@ dequantize_kernel(const uint8_t* __restrict__ codes, const uint8_t* __restrict__
     __shared__ QuantSmem S;
     const float Lf = (float)((1 << (bits - 1)) - 1);
     const int qmask = (1 << (bits - 1)) - 1;
+    const int sign_shift = 32 - bits;                 // moves a code's sign bit to bit 31
     const int64_t nspans = (total + kQSpan - 1) / kQSpan;
     CodeRegs<PACKED> cur, nxt;
     RowState rs;                                    // survives from span to span
@@ -309,16 +340,20 @@ dequantize_kernel(const uint8_t* __restrict__ codes, const uint8_t* __restrict__
                 // all eight values in one row; the level becomes a float through the mantissa of
                 // 1.5 * 2^23 (exact for q < 2^22) instead of an integer conversion
                 const PieceParams P = rs.P;
-                const bool live = rs.m > 0.0f;
 #pragma unroll
-                for (int t = 0; t < 8; ++t) {
-                    const uint32_t code = cur.code(c, t);
-                    const bool tail = (cur.mb[c] >> t) & 1u;
-                    const float q = __fsub_rn(__uint_as_float(0x4B400000u | (code & (uint32_t)qmask)),
-                                              12582912.0f);
-                    const float v = __fadd_rn(__fmul_rn(q, tail ? P.s2 : P.s1), tail ? P.p : 0.0f);
-                    const uint32_t sb = (code >> (bits - 1)) & 1u;
-                    yv[t] = live ? __uint_as_float(__float_as_uint(v) | (sb << 31)) : 0.0f;
+                for (int t = 0; t < 8; ++t) yv[t] = 0.0f;
+                if (rs.m > 0.0f) {                     // one test per chunk; no branch per value
+                    const uint32_t mb = cur.mb[c];
+#pragma unroll
+                    for (int t = 0; t < 8; ++t) {
+                        const uint32_t code = cur.code(c, t);
+                        const bool tail = (mb & (1u << t)) != 0;
+                        const float q = __fsub_rn(__uint_as_float(0x4B400000u | (code & (uint32_t)qmask)),
+                                                  12582912.0f);
+                        const float v = __fadd_rn(__fmul_rn(q, tail ? P.s2 : P.s1), tail ? P.p : 0.0f);
+                        // the code's sign bit moved to bit 31
+                        yv[t] = __uint_as_float(__float_as_uint(v) | ((code << sign_shift) & 0x80000000u));
+                    }
                 }
             } else {
 #pragma unroll
@@ -394,7 +429,7 @@ cudaError_t launch_quantize(const float* x, const int64_t* row_offsets, int64_t 
                             uint8_t* codes, uint8_t* mask, float* fake, int layout,
                             cudaStream_t stream) {
     if (total == 0) return cudaSuccess;
-    Rows rows{row_offsets, C, n};
+    Rows rows{row_offsets, C, n, n > 0 ? 1.0 / (double)n : 0.0};
     const bool packed = (layout == 1 && bits <= 4);
     const int64_t nspans = (total + kQSpan - 1) / kQSpan;
     const int vec_in = aligned(x, 16), vec_fake = fake ? aligned(fake, 16) : 0;
@@ -416,7 +451,7 @@ cudaError_t launch_dequantize(const uint8_t* codes, const uint8_t* mask,
                               int bits, const float* m, const float* p, float* y, int layout,
                               cudaStream_t stream) {
     if (total == 0) return cudaSuccess;
-    Rows rows{row_offsets, C, n};
+    Rows rows{row_offsets, C, n, n > 0 ? 1.0 / (double)n : 0.0};
     const bool packed = (layout == 1 && bits <= 4);
     const int64_t nspans = (total + kQSpan - 1) / kQSpan;
     if (packed)

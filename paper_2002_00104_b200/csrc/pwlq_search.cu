@@ -708,7 +708,7 @@ cudaError_t launch_search(const float* x, const int64_t* row_offsets, int64_t C,
     }
     SearchArgs a;
     a.x = x;
-    a.rows = Rows{row_offsets, C, n};
+    a.rows = Rows{row_offsets, C, n, n > 0 ? 1.0 / (double)n : 0.0};
     a.m = m;
     a.ratios = ratios;
     a.K = K;
