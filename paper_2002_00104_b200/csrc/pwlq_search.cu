@@ -340,8 +340,8 @@ __host__ __device__ inline int slices_sorted(int K, int cw, int warps) {
     const int E = (4 * warps + G - 1) / G;
     return E < 1 ? 1 : (E > 8 ? 8 : E);
 }
-__host__ __device__ inline int max_slices_sorted(int K) {
-    return slices_sorted(K, kCwShortTile, kSWarps);    // fewest groups, most warps: most slices
+__host__ __device__ inline int max_slices_sorted(int K, int warps) {
+    return slices_sorted(K, kCwShortTile, warps);      // fewest groups: most slices
 }
 
 // Shared memory: sorted tile | bucket ids | candidate breakpoints | candidate constants | bucket
@@ -355,7 +355,8 @@ struct SortedSmem {
     uint16_t* hist;     // [kSWarps][K + 2]
     double* part;       // [E][K]
 };
-__host__ __device__ inline size_t sorted_smem_layout(int cap, int K, int E, size_t off[7]) {
+__host__ __device__ inline size_t sorted_smem_layout(int cap, int K, int warps, size_t off[7]) {
+    const int E = max_slices_sorted(K, warps);
     size_t o = 0;
     auto take = [&](size_t bytes) { size_t r = o; o = (o + bytes + 15) & ~(size_t)15; return r; };
     off[0] = take(sizeof(float) * (size_t)(cap + 4));
@@ -363,7 +364,7 @@ __host__ __device__ inline size_t sorted_smem_layout(int cap, int K, int E, size
     off[2] = take(sizeof(float) * (size_t)K);
     off[3] = take(sizeof(float4) * (size_t)K);
     off[4] = take(sizeof(int) * (size_t)(K + 2));
-    off[5] = take(sizeof(uint16_t) * (size_t)kSWarps * (size_t)(K + 2));
+    off[5] = take(sizeof(uint16_t) * (size_t)warps * (size_t)(K + 2));
     off[6] = take(sizeof(double) * (size_t)E * (size_t)K);
     return o;
 }
@@ -440,6 +441,9 @@ search_sorted_kernel(SearchArgs a) {
     __shared__ int red_idx[kSWarps];
     __shared__ int warp_sums[kSWarps];
     __shared__ int next_item;
+    // The launches of the other row-length classes touch other rows only: let the next one start
+    // filling the SMs as soon as every CTA of this grid is resident or done.
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     int64_t row, tile, t_beg;
     int cnt;
     float m;
@@ -450,7 +454,7 @@ search_sorted_kernel(SearchArgs a) {
     const int cw = group_width(cnt);
     const int E = min(slices_sorted(K, cw, nwarps), max(1, cnt / 512));   // a slice is worth >= 128 vectors
     size_t off[7];
-    sorted_smem_layout(a.cap, K, max_slices_sorted(K), off);
+    sorted_smem_layout(a.cap, K, nwarps, off);
     SortedSmem S;
     S.tile = reinterpret_cast<float*>(smem_raw + off[0]);
     S.jr = reinterpret_cast<uint32_t*>(smem_raw + off[1]);
@@ -728,15 +732,16 @@ cudaError_t launch_search(const float* x, const int64_t* row_offsets, int64_t C,
         // more small CTAs per SM.  One launch per class; a CTA whose row belongs to another
         // class exits at once.  A dense tensor has one class.
         struct RowClass { int64_t n_min, n_max; int threads; };
-        const RowClass classes[3] = {{0, 256, 64}, {257, 1152, 128}, {1153, INT64_MAX, 256}};
+        const RowClass classes[3] = {{1153, INT64_MAX, 256}, {257, 1152, 128}, {0, 256, 64}};
         size_t off[7];
-        const size_t smem_max = sorted_smem_layout(a.cap, K, max_slices_sorted(K), off);
+        const size_t smem_max = sorted_smem_layout(a.cap, K, kSWarps, off);
         if (smem_max > 48 * 1024) {  // above the default limit: opt in (idempotent, per device)
             e = cudaFuncSetAttribute(search_sorted_kernel,
                                      cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_max);
             if (e != cudaSuccess) return e;
         }
         const int full_cap = a.cap;
+        int launched = 0;
         for (const RowClass& rc : classes) {
             if (plan.max_n < rc.n_min) continue;
             if (!row_offsets && n > rc.n_max) continue;           // dense: every row has length n
@@ -746,10 +751,23 @@ cudaError_t launch_search(const float* x, const int64_t* row_offsets, int64_t C,
             a.grid_tiles = longest ? plan.tiles : 1;
             a.cap = longest ? full_cap
                             : (int)((std::min<int64_t>(plan.max_n, rc.n_max) + 3) / 4 * 4);
-            const size_t smem = sorted_smem_layout(a.cap, K, max_slices_sorted(K), off);
-            search_sorted_kernel<<<(unsigned)(C * a.grid_tiles), rc.threads, smem, stream>>>(a);
-            e = cudaGetLastError();
+            const size_t smem = sorted_smem_layout(a.cap, K, rc.threads / 32, off);
+            // Launches after the first may overlap the tail of the one before (they are
+            // independent of each other; all of them were ordered after the abs-max above by the
+            // first, ordinary launch).
+            cudaLaunchConfig_t cfg = {};
+            cfg.gridDim = dim3((unsigned)(C * a.grid_tiles));
+            cfg.blockDim = dim3((unsigned)rc.threads);
+            cfg.dynamicSmemBytes = smem;
+            cfg.stream = stream;
+            cudaLaunchAttribute attr[1];
+            attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+            attr[0].val.programmaticStreamSerializationAllowed = 1;
+            cfg.attrs = attr;
+            cfg.numAttrs = launched > 0 ? 1 : 0;
+            e = cudaLaunchKernelEx(&cfg, search_sorted_kernel, a);
             if (e != cudaSuccess) return e;
+            ++launched;
         }
         a.cap = full_cap;
     } else {

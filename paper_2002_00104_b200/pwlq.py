@@ -15,7 +15,8 @@ from typing import Optional
 import torch
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-_LIB_PATH = os.path.join(_HERE, "libpwlq.so")
+# PWLQ_LIBRARY selects another build of the same C ABI (e.g. one compiled with other options)
+_LIB_PATH = os.environ.get("PWLQ_LIBRARY") or os.path.join(_HERE, "libpwlq.so")
 _lib = None
 
 OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_WORKSPACE, ERR_CUDA, ERR_NONFINITE, ERR_TIMEOUT = range(7)
