@@ -3,7 +3,7 @@
 // Both are single streaming passes bound by HBM.  A thread owns 8 consecutive values: two
 // 128-bit loads of x, then one 64-bit store of byte codes (or one 32-bit store of nibble-packed
 // codes) and one region-mask byte, so that a warp writes contiguous 256 / 128 / 32-byte runs.
-// CTAs are persistent and walk spans of 4096 values; the rows that overlap a span are staged in
+// CTAs are persistent and walk spans of 8192 values; the rows that overlap a span are staged in
 // shared memory with their constants (four divisions per row, done once per span), so a thread's
 // row lookups and constant fetches stay on chip, and the next span's loads are already in flight
 // while the current one is staged and computed.
@@ -17,10 +17,10 @@ namespace pwlq {
 
 constexpr int kQThreads = 256;
 constexpr int kQChunk = kQThreads * 8;           // values one pass of the CTA covers
-constexpr int kQChunks = 2;                      // passes per span
+constexpr int kQChunks = 4;                      // passes per span
 constexpr int kQSpan = kQChunk * kQChunks;       // values per span (one staged row table)
 constexpr int kQRows = 512;                      // rows staged per span
-constexpr int kQStages = 3;                      // spans in flight per CTA (quantize)
+constexpr int kQStages = 2;                      // spans in flight per CTA (quantize)
 
 static __device__ int g_quantize_timeout;        // set when a bounded wait expired
 
