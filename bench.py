@@ -361,8 +361,12 @@ def run_ours(args, rank, world, local_rank):
             cores = os.cpu_count() or 1
             spans, _ = oracle_sample(w, 2e8)                 # short calibration
             ev, dt = time_oracle(w, spans, cores)
-            spans, what = oracle_sample(w, min(w.elem_cand, 15.0 * ev / dt))   # about 15 s
-            ev, dt = time_oracle(w, spans, cores)
+            spans, what = oracle_sample(w, min(w.elem_cand, 15.0 * ev / dt))   # about 15 s ...
+            ev, dt, passes = 0, 0.0, 0
+            while dt < 10.0 and passes < 8:                  # ... repeated if the box is faster
+                e1, d1 = time_oracle(w, spans, cores)
+                ev += e1; dt += d1; passes += 1
+            what += f", {passes} pass(es)"
             line["cpu_baseline"] = {"value": ev / dt / 1e9, "unit": UNIT, "cores": cores,
                                     "kind": "oracle", "sample": what, "seconds": dt}
         print(json.dumps(line), flush=True)
