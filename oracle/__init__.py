@@ -4,5 +4,5 @@ Only the tests, the smoke check and the benchmark's CPU-baseline leg import
 this package.  It shares no code with the CUDA path.
 """
 from .pwlq_oracle import (  # noqa: F401
-    OracleError, OracleLib, absmax, build, code_bytes, dequantize, elem, params, quantize, search,
+    OracleError, OracleLib, absmax, analytic_p, build, code_bytes, dequantize, elem, params, quantize, search, select_analytic,
 )

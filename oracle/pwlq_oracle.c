@@ -243,3 +243,75 @@ void pwlq_oracle_params(float m, float p, int bits, float *out5)
     pw_params P = make_params(m, p, bits);
     out5[0] = P.Lf; out5[1] = P.s1; out5[2] = P.inv1; out5[3] = P.s2; out5[4] = P.inv2;
 }
+
+/* ------------------------------------------------------------------------------------------
+ * Analytic breakpoint selection (Sec. 3.3 and Sec. 5.1): instead of searching a grid, assume a
+ * zero-mean Gaussian or Laplacian density for the row and take the breakpoint that minimises the
+ * expected error of Eq. 5, i.e. the root of the stationarity condition Eq. 9 on (0, m/2), or the
+ * closed-form approximation of Sec. 5.1.  All in binary64.
+ *
+ *   model 0: Gaussian, p = sigma * ln(0.8614 m / sigma + 0.6079)    (Sec. 5.1, read with m and p
+ *            in units of sigma: the printed form p / m = ln(0.8614 m + 0.6079) exceeds 1)
+ *   model 1: Gaussian, root of Eq. 9
+ *   model 2: Laplacian, root of Eq. 9
+ * Scale estimates (the paper does not say how the density is fitted; these are the maximum
+ * likelihood fits of the zero-mean models): sigma = sqrt(mean x^2), Laplace b = mean |x|.
+ * The result is clamped to (0, m/2] (the domain of Eq. 6); if Eq. 9 has no sign change there
+ * (a row that is flatter than the model allows), p = m/2. */
+static double model_cdf(int model, double scale, double p)
+{
+    if (model == 2) return 1.0 - 0.5 * exp(-p / scale);              /* Laplace, p >= 0 */
+    return 0.5 * erfc(-p / (scale * 1.4142135623730951));            /* Gaussian */
+}
+static double model_pdf(int model, double scale, double p)
+{
+    if (model == 2) return 0.5 / scale * exp(-p / scale);
+    return exp(-0.5 * (p / scale) * (p / scale)) / (scale * 2.5066282746310002);
+}
+/* Eq. 9 written as g(p) = 2 m F(p) - [2 m - p + m (m - 2 p) f(p)]; g < 0 left of the root. */
+static double eq9_residual(int model, double scale, double m, double p)
+{
+    return 2.0 * m * model_cdf(model, scale, p)
+           - (2.0 * m - p + m * (m - 2.0 * p) * model_pdf(model, scale, p));
+}
+
+double pwlq_oracle_analytic_p(double m, double scale, int model)
+{
+    double lo, hi, p;
+    int it;
+    if (!(m > 0.0) || !(scale > 0.0)) return 0.0;
+    if (model == 0) {
+        p = scale * log(0.8614 * (m / scale) + 0.6079);
+    } else {
+        lo = 0.0; hi = 0.5 * m;
+        if (!(eq9_residual(model, scale, m, hi) > 0.0)) return 0.5 * m;
+        for (it = 0; it < 80; ++it) {
+            double mid = 0.5 * (lo + hi);
+            if (eq9_residual(model, scale, m, mid) < 0.0) lo = mid; else hi = mid;
+        }
+        p = 0.5 * (lo + hi);
+    }
+    if (!(p > 0.0)) p = 0.5 * m * 1e-6;     /* the approximation's logarithm can go negative */
+    if (p > 0.5 * m) p = 0.5 * m;
+    return p;
+}
+
+int pwlq_oracle_select_analytic(const float *x, const int64_t *row_offsets, int64_t C, int64_t n,
+                                const float *m_in, int model, float *p_out, double *scale_out)
+{
+    int64_t c, i;
+    if (!x || !m_in || !p_out || C < 1 || model < 0 || model > 2) return ORACLE_ERR_ARG;
+    for (c = 0; c < C; ++c) {
+        int64_t b = row_begin(row_offsets, n, c), e = row_begin(row_offsets, n, c + 1);
+        double s2 = 0.0, s1 = 0.0, scale = 0.0;
+        for (i = b; i < e; ++i) {
+            double v = (double)x[i];
+            s2 += v * v;
+            s1 += fabs(v);
+        }
+        if (e > b) scale = (model == 2) ? s1 / (double)(e - b) : sqrt(s2 / (double)(e - b));
+        if (scale_out) scale_out[c] = scale;
+        p_out[c] = (float)pwlq_oracle_analytic_p((double)m_in[c], scale, model);
+    }
+    return ORACLE_OK;
+}

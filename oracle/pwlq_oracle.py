@@ -84,6 +84,9 @@ class OracleLib:
         lib.pwlq_oracle_elem.restype = None
         lib.pwlq_oracle_params.argtypes = [ctypes.c_float, ctypes.c_float, ctypes.c_int, P]
         lib.pwlq_oracle_params.restype = None
+        lib.pwlq_oracle_analytic_p.argtypes = [ctypes.c_double, ctypes.c_double, ctypes.c_int]
+        lib.pwlq_oracle_analytic_p.restype = ctypes.c_double
+        lib.pwlq_oracle_select_analytic.argtypes = [P, P, I64, I64, P, ctypes.c_int, P, P]
         self._lib = lib
 
     def absmax(self, x, row_offsets=None):
@@ -142,6 +145,23 @@ class OracleLib:
                                                 int(layout)), "dequantize")
         return y
 
+    def analytic_p(self, m, scale, model):
+        """Breakpoint of the assumed density (0: Gaussian ln-approximation, 1: Gaussian Eq. 9
+        root, 2: Laplacian Eq. 9 root), clamped to (0, m/2]."""
+        return float(self._lib.pwlq_oracle_analytic_p(float(m), float(scale), int(model)))
+
+    def select_analytic(self, x, m, model, row_offsets=None):
+        """Returns (p float32 [C], scale float64 [C]) for every row."""
+        flat, ro, C, n = _rows(x, row_offsets)
+        m = np.ascontiguousarray(m, dtype=np.float32)
+        assert m.size == C
+        p = np.empty(C, dtype=np.float32)
+        scale = np.empty(C, dtype=np.float64)
+        _check(self._lib.pwlq_oracle_select_analytic(_ptr(flat), _ptr(ro), C, n, _ptr(m),
+                                                     int(model), _ptr(p), _ptr(scale)),
+               "select_analytic")
+        return p, scale
+
     def elem(self, x, m, p, bits):
         """One value through Eq. 3: returns (code, region, q, y)."""
         code, region, q = ctypes.c_int(), ctypes.c_int(), ctypes.c_int()
@@ -185,6 +205,14 @@ def dequantize(*a, **k):
 
 def elem(*a, **k):
     return _get().elem(*a, **k)
+
+
+def analytic_p(*a, **k):
+    return _get().analytic_p(*a, **k)
+
+
+def select_analytic(*a, **k):
+    return _get().select_analytic(*a, **k)
 
 
 def params(*a, **k):

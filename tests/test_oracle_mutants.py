@@ -36,6 +36,12 @@ MUTANTS = {
                       "float a = x[i];\n            if (!(a <= 3.402823466e+38f)) return ORACLE_ERR_NONFINITE;\n            if (a > m) m = a;\n        }\n        m_out[c] = m;"),
     "dequant_ignores_region": ("float z = r ? p : 0.0f;\n            float v = q * s;", "float z = 0.0f;\n            float v = q * s;"),
     "p_from_wrong_ratio": ("float p = m * ratios[k];", "float p = m * ratios[K - 1 - k];"),
+    "eq9_wrong_sign": ("- (2.0 * m - p + m * (m - 2.0 * p) * model_pdf(model, scale, p));",
+                       "- (2.0 * m - p - m * (m - 2.0 * p) * model_pdf(model, scale, p));"),
+    "eq9_dropped_p": ("- (2.0 * m - p + m", "- (2.0 * m + m"),
+    "sigma_without_sqrt": (": sqrt(s2 / (double)(e - b));", ": (s2 / (double)(e - b));"),
+    "laplace_cdf_as_gauss_tail": ("return 1.0 - 0.5 * exp(-p / scale);", "return 1.0 - exp(-p / scale);"),
+    "approx_constant": ("0.8614 * (m / scale) + 0.6079", "0.8614 * (m / scale) + 0.06079"),
     "divide_not_reciprocal_free_pass": None,   # placeholder documented below
 }
 # 'divide_not_reciprocal': evaluating (|r| - z) / s by a true division instead of multiplying by
@@ -54,6 +60,9 @@ PIN_CALLS = [
     lambda o: pins.test_zero_rows_and_single_values(o),
     lambda o: pins.test_ragged_rows_equal_dense_rows(o),
     lambda o: pins.test_uniform_data_matches_eq2(o),
+    lambda o: pins.test_analytic_root_matches_an_independent_solver(o, 1, pins.stats.norm),
+    lambda o: pins.test_analytic_root_matches_an_independent_solver(o, 2, pins.stats.laplace),
+    lambda o: pins.test_analytic_approximation_and_scales(o),
 ]
 
 

@@ -339,3 +339,54 @@ def test_ln_approximation_reading(oracle):
     m = float(oracle.absmax(x)[0])
     res = oracle.search(x, 4, W.ratio_grid(400))
     assert abs(res["p"][0] - math.log(0.8614 * m + 0.6079)) < 0.12
+
+
+# ---------------------------------------------------------------- analytic selection (Eq. 9, Sec. 5.1)
+@pytest.mark.parametrize("model,dist", [(1, stats.norm), (2, stats.laplace)])
+def test_analytic_root_matches_an_independent_solver(oracle, model, dist):
+    """The oracle's bisection on Eq. 9 against scipy's Brent solver on the same equation written
+    with scipy's CDF / PDF."""
+    from scipy.optimize import brentq
+    for m, scale in ((4.0, 1.0), (6.5, 1.0), (0.31, 0.05), (12.0, 1.3), (3.0, 0.4)):
+        d = dist(0, scale)
+        g = lambda p: 2 * m * d.cdf(p) - (2 * m - p + m * (m - 2 * p) * d.pdf(p))
+        if g(0.5 * m) <= 0:
+            assert oracle.analytic_p(m, scale, model) == 0.5 * m
+            continue
+        want = brentq(g, 1e-12 * m, 0.5 * m, xtol=1e-15, rtol=1e-14)
+        assert math.isclose(oracle.analytic_p(m, scale, model), want, rel_tol=1e-9)
+    # a row much flatter than the model: no stationary point inside (0, m/2), the bound is taken
+    assert oracle.analytic_p(1.0, 5.0, 1) == 0.5
+
+
+def test_analytic_approximation_and_scales(oracle):
+    # Sec. 5.1 closed form in units of sigma, clamped to (0, m/2]
+    assert math.isclose(oracle.analytic_p(5.0, 1.0, 0), math.log(0.8614 * 5.0 + 0.6079), rel_tol=1e-12)
+    assert math.isclose(oracle.analytic_p(0.5, 0.1, 0), 0.1 * math.log(0.8614 * 5.0 + 0.6079), rel_tol=1e-12)
+    assert oracle.analytic_p(2.0, 1.0, 0) == min(math.log(0.8614 * 2.0 + 0.6079), 1.0)
+    assert oracle.analytic_p(0.0, 1.0, 0) == 0.0 and oracle.analytic_p(1.0, 0.0, 1) == 0.0
+    rng = np.random.default_rng(17)
+    x = rng.normal(0, 0.05, (3, 5000)).astype(np.float32)
+    m = oracle.absmax(x)
+    for model in (0, 1, 2):
+        p, scale = oracle.select_analytic(x, m, model)
+        ref = np.mean(np.abs(x.astype(np.float64)), axis=1) if model == 2 else \
+            np.sqrt(np.mean(x.astype(np.float64) ** 2, axis=1))
+        assert np.allclose(scale, ref, rtol=1e-12)
+        want = [oracle.analytic_p(float(m[c]), float(scale[c]), model) for c in range(3)]
+        assert np.array_equal(p, np.array(want, dtype=np.float32))
+
+
+@pytest.mark.parametrize("name,model", [("gauss", 0), ("gauss", 1), ("laplace", 2)])
+def test_analytic_choice_is_close_to_the_searched_optimum(oracle, name, model):
+    """Sec. 5.1: the analytic breakpoint gives almost the same error as the minimiser.  Here: its
+    squared error on the sample is within 3 % of the best grid candidate's (b = 4)."""
+    rng = np.random.default_rng(23)
+    n = 100000
+    x = (rng.standard_normal(n) if name == "gauss" else rng.laplace(0, 1, n)).astype(np.float32)
+    m = oracle.absmax(x)
+    p, _ = oracle.select_analytic(x, m, model)
+    grid = oracle.search(x, 4, W.ratio_grid(400))
+    at_p = oracle.search(x, 4, [p[0] / m[0]])
+    assert at_p["sse64"][0, 0] <= grid["sse64"][0].min() * 1.03
+    assert 0 < p[0] <= m[0] / 2
