@@ -122,6 +122,29 @@ int pwlq_dequantize_ragged(const uint8_t* codes, const uint8_t* region_mask,
                            const float* m, const float* p, float* y, int code_layout,
                            void* stream);
 
+/* Analytic breakpoint selection, the paper's own way of choosing p (Sec. 3.3, Sec. 5.1): assume a
+ * zero-mean density for each row, fit its scale, and take the breakpoint that minimises the
+ * expected error of Eq. 5 -- the root of Eq. 9 on (0, m/2) -- or the closed form of Sec. 5.1.
+ * O(n) per row instead of O(n K); the result can be fed to pwlq_quantize directly.
+ *   model      PWLQ_MODEL_GAUSS_APPROX   p = sigma ln(0.8614 m / sigma + 0.6079)  (Sec. 5.1, m and p
+ *                                        in units of sigma)
+ *              PWLQ_MODEL_GAUSS_ROOT     Gaussian, root of Eq. 9 (80 bisection steps, binary64)
+ *              PWLQ_MODEL_LAPLACE        Laplacian, root of Eq. 9
+ *   scale fit  sigma = sqrt(mean x^2) (Gaussian), b = mean |x| (Laplacian), binary64 sums in a
+ *              fixed order
+ *   m          [C] ranges (pwlq_absmax);  p_out [C], 0 < p <= m/2 (m/2 when Eq. 9 has no root
+ *              inside, 0 for an all-zero row);  scale_out [C] or NULL
+ *   workspace  pwlq_select_workspace_bytes(C, longest row) bytes, 256-byte aligned */
+enum { PWLQ_MODEL_GAUSS_APPROX = 0, PWLQ_MODEL_GAUSS_ROOT = 1, PWLQ_MODEL_LAPLACE = 2 };
+size_t pwlq_select_workspace_bytes(int64_t C, int64_t n);
+int pwlq_select_analytic(const float* x, int64_t C, int64_t n, const float* m, int model,
+                         float* p_out, float* scale_out, void* workspace, size_t workspace_bytes,
+                         void* stream);
+int pwlq_select_analytic_ragged(const float* x, const int64_t* row_offsets, int64_t C,
+                                int64_t total, int64_t max_n, const float* m, int model,
+                                float* p_out, float* scale_out, void* workspace,
+                                size_t workspace_bytes, void* stream);
+
 /* Whole path from HOST buffers: copies x (and row_offsets, ratios) to the device, runs abs-max,
  * search, quantize and dequantize there, and copies m, p, err, idx, codes and region_mask back.
  * All *_host pointers are host memory (pinned memory makes the copies asynchronous); NULL

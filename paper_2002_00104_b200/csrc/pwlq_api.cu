@@ -242,6 +242,46 @@ int pwlq_encode_host(const float* x_host, const int64_t* row_offsets_host, int64
     return PWLQ_OK;
 }
 
+size_t pwlq_select_workspace_bytes(int64_t C, int64_t n) {
+    if (C < 1 || n < 1) return 0;
+    return pwlq::select_workspace_bytes(C, n);
+}
+
+static int select_impl(const float* x, const int64_t* ro, int64_t C, int64_t n, int64_t total,
+                       int64_t max_n, const float* m, int model, float* p_out, float* scale_out,
+                       void* ws, size_t ws_bytes, void* stream) {
+    if (!x || !m || !p_out || model < PWLQ_MODEL_GAUSS_APPROX || model > PWLQ_MODEL_LAPLACE ||
+        max_n < 1 || max_n > total)
+        return PWLQ_ERR_INVALID_ARG;
+    if (misaligned(x, 4) || misaligned(m, 4) || misaligned(p_out, 4) || misaligned(scale_out, 4) ||
+        misaligned(ro, 8))
+        return PWLQ_ERR_INVALID_ARG;
+    const int64_t tiles = (max_n + 8191) / 8192;
+    if (total > kMaxTotal || C * tiles > ((int64_t)1 << 31) - 1) return PWLQ_ERR_UNSUPPORTED;
+    if (!ws || ws_bytes < pwlq::select_workspace_bytes(C, max_n)) return PWLQ_ERR_WORKSPACE;
+    if (misaligned(ws, 256)) return PWLQ_ERR_INVALID_ARG;
+    return from_cuda(pwlq::launch_select_analytic(x, ro, C, n, max_n, m, model, p_out, scale_out,
+                                                  ws, as_stream(stream)));
+}
+
+int pwlq_select_analytic(const float* x, int64_t C, int64_t n, const float* m, int model,
+                         float* p_out, float* scale_out, void* workspace, size_t workspace_bytes,
+                         void* stream) {
+    if (int rc = check_rows(C, n)) return rc;
+    return select_impl(x, nullptr, C, n, C * n, n, m, model, p_out, scale_out, workspace,
+                       workspace_bytes, stream);
+}
+
+int pwlq_select_analytic_ragged(const float* x, const int64_t* row_offsets, int64_t C,
+                                int64_t total, int64_t max_n, const float* m, int model,
+                                float* p_out, float* scale_out, void* workspace,
+                                size_t workspace_bytes, void* stream) {
+    if (int rc = check_rows(C, total)) return rc;
+    if (!row_offsets) return PWLQ_ERR_INVALID_ARG;
+    return select_impl(x, row_offsets, C, 0, total, max_n, m, model, p_out, scale_out, workspace,
+                       workspace_bytes, stream);
+}
+
 int pwlq_device_status(void) {
     const int expired = pwlq::absmax_timeout_flag() | pwlq::quantize_timeout_flag();
     return expired ? (1 << PWLQ_ERR_TIMEOUT) : 0;

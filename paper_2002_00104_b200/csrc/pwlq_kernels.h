@@ -39,6 +39,12 @@ cudaError_t launch_dequantize(const uint8_t* codes, const uint8_t* mask,
                               int bits, const float* m, const float* p, float* y, int layout,
                               cudaStream_t stream);
 
+size_t select_workspace_bytes(int64_t C, int64_t max_n);
+cudaError_t launch_select_analytic(const float* x, const int64_t* row_offsets, int64_t C,
+                                   int64_t n, int64_t max_n, const float* m, int model,
+                                   float* p_out, float* scale_out, void* workspace,
+                                   cudaStream_t stream);
+
 // 1 when a bounded wait of the kernel family expired since the library was loaded (reads a
 // device flag: synchronises with the device).
 int absmax_timeout_flag();

@@ -21,6 +21,7 @@ _lib = None
 
 OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_WORKSPACE, ERR_CUDA, ERR_NONFINITE, ERR_TIMEOUT = range(7)
 CODES_U8, CODES_PACKED = 0, 1
+MODEL_GAUSS_APPROX, MODEL_GAUSS_ROOT, MODEL_LAPLACE = 0, 1, 2
 MAX_K = 4096
 
 _P, _I64, _INT, _SZ = ctypes.c_void_p, ctypes.c_int64, ctypes.c_int, ctypes.c_size_t
@@ -40,6 +41,9 @@ _SIGNATURES = {
                                 _INT, _P, _SZ, _P, _P]),
     "pwlq_search_noalloc": (_INT, [_P, _I64, _I64, _INT, _P, _INT, _P, _P, _P, _P, _P, _P, _P]),
     "pwlq_search_noalloc_max_bytes": (_SZ, []),
+    "pwlq_select_workspace_bytes": (_SZ, [_I64, _I64]),
+    "pwlq_select_analytic": (_INT, [_P, _I64, _I64, _P, _INT, _P, _P, _P, _SZ, _P]),
+    "pwlq_select_analytic_ragged": (_INT, [_P, _P, _I64, _I64, _I64, _P, _INT, _P, _P, _P, _SZ, _P]),
     "pwlq_device_status": (_INT, []),
     "pwlq_status_string": (ctypes.c_char_p, [_INT]),
     "pwlq_version": (ctypes.c_char_p, []),
@@ -196,6 +200,28 @@ def search_noalloc(x, bits, ratios, m=None, want_sse=False, stream=None):
 
 def noalloc_max_bytes() -> int:
     return int(load_library().pwlq_search_noalloc_max_bytes())
+
+
+def select_analytic(x, m, model, row_offsets=None, max_n=None, want_scale=False, stream=None):
+    """Analytic breakpoint per row (the paper's own selection rule).  Returns (p, scale or None)."""
+    lib = load_library()
+    C, n, total = _shape(x, row_offsets)
+    longest = n if row_offsets is None else int(max_n)
+    need = int(lib.pwlq_select_workspace_bytes(C, longest))
+    ws = torch.empty(max(need, 256), dtype=torch.uint8, device=x.device)
+    p = torch.empty(C, dtype=torch.float32, device=x.device)
+    scale = torch.empty(C, dtype=torch.float32, device=x.device) if want_scale else None
+    tail = (_dev(m, torch.float32, "m"), int(model), _dev(p, torch.float32, "p"),
+            _dev(scale, torch.float32, "scale"), _dev(ws, torch.uint8, "workspace"), ws.numel(),
+            _stream(stream))
+    if row_offsets is None:
+        rc = lib.pwlq_select_analytic(_dev(x, torch.float32, "x"), C, n, *tail)
+    else:
+        rc = lib.pwlq_select_analytic_ragged(_dev(x, torch.float32, "x"),
+                                             _dev(row_offsets, torch.int64, "row_offsets"), C,
+                                             total, longest, *tail)
+    _check(rc, "pwlq_select_analytic")
+    return p, scale
 
 
 def search_status(workspace) -> int:
