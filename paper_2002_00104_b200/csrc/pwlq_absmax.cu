@@ -89,7 +89,7 @@ absmax_kernel(const float* __restrict__ x, Rows rows, int64_t total, uint32_t* _
         const bool has_next = use_table && span + 1 < s1;
         if (has_next) {
             const int l = S.T.find(span_end);
-            next_row0 = (l >= 0) ? row0 + l : rows.row_of(span_end);
+            next_row0 = (l >= 0) ? row0 + l : warp_row_of(rows, span_end);
             S.T.fetch(rows, nullptr, nullptr, next_row0, nf);
         }
         if (!single) {                                 // several rows: nothing is carried across

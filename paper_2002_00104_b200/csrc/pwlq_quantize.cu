@@ -19,34 +19,12 @@ constexpr int kQThreads = 256;
 constexpr int kQChunk = kQThreads * 8;           // values one pass of the CTA covers
 constexpr int kQChunks = 4;                      // passes per span
 constexpr int kQSpan = kQChunk * kQChunks;       // values per span (one staged row table)
-constexpr int kQRows = 512;                      // rows staged per span
 constexpr int kQStages = 2;                      // spans in flight per CTA (quantize)
 
 static __device__ int g_quantize_timeout;        // set when a bounded wait expired
 
-// Rows overlapping the CTA's span with their constants, computed once per span.
-struct QuantSmem {
-    RowTable<kQRows> T;
-    float m[kQRows];
-    PieceParams P[kQRows];
-
-    // All threads call this (three barriers).  The ranges and breakpoints of all staged rows are
-    // requested together with the row offsets; constants are computed for the rows that start
-    // inside the span (and for the row the span starts in).
-    __device__ __forceinline__ void load(const Rows& rows, const float* __restrict__ m_arr,
-                                         const float* __restrict__ p_arr, float Lf,
-                                         int64_t span_beg, int64_t span_end) {
-        T.load(rows, span_beg);
-        for (int r = threadIdx.x; r < kQRows; r += blockDim.x) {
-            if (T.row0 + r < rows.C && T.off[r] < span_end) {
-                const float mr = m_arr[T.row0 + r];
-                m[r] = mr;
-                P[r] = make_params(mr, p_arr[T.row0 + r], Lf);
-            }
-        }
-        __syncthreads();
-    }
-};
+// Ragged rows: the rows overlapping the CTA's current span, with their constants.
+typedef SpanTable<true> QuantSmem;
 
 // The row a thread is currently in: constants in registers, refreshed when it crosses a boundary.
 struct RowState {
@@ -66,10 +44,10 @@ struct RowState {
             P = make_params(m, __ldg(p_arr + row), Lf);
             return;
         }
-        const int loc = S.T.find(i);
+        const int loc = S.find(i);
         if (loc >= 0) {
-            beg = S.T.off[loc];
-            end = S.T.off[loc + 1];
+            beg = S.off[loc];
+            end = S.off[loc + 1];
             m = S.m[loc];
             P = S.P[loc];
         } else {                                   // beyond the staged rows (very many tiny rows)
@@ -97,7 +75,7 @@ __device__ __forceinline__ unsigned q_bulk_bytes(int64_t span, int64_t total, in
 // Persistent CTAs: each walks spans blockIdx.x, blockIdx.x + gridDim.x, ...; the values of the
 // next three spans are already on their way into a ring of shared-memory slots (bulk
 // asynchronous copies) while the rows of the current span are staged and its values quantized.
-template <bool PACKED, bool WANT_FAKE>
+template <bool PACKED, bool WANT_FAKE, bool RAGGED>
 __global__ void __launch_bounds__(kQThreads)
 quantize_kernel(const float* __restrict__ x, Rows rows, int64_t total, int bits,
                 const float* __restrict__ m_arr, const float* __restrict__ p_arr,
@@ -112,20 +90,38 @@ quantize_kernel(const float* __restrict__ x, Rows rows, int64_t total, int bits,
     const uint32_t sign_unit = 1u << (bits - 1);      // value of the sign bit inside a code
     const int sign_shift = 32 - bits;                 // moves bit 31 onto the code's sign bit
     const int64_t nspans = (total + kQSpan - 1) / kQSpan;
+    // The CTA's spans: ragged rows -> a block of consecutive spans (the next span's first row is
+    // then the row this span ends in, so its table can be requested without a search); dense rows
+    // -> every gridDim.x-th span.
+    const int64_t first = RAGGED ? nspans * blockIdx.x / gridDim.x : blockIdx.x;
+    const int64_t stride = RAGGED ? 1 : gridDim.x;
+    const int64_t last = RAGGED ? nspans * (blockIdx.x + 1) / gridDim.x : nspans;   // exclusive
     if (threadIdx.x == 0) s_abort = 0;
     Q.ring.init();
     for (int it = 0; it < kQStages; ++it) {
-        const int64_t span = blockIdx.x + (int64_t)it * gridDim.x;
-        if (span < nspans) Q.ring.issue(it, x + span * kQSpan, q_bulk_bytes(span, total, vec_in));
+        const int64_t span = first + (int64_t)it * stride;
+        if (span < last) Q.ring.issue(it, x + span * kQSpan, q_bulk_bytes(span, total, vec_in));
+    }
+    int64_t row0 = 0;                               // first staged row of the current span
+    RowFetch nf;
+    if (RAGGED && first < last) {
+        row0 = warp_row_of(rows, first * kQSpan);   // every warp finds the same row
+        S.fetch(rows, m_arr, p_arr, row0, nf);
+        S.commit(nf, min((first + 1) * kQSpan, total), Lf);
+        __syncthreads();
     }
     RowState rs;                                    // survives from span to span
     int64_t it = 0;
-    for (int64_t span = blockIdx.x; span < nspans; span += gridDim.x, ++it) {
+    for (int64_t span = first; span < last; span += stride, ++it) {
         const int64_t span_beg = span * kQSpan;
         const int64_t span_end = min(span_beg + kQSpan, total);
-        if (rows.offsets) {                            // ragged rows: stage the span's rows
-            S.load(rows, m_arr, p_arr, Lf, span_beg, span_end);
-            rs.beg = rs.end = 0;                       // staged constants are per span
+        // ragged rows: request the next span's table now, write it when this span is done
+        int64_t next_row0 = 0;
+        const bool has_next = RAGGED && span + 1 < last;
+        if (has_next) {
+            const int l = S.find(span_end);
+            next_row0 = (l >= 0) ? row0 + l : warp_row_of(rows, span_end);
+            S.fetch(rows, m_arr, p_arr, next_row0, nf);
         }
         float* xs = reinterpret_cast<float*>(Q.ring.slot(it));
         if (q_bulk_bytes(span, total, vec_in) != 0) {
@@ -259,9 +255,15 @@ quantize_kernel(const float* __restrict__ x, Rows rows, int64_t total, int bits,
             if (threadIdx.x == 0) atomicExch(&g_quantize_timeout, 1);
             return;
         }
-        const int64_t ahead = span + (int64_t)kQStages * gridDim.x;
-        if (ahead < nspans)
+        if (has_next) {
+            S.commit(nf, min(span_end + kQSpan, total), Lf);
+            row0 = next_row0;
+            rs.beg = rs.end = 0;                     // staged constants are per span
+        }
+        const int64_t ahead = span + (int64_t)kQStages * stride;
+        if (ahead < last)
             Q.ring.issue(it + kQStages, x + ahead * kQSpan, q_bulk_bytes(ahead, total, vec_in));
+        if (RAGGED) __syncthreads();                // the next table is published
     }
 }
 
@@ -307,7 +309,7 @@ struct CodeRegs {
     }
 };
 
-template <bool PACKED>
+template <bool PACKED, bool RAGGED>
 __global__ void __launch_bounds__(kQThreads)
 dequantize_kernel(const uint8_t* __restrict__ codes, const uint8_t* __restrict__ mask, Rows rows,
                   int64_t total, int bits, const float* __restrict__ m_arr,
@@ -318,16 +320,31 @@ dequantize_kernel(const uint8_t* __restrict__ codes, const uint8_t* __restrict__
     const int qmask = (1 << (bits - 1)) - 1;
     const int sign_shift = 32 - bits;                 // moves a code's sign bit to bit 31
     const int64_t nspans = (total + kQSpan - 1) / kQSpan;
+    // the CTA's spans: consecutive for ragged rows (chained row tables), strided for dense rows
+    const int64_t first = RAGGED ? nspans * blockIdx.x / gridDim.x : blockIdx.x;
+    const int64_t stride = RAGGED ? 1 : gridDim.x;
+    const int64_t last = RAGGED ? nspans * (blockIdx.x + 1) / gridDim.x : nspans;   // exclusive
     CodeRegs<PACKED> cur, nxt;
     RowState rs;                                    // survives from span to span
-    cur.load(codes, mask, (int64_t)blockIdx.x * kQSpan, total, vec_codes);
-    for (int64_t span = blockIdx.x; span < nspans; span += gridDim.x) {
+    cur.load(codes, mask, first * kQSpan, total, vec_codes);
+    int64_t row0 = 0;                               // first staged row of the current span
+    RowFetch nf;
+    if (RAGGED && first < last) {
+        row0 = warp_row_of(rows, first * kQSpan);
+        S.fetch(rows, m_arr, p_arr, row0, nf);
+        S.commit(nf, min((first + 1) * kQSpan, total), Lf);
+        __syncthreads();
+    }
+    for (int64_t span = first; span < last; span += stride) {
         const int64_t span_beg = span * kQSpan;
-        if (span + gridDim.x < nspans)
-            nxt.load(codes, mask, (span + gridDim.x) * kQSpan, total, vec_codes);
-        if (rows.offsets) {                            // ragged rows: stage the span's rows
-            S.load(rows, m_arr, p_arr, Lf, span_beg, min(span_beg + kQSpan, total));
-            rs.beg = rs.end = 0;
+        const int64_t span_end = min(span_beg + kQSpan, total);
+        if (span + stride < last) nxt.load(codes, mask, (span + stride) * kQSpan, total, vec_codes);
+        int64_t next_row0 = 0;
+        const bool has_next = RAGGED && span + 1 < last;
+        if (has_next) {
+            const int l = S.find(span_end);
+            next_row0 = (l >= 0) ? row0 + l : warp_row_of(rows, span_end);
+            S.fetch(rows, m_arr, p_arr, next_row0, nf);
         }
 #pragma unroll
         for (int c = 0; c < kQChunks; ++c) {
@@ -382,7 +399,15 @@ dequantize_kernel(const uint8_t* __restrict__ codes, const uint8_t* __restrict__
                 for (int t = 0; t < cnt; ++t) y[i0 + t] = yv[t];
             }
         }
-        if (rows.offsets) __syncthreads();          // the row table is rebuilt for the next span
+        if (RAGGED) {
+            __syncthreads();                        // the row table is no longer read
+            if (has_next) {
+                S.commit(nf, min(span_end + kQSpan, total), Lf);
+                row0 = next_row0;
+                rs.beg = rs.end = 0;
+            }
+            __syncthreads();                        // the next table is published
+        }
         cur = nxt;
     }
 }
@@ -435,13 +460,17 @@ cudaError_t launch_quantize(const float* x, const int64_t* row_offsets, int64_t 
     const int vec_in = aligned(x, 16), vec_fake = fake ? aligned(fake, 16) : 0;
     const size_t smem = sizeof(QuantizeSmem);
     const int vec_codes = packed ? aligned(codes, 4) : aligned(codes, 8);
-#define PWLQ_LAUNCH_QUANTIZE(PK, FK)                                                              \
-    quantize_kernel<PK, FK><<<persistent_grid((const void*)quantize_kernel<PK, FK>, kQThreads,    \
-                                              smem, nspans),                                      \
-                              kQThreads, smem, stream>>>(x, rows, total, bits, m, p, codes, mask, \
-                                                         fake, vec_in, vec_fake, vec_codes)
-    if (packed) { if (fake) PWLQ_LAUNCH_QUANTIZE(true, true); else PWLQ_LAUNCH_QUANTIZE(true, false); }
-    else        { if (fake) PWLQ_LAUNCH_QUANTIZE(false, true); else PWLQ_LAUNCH_QUANTIZE(false, false); }
+#define PWLQ_LAUNCH_QUANTIZE(PK, FK, RG)                                                          \
+    quantize_kernel<PK, FK, RG><<<persistent_grid((const void*)quantize_kernel<PK, FK, RG>,       \
+                                                  kQThreads, smem, nspans),                       \
+                                  kQThreads, smem, stream>>>(x, rows, total, bits, m, p, codes,   \
+                                                             mask, fake, vec_in, vec_fake,        \
+                                                             vec_codes)
+#define PWLQ_LAUNCH_QUANTIZE_RG(PK, FK) \
+    do { if (row_offsets) PWLQ_LAUNCH_QUANTIZE(PK, FK, true); else PWLQ_LAUNCH_QUANTIZE(PK, FK, false); } while (0)
+    if (packed) { if (fake) PWLQ_LAUNCH_QUANTIZE_RG(true, true); else PWLQ_LAUNCH_QUANTIZE_RG(true, false); }
+    else        { if (fake) PWLQ_LAUNCH_QUANTIZE_RG(false, true); else PWLQ_LAUNCH_QUANTIZE_RG(false, false); }
+#undef PWLQ_LAUNCH_QUANTIZE_RG
 #undef PWLQ_LAUNCH_QUANTIZE
     return cudaGetLastError();
 }
@@ -454,14 +483,14 @@ cudaError_t launch_dequantize(const uint8_t* codes, const uint8_t* mask,
     Rows rows{row_offsets, C, n, n > 0 ? 1.0 / (double)n : 0.0};
     const bool packed = (layout == 1 && bits <= 4);
     const int64_t nspans = (total + kQSpan - 1) / kQSpan;
-    if (packed)
-        dequantize_kernel<true><<<persistent_grid((const void*)dequantize_kernel<true>, kQThreads, 0, nspans),
-                                  kQThreads, 0, stream>>>(codes, mask, rows, total, bits, m, p, y,
-                                                          aligned(codes, 4), aligned(y, 16));
-    else
-        dequantize_kernel<false><<<persistent_grid((const void*)dequantize_kernel<false>, kQThreads, 0, nspans),
-                                   kQThreads, 0, stream>>>(codes, mask, rows, total, bits, m, p, y,
-                                                           aligned(codes, 8), aligned(y, 16));
+#define PWLQ_LAUNCH_DEQUANTIZE(PK, RG)                                                            \
+    dequantize_kernel<PK, RG><<<persistent_grid((const void*)dequantize_kernel<PK, RG>, kQThreads, \
+                                                0, nspans),                                       \
+                                kQThreads, 0, stream>>>(codes, mask, rows, total, bits, m, p, y,   \
+                                                        aligned(codes, PK ? 4 : 8), aligned(y, 16))
+    if (packed) { if (row_offsets) PWLQ_LAUNCH_DEQUANTIZE(true, true); else PWLQ_LAUNCH_DEQUANTIZE(true, false); }
+    else        { if (row_offsets) PWLQ_LAUNCH_DEQUANTIZE(false, true); else PWLQ_LAUNCH_DEQUANTIZE(false, false); }
+#undef PWLQ_LAUNCH_DEQUANTIZE
     return cudaGetLastError();
 }
 
