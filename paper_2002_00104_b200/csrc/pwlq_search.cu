@@ -151,12 +151,12 @@ __device__ __forceinline__ void finish_tile(const SearchArgs& a, int64_t row, in
         if (a.tiles > 1) {
             a.partials[((size_t)row * a.tiles + tile) * K + k] = tot;
         } else {
-            part[k] = tot;
+            if (E > 1) part[k] = tot;
             if (a.sse_all) a.sse_all[row * K + k] = (float)tot;
         }
     }
     if (a.tiles > 1) return;
-    __syncthreads();
+    if (E > 1) __syncthreads();                      // E == 1: part[] already holds the sums
     double best; int idx;
     block_argmin(part, K, red_val, red_idx, best, idx);
     if (threadIdx.x == 0) write_row_result(a, row, m, best, idx);
@@ -350,7 +350,6 @@ struct SortedSmem {
     float* tile;        // [cap + 4]
     uint32_t* jr;       // [cap]  bucket | rank << 11
     float* ps;          // [K]
-    float4* pa;         // [K]  (inv1, -s1, inv2, -s2)
     int* start;         // [K + 2]
     uint16_t* hist;     // [kSWarps][K + 2]
     double* part;       // [E][K]
@@ -362,7 +361,7 @@ __host__ __device__ inline size_t sorted_smem_layout(int cap, int K, int warps, 
     off[0] = take(sizeof(float) * (size_t)(cap + 4));
     off[1] = take(sizeof(uint32_t) * (size_t)cap);
     off[2] = take(sizeof(float) * (size_t)K);
-    off[3] = take(sizeof(float4) * (size_t)K);
+    off[3] = o;
     off[4] = take(sizeof(int) * (size_t)(K + 2));
     off[5] = take(sizeof(uint16_t) * (size_t)warps * (size_t)(K + 2));
     off[6] = take(sizeof(double) * (size_t)E * (size_t)K);
@@ -390,10 +389,11 @@ __device__ __forceinline__ int bucket_of(const float* ps, int K, float a, float 
 }
 
 template <int kCW, bool EXACT_V>
-__device__ __forceinline__ void eval_sorted(const SearchArgs& a, const SortedSmem& S, int n4,
-                                            int pad, int E, int* next_item) {
+__device__ __forceinline__ void eval_sorted(const SearchArgs& a, const SortedSmem& S, float m,
+                                            int n4, int pad, int E, int* next_item) {
     constexpr int kPhases = 32 / kCW;
     const int K = a.K;
+    const float Lf = (float)((1 << (a.bits - 1)) - 1);
     const int G = (K + kCW - 1) / kCW;
     const int lane = threadIdx.x & 31;
     const int ci = lane % kCW, ph = lane / kCW;
@@ -412,12 +412,12 @@ __device__ __forceinline__ void eval_sorted(const SearchArgs& a, const SortedSme
         // entries [0, B_k) of the sorted tile are the center values of candidate k
         const int c_hi = min(hi, (pad + S.start[k0 + 1]) >> 2);      // vectors below every boundary
         const int t_lo = max(lo, (pad + S.start[k1 + 1] + 3) >> 2);  // vectors above every boundary
-        const float4 pa = S.pa[k];
-        PieceParams P;
-        P.p = S.ps[k]; P.inv1 = pa.x; P.s1 = -pa.y; P.inv2 = pa.z; P.s2 = -pa.w;
+        // the candidate's constants (four divisions) are computed here, by the lanes that use
+        // them, while other warps keep the FP32 pipe busy -- not in a serial phase of the CTA
+        const PieceParams P = make_params(m, S.ps[k], Lf);
         Pairs c;
-        c.inv1 = pack2(pa.x, pa.x); c.ns1 = pack2(pa.y, pa.y);
-        c.inv2 = pack2(pa.z, pa.z); c.ns2 = pack2(pa.w, pa.w);
+        c.inv1 = pack2(P.inv1, P.inv1); c.ns1 = pack2(-P.s1, -P.s1);
+        c.inv2 = pack2(P.inv2, P.inv2); c.ns2 = pack2(-P.s2, -P.s2);
         c.np = pack2(-P.p, -P.p);
         c.magic = pack2(kMagic, kMagic); c.nmagic = pack2(-kMagic, -kMagic);
         Acc A;
@@ -459,7 +459,6 @@ search_sorted_kernel(SearchArgs a) {
     S.tile = reinterpret_cast<float*>(smem_raw + off[0]);
     S.jr = reinterpret_cast<uint32_t*>(smem_raw + off[1]);
     S.ps = reinterpret_cast<float*>(smem_raw + off[2]);
-    S.pa = reinterpret_cast<float4*>(smem_raw + off[3]);
     S.start = reinterpret_cast<int*>(smem_raw + off[4]);
     S.hist = reinterpret_cast<uint16_t*>(smem_raw + off[5]);
     S.part = reinterpret_cast<double*>(smem_raw + off[6]);
@@ -467,17 +466,16 @@ search_sorted_kernel(SearchArgs a) {
     const unsigned full = 0xffffffffu;
     const int HS = K + 2;                           // histogram stride; bucket K + 1 = "no value"
 
-    const float Lf = (float)((1 << (a.bits - 1)) - 1);
+    // candidate breakpoints p_k = m * ratio_k; they ascend exactly when the ratios do (m > 0 and
+    // the multiplication rounds monotonically)
+    int unordered = 0;
     for (int k = threadIdx.x; k < K; k += nthreads) {
-        const PieceParams P = make_params(m, __fmul_rn(m, a.ratios[k]), Lf);
-        S.ps[k] = P.p;
-        S.pa[k] = make_float4(P.inv1, -P.s1, P.inv2, -P.s2);
+        const float rk = __ldg(a.ratios + k);
+        if (k > 0) unordered |= (rk < __ldg(a.ratios + k - 1));
+        S.ps[k] = __fmul_rn(m, rk);
     }
     for (int i = threadIdx.x; i < nwarps * HS; i += nthreads) S.hist[i] = 0;
     if (threadIdx.x == 0) next_item = 0;
-    __syncthreads();
-    int unordered = 0;
-    for (int k = threadIdx.x + 1; k < K; k += nthreads) unordered |= (S.ps[k] < S.ps[k - 1]);
     if (__syncthreads_or(unordered)) {
         // the grid is not ascending: no sorted structure to exploit
         const int cnt4 = (cnt + 3) >> 2;
@@ -586,14 +584,14 @@ search_sorted_kernel(SearchArgs a) {
     const int64_t L = (1 << (a.bits - 1)) - 1;
     const bool fused = 2 * n_row >= L * L;
     if (cw == kCwLongTile) {
-        if (fused) eval_sorted<kCwLongTile, false>(a, S, n4, pad, E, &next_item);
-        else       eval_sorted<kCwLongTile, true>(a, S, n4, pad, E, &next_item);
+        if (fused) eval_sorted<kCwLongTile, false>(a, S, m, n4, pad, E, &next_item);
+        else       eval_sorted<kCwLongTile, true>(a, S, m, n4, pad, E, &next_item);
     } else if (cw == kCwMidTile) {
-        if (fused) eval_sorted<kCwMidTile, false>(a, S, n4, pad, E, &next_item);
-        else       eval_sorted<kCwMidTile, true>(a, S, n4, pad, E, &next_item);
+        if (fused) eval_sorted<kCwMidTile, false>(a, S, m, n4, pad, E, &next_item);
+        else       eval_sorted<kCwMidTile, true>(a, S, m, n4, pad, E, &next_item);
     } else {
-        if (fused) eval_sorted<kCwShortTile, false>(a, S, n4, pad, E, &next_item);
-        else       eval_sorted<kCwShortTile, true>(a, S, n4, pad, E, &next_item);
+        if (fused) eval_sorted<kCwShortTile, false>(a, S, m, n4, pad, E, &next_item);
+        else       eval_sorted<kCwShortTile, true>(a, S, m, n4, pad, E, &next_item);
     }
     __syncthreads();
     finish_tile(a, row, tile, m, S.part, E, red_val, red_idx);
