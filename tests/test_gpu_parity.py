@@ -227,3 +227,87 @@ def test_argument_errors_launch_nothing(pwlq):
 def test_no_bounded_wait_expired(pwlq):
     """Runs after the parity tests of this file: none of their kernels gave up on a wait."""
     assert pwlq.device_status() == 0
+
+
+# ------------------------------------------------------------------ awkward layouts, host entry
+def awkward_rows(seed=3):
+    """Ragged rows with empty rows, single values, lengths that straddle every vector width, one
+    all-zero row and one row longer than a search tile."""
+    lengths = [0, 1, 0, 3, 7, 8, 9, 0, 15, 16, 17, 31, 33, 100, 0, 255, 257, 1000, 4097, 8193, 5, 0]
+    rng = np.random.default_rng(seed)
+    parts = [rng.laplace(0, 0.03, n).astype(np.float32) for n in lengths]
+    parts[13][:] = 0.0
+    ro = np.concatenate([[0], np.cumsum(lengths)]).astype(np.int64)
+    return np.concatenate(parts), ro
+
+
+@pytest.mark.parametrize("misalign", [0, 1, 2, 3])
+@pytest.mark.parametrize("bits,layout", [(4, 1), (8, 0)])
+def test_whole_path_on_awkward_rows_and_unaligned_buffers(pwlq, oracle, misalign, bits, layout):
+    """Empty rows, tiny rows, a ragged tail, and every buffer shifted off its natural vector
+    alignment by `misalign` elements: the vector and bulk-copy fast paths must step aside."""
+    x, ro = awkward_rows()
+    total = x.size
+    ratios = W.ratio_grid(32)
+    xb = dev(np.concatenate([np.zeros(misalign, np.float32), x]))[misalign:]
+    m = pwlq.absmax(xb, row_offsets=dev(ro))
+    om = oracle.absmax(x, ro)
+    assert np.array_equal(np_(m), om)
+    s = pwlq.search(xb, bits, dev(ratios), m=m, row_offsets=dev(ro), max_n=8193, want_sse=True)
+    ora = oracle.search(x, bits, ratios, row_offsets=ro)
+    check_search({k: np_(s[k]) for k in ("p", "err", "idx", "sse")}, ora, ratios, om, np.diff(ro))
+    p = s["p"]
+    nbytes = pwlq.code_bytes(total, bits, layout)
+    cbuf = torch.zeros(nbytes + 16, dtype=torch.uint8, device="cuda")
+    mbuf = torch.zeros((total + 7) // 8 + 16, dtype=torch.uint8, device="cuda")
+    fbuf = torch.zeros(total + 16, dtype=torch.float32, device="cuda")
+    codes, mask, fake = cbuf[misalign:misalign + nbytes], mbuf[misalign:misalign + (total + 7) // 8], \
+        fbuf[misalign:misalign + total]
+    pwlq.quantize(xb, bits, m, p, layout=layout, row_offsets=dev(ro), out=(codes, mask, fake))
+    oc, ok, of = oracle.quantize(x, bits, om, np_(p), layout=layout, row_offsets=ro)
+    assert np.array_equal(np_(codes), oc) and np.array_equal(np_(mask), ok)
+    assert np_(fake).tobytes() == of.tobytes()
+    ybuf = torch.zeros(total + 16, dtype=torch.float32, device="cuda")
+    y = ybuf[misalign:misalign + total]
+    pwlq.dequantize(codes, mask, bits, m, p, layout=layout, row_offsets=dev(ro), out=y)
+    assert np_(y).tobytes() == of.tobytes()
+    assert float(ybuf[:misalign].abs().sum()) == 0 and float(ybuf[misalign + total:].abs().sum()) == 0
+    assert pwlq.device_status() == 0
+
+
+@pytest.mark.parametrize("ragged", [False, True])
+def test_encode_host_matches_oracle(pwlq, oracle, ragged):
+    """The host-buffer entry point (copies in, abs-max, search, quantize, dequantize, copies out)."""
+    if ragged:
+        w = W.small_mixed(seed=41, bits=4, K=64)
+        x, ro, C = w.x, w.row_offsets, w.C
+    else:
+        rng = np.random.default_rng(2)
+        x = rng.normal(0, 0.05, (12, 300)).astype(np.float32).reshape(-1)
+        ro, C = None, 12
+    total = x.size
+    max_n = int(np.diff(ro).max()) if ragged else 300
+    ratios = W.ratio_grid(64)
+    hx = torch.from_numpy(x).pin_memory()
+    hro = torch.from_numpy(ro).pin_memory() if ragged else None
+    out = {"m": torch.empty(C, dtype=torch.float32).pin_memory(),
+           "p": torch.empty(C, dtype=torch.float32).pin_memory(),
+           "err": torch.empty(C, dtype=torch.float32).pin_memory(),
+           "idx": torch.empty(C, dtype=torch.int32).pin_memory(),
+           "codes": torch.empty((total + 1) // 2, dtype=torch.uint8).pin_memory(),
+           "mask": torch.empty((total + 7) // 8, dtype=torch.uint8).pin_memory()}
+    scratch = torch.empty(pwlq.encode_host_scratch_bytes(C, total, max_n, 64), dtype=torch.uint8,
+                          device="cuda")
+    pwlq.encode_host(hx, hro, C, max_n, 4, torch.from_numpy(ratios).pin_memory(), out,
+                     pwlq.CODES_PACKED, scratch)
+    torch.cuda.synchronize()
+    xo = x if ragged else x.reshape(C, -1)
+    om = oracle.absmax(xo, ro)
+    assert np.array_equal(out["m"].numpy(), om)
+    ora = oracle.search(xo, 4, ratios, row_offsets=ro)
+    rows = np.arange(C)
+    gi = out["idx"].numpy()
+    gap = np.abs(ora["sse64"][rows, gi] - ora["sse64"][rows, ora["idx"]])
+    assert np.all(gap <= 1e-5 * ora["sse64"][rows, ora["idx"]] + 1e-30)
+    oc, ok, _ = oracle.quantize(xo, 4, om, out["p"].numpy(), layout=1, row_offsets=ro)
+    assert np.array_equal(out["codes"].numpy(), oc) and np.array_equal(out["mask"].numpy(), ok)
