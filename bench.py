@@ -40,6 +40,10 @@ SM_COUNT, FP32_LANES_PER_SM, SM_MAX_GHZ = 148, 128, 1.965
 ALU_PEAK_TLANEOPS = SM_COUNT * FP32_LANES_PER_SM * SM_MAX_GHZ / 1e3     # 37.2 T lane-ops/s
 LANE_OPS_PER_ELEM_CAND = 6      # sub, mul, 2 adds (round to nearest even), fma, fma
 L2_FLUSH_BYTES = 256 << 20
+# dram__bytes_read.sum + dram__bytes_write.sum of the search kernels of ONE step, from the ncu
+# capture summarised in profiles/search_sorted_kernel_resnet50.md (103.06 MB read, 0.66 MB
+# written; the values themselves are 102.0 MB).  Keyed by (workload, bits, K); None elsewhere.
+SEARCH_DRAM_BYTES = {("resnet50", 4, 256): 103.71e6}
 
 WORKLOADS = {
     "resnet50": W.resnet50,
@@ -340,7 +344,8 @@ def run_ours(args, rank, world, local_rank):
                           "dequantize": stage_tot[3] / args.steps},
             "roofline": {"bound": "alu", "achieved": achieved, "peak": ALU_PEAK_TLANEOPS,
                          "unit": "Tlaneop/s", "frac": achieved / ALU_PEAK_TLANEOPS,
-                         "traffic": None, "kernel": "search_kernel",
+                         "traffic": SEARCH_DRAM_BYTES.get((args.workload, w.bits, w.K)),
+                         "kernel": "search_sorted_kernel",
                          "peak_source": "148 SMs x 128 FP32 lanes x 1.965 GHz (derived)",
                          "search_gelem_cand_per_s": ec / (search_ms * 1e-3) / 1e9},
             "hbm_stages": {

@@ -8,6 +8,8 @@
 // atomic per warp when the row ends); a span that holds several rows is cut into one slice per
 // warp, and the warp walks the rows overlapping its slice (offsets staged in shared memory) with
 // a strided read, a shuffle reduction and one atomicMax per piece.
+#include <algorithm>
+
 #include "pwlq_common.cuh"
 #include "pwlq_kernels.h"
 #include "pwlq_pipeline.cuh"
@@ -18,12 +20,13 @@ constexpr int kAbsThreads = 256;
 constexpr int kAbsUnroll = 4;
 constexpr int kAbsSpan = kAbsThreads * 4 * kAbsUnroll;  // values per span
 constexpr int kAbsStages = 3;                            // spans in flight per CTA
+constexpr int kAbsTableRows = 512;                       // staged rows per span (rows of >= 8 values fit)
 
 static __device__ int g_absmax_timeout;                  // set when a bounded wait expired
 
 struct AbsSmem {
     BulkRing<kAbsStages, kAbsSpan * 4> ring;
-    SpanTable<false> T;
+    SpanTable<false, kAbsTableRows> T;
 };
 
 // Bytes of span `span` if it can be fetched by a bulk copy (aligned base, whole 16-byte units).
@@ -35,13 +38,13 @@ __device__ __forceinline__ unsigned abs_bulk_bytes(int64_t span, int64_t total, 
 
 __global__ void __launch_bounds__(kAbsThreads)
 absmax_kernel(const float* __restrict__ x, Rows rows, int64_t total, uint32_t* __restrict__ m_bits,
-              int vec_ok) {
+              int vec_ok, int64_t spans_per_cta) {
     extern __shared__ __align__(128) unsigned char smem_raw[];
     AbsSmem& S = *reinterpret_cast<AbsSmem*>(smem_raw);
     __shared__ int s_abort;
     const int64_t nspans = (total + kAbsSpan - 1) / kAbsSpan;
     // this CTA's consecutive spans
-    const int64_t s0 = nspans * blockIdx.x / gridDim.x, s1 = nspans * (blockIdx.x + 1) / gridDim.x;
+    const int64_t s0 = blockIdx.x * spans_per_cta, s1 = min(s0 + spans_per_cta, nspans);
     const bool use_table = rows.offsets != nullptr || rows.n < kAbsSpan;   // several rows per span
     if (threadIdx.x == 0) s_abort = 0;
     S.ring.init();
@@ -50,11 +53,11 @@ absmax_kernel(const float* __restrict__ x, Rows rows, int64_t total, uint32_t* _
             S.ring.issue(it, x + (s0 + it) * kAbsSpan, abs_bulk_bytes(s0 + it, total, vec_ok));
 
     int64_t row0 = 0;                                  // first staged row of the current span
-    RowFetch nf;
+    RowFetch<kAbsTableRows> nf;
     if (use_table && s0 < s1) {
-        row0 = warp_row_of(rows, s0 * kAbsSpan);       // every warp finds the same row
+        row0 = cta_row_near(rows, s0 * kAbsSpan);
         S.T.fetch(rows, nullptr, nullptr, row0, nf);
-        S.T.commit(nf, 0, 0.0f);
+        S.T.commit(nf, 0.0f);
         __syncthreads();
     }
 
@@ -78,15 +81,18 @@ absmax_kernel(const float* __restrict__ x, Rows rows, int64_t total, uint32_t* _
         bool single;
         int64_t first_row;
         if (use_table) {
-            first_row = row0;
-            single = S.T.off[1] >= span_end;
+            const int l0 = S.T.find(span_beg);          // -1: more rows than the window holds
+            first_row = row0 + l0;
+            single = l0 >= 0 && S.T.off[l0 + 1] >= span_end;
         } else {
             first_row = rows.dense_row(span_beg);
             single = (first_row + 1) * rows.n >= span_end;
         }
-        // the next span starts in the row in which this one ends: request its table now
+        // the staged rows end before the next span does: request the window that starts in the
+        // row in which this span ends
         int64_t next_row0 = 0;
-        const bool has_next = use_table && span + 1 < s1;
+        const bool has_next = use_table && span + 1 < s1 &&
+                              !S.T.covers(min(span_end + kAbsSpan, total));
         if (has_next) {
             const int l = S.T.find(span_end);
             next_row0 = (l >= 0) ? row0 + l : warp_row_of(rows, span_end);
@@ -123,32 +129,70 @@ absmax_kernel(const float* __restrict__ x, Rows rows, int64_t total, uint32_t* _
                 }
             }
         } else {
-            // several rows: every warp takes a contiguous slice of the span and walks the rows
-            // that overlap it; per (slice, row) piece a strided read, a shuffle reduction and one
-            // atomic.  No per-value row lookup, no divergence.
+            // several rows: every warp takes a contiguous slice of the span and walks it in
+            // windows of 128 values (one 128-bit read per lane).  The maximum of the row the warp
+            // is in stays in per-lane registers from window to window; when the row ends inside a
+            // window the lanes' values are split at the boundary, the finished row is reduced with
+            // one warp-wide maximum and one atomic, and the next row starts.  All control flow is
+            // warp-uniform.
             const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
             constexpr int kSlice = kAbsSpan / (kAbsThreads / 32);
-            const int64_t sl_beg = span_beg + (int64_t)warp * kSlice;
-            const int64_t sl_end = min(sl_beg + kSlice, span_end);
-            int64_t pos = sl_beg;
-            int l = (pos < sl_end && use_table) ? S.T.find(pos) : -1;
-            while (pos < sl_end) {
-                int64_t r_glob, r_end;
-                if (l >= 0 && l < kTableRows) {            // staged row
-                    r_glob = row0 + l;
-                    r_end = S.T.off[l + 1];
-                    ++l;
-                } else {                                   // long dense rows, or beyond the staged rows
-                    r_glob = rows.row_of(pos);
-                    r_end = rows.begin(r_glob + 1);
-                }
-                const int64_t e = min(r_end, sl_end);
+            const int sl_beg = warp * kSlice;                              // relative to the span
+            const int sl_end = min(sl_beg + kSlice, (int)(span_end - span_beg));
+            if (sl_beg < sl_end) {
+                int l = use_table ? S.T.find(span_beg + sl_beg) : -1;
+                int64_t r_glob = 0;
+                int r_end = 0;                                             // relative to the span
+                auto enter_row = [&](int pos) {            // the row that contains / follows pos
+                    int64_t e;
+                    if (l >= 0 && l < kAbsTableRows) {     // staged row
+                        r_glob = row0 + l;
+                        e = S.T.off[l + 1];
+                        ++l;
+                    } else {                               // long dense rows, or beyond the table
+                        r_glob = rows.row_of(span_beg + pos);
+                        e = rows.begin(r_glob + 1);
+                        l = -1;
+                    }
+                    r_end = (int)min(e - span_beg, (int64_t)kAbsSpan);
+                };
+                enter_row(sl_beg);
                 uint32_t v = 0;
-                for (int64_t i = pos + lane; i < e; i += 32) v = max(v, abs_bits(xs[i - span_beg]));
+                for (int wb = sl_beg; wb < sl_end; wb += 128) {
+                    const int we = min(wb + 128, sl_end);
+                    const int i0 = wb + 4 * lane;
+                    uint32_t b[4] = {0u, 0u, 0u, 0u};
+                    if (i0 + 4 <= we) {
+                        const float4 f = *reinterpret_cast<const float4*>(xs + i0);
+                        b[0] = abs_bits(f.x); b[1] = abs_bits(f.y);
+                        b[2] = abs_bits(f.z); b[3] = abs_bits(f.w);
+                    } else {
 #pragma unroll
-                for (int o = 16; o > 0; o >>= 1) v = max(v, __shfl_xor_sync(0xffffffffu, v, o));
+                        for (int t = 0; t < 4; ++t)
+                            if (i0 + t < we) b[t] = abs_bits(xs[i0 + t]);
+                    }
+                    if (r_end >= we) {                     // the window lies inside the current row
+                        v = max(max(v, b[0]), max(b[1], max(b[2], b[3])));
+                        continue;
+                    }
+                    int pos = wb;                          // values before pos are accounted for
+                    while (true) {
+                        const int e = min(r_end, we);
+#pragma unroll
+                        for (int t = 0; t < 4; ++t)
+                            if (i0 + t >= pos && i0 + t < e) v = max(v, b[t]);
+                        if (r_end > we) break;             // the row continues in the next window
+                        v = __reduce_max_sync(0xffffffffu, v);
+                        if (lane == 0 && v != 0) atomicMax(m_bits + r_glob, v);
+                        v = 0;
+                        pos = e;
+                        if (pos >= sl_end) break;          // the slice ends with this row
+                        enter_row(pos);
+                        if (pos >= we) break;              // the new row starts with the next window
+                    }
+                }
+                v = __reduce_max_sync(0xffffffffu, v);     // the row the slice ends in
                 if (lane == 0 && v != 0) atomicMax(m_bits + r_glob, v);
-                pos = e;
             }
         }
         __syncthreads();                              // slot and table are no longer read
@@ -156,11 +200,11 @@ absmax_kernel(const float* __restrict__ x, Rows rows, int64_t total, uint32_t* _
             if (threadIdx.x == 0) atomicExch(&g_absmax_timeout, 1);
             return;
         }
-        if (has_next) { S.T.commit(nf, 0, 0.0f); row0 = next_row0; }
+        if (has_next) { S.T.commit(nf, 0.0f); row0 = next_row0; }
         if (span + kAbsStages < s1)
             S.ring.issue(it + kAbsStages, x + (span + kAbsStages) * kAbsSpan,
                          abs_bulk_bytes(span + kAbsStages, total, vec_ok));
-        if (use_table) __syncthreads();               // the next table is published
+        if (has_next) __syncthreads();                // the next window is published
     }
     flush_merged();                                   // what is still carried at the end
 }
@@ -192,10 +236,17 @@ cudaError_t launch_absmax(const float* x, const int64_t* row_offsets, int64_t C,
                                                       sizeof(AbsSmem));
         cached[dev] = (sms > 0 && per_sm > 0) ? sms * per_sm : 148;
     }
-    const unsigned grid = (unsigned)(nspans < cached[dev] ? nspans : cached[dev]);
+    // Long dense rows cost the same everywhere: one CTA per slot of the device, equal shares.
+    // Where spans hold several rows the cost per span depends on the row lengths, so the spans are
+    // handed out in small blocks (about four per slot) and the hardware scheduler balances them.
+    const int64_t slots = cached[dev];
+    const bool several_rows = row_offsets != nullptr || n < kAbsSpan;
+    int64_t per_cta = (nspans + slots - 1) / slots;
+    if (several_rows) per_cta = std::min<int64_t>(std::max<int64_t>((nspans + 4 * slots - 1) / (4 * slots), 4), 32);
+    const unsigned grid = (unsigned)((nspans + per_cta - 1) / per_cta);
     const int vec_ok = (reinterpret_cast<uintptr_t>(x) & 15u) == 0;
     absmax_kernel<<<grid, kAbsThreads, sizeof(AbsSmem), stream>>>(
-        x, rows, total, reinterpret_cast<uint32_t*>(m_out), vec_ok);
+        x, rows, total, reinterpret_cast<uint32_t*>(m_out), vec_ok, per_cta);
     return cudaGetLastError();
 }
 

@@ -103,41 +103,68 @@ __device__ __forceinline__ int64_t warp_row_of(const Rows& rows, int64_t i) {
     return lo;
 }
 
-// The rows that overlap one CTA's span of the flat storage, staged in shared memory so that the
-// per-thread row lookups never touch global memory.  A persistent CTA walks consecutive spans, so
-// the first row of the next span is the row in which the current span ends: the next table's
-// offsets (and ranges / breakpoints) are requested into registers before the current span is
-// processed and written to shared memory after it, which keeps every global round trip off the
-// critical path.  Values that lie beyond the last staged row (spans made of very many tiny or
-// empty rows) use the global search.
-constexpr int kTableRows = 512;
+// A row at or shortly before the row that contains flat index i (at most three rows before it),
+// found by a whole CTA together in rounds of blockDim.x-way search: two dependent rounds of loads
+// for up to 65536 rows with 256 threads.  Every thread calls it with the same i (it contains CTA
+// barriers) and gets the same answer.
+__device__ __forceinline__ int64_t cta_row_near(const Rows& rows, int64_t i) {
+    if (!rows.offsets) return rows.dense_row(i);
+    const int64_t T = blockDim.x;
+    int64_t lo = 0, hi = rows.C;                     // offsets[lo] <= i < offsets[hi]
+    while (hi - lo > 4) {
+        const int64_t step = (hi - lo + T - 1) / T;
+        const int64_t q = lo + (int64_t)(threadIdx.x + 1) * step;
+        const int le = (q < hi) && (rows.offsets[q] <= i);       // true for a prefix of the threads
+        const int cnt = __syncthreads_count(le);
+        const int64_t new_lo = lo + (int64_t)cnt * step;
+        hi = min(hi, new_lo + step);
+        lo = new_lo;
+    }
+    return lo;
+}
+
+// A window of CAP consecutive rows of the flat storage, staged in shared memory so that the
+// per-thread row lookups of a CTA never touch global memory.  The CTA walks consecutive spans and
+// keeps the window for as long as it reaches to the end of the next span: with long
+// rows it is filled once per CTA.  When the next span will run past it, the window that starts at
+// the row in which the current span ends is requested into registers before the current span is
+// processed and written to shared memory after it, which keeps the global round trip off the
+// critical path.  Values that lie beyond the last staged row (spans with more than CAP rows) use
+// the global search.
 constexpr int kTableThreads = 256;        // CTA size the fetch / commit pattern is written for
 
-struct RowFetch {                          // what one thread holds of the next table
-    int64_t off[3];                        // rows tid, tid + 256, and (thread 0) the end entry
-    float m[2], p[2];
+template <int CAP>
+struct RowFetch {                          // what one thread holds of the next window
+    static constexpr int kPerThread = CAP / kTableThreads;
+    int64_t off[kPerThread + 1];           // rows tid + u * 256, and (thread 0) the entry CAP
+    float m[kPerThread], p[kPerThread];
 };
 
-template <bool PARAMS>
+template <bool PARAMS, int CAP>
 struct SpanTable {
-    int64_t off[kTableRows + 1];  // off[r] = first flat index of row row0 + r (INT64_MAX past the end)
-    float m[PARAMS ? kTableRows : 1];
-    PieceParams P[PARAMS ? kTableRows : 1];
+    static constexpr int kPerThread = CAP / kTableThreads;
+    static_assert(CAP % kTableThreads == 0, "whole rounds of the CTA");
+    int64_t off[CAP + 1];     // off[r] = first flat index of row row0 + r (INT64_MAX past the last row)
+    float m[PARAMS ? CAP : 1];
+    PieceParams P[PARAMS ? CAP : 1];
+
+    // True when every flat index below `end` lies in a staged row (or past the last row).
+    __device__ __forceinline__ bool covers(int64_t end) const { return off[CAP] >= end; }
 
     // Local index of the staged row containing i, or -1 when i lies beyond the staged rows.
-    // Rows inside one span are mostly equally long (one layer), so a proportional guess is tried
-    // first and corrected by a few neighbour steps; irregular tables fall back to bisection.
+    // Neighbouring rows are mostly equally long (one layer), so a proportional guess is tried
+    // first and corrected by a few neighbour steps; irregular windows fall back to bisection.
     __device__ __forceinline__ int find(int64_t i) const {
-        const int64_t last = off[kTableRows];
+        const int64_t last = off[CAP];
         if (i >= last) return -1;
-        int lo = 0, hi = kTableRows;                  // off[lo] <= i < off[hi]
+        int lo = 0, hi = CAP;                         // off[lo] <= i < off[hi]
         if (last != INT64_MAX) {
-            const float scale = (float)kTableRows / (float)(last - off[0]);
-            int g = min(max((int)((float)(i - off[0]) * scale), 0), kTableRows - 1);
+            const float scale = (float)CAP / (float)(last - off[0]);
+            int g = min(max((int)((float)(i - off[0]) * scale), 0), CAP - 1);
 #pragma unroll
             for (int t = 0; t < 4; ++t) {
                 if (off[g] > i) { hi = g; g = max(g - 1, 0); }
-                else if (off[g + 1] <= i) { lo = g + 1; g = min(g + 1, kTableRows - 1); }
+                else if (off[g + 1] <= i) { lo = g + 1; g = min(g + 1, CAP - 1); }
                 else return g;
             }
         }
@@ -147,68 +174,33 @@ struct SpanTable {
         }
         return lo;
     }
-    // Requests the table that starts at row r0 (no barrier; the values stay in registers).
+    // Requests the window that starts at row r0 (no barrier; the values stay in registers).
     __device__ __forceinline__ void fetch(const Rows& rows, const float* __restrict__ m_arr,
                                           const float* __restrict__ p_arr, int64_t r0,
-                                          RowFetch& f) const {
+                                          RowFetch<CAP>& f) const {
 #pragma unroll
-        for (int u = 0; u < 2; ++u) {
-            const int64_t row = r0 + threadIdx.x + u * kTableThreads;
+        for (int u = 0; u < kPerThread; ++u) {
+            const int64_t row = r0 + (int)threadIdx.x + u * kTableThreads;
             f.off[u] = (row <= rows.C) ? rows.begin(row) : INT64_MAX;
             f.m[u] = f.p[u] = 0.0f;
             if (PARAMS && row < rows.C) { f.m[u] = __ldg(m_arr + row); f.p[u] = __ldg(p_arr + row); }
         }
-        f.off[2] = (threadIdx.x == 0 && r0 + kTableRows <= rows.C) ? rows.begin(r0 + kTableRows)
-                                                                   : INT64_MAX;
+        f.off[kPerThread] = (threadIdx.x == 0 && r0 + CAP <= rows.C) ? rows.begin(r0 + CAP)
+                                                                     : INT64_MAX;
     }
-    // Writes what fetch() requested; call between the barrier that retires the previous table and
-    // the barrier that publishes this one.  Constants are computed for rows that start before
-    // span_end only.
-    __device__ __forceinline__ void commit(const RowFetch& f, int64_t span_end, float Lf) {
+    // Writes what fetch() requested, with the rows' constants; call between the barrier that
+    // retires the previous window and the barrier that publishes this one.
+    __device__ __forceinline__ void commit(const RowFetch<CAP>& f, float Lf) {
 #pragma unroll
-        for (int u = 0; u < 2; ++u) {
-            const int r = threadIdx.x + u * kTableThreads;
+        for (int u = 0; u < kPerThread; ++u) {
+            const int r = (int)threadIdx.x + u * kTableThreads;
             off[r] = f.off[u];
-            if (PARAMS && f.off[u] < span_end) {
+            if (PARAMS) {
                 m[r] = f.m[u];
                 P[r] = make_params(f.m[u], f.p[u], Lf);
             }
         }
-        if (threadIdx.x == 0) off[kTableRows] = f.off[2];
-    }
-};
-
-// Stand-alone variant used by the quantize / dequantize kernels (their spans are not consecutive):
-// the rows that overlap one CTA's span, staged in shared memory so that the per-thread row lookups
-// never touch global memory.  R = table capacity; values that lie beyond
-// the last staged row (spans made of very many tiny or empty rows) use the global search.
-template <int R>
-struct RowTable {
-    int64_t off[R + 1];       // off[r] = first flat index of row row0 + r (INT64_MAX past the end)
-    int64_t row0;
-
-    // All threads of the CTA call this (two barriers); afterwards thread r still holds off[r] of
-    // the rows r = threadIdx.x, threadIdx.x + blockDim.x, ... it loaded.
-    __device__ __forceinline__ void load(const Rows& rows, int64_t span_beg) {
-        if (threadIdx.x < 32) {
-            const int64_t r0 = warp_row_of(rows, span_beg);
-            if (threadIdx.x == 0) row0 = r0;
-        }
-        __syncthreads();
-        const int64_t r0 = row0;
-        for (int r = threadIdx.x; r <= R; r += blockDim.x)
-            off[r] = (r0 + r <= rows.C) ? rows.begin(r0 + r) : INT64_MAX;
-        __syncthreads();
-    }
-    // Local index of the staged row containing i, or -1 when i lies beyond the staged rows.
-    __device__ __forceinline__ int find(int64_t i) const {
-        if (i >= off[R]) return -1;
-        int lo = 0, hi = R;                           // off[lo] <= i < off[hi]
-        while (hi - lo > 1) {
-            const int mid = (lo + hi) >> 1;
-            if (off[mid] <= i) lo = mid; else hi = mid;
-        }
-        return lo;
+        if (threadIdx.x == 0) off[CAP] = f.off[kPerThread];
     }
 };
 

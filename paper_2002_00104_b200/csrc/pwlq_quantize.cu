@@ -7,6 +7,7 @@
 // shared memory with their constants (four divisions per row, done once per span), so a thread's
 // row lookups and constant fetches stay on chip, and the next span's loads are already in flight
 // while the current one is staged and computed.
+#include <algorithm>
 #include <mutex>
 
 #include "pwlq_common.cuh"
@@ -17,46 +18,82 @@ namespace pwlq {
 
 constexpr int kQThreads = 256;
 constexpr int kQChunk = kQThreads * 8;           // values one pass of the CTA covers
-constexpr int kQChunks = 4;                      // passes per span
+constexpr int kQChunks = 2;                      // passes per span
 constexpr int kQSpan = kQChunk * kQChunks;       // values per span (one staged row table)
 constexpr int kQStages = 2;                      // spans in flight per CTA (quantize)
 
 static __device__ int g_quantize_timeout;        // set when a bounded wait expired
 
-// Ragged rows: the rows overlapping the CTA's current span, with their constants.
-typedef SpanTable<true> QuantSmem;
+// Offset inside the span of the eight values a thread handles in pass c.  A warp owns one
+// contiguous eighth of the span and walks it in passes of 256 values, so that a thread's
+// successive passes mostly stay inside one row (its row constants stay in registers) while a
+// warp's reads and writes of one pass remain contiguous.
+__device__ __forceinline__ int chunk_offset(int c) {
+    return ((int)threadIdx.x >> 5) * (kQSpan / (kQThreads / 32)) + c * 256 + ((int)threadIdx.x & 31) * 8;
+}
+
+// The rows overlapping the CTA's current span, with their constants (ragged rows, and dense rows
+// shorter than a span).
+constexpr int kQTableRows = 512;                 // rows of >= 8 values always fit
+typedef SpanTable<true, kQTableRows> QuantSmem;
+typedef RowFetch<kQTableRows> QuantFetch;
 
 // The row a thread is currently in: constants in registers, refreshed when it crosses a boundary.
 struct RowState {
     int64_t beg = 0, end = 0;
     float m = 0.0f;
     PieceParams P;
+    int loc = -1;                                  // index in the staged table (-1: not from it)
 
+    template <bool TABLE>
     __device__ __forceinline__ void seek(const QuantSmem& S, const Rows& rows,
                                          const float* __restrict__ m_arr,
                                          const float* __restrict__ p_arr, float Lf, int64_t i) {
         if (i >= beg && i < end) return;
-        if (!rows.offsets) {                       // dense: arithmetic, constants from L1 / L2
-            const int64_t row = rows.dense_row(i);
-            beg = row * rows.n;
-            end = beg + rows.n;
-            m = __ldg(m_arr + row);
-            P = make_params(m, __ldg(p_arr + row), Lf);
-            return;
-        }
-        const int loc = S.find(i);
+        loc = TABLE ? S.find(i) : -1;
         if (loc >= 0) {
             beg = S.off[loc];
             end = S.off[loc + 1];
             m = S.m[loc];
             P = S.P[loc];
-        } else {                                   // beyond the staged rows (very many tiny rows)
+        } else {                                   // long dense rows, or beyond the staged rows
             const int64_t row = rows.row_of(i);
             beg = rows.begin(row);
             end = rows.begin(row + 1);
-            m = m_arr[row];
-            P = make_params(m, p_arr[row], Lf);
+            m = __ldg(m_arr + row);
+            P = make_params(m, __ldg(p_arr + row), Lf);
         }
+    }
+    // Constants of the row that follows, if that row reaches at least to need_end.
+    template <bool TABLE>
+    __device__ __forceinline__ bool next_row(const QuantSmem& S, const Rows& rows,
+                                             const float* __restrict__ m_arr,
+                                             const float* __restrict__ p_arr, float Lf,
+                                             int64_t need_end, float& mB, PieceParams& PB,
+                                             int64_t& endB) const {
+        if (TABLE) {
+            if (loc < 0 || loc + 1 >= kQTableRows) return false;
+            endB = S.off[loc + 2];
+            if (endB < need_end) return false;
+            mB = S.m[loc + 1];
+            PB = S.P[loc + 1];
+            return true;
+        }
+        if (rows.offsets || rows.n < need_end - end) return false;
+        const int64_t row = rows.dense_row(end);
+        if (row >= rows.C) return false;
+        endB = end + rows.n;
+        mB = __ldg(m_arr + row);
+        PB = make_params(mB, __ldg(p_arr + row), Lf);
+        return true;
+    }
+    // Moves on to the row that next_row() returned.
+    __device__ __forceinline__ void advance(float mB, const PieceParams& PB, int64_t endB) {
+        beg = end;
+        end = endB;
+        m = mB;
+        P = PB;
+        if (loc >= 0) ++loc;
     }
 };
 
@@ -72,30 +109,77 @@ __device__ __forceinline__ unsigned q_bulk_bytes(int64_t span, int64_t total, in
     return (vec_in && (cnt & 3) == 0) ? (unsigned)(cnt * 4) : 0u;
 }
 
-// Persistent CTAs: each walks spans blockIdx.x, blockIdx.x + gridDim.x, ...; the values of the
-// next three spans are already on their way into a ring of shared-memory slots (bulk
-// asynchronous copies) while the rows of the current span are staged and its values quantized.
-template <bool PACKED, bool WANT_FAKE, bool RAGGED>
+// Eight consecutive values, the first `split` of them in row A and the rest in row B (TWO = false:
+// all in row A), both rows with m > 0.  The sequence of quantize_mag with the per-row tests
+// hoisted, the level taken from the mantissa of t + 1.5 * 2^23, and the sign flag (x < 0, false
+// for -0.0) read off the sign bit of x + 0.0.  Codes are packed and region bits gathered on the
+// fly; there is no branch per value.
+template <bool PACKED, bool WANT_FAKE, bool TWO>
+__device__ __forceinline__ void quantize8(const float (&xv)[8], int split, float mA,
+                                          const PieceParams& A, float mB, const PieceParams& B,
+                                          float Lf, int Li, uint32_t sign_unit, int sign_shift,
+                                          uint32_t& w0, uint32_t& w1, uint32_t& mb, float (&yv)[8]) {
+    w0 = w1 = mb = 0;
+#pragma unroll
+    for (int t = 0; t < 8; ++t) {
+        const bool second = TWO && t >= split;
+        const float m = second ? mB : mA;
+        const float p = second ? B.p : A.p;
+        const float inv1 = second ? B.inv1 : A.inv1;
+        const float inv2 = second ? B.inv2 : A.inv2;
+        const float xi = xv[t];
+        const float a = fminf(fabsf(xi), m);
+        const bool tail = a > p;
+        const float z = tail ? p : 0.0f;
+        const float inv = tail ? inv2 : inv1;
+        const float r = __fadd_rn(__fmul_rn(__fsub_rn(a, z), inv), 12582912.0f);
+        const uint32_t q = (uint32_t)min(__float_as_int(r) - 0x4B400000, Li);
+        const uint32_t xs0 = __float_as_uint(__fadd_rn(xi, 0.0f));   // sign bit = (x < 0)
+        const uint32_t code = ((xs0 >> sign_shift) & sign_unit) | q;
+        if (PACKED) w0 += code << (4 * t);
+        else if (t < 4) w0 += code << (8 * t);
+        else w1 += code << (8 * (t - 4));
+        mb += tail ? (1u << t) : 0u;
+        if (WANT_FAKE) {
+            const float s1 = second ? B.s1 : A.s1;
+            const float s2 = second ? B.s2 : A.s2;
+            const float s = tail ? s2 : s1;
+            const float qf = fminf(__fsub_rn(r, 12582912.0f), Lf);
+            const float v = __fadd_rn(__fmul_rn(qf, s), z);
+            yv[t] = __uint_as_float(__float_as_uint(v) | (xs0 & 0x80000000u));
+        }
+    }
+}
+
+// Persistent CTAs.  TABLE (ragged rows, or dense rows shorter than a span): each CTA walks a block
+// of consecutive spans, so the next span's first row is the row this span ends in and its row
+// table can be requested without a search.  Otherwise every gridDim.x-th span.  The values of
+// the next spans are already on their way into a ring of shared-memory slots (bulk asynchronous
+// copies) while the current span is quantized.
+//
+// A warp's 256 values of one pass are handled by one of three warp-uniform variants: all lanes
+// have their eight values inside one row; some lanes have them in two rows (per-value selects
+// between the two rows' constants); anything else (the tensor's tail, rows with m = 0, more than
+// two rows in eight values) takes the per-value path.
+template <bool PACKED, bool WANT_FAKE, bool TABLE>
 __global__ void __launch_bounds__(kQThreads)
 quantize_kernel(const float* __restrict__ x, Rows rows, int64_t total, int bits,
                 const float* __restrict__ m_arr, const float* __restrict__ p_arr,
                 uint8_t* __restrict__ codes, uint8_t* __restrict__ mask, float* __restrict__ fake,
-                int vec_in, int vec_fake, int vec_codes) {
+                int vec_in, int vec_fake, int vec_codes, int64_t spans_per_cta) {
     extern __shared__ __align__(128) unsigned char smem_raw[];
     QuantizeSmem& Q = *reinterpret_cast<QuantizeSmem*>(smem_raw);
     QuantSmem& S = Q.rows;
     __shared__ int s_abort;
+    const unsigned full = 0xffffffffu;
     const float Lf = (float)((1 << (bits - 1)) - 1);
     const int Li = (1 << (bits - 1)) - 1;
     const uint32_t sign_unit = 1u << (bits - 1);      // value of the sign bit inside a code
     const int sign_shift = 32 - bits;                 // moves bit 31 onto the code's sign bit
     const int64_t nspans = (total + kQSpan - 1) / kQSpan;
-    // The CTA's spans: ragged rows -> a block of consecutive spans (the next span's first row is
-    // then the row this span ends in, so its table can be requested without a search); dense rows
-    // -> every gridDim.x-th span.
-    const int64_t first = RAGGED ? nspans * blockIdx.x / gridDim.x : blockIdx.x;
-    const int64_t stride = RAGGED ? 1 : gridDim.x;
-    const int64_t last = RAGGED ? nspans * (blockIdx.x + 1) / gridDim.x : nspans;   // exclusive
+    const int64_t first = TABLE ? blockIdx.x * spans_per_cta : blockIdx.x;
+    const int64_t stride = TABLE ? 1 : gridDim.x;
+    const int64_t last = TABLE ? min(first + spans_per_cta, nspans) : nspans;        // exclusive
     if (threadIdx.x == 0) s_abort = 0;
     Q.ring.init();
     for (int it = 0; it < kQStages; ++it) {
@@ -103,21 +187,22 @@ quantize_kernel(const float* __restrict__ x, Rows rows, int64_t total, int bits,
         if (span < last) Q.ring.issue(it, x + span * kQSpan, q_bulk_bytes(span, total, vec_in));
     }
     int64_t row0 = 0;                               // first staged row of the current span
-    RowFetch nf;
-    if (RAGGED && first < last) {
-        row0 = warp_row_of(rows, first * kQSpan);   // every warp finds the same row
+    QuantFetch nf;
+    if (TABLE && first < last) {
+        row0 = cta_row_near(rows, first * kQSpan);
         S.fetch(rows, m_arr, p_arr, row0, nf);
-        S.commit(nf, min((first + 1) * kQSpan, total), Lf);
+        S.commit(nf, Lf);
         __syncthreads();
     }
-    RowState rs;                                    // survives from span to span
+    RowState ws;                                    // the row a warp's pass starts in (warp-uniform)
     int64_t it = 0;
     for (int64_t span = first; span < last; span += stride, ++it) {
         const int64_t span_beg = span * kQSpan;
         const int64_t span_end = min(span_beg + kQSpan, total);
-        // ragged rows: request the next span's table now, write it when this span is done
+        // the staged rows end before the next span does: request the window that starts in the
+        // row in which this span ends now, write it when this span is done
         int64_t next_row0 = 0;
-        const bool has_next = RAGGED && span + 1 < last;
+        const bool has_next = TABLE && span + 1 < last && !S.covers(min(span_end + kQSpan, total));
         if (has_next) {
             const int l = S.find(span_end);
             next_row0 = (l >= 0) ? row0 + l : warp_row_of(rows, span_end);
@@ -131,114 +216,119 @@ quantize_kernel(const float* __restrict__ x, Rows rows, int64_t total, int bits,
                 xs[i] = x[span_beg + i];
             __syncthreads();
         }
-#pragma unroll
+#pragma unroll 1
         for (int c = 0; c < kQChunks; ++c) {
-            const int li = c * kQChunk + (int)threadIdx.x * 8;
+            const int li = chunk_offset(c);
             const int64_t i0 = span_beg + li;
             const int cnt = (int)max((int64_t)0, min((int64_t)8, total - i0));
-            if (cnt == 0) continue;
             const float4 xa = *reinterpret_cast<const float4*>(xs + li);
             const float4 xb = *reinterpret_cast<const float4*>(xs + li + 4);
             const float xv[8] = {xa.x, xa.y, xa.z, xa.w, xb.x, xb.y, xb.z, xb.w};
-            uint32_t code[8];
+            uint32_t w0 = 0, w1 = 0, mb = 0;
             float yv[8];
-            uint32_t mbyte = 0;
-            rs.seek(S, rows, m_arr, p_arr, Lf, i0);
-            if (cnt == 8 && i0 + 8 <= rs.end) {
-                // all eight values in one row: the sequence of quantize_mag with the per-row
-                // tests hoisted, the level taken from the mantissa of t + 1.5 * 2^23, and the sign
-                // flag (x < 0, false for -0.0) read off the sign bit of x + 0.0
-                // Codes are packed and region bits gathered on the fly (no per-value branch).
-                const float m = rs.m;
-                const PieceParams P = rs.P;
-                uint32_t w0 = 0, w1 = 0, mb = 0;       // packed codes (w1: upper four, byte layout)
-                if (m > 0.0f) {
-#pragma unroll
-                    for (int t = 0; t < 8; ++t) {
-                        const float xi = xv[t];
-                        const float a = fminf(fabsf(xi), m);
-                        const bool tail = a > P.p;
-                        const float z = tail ? P.p : 0.0f;
-                        const float inv = tail ? P.inv2 : P.inv1;
-                        const float r = __fadd_rn(__fmul_rn(__fsub_rn(a, z), inv), 12582912.0f);
-                        const uint32_t q = (uint32_t)min(__float_as_int(r) - 0x4B400000, Li);
-                        const uint32_t xs0 = __float_as_uint(__fadd_rn(xi, 0.0f));   // sign bit = (x < 0)
-                        const uint32_t code = ((xs0 >> sign_shift) & sign_unit) | q;
-                        if (PACKED) w0 += code << (4 * t);
-                        else if (t < 4) w0 += code << (8 * t);
-                        else w1 += code << (8 * (t - 4));
-                        mb += tail ? (1u << t) : 0u;
-                        if (WANT_FAKE) {
-                            const float s = tail ? P.s2 : P.s1;
-                            const float qf = fminf(__fsub_rn(r, 12582912.0f), Lf);
-                            const float v = __fadd_rn(__fmul_rn(qf, s), z);
-                            yv[t] = __uint_as_float(__float_as_uint(v) | (xs0 & 0x80000000u));
-                        }
-                    }
-                } else if (WANT_FAKE) {
-#pragma unroll
-                    for (int t = 0; t < 8; ++t) yv[t] = 0.0f;
-                }
-                mask[i0 >> 3] = (uint8_t)mb;
-                if (PACKED) {
-                    uint8_t* dst = codes + (i0 >> 1);
-                    if (vec_codes) *reinterpret_cast<uint32_t*>(dst) = w0;
-                    else for (int b = 0; b < 4; ++b) dst[b] = (uint8_t)(w0 >> (8 * b));
-                } else {
-                    uint8_t* dst = codes + i0;
-                    if (vec_codes) *reinterpret_cast<uint2*>(dst) = make_uint2(w0, w1);
-                    else for (int b = 0; b < 8; ++b) dst[b] = (uint8_t)((b < 4 ? w0 : w1) >> (8 * (b & 3)));
-                }
-                if (WANT_FAKE) {
-                    if (vec_fake) {
-                        __stcs(reinterpret_cast<float4*>(fake + i0), make_float4(yv[0], yv[1], yv[2], yv[3]));
-                        __stcs(reinterpret_cast<float4*>(fake + i0 + 4), make_float4(yv[4], yv[5], yv[6], yv[7]));
+            // Warp-uniform part: the pass starts in row A (kept in ws from pass to pass); if the
+            // row ends inside the pass, row B follows and must reach to the end of the pass.
+            const int64_t pass_beg = i0 - ((int)threadIdx.x & 31) * 8, pass_end = pass_beg + 256;
+            bool done = false;
+            if (pass_end <= total) {
+                ws.seek<TABLE>(S, rows, m_arr, p_arr, Lf, pass_beg);
+                if (ws.m > 0.0f) {
+                    if (ws.end >= pass_end) {
+                        quantize8<PACKED, WANT_FAKE, false>(xv, 8, ws.m, ws.P, ws.m, ws.P, Lf, Li,
+                                                            sign_unit, sign_shift, w0, w1, mb, yv);
+                        done = true;
                     } else {
-                        for (int t = 0; t < 8; ++t) fake[i0 + t] = yv[t];
-                    }
-                }
-                continue;
-            } else {
-#pragma unroll
-                for (int t = 0; t < 8; ++t) {
-                    code[t] = 0;
-                    yv[t] = 0.0f;
-                    if (t < cnt) {
-                        rs.seek(S, rows, m_arr, p_arr, Lf, i0 + t);
-                        if (rs.m > 0.0f) {
-                            const float xi = xv[t];
-                            const int neg = xi < 0.0f;
-                            int q, tail;
-                            float v;
-                            quantize_mag(fminf(fabsf(xi), rs.m), rs.P, Lf, q, tail, v);
-                            code[t] = (uint32_t)((neg << (bits - 1)) | q);
-                            mbyte |= (uint32_t)tail << t;
-                            yv[t] = neg ? -v : v;
+                        float mB = 0.0f;
+                        PieceParams PB = ws.P;
+                        int64_t endB = 0;
+                        if (ws.next_row<TABLE>(S, rows, m_arr, p_arr, Lf, pass_end, mB, PB, endB) &&
+                            mB > 0.0f) {
+                            const int split = (int)max((int64_t)0, min((int64_t)8, ws.end - i0));
+                            if (__any_sync(full, split > 0 && split < 8)) {   // a lane holds both rows
+                                quantize8<PACKED, WANT_FAKE, true>(xv, split, ws.m, ws.P, mB, PB, Lf,
+                                                                   Li, sign_unit, sign_shift, w0, w1,
+                                                                   mb, yv);
+                            } else {
+                                const bool second = split == 0;
+                                PieceParams PL;
+                                PL.p = second ? PB.p : ws.P.p;
+                                PL.s1 = second ? PB.s1 : ws.P.s1;
+                                PL.inv1 = second ? PB.inv1 : ws.P.inv1;
+                                PL.s2 = second ? PB.s2 : ws.P.s2;
+                                PL.inv2 = second ? PB.inv2 : ws.P.inv2;
+                                const float mL = second ? mB : ws.m;
+                                quantize8<PACKED, WANT_FAKE, false>(xv, 8, mL, PL, mL, PL, Lf, Li,
+                                                                    sign_unit, sign_shift, w0, w1,
+                                                                    mb, yv);
+                            }
+                            ws.advance(mB, PB, endB);
+                            done = true;
                         }
                     }
                 }
             }
-            mask[i0 >> 3] = (uint8_t)mbyte;
+            if (!done) {
+                // Per-thread part (short rows, rows with m = 0, the tensor's tail): every lane
+                // looks up its own row; lanes whose eight values lie in two rows select between
+                // the two rows' constants per value; anything else takes the per-value path.
+                RowState rs;
+                int split = 8;
+                bool simple = true, two = false;
+                float mB = 0.0f;
+                PieceParams PB = ws.P;
+                int64_t endB = 0;
+                if (cnt > 0) {
+                    rs.seek<TABLE>(S, rows, m_arr, p_arr, Lf, i0);
+                    split = (int)min((int64_t)8, rs.end - i0);
+                    simple = cnt == 8 && split == 8 && rs.m > 0.0f;
+                    if (cnt == 8 && split < 8 && rs.m > 0.0f)
+                        two = rs.next_row<TABLE>(S, rows, m_arr, p_arr, Lf, i0 + 8, mB, PB, endB) &&
+                              mB > 0.0f;
+                }
+                if (__all_sync(full, simple || two)) {
+                    if (!two) { mB = rs.m; PB = rs.P; split = 8; }
+                    quantize8<PACKED, WANT_FAKE, true>(xv, split, rs.m, rs.P, mB, PB, Lf, Li,
+                                                       sign_unit, sign_shift, w0, w1, mb, yv);
+                } else {
+#pragma unroll
+                    for (int t = 0; t < 8; ++t) {
+                        yv[t] = 0.0f;
+                        if (t < cnt) {
+                            rs.seek<TABLE>(S, rows, m_arr, p_arr, Lf, i0 + t);
+                            if (rs.m > 0.0f) {
+                                const float xi = xv[t];
+                                const int neg = xi < 0.0f;
+                                int q, tail;
+                                float v;
+                                quantize_mag(fminf(fabsf(xi), rs.m), rs.P, Lf, q, tail, v);
+                                const uint32_t code = (uint32_t)((neg << (bits - 1)) | q);
+                                if (PACKED) w0 |= code << (4 * t);
+                                else if (t < 4) w0 |= code << (8 * t);
+                                else w1 |= code << (8 * (t - 4));
+                                mb |= (uint32_t)tail << t;
+                                yv[t] = neg ? -v : v;
+                            }
+                        }
+                    }
+                }
+            }
+            if (cnt == 0) continue;
+            mask[i0 >> 3] = (uint8_t)mb;
             if (PACKED) {
-                const uint32_t w = code[0] | (code[1] << 4) | (code[2] << 8) | (code[3] << 12) |
-                                   (code[4] << 16) | (code[5] << 20) | (code[6] << 24) |
-                                   (code[7] << 28);
                 uint8_t* dst = codes + (i0 >> 1);
                 if (vec_codes && cnt == 8) {
-                    *reinterpret_cast<uint32_t*>(dst) = w;
+                    *reinterpret_cast<uint32_t*>(dst) = w0;
                 } else {
                     const int nb = (cnt + 1) >> 1;
-                    for (int b = 0; b < nb; ++b) dst[b] = (uint8_t)(w >> (8 * b));
+                    for (int b = 0; b < nb; ++b) dst[b] = (uint8_t)(w0 >> (8 * b));
                 }
             } else {
                 uint8_t* dst = codes + i0;
                 if (vec_codes && cnt == 8) {
-                    uint2 w;
-                    w.x = code[0] | (code[1] << 8) | (code[2] << 16) | (code[3] << 24);
-                    w.y = code[4] | (code[5] << 8) | (code[6] << 16) | (code[7] << 24);
-                    *reinterpret_cast<uint2*>(dst) = w;
+                    *reinterpret_cast<uint2*>(dst) = make_uint2(w0, w1);
                 } else {
-                    for (int t = 0; t < cnt; ++t) dst[t] = (uint8_t)code[t];
+                    for (int t = 0; t < cnt; ++t)
+                        dst[t] = (uint8_t)((t < 4 ? w0 : w1) >> (8 * (t & 3)));
                 }
             }
             if (WANT_FAKE) {
@@ -255,15 +345,15 @@ quantize_kernel(const float* __restrict__ x, Rows rows, int64_t total, int bits,
             if (threadIdx.x == 0) atomicExch(&g_quantize_timeout, 1);
             return;
         }
-        if (has_next) {
-            S.commit(nf, min(span_end + kQSpan, total), Lf);
-            row0 = next_row0;
-            rs.beg = rs.end = 0;                     // staged constants are per span
-        }
         const int64_t ahead = span + (int64_t)kQStages * stride;
         if (ahead < last)
             Q.ring.issue(it + kQStages, x + ahead * kQSpan, q_bulk_bytes(ahead, total, vec_in));
-        if (RAGGED) __syncthreads();                // the next table is published
+        if (has_next) {
+            S.commit(nf, Lf);
+            row0 = next_row0;
+            ws.beg = ws.end = 0;                     // indices into the window are stale
+            __syncthreads();                        // the next window is published
+        }
     }
 }
 
@@ -276,7 +366,7 @@ struct CodeRegs {
                                          int64_t total, int vec_codes) {
 #pragma unroll
         for (int c = 0; c < kQChunks; ++c) {
-            const int64_t i0 = span_beg + (int64_t)c * kQChunk + (int64_t)threadIdx.x * 8;
+            const int64_t i0 = span_beg + chunk_offset(c);
             const int cnt = (int)max((int64_t)0, min((int64_t)8, total - i0));
             w0[c] = w1[c] = mb[c] = 0;
             if (cnt == 0) continue;
@@ -303,36 +393,61 @@ struct CodeRegs {
             mb[c] = mask[i0 >> 3];
         }
     }
-    __device__ __forceinline__ uint32_t code(int c, int t) const {
-        if (PACKED) return (w0[c] >> (4 * t)) & 0xFu;
-        return ((t < 4 ? w0[c] : w1[c]) >> (8 * (t & 3))) & 0xFFu;
-    }
 };
 
-template <bool PACKED, bool RAGGED>
+template <bool PACKED>
+__device__ __forceinline__ uint32_t code_of(uint32_t w0, uint32_t w1, int t) {
+    if (PACKED) return (w0 >> (4 * t)) & 0xFu;
+    return ((t < 4 ? w0 : w1) >> (8 * (t & 3))) & 0xFFu;
+}
+
+// Eight consecutive codes, the first `split` of them in row A and the rest in row B (TWO = false:
+// all in row A), both rows with m > 0.  The level becomes a float through the mantissa of
+// 1.5 * 2^23 (exact for q < 2^22) instead of an integer conversion.
+template <bool PACKED, bool TWO>
+__device__ __forceinline__ void dequantize8(uint32_t w0, uint32_t w1, uint32_t mb, int split,
+                                            const PieceParams& A, const PieceParams& B, int qmask,
+                                            int sign_shift, float (&yv)[8]) {
+#pragma unroll
+    for (int t = 0; t < 8; ++t) {
+        const bool second = TWO && t >= split;
+        const float p = second ? B.p : A.p;
+        const float s1 = second ? B.s1 : A.s1;
+        const float s2 = second ? B.s2 : A.s2;
+        const uint32_t code = code_of<PACKED>(w0, w1, t);
+        const bool tail = (mb & (1u << t)) != 0;
+        const float q = __fsub_rn(__uint_as_float(0x4B400000u | (code & (uint32_t)qmask)), 12582912.0f);
+        const float v = __fadd_rn(__fmul_rn(q, tail ? s2 : s1), tail ? p : 0.0f);
+        // the code's sign bit moved to bit 31
+        yv[t] = __uint_as_float(__float_as_uint(v) | ((code << sign_shift) & 0x80000000u));
+    }
+}
+
+template <bool PACKED, bool TABLE>
 __global__ void __launch_bounds__(kQThreads)
 dequantize_kernel(const uint8_t* __restrict__ codes, const uint8_t* __restrict__ mask, Rows rows,
                   int64_t total, int bits, const float* __restrict__ m_arr,
                   const float* __restrict__ p_arr, float* __restrict__ y, int vec_codes,
-                  int vec_out) {
+                  int vec_out, int64_t spans_per_cta) {
     __shared__ QuantSmem S;
+    const unsigned full = 0xffffffffu;
     const float Lf = (float)((1 << (bits - 1)) - 1);
     const int qmask = (1 << (bits - 1)) - 1;
     const int sign_shift = 32 - bits;                 // moves a code's sign bit to bit 31
     const int64_t nspans = (total + kQSpan - 1) / kQSpan;
-    // the CTA's spans: consecutive for ragged rows (chained row tables), strided for dense rows
-    const int64_t first = RAGGED ? nspans * blockIdx.x / gridDim.x : blockIdx.x;
-    const int64_t stride = RAGGED ? 1 : gridDim.x;
-    const int64_t last = RAGGED ? nspans * (blockIdx.x + 1) / gridDim.x : nspans;   // exclusive
+    // the CTA's spans: consecutive with a row table (chained tables), strided otherwise
+    const int64_t first = TABLE ? blockIdx.x * spans_per_cta : blockIdx.x;
+    const int64_t stride = TABLE ? 1 : gridDim.x;
+    const int64_t last = TABLE ? min(first + spans_per_cta, nspans) : nspans;        // exclusive
     CodeRegs<PACKED> cur, nxt;
-    RowState rs;                                    // survives from span to span
+    RowState ws;                                    // the row a warp's pass starts in (warp-uniform)
     cur.load(codes, mask, first * kQSpan, total, vec_codes);
     int64_t row0 = 0;                               // first staged row of the current span
-    RowFetch nf;
-    if (RAGGED && first < last) {
-        row0 = warp_row_of(rows, first * kQSpan);
+    QuantFetch nf;
+    if (TABLE && first < last) {
+        row0 = cta_row_near(rows, first * kQSpan);
         S.fetch(rows, m_arr, p_arr, row0, nf);
-        S.commit(nf, min((first + 1) * kQSpan, total), Lf);
+        S.commit(nf, Lf);
         __syncthreads();
     }
     for (int64_t span = first; span < last; span += stride) {
@@ -340,7 +455,7 @@ dequantize_kernel(const uint8_t* __restrict__ codes, const uint8_t* __restrict__
         const int64_t span_end = min(span_beg + kQSpan, total);
         if (span + stride < last) nxt.load(codes, mask, (span + stride) * kQSpan, total, vec_codes);
         int64_t next_row0 = 0;
-        const bool has_next = RAGGED && span + 1 < last;
+        const bool has_next = TABLE && span + 1 < last && !S.covers(min(span_end + kQSpan, total));
         if (has_next) {
             const int l = S.find(span_end);
             next_row0 = (l >= 0) ? row0 + l : warp_row_of(rows, span_end);
@@ -348,50 +463,86 @@ dequantize_kernel(const uint8_t* __restrict__ codes, const uint8_t* __restrict__
         }
 #pragma unroll
         for (int c = 0; c < kQChunks; ++c) {
-            const int64_t i0 = span_beg + (int64_t)c * kQChunk + (int64_t)threadIdx.x * 8;
+            const int64_t i0 = span_beg + chunk_offset(c);
             const int cnt = (int)max((int64_t)0, min((int64_t)8, total - i0));
-            if (cnt == 0) continue;
             float yv[8];
-            rs.seek(S, rows, m_arr, p_arr, Lf, i0);
-            if (cnt == 8 && i0 + 8 <= rs.end) {
-                // all eight values in one row; the level becomes a float through the mantissa of
-                // 1.5 * 2^23 (exact for q < 2^22) instead of an integer conversion
-                const PieceParams P = rs.P;
-#pragma unroll
-                for (int t = 0; t < 8; ++t) yv[t] = 0.0f;
-                if (rs.m > 0.0f) {                     // one test per chunk; no branch per value
-                    const uint32_t mb = cur.mb[c];
-#pragma unroll
-                    for (int t = 0; t < 8; ++t) {
-                        const uint32_t code = cur.code(c, t);
-                        const bool tail = (mb & (1u << t)) != 0;
-                        const float q = __fsub_rn(__uint_as_float(0x4B400000u | (code & (uint32_t)qmask)),
-                                                  12582912.0f);
-                        const float v = __fadd_rn(__fmul_rn(q, tail ? P.s2 : P.s1), tail ? P.p : 0.0f);
-                        // the code's sign bit moved to bit 31
-                        yv[t] = __uint_as_float(__float_as_uint(v) | ((code << sign_shift) & 0x80000000u));
-                    }
-                }
-            } else {
-#pragma unroll
-                for (int t = 0; t < 8; ++t) {
-                    yv[t] = 0.0f;
-                    if (t < cnt) {
-                        rs.seek(S, rows, m_arr, p_arr, Lf, i0 + t);
-                        if (rs.m > 0.0f) {
-                            const uint32_t code = cur.code(c, t);
-                            const int tail = (cur.mb[c] >> t) & 1;
-                            const int neg = (code >> (bits - 1)) & 1;
-                            const float q = (float)(code & qmask);
-                            const float s = tail ? rs.P.s2 : rs.P.s1;
-                            const float z = tail ? rs.P.p : 0.0f;
-                            float v = __fmul_rn(q, s);
-                            v = __fadd_rn(v, z);
-                            yv[t] = neg ? -v : v;
+            // warp-uniform part and per-thread part as in quantize_kernel
+            const int64_t pass_beg = i0 - ((int)threadIdx.x & 31) * 8, pass_end = pass_beg + 256;
+            bool done = false;
+            if (pass_end <= total) {
+                ws.seek<TABLE>(S, rows, m_arr, p_arr, Lf, pass_beg);
+                if (ws.m > 0.0f) {
+                    if (ws.end >= pass_end) {
+                        dequantize8<PACKED, false>(cur.w0[c], cur.w1[c], cur.mb[c], 8, ws.P, ws.P,
+                                                   qmask, sign_shift, yv);
+                        done = true;
+                    } else {
+                        float mB = 0.0f;
+                        PieceParams PB = ws.P;
+                        int64_t endB = 0;
+                        if (ws.next_row<TABLE>(S, rows, m_arr, p_arr, Lf, pass_end, mB, PB, endB) &&
+                            mB > 0.0f) {
+                            const int split = (int)max((int64_t)0, min((int64_t)8, ws.end - i0));
+                            if (__any_sync(full, split > 0 && split < 8)) {   // a lane holds both rows
+                                dequantize8<PACKED, true>(cur.w0[c], cur.w1[c], cur.mb[c], split,
+                                                          ws.P, PB, qmask, sign_shift, yv);
+                            } else {
+                                const bool second = split == 0;
+                                PieceParams PL;
+                                PL.p = second ? PB.p : ws.P.p;
+                                PL.s1 = second ? PB.s1 : ws.P.s1;
+                                PL.s2 = second ? PB.s2 : ws.P.s2;
+                                PL.inv1 = PL.inv2 = 0.0f;
+                                dequantize8<PACKED, false>(cur.w0[c], cur.w1[c], cur.mb[c], 8, PL, PL,
+                                                           qmask, sign_shift, yv);
+                            }
+                            ws.advance(mB, PB, endB);
+                            done = true;
                         }
                     }
                 }
             }
+            if (!done) {
+                RowState rs;
+                int split = 8;
+                bool simple = true, two = false;
+                float mB = 0.0f;
+                PieceParams PB = ws.P;
+                int64_t endB = 0;
+                if (cnt > 0) {
+                    rs.seek<TABLE>(S, rows, m_arr, p_arr, Lf, i0);
+                    split = (int)min((int64_t)8, rs.end - i0);
+                    simple = cnt == 8 && split == 8 && rs.m > 0.0f;
+                    if (cnt == 8 && split < 8 && rs.m > 0.0f)
+                        two = rs.next_row<TABLE>(S, rows, m_arr, p_arr, Lf, i0 + 8, mB, PB, endB) &&
+                              mB > 0.0f;
+                }
+                if (__all_sync(full, simple || two)) {
+                    if (!two) { PB = rs.P; split = 8; }
+                    dequantize8<PACKED, true>(cur.w0[c], cur.w1[c], cur.mb[c], split, rs.P, PB, qmask,
+                                              sign_shift, yv);
+                } else {
+#pragma unroll
+                    for (int t = 0; t < 8; ++t) {
+                        yv[t] = 0.0f;
+                        if (t < cnt) {
+                            rs.seek<TABLE>(S, rows, m_arr, p_arr, Lf, i0 + t);
+                            if (rs.m > 0.0f) {
+                                const uint32_t code = code_of<PACKED>(cur.w0[c], cur.w1[c], t);
+                                const int tail = (cur.mb[c] >> t) & 1;
+                                const int neg = (code >> (bits - 1)) & 1;
+                                const float q = (float)(code & qmask);
+                                const float s = tail ? rs.P.s2 : rs.P.s1;
+                                const float z = tail ? rs.P.p : 0.0f;
+                                float v = __fmul_rn(q, s);
+                                v = __fadd_rn(v, z);
+                                yv[t] = neg ? -v : v;
+                            }
+                        }
+                    }
+                }
+            }
+            if (cnt == 0) continue;
             if (vec_out && cnt == 8) {
                 __stcs(reinterpret_cast<float4*>(y + i0), make_float4(yv[0], yv[1], yv[2], yv[3]));
                 __stcs(reinterpret_cast<float4*>(y + i0 + 4), make_float4(yv[4], yv[5], yv[6], yv[7]));
@@ -399,14 +550,12 @@ dequantize_kernel(const uint8_t* __restrict__ codes, const uint8_t* __restrict__
                 for (int t = 0; t < cnt; ++t) y[i0 + t] = yv[t];
             }
         }
-        if (RAGGED) {
-            __syncthreads();                        // the row table is no longer read
-            if (has_next) {
-                S.commit(nf, min(span_end + kQSpan, total), Lf);
-                row0 = next_row0;
-                rs.beg = rs.end = 0;
-            }
-            __syncthreads();                        // the next table is published
+        if (has_next) {
+            __syncthreads();                        // the window is no longer read
+            S.commit(nf, Lf);
+            row0 = next_row0;
+            ws.beg = ws.end = 0;                     // indices into the window are stale
+            __syncthreads();                        // the next window is published
         }
         cur = nxt;
     }
@@ -416,9 +565,9 @@ static inline bool aligned(const void* p, size_t a) {
     return (reinterpret_cast<uintptr_t>(p) & (a - 1)) == 0;
 }
 
-// CTAs that fit the device at once: the persistent grid.  Looked up once per (kernel, device);
-// the first lookup also opts the kernel in to its dynamic shared memory size.
-static unsigned persistent_grid(const void* kernel, int threads, size_t smem, int64_t nspans) {
+// CTAs of `kernel` that fit the device at once.  Looked up once per (kernel, device); the first
+// lookup also opts the kernel in to its dynamic shared memory size.
+static int64_t device_slots(const void* kernel, int threads, size_t smem) {
     struct Entry { const void* kernel; int dev; int ctas; };
     static Entry table[64];
     static int used = 0;
@@ -426,21 +575,32 @@ static unsigned persistent_grid(const void* kernel, int threads, size_t smem, in
     int dev = 0;
     cudaGetDevice(&dev);
     int ctas = 0;
-    {
-        std::lock_guard<std::mutex> lock(mu);
-        for (int i = 0; i < used; ++i)
-            if (table[i].kernel == kernel && table[i].dev == dev) ctas = table[i].ctas;
-        if (ctas == 0) {
-            if (smem > 0)
-                cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-            int sms = 0, per_sm = 0;
-            cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-            cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kernel, threads, smem);
-            ctas = (sms > 0 && per_sm > 0) ? sms * per_sm : 148;
-            if (used < 64) table[used++] = Entry{kernel, dev, ctas};
-        }
+    std::lock_guard<std::mutex> lock(mu);
+    for (int i = 0; i < used; ++i)
+        if (table[i].kernel == kernel && table[i].dev == dev) ctas = table[i].ctas;
+    if (ctas == 0) {
+        if (smem > 0)
+            cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        int sms = 0, per_sm = 0;
+        cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+        cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kernel, threads, smem);
+        ctas = (sms > 0 && per_sm > 0) ? sms * per_sm : 148;
+        if (used < 64) table[used++] = Entry{kernel, dev, ctas};
     }
-    return (unsigned)(nspans < ctas ? nspans : ctas);
+    return ctas;
+}
+
+// Grid and spans per CTA.  Without a row table (long dense rows) the cost per span is the same
+// everywhere: a persistent grid, one CTA per slot, walks the spans with a stride.  With a row
+// table the cost per span depends on the row lengths, so consecutive spans are handed out in
+// small blocks (about four per slot) and the hardware scheduler balances them.
+struct SpanGrid { unsigned grid; int64_t per_cta; };
+static SpanGrid span_grid(const void* kernel, int threads, size_t smem, int64_t nspans, bool table) {
+    const int64_t slots = device_slots(kernel, threads, smem);
+    if (!table) return SpanGrid{(unsigned)std::min(nspans, slots), 0};
+    const int64_t per_cta =
+        std::min<int64_t>(std::max<int64_t>((nspans + 4 * slots - 1) / (4 * slots), 4), 32);
+    return SpanGrid{(unsigned)((nspans + per_cta - 1) / per_cta), per_cta};
 }
 
 int quantize_timeout_flag() {
@@ -460,14 +620,17 @@ cudaError_t launch_quantize(const float* x, const int64_t* row_offsets, int64_t 
     const int vec_in = aligned(x, 16), vec_fake = fake ? aligned(fake, 16) : 0;
     const size_t smem = sizeof(QuantizeSmem);
     const int vec_codes = packed ? aligned(codes, 4) : aligned(codes, 8);
+    const bool table = row_offsets != nullptr || n < kQSpan;    // several rows per span
 #define PWLQ_LAUNCH_QUANTIZE(PK, FK, RG)                                                          \
-    quantize_kernel<PK, FK, RG><<<persistent_grid((const void*)quantize_kernel<PK, FK, RG>,       \
-                                                  kQThreads, smem, nspans),                       \
-                                  kQThreads, smem, stream>>>(x, rows, total, bits, m, p, codes,   \
-                                                             mask, fake, vec_in, vec_fake,        \
-                                                             vec_codes)
+    do {                                                                                          \
+        const SpanGrid g = span_grid((const void*)quantize_kernel<PK, FK, RG>, kQThreads, smem,   \
+                                     nspans, RG);                                                 \
+        quantize_kernel<PK, FK, RG><<<g.grid, kQThreads, smem, stream>>>(                         \
+            x, rows, total, bits, m, p, codes, mask, fake, vec_in, vec_fake, vec_codes,           \
+            g.per_cta);                                                                           \
+    } while (0)
 #define PWLQ_LAUNCH_QUANTIZE_RG(PK, FK) \
-    do { if (row_offsets) PWLQ_LAUNCH_QUANTIZE(PK, FK, true); else PWLQ_LAUNCH_QUANTIZE(PK, FK, false); } while (0)
+    do { if (table) PWLQ_LAUNCH_QUANTIZE(PK, FK, true); else PWLQ_LAUNCH_QUANTIZE(PK, FK, false); } while (0)
     if (packed) { if (fake) PWLQ_LAUNCH_QUANTIZE_RG(true, true); else PWLQ_LAUNCH_QUANTIZE_RG(true, false); }
     else        { if (fake) PWLQ_LAUNCH_QUANTIZE_RG(false, true); else PWLQ_LAUNCH_QUANTIZE_RG(false, false); }
 #undef PWLQ_LAUNCH_QUANTIZE_RG
@@ -484,12 +647,16 @@ cudaError_t launch_dequantize(const uint8_t* codes, const uint8_t* mask,
     const bool packed = (layout == 1 && bits <= 4);
     const int64_t nspans = (total + kQSpan - 1) / kQSpan;
 #define PWLQ_LAUNCH_DEQUANTIZE(PK, RG)                                                            \
-    dequantize_kernel<PK, RG><<<persistent_grid((const void*)dequantize_kernel<PK, RG>, kQThreads, \
-                                                0, nspans),                                       \
-                                kQThreads, 0, stream>>>(codes, mask, rows, total, bits, m, p, y,   \
-                                                        aligned(codes, PK ? 4 : 8), aligned(y, 16))
-    if (packed) { if (row_offsets) PWLQ_LAUNCH_DEQUANTIZE(true, true); else PWLQ_LAUNCH_DEQUANTIZE(true, false); }
-    else        { if (row_offsets) PWLQ_LAUNCH_DEQUANTIZE(false, true); else PWLQ_LAUNCH_DEQUANTIZE(false, false); }
+    do {                                                                                          \
+        const SpanGrid g = span_grid((const void*)dequantize_kernel<PK, RG>, kQThreads, 0,        \
+                                     nspans, RG);                                                 \
+        dequantize_kernel<PK, RG><<<g.grid, kQThreads, 0, stream>>>(                              \
+            codes, mask, rows, total, bits, m, p, y, aligned(codes, PK ? 4 : 8), aligned(y, 16),  \
+            g.per_cta);                                                                           \
+    } while (0)
+    const bool table = row_offsets != nullptr || n < kQSpan;    // several rows per span
+    if (packed) { if (table) PWLQ_LAUNCH_DEQUANTIZE(true, true); else PWLQ_LAUNCH_DEQUANTIZE(true, false); }
+    else        { if (table) PWLQ_LAUNCH_DEQUANTIZE(false, true); else PWLQ_LAUNCH_DEQUANTIZE(false, false); }
 #undef PWLQ_LAUNCH_DEQUANTIZE
     return cudaGetLastError();
 }
