@@ -4,5 +4,6 @@ Only the tests, the smoke check and the benchmark's CPU-baseline leg import
 this package.  It shares no code with the CUDA path.
 """
 from .pwlq_oracle import (  # noqa: F401
-    OracleError, OracleLib, absmax, analytic_p, build, code_bytes, dequantize, elem, params, quantize, search, select_analytic,
+    OracleError, OracleLib, absmax, analytic_p, build, code_bytes, dequantize, dequantize_u, elem,
+    elem_u, minmax, params, quantize, quantize_u, search, search_u, select_analytic,
 )

@@ -315,3 +315,173 @@ int pwlq_oracle_select_analytic(const float *x, const int64_t *row_offsets, int6
     }
     return ORACLE_OK;
 }
+
+/* ------------------------------------------------------------------------------------------
+ * One-sided ranges (unsigned tensors such as ReLU activations; asymmetric ranges [m1, m2]).
+ *
+ * Sec. 3.2 (footnote to the range) says the scheme extends to asymmetric ranges [m1, m2], and
+ * Eq. 1 takes the offset z = r_l and the unsigned integer domain {0, ..., 2^b - 1} for one-sided
+ * distributions.  The paper does not spell the piecewise form out; the reading taken here:
+ *   - a row's range [lo, hi] is shifted to [0, m] with m = hi - lo (binary32), its dense end
+ *     being the lower bound (as for ReLU outputs, lo = 0);
+ *   - one breakpoint p splits [0, m] into the center [0, p] and the tail (p, m];
+ *   - no sign is stored, so each of the two pieces keeps the whole b-bit level set:
+ *     N = 2^b levels, s = Delta / (2^b - 1) (Eq. 1 with N = 2^b);
+ *   - a = min(max(x - lo, 0), m) (one binary32 subtraction, then the clamp of Eq. 1), after which
+ *     the steps are those of the positive half of Eq. 3; the delivered value is y = v + lo;
+ *   - the squared error is taken in the shifted domain, (v - a)^2, which for lo = 0 is the
+ *     error of the delivered value itself;
+ *   - a constant row (m = 0) gets code 0 everywhere and y = lo.
+ * The stored integer is the b-bit level q; the region bit is kept separately as before.
+ * With x >= 0 and lo = 0 this is exactly the positive half of the signed scheme at b + 1 bits
+ * (same L = 2^b - 1), which is what the tests pin it to.
+ */
+static pw_params make_params_u(float m, float p, int bits)
+{
+    return make_params(m, p, bits + 1);          /* L = 2^b - 1 */
+}
+
+static float shifted_mag(float x, float lo, float m)
+{
+    float a = x - lo;
+    a = fmaxf(a, 0.0f);
+    return fminf(a, m);
+}
+
+/* Per-row minimum and maximum (the range [m1, m2]); an empty row gets lo = hi = 0. */
+int pwlq_oracle_minmax(const float *x, const int64_t *row_offsets, int64_t C, int64_t n,
+                       float *lo_out, float *hi_out)
+{
+    int64_t c, i;
+    if (!x || !lo_out || !hi_out || C < 1) return ORACLE_ERR_ARG;
+    for (c = 0; c < C; ++c) {
+        int64_t b = row_begin(row_offsets, n, c), e = row_begin(row_offsets, n, c + 1);
+        float lo = 0.0f, hi = 0.0f;
+        for (i = b; i < e; ++i) {
+            if (!(fabsf(x[i]) <= 3.402823466e+38f)) return ORACLE_ERR_NONFINITE;
+            if (i == b || x[i] < lo) lo = x[i];
+            if (i == b || x[i] > hi) hi = x[i];
+        }
+        lo_out[c] = lo;
+        hi_out[c] = hi;
+    }
+    return ORACLE_OK;
+}
+
+/* Grid search of the breakpoint for one-sided ranges: p_k = m * ratios[k], m = hi - lo. */
+int pwlq_oracle_search_u(const float *x, const int64_t *row_offsets, int64_t C, int64_t n,
+                         int bits, const float *ratios, int K, const float *lo_in,
+                         const float *hi_in, float *p_out, float *err_out, int32_t *idx_out,
+                         float *sse_f32, double *sse_f64)
+{
+    int64_t c, i;
+    int k;
+    if (!x || !ratios || !lo_in || !hi_in || C < 1 || K < 1 || bits < 2 || bits > 8)
+        return ORACLE_ERR_ARG;
+    for (c = 0; c < C; ++c) {
+        int64_t b = row_begin(row_offsets, n, c), e = row_begin(row_offsets, n, c + 1);
+        float lo = lo_in[c];
+        float m = hi_in[c] - lo;
+        double best = 0.0;
+        int best_k = 0;
+        if (!(fabsf(m) <= 3.402823466e+38f) || !(fabsf(lo) <= 3.402823466e+38f))
+            return ORACLE_ERR_NONFINITE;
+        for (k = 0; k < K; ++k) {
+            double sse = 0.0;
+            if (m > 0.0f) {
+                float p = m * ratios[k];
+                pw_params P = make_params_u(m, p, bits);
+                for (i = b; i < e; ++i) {
+                    int q, r; float a;
+                    float v = pw_elem(shifted_mag(x[i], lo, m), m, p, &P, &q, &r, &a);
+                    double d = (double)v - (double)a;
+                    sse += d * d;
+                }
+            }
+            if (sse_f32) sse_f32[c * (int64_t)K + k] = (float)sse;
+            if (sse_f64) sse_f64[c * (int64_t)K + k] = sse;
+            if (k == 0 || sse < best) { best = sse; best_k = k; }
+        }
+        if (idx_out) idx_out[c] = best_k;
+        if (p_out)   p_out[c] = (m > 0.0f) ? m * ratios[best_k] : 0.0f;
+        if (err_out) err_out[c] = (float)best;
+    }
+    return ORACLE_OK;
+}
+
+/* One-sided quantizer: b-bit level (no sign), region bit, optional delivered value v + lo.
+ * Code and mask layouts as in pwlq_oracle_quantize. */
+int pwlq_oracle_quantize_u(const float *x, const int64_t *row_offsets, int64_t C, int64_t n,
+                           int bits, const float *lo_in, const float *hi_in, const float *p_in,
+                           uint8_t *codes, uint8_t *region_mask, float *fake_out, int layout)
+{
+    int64_t c, i, total;
+    int packed = (layout == 1 && bits <= 4);
+    if (!x || !lo_in || !hi_in || !p_in || C < 1 || bits < 2 || bits > 8) return ORACLE_ERR_ARG;
+    total = row_begin(row_offsets, n, C);
+    if (codes)       for (i = 0; i < (packed ? (total + 1) / 2 : total); ++i) codes[i] = 0;
+    if (region_mask) for (i = 0; i < (total + 7) / 8; ++i) region_mask[i] = 0;
+    for (c = 0; c < C; ++c) {
+        int64_t b = row_begin(row_offsets, n, c), e = row_begin(row_offsets, n, c + 1);
+        float lo = lo_in[c], p = p_in[c];
+        float m = hi_in[c] - lo;
+        pw_params P = make_params_u(m, p, bits);
+        for (i = b; i < e; ++i) {
+            int q = 0, r = 0;
+            float a, v = 0.0f;
+            if (m > 0.0f) v = pw_elem(shifted_mag(x[i], lo, m), m, p, &P, &q, &r, &a);
+            if (codes) {
+                if (packed) codes[i >> 1] |= (uint8_t)(q << ((i & 1) * 4));
+                else        codes[i] = (uint8_t)q;
+            }
+            if (region_mask && r) region_mask[i >> 3] |= (uint8_t)(1u << (i & 7));
+            if (fake_out) fake_out[i] = v + lo;
+        }
+    }
+    return ORACLE_OK;
+}
+
+/* Inverse of the one-sided quantizer: y = (s * q + z) + lo with (s, z) of the stored region. */
+int pwlq_oracle_dequantize_u(const uint8_t *codes, const uint8_t *region_mask,
+                             const int64_t *row_offsets, int64_t C, int64_t n, int bits,
+                             const float *lo_in, const float *hi_in, const float *p_in, float *y,
+                             int layout)
+{
+    int64_t c, i;
+    int packed = (layout == 1 && bits <= 4);
+    int qmask = (1 << bits) - 1;
+    if (!codes || !region_mask || !lo_in || !hi_in || !p_in || !y || C < 1 || bits < 2 || bits > 8)
+        return ORACLE_ERR_ARG;
+    for (c = 0; c < C; ++c) {
+        int64_t b = row_begin(row_offsets, n, c), e = row_begin(row_offsets, n, c + 1);
+        float lo = lo_in[c], p = p_in[c];
+        float m = hi_in[c] - lo;
+        pw_params P = make_params_u(m, p, bits);
+        for (i = b; i < e; ++i) {
+            int code = packed ? ((codes[i >> 1] >> ((i & 1) * 4)) & 0xF) : codes[i];
+            int r = (region_mask[i >> 3] >> (i & 7)) & 1;
+            float q = (float)(code & qmask);
+            float s = r ? P.s2 : P.s1;
+            float z = r ? p : 0.0f;
+            float v = q * s;
+            v = v + z;
+            if (!(m > 0.0f)) v = 0.0f;
+            y[i] = v + lo;
+        }
+    }
+    return ORACLE_OK;
+}
+
+/* One value of the one-sided quantizer, for hand-checkable tests. */
+void pwlq_oracle_elem_u(float x, float lo, float hi, float p, int bits,
+                        int *code_out, int *region_out, float *y_out)
+{
+    float m = hi - lo;
+    pw_params P = make_params_u(m, p, bits);
+    int q = 0, r = 0;
+    float a, v = 0.0f;
+    if (m > 0.0f) v = pw_elem(shifted_mag(x, lo, m), m, p, &P, &q, &r, &a);
+    *code_out = q;
+    *region_out = r;
+    *y_out = v + lo;
+}

@@ -87,6 +87,16 @@ class OracleLib:
         lib.pwlq_oracle_analytic_p.argtypes = [ctypes.c_double, ctypes.c_double, ctypes.c_int]
         lib.pwlq_oracle_analytic_p.restype = ctypes.c_double
         lib.pwlq_oracle_select_analytic.argtypes = [P, P, I64, I64, P, ctypes.c_int, P, P]
+        lib.pwlq_oracle_minmax.argtypes = [P, P, I64, I64, P, P]
+        lib.pwlq_oracle_search_u.argtypes = [P, P, I64, I64, ctypes.c_int, P, ctypes.c_int, P, P,
+                                             P, P, P, P, P]
+        lib.pwlq_oracle_quantize_u.argtypes = [P, P, I64, I64, ctypes.c_int, P, P, P, P, P, P,
+                                               ctypes.c_int]
+        lib.pwlq_oracle_dequantize_u.argtypes = [P, P, P, I64, I64, ctypes.c_int, P, P, P, P,
+                                                 ctypes.c_int]
+        lib.pwlq_oracle_elem_u.argtypes = [ctypes.c_float, ctypes.c_float, ctypes.c_float,
+                                           ctypes.c_float, ctypes.c_int, P, P, P]
+        lib.pwlq_oracle_elem_u.restype = None
         self._lib = lib
 
     def absmax(self, x, row_offsets=None):
@@ -170,6 +180,76 @@ class OracleLib:
                                    ctypes.byref(region), ctypes.byref(q), ctypes.byref(y))
         return code.value, region.value, q.value, y.value
 
+    # ---- one-sided ranges [lo, hi] (unsigned tensors): b-bit levels, no sign bit
+    def minmax(self, x, row_offsets=None):
+        flat, ro, C, n = _rows(x, row_offsets)
+        lo = np.empty(C, dtype=np.float32)
+        hi = np.empty(C, dtype=np.float32)
+        _check(self._lib.pwlq_oracle_minmax(_ptr(flat), _ptr(ro), C, n, _ptr(lo), _ptr(hi)),
+               "minmax")
+        return lo, hi
+
+    def search_u(self, x, bits, ratios, lo, hi, row_offsets=None, want_sse=True):
+        """Returns dict(p, err, idx, sse (float32 [C,K]), sse64 (float64 [C,K]))."""
+        flat, ro, C, n = _rows(x, row_offsets)
+        ratios = np.ascontiguousarray(ratios, dtype=np.float32)
+        K = int(ratios.size)
+        lo = np.ascontiguousarray(lo, dtype=np.float32)
+        hi = np.ascontiguousarray(hi, dtype=np.float32)
+        assert lo.size == C and hi.size == C
+        p = np.empty(C, dtype=np.float32)
+        err = np.empty(C, dtype=np.float32)
+        idx = np.empty(C, dtype=np.int32)
+        sse = np.empty((C, K), dtype=np.float32) if want_sse else None
+        sse64 = np.empty((C, K), dtype=np.float64) if want_sse else None
+        _check(self._lib.pwlq_oracle_search_u(_ptr(flat), _ptr(ro), C, n, int(bits), _ptr(ratios),
+                                              K, _ptr(lo), _ptr(hi), _ptr(p), _ptr(err),
+                                              _ptr(idx), _ptr(sse), _ptr(sse64)), "search_u")
+        return {"p": p, "err": err, "idx": idx, "sse": sse, "sse64": sse64}
+
+    def quantize_u(self, x, bits, lo, hi, p, layout=0, row_offsets=None, want_fake=True):
+        """Returns (codes uint8, region_mask uint8, fake fp32 or None)."""
+        flat, ro, C, n = _rows(x, row_offsets)
+        total = flat.size
+        lo = np.ascontiguousarray(lo, dtype=np.float32)
+        hi = np.ascontiguousarray(hi, dtype=np.float32)
+        p = np.ascontiguousarray(p, dtype=np.float32)
+        assert lo.size == C and hi.size == C and p.size == C
+        codes = np.empty(code_bytes(total, bits, layout), dtype=np.uint8)
+        mask = np.empty((total + 7) // 8, dtype=np.uint8)
+        fake = np.empty(total, dtype=np.float32) if want_fake else None
+        _check(self._lib.pwlq_oracle_quantize_u(_ptr(flat), _ptr(ro), C, n, int(bits), _ptr(lo),
+                                                _ptr(hi), _ptr(p), _ptr(codes), _ptr(mask),
+                                                _ptr(fake), int(layout)), "quantize_u")
+        return codes, mask, fake
+
+    def dequantize_u(self, codes, mask, bits, lo, hi, p, C=None, n=None, layout=0,
+                     row_offsets=None):
+        codes = np.ascontiguousarray(codes, dtype=np.uint8)
+        mask = np.ascontiguousarray(mask, dtype=np.uint8)
+        lo = np.ascontiguousarray(lo, dtype=np.float32)
+        hi = np.ascontiguousarray(hi, dtype=np.float32)
+        p = np.ascontiguousarray(p, dtype=np.float32)
+        if row_offsets is not None:
+            ro = np.ascontiguousarray(row_offsets, dtype=np.int64)
+            C, n, total = ro.size - 1, 0, int(ro[-1])
+        else:
+            ro, total = None, int(C) * int(n)
+        assert lo.size == C and hi.size == C and p.size == C
+        y = np.empty(total, dtype=np.float32)
+        _check(self._lib.pwlq_oracle_dequantize_u(_ptr(codes), _ptr(mask), _ptr(ro), C, n,
+                                                  int(bits), _ptr(lo), _ptr(hi), _ptr(p),
+                                                  _ptr(y), int(layout)), "dequantize_u")
+        return y
+
+    def elem_u(self, x, lo, hi, p, bits):
+        """One value through the one-sided quantizer: returns (code, region, y)."""
+        code, region = ctypes.c_int(), ctypes.c_int()
+        y = ctypes.c_float()
+        self._lib.pwlq_oracle_elem_u(float(x), float(lo), float(hi), float(p), int(bits),
+                                     ctypes.byref(code), ctypes.byref(region), ctypes.byref(y))
+        return code.value, region.value, y.value
+
     def params(self, m, p, bits):
         """(L, s1, inv1, s2, inv2) as binary32 values."""
         out = np.empty(5, dtype=np.float32)
@@ -217,3 +297,23 @@ def select_analytic(*a, **k):
 
 def params(*a, **k):
     return _get().params(*a, **k)
+
+
+def minmax(*a, **k):
+    return _get().minmax(*a, **k)
+
+
+def search_u(*a, **k):
+    return _get().search_u(*a, **k)
+
+
+def quantize_u(*a, **k):
+    return _get().quantize_u(*a, **k)
+
+
+def dequantize_u(*a, **k):
+    return _get().dequantize_u(*a, **k)
+
+
+def elem_u(*a, **k):
+    return _get().elem_u(*a, **k)

@@ -6,6 +6,7 @@ import subprocess
 import pytest
 
 import test_oracle_pins as pins
+import test_oracle_unsigned_pins as upins
 
 ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
 SRC = os.path.join(ROOT, "oracle", "pwlq_oracle.c")
@@ -42,6 +43,14 @@ MUTANTS = {
     "sigma_without_sqrt": (": sqrt(s2 / (double)(e - b));", ": (s2 / (double)(e - b));"),
     "laplace_cdf_as_gauss_tail": ("return 1.0 - 0.5 * exp(-p / scale);", "return 1.0 - exp(-p / scale);"),
     "approx_constant": ("0.8614 * (m / scale) + 0.6079", "0.8614 * (m / scale) + 0.06079"),
+    "unsigned_levels_as_signed": ("return make_params(m, p, bits + 1);", "return make_params(m, p, bits);"),
+    "unsigned_no_shift": ("    float a = x - lo;\n    a = fmaxf(a, 0.0f);", "    float a = x;\n    a = fmaxf(a, 0.0f);"),
+    "unsigned_no_clamp_below": ("    a = fmaxf(a, 0.0f);", "    a = a + 0.0f;"),
+    "unsigned_offset_not_added": ("if (fake_out) fake_out[i] = v + lo;", "if (fake_out) fake_out[i] = v;"),
+    "unsigned_dequant_offset": ("            y[i] = v + lo;", "            y[i] = v;"),
+    "unsigned_dequant_level_mask": ("int qmask = (1 << bits) - 1;", "int qmask = (1 << (bits - 1)) - 1;"),
+    "minmax_min_is_max": ("if (i == b || x[i] < lo) lo = x[i];", "if (i == b || x[i] > lo) lo = x[i];"),
+    "unsigned_range_is_hi": ("        float m = hi_in[c] - lo;\n        double best = 0.0;", "        float m = hi_in[c];\n        double best = 0.0;"),
     "divide_not_reciprocal_free_pass": None,   # placeholder documented below
 }
 # 'divide_not_reciprocal': evaluating (|r| - z) / s by a true division instead of multiplying by
@@ -63,6 +72,11 @@ PIN_CALLS = [
     lambda o: pins.test_analytic_root_matches_an_independent_solver(o, 1, pins.stats.norm),
     lambda o: pins.test_analytic_root_matches_an_independent_solver(o, 2, pins.stats.laplace),
     lambda o: pins.test_analytic_approximation_and_scales(o),
+    lambda o: upins.test_worked_example_unsigned_b2(o),
+    lambda o: upins.test_minmax_rows(o),
+    lambda o: upins.test_nonnegative_rows_equal_the_signed_scheme_with_one_more_bit(o, 3),
+    lambda o: upins.test_levels_regions_and_half_step_bound_unsigned(o, 4),
+    lambda o: upins.test_bruteforce_true_division_tiny_rows(o, 4, 32),
 ]
 
 
