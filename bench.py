@@ -220,6 +220,8 @@ def run_ours(args, rank, world, local_rank):
         ro = torch.from_numpy(w.row_offsets).to(dev)
     ratios = torch.from_numpy(ratios_np).to(dev)
     m = torch.empty(w.C, dtype=torch.float32, device=dev)
+    lo = torch.empty(w.C, dtype=torch.float32, device=dev)      # one-sided scheme: range [lo, m]
+    unsigned = args.scheme == "unsigned"
     sout = {"p": torch.empty(w.C, dtype=torch.float32, device=dev),
             "err": torch.empty(w.C, dtype=torch.float32, device=dev),
             "idx": torch.empty(w.C, dtype=torch.int32, device=dev), "sse": None}
@@ -233,6 +235,19 @@ def run_ours(args, rank, world, local_rank):
     def step(ev=None):
         """One pass of the whole path; ev = 5 CUDA events to record between the stages."""
         if ev: ev[0].record(stream)
+        if unsigned:
+            pwlq.minmax(x, row_offsets=ro, out=(lo, m))
+            if ev: ev[1].record(stream)
+            pwlq.search_unsigned(x, w.bits, ratios, lo, m, row_offsets=ro, max_n=max_n,
+                                 workspace=ws, out=sout)
+            if ev: ev[2].record(stream)
+            pwlq.quantize_unsigned(x, w.bits, lo, m, sout["p"], layout=layout, row_offsets=ro,
+                                   out=(codes, mask, None))
+            if ev: ev[3].record(stream)
+            pwlq.dequantize_unsigned(codes, mask, w.bits, lo, m, sout["p"], C=w.C, n=dense_n,
+                                     layout=layout, row_offsets=ro, out=y)
+            if ev: ev[4].record(stream)
+            return
         pwlq.absmax(x, row_offsets=ro, out=m)
         if ev: ev[1].record(stream)
         pwlq.search(x, w.bits, ratios, m=m, row_offsets=ro, max_n=max_n, workspace=ws, out=sout)
@@ -300,6 +315,8 @@ def run_ours(args, rank, world, local_rank):
 
     # the end-to-end outputs must equal the resident-path outputs (same kernels, same inputs)
     same = bool(torch.equal(hout["codes"], codes.cpu()) and torch.equal(hout["idx"], sout["idx"].cpu()))
+    if unsigned:
+        same = None          # the host-buffer entry point runs the signed scheme only
 
     # ---- max over ranks
     if dist is not None:
@@ -337,6 +354,7 @@ def run_ours(args, rank, world, local_rank):
             "data": "synthetic",
             "config": {"workload": w.name, "bits": w.bits, "K": w.K, "rows": w.C,
                        "values": w.total, "elem_cand_per_step": ec, "code_layout": "packed",
+                       "scheme": args.scheme,
                        "l2": f"flushed between steps by writing {L2_FLUSH_BYTES >> 20} MiB",
                        "parallelism": f"independent batches x{world}"},
             "stages_ms": {"absmax": stage_tot[0] / args.steps, "search": search_ms,
@@ -356,13 +374,16 @@ def run_ours(args, rank, world, local_rank):
             "e2e": {"value": world * ec * e2e_steps / (e2e_ms * 1e-3) / 1e9, "unit": UNIT,
                     "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                     "ms_per_step": e2e_ms / e2e_steps, "matches_resident_path": same},
-            "gpu_launches": per_step * (args.steps + e2e_steps + 2 + max(3, args.warmup)),
+            "gpu_launches": (per_step + int(unsigned)) * (args.steps + max(3, args.warmup)) +
+                            per_step * (e2e_steps + 2),
             "kernels_per_step": per_step,
             "clocks": clocks, "device_status": status,
         }
         for k in ("absmax", "quantize", "dequantize"):
             line["hbm_stages"][k]["frac"] = line["hbm_stages"][k]["gbs"] / hbm
-        if world == 1 and not args.no_cpu_baseline:
+        if unsigned:
+            line["e2e"]["scheme"] = "signed (the host-buffer entry point has no one-sided form)"
+        if world == 1 and not args.no_cpu_baseline and not unsigned:
             cores = os.cpu_count() or 1
             spans, _ = oracle_sample(w, 2e8)                 # short calibration
             ev, dt = time_oracle(w, spans, cores)
@@ -388,6 +409,9 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="resnet50", choices=sorted(WORKLOADS))
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--scheme", default="signed", choices=["signed", "unsigned"],
+                    help="unsigned: min/max + one-sided search / quantize / dequantize (b-bit "
+                         "levels, no sign bit); a side measurement, not the headline")
     ap.add_argument("--bits", type=int, default=0, help="override the workload's bit-width")
     ap.add_argument("--K", type=int, default=0, help="override the number of candidates")
     ap.add_argument("--rows", type=int, default=0, help="laplace4096 only: number of rows")

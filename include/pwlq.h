@@ -122,6 +122,52 @@ int pwlq_dequantize_ragged(const uint8_t* codes, const uint8_t* region_mask,
                            const float* m, const float* p, float* y, int code_layout,
                            void* stream);
 
+/* One-sided ranges: unsigned tensors such as ReLU activations, or any asymmetric range [m1, m2]
+ * (Sec. 3.2, footnote to the range; Eq. 1 with z = r_l and the unsigned integer domain
+ * {0, ..., 2^b - 1} for one-sided distributions).  The paper does not spell the piecewise form
+ * out; this library takes the range [lo, hi] of a row, shifts it to [0, m], m = hi - lo, with the
+ * dense end at the lower bound, and splits it at one breakpoint p into the center [0, p] and the
+ * tail (p, m].  No sign is stored, so each piece keeps all 2^b levels, s = Delta / (2^b - 1):
+ *   a = min(max(x - lo, 0), m)           (one binary32 subtraction, then the clamp of Eq. 1)
+ *   tail = a > p;  q, v as in pwlq_quantize with L = 2^b - 1;  delivered value y = v + lo.
+ * The stored code is the level q (b bits); code and region-mask layouts are those of
+ * pwlq_quantize.  The squared error of the search is (v - a)^2, i.e. taken in the shifted domain
+ * (for lo = 0 the error of the delivered value).  A constant row (hi <= lo) gets code 0, y = lo,
+ * index 0, p = 0 and error 0.  On non-negative data with lo = 0 the result equals the signed
+ * scheme at b + 1 bits with the sign bit dropped.
+ *
+ * pwlq_minmax: lo_out[c] = min_i x[c, i], hi_out[c] = max_i x[c, i] (device, [C] each, distinct
+ * buffers); an empty row gets 0, 0; zeros are written as +0.  The other calls take lo and hi
+ * (device, [C], both required) where their signed counterparts take m; p, workspace, layouts,
+ * asynchrony, ownership and error behaviour are the same (workspace size:
+ * pwlq_search_workspace_bytes). */
+int pwlq_minmax(const float* x, int64_t C, int64_t n, float* lo_out, float* hi_out, void* stream);
+int pwlq_minmax_ragged(const float* x, const int64_t* row_offsets, int64_t C, int64_t total,
+                       float* lo_out, float* hi_out, void* stream);
+int pwlq_search_unsigned(const float* x, int64_t C, int64_t n, int bits, const float* ratios,
+                         int K, const float* lo, const float* hi, float* p_out, float* err_out,
+                         int32_t* idx_out, float* sse_all, void* workspace,
+                         size_t workspace_bytes, void* stream);
+int pwlq_search_unsigned_ragged(const float* x, const int64_t* row_offsets, int64_t C,
+                                int64_t total, int64_t max_n, int bits, const float* ratios,
+                                int K, const float* lo, const float* hi, float* p_out,
+                                float* err_out, int32_t* idx_out, float* sse_all, void* workspace,
+                                size_t workspace_bytes, void* stream);
+int pwlq_quantize_unsigned(const float* x, int64_t C, int64_t n, int bits, const float* lo,
+                           const float* hi, const float* p, uint8_t* codes,
+                           uint8_t* region_mask, float* fake_out, int code_layout, void* stream);
+int pwlq_quantize_unsigned_ragged(const float* x, const int64_t* row_offsets, int64_t C,
+                                  int64_t total, int bits, const float* lo, const float* hi,
+                                  const float* p, uint8_t* codes, uint8_t* region_mask,
+                                  float* fake_out, int code_layout, void* stream);
+int pwlq_dequantize_unsigned(const uint8_t* codes, const uint8_t* region_mask, int64_t C,
+                             int64_t n, int bits, const float* lo, const float* hi,
+                             const float* p, float* y, int code_layout, void* stream);
+int pwlq_dequantize_unsigned_ragged(const uint8_t* codes, const uint8_t* region_mask,
+                                    const int64_t* row_offsets, int64_t C, int64_t total,
+                                    int bits, const float* lo, const float* hi, const float* p,
+                                    float* y, int code_layout, void* stream);
+
 /* Analytic breakpoint selection, the paper's own way of choosing p (Sec. 3.3, Sec. 5.1): assume a
  * zero-mean density for each row, fit its scale, and take the breakpoint that minimises the
  * expected error of Eq. 5 -- the root of Eq. 9 on (0, m/2) -- or the closed form of Sec. 5.1.

@@ -24,6 +24,43 @@ constexpr int kAbsTableRows = 512;                       // staged rows per span
 
 static __device__ int g_absmax_timeout;                  // set when a bounded wait expired
 
+// Order-preserving map of binary32 values onto unsigned integers (and back), so that minima and
+// maxima of signed values can use integer atomics.
+__device__ __forceinline__ uint32_t ordered_key(float x) {
+    const uint32_t b = __float_as_uint(x);
+    return b ^ ((uint32_t)((int32_t)b >> 31) | 0x80000000u);
+}
+__device__ __forceinline__ float from_ordered_key(uint32_t k) {
+    return __uint_as_float((k & 0x80000000u) ? (k ^ 0x80000000u) : ~k);
+}
+
+// What is folded over a row.  MINMAX = false: the maximum of the magnitude bit patterns (exact and
+// order-free).  MINMAX = true: the maximum of the ordered keys and the maximum of the inverted
+// keys (i.e. the minimum); 0 means "nothing seen" in both.
+template <bool MINMAX>
+struct Fold {
+    uint32_t a = 0, b = 0;
+    __device__ __forceinline__ void add(float x) {
+        if (MINMAX) {
+            const uint32_t k = ordered_key(x);
+            a = max(a, k);
+            b = max(b, ~k);
+        } else {
+            a = max(a, abs_bits(x));
+        }
+    }
+    __device__ __forceinline__ void add4(const float4 v) { add(v.x); add(v.y); add(v.z); add(v.w); }
+    __device__ __forceinline__ void reduce_warp() {
+        a = __reduce_max_sync(0xffffffffu, a);
+        if (MINMAX) b = __reduce_max_sync(0xffffffffu, b);
+    }
+    __device__ __forceinline__ void store(uint32_t* hi, uint32_t* lo, int64_t row) const {
+        if (a != 0) atomicMax(hi + row, a);
+        if (MINMAX && b != 0) atomicMax(lo + row, b);
+    }
+    __device__ __forceinline__ void clear() { a = b = 0; }
+};
+
 struct AbsSmem {
     BulkRing<kAbsStages, kAbsSpan * 4> ring;
     SpanTable<false, kAbsTableRows> T;
@@ -36,9 +73,10 @@ __device__ __forceinline__ unsigned abs_bulk_bytes(int64_t span, int64_t total, 
     return (vec_ok && (cnt & 3) == 0) ? (unsigned)(cnt * 4) : 0u;
 }
 
+template <bool MINMAX>
 __global__ void __launch_bounds__(kAbsThreads)
 absmax_kernel(const float* __restrict__ x, Rows rows, int64_t total, uint32_t* __restrict__ m_bits,
-              int vec_ok, int64_t spans_per_cta) {
+              uint32_t* __restrict__ lo_bits, int vec_ok, int64_t spans_per_cta) {
     extern __shared__ __align__(128) unsigned char smem_raw[];
     AbsSmem& S = *reinterpret_cast<AbsSmem*>(smem_raw);
     __shared__ int s_abort;
@@ -56,7 +94,7 @@ absmax_kernel(const float* __restrict__ x, Rows rows, int64_t total, uint32_t* _
     RowFetch<kAbsTableRows> nf;
     if (use_table && s0 < s1) {
         row0 = cta_row_near(rows, s0 * kAbsSpan);
-        S.T.fetch(rows, nullptr, nullptr, row0, nf);
+        S.T.fetch(rows, nullptr, nullptr, nullptr, row0, nf);
         S.T.commit(nf, 0.0f);
         __syncthreads();
     }
@@ -65,12 +103,11 @@ absmax_kernel(const float* __restrict__ x, Rows rows, int64_t total, uint32_t* _
     // maximum over it; both survive from span to span, so a long row costs one atomic per warp
     // for the whole kernel.
     int64_t grow = -1;
-    uint32_t mx = 0;
+    Fold<MINMAX> mx;
     auto flush_merged = [&]() {                        // every lane of the warp calls this
-#pragma unroll
-        for (int o = 16; o > 0; o >>= 1) mx = max(mx, __shfl_xor_sync(0xffffffffu, mx, o));
-        if ((threadIdx.x & 31) == 0 && mx != 0 && grow >= 0) atomicMax(m_bits + grow, mx);
-        mx = 0;
+        mx.reduce_warp();
+        if ((threadIdx.x & 31) == 0 && grow >= 0) mx.store(m_bits, lo_bits, grow);
+        mx.clear();
     };
 
     for (int64_t span = s0; span < s1; ++span) {
@@ -96,7 +133,7 @@ absmax_kernel(const float* __restrict__ x, Rows rows, int64_t total, uint32_t* _
         if (has_next) {
             const int l = S.T.find(span_end);
             next_row0 = (l >= 0) ? row0 + l : warp_row_of(rows, span_end);
-            S.T.fetch(rows, nullptr, nullptr, next_row0, nf);
+            S.T.fetch(rows, nullptr, nullptr, nullptr, next_row0, nf);
         }
         if (!single) {                                 // several rows: nothing is carried across
             flush_merged();
@@ -120,12 +157,10 @@ absmax_kernel(const float* __restrict__ x, Rows rows, int64_t total, uint32_t* _
             for (int j = 0; j < kAbsUnroll; ++j) {
                 const int li = (j * kAbsThreads + threadIdx.x) * 4;
                 if (span_beg + li + 4 <= span_end) {
-                    const float4 v = *reinterpret_cast<const float4*>(xs + li);
-                    mx = max(max(mx, abs_bits(v.x)),
-                             max(abs_bits(v.y), max(abs_bits(v.z), abs_bits(v.w))));
+                    mx.add4(*reinterpret_cast<const float4*>(xs + li));
                 } else {
                     for (int t = 0; t < 4; ++t)
-                        if (span_beg + li + t < span_end) mx = max(mx, abs_bits(xs[li + t]));
+                        if (span_beg + li + t < span_end) mx.add(xs[li + t]);
                 }
             }
         } else {
@@ -157,22 +192,28 @@ absmax_kernel(const float* __restrict__ x, Rows rows, int64_t total, uint32_t* _
                     r_end = (int)min(e - span_beg, (int64_t)kAbsSpan);
                 };
                 enter_row(sl_beg);
-                uint32_t v = 0;
+                Fold<MINMAX> v;
                 for (int wb = sl_beg; wb < sl_end; wb += 128) {
                     const int we = min(wb + 128, sl_end);
                     const int i0 = wb + 4 * lane;
-                    uint32_t b[4] = {0u, 0u, 0u, 0u};
-                    if (i0 + 4 <= we) {
-                        const float4 f = *reinterpret_cast<const float4*>(xs + i0);
-                        b[0] = abs_bits(f.x); b[1] = abs_bits(f.y);
-                        b[2] = abs_bits(f.z); b[3] = abs_bits(f.w);
+                    float f[4] = {0.0f, 0.0f, 0.0f, 0.0f};
+                    const bool whole = i0 + 4 <= we;       // all four values lie inside the window
+                    if (whole) {
+                        const float4 q = *reinterpret_cast<const float4*>(xs + i0);
+                        f[0] = q.x; f[1] = q.y; f[2] = q.z; f[3] = q.w;
                     } else {
 #pragma unroll
                         for (int t = 0; t < 4; ++t)
-                            if (i0 + t < we) b[t] = abs_bits(xs[i0 + t]);
+                            if (i0 + t < we) f[t] = xs[i0 + t];
                     }
                     if (r_end >= we) {                     // the window lies inside the current row
-                        v = max(max(v, b[0]), max(b[1], max(b[2], b[3])));
+                        if (whole) {
+                            v.add4(make_float4(f[0], f[1], f[2], f[3]));
+                        } else {
+#pragma unroll
+                            for (int t = 0; t < 4; ++t)
+                                if (i0 + t < we) v.add(f[t]);
+                        }
                         continue;
                     }
                     int pos = wb;                          // values before pos are accounted for
@@ -180,19 +221,19 @@ absmax_kernel(const float* __restrict__ x, Rows rows, int64_t total, uint32_t* _
                         const int e = min(r_end, we);
 #pragma unroll
                         for (int t = 0; t < 4; ++t)
-                            if (i0 + t >= pos && i0 + t < e) v = max(v, b[t]);
+                            if (i0 + t >= pos && i0 + t < e) v.add(f[t]);
                         if (r_end > we) break;             // the row continues in the next window
-                        v = __reduce_max_sync(0xffffffffu, v);
-                        if (lane == 0 && v != 0) atomicMax(m_bits + r_glob, v);
-                        v = 0;
+                        v.reduce_warp();
+                        if (lane == 0) v.store(m_bits, lo_bits, r_glob);
+                        v.clear();
                         pos = e;
                         if (pos >= sl_end) break;          // the slice ends with this row
                         enter_row(pos);
                         if (pos >= we) break;              // the new row starts with the next window
                     }
                 }
-                v = __reduce_max_sync(0xffffffffu, v);     // the row the slice ends in
-                if (lane == 0 && v != 0) atomicMax(m_bits + r_glob, v);
+                v.reduce_warp();                           // the row the slice ends in
+                if (lane == 0) v.store(m_bits, lo_bits, r_glob);
             }
         }
         __syncthreads();                              // slot and table are no longer read
@@ -215,10 +256,35 @@ int absmax_timeout_flag() {
     return v;
 }
 
-cudaError_t launch_absmax(const float* x, const int64_t* row_offsets, int64_t C, int64_t n,
-                          int64_t total, float* m_out, cudaStream_t stream) {
-    cudaError_t e = cudaMemsetAsync(m_out, 0, sizeof(float) * (size_t)C, stream);
+// Turns the folded keys of minmax into values, in place.  A row in which nothing was seen (an
+// empty row) gets lo = hi = 0; zeros are delivered as +0.
+__global__ void minmax_finalize_kernel(uint32_t* __restrict__ lo_bits,
+                                       uint32_t* __restrict__ hi_bits, int64_t C) {
+    const int64_t c = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (c >= C) return;
+    const uint32_t kh = hi_bits[c], kl = lo_bits[c];
+    float hi = 0.0f, lo = 0.0f;
+    if (kh != 0 || kl != 0) {
+        hi = from_ordered_key(kh);
+        lo = from_ordered_key(~kl);
+    }
+    if (hi == 0.0f) hi = 0.0f;
+    if (lo == 0.0f) lo = 0.0f;
+    hi_bits[c] = __float_as_uint(hi);
+    lo_bits[c] = __float_as_uint(lo);
+}
+
+// Launches the folding kernel: MINMAX = false writes the abs-max bit patterns to out_a;
+// MINMAX = true folds ordered keys of the maxima into out_a and of the minima into out_b.
+template <bool MINMAX>
+static cudaError_t launch_fold(const float* x, const int64_t* row_offsets, int64_t C, int64_t n,
+                               int64_t total, float* out_a, float* out_b, cudaStream_t stream) {
+    cudaError_t e = cudaMemsetAsync(out_a, 0, sizeof(float) * (size_t)C, stream);
     if (e != cudaSuccess) return e;
+    if (MINMAX) {
+        e = cudaMemsetAsync(out_b, 0, sizeof(float) * (size_t)C, stream);
+        if (e != cudaSuccess) return e;
+    }
     if (total == 0) return cudaSuccess;
     Rows rows{row_offsets, C, n, n > 0 ? 1.0 / (double)n : 0.0};
     const int64_t nspans = (total + kAbsSpan - 1) / kAbsSpan;
@@ -227,12 +293,12 @@ cudaError_t launch_absmax(const float* x, const int64_t* row_offsets, int64_t C,
     cudaGetDevice(&dev);
     if (dev < 0 || dev >= 64) dev = 0;
     if (cached[dev] == 0) {
-        e = cudaFuncSetAttribute(absmax_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+        e = cudaFuncSetAttribute(absmax_kernel<MINMAX>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                  (int)sizeof(AbsSmem));
         if (e != cudaSuccess) return e;
         int sms = 0, per_sm = 0;
         cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-        cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, absmax_kernel, kAbsThreads,
+        cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, absmax_kernel<MINMAX>, kAbsThreads,
                                                       sizeof(AbsSmem));
         cached[dev] = (sms > 0 && per_sm > 0) ? sms * per_sm : 148;
     }
@@ -242,11 +308,27 @@ cudaError_t launch_absmax(const float* x, const int64_t* row_offsets, int64_t C,
     const int64_t slots = cached[dev];
     const bool several_rows = row_offsets != nullptr || n < kAbsSpan;
     int64_t per_cta = (nspans + slots - 1) / slots;
-    if (several_rows) per_cta = std::min<int64_t>(std::max<int64_t>((nspans + 4 * slots - 1) / (4 * slots), 4), 32);
+    if (several_rows)
+        per_cta = std::min<int64_t>(std::max<int64_t>((nspans + 4 * slots - 1) / (4 * slots), 4), 32);
     const unsigned grid = (unsigned)((nspans + per_cta - 1) / per_cta);
     const int vec_ok = (reinterpret_cast<uintptr_t>(x) & 15u) == 0;
-    absmax_kernel<<<grid, kAbsThreads, sizeof(AbsSmem), stream>>>(
-        x, rows, total, reinterpret_cast<uint32_t*>(m_out), vec_ok, per_cta);
+    absmax_kernel<MINMAX><<<grid, kAbsThreads, sizeof(AbsSmem), stream>>>(
+        x, rows, total, reinterpret_cast<uint32_t*>(out_a), reinterpret_cast<uint32_t*>(out_b),
+        vec_ok, per_cta);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_absmax(const float* x, const int64_t* row_offsets, int64_t C, int64_t n,
+                          int64_t total, float* m_out, cudaStream_t stream) {
+    return launch_fold<false>(x, row_offsets, C, n, total, m_out, nullptr, stream);
+}
+
+cudaError_t launch_minmax(const float* x, const int64_t* row_offsets, int64_t C, int64_t n,
+                          int64_t total, float* lo_out, float* hi_out, cudaStream_t stream) {
+    cudaError_t e = launch_fold<true>(x, row_offsets, C, n, total, hi_out, lo_out, stream);
+    if (e != cudaSuccess) return e;
+    minmax_finalize_kernel<<<(unsigned)((C + 255) / 256), 256, 0, stream>>>(
+        reinterpret_cast<uint32_t*>(lo_out), reinterpret_cast<uint32_t*>(hi_out), C);
     return cudaGetLastError();
 }
 

@@ -28,13 +28,27 @@ int absmax_impl(const float* x, const int64_t* ro, int64_t C, int64_t n, int64_t
     return from_cuda(pwlq::launch_absmax(x, ro, C, n, total, m_out, as_stream(stream)));
 }
 
+int minmax_impl(const float* x, const int64_t* ro, int64_t C, int64_t n, int64_t total,
+                float* lo_out, float* hi_out, void* stream) {
+    if (!x || !lo_out || !hi_out || lo_out == hi_out || misaligned(x, 4) ||
+        misaligned(lo_out, 4) || misaligned(hi_out, 4) || misaligned(ro, 8))
+        return PWLQ_ERR_INVALID_ARG;
+    if (total > kMaxTotal) return PWLQ_ERR_UNSUPPORTED;
+    return from_cuda(pwlq::launch_minmax(x, ro, C, n, total, lo_out, hi_out, as_stream(stream)));
+}
+
+// lo == nullptr: signed scheme (m = abs-max, may be null: computed internally);
+// lo != nullptr: one-sided ranges [lo, m], both required.
 int search_impl(const float* x, const int64_t* ro, int64_t C, int64_t n, int64_t total,
-                int64_t max_n, int bits, const float* ratios, int K, const float* m, float* p_out,
+                int64_t max_n, int bits, const float* ratios, int K, const float* m,
+                const float* lo, float* p_out,
                 float* err_out, int32_t* idx_out, float* sse_all, void* ws, size_t ws_bytes,
                 void* stream) {
-    if (!x || !ratios || !p_out || !idx_out || bits < 2 || bits > 8 || K < 1 || max_n < 1)
+    if (!x || !ratios || !p_out || !idx_out || bits < 2 || bits > 8 || K < 1 || max_n < 1 ||
+        (lo && !m))
         return PWLQ_ERR_INVALID_ARG;
-    if (misaligned(x, 4) || misaligned(ratios, 4) || misaligned(m, 4) || misaligned(p_out, 4) ||
+    if (misaligned(x, 4) || misaligned(ratios, 4) || misaligned(m, 4) || misaligned(lo, 4) ||
+        misaligned(p_out, 4) ||
         misaligned(err_out, 4) || misaligned(idx_out, 4) || misaligned(sse_all, 4) ||
         misaligned(ro, 8))
         return PWLQ_ERR_INVALID_ARG;
@@ -44,35 +58,36 @@ int search_impl(const float* x, const int64_t* ro, int64_t C, int64_t n, int64_t
         return PWLQ_ERR_UNSUPPORTED;
     if (!ws || ws_bytes < plan.bytes) return PWLQ_ERR_WORKSPACE;
     if (misaligned(ws, 256)) return PWLQ_ERR_INVALID_ARG;
-    return from_cuda(pwlq::launch_search(x, ro, C, n, total, bits, ratios, K, m, p_out, err_out,
-                                         idx_out, sse_all, ws, plan, as_stream(stream)));
+    return from_cuda(pwlq::launch_search(x, ro, C, n, total, bits, ratios, K, m, lo, p_out,
+                                         err_out, idx_out, sse_all, ws, plan, as_stream(stream)));
 }
 
 int quantize_impl(const float* x, const int64_t* ro, int64_t C, int64_t n, int64_t total,
-                  int bits, const float* m, const float* p, uint8_t* codes, uint8_t* mask,
-                  float* fake, int layout, void* stream) {
+                  int bits, const float* m, const float* lo, const float* p, uint8_t* codes,
+                  uint8_t* mask, float* fake, int layout, void* stream) {
     if (!x || !m || !p || !codes || !mask || bits < 2 || bits > 8 ||
         (layout != PWLQ_CODES_U8 && layout != PWLQ_CODES_PACKED))
         return PWLQ_ERR_INVALID_ARG;
-    if (misaligned(x, 4) || misaligned(m, 4) || misaligned(p, 4) || misaligned(fake, 4) ||
-        misaligned(ro, 8))
+    if (misaligned(x, 4) || misaligned(m, 4) || misaligned(lo, 4) || misaligned(p, 4) ||
+        misaligned(fake, 4) || misaligned(ro, 8))
         return PWLQ_ERR_INVALID_ARG;
     if (total > kMaxTotal) return PWLQ_ERR_UNSUPPORTED;
-    return from_cuda(pwlq::launch_quantize(x, ro, C, n, total, bits, m, p, codes, mask, fake,
+    return from_cuda(pwlq::launch_quantize(x, ro, C, n, total, bits, m, lo, p, codes, mask, fake,
                                            layout, as_stream(stream)));
 }
 
 int dequantize_impl(const uint8_t* codes, const uint8_t* mask, const int64_t* ro, int64_t C,
-                    int64_t n, int64_t total, int bits, const float* m, const float* p, float* y,
-                    int layout, void* stream) {
+                    int64_t n, int64_t total, int bits, const float* m, const float* lo,
+                    const float* p, float* y, int layout, void* stream) {
     if (!codes || !mask || !m || !p || !y || bits < 2 || bits > 8 ||
         (layout != PWLQ_CODES_U8 && layout != PWLQ_CODES_PACKED))
         return PWLQ_ERR_INVALID_ARG;
-    if (misaligned(m, 4) || misaligned(p, 4) || misaligned(y, 4) || misaligned(ro, 8))
+    if (misaligned(m, 4) || misaligned(lo, 4) || misaligned(p, 4) || misaligned(y, 4) ||
+        misaligned(ro, 8))
         return PWLQ_ERR_INVALID_ARG;
     if (total > kMaxTotal) return PWLQ_ERR_UNSUPPORTED;
-    return from_cuda(pwlq::launch_dequantize(codes, mask, ro, C, n, total, bits, m, p, y, layout,
-                                             as_stream(stream)));
+    return from_cuda(pwlq::launch_dequantize(codes, mask, ro, C, n, total, bits, m, lo, p, y,
+                                             layout, as_stream(stream)));
 }
 
 inline size_t code_bytes(int64_t total, int bits, int layout) {
@@ -129,8 +144,8 @@ int pwlq_search(const float* x, int64_t C, int64_t n, int bits, const float* rat
                 const float* m, float* p_out, float* err_out, int32_t* idx_out, float* sse_all,
                 void* workspace, size_t workspace_bytes, void* stream) {
     if (int rc = check_rows(C, n)) return rc;
-    return search_impl(x, nullptr, C, n, C * n, n, bits, ratios, K, m, p_out, err_out, idx_out,
-                       sse_all, workspace, workspace_bytes, stream);
+    return search_impl(x, nullptr, C, n, C * n, n, bits, ratios, K, m, nullptr, p_out, err_out,
+                       idx_out, sse_all, workspace, workspace_bytes, stream);
 }
 
 int pwlq_search_ragged(const float* x, const int64_t* row_offsets, int64_t C, int64_t total,
@@ -139,16 +154,16 @@ int pwlq_search_ragged(const float* x, const int64_t* row_offsets, int64_t C, in
                        void* workspace, size_t workspace_bytes, void* stream) {
     if (int rc = check_rows(C, total)) return rc;
     if (!row_offsets || max_n > total) return PWLQ_ERR_INVALID_ARG;
-    return search_impl(x, row_offsets, C, 0, total, max_n, bits, ratios, K, m, p_out, err_out,
-                       idx_out, sse_all, workspace, workspace_bytes, stream);
+    return search_impl(x, row_offsets, C, 0, total, max_n, bits, ratios, K, m, nullptr, p_out,
+                       err_out, idx_out, sse_all, workspace, workspace_bytes, stream);
 }
 
 int pwlq_quantize(const float* x, int64_t C, int64_t n, int bits, const float* m, const float* p,
                   uint8_t* codes, uint8_t* region_mask, float* fake_out, int code_layout,
                   void* stream) {
     if (int rc = check_rows(C, n)) return rc;
-    return quantize_impl(x, nullptr, C, n, C * n, bits, m, p, codes, region_mask, fake_out,
-                         code_layout, stream);
+    return quantize_impl(x, nullptr, C, n, C * n, bits, m, nullptr, p, codes, region_mask,
+                         fake_out, code_layout, stream);
 }
 
 int pwlq_quantize_ragged(const float* x, const int64_t* row_offsets, int64_t C, int64_t total,
@@ -156,16 +171,16 @@ int pwlq_quantize_ragged(const float* x, const int64_t* row_offsets, int64_t C, 
                          uint8_t* region_mask, float* fake_out, int code_layout, void* stream) {
     if (int rc = check_rows(C, total)) return rc;
     if (!row_offsets) return PWLQ_ERR_INVALID_ARG;
-    return quantize_impl(x, row_offsets, C, 0, total, bits, m, p, codes, region_mask, fake_out,
-                         code_layout, stream);
+    return quantize_impl(x, row_offsets, C, 0, total, bits, m, nullptr, p, codes, region_mask,
+                         fake_out, code_layout, stream);
 }
 
 int pwlq_dequantize(const uint8_t* codes, const uint8_t* region_mask, int64_t C, int64_t n,
                     int bits, const float* m, const float* p, float* y, int code_layout,
                     void* stream) {
     if (int rc = check_rows(C, n)) return rc;
-    return dequantize_impl(codes, region_mask, nullptr, C, n, C * n, bits, m, p, y, code_layout,
-                           stream);
+    return dequantize_impl(codes, region_mask, nullptr, C, n, C * n, bits, m, nullptr, p, y,
+                           code_layout, stream);
 }
 
 int pwlq_dequantize_ragged(const uint8_t* codes, const uint8_t* region_mask,
@@ -174,7 +189,79 @@ int pwlq_dequantize_ragged(const uint8_t* codes, const uint8_t* region_mask,
                            void* stream) {
     if (int rc = check_rows(C, total)) return rc;
     if (!row_offsets) return PWLQ_ERR_INVALID_ARG;
-    return dequantize_impl(codes, region_mask, row_offsets, C, 0, total, bits, m, p, y,
+    return dequantize_impl(codes, region_mask, row_offsets, C, 0, total, bits, m, nullptr, p, y,
+                           code_layout, stream);
+}
+
+int pwlq_minmax(const float* x, int64_t C, int64_t n, float* lo_out, float* hi_out,
+                void* stream) {
+    if (int rc = check_rows(C, n)) return rc;
+    return minmax_impl(x, nullptr, C, n, C * n, lo_out, hi_out, stream);
+}
+
+int pwlq_minmax_ragged(const float* x, const int64_t* row_offsets, int64_t C, int64_t total,
+                       float* lo_out, float* hi_out, void* stream) {
+    if (int rc = check_rows(C, total)) return rc;
+    if (!row_offsets) return PWLQ_ERR_INVALID_ARG;
+    return minmax_impl(x, row_offsets, C, 0, total, lo_out, hi_out, stream);
+}
+
+int pwlq_search_unsigned(const float* x, int64_t C, int64_t n, int bits, const float* ratios,
+                         int K, const float* lo, const float* hi, float* p_out, float* err_out,
+                         int32_t* idx_out, float* sse_all, void* workspace,
+                         size_t workspace_bytes, void* stream) {
+    if (int rc = check_rows(C, n)) return rc;
+    if (!lo || !hi) return PWLQ_ERR_INVALID_ARG;
+    return search_impl(x, nullptr, C, n, C * n, n, bits, ratios, K, hi, lo, p_out, err_out,
+                       idx_out, sse_all, workspace, workspace_bytes, stream);
+}
+
+int pwlq_search_unsigned_ragged(const float* x, const int64_t* row_offsets, int64_t C,
+                                int64_t total, int64_t max_n, int bits, const float* ratios,
+                                int K, const float* lo, const float* hi, float* p_out,
+                                float* err_out, int32_t* idx_out, float* sse_all, void* workspace,
+                                size_t workspace_bytes, void* stream) {
+    if (int rc = check_rows(C, total)) return rc;
+    if (!row_offsets || max_n > total || !lo || !hi) return PWLQ_ERR_INVALID_ARG;
+    return search_impl(x, row_offsets, C, 0, total, max_n, bits, ratios, K, hi, lo, p_out,
+                       err_out, idx_out, sse_all, workspace, workspace_bytes, stream);
+}
+
+int pwlq_quantize_unsigned(const float* x, int64_t C, int64_t n, int bits, const float* lo,
+                           const float* hi, const float* p, uint8_t* codes,
+                           uint8_t* region_mask, float* fake_out, int code_layout, void* stream) {
+    if (int rc = check_rows(C, n)) return rc;
+    if (!lo) return PWLQ_ERR_INVALID_ARG;
+    return quantize_impl(x, nullptr, C, n, C * n, bits, hi, lo, p, codes, region_mask, fake_out,
+                         code_layout, stream);
+}
+
+int pwlq_quantize_unsigned_ragged(const float* x, const int64_t* row_offsets, int64_t C,
+                                  int64_t total, int bits, const float* lo, const float* hi,
+                                  const float* p, uint8_t* codes, uint8_t* region_mask,
+                                  float* fake_out, int code_layout, void* stream) {
+    if (int rc = check_rows(C, total)) return rc;
+    if (!row_offsets || !lo) return PWLQ_ERR_INVALID_ARG;
+    return quantize_impl(x, row_offsets, C, 0, total, bits, hi, lo, p, codes, region_mask,
+                         fake_out, code_layout, stream);
+}
+
+int pwlq_dequantize_unsigned(const uint8_t* codes, const uint8_t* region_mask, int64_t C,
+                             int64_t n, int bits, const float* lo, const float* hi,
+                             const float* p, float* y, int code_layout, void* stream) {
+    if (int rc = check_rows(C, n)) return rc;
+    if (!lo) return PWLQ_ERR_INVALID_ARG;
+    return dequantize_impl(codes, region_mask, nullptr, C, n, C * n, bits, hi, lo, p, y,
+                           code_layout, stream);
+}
+
+int pwlq_dequantize_unsigned_ragged(const uint8_t* codes, const uint8_t* region_mask,
+                                    const int64_t* row_offsets, int64_t C, int64_t total,
+                                    int bits, const float* lo, const float* hi, const float* p,
+                                    float* y, int code_layout, void* stream) {
+    if (int rc = check_rows(C, total)) return rc;
+    if (!row_offsets || !lo) return PWLQ_ERR_INVALID_ARG;
+    return dequantize_impl(codes, region_mask, row_offsets, C, 0, total, bits, hi, lo, p, y,
                            code_layout, stream);
 }
 
@@ -225,11 +312,12 @@ int pwlq_encode_host(const float* x_host, const int64_t* row_offsets_host, int64
                                  cudaMemcpyHostToDevice, st));
     PWLQ_TRY(cudaMemcpyAsync(dr, ratios_host, sizeof(float) * (size_t)K, cudaMemcpyHostToDevice, st));
     PWLQ_TRY(pwlq::launch_absmax(dx, dro, C, n, total, dm, st));
-    PWLQ_TRY(pwlq::launch_search(dx, dro, C, n, total, bits, dr, K, dm, dp, de, di, nullptr,
-                                 d + h.ws, h.sp, st));
-    PWLQ_TRY(pwlq::launch_quantize(dx, dro, C, n, total, bits, dm, dp, dc, dk, nullptr,
+    PWLQ_TRY(pwlq::launch_search(dx, dro, C, n, total, bits, dr, K, dm, nullptr, dp, de, di,
+                                 nullptr, d + h.ws, h.sp, st));
+    PWLQ_TRY(pwlq::launch_quantize(dx, dro, C, n, total, bits, dm, nullptr, dp, dc, dk, nullptr,
                                    code_layout, st));
-    PWLQ_TRY(pwlq::launch_dequantize(dc, dk, dro, C, n, total, bits, dm, dp, dy, code_layout, st));
+    PWLQ_TRY(pwlq::launch_dequantize(dc, dk, dro, C, n, total, bits, dm, nullptr, dp, dy,
+                                     code_layout, st));
     PWLQ_TRY(cudaMemcpyAsync(m_host, dm, sizeof(float) * (size_t)C, cudaMemcpyDeviceToHost, st));
     PWLQ_TRY(cudaMemcpyAsync(p_host, dp, sizeof(float) * (size_t)C, cudaMemcpyDeviceToHost, st));
     if (err_host)

@@ -137,7 +137,7 @@ template <int CAP>
 struct RowFetch {                          // what one thread holds of the next window
     static constexpr int kPerThread = CAP / kTableThreads;
     int64_t off[kPerThread + 1];           // rows tid + u * 256, and (thread 0) the entry CAP
-    float m[kPerThread], p[kPerThread];
+    float m[kPerThread], p[kPerThread], lo[kPerThread];
 };
 
 template <bool PARAMS, int CAP>
@@ -145,7 +145,8 @@ struct SpanTable {
     static constexpr int kPerThread = CAP / kTableThreads;
     static_assert(CAP % kTableThreads == 0, "whole rounds of the CTA");
     int64_t off[CAP + 1];     // off[r] = first flat index of row row0 + r (INT64_MAX past the last row)
-    float m[PARAMS ? CAP : 1];
+    float m[PARAMS ? CAP : 1];    // range width: abs-max, or hi - lo for one-sided ranges
+    float lo[PARAMS ? CAP : 1];   // lower bound of a one-sided range (0 otherwise)
     PieceParams P[PARAMS ? CAP : 1];
 
     // True when every flat index below `end` lies in a staged row (or past the last row).
@@ -175,15 +176,24 @@ struct SpanTable {
         return lo;
     }
     // Requests the window that starts at row r0 (no barrier; the values stay in registers).
+    // lo_arr != nullptr: one-sided ranges, m_arr holds the upper bounds.
     __device__ __forceinline__ void fetch(const Rows& rows, const float* __restrict__ m_arr,
-                                          const float* __restrict__ p_arr, int64_t r0,
+                                          const float* __restrict__ p_arr,
+                                          const float* __restrict__ lo_arr, int64_t r0,
                                           RowFetch<CAP>& f) const {
 #pragma unroll
         for (int u = 0; u < kPerThread; ++u) {
             const int64_t row = r0 + (int)threadIdx.x + u * kTableThreads;
             f.off[u] = (row <= rows.C) ? rows.begin(row) : INT64_MAX;
-            f.m[u] = f.p[u] = 0.0f;
-            if (PARAMS && row < rows.C) { f.m[u] = __ldg(m_arr + row); f.p[u] = __ldg(p_arr + row); }
+            f.m[u] = f.p[u] = f.lo[u] = 0.0f;
+            if (PARAMS && row < rows.C) {
+                f.m[u] = __ldg(m_arr + row);
+                f.p[u] = __ldg(p_arr + row);
+                if (lo_arr) {
+                    f.lo[u] = __ldg(lo_arr + row);
+                    f.m[u] = __fsub_rn(f.m[u], f.lo[u]);
+                }
+            }
         }
         f.off[kPerThread] = (threadIdx.x == 0 && r0 + CAP <= rows.C) ? rows.begin(r0 + CAP)
                                                                      : INT64_MAX;
@@ -197,6 +207,7 @@ struct SpanTable {
             off[r] = f.off[u];
             if (PARAMS) {
                 m[r] = f.m[u];
+                lo[r] = f.lo[u];
                 P[r] = make_params(f.m[u], f.p[u], Lf);
             }
         }

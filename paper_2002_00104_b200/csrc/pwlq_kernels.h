@@ -14,6 +14,10 @@ constexpr int kSearchTile = 8192;
 cudaError_t launch_absmax(const float* x, const int64_t* row_offsets, int64_t C, int64_t n,
                           int64_t total, float* m_out, cudaStream_t stream);
 
+// Per-row minimum and maximum (the range [m1, m2] of a one-sided / asymmetric tensor).
+cudaError_t launch_minmax(const float* x, const int64_t* row_offsets, int64_t C, int64_t n,
+                          int64_t total, float* lo_out, float* hi_out, cudaStream_t stream);
+
 struct SearchPlan {
     int64_t max_n;         // longest row
     int64_t tiles;         // tiles per row (by the longest row)
@@ -26,18 +30,21 @@ SearchPlan plan_search(int64_t C, int64_t max_n, int K);
 
 cudaError_t launch_search(const float* x, const int64_t* row_offsets, int64_t C, int64_t n,
                           int64_t total, int bits, const float* ratios, int K, const float* m,
-                          float* p_out, float* err_out, int32_t* idx_out, float* sse_all,
+                          const float* lo, float* p_out, float* err_out, int32_t* idx_out, float* sse_all,
                           void* workspace, const SearchPlan& plan, cudaStream_t stream);
 
+// lo == nullptr: signed scheme with m = abs-max; lo != nullptr: one-sided ranges [lo, m] (m = upper
+// bounds), unsigned b-bit levels.  The same convention holds for launch_dequantize and
+// launch_search.
 cudaError_t launch_quantize(const float* x, const int64_t* row_offsets, int64_t C, int64_t n,
-                            int64_t total, int bits, const float* m, const float* p,
-                            uint8_t* codes, uint8_t* mask, float* fake, int layout,
+                            int64_t total, int bits, const float* m, const float* lo,
+                            const float* p, uint8_t* codes, uint8_t* mask, float* fake, int layout,
                             cudaStream_t stream);
 
 cudaError_t launch_dequantize(const uint8_t* codes, const uint8_t* mask,
                               const int64_t* row_offsets, int64_t C, int64_t n, int64_t total,
-                              int bits, const float* m, const float* p, float* y, int layout,
-                              cudaStream_t stream);
+                              int bits, const float* m, const float* lo, const float* p, float* y,
+                              int layout, cudaStream_t stream);
 
 size_t select_workspace_bytes(int64_t C, int64_t max_n);
 cudaError_t launch_select_analytic(const float* x, const int64_t* row_offsets, int64_t C,

@@ -65,7 +65,7 @@ extern "C" int pwlq_search_noalloc(const float* x, int64_t C, int64_t n, int bit
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     // launch_search clears the status word and writes every range and partial sum it later
     // reads, so nothing of the previous call's contents is consumed.
-    cudaError_t e = pwlq::launch_search(x, nullptr, C, n, C * n, bits, ratios, K, m, p_out,
+    cudaError_t e = pwlq::launch_search(x, nullptr, C, n, C * n, bits, ratios, K, m, nullptr, p_out,
                                         err_out, idx_out, sse_all, scratch, plan, st);
     if (e != cudaSuccess) return PWLQ_ERR_CUDA;
     if (status_out) {

@@ -38,44 +38,60 @@ constexpr int kQTableRows = 512;                 // rows of >= 8 values always f
 typedef SpanTable<true, kQTableRows> QuantSmem;
 typedef RowFetch<kQTableRows> QuantFetch;
 
+// Per-row inputs: m = abs-max and lo = nullptr (signed scheme), or m = upper and lo = lower
+// bound of a one-sided range; p = breakpoint.
+struct RowArrays {
+    const float* __restrict__ m;
+    const float* __restrict__ lo;
+    const float* __restrict__ p;
+};
+
 // The row a thread is currently in: constants in registers, refreshed when it crosses a boundary.
 struct RowState {
     int64_t beg = 0, end = 0;
-    float m = 0.0f;
+    float m = 0.0f;                                // range width (abs-max, or hi - lo)
+    float lo = 0.0f;                               // lower bound of a one-sided range, else 0
     PieceParams P;
     int loc = -1;                                  // index in the staged table (-1: not from it)
 
+    // Range width and lower bound of `row` straight from global memory.
+    static __device__ __forceinline__ void load_range(const RowArrays& A, int64_t row, float& m,
+                                                      float& lo) {
+        m = __ldg(A.m + row);
+        lo = 0.0f;
+        if (A.lo) { lo = __ldg(A.lo + row); m = __fsub_rn(m, lo); }
+    }
     template <bool TABLE>
-    __device__ __forceinline__ void seek(const QuantSmem& S, const Rows& rows,
-                                         const float* __restrict__ m_arr,
-                                         const float* __restrict__ p_arr, float Lf, int64_t i) {
+    __device__ __forceinline__ void seek(const QuantSmem& S, const Rows& rows, const RowArrays& A,
+                                         float Lf, int64_t i) {
         if (i >= beg && i < end) return;
         loc = TABLE ? S.find(i) : -1;
         if (loc >= 0) {
             beg = S.off[loc];
             end = S.off[loc + 1];
             m = S.m[loc];
+            lo = S.lo[loc];
             P = S.P[loc];
         } else {                                   // long dense rows, or beyond the staged rows
             const int64_t row = rows.row_of(i);
             beg = rows.begin(row);
             end = rows.begin(row + 1);
-            m = __ldg(m_arr + row);
-            P = make_params(m, __ldg(p_arr + row), Lf);
+            load_range(A, row, m, lo);
+            P = make_params(m, __ldg(A.p + row), Lf);
         }
     }
     // Constants of the row that follows, if that row reaches at least to need_end.
     template <bool TABLE>
     __device__ __forceinline__ bool next_row(const QuantSmem& S, const Rows& rows,
-                                             const float* __restrict__ m_arr,
-                                             const float* __restrict__ p_arr, float Lf,
-                                             int64_t need_end, float& mB, PieceParams& PB,
+                                             const RowArrays& A, float Lf, int64_t need_end,
+                                             float& mB, float& loB, PieceParams& PB,
                                              int64_t& endB) const {
         if (TABLE) {
             if (loc < 0 || loc + 1 >= kQTableRows) return false;
             endB = S.off[loc + 2];
             if (endB < need_end) return false;
             mB = S.m[loc + 1];
+            loB = S.lo[loc + 1];
             PB = S.P[loc + 1];
             return true;
         }
@@ -83,15 +99,17 @@ struct RowState {
         const int64_t row = rows.dense_row(end);
         if (row >= rows.C) return false;
         endB = end + rows.n;
-        mB = __ldg(m_arr + row);
-        PB = make_params(mB, __ldg(p_arr + row), Lf);
+        load_range(A, row, mB, loB);
+        PB = make_params(mB, __ldg(A.p + row), Lf);
         return true;
     }
     // Moves on to the row that next_row() returned.
-    __device__ __forceinline__ void advance(float mB, const PieceParams& PB, int64_t endB) {
+    __device__ __forceinline__ void advance(float mB, float loB, const PieceParams& PB,
+                                            int64_t endB) {
         beg = end;
         end = endB;
         m = mB;
+        lo = loB;
         P = PB;
         if (loc >= 0) ++loc;
     }
@@ -114,28 +132,32 @@ __device__ __forceinline__ unsigned q_bulk_bytes(int64_t span, int64_t total, in
 // hoisted, the level taken from the mantissa of t + 1.5 * 2^23, and the sign flag (x < 0, false
 // for -0.0) read off the sign bit of x + 0.0.  Codes are packed and region bits gathered on the
 // fly; there is no branch per value.
-template <bool PACKED, bool WANT_FAKE, bool TWO>
-__device__ __forceinline__ void quantize8(const float (&xv)[8], int split, float mA,
-                                          const PieceParams& A, float mB, const PieceParams& B,
-                                          float Lf, int Li, uint32_t sign_unit, int sign_shift,
-                                          uint32_t& w0, uint32_t& w1, uint32_t& mb, float (&yv)[8]) {
+// UNS: one-sided range, a = min(max(x - lo, 0), m), the code is the level itself and the delivered
+// value is v + lo.
+template <bool PACKED, bool WANT_FAKE, bool TWO, bool UNS>
+__device__ __forceinline__ void quantize8(const float (&xv)[8], int split, float mA, float loA,
+                                          const PieceParams& A, float mB, float loB,
+                                          const PieceParams& B, float Lf, int Li,
+                                          uint32_t sign_unit, int sign_shift, uint32_t& w0,
+                                          uint32_t& w1, uint32_t& mb, float (&yv)[8]) {
     w0 = w1 = mb = 0;
 #pragma unroll
     for (int t = 0; t < 8; ++t) {
         const bool second = TWO && t >= split;
         const float m = second ? mB : mA;
+        const float lo = second ? loB : loA;
         const float p = second ? B.p : A.p;
         const float inv1 = second ? B.inv1 : A.inv1;
         const float inv2 = second ? B.inv2 : A.inv2;
         const float xi = xv[t];
-        const float a = fminf(fabsf(xi), m);
+        const float a = UNS ? fminf(fmaxf(__fsub_rn(xi, lo), 0.0f), m) : fminf(fabsf(xi), m);
         const bool tail = a > p;
         const float z = tail ? p : 0.0f;
         const float inv = tail ? inv2 : inv1;
         const float r = __fadd_rn(__fmul_rn(__fsub_rn(a, z), inv), 12582912.0f);
         const uint32_t q = (uint32_t)min(__float_as_int(r) - 0x4B400000, Li);
-        const uint32_t xs0 = __float_as_uint(__fadd_rn(xi, 0.0f));   // sign bit = (x < 0)
-        const uint32_t code = ((xs0 >> sign_shift) & sign_unit) | q;
+        const uint32_t xs0 = UNS ? 0u : __float_as_uint(__fadd_rn(xi, 0.0f));   // sign bit = (x < 0)
+        const uint32_t code = UNS ? q : (((xs0 >> sign_shift) & sign_unit) | q);
         if (PACKED) w0 += code << (4 * t);
         else if (t < 4) w0 += code << (8 * t);
         else w1 += code << (8 * (t - 4));
@@ -146,7 +168,7 @@ __device__ __forceinline__ void quantize8(const float (&xv)[8], int split, float
             const float s = tail ? s2 : s1;
             const float qf = fminf(__fsub_rn(r, 12582912.0f), Lf);
             const float v = __fadd_rn(__fmul_rn(qf, s), z);
-            yv[t] = __uint_as_float(__float_as_uint(v) | (xs0 & 0x80000000u));
+            yv[t] = UNS ? __fadd_rn(v, lo) : __uint_as_float(__float_as_uint(v) | (xs0 & 0x80000000u));
         }
     }
 }
@@ -161,10 +183,9 @@ __device__ __forceinline__ void quantize8(const float (&xv)[8], int split, float
 // have their eight values inside one row; some lanes have them in two rows (per-value selects
 // between the two rows' constants); anything else (the tensor's tail, rows with m = 0, more than
 // two rows in eight values) takes the per-value path.
-template <bool PACKED, bool WANT_FAKE, bool TABLE>
+template <bool PACKED, bool WANT_FAKE, bool TABLE, bool UNS>
 __global__ void __launch_bounds__(kQThreads)
-quantize_kernel(const float* __restrict__ x, Rows rows, int64_t total, int bits,
-                const float* __restrict__ m_arr, const float* __restrict__ p_arr,
+quantize_kernel(const float* __restrict__ x, Rows rows, int64_t total, int bits, RowArrays A,
                 uint8_t* __restrict__ codes, uint8_t* __restrict__ mask, float* __restrict__ fake,
                 int vec_in, int vec_fake, int vec_codes, int64_t spans_per_cta) {
     extern __shared__ __align__(128) unsigned char smem_raw[];
@@ -172,8 +193,8 @@ quantize_kernel(const float* __restrict__ x, Rows rows, int64_t total, int bits,
     QuantSmem& S = Q.rows;
     __shared__ int s_abort;
     const unsigned full = 0xffffffffu;
-    const float Lf = (float)((1 << (bits - 1)) - 1);
-    const int Li = (1 << (bits - 1)) - 1;
+    const int Li = UNS ? (1 << bits) - 1 : (1 << (bits - 1)) - 1;    // largest level of a piece
+    const float Lf = (float)Li;
     const uint32_t sign_unit = 1u << (bits - 1);      // value of the sign bit inside a code
     const int sign_shift = 32 - bits;                 // moves bit 31 onto the code's sign bit
     const int64_t nspans = (total + kQSpan - 1) / kQSpan;
@@ -190,7 +211,7 @@ quantize_kernel(const float* __restrict__ x, Rows rows, int64_t total, int bits,
     QuantFetch nf;
     if (TABLE && first < last) {
         row0 = cta_row_near(rows, first * kQSpan);
-        S.fetch(rows, m_arr, p_arr, row0, nf);
+        S.fetch(rows, A.m, A.p, A.lo, row0, nf);
         S.commit(nf, Lf);
         __syncthreads();
     }
@@ -206,7 +227,7 @@ quantize_kernel(const float* __restrict__ x, Rows rows, int64_t total, int bits,
         if (has_next) {
             const int l = S.find(span_end);
             next_row0 = (l >= 0) ? row0 + l : warp_row_of(rows, span_end);
-            S.fetch(rows, m_arr, p_arr, next_row0, nf);
+            S.fetch(rows, A.m, A.p, A.lo, next_row0, nf);
         }
         float* xs = reinterpret_cast<float*>(Q.ring.slot(it));
         if (q_bulk_bytes(span, total, vec_in) != 0) {
@@ -231,23 +252,24 @@ quantize_kernel(const float* __restrict__ x, Rows rows, int64_t total, int bits,
             const int64_t pass_beg = i0 - ((int)threadIdx.x & 31) * 8, pass_end = pass_beg + 256;
             bool done = false;
             if (pass_end <= total) {
-                ws.seek<TABLE>(S, rows, m_arr, p_arr, Lf, pass_beg);
+                ws.seek<TABLE>(S, rows, A, Lf, pass_beg);
                 if (ws.m > 0.0f) {
                     if (ws.end >= pass_end) {
-                        quantize8<PACKED, WANT_FAKE, false>(xv, 8, ws.m, ws.P, ws.m, ws.P, Lf, Li,
-                                                            sign_unit, sign_shift, w0, w1, mb, yv);
+                        quantize8<PACKED, WANT_FAKE, false, UNS>(xv, 8, ws.m, ws.lo, ws.P, ws.m, ws.lo,
+                                                                 ws.P, Lf, Li, sign_unit, sign_shift,
+                                                                 w0, w1, mb, yv);
                         done = true;
                     } else {
-                        float mB = 0.0f;
+                        float mB = 0.0f, loB = 0.0f;
                         PieceParams PB = ws.P;
                         int64_t endB = 0;
-                        if (ws.next_row<TABLE>(S, rows, m_arr, p_arr, Lf, pass_end, mB, PB, endB) &&
+                        if (ws.next_row<TABLE>(S, rows, A, Lf, pass_end, mB, loB, PB, endB) &&
                             mB > 0.0f) {
                             const int split = (int)max((int64_t)0, min((int64_t)8, ws.end - i0));
                             if (__any_sync(full, split > 0 && split < 8)) {   // a lane holds both rows
-                                quantize8<PACKED, WANT_FAKE, true>(xv, split, ws.m, ws.P, mB, PB, Lf,
-                                                                   Li, sign_unit, sign_shift, w0, w1,
-                                                                   mb, yv);
+                                quantize8<PACKED, WANT_FAKE, true, UNS>(xv, split, ws.m, ws.lo, ws.P, mB,
+                                                                        loB, PB, Lf, Li, sign_unit,
+                                                                        sign_shift, w0, w1, mb, yv);
                             } else {
                                 const bool second = split == 0;
                                 PieceParams PL;
@@ -257,11 +279,12 @@ quantize_kernel(const float* __restrict__ x, Rows rows, int64_t total, int bits,
                                 PL.s2 = second ? PB.s2 : ws.P.s2;
                                 PL.inv2 = second ? PB.inv2 : ws.P.inv2;
                                 const float mL = second ? mB : ws.m;
-                                quantize8<PACKED, WANT_FAKE, false>(xv, 8, mL, PL, mL, PL, Lf, Li,
-                                                                    sign_unit, sign_shift, w0, w1,
-                                                                    mb, yv);
+                                const float loL = second ? loB : ws.lo;
+                                quantize8<PACKED, WANT_FAKE, false, UNS>(xv, 8, mL, loL, PL, mL, loL,
+                                                                         PL, Lf, Li, sign_unit,
+                                                                         sign_shift, w0, w1, mb, yv);
                             }
-                            ws.advance(mB, PB, endB);
+                            ws.advance(mB, loB, PB, endB);
                             done = true;
                         }
                     }
@@ -274,39 +297,43 @@ quantize_kernel(const float* __restrict__ x, Rows rows, int64_t total, int bits,
                 RowState rs;
                 int split = 8;
                 bool simple = true, two = false;
-                float mB = 0.0f;
+                float mB = 0.0f, loB = 0.0f;
                 PieceParams PB = ws.P;
                 int64_t endB = 0;
                 if (cnt > 0) {
-                    rs.seek<TABLE>(S, rows, m_arr, p_arr, Lf, i0);
+                    rs.seek<TABLE>(S, rows, A, Lf, i0);
                     split = (int)min((int64_t)8, rs.end - i0);
                     simple = cnt == 8 && split == 8 && rs.m > 0.0f;
                     if (cnt == 8 && split < 8 && rs.m > 0.0f)
-                        two = rs.next_row<TABLE>(S, rows, m_arr, p_arr, Lf, i0 + 8, mB, PB, endB) &&
+                        two = rs.next_row<TABLE>(S, rows, A, Lf, i0 + 8, mB, loB, PB, endB) &&
                               mB > 0.0f;
                 }
                 if (__all_sync(full, simple || two)) {
-                    if (!two) { mB = rs.m; PB = rs.P; split = 8; }
-                    quantize8<PACKED, WANT_FAKE, true>(xv, split, rs.m, rs.P, mB, PB, Lf, Li,
-                                                       sign_unit, sign_shift, w0, w1, mb, yv);
+                    if (!two) { mB = rs.m; loB = rs.lo; PB = rs.P; split = 8; }
+                    quantize8<PACKED, WANT_FAKE, true, UNS>(xv, split, rs.m, rs.lo, rs.P, mB, loB, PB,
+                                                            Lf, Li, sign_unit, sign_shift, w0, w1, mb,
+                                                            yv);
                 } else {
 #pragma unroll
                     for (int t = 0; t < 8; ++t) {
                         yv[t] = 0.0f;
                         if (t < cnt) {
-                            rs.seek<TABLE>(S, rows, m_arr, p_arr, Lf, i0 + t);
+                            rs.seek<TABLE>(S, rows, A, Lf, i0 + t);
+                            if (UNS) yv[t] = rs.lo;                // a constant row delivers lo
                             if (rs.m > 0.0f) {
                                 const float xi = xv[t];
-                                const int neg = xi < 0.0f;
+                                const int neg = !UNS && xi < 0.0f;
                                 int q, tail;
                                 float v;
-                                quantize_mag(fminf(fabsf(xi), rs.m), rs.P, Lf, q, tail, v);
+                                const float a = UNS ? fminf(fmaxf(__fsub_rn(xi, rs.lo), 0.0f), rs.m)
+                                                    : fminf(fabsf(xi), rs.m);
+                                quantize_mag(a, rs.P, Lf, q, tail, v);
                                 const uint32_t code = (uint32_t)((neg << (bits - 1)) | q);
                                 if (PACKED) w0 |= code << (4 * t);
                                 else if (t < 4) w0 |= code << (8 * t);
                                 else w1 |= code << (8 * (t - 4));
                                 mb |= (uint32_t)tail << t;
-                                yv[t] = neg ? -v : v;
+                                yv[t] = UNS ? __fadd_rn(v, rs.lo) : (neg ? -v : v);
                             }
                         }
                     }
@@ -404,13 +431,15 @@ __device__ __forceinline__ uint32_t code_of(uint32_t w0, uint32_t w1, int t) {
 // Eight consecutive codes, the first `split` of them in row A and the rest in row B (TWO = false:
 // all in row A), both rows with m > 0.  The level becomes a float through the mantissa of
 // 1.5 * 2^23 (exact for q < 2^22) instead of an integer conversion.
-template <bool PACKED, bool TWO>
+// UNS: one-sided range, the code is the level and the delivered value is v + lo.
+template <bool PACKED, bool TWO, bool UNS>
 __device__ __forceinline__ void dequantize8(uint32_t w0, uint32_t w1, uint32_t mb, int split,
-                                            const PieceParams& A, const PieceParams& B, int qmask,
-                                            int sign_shift, float (&yv)[8]) {
+                                            const PieceParams& A, float loA, const PieceParams& B,
+                                            float loB, int qmask, int sign_shift, float (&yv)[8]) {
 #pragma unroll
     for (int t = 0; t < 8; ++t) {
         const bool second = TWO && t >= split;
+        const float lo = second ? loB : loA;
         const float p = second ? B.p : A.p;
         const float s1 = second ? B.s1 : A.s1;
         const float s2 = second ? B.s2 : A.s2;
@@ -418,21 +447,21 @@ __device__ __forceinline__ void dequantize8(uint32_t w0, uint32_t w1, uint32_t m
         const bool tail = (mb & (1u << t)) != 0;
         const float q = __fsub_rn(__uint_as_float(0x4B400000u | (code & (uint32_t)qmask)), 12582912.0f);
         const float v = __fadd_rn(__fmul_rn(q, tail ? s2 : s1), tail ? p : 0.0f);
-        // the code's sign bit moved to bit 31
-        yv[t] = __uint_as_float(__float_as_uint(v) | ((code << sign_shift) & 0x80000000u));
+        // signed scheme: the code's sign bit moved to bit 31
+        yv[t] = UNS ? __fadd_rn(v, lo)
+                    : __uint_as_float(__float_as_uint(v) | ((code << sign_shift) & 0x80000000u));
     }
 }
 
-template <bool PACKED, bool TABLE>
+template <bool PACKED, bool TABLE, bool UNS>
 __global__ void __launch_bounds__(kQThreads)
 dequantize_kernel(const uint8_t* __restrict__ codes, const uint8_t* __restrict__ mask, Rows rows,
-                  int64_t total, int bits, const float* __restrict__ m_arr,
-                  const float* __restrict__ p_arr, float* __restrict__ y, int vec_codes,
+                  int64_t total, int bits, RowArrays A, float* __restrict__ y, int vec_codes,
                   int vec_out, int64_t spans_per_cta) {
     __shared__ QuantSmem S;
     const unsigned full = 0xffffffffu;
-    const float Lf = (float)((1 << (bits - 1)) - 1);
-    const int qmask = (1 << (bits - 1)) - 1;
+    const int qmask = UNS ? (1 << bits) - 1 : (1 << (bits - 1)) - 1;   // the level inside a code
+    const float Lf = (float)qmask;
     const int sign_shift = 32 - bits;                 // moves a code's sign bit to bit 31
     const int64_t nspans = (total + kQSpan - 1) / kQSpan;
     // the CTA's spans: consecutive with a row table (chained tables), strided otherwise
@@ -446,7 +475,7 @@ dequantize_kernel(const uint8_t* __restrict__ codes, const uint8_t* __restrict__
     QuantFetch nf;
     if (TABLE && first < last) {
         row0 = cta_row_near(rows, first * kQSpan);
-        S.fetch(rows, m_arr, p_arr, row0, nf);
+        S.fetch(rows, A.m, A.p, A.lo, row0, nf);
         S.commit(nf, Lf);
         __syncthreads();
     }
@@ -459,7 +488,7 @@ dequantize_kernel(const uint8_t* __restrict__ codes, const uint8_t* __restrict__
         if (has_next) {
             const int l = S.find(span_end);
             next_row0 = (l >= 0) ? row0 + l : warp_row_of(rows, span_end);
-            S.fetch(rows, m_arr, p_arr, next_row0, nf);
+            S.fetch(rows, A.m, A.p, A.lo, next_row0, nf);
         }
 #pragma unroll
         for (int c = 0; c < kQChunks; ++c) {
@@ -470,22 +499,23 @@ dequantize_kernel(const uint8_t* __restrict__ codes, const uint8_t* __restrict__
             const int64_t pass_beg = i0 - ((int)threadIdx.x & 31) * 8, pass_end = pass_beg + 256;
             bool done = false;
             if (pass_end <= total) {
-                ws.seek<TABLE>(S, rows, m_arr, p_arr, Lf, pass_beg);
+                ws.seek<TABLE>(S, rows, A, Lf, pass_beg);
                 if (ws.m > 0.0f) {
                     if (ws.end >= pass_end) {
-                        dequantize8<PACKED, false>(cur.w0[c], cur.w1[c], cur.mb[c], 8, ws.P, ws.P,
-                                                   qmask, sign_shift, yv);
+                        dequantize8<PACKED, false, UNS>(cur.w0[c], cur.w1[c], cur.mb[c], 8, ws.P, ws.lo,
+                                                        ws.P, ws.lo, qmask, sign_shift, yv);
                         done = true;
                     } else {
-                        float mB = 0.0f;
+                        float mB = 0.0f, loB = 0.0f;
                         PieceParams PB = ws.P;
                         int64_t endB = 0;
-                        if (ws.next_row<TABLE>(S, rows, m_arr, p_arr, Lf, pass_end, mB, PB, endB) &&
+                        if (ws.next_row<TABLE>(S, rows, A, Lf, pass_end, mB, loB, PB, endB) &&
                             mB > 0.0f) {
                             const int split = (int)max((int64_t)0, min((int64_t)8, ws.end - i0));
                             if (__any_sync(full, split > 0 && split < 8)) {   // a lane holds both rows
-                                dequantize8<PACKED, true>(cur.w0[c], cur.w1[c], cur.mb[c], split,
-                                                          ws.P, PB, qmask, sign_shift, yv);
+                                dequantize8<PACKED, true, UNS>(cur.w0[c], cur.w1[c], cur.mb[c], split,
+                                                               ws.P, ws.lo, PB, loB, qmask,
+                                                               sign_shift, yv);
                             } else {
                                 const bool second = split == 0;
                                 PieceParams PL;
@@ -493,10 +523,11 @@ dequantize_kernel(const uint8_t* __restrict__ codes, const uint8_t* __restrict__
                                 PL.s1 = second ? PB.s1 : ws.P.s1;
                                 PL.s2 = second ? PB.s2 : ws.P.s2;
                                 PL.inv1 = PL.inv2 = 0.0f;
-                                dequantize8<PACKED, false>(cur.w0[c], cur.w1[c], cur.mb[c], 8, PL, PL,
-                                                           qmask, sign_shift, yv);
+                                const float loL = second ? loB : ws.lo;
+                                dequantize8<PACKED, false, UNS>(cur.w0[c], cur.w1[c], cur.mb[c], 8, PL,
+                                                                loL, PL, loL, qmask, sign_shift, yv);
                             }
-                            ws.advance(mB, PB, endB);
+                            ws.advance(mB, loB, PB, endB);
                             done = true;
                         }
                     }
@@ -506,37 +537,38 @@ dequantize_kernel(const uint8_t* __restrict__ codes, const uint8_t* __restrict__
                 RowState rs;
                 int split = 8;
                 bool simple = true, two = false;
-                float mB = 0.0f;
+                float mB = 0.0f, loB = 0.0f;
                 PieceParams PB = ws.P;
                 int64_t endB = 0;
                 if (cnt > 0) {
-                    rs.seek<TABLE>(S, rows, m_arr, p_arr, Lf, i0);
+                    rs.seek<TABLE>(S, rows, A, Lf, i0);
                     split = (int)min((int64_t)8, rs.end - i0);
                     simple = cnt == 8 && split == 8 && rs.m > 0.0f;
                     if (cnt == 8 && split < 8 && rs.m > 0.0f)
-                        two = rs.next_row<TABLE>(S, rows, m_arr, p_arr, Lf, i0 + 8, mB, PB, endB) &&
+                        two = rs.next_row<TABLE>(S, rows, A, Lf, i0 + 8, mB, loB, PB, endB) &&
                               mB > 0.0f;
                 }
                 if (__all_sync(full, simple || two)) {
-                    if (!two) { PB = rs.P; split = 8; }
-                    dequantize8<PACKED, true>(cur.w0[c], cur.w1[c], cur.mb[c], split, rs.P, PB, qmask,
-                                              sign_shift, yv);
+                    if (!two) { PB = rs.P; loB = rs.lo; split = 8; }
+                    dequantize8<PACKED, true, UNS>(cur.w0[c], cur.w1[c], cur.mb[c], split, rs.P, rs.lo,
+                                                   PB, loB, qmask, sign_shift, yv);
                 } else {
 #pragma unroll
                     for (int t = 0; t < 8; ++t) {
                         yv[t] = 0.0f;
                         if (t < cnt) {
-                            rs.seek<TABLE>(S, rows, m_arr, p_arr, Lf, i0 + t);
+                            rs.seek<TABLE>(S, rows, A, Lf, i0 + t);
+                            if (UNS) yv[t] = rs.lo;                // a constant row delivers lo
                             if (rs.m > 0.0f) {
                                 const uint32_t code = code_of<PACKED>(cur.w0[c], cur.w1[c], t);
                                 const int tail = (cur.mb[c] >> t) & 1;
-                                const int neg = (code >> (bits - 1)) & 1;
+                                const int neg = !UNS && ((code >> (bits - 1)) & 1);
                                 const float q = (float)(code & qmask);
                                 const float s = tail ? rs.P.s2 : rs.P.s1;
                                 const float z = tail ? rs.P.p : 0.0f;
                                 float v = __fmul_rn(q, s);
                                 v = __fadd_rn(v, z);
-                                yv[t] = neg ? -v : v;
+                                yv[t] = UNS ? __fadd_rn(v, rs.lo) : (neg ? -v : v);
                             }
                         }
                     }
@@ -609,54 +641,62 @@ int quantize_timeout_flag() {
     return v;
 }
 
+// lo == nullptr: signed scheme, m = abs-max.  lo != nullptr: one-sided ranges [lo, m].
 cudaError_t launch_quantize(const float* x, const int64_t* row_offsets, int64_t C, int64_t n,
-                            int64_t total, int bits, const float* m, const float* p,
-                            uint8_t* codes, uint8_t* mask, float* fake, int layout,
+                            int64_t total, int bits, const float* m, const float* lo,
+                            const float* p, uint8_t* codes, uint8_t* mask, float* fake, int layout,
                             cudaStream_t stream) {
     if (total == 0) return cudaSuccess;
     Rows rows{row_offsets, C, n, n > 0 ? 1.0 / (double)n : 0.0};
+    const RowArrays A{m, lo, p};
     const bool packed = (layout == 1 && bits <= 4);
     const int64_t nspans = (total + kQSpan - 1) / kQSpan;
     const int vec_in = aligned(x, 16), vec_fake = fake ? aligned(fake, 16) : 0;
     const size_t smem = sizeof(QuantizeSmem);
     const int vec_codes = packed ? aligned(codes, 4) : aligned(codes, 8);
     const bool table = row_offsets != nullptr || n < kQSpan;    // several rows per span
-#define PWLQ_LAUNCH_QUANTIZE(PK, FK, RG)                                                          \
+#define PWLQ_LAUNCH_QUANTIZE(PK, FK, RG, UN)                                                      \
     do {                                                                                          \
-        const SpanGrid g = span_grid((const void*)quantize_kernel<PK, FK, RG>, kQThreads, smem,   \
-                                     nspans, RG);                                                 \
-        quantize_kernel<PK, FK, RG><<<g.grid, kQThreads, smem, stream>>>(                         \
-            x, rows, total, bits, m, p, codes, mask, fake, vec_in, vec_fake, vec_codes,           \
-            g.per_cta);                                                                           \
+        const SpanGrid g = span_grid((const void*)quantize_kernel<PK, FK, RG, UN>, kQThreads,     \
+                                     smem, nspans, RG);                                           \
+        quantize_kernel<PK, FK, RG, UN><<<g.grid, kQThreads, smem, stream>>>(                     \
+            x, rows, total, bits, A, codes, mask, fake, vec_in, vec_fake, vec_codes, g.per_cta);  \
     } while (0)
+#define PWLQ_LAUNCH_QUANTIZE_UN(PK, FK, RG) \
+    do { if (lo) PWLQ_LAUNCH_QUANTIZE(PK, FK, RG, true); else PWLQ_LAUNCH_QUANTIZE(PK, FK, RG, false); } while (0)
 #define PWLQ_LAUNCH_QUANTIZE_RG(PK, FK) \
-    do { if (table) PWLQ_LAUNCH_QUANTIZE(PK, FK, true); else PWLQ_LAUNCH_QUANTIZE(PK, FK, false); } while (0)
+    do { if (table) PWLQ_LAUNCH_QUANTIZE_UN(PK, FK, true); else PWLQ_LAUNCH_QUANTIZE_UN(PK, FK, false); } while (0)
     if (packed) { if (fake) PWLQ_LAUNCH_QUANTIZE_RG(true, true); else PWLQ_LAUNCH_QUANTIZE_RG(true, false); }
     else        { if (fake) PWLQ_LAUNCH_QUANTIZE_RG(false, true); else PWLQ_LAUNCH_QUANTIZE_RG(false, false); }
 #undef PWLQ_LAUNCH_QUANTIZE_RG
+#undef PWLQ_LAUNCH_QUANTIZE_UN
 #undef PWLQ_LAUNCH_QUANTIZE
     return cudaGetLastError();
 }
 
 cudaError_t launch_dequantize(const uint8_t* codes, const uint8_t* mask,
                               const int64_t* row_offsets, int64_t C, int64_t n, int64_t total,
-                              int bits, const float* m, const float* p, float* y, int layout,
-                              cudaStream_t stream) {
+                              int bits, const float* m, const float* lo, const float* p, float* y,
+                              int layout, cudaStream_t stream) {
     if (total == 0) return cudaSuccess;
     Rows rows{row_offsets, C, n, n > 0 ? 1.0 / (double)n : 0.0};
+    const RowArrays A{m, lo, p};
     const bool packed = (layout == 1 && bits <= 4);
     const int64_t nspans = (total + kQSpan - 1) / kQSpan;
-#define PWLQ_LAUNCH_DEQUANTIZE(PK, RG)                                                            \
+#define PWLQ_LAUNCH_DEQUANTIZE(PK, RG, UN)                                                        \
     do {                                                                                          \
-        const SpanGrid g = span_grid((const void*)dequantize_kernel<PK, RG>, kQThreads, 0,        \
+        const SpanGrid g = span_grid((const void*)dequantize_kernel<PK, RG, UN>, kQThreads, 0,    \
                                      nspans, RG);                                                 \
-        dequantize_kernel<PK, RG><<<g.grid, kQThreads, 0, stream>>>(                              \
-            codes, mask, rows, total, bits, m, p, y, aligned(codes, PK ? 4 : 8), aligned(y, 16),  \
+        dequantize_kernel<PK, RG, UN><<<g.grid, kQThreads, 0, stream>>>(                          \
+            codes, mask, rows, total, bits, A, y, aligned(codes, PK ? 4 : 8), aligned(y, 16),     \
             g.per_cta);                                                                           \
     } while (0)
+#define PWLQ_LAUNCH_DEQUANTIZE_UN(PK, RG) \
+    do { if (lo) PWLQ_LAUNCH_DEQUANTIZE(PK, RG, true); else PWLQ_LAUNCH_DEQUANTIZE(PK, RG, false); } while (0)
     const bool table = row_offsets != nullptr || n < kQSpan;    // several rows per span
-    if (packed) { if (table) PWLQ_LAUNCH_DEQUANTIZE(true, true); else PWLQ_LAUNCH_DEQUANTIZE(true, false); }
-    else        { if (table) PWLQ_LAUNCH_DEQUANTIZE(false, true); else PWLQ_LAUNCH_DEQUANTIZE(false, false); }
+    if (packed) { if (table) PWLQ_LAUNCH_DEQUANTIZE_UN(true, true); else PWLQ_LAUNCH_DEQUANTIZE_UN(true, false); }
+    else        { if (table) PWLQ_LAUNCH_DEQUANTIZE_UN(false, true); else PWLQ_LAUNCH_DEQUANTIZE_UN(false, false); }
+#undef PWLQ_LAUNCH_DEQUANTIZE_UN
 #undef PWLQ_LAUNCH_DEQUANTIZE
     return cudaGetLastError();
 }

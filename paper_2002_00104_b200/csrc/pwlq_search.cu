@@ -41,10 +41,11 @@ constexpr float kMagic = 12582912.0f;   // 1.5 * 2^23: adding it rounds to the n
 struct SearchArgs {
     const float* x;
     Rows rows;
-    const float* m;
+    const float* m;     // per-row abs-max (signed scheme) or upper bound (one-sided ranges)
+    const float* lo;    // per-row lower bound of a one-sided range; nullptr: signed scheme
     const float* ratios;
     int K;
-    int bits;
+    int levels;         // L: largest level of a piece, 2^(b-1) - 1 signed, 2^b - 1 one-sided
     int cap;            // tile capacity in values (multiple of 4, <= kSearchTile)
     int64_t n_min, n_max;   // this launch handles the rows with n_min <= length <= n_max
     int64_t grid_tiles;     // blockIdx.x = row * grid_tiles + tile
@@ -283,7 +284,7 @@ __device__ __forceinline__ void eval_unsorted(const SearchArgs& a, const float* 
                                               double* part, int cnt4, float m, int E) {
     const int K = a.K;
     const int G = (K + 31) / 32;
-    const float Lf = (float)((1 << (a.bits - 1)) - 1);
+    const float Lf = (float)a.levels;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const Pairs unused = {};
     for (int item = warp; item < G * E; item += (int)(blockDim.x >> 5)) {
@@ -302,8 +303,20 @@ __device__ __forceinline__ void eval_unsorted(const SearchArgs& a, const float* 
     }
 }
 
+// Range width of a row (abs-max, or hi - lo) and its lower bound (0 for the signed scheme).
+__device__ __forceinline__ float row_range(const SearchArgs& a, int64_t row, float& lo) {
+    float m = a.m[row];
+    lo = 0.0f;
+    if (a.lo) { lo = a.lo[row]; m = __fsub_rn(m, lo); }
+    return m;
+}
+// Magnitude the quantizer sees: min(|x|, m), or min(max(x - lo, 0), m) for a one-sided range.
+__device__ __forceinline__ float mag_of(const SearchArgs& a, float x, float m, float lo) {
+    return a.lo ? fminf(fmaxf(__fsub_rn(x, lo), 0.0f), m) : fminf(fabsf(x), m);
+}
+
 __device__ __forceinline__ bool row_setup(const SearchArgs& a, int64_t& row, int64_t& tile,
-                                          int64_t& t_beg, int& cnt, float& m) {
+                                          int64_t& t_beg, int& cnt, float& m, float& lo) {
     row = blockIdx.x / a.grid_tiles;
     tile = blockIdx.x - row * a.grid_tiles;
     const int64_t beg = a.rows.begin(row), end = a.rows.begin(row + 1);
@@ -311,8 +324,9 @@ __device__ __forceinline__ bool row_setup(const SearchArgs& a, int64_t& row, int
     t_beg = beg + tile * (int64_t)a.cap;
     if (t_beg >= end && tile > 0) return false;      // this row has fewer tiles than the longest
     cnt = (int)min((int64_t)a.cap, end - t_beg);
-    m = a.m[row];
-    const bool finite = __float_as_uint(m) < 0x7f800000u;
+    m = row_range(a, row, lo);
+    const bool finite = (__float_as_uint(m) & 0x7fffffffu) < 0x7f800000u &&
+                        (__float_as_uint(lo) & 0x7fffffffu) < 0x7f800000u;
     if (!finite || !(m > 0.0f) || cnt <= 0) {
         if (!finite && threadIdx.x == 0 && tile == 0) atomicOr(a.status, kStatusNonFinite);
         if (a.tiles == 1) write_degenerate_row(a, row);
@@ -393,7 +407,7 @@ __device__ __forceinline__ void eval_sorted(const SearchArgs& a, const SortedSme
                                             int n4, int pad, int E, int* next_item) {
     constexpr int kPhases = 32 / kCW;
     const int K = a.K;
-    const float Lf = (float)((1 << (a.bits - 1)) - 1);
+    const float Lf = (float)a.levels;
     const int G = (K + kCW - 1) / kCW;
     const int lane = threadIdx.x & 31;
     const int ci = lane % kCW, ph = lane / kCW;
@@ -446,8 +460,8 @@ search_sorted_kernel(SearchArgs a) {
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     int64_t row, tile, t_beg;
     int cnt;
-    float m;
-    if (!row_setup(a, row, tile, t_beg, cnt, m)) return;
+    float m, lo;
+    if (!row_setup(a, row, tile, t_beg, cnt, m, lo)) return;
 
     const int K = a.K;
     const int nwarps = (int)(blockDim.x >> 5), nthreads = (int)blockDim.x;
@@ -480,7 +494,7 @@ search_sorted_kernel(SearchArgs a) {
         // the grid is not ascending: no sorted structure to exploit
         const int cnt4 = (cnt + 3) >> 2;
         for (int i = threadIdx.x; i < cnt4 * 4; i += nthreads)
-            S.tile[i] = (i < cnt) ? fminf(fabsf(a.x[t_beg + i]), m) : 0.0f;
+            S.tile[i] = (i < cnt) ? mag_of(a, a.x[t_beg + i], m, lo) : 0.0f;
         __syncthreads();
         const int Eu = slices_for(K, nwarps);         // never more slices than the sorted layout
         eval_unsorted(a, S.tile, S.part, cnt4, m, Eu);
@@ -509,7 +523,7 @@ search_sorted_kernel(SearchArgs a) {
         int jv[4];
 #pragma unroll
         for (int u = 0; u < 4; ++u) {
-            av[u] = fminf(fabsf(nxt[u]), m);
+            av[u] = mag_of(a, nxt[u], m, lo);
             const int i = base + 128 + u * 32 + lane;
             nxt[u] = (i < w_end) ? __ldg(a.x + t_beg + i) : 0.0f;
         }
@@ -572,7 +586,7 @@ search_sorted_kernel(SearchArgs a) {
             const int i = base + u * 32 + lane;
             if (i < w_end) {
                 const uint32_t jr = S.jr[i];
-                S.tile[pad + myhist[jr & 0x7ffu] + (jr >> 11)] = fminf(fabsf(a.x[t_beg + i]), m);
+                S.tile[pad + myhist[jr & 0x7ffu] + (jr >> 11)] = mag_of(a, a.x[t_beg + i], m, lo);
             }
         }
     }
@@ -581,7 +595,7 @@ search_sorted_kernel(SearchArgs a) {
     // ---- evaluation
     const int n4 = (pad + cnt) >> 2;
     const int64_t n_row = a.rows.begin(row + 1) - a.rows.begin(row);
-    const int64_t L = (1 << (a.bits - 1)) - 1;
+    const int64_t L = a.levels;
     const bool fused = 2 * n_row >= L * L;
     if (cw == kCwLongTile) {
         if (fused) eval_sorted<kCwLongTile, false>(a, S, m, n4, pad, E, &next_item);
@@ -606,14 +620,14 @@ search_generic_kernel(SearchArgs a) {
     __shared__ int red_idx[kSWarps];
     int64_t row, tile, t_beg;
     int cnt;
-    float m;
-    if (!row_setup(a, row, tile, t_beg, cnt, m)) return;
+    float m, lo;
+    if (!row_setup(a, row, tile, t_beg, cnt, m, lo)) return;
     const int E = slices_for(a.K, kSWarps);
     const int cnt4 = (cnt + 3) >> 2;
     float* tile_s = reinterpret_cast<float*>(smem_raw);
     double* part = reinterpret_cast<double*>(smem_raw + (((size_t)a.cap * 4 + 15) & ~(size_t)15));
     for (int i = threadIdx.x; i < cnt4 * 4; i += kSThreads)
-        tile_s[i] = (i < cnt) ? fminf(fabsf(a.x[t_beg + i]), m) : 0.0f;   // zero padding: error 0
+        tile_s[i] = (i < cnt) ? mag_of(a, a.x[t_beg + i], m, lo) : 0.0f;   // zero padding: error 0
     __syncthreads();
     eval_unsorted(a, tile_s, part, cnt4, m, E);
     __syncthreads();
@@ -632,8 +646,10 @@ search_combine_kernel(SearchArgs a, double* __restrict__ sums) {
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int k = chunk * 32 + lane;
     const int64_t n_row = a.rows.begin(row + 1) - a.rows.begin(row);
-    const float m = a.m[row];
-    const bool finite = __float_as_uint(m) < 0x7f800000u;
+    float lo;
+    const float m = row_range(a, row, lo);
+    const bool finite = (__float_as_uint(m) & 0x7fffffffu) < 0x7f800000u &&
+                        (__float_as_uint(lo) & 0x7fffffffu) < 0x7f800000u;
     const bool degenerate = !finite || !(m > 0.0f) || n_row <= 0;
     const int64_t nt = degenerate ? 0 : (n_row + a.cap - 1) / a.cap;
     const int64_t t0 = nt * warp / kSWarps, t1 = nt * (warp + 1) / kSWarps;
@@ -659,8 +675,10 @@ search_argmin_kernel(SearchArgs a, const double* __restrict__ sums) {
     __shared__ int red_idx[kSWarps];
     const int64_t row = blockIdx.x;
     const int64_t n_row = a.rows.begin(row + 1) - a.rows.begin(row);
-    const float m = a.m[row];
-    const bool finite = __float_as_uint(m) < 0x7f800000u;
+    float lo;
+    const float m = row_range(a, row, lo);
+    const bool finite = (__float_as_uint(m) & 0x7fffffffu) < 0x7f800000u &&
+                        (__float_as_uint(lo) & 0x7fffffffu) < 0x7f800000u;
     if (!finite || !(m > 0.0f) || n_row <= 0) {
         if (threadIdx.x == 0) {
             a.idx_out[row] = 0;
@@ -697,12 +715,13 @@ SearchPlan plan_search(int64_t C, int64_t max_n, int K) {
 
 cudaError_t launch_search(const float* x, const int64_t* row_offsets, int64_t C, int64_t n,
                           int64_t total, int bits, const float* ratios, int K, const float* m,
-                          float* p_out, float* err_out, int32_t* idx_out, float* sse_all,
-                          void* workspace, const SearchPlan& plan, cudaStream_t stream) {
+                          const float* lo, float* p_out, float* err_out, int32_t* idx_out,
+                          float* sse_all, void* workspace, const SearchPlan& plan,
+                          cudaStream_t stream) {
     unsigned char* ws = static_cast<unsigned char*>(workspace);
     cudaError_t e = cudaMemsetAsync(ws, 0, 256, stream);          // status word
     if (e != cudaSuccess) return e;
-    if (!m) {
+    if (!m && !lo) {
         float* m_ws = reinterpret_cast<float*>(ws + plan.off_m);
         e = launch_absmax(x, row_offsets, C, n, total, m_ws, stream);
         if (e != cudaSuccess) return e;
@@ -714,7 +733,8 @@ cudaError_t launch_search(const float* x, const int64_t* row_offsets, int64_t C,
     a.m = m;
     a.ratios = ratios;
     a.K = K;
-    a.bits = bits;
+    a.lo = lo;
+    a.levels = lo ? (1 << bits) - 1 : (1 << (bits - 1)) - 1;
     a.tiles = plan.tiles;
     a.cap = (plan.tiles > 1) ? kSearchTile : (int)((plan.max_n + 3) / 4 * 4);
     a.partials = reinterpret_cast<double*>(ws + plan.off_partials);

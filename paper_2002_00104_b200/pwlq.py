@@ -36,6 +36,18 @@ _SIGNATURES = {
     "pwlq_quantize_ragged": (_INT, [_P, _P, _I64, _I64, _INT, _P, _P, _P, _P, _P, _INT, _P]),
     "pwlq_dequantize": (_INT, [_P, _P, _I64, _I64, _INT, _P, _P, _P, _INT, _P]),
     "pwlq_dequantize_ragged": (_INT, [_P, _P, _P, _I64, _I64, _INT, _P, _P, _P, _INT, _P]),
+    "pwlq_minmax": (_INT, [_P, _I64, _I64, _P, _P, _P]),
+    "pwlq_minmax_ragged": (_INT, [_P, _P, _I64, _I64, _P, _P, _P]),
+    "pwlq_search_unsigned": (_INT, [_P, _I64, _I64, _INT, _P, _INT, _P, _P, _P, _P, _P, _P, _P, _SZ,
+                                    _P]),
+    "pwlq_search_unsigned_ragged": (_INT, [_P, _P, _I64, _I64, _I64, _INT, _P, _INT, _P, _P, _P, _P,
+                                           _P, _P, _P, _SZ, _P]),
+    "pwlq_quantize_unsigned": (_INT, [_P, _I64, _I64, _INT, _P, _P, _P, _P, _P, _P, _INT, _P]),
+    "pwlq_quantize_unsigned_ragged": (_INT, [_P, _P, _I64, _I64, _INT, _P, _P, _P, _P, _P, _P, _INT,
+                                             _P]),
+    "pwlq_dequantize_unsigned": (_INT, [_P, _P, _I64, _I64, _INT, _P, _P, _P, _P, _INT, _P]),
+    "pwlq_dequantize_unsigned_ragged": (_INT, [_P, _P, _P, _I64, _I64, _INT, _P, _P, _P, _P, _INT,
+                                               _P]),
     "pwlq_encode_host_scratch_bytes": (_SZ, [_I64, _I64, _I64, _INT]),
     "pwlq_encode_host": (_INT, [_P, _P, _I64, _I64, _I64, _INT, _P, _INT, _P, _P, _P, _P, _P, _P,
                                 _INT, _P, _SZ, _P, _P]),
@@ -272,6 +284,105 @@ def dequantize(codes, mask, bits, m, p, C=None, n=None, layout=CODES_U8, row_off
                                         _dev(row_offsets, torch.int64, "row_offsets"), C, total,
                                         *tail)
     _check(rc, "pwlq_dequantize")
+    return y
+
+
+# ---- one-sided ranges [lo, hi] (unsigned tensors): b-bit levels, no sign bit
+def minmax(x, row_offsets=None, out=None, stream=None):
+    """Returns (lo, hi), the per-row minimum and maximum."""
+    lib = load_library()
+    C, n, total = _shape(x, row_offsets)
+    lo, hi = out if out is not None else (torch.empty(C, dtype=torch.float32, device=x.device),
+                                          torch.empty(C, dtype=torch.float32, device=x.device))
+    if row_offsets is None:
+        rc = lib.pwlq_minmax(_dev(x, torch.float32, "x"), C, n, _dev(lo, torch.float32, "lo"),
+                             _dev(hi, torch.float32, "hi"), _stream(stream))
+    else:
+        rc = lib.pwlq_minmax_ragged(_dev(x, torch.float32, "x"),
+                                    _dev(row_offsets, torch.int64, "row_offsets"), C, total,
+                                    _dev(lo, torch.float32, "lo"), _dev(hi, torch.float32, "hi"),
+                                    _stream(stream))
+    _check(rc, "pwlq_minmax")
+    return lo, hi
+
+
+def search_unsigned(x, bits, ratios, lo, hi, row_offsets=None, max_n=None, want_sse=False,
+                    workspace=None, out=None, stream=None):
+    """Returns dict(p, err, idx, sse or None, workspace).  ``workspace[:4]`` holds the status."""
+    lib = load_library()
+    C, n, total = _shape(x, row_offsets)
+    K = ratios.numel()
+    longest = n if row_offsets is None else int(max_n)
+    need = search_workspace_bytes(C, longest, K)
+    if workspace is None:
+        workspace = torch.empty(max(need, 256), dtype=torch.uint8, device=x.device)
+    if out is None:
+        out = {"p": torch.empty(C, dtype=torch.float32, device=x.device),
+               "err": torch.empty(C, dtype=torch.float32, device=x.device),
+               "idx": torch.empty(C, dtype=torch.int32, device=x.device),
+               "sse": torch.empty((C, K), dtype=torch.float32, device=x.device) if want_sse else None}
+    args_tail = (int(bits), _dev(ratios, torch.float32, "ratios"), K, _dev(lo, torch.float32, "lo"),
+                 _dev(hi, torch.float32, "hi"),
+                 _dev(out["p"], torch.float32, "p"), _dev(out["err"], torch.float32, "err"),
+                 _dev(out["idx"], torch.int32, "idx"), _dev(out.get("sse"), torch.float32, "sse"),
+                 _dev(workspace, torch.uint8, "workspace"), workspace.numel(), _stream(stream))
+    if row_offsets is None:
+        rc = lib.pwlq_search_unsigned(_dev(x, torch.float32, "x"), C, n, *args_tail)
+    else:
+        rc = lib.pwlq_search_unsigned_ragged(_dev(x, torch.float32, "x"),
+                                             _dev(row_offsets, torch.int64, "row_offsets"), C,
+                                             total, longest, *args_tail)
+    _check(rc, "pwlq_search_unsigned")
+    out = dict(out)
+    out["workspace"] = workspace
+    return out
+
+
+def quantize_unsigned(x, bits, lo, hi, p, layout=CODES_U8, row_offsets=None, want_fake=False,
+                      out=None, stream=None):
+    """Returns (codes uint8, region_mask uint8, fake fp32 or None)."""
+    lib = load_library()
+    C, n, total = _shape(x, row_offsets)
+    if out is None:
+        codes = torch.empty(code_bytes(total, bits, layout), dtype=torch.uint8, device=x.device)
+        mask = torch.empty((total + 7) // 8, dtype=torch.uint8, device=x.device)
+        fake = torch.empty(total, dtype=torch.float32, device=x.device) if want_fake else None
+    else:
+        codes, mask, fake = out
+    tail = (int(bits), _dev(lo, torch.float32, "lo"), _dev(hi, torch.float32, "hi"),
+            _dev(p, torch.float32, "p"), _dev(codes, torch.uint8, "codes"),
+            _dev(mask, torch.uint8, "mask"), _dev(fake, torch.float32, "fake"), int(layout),
+            _stream(stream))
+    if row_offsets is None:
+        rc = lib.pwlq_quantize_unsigned(_dev(x, torch.float32, "x"), C, n, *tail)
+    else:
+        rc = lib.pwlq_quantize_unsigned_ragged(_dev(x, torch.float32, "x"),
+                                               _dev(row_offsets, torch.int64, "row_offsets"), C,
+                                               total, *tail)
+    _check(rc, "pwlq_quantize_unsigned")
+    return codes, mask, fake
+
+
+def dequantize_unsigned(codes, mask, bits, lo, hi, p, C=None, n=None, layout=CODES_U8,
+                        row_offsets=None, out=None, stream=None):
+    lib = load_library()
+    if row_offsets is None:
+        total = int(C) * int(n)
+    else:
+        C = row_offsets.numel() - 1
+        total = int(out.numel()) if out is not None else int(row_offsets[-1].item())
+    y = out if out is not None else torch.empty(total, dtype=torch.float32, device=codes.device)
+    tail = (int(bits), _dev(lo, torch.float32, "lo"), _dev(hi, torch.float32, "hi"),
+            _dev(p, torch.float32, "p"), _dev(y, torch.float32, "y"), int(layout), _stream(stream))
+    if row_offsets is None:
+        rc = lib.pwlq_dequantize_unsigned(_dev(codes, torch.uint8, "codes"),
+                                          _dev(mask, torch.uint8, "mask"), int(C), int(n), *tail)
+    else:
+        rc = lib.pwlq_dequantize_unsigned_ragged(_dev(codes, torch.uint8, "codes"),
+                                                 _dev(mask, torch.uint8, "mask"),
+                                                 _dev(row_offsets, torch.int64, "row_offsets"), C,
+                                                 total, *tail)
+    _check(rc, "pwlq_dequantize_unsigned")
     return y
 
 
