@@ -485,3 +485,154 @@ void pwlq_oracle_elem_u(float x, float lo, float hi, float p, int bits,
     *region_out = r;
     *y_out = v + lo;
 }
+
+/* ------------------------------------------------------------------------------------------
+ * Two breakpoints (Sec. 5.1, "Multiple Breakpoints"): the paper says only that more breakpoints
+ * give more non-overlapping regions, each quantized uniformly, and that they are found by
+ * minimising the same error in an enlarged search space.  Reading taken here: breakpoints
+ * 0 < p1 < p2 <= m split [0, m] into R1 = [0, p1], R2 = (p1, p2], R3 = (p2, m]; inside every
+ * region (and sign) Eq. 1 is applied with b-1 bits, range [z, z + Delta] and offset z equal to
+ * the region's lower end (z = 0, p1, p2; Delta = p1, p2 - p1, m - p2), exactly as Eq. 3 does for
+ * its two regions.  The stored integer is the sign-magnitude code of Eq. 3; the region index
+ * (0, 1, 2) takes two bits per value: bits 2 (i & 3) and 2 (i & 3) + 1 of byte i >> 2.
+ * The search minimises the empirical squared error over all pairs i < j of the K candidate ratios,
+ * p1 = m * ratios[i], p2 = m * ratios[j]; the first minimal pair in the order (i, j) wins.
+ * With p2 = m the scheme is the one-breakpoint scheme with p = p1, which is what the tests pin
+ * it to first.
+ */
+typedef struct { float z[3], s[3], inv[3], Lf; } pw2_params;
+
+static pw2_params make_params2(float m, float p1, float p2, int bits)
+{
+    pw2_params P;
+    float d[3];
+    int r;
+    P.Lf = (float)((1 << (bits - 1)) - 1);
+    P.z[0] = 0.0f; P.z[1] = p1; P.z[2] = p2;
+    d[0] = p1; d[1] = p2 - p1; d[2] = m - p2;
+    for (r = 0; r < 3; ++r) {
+        if (d[r] > 0.0f) { P.s[r] = d[r] / P.Lf; P.inv[r] = P.Lf / d[r]; }
+        else             { P.s[r] = 0.0f;        P.inv[r] = 0.0f; }
+    }
+    return P;
+}
+
+static float pw2_elem(float x, float m, float p1, float p2, const pw2_params *P,
+                      int *q_out, int *region_out, float *a_out)
+{
+    float a = fminf(fabsf(x), m);
+    int r = (a > p1) + (a > p2);
+    float u = a - P->z[r];
+    float t = u * P->inv[r];
+    float q = fminf(rintf(t), P->Lf);
+    float v = q * P->s[r];
+    v = v + P->z[r];
+    *q_out = (int)q;
+    *region_out = r;
+    *a_out = a;
+    return v;
+}
+
+/* sse_f32 / sse_f64 (either may be NULL): [C, K, K], entry (i, j) valid for i < j, others 0. */
+int pwlq_oracle_search2(const float *x, const int64_t *row_offsets, int64_t C, int64_t n,
+                        int bits, const float *ratios, int K, const float *m_in,
+                        float *p1_out, float *p2_out, float *err_out, int32_t *idx1_out,
+                        int32_t *idx2_out, float *sse_f32, double *sse_f64)
+{
+    int64_t c, e, b, t;
+    int i, j;
+    if (!x || !ratios || !m_in || C < 1 || K < 2 || bits < 2 || bits > 8) return ORACLE_ERR_ARG;
+    for (c = 0; c < C; ++c) {
+        float m = m_in[c];
+        double best = 0.0;
+        int bi = 0, bj = 1, first = 1;
+        b = row_begin(row_offsets, n, c);
+        e = row_begin(row_offsets, n, c + 1);
+        if (!(m <= 3.402823466e+38f)) return ORACLE_ERR_NONFINITE;
+        for (i = 0; i < K; ++i) for (j = 0; j < K; ++j) {
+            double sse = 0.0;
+            if (i < j && m > 0.0f) {
+                float p1 = m * ratios[i], p2 = m * ratios[j];
+                pw2_params P = make_params2(m, p1, p2, bits);
+                for (t = b; t < e; ++t) {
+                    int q, r; float a;
+                    float v = pw2_elem(x[t], m, p1, p2, &P, &q, &r, &a);
+                    double d = (double)v - (double)a;
+                    sse += d * d;
+                }
+            }
+            if (sse_f32) sse_f32[(c * (int64_t)K + i) * K + j] = (float)sse;
+            if (sse_f64) sse_f64[(c * (int64_t)K + i) * K + j] = sse;
+            if (i < j && (first || sse < best)) { best = sse; bi = i; bj = j; first = 0; }
+        }
+        if (idx1_out) idx1_out[c] = bi;
+        if (idx2_out) idx2_out[c] = bj;
+        if (p1_out) p1_out[c] = (m > 0.0f) ? m * ratios[bi] : 0.0f;
+        if (p2_out) p2_out[c] = (m > 0.0f) ? m * ratios[bj] : 0.0f;
+        if (err_out) err_out[c] = (float)best;
+    }
+    return ORACLE_OK;
+}
+
+int pwlq_oracle_quantize2(const float *x, const int64_t *row_offsets, int64_t C, int64_t n,
+                          int bits, const float *m_in, const float *p1_in, const float *p2_in,
+                          uint8_t *codes, uint8_t *region2, float *fake_out, int layout)
+{
+    int64_t c, i, total;
+    int packed = (layout == 1 && bits <= 4);
+    if (!x || !m_in || !p1_in || !p2_in || C < 1 || bits < 2 || bits > 8) return ORACLE_ERR_ARG;
+    total = row_begin(row_offsets, n, C);
+    if (codes)   for (i = 0; i < (packed ? (total + 1) / 2 : total); ++i) codes[i] = 0;
+    if (region2) for (i = 0; i < (total + 3) / 4; ++i) region2[i] = 0;
+    for (c = 0; c < C; ++c) {
+        int64_t b = row_begin(row_offsets, n, c), e = row_begin(row_offsets, n, c + 1);
+        float m = m_in[c], p1 = p1_in[c], p2 = p2_in[c];
+        pw2_params P = make_params2(m, p1, p2, bits);
+        for (i = b; i < e; ++i) {
+            int q = 0, r = 0, neg = 0, code;
+            float a, v = 0.0f;
+            if (m > 0.0f) {
+                neg = (x[i] < 0.0f);
+                v = pw2_elem(x[i], m, p1, p2, &P, &q, &r, &a);
+            }
+            code = (neg << (bits - 1)) | q;
+            if (codes) {
+                if (packed) codes[i >> 1] |= (uint8_t)(code << ((i & 1) * 4));
+                else        codes[i] = (uint8_t)code;
+            }
+            if (region2) region2[i >> 2] |= (uint8_t)(r << ((i & 3) * 2));
+            if (fake_out) fake_out[i] = neg ? -v : v;
+        }
+    }
+    return ORACLE_OK;
+}
+
+int pwlq_oracle_dequantize2(const uint8_t *codes, const uint8_t *region2,
+                            const int64_t *row_offsets, int64_t C, int64_t n, int bits,
+                            const float *m_in, const float *p1_in, const float *p2_in, float *y,
+                            int layout)
+{
+    int64_t c, i;
+    int packed = (layout == 1 && bits <= 4);
+    int qmask = (1 << (bits - 1)) - 1;
+    if (!codes || !region2 || !m_in || !p1_in || !p2_in || !y || C < 1 || bits < 2 || bits > 8)
+        return ORACLE_ERR_ARG;
+    for (c = 0; c < C; ++c) {
+        int64_t b = row_begin(row_offsets, n, c), e = row_begin(row_offsets, n, c + 1);
+        float m = m_in[c];
+        pw2_params P = make_params2(m, p1_in[c], p2_in[c], bits);
+        for (i = b; i < e; ++i) {
+            int code = packed ? ((codes[i >> 1] >> ((i & 1) * 4)) & 0xF) : codes[i];
+            int r = (region2[i >> 2] >> ((i & 3) * 2)) & 3;
+            int neg = (code >> (bits - 1)) & 1;
+            float q = (float)(code & qmask);
+            float v;
+            if (r > 2) r = 2;
+            v = q * P.s[r];
+            v = v + P.z[r];
+            if (!(m > 0.0f)) { v = 0.0f; neg = 0; }
+            y[i] = neg ? -v : v;
+        }
+    }
+    return ORACLE_OK;
+}

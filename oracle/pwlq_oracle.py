@@ -97,6 +97,12 @@ class OracleLib:
         lib.pwlq_oracle_elem_u.argtypes = [ctypes.c_float, ctypes.c_float, ctypes.c_float,
                                            ctypes.c_float, ctypes.c_int, P, P, P]
         lib.pwlq_oracle_elem_u.restype = None
+        lib.pwlq_oracle_search2.argtypes = [P, P, I64, I64, ctypes.c_int, P, ctypes.c_int, P, P, P,
+                                            P, P, P, P, P]
+        lib.pwlq_oracle_quantize2.argtypes = [P, P, I64, I64, ctypes.c_int, P, P, P, P, P, P,
+                                              ctypes.c_int]
+        lib.pwlq_oracle_dequantize2.argtypes = [P, P, P, I64, I64, ctypes.c_int, P, P, P, P,
+                                                ctypes.c_int]
         self._lib = lib
 
     def absmax(self, x, row_offsets=None):
@@ -250,6 +256,56 @@ class OracleLib:
                                      ctypes.byref(code), ctypes.byref(region), ctypes.byref(y))
         return code.value, region.value, y.value
 
+    # ---- two breakpoints: regions [0, p1], (p1, p2], (p2, m]; region index in two bits per value
+    def search2(self, x, bits, ratios, m, row_offsets=None, want_sse=True):
+        """Returns dict(p1, p2, err, idx1, idx2, sse64 [C,K,K] (entries i < j valid))."""
+        flat, ro, C, n = _rows(x, row_offsets)
+        ratios = np.ascontiguousarray(ratios, dtype=np.float32)
+        K = int(ratios.size)
+        m = np.ascontiguousarray(m, dtype=np.float32)
+        assert m.size == C
+        p1 = np.empty(C, dtype=np.float32)
+        p2 = np.empty(C, dtype=np.float32)
+        err = np.empty(C, dtype=np.float32)
+        i1 = np.empty(C, dtype=np.int32)
+        i2 = np.empty(C, dtype=np.int32)
+        sse64 = np.empty((C, K, K), dtype=np.float64) if want_sse else None
+        _check(self._lib.pwlq_oracle_search2(_ptr(flat), _ptr(ro), C, n, int(bits), _ptr(ratios),
+                                             K, _ptr(m), _ptr(p1), _ptr(p2), _ptr(err), _ptr(i1),
+                                             _ptr(i2), None, _ptr(sse64)), "search2")
+        return {"p1": p1, "p2": p2, "err": err, "idx1": i1, "idx2": i2, "sse64": sse64}
+
+    def quantize2(self, x, bits, m, p1, p2, layout=0, row_offsets=None, want_fake=True):
+        """Returns (codes uint8, region2 uint8 (two bits per value), fake fp32 or None)."""
+        flat, ro, C, n = _rows(x, row_offsets)
+        total = flat.size
+        m, p1, p2 = (np.ascontiguousarray(v, dtype=np.float32) for v in (m, p1, p2))
+        assert m.size == C and p1.size == C and p2.size == C
+        codes = np.empty(code_bytes(total, bits, layout), dtype=np.uint8)
+        region = np.empty((total + 3) // 4, dtype=np.uint8)
+        fake = np.empty(total, dtype=np.float32) if want_fake else None
+        _check(self._lib.pwlq_oracle_quantize2(_ptr(flat), _ptr(ro), C, n, int(bits), _ptr(m),
+                                               _ptr(p1), _ptr(p2), _ptr(codes), _ptr(region),
+                                               _ptr(fake), int(layout)), "quantize2")
+        return codes, region, fake
+
+    def dequantize2(self, codes, region, bits, m, p1, p2, C=None, n=None, layout=0,
+                    row_offsets=None):
+        codes = np.ascontiguousarray(codes, dtype=np.uint8)
+        region = np.ascontiguousarray(region, dtype=np.uint8)
+        m, p1, p2 = (np.ascontiguousarray(v, dtype=np.float32) for v in (m, p1, p2))
+        if row_offsets is not None:
+            ro = np.ascontiguousarray(row_offsets, dtype=np.int64)
+            C, n, total = ro.size - 1, 0, int(ro[-1])
+        else:
+            ro, total = None, int(C) * int(n)
+        assert m.size == C and p1.size == C and p2.size == C
+        y = np.empty(total, dtype=np.float32)
+        _check(self._lib.pwlq_oracle_dequantize2(_ptr(codes), _ptr(region), _ptr(ro), C, n,
+                                                 int(bits), _ptr(m), _ptr(p1), _ptr(p2), _ptr(y),
+                                                 int(layout)), "dequantize2")
+        return y
+
     def params(self, m, p, bits):
         """(L, s1, inv1, s2, inv2) as binary32 values."""
         out = np.empty(5, dtype=np.float32)
@@ -317,3 +373,15 @@ def dequantize_u(*a, **k):
 
 def elem_u(*a, **k):
     return _get().elem_u(*a, **k)
+
+
+def search2(*a, **k):
+    return _get().search2(*a, **k)
+
+
+def quantize2(*a, **k):
+    return _get().quantize2(*a, **k)
+
+
+def dequantize2(*a, **k):
+    return _get().dequantize2(*a, **k)

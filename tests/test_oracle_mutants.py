@@ -6,6 +6,7 @@ import subprocess
 import pytest
 
 import test_oracle_pins as pins
+import test_oracle_two_breakpoints_pins as tpins
 import test_oracle_unsigned_pins as upins
 
 ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
@@ -51,6 +52,13 @@ MUTANTS = {
     "unsigned_dequant_level_mask": ("int qmask = (1 << bits) - 1;", "int qmask = (1 << (bits - 1)) - 1;"),
     "minmax_min_is_max": ("if (i == b || x[i] < lo) lo = x[i];", "if (i == b || x[i] > lo) lo = x[i];"),
     "unsigned_range_is_hi": ("        float m = hi_in[c] - lo;\n        double best = 0.0;", "        float m = hi_in[c];\n        double best = 0.0;"),
+    "two_bp_region_closed_at_p1": ("int r = (a > p1) + (a > p2);", "int r = (a >= p1) + (a > p2);"),
+    "two_bp_middle_range": ("d[0] = p1; d[1] = p2 - p1; d[2] = m - p2;", "d[0] = p1; d[1] = p2; d[2] = m - p2;"),
+    "two_bp_third_offset": ("P.z[0] = 0.0f; P.z[1] = p1; P.z[2] = p2;", "P.z[0] = 0.0f; P.z[1] = p1; P.z[2] = p1;"),
+    "two_bp_last_pair_on_ties": ("if (i < j && (first || sse < best))", "if (i < j && (first || sse <= best))"),
+    "two_bp_region_bit_order": ("region2[i >> 2] |= (uint8_t)(r << ((i & 3) * 2));",
+                                "region2[i >> 2] |= (uint8_t)(r << ((3 - (i & 3)) * 2));"),
+    "two_bp_pairs_not_ordered": ("if (i < j && m > 0.0f) {", "if (i != j && m > 0.0f) {"),
     "divide_not_reciprocal_free_pass": None,   # placeholder documented below
 }
 # 'divide_not_reciprocal': evaluating (|r| - z) / s by a true division instead of multiplying by
@@ -77,6 +85,10 @@ PIN_CALLS = [
     lambda o: upins.test_nonnegative_rows_equal_the_signed_scheme_with_one_more_bit(o, 3),
     lambda o: upins.test_levels_regions_and_half_step_bound_unsigned(o, 4),
     lambda o: upins.test_bruteforce_true_division_tiny_rows(o, 4, 32),
+    lambda o: tpins.test_worked_example_two_breakpoints(o),
+    lambda o: tpins.test_second_breakpoint_at_m_is_the_one_breakpoint_scheme(o, 3),
+    lambda o: tpins.test_pair_order_and_degenerate_rows(o),
+    lambda o: tpins.test_half_step_bound_per_region(o, 4),
 ]
 
 
