@@ -168,6 +168,52 @@ int pwlq_dequantize_unsigned_ragged(const uint8_t* codes, const uint8_t* region_
                                     int bits, const float* lo, const float* hi, const float* p,
                                     float* y, int code_layout, void* stream);
 
+/* Two breakpoints (Sec. 5.1, "Multiple Breakpoints": more non-overlapping regions, found by
+ * minimising the same error over an enlarged search space).  The paper gives no formulas beyond
+ * that; this library extends Eq. 3 in the obvious way: breakpoints 0 < p1 < p2 <= m split [0, m]
+ * into R1 = [0, p1], R2 = (p1, p2], R3 = (p2, m]; inside every region (and sign) Eq. 1 is applied
+ * with b-1 bits on the range [z, z + Delta], z = 0, p1, p2 and Delta = p1, p2 - p1, m - p2, with
+ * the arithmetic of pwlq_quantize.  The code is the sign-magnitude code of pwlq_quantize; the region
+ * index r in {0, 1, 2} takes two bits per value: bits 2 (i & 3), 2 (i & 3) + 1 of byte i >> 2 of
+ * region2 (ceil(total / 4) bytes), i the flat index.  With p2 = m the scheme is pwlq_quantize's.
+ *
+ * pwlq_search2: for every row, all pairs i < j of the K candidate ratios (ascending, K in
+ * [2, PWLQ_MAX_K2]), p1 = m * ratios[i], p2 = m * ratios[j]; squared error summed as in
+ * pwlq_search; the first minimal pair in the order (i, j) wins.  Rows are limited to 8192 values
+ * (PWLQ_ERR_UNSUPPORTED beyond).  m (device, [C]) is required.
+ *   p1_out, p2_out, idx1_out, idx2_out   device, [C]; err_out device [C] or NULL
+ *   sse_pairs   device, [C, K, K] or NULL; entry (i, j) is written with the sum for i < j, 0 otherwise
+ *   workspace   device, 256-byte aligned, pwlq_search2_workspace_bytes(...) bytes; its first word
+ *               is a status word as in pwlq_search (bit 1 << PWLQ_ERR_INVALID_ARG: the ratios do
+ *               not ascend, results of the launch are zeros)
+ * A row with m = 0 or no values gets indices (0, 1), p1 = p2 = 0, error 0.
+ * Asynchrony, ownership and error behaviour as for the one-breakpoint calls. */
+#define PWLQ_MAX_K2 64
+size_t pwlq_search2_workspace_bytes(int64_t C, int64_t max_n, int K);
+int pwlq_search2(const float* x, int64_t C, int64_t n, int bits, const float* ratios, int K,
+                 const float* m, float* p1_out, float* p2_out, float* err_out, int32_t* idx1_out,
+                 int32_t* idx2_out, float* sse_pairs, void* workspace, size_t workspace_bytes,
+                 void* stream);
+int pwlq_search2_ragged(const float* x, const int64_t* row_offsets, int64_t C, int64_t total,
+                        int64_t max_n, int bits, const float* ratios, int K, const float* m,
+                        float* p1_out, float* p2_out, float* err_out, int32_t* idx1_out,
+                        int32_t* idx2_out, float* sse_pairs, void* workspace,
+                        size_t workspace_bytes, void* stream);
+int pwlq_quantize2(const float* x, int64_t C, int64_t n, int bits, const float* m,
+                   const float* p1, const float* p2, uint8_t* codes, uint8_t* region2,
+                   float* fake_out, int code_layout, void* stream);
+int pwlq_quantize2_ragged(const float* x, const int64_t* row_offsets, int64_t C, int64_t total,
+                          int bits, const float* m, const float* p1, const float* p2,
+                          uint8_t* codes, uint8_t* region2, float* fake_out, int code_layout,
+                          void* stream);
+int pwlq_dequantize2(const uint8_t* codes, const uint8_t* region2, int64_t C, int64_t n,
+                     int bits, const float* m, const float* p1, const float* p2, float* y,
+                     int code_layout, void* stream);
+int pwlq_dequantize2_ragged(const uint8_t* codes, const uint8_t* region2,
+                            const int64_t* row_offsets, int64_t C, int64_t total, int bits,
+                            const float* m, const float* p1, const float* p2, float* y,
+                            int code_layout, void* stream);
+
 /* Analytic breakpoint selection, the paper's own way of choosing p (Sec. 3.3, Sec. 5.1): assume a
  * zero-mean density for each row, fit its scale, and take the breakpoint that minimises the
  * expected error of Eq. 5 -- the root of Eq. 9 on (0, m/2) -- or the closed form of Sec. 5.1.

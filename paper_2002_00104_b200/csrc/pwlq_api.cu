@@ -265,6 +265,117 @@ int pwlq_dequantize_unsigned_ragged(const uint8_t* codes, const uint8_t* region_
                            code_layout, stream);
 }
 
+size_t pwlq_search2_workspace_bytes(int64_t C, int64_t max_n, int K) {
+    if (C < 1 || max_n < 1 || max_n > pwlq::kSearchTile || K < 2 || K > PWLQ_MAX_K2) return 0;
+    return 256;
+}
+
+static int search2_impl(const float* x, const int64_t* ro, int64_t C, int64_t n, int64_t total,
+                        int64_t max_n, int bits, const float* ratios, int K, const float* m,
+                        float* p1_out, float* p2_out, float* err_out, int32_t* idx1_out,
+                        int32_t* idx2_out, float* sse_pairs, void* ws, size_t ws_bytes,
+                        void* stream) {
+    if (!x || !ratios || !m || !p1_out || !p2_out || !idx1_out || !idx2_out || bits < 2 ||
+        bits > 8 || K < 2 || max_n < 1)
+        return PWLQ_ERR_INVALID_ARG;
+    if (misaligned(x, 4) || misaligned(ratios, 4) || misaligned(m, 4) || misaligned(p1_out, 4) ||
+        misaligned(p2_out, 4) || misaligned(err_out, 4) || misaligned(idx1_out, 4) ||
+        misaligned(idx2_out, 4) || misaligned(sse_pairs, 4) || misaligned(ro, 8))
+        return PWLQ_ERR_INVALID_ARG;
+    if (K > PWLQ_MAX_K2 || max_n > pwlq::kSearchTile || total > kMaxTotal) return PWLQ_ERR_UNSUPPORTED;
+    if (!ws || ws_bytes < 256) return PWLQ_ERR_WORKSPACE;
+    if (misaligned(ws, 256)) return PWLQ_ERR_INVALID_ARG;
+    return from_cuda(pwlq::launch_search2(x, ro, C, n, max_n, bits, ratios, K, m, p1_out, p2_out,
+                                          err_out, idx1_out, idx2_out, sse_pairs, ws,
+                                          as_stream(stream)));
+}
+
+int pwlq_search2(const float* x, int64_t C, int64_t n, int bits, const float* ratios, int K,
+                 const float* m, float* p1_out, float* p2_out, float* err_out, int32_t* idx1_out,
+                 int32_t* idx2_out, float* sse_pairs, void* workspace, size_t workspace_bytes,
+                 void* stream) {
+    if (int rc = check_rows(C, n)) return rc;
+    return search2_impl(x, nullptr, C, n, C * n, n, bits, ratios, K, m, p1_out, p2_out, err_out,
+                        idx1_out, idx2_out, sse_pairs, workspace, workspace_bytes, stream);
+}
+
+int pwlq_search2_ragged(const float* x, const int64_t* row_offsets, int64_t C, int64_t total,
+                        int64_t max_n, int bits, const float* ratios, int K, const float* m,
+                        float* p1_out, float* p2_out, float* err_out, int32_t* idx1_out,
+                        int32_t* idx2_out, float* sse_pairs, void* workspace,
+                        size_t workspace_bytes, void* stream) {
+    if (int rc = check_rows(C, total)) return rc;
+    if (!row_offsets || max_n > total) return PWLQ_ERR_INVALID_ARG;
+    return search2_impl(x, row_offsets, C, 0, total, max_n, bits, ratios, K, m, p1_out, p2_out,
+                        err_out, idx1_out, idx2_out, sse_pairs, workspace, workspace_bytes, stream);
+}
+
+static int quantize2_impl(const float* x, const int64_t* ro, int64_t C, int64_t n, int64_t total,
+                          int bits, const float* m, const float* p1, const float* p2,
+                          uint8_t* codes, uint8_t* region2, float* fake, int layout,
+                          void* stream) {
+    if (!x || !m || !p1 || !p2 || !codes || !region2 || bits < 2 || bits > 8 ||
+        (layout != PWLQ_CODES_U8 && layout != PWLQ_CODES_PACKED))
+        return PWLQ_ERR_INVALID_ARG;
+    if (misaligned(x, 4) || misaligned(m, 4) || misaligned(p1, 4) || misaligned(p2, 4) ||
+        misaligned(fake, 4) || misaligned(ro, 8))
+        return PWLQ_ERR_INVALID_ARG;
+    if (total > kMaxTotal) return PWLQ_ERR_UNSUPPORTED;
+    return from_cuda(pwlq::launch_quantize2(x, ro, C, n, total, bits, m, p1, p2, codes, region2,
+                                            fake, layout, as_stream(stream)));
+}
+
+int pwlq_quantize2(const float* x, int64_t C, int64_t n, int bits, const float* m,
+                   const float* p1, const float* p2, uint8_t* codes, uint8_t* region2,
+                   float* fake_out, int code_layout, void* stream) {
+    if (int rc = check_rows(C, n)) return rc;
+    return quantize2_impl(x, nullptr, C, n, C * n, bits, m, p1, p2, codes, region2, fake_out,
+                          code_layout, stream);
+}
+
+int pwlq_quantize2_ragged(const float* x, const int64_t* row_offsets, int64_t C, int64_t total,
+                          int bits, const float* m, const float* p1, const float* p2,
+                          uint8_t* codes, uint8_t* region2, float* fake_out, int code_layout,
+                          void* stream) {
+    if (int rc = check_rows(C, total)) return rc;
+    if (!row_offsets) return PWLQ_ERR_INVALID_ARG;
+    return quantize2_impl(x, row_offsets, C, 0, total, bits, m, p1, p2, codes, region2, fake_out,
+                          code_layout, stream);
+}
+
+static int dequantize2_impl(const uint8_t* codes, const uint8_t* region2, const int64_t* ro,
+                            int64_t C, int64_t n, int64_t total, int bits, const float* m,
+                            const float* p1, const float* p2, float* y, int layout,
+                            void* stream) {
+    if (!codes || !region2 || !m || !p1 || !p2 || !y || bits < 2 || bits > 8 ||
+        (layout != PWLQ_CODES_U8 && layout != PWLQ_CODES_PACKED))
+        return PWLQ_ERR_INVALID_ARG;
+    if (misaligned(m, 4) || misaligned(p1, 4) || misaligned(p2, 4) || misaligned(y, 4) ||
+        misaligned(ro, 8))
+        return PWLQ_ERR_INVALID_ARG;
+    if (total > kMaxTotal) return PWLQ_ERR_UNSUPPORTED;
+    return from_cuda(pwlq::launch_dequantize2(codes, region2, ro, C, n, total, bits, m, p1, p2, y,
+                                              layout, as_stream(stream)));
+}
+
+int pwlq_dequantize2(const uint8_t* codes, const uint8_t* region2, int64_t C, int64_t n,
+                     int bits, const float* m, const float* p1, const float* p2, float* y,
+                     int code_layout, void* stream) {
+    if (int rc = check_rows(C, n)) return rc;
+    return dequantize2_impl(codes, region2, nullptr, C, n, C * n, bits, m, p1, p2, y, code_layout,
+                            stream);
+}
+
+int pwlq_dequantize2_ragged(const uint8_t* codes, const uint8_t* region2,
+                            const int64_t* row_offsets, int64_t C, int64_t total, int bits,
+                            const float* m, const float* p1, const float* p2, float* y,
+                            int code_layout, void* stream) {
+    if (int rc = check_rows(C, total)) return rc;
+    if (!row_offsets) return PWLQ_ERR_INVALID_ARG;
+    return dequantize2_impl(codes, region2, row_offsets, C, 0, total, bits, m, p1, p2, y,
+                            code_layout, stream);
+}
+
 size_t pwlq_encode_host_scratch_bytes(int64_t C, int64_t total, int64_t max_n, int K) {
     if (C < 1 || total < 1 || max_n < 1 || K < 1 || K > PWLQ_MAX_K) return 0;
     return plan_host(C, total, max_n, K).bytes;

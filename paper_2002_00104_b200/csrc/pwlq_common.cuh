@@ -11,6 +11,7 @@ namespace pwlq {
 
 constexpr int kWarp = 32;
 constexpr int kStatusNonFinite = 1 << 5;   // device status bit: 1 << PWLQ_ERR_NONFINITE
+constexpr int kStatusBadGrid = 1 << 1;     // device status bit: 1 << PWLQ_ERR_INVALID_ARG
 
 struct PieceParams {
     float p;     // breakpoint (offset z of the tail pieces, Eq. 3)

@@ -46,6 +46,23 @@ cudaError_t launch_dequantize(const uint8_t* codes, const uint8_t* mask,
                               int bits, const float* m, const float* lo, const float* p, float* y,
                               int layout, cudaStream_t stream);
 
+// Two breakpoints (three regions): pair search over a grid of K <= kSearch2MaxK ascending ratios
+// for rows of at most kSearchTile values; quantize / dequantize with a two-bit region index.
+constexpr int kSearch2MaxK = 64;
+cudaError_t launch_search2(const float* x, const int64_t* row_offsets, int64_t C, int64_t n,
+                           int64_t max_n, int bits, const float* ratios, int K, const float* m,
+                           float* p1_out, float* p2_out, float* err_out, int32_t* idx1_out,
+                           int32_t* idx2_out, float* sse_pairs, void* workspace,
+                           cudaStream_t stream);
+cudaError_t launch_quantize2(const float* x, const int64_t* row_offsets, int64_t C, int64_t n,
+                             int64_t total, int bits, const float* m, const float* p1,
+                             const float* p2, uint8_t* codes, uint8_t* region2, float* fake,
+                             int layout, cudaStream_t stream);
+cudaError_t launch_dequantize2(const uint8_t* codes, const uint8_t* region2,
+                               const int64_t* row_offsets, int64_t C, int64_t n, int64_t total,
+                               int bits, const float* m, const float* p1, const float* p2,
+                               float* y, int layout, cudaStream_t stream);
+
 size_t select_workspace_bytes(int64_t C, int64_t max_n);
 cudaError_t launch_select_analytic(const float* x, const int64_t* row_offsets, int64_t C,
                                    int64_t n, int64_t max_n, const float* m, int model,
