@@ -636,3 +636,117 @@ int pwlq_oracle_dequantize2(const uint8_t *codes, const uint8_t *region2,
     }
     return ORACLE_OK;
 }
+
+/* ------------------------------------------------------------------------------------------
+ * Bias correction (Sec. 5.1, "Bias Correction"): quantization shifts the mean and the variance of
+ * a row; the paper compensates this by folding correction terms into the scale and the offset,
+ * citing earlier work, and prints no formula.  Reading taken here: with y_i = pw(x_i) the
+ * delivered value of the quantizer for row c,
+ *     xi_c   = sqrt( sum_i (x_i - mean x)^2 / sum_i (y_i - mean y)^2 )     (1 if a sum is 0)
+ *     beta_c = mean x - xi_c * mean y
+ * and the corrected value is y'_i = xi_c * y_i + beta_c, so that the corrected row has exactly
+ * the mean and the centred norm of the original row.  Means and sums in binary64 (two passes);
+ * xi and beta are delivered in binary32 and applied as one binary32 multiply and one add.
+ * An empty row gets xi = 1, beta = 0.
+ */
+int pwlq_oracle_bias_correction(const float *x, const int64_t *row_offsets, int64_t C, int64_t n,
+                                int bits, const float *m_in, const float *p_in, float *xi_out,
+                                float *beta_out)
+{
+    int64_t c, i;
+    if (!x || !m_in || !p_in || !xi_out || !beta_out || C < 1 || bits < 2 || bits > 8)
+        return ORACLE_ERR_ARG;
+    for (c = 0; c < C; ++c) {
+        int64_t b = row_begin(row_offsets, n, c), e = row_begin(row_offsets, n, c + 1);
+        float m = m_in[c], p = p_in[c];
+        pw_params P = make_params(m, p, bits);
+        double sx = 0.0, sy = 0.0, vx = 0.0, vy = 0.0, mx, my, xi = 1.0;
+        if (e <= b) { xi_out[c] = 1.0f; beta_out[c] = 0.0f; continue; }
+        for (i = b; i < e; ++i) {
+            int q, r; float a, v = 0.0f;
+            if (m > 0.0f) v = pw_elem(x[i], m, p, &P, &q, &r, &a);
+            sx += (double)x[i];
+            sy += (double)((m > 0.0f && x[i] < 0.0f) ? -v : v);
+        }
+        mx = sx / (double)(e - b);
+        my = sy / (double)(e - b);
+        for (i = b; i < e; ++i) {
+            int q, r; float a, v = 0.0f;
+            double y;
+            if (m > 0.0f) v = pw_elem(x[i], m, p, &P, &q, &r, &a);
+            y = (double)((m > 0.0f && x[i] < 0.0f) ? -v : v);
+            vx += ((double)x[i] - mx) * ((double)x[i] - mx);
+            vy += (y - my) * (y - my);
+        }
+        if (vx > 0.0 && vy > 0.0) xi = sqrt(vx / vy);
+        xi_out[c] = (float)xi;
+        beta_out[c] = (float)(mx - xi * my);
+    }
+    return ORACLE_OK;
+}
+
+/* Dequantize with the folded correction: y' = xi * y + beta (binary32, two roundings). */
+int pwlq_oracle_dequantize_bc(const uint8_t *codes, const uint8_t *region_mask,
+                              const int64_t *row_offsets, int64_t C, int64_t n, int bits,
+                              const float *m_in, const float *p_in, const float *xi_in,
+                              const float *beta_in, float *y, int layout)
+{
+    int64_t c, i;
+    int rc = pwlq_oracle_dequantize(codes, region_mask, row_offsets, C, n, bits, m_in, p_in, y,
+                                    layout);
+    if (rc != ORACLE_OK) return rc;
+    if (!xi_in || !beta_in) return ORACLE_ERR_ARG;
+    for (c = 0; c < C; ++c) {
+        int64_t b = row_begin(row_offsets, n, c), e = row_begin(row_offsets, n, c + 1);
+        for (i = b; i < e; ++i) {
+            float t = xi_in[c] * y[i];
+            y[i] = t + beta_in[c];
+        }
+    }
+    return ORACLE_OK;
+}
+
+/* ------------------------------------------------------------------------------------------
+ * Dense storage: Sec. 4 counts b bits per value plus one bit for the region.  Here the two are
+ * stored together as a (b+1)-bit field, field = code | region << b, value i occupying bits
+ * [i (b+1), (i+1) (b+1)) of a little-endian bit stream (bit k of the stream is bit k & 7 of byte
+ * k >> 3).  ceil(total (b+1) / 8) bytes.
+ */
+int pwlq_oracle_pack_dense(const uint8_t *codes_u8, const uint8_t *region_mask, int64_t total,
+                           int bits, uint8_t *stream)
+{
+    int64_t i, nbytes = (total * (bits + 1) + 7) / 8;
+    int k;
+    if (!codes_u8 || !region_mask || !stream || bits < 2 || bits > 8 || total < 0)
+        return ORACLE_ERR_ARG;
+    for (i = 0; i < nbytes; ++i) stream[i] = 0;
+    for (i = 0; i < total; ++i) {
+        int r = (region_mask[i >> 3] >> (i & 7)) & 1;
+        int field = (codes_u8[i] & ((1 << bits) - 1)) | (r << bits);
+        for (k = 0; k <= bits; ++k) {
+            int64_t pos = i * (bits + 1) + k;
+            if ((field >> k) & 1) stream[pos >> 3] |= (uint8_t)(1u << (pos & 7));
+        }
+    }
+    return ORACLE_OK;
+}
+
+int pwlq_oracle_unpack_dense(const uint8_t *stream, int64_t total, int bits, uint8_t *codes_u8,
+                             uint8_t *region_mask)
+{
+    int64_t i;
+    int k;
+    if (!codes_u8 || !region_mask || !stream || bits < 2 || bits > 8 || total < 0)
+        return ORACLE_ERR_ARG;
+    for (i = 0; i < (total + 7) / 8; ++i) region_mask[i] = 0;
+    for (i = 0; i < total; ++i) {
+        int field = 0;
+        for (k = 0; k <= bits; ++k) {
+            int64_t pos = i * (bits + 1) + k;
+            field |= ((stream[pos >> 3] >> (pos & 7)) & 1) << k;
+        }
+        codes_u8[i] = (uint8_t)(field & ((1 << bits) - 1));
+        if (field >> bits) region_mask[i >> 3] |= (uint8_t)(1u << (i & 7));
+    }
+    return ORACLE_OK;
+}

@@ -103,6 +103,11 @@ class OracleLib:
                                               ctypes.c_int]
         lib.pwlq_oracle_dequantize2.argtypes = [P, P, P, I64, I64, ctypes.c_int, P, P, P, P,
                                                 ctypes.c_int]
+        lib.pwlq_oracle_bias_correction.argtypes = [P, P, I64, I64, ctypes.c_int, P, P, P, P]
+        lib.pwlq_oracle_dequantize_bc.argtypes = [P, P, P, I64, I64, ctypes.c_int, P, P, P, P, P,
+                                                  ctypes.c_int]
+        lib.pwlq_oracle_pack_dense.argtypes = [P, P, I64, ctypes.c_int, P]
+        lib.pwlq_oracle_unpack_dense.argtypes = [P, I64, ctypes.c_int, P, P]
         self._lib = lib
 
     def absmax(self, x, row_offsets=None):
@@ -306,6 +311,55 @@ class OracleLib:
                                                  int(layout)), "dequantize2")
         return y
 
+    # ---- bias correction (folded scale xi and offset beta per row) and dense (b+1)-bit storage
+    def bias_correction(self, x, bits, m, p, row_offsets=None):
+        """Returns (xi float32 [C], beta float32 [C])."""
+        flat, ro, C, n = _rows(x, row_offsets)
+        m = np.ascontiguousarray(m, dtype=np.float32)
+        p = np.ascontiguousarray(p, dtype=np.float32)
+        assert m.size == C and p.size == C
+        xi = np.empty(C, dtype=np.float32)
+        beta = np.empty(C, dtype=np.float32)
+        _check(self._lib.pwlq_oracle_bias_correction(_ptr(flat), _ptr(ro), C, n, int(bits), _ptr(m),
+                                                     _ptr(p), _ptr(xi), _ptr(beta)),
+               "bias_correction")
+        return xi, beta
+
+    def dequantize_bc(self, codes, mask, bits, m, p, xi, beta, C=None, n=None, layout=0,
+                      row_offsets=None):
+        codes = np.ascontiguousarray(codes, dtype=np.uint8)
+        mask = np.ascontiguousarray(mask, dtype=np.uint8)
+        m, p, xi, beta = (np.ascontiguousarray(v, dtype=np.float32) for v in (m, p, xi, beta))
+        if row_offsets is not None:
+            ro = np.ascontiguousarray(row_offsets, dtype=np.int64)
+            C, n, total = ro.size - 1, 0, int(ro[-1])
+        else:
+            ro, total = None, int(C) * int(n)
+        assert m.size == C and p.size == C and xi.size == C and beta.size == C
+        y = np.empty(total, dtype=np.float32)
+        _check(self._lib.pwlq_oracle_dequantize_bc(_ptr(codes), _ptr(mask), _ptr(ro), C, n,
+                                                   int(bits), _ptr(m), _ptr(p), _ptr(xi),
+                                                   _ptr(beta), _ptr(y), int(layout)),
+               "dequantize_bc")
+        return y
+
+    def pack_dense(self, codes_u8, mask, bits):
+        codes_u8 = np.ascontiguousarray(codes_u8, dtype=np.uint8)
+        mask = np.ascontiguousarray(mask, dtype=np.uint8)
+        total = codes_u8.size
+        out = np.empty((total * (bits + 1) + 7) // 8, dtype=np.uint8)
+        _check(self._lib.pwlq_oracle_pack_dense(_ptr(codes_u8), _ptr(mask), total, int(bits),
+                                                _ptr(out)), "pack_dense")
+        return out
+
+    def unpack_dense(self, stream, total, bits):
+        stream = np.ascontiguousarray(stream, dtype=np.uint8)
+        codes = np.empty(total, dtype=np.uint8)
+        mask = np.empty((total + 7) // 8, dtype=np.uint8)
+        _check(self._lib.pwlq_oracle_unpack_dense(_ptr(stream), int(total), int(bits), _ptr(codes),
+                                                  _ptr(mask)), "unpack_dense")
+        return codes, mask
+
     def params(self, m, p, bits):
         """(L, s1, inv1, s2, inv2) as binary32 values."""
         out = np.empty(5, dtype=np.float32)
@@ -385,3 +439,19 @@ def quantize2(*a, **k):
 
 def dequantize2(*a, **k):
     return _get().dequantize2(*a, **k)
+
+
+def bias_correction(*a, **k):
+    return _get().bias_correction(*a, **k)
+
+
+def dequantize_bc(*a, **k):
+    return _get().dequantize_bc(*a, **k)
+
+
+def pack_dense(*a, **k):
+    return _get().pack_dense(*a, **k)
+
+
+def unpack_dense(*a, **k):
+    return _get().unpack_dense(*a, **k)

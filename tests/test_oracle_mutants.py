@@ -6,6 +6,7 @@ import subprocess
 import pytest
 
 import test_oracle_pins as pins
+import test_oracle_bias_and_packing_pins as bpins
 import test_oracle_two_breakpoints_pins as tpins
 import test_oracle_unsigned_pins as upins
 
@@ -59,6 +60,15 @@ MUTANTS = {
     "two_bp_region_bit_order": ("region2[i >> 2] |= (uint8_t)(r << ((i & 3) * 2));",
                                 "region2[i >> 2] |= (uint8_t)(r << ((3 - (i & 3)) * 2));"),
     "two_bp_pairs_not_ordered": ("if (i < j && m > 0.0f) {", "if (i != j && m > 0.0f) {"),
+    "bc_ratio_inverted": ("xi = sqrt(vx / vy);", "xi = sqrt(vy / vx);"),
+    "bc_variance_ratio_without_sqrt": ("xi = sqrt(vx / vy);", "xi = (vx / vy);"),
+    "bc_offset_sign": ("beta_out[c] = (float)(mx - xi * my);", "beta_out[c] = (float)(mx + xi * my);"),
+    "bc_offset_before_scale": ("            float t = xi_in[c] * y[i];\n            y[i] = t + beta_in[c];",
+                               "            float t = y[i] + beta_in[c];\n            y[i] = xi_in[c] * t;"),
+    "dense_region_in_low_bit": ("int field = (codes_u8[i] & ((1 << bits) - 1)) | (r << bits);",
+                                "int field = ((codes_u8[i] & ((1 << bits) - 1)) << 1) | r;"),
+    "dense_msb_first": ("if ((field >> k) & 1) stream[pos >> 3] |= (uint8_t)(1u << (pos & 7));",
+                        "if ((field >> k) & 1) stream[pos >> 3] |= (uint8_t)(0x80u >> (pos & 7));"),
     "divide_not_reciprocal_free_pass": None,   # placeholder documented below
 }
 # 'divide_not_reciprocal': evaluating (|r| - z) / s by a true division instead of multiplying by
@@ -89,6 +99,10 @@ PIN_CALLS = [
     lambda o: tpins.test_second_breakpoint_at_m_is_the_one_breakpoint_scheme(o, 3),
     lambda o: tpins.test_pair_order_and_degenerate_rows(o),
     lambda o: tpins.test_half_step_bound_per_region(o, 4),
+    lambda o: bpins.test_corrected_rows_keep_mean_and_centred_norm(o, 4),
+    lambda o: bpins.test_hand_computed_row(o),
+    lambda o: bpins.test_dequantize_with_correction_applies_scale_then_offset(o),
+    lambda o: bpins.test_dense_stream_hand_example(o),
 ]
 
 
