@@ -214,6 +214,45 @@ int pwlq_dequantize2_ragged(const uint8_t* codes, const uint8_t* region2,
                             const float* m, const float* p1, const float* p2, float* y,
                             int code_layout, void* stream);
 
+/* Bias correction (Sec. 5.1, "Bias Correction"): quantization shifts the mean and the variance of
+ * a row; the paper compensates this by folding correction terms into the scale and the offset and
+ * prints no formula.  This library computes, per row, with y = the value pwlq_quantize delivers,
+ *     xi   = sqrt( sum (x - mean x)^2 / sum (y - mean y)^2 )      (1 when either sum is 0)
+ *     beta = mean x - xi * mean y
+ * in binary64, delivered in binary32, so that xi * y + beta has the mean and the centred norm of
+ * x.  An empty row gets xi = 1, beta = 0.
+ *   xi_out, beta_out   device, [C]
+ *   workspace          device, 256-byte aligned, pwlq_bias_workspace_bytes(C, longest row) bytes
+ * pwlq_dequantize_bc is pwlq_dequantize followed by y' = xi * y + beta in binary32 (one multiply,
+ * one add).  Asynchrony, ownership and error behaviour as for the other calls. */
+size_t pwlq_bias_workspace_bytes(int64_t C, int64_t max_n);
+int pwlq_bias_correction(const float* x, int64_t C, int64_t n, int bits, const float* m,
+                         const float* p, float* xi_out, float* beta_out, void* workspace,
+                         size_t workspace_bytes, void* stream);
+int pwlq_bias_correction_ragged(const float* x, const int64_t* row_offsets, int64_t C,
+                                int64_t total, int64_t max_n, int bits, const float* m,
+                                const float* p, float* xi_out, float* beta_out, void* workspace,
+                                size_t workspace_bytes, void* stream);
+int pwlq_dequantize_bc(const uint8_t* codes, const uint8_t* region_mask, int64_t C, int64_t n,
+                       int bits, const float* m, const float* p, const float* xi,
+                       const float* beta, float* y, int code_layout, void* stream);
+int pwlq_dequantize_bc_ragged(const uint8_t* codes, const uint8_t* region_mask,
+                              const int64_t* row_offsets, int64_t C, int64_t total, int bits,
+                              const float* m, const float* p, const float* xi, const float* beta,
+                              float* y, int code_layout, void* stream);
+
+/* Dense storage (Sec. 4: b bits per value plus one bit for the region): code and region bit of
+ * value i as one (b+1)-bit field, field = code | region << b, in bits [i (b+1), (i+1) (b+1)) of a
+ * little-endian bit stream (bit k of the stream is bit k & 7 of byte k >> 3);
+ * pwlq_dense_bytes(total, bits) = ceil(total (b+1) / 8) bytes.  pwlq_pack_dense reads codes in the
+ * PWLQ_CODES_U8 layout and the region mask of pwlq_quantize; pwlq_unpack_dense restores both.
+ * All pointers are device pointers owned by the caller. */
+size_t pwlq_dense_bytes(int64_t total, int bits);
+int pwlq_pack_dense(const uint8_t* codes_u8, const uint8_t* region_mask, int64_t total, int bits,
+                    uint8_t* stream_out, void* stream);
+int pwlq_unpack_dense(const uint8_t* stream_in, int64_t total, int bits, uint8_t* codes_u8,
+                      uint8_t* region_mask, void* stream);
+
 /* Analytic breakpoint selection, the paper's own way of choosing p (Sec. 3.3, Sec. 5.1): assume a
  * zero-mean density for each row, fit its scale, and take the breakpoint that minimises the
  * expected error of Eq. 5 -- the root of Eq. 9 on (0, m/2) -- or the closed form of Sec. 5.1.

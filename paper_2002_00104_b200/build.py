@@ -9,7 +9,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libpwlq.so")
 SOURCES = ["pwlq_api.cu", "pwlq_absmax.cu", "pwlq_search.cu", "pwlq_quantize.cu",
-           "pwlq_noalloc.cu", "pwlq_select.cu", "pwlq_search2.cu"]
+           "pwlq_noalloc.cu", "pwlq_select.cu", "pwlq_search2.cu", "pwlq_bias.cu"]
 NVCC_FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a", "-O3", "-std=c++17", "-lineinfo",
     "-fmad=false",            # no implicit FMA contraction: every fused op is an explicit fmaf

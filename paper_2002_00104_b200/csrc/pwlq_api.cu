@@ -376,6 +376,102 @@ int pwlq_dequantize2_ragged(const uint8_t* codes, const uint8_t* region2,
                             code_layout, stream);
 }
 
+size_t pwlq_bias_workspace_bytes(int64_t C, int64_t max_n) {
+    if (C < 1 || max_n < 1) return 0;
+    return pwlq::bias_workspace_bytes(C, max_n);
+}
+
+static int bias_impl(const float* x, const int64_t* ro, int64_t C, int64_t n, int64_t total,
+                     int64_t max_n, int bits, const float* m, const float* p, float* xi_out,
+                     float* beta_out, void* ws, size_t ws_bytes, void* stream) {
+    if (!x || !m || !p || !xi_out || !beta_out || bits < 2 || bits > 8 || max_n < 1)
+        return PWLQ_ERR_INVALID_ARG;
+    if (misaligned(x, 4) || misaligned(m, 4) || misaligned(p, 4) || misaligned(xi_out, 4) ||
+        misaligned(beta_out, 4) || misaligned(ro, 8))
+        return PWLQ_ERR_INVALID_ARG;
+    if (total > kMaxTotal) return PWLQ_ERR_UNSUPPORTED;
+    const int64_t tiles = (max_n + 8191) / 8192;
+    if (C * tiles > ((int64_t)1 << 31) - 1) return PWLQ_ERR_UNSUPPORTED;
+    if (!ws || ws_bytes < pwlq::bias_workspace_bytes(C, max_n)) return PWLQ_ERR_WORKSPACE;
+    if (misaligned(ws, 256)) return PWLQ_ERR_INVALID_ARG;
+    return from_cuda(pwlq::launch_bias_correction(x, ro, C, n, max_n, bits, m, p, xi_out, beta_out,
+                                                  ws, as_stream(stream)));
+}
+
+int pwlq_bias_correction(const float* x, int64_t C, int64_t n, int bits, const float* m,
+                         const float* p, float* xi_out, float* beta_out, void* workspace,
+                         size_t workspace_bytes, void* stream) {
+    if (int rc = check_rows(C, n)) return rc;
+    return bias_impl(x, nullptr, C, n, C * n, n, bits, m, p, xi_out, beta_out, workspace,
+                     workspace_bytes, stream);
+}
+
+int pwlq_bias_correction_ragged(const float* x, const int64_t* row_offsets, int64_t C,
+                                int64_t total, int64_t max_n, int bits, const float* m,
+                                const float* p, float* xi_out, float* beta_out, void* workspace,
+                                size_t workspace_bytes, void* stream) {
+    if (int rc = check_rows(C, total)) return rc;
+    if (!row_offsets || max_n > total) return PWLQ_ERR_INVALID_ARG;
+    return bias_impl(x, row_offsets, C, 0, total, max_n, bits, m, p, xi_out, beta_out, workspace,
+                     workspace_bytes, stream);
+}
+
+static int dequantize_bc_impl(const uint8_t* codes, const uint8_t* mask, const int64_t* ro,
+                              int64_t C, int64_t n, int64_t total, int bits, const float* m,
+                              const float* p, const float* xi, const float* beta, float* y,
+                              int layout, void* stream) {
+    if (!codes || !mask || !m || !p || !xi || !beta || !y || bits < 2 || bits > 8 ||
+        (layout != PWLQ_CODES_U8 && layout != PWLQ_CODES_PACKED))
+        return PWLQ_ERR_INVALID_ARG;
+    if (misaligned(m, 4) || misaligned(p, 4) || misaligned(xi, 4) || misaligned(beta, 4) ||
+        misaligned(y, 4) || misaligned(ro, 8))
+        return PWLQ_ERR_INVALID_ARG;
+    if (total > kMaxTotal) return PWLQ_ERR_UNSUPPORTED;
+    return from_cuda(pwlq::launch_dequantize_bc(codes, mask, ro, C, n, total, bits, m, p, xi, beta,
+                                                y, layout, as_stream(stream)));
+}
+
+int pwlq_dequantize_bc(const uint8_t* codes, const uint8_t* region_mask, int64_t C, int64_t n,
+                       int bits, const float* m, const float* p, const float* xi,
+                       const float* beta, float* y, int code_layout, void* stream) {
+    if (int rc = check_rows(C, n)) return rc;
+    return dequantize_bc_impl(codes, region_mask, nullptr, C, n, C * n, bits, m, p, xi, beta, y,
+                              code_layout, stream);
+}
+
+int pwlq_dequantize_bc_ragged(const uint8_t* codes, const uint8_t* region_mask,
+                              const int64_t* row_offsets, int64_t C, int64_t total, int bits,
+                              const float* m, const float* p, const float* xi, const float* beta,
+                              float* y, int code_layout, void* stream) {
+    if (int rc = check_rows(C, total)) return rc;
+    if (!row_offsets) return PWLQ_ERR_INVALID_ARG;
+    return dequantize_bc_impl(codes, region_mask, row_offsets, C, 0, total, bits, m, p, xi, beta,
+                              y, code_layout, stream);
+}
+
+size_t pwlq_dense_bytes(int64_t total, int bits) {
+    if (total < 0 || bits < 2 || bits > 8) return 0;
+    return (size_t)((total * (bits + 1) + 7) / 8);
+}
+
+int pwlq_pack_dense(const uint8_t* codes_u8, const uint8_t* region_mask, int64_t total, int bits,
+                    uint8_t* stream_out, void* stream) {
+    if (!codes_u8 || !region_mask || !stream_out || total < 1 || bits < 2 || bits > 8)
+        return PWLQ_ERR_INVALID_ARG;
+    if (total > kMaxTotal) return PWLQ_ERR_UNSUPPORTED;
+    return from_cuda(pwlq::launch_pack_dense(codes_u8, region_mask, total, bits, stream_out,
+                                             as_stream(stream)));
+}
+
+int pwlq_unpack_dense(const uint8_t* stream_in, int64_t total, int bits, uint8_t* codes_u8,
+                      uint8_t* region_mask, void* stream) {
+    if (!codes_u8 || !region_mask || !stream_in || total < 1 || bits < 2 || bits > 8)
+        return PWLQ_ERR_INVALID_ARG;
+    if (total > kMaxTotal) return PWLQ_ERR_UNSUPPORTED;
+    return from_cuda(pwlq::launch_unpack_dense(stream_in, total, bits, codes_u8, region_mask,
+                                               as_stream(stream)));
+}
+
 size_t pwlq_encode_host_scratch_bytes(int64_t C, int64_t total, int64_t max_n, int K) {
     if (C < 1 || total < 1 || max_n < 1 || K < 1 || K > PWLQ_MAX_K) return 0;
     return plan_host(C, total, max_n, K).bytes;

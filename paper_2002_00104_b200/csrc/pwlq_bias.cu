@@ -1,0 +1,272 @@
+// Bias correction (Sec. 5.1, "Bias Correction") and dense (b+1)-bit storage (Sec. 4: b bits per
+// value plus one region bit).
+//
+// Bias correction: quantization shifts the mean and the variance of a row; the correction is
+// folded into one scale xi and one offset beta per row,
+//     xi   = sqrt( sum (x - mean x)^2 / sum (y - mean y)^2 ),   beta = mean x - xi * mean y,
+// with y = pw(x) the quantizer's delivered value, so that xi * y + beta has the mean and the
+// centred norm of x.  One streaming pass: sums of (x - x0), (y - y0) and their squares in binary64
+// around a pivot (the row's first value and its quantized value), which keeps constant rows exact
+// and the variance formula well conditioned; fixed summation order.
+#include <algorithm>
+
+#include "pwlq_common.cuh"
+#include "pwlq_kernels.h"
+
+namespace pwlq {
+
+constexpr int kBcThreads = 128;
+constexpr int kBcTile = 8192;
+
+// Delivered value of the quantizer (Eq. 3) for one input.
+__device__ __forceinline__ float fake_value(float x, float m, const PieceParams& P, float Lf) {
+    if (!(m > 0.0f)) return 0.0f;
+    int q, tail;
+    float v;
+    quantize_mag(fminf(fabsf(x), m), P, Lf, q, tail, v);
+    return x < 0.0f ? -v : v;
+}
+
+__device__ __forceinline__ void finish_bias_row(int64_t row, int64_t n_row, double x0, double y0,
+                                                const double s[4], float* __restrict__ xi_out,
+                                                float* __restrict__ beta_out) {
+    double xi = 1.0, beta = 0.0;
+    if (n_row > 0) {
+        const double n = (double)n_row;
+        const double mx = x0 + s[0] / n, my = y0 + s[1] / n;
+        const double vx = s[2] - s[0] * s[0] / n, vy = s[3] - s[1] * s[1] / n;
+        if (vx > 0.0 && vy > 0.0) xi = sqrt(vx / vy);
+        beta = mx - xi * my;
+    }
+    xi_out[row] = (float)xi;
+    beta_out[row] = (float)beta;
+}
+
+// One CTA per (row, tile): sums of (x - x0), (y - y0), (x - x0)^2, (y - y0)^2 over the tile.
+__global__ void __launch_bounds__(kBcThreads)
+bias_moments_kernel(const float* __restrict__ x, Rows rows, int64_t tiles, int bits,
+                    const float* __restrict__ m_arr, const float* __restrict__ p_arr,
+                    double* __restrict__ partial, float* __restrict__ xi_out,
+                    float* __restrict__ beta_out) {
+    __shared__ double red[4][kBcThreads / 32];
+    const int64_t row = blockIdx.x / tiles, tile = blockIdx.x - row * tiles;
+    const int64_t beg = rows.begin(row), end = rows.begin(row + 1);
+    const int64_t t_beg = beg + tile * kBcTile;
+    const int64_t t_end = min(t_beg + kBcTile, end);
+    const float Lf = (float)((1 << (bits - 1)) - 1);
+    const float m = m_arr[row];
+    const PieceParams P = make_params(m, p_arr[row], Lf);
+    double x0 = 0.0, y0 = 0.0;
+    if (end > beg) {
+        const float xf = __ldg(x + beg);
+        x0 = (double)xf;
+        y0 = (double)fake_value(xf, m, P, Lf);
+    }
+    double s[4] = {0.0, 0.0, 0.0, 0.0};
+    for (int64_t i = t_beg + threadIdx.x; i < t_end; i += kBcThreads) {
+        const float xf = x[i];
+        const double dx = (double)xf - x0;
+        const double dy = (double)fake_value(xf, m, P, Lf) - y0;
+        s[0] += dx; s[1] += dy; s[2] += dx * dx; s[3] += dy * dy;
+    }
+#pragma unroll
+    for (int k = 0; k < 4; ++k)
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) s[k] += __shfl_xor_sync(0xffffffffu, s[k], o);
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    if (lane == 0)
+        for (int k = 0; k < 4; ++k) red[k][warp] = s[k];
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        for (int k = 0; k < 4; ++k) {
+            s[k] = red[k][0];
+            for (int w = 1; w < kBcThreads / 32; ++w) s[k] += red[k][w];
+        }
+        if (tiles == 1) {
+            finish_bias_row(row, end - beg, x0, y0, s, xi_out, beta_out);
+        } else {
+            for (int k = 0; k < 4; ++k) partial[4 * blockIdx.x + k] = s[k];
+        }
+    }
+}
+
+// Long rows: the tiles' sums in ascending order, then xi and beta.
+__global__ void bias_finish_kernel(const float* __restrict__ x, Rows rows, int64_t tiles, int bits,
+                                   const float* __restrict__ m_arr,
+                                   const float* __restrict__ p_arr,
+                                   const double* __restrict__ partial, float* __restrict__ xi_out,
+                                   float* __restrict__ beta_out) {
+    const int64_t row = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (row >= rows.C) return;
+    const int64_t beg = rows.begin(row), end = rows.begin(row + 1);
+    const int64_t nt = (end - beg + kBcTile - 1) / kBcTile;
+    const float Lf = (float)((1 << (bits - 1)) - 1);
+    double x0 = 0.0, y0 = 0.0;
+    if (end > beg) {
+        const float m = m_arr[row];
+        const PieceParams P = make_params(m, p_arr[row], Lf);
+        const float xf = x[beg];
+        x0 = (double)xf;
+        y0 = (double)fake_value(xf, m, P, Lf);
+    }
+    double s[4] = {0.0, 0.0, 0.0, 0.0};
+    for (int64_t t = 0; t < nt; ++t)
+        for (int k = 0; k < 4; ++k) s[k] += partial[4 * (row * tiles + t) + k];
+    finish_bias_row(row, end - beg, x0, y0, s, xi_out, beta_out);
+}
+
+size_t bias_workspace_bytes(int64_t C, int64_t max_n) {
+    const int64_t tiles = (max_n + kBcTile - 1) / kBcTile;
+    return tiles > 1 ? (size_t)(32 * C * tiles + 255) / 256 * 256 : 256;
+}
+
+cudaError_t launch_bias_correction(const float* x, const int64_t* row_offsets, int64_t C,
+                                   int64_t n, int64_t max_n, int bits, const float* m,
+                                   const float* p, float* xi_out, float* beta_out, void* workspace,
+                                   cudaStream_t stream) {
+    Rows rows{row_offsets, C, n, n > 0 ? 1.0 / (double)n : 0.0};
+    const int64_t tiles = std::max<int64_t>(1, (max_n + kBcTile - 1) / kBcTile);
+    double* partial = static_cast<double*>(workspace);
+    bias_moments_kernel<<<(unsigned)(C * tiles), kBcThreads, 0, stream>>>(
+        x, rows, tiles, bits, m, p, partial, xi_out, beta_out);
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess || tiles == 1) return e;
+    bias_finish_kernel<<<(unsigned)((C + 127) / 128), 128, 0, stream>>>(
+        x, rows, tiles, bits, m, p, partial, xi_out, beta_out);
+    return cudaGetLastError();
+}
+
+// ---------------------------------------------------------------- dequantize with the correction
+constexpr int kDbThreads = 256;
+constexpr int kDbPerThread = 16;
+
+// y' = xi * y + beta with y the value pwlq_dequantize delivers (one multiply, one add).
+template <bool PACKED>
+__global__ void __launch_bounds__(kDbThreads)
+dequantize_bc_kernel(const uint8_t* __restrict__ codes, const uint8_t* __restrict__ mask, Rows rows,
+                     int64_t total, int bits, const float* __restrict__ m_arr,
+                     const float* __restrict__ p_arr, const float* __restrict__ xi_arr,
+                     const float* __restrict__ beta_arr, float* __restrict__ y) {
+    const int64_t i0 = ((int64_t)blockIdx.x * kDbThreads + threadIdx.x) * kDbPerThread;
+    if (i0 >= total) return;
+    const float Lf = (float)((1 << (bits - 1)) - 1);
+    const int qmask = (1 << (bits - 1)) - 1;
+    const int cnt = (int)min((int64_t)kDbPerThread, total - i0);
+    int64_t row = -1, end = 0;
+    float m = 0.0f, xi = 1.0f, beta = 0.0f;
+    PieceParams P = {};
+#pragma unroll
+    for (int t = 0; t < kDbPerThread; ++t) {
+        if (t < cnt) {
+            const int64_t i = i0 + t;
+            if (row < 0 || i >= end) {
+                row = (row < 0) ? rows.row_of(i) : row + 1;
+                while (rows.begin(row + 1) <= i) ++row;          // skips empty rows
+                end = rows.begin(row + 1);
+                m = __ldg(m_arr + row);
+                P = make_params(m, __ldg(p_arr + row), Lf);
+                xi = __ldg(xi_arr + row);
+                beta = __ldg(beta_arr + row);
+            }
+            const int code = PACKED ? ((codes[i >> 1] >> ((i & 1) * 4)) & 0xF) : codes[i];
+            const int tail = (mask[i >> 3] >> (i & 7)) & 1;
+            float v = __fadd_rn(__fmul_rn((float)(code & qmask), tail ? P.s2 : P.s1),
+                                tail ? P.p : 0.0f);
+            int neg = (code >> (bits - 1)) & 1;
+            if (!(m > 0.0f)) { v = 0.0f; neg = 0; }
+            y[i] = __fadd_rn(__fmul_rn(xi, neg ? -v : v), beta);
+        }
+    }
+}
+
+cudaError_t launch_dequantize_bc(const uint8_t* codes, const uint8_t* mask,
+                                 const int64_t* row_offsets, int64_t C, int64_t n, int64_t total,
+                                 int bits, const float* m, const float* p, const float* xi,
+                                 const float* beta, float* y, int layout, cudaStream_t stream) {
+    if (total == 0) return cudaSuccess;
+    Rows rows{row_offsets, C, n, n > 0 ? 1.0 / (double)n : 0.0};
+    const bool packed = (layout == 1 && bits <= 4);
+    const int64_t per_cta = (int64_t)kDbThreads * kDbPerThread;
+    const unsigned grid = (unsigned)((total + per_cta - 1) / per_cta);
+    if (packed) dequantize_bc_kernel<true><<<grid, kDbThreads, 0, stream>>>(codes, mask, rows, total, bits, m, p, xi, beta, y);
+    else        dequantize_bc_kernel<false><<<grid, kDbThreads, 0, stream>>>(codes, mask, rows, total, bits, m, p, xi, beta, y);
+    return cudaGetLastError();
+}
+
+// ------------------------------------------------------------------------- dense bit stream
+// Value i occupies bits [i (b+1), (i+1) (b+1)) of a little-endian bit stream, field =
+// code | region << b.  Eight values make b + 1 whole bytes, so a thread that owns eight values
+// owns whole bytes of the stream.
+constexpr int kPkThreads = 256;
+
+__global__ void __launch_bounds__(kPkThreads)
+pack_dense_kernel(const uint8_t* __restrict__ codes, const uint8_t* __restrict__ mask,
+                  int64_t total, int bits, uint8_t* __restrict__ out) {
+    const int64_t g = (int64_t)blockIdx.x * kPkThreads + threadIdx.x;
+    const int64_t i0 = g * 8;
+    if (i0 >= total) return;
+    const int cnt = (int)min((int64_t)8, total - i0);
+    const int w = bits + 1;
+    const uint32_t cmask = (1u << bits) - 1u;
+    const uint32_t mb = mask[i0 >> 3];
+    unsigned long long lo = 0;
+    uint32_t hi = 0;                                  // bits 64.. of the 8 (b+1)-bit fields (b = 8)
+    for (int t = 0; t < cnt; ++t) {
+        const unsigned long long field = (codes[i0 + t] & cmask) | (((mb >> t) & 1u) << bits);
+        const int sh = t * w;
+        lo |= field << sh;
+        if (sh + w > 64) hi |= (uint32_t)(field >> (64 - sh));
+    }
+    const int nbytes = (cnt * w + 7) / 8;
+    uint8_t* dst = out + g * w;
+    for (int b = 0; b < nbytes; ++b)
+        dst[b] = (uint8_t)(b < 8 ? (lo >> (8 * b)) : (hi >> (8 * (b - 8))));
+}
+
+__global__ void __launch_bounds__(kPkThreads)
+unpack_dense_kernel(const uint8_t* __restrict__ in, int64_t total, int bits,
+                    uint8_t* __restrict__ codes, uint8_t* __restrict__ mask) {
+    const int64_t g = (int64_t)blockIdx.x * kPkThreads + threadIdx.x;
+    const int64_t i0 = g * 8;
+    if (i0 >= total) return;
+    const int cnt = (int)min((int64_t)8, total - i0);
+    const int w = bits + 1;
+    const uint32_t cmask = (1u << bits) - 1u;
+    const int nbytes = (cnt * w + 7) / 8;
+    const uint8_t* src = in + g * w;
+    unsigned long long lo = 0;
+    uint32_t hi = 0;
+    for (int b = 0; b < nbytes; ++b) {
+        if (b < 8) lo |= (unsigned long long)src[b] << (8 * b);
+        else hi |= (uint32_t)src[b] << (8 * (b - 8));
+    }
+    uint32_t mb = 0;
+    for (int t = 0; t < cnt; ++t) {
+        const int sh = t * w;
+        unsigned long long field = lo >> sh;
+        if (sh + w > 64) field |= (unsigned long long)hi << (64 - sh);
+        codes[i0 + t] = (uint8_t)((uint32_t)field & cmask);
+        mb |= (uint32_t)((field >> bits) & 1ull) << t;
+    }
+    mask[i0 >> 3] = (uint8_t)mb;
+}
+
+cudaError_t launch_pack_dense(const uint8_t* codes, const uint8_t* mask, int64_t total, int bits,
+                              uint8_t* out, cudaStream_t stream) {
+    if (total == 0) return cudaSuccess;
+    const int64_t groups = (total + 7) / 8;
+    pack_dense_kernel<<<(unsigned)((groups + kPkThreads - 1) / kPkThreads), kPkThreads, 0, stream>>>(
+        codes, mask, total, bits, out);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_unpack_dense(const uint8_t* in, int64_t total, int bits, uint8_t* codes,
+                                uint8_t* mask, cudaStream_t stream) {
+    if (total == 0) return cudaSuccess;
+    const int64_t groups = (total + 7) / 8;
+    unpack_dense_kernel<<<(unsigned)((groups + kPkThreads - 1) / kPkThreads), kPkThreads, 0, stream>>>(
+        in, total, bits, codes, mask);
+    return cudaGetLastError();
+}
+
+}  // namespace pwlq

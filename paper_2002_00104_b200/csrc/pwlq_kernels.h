@@ -63,6 +63,22 @@ cudaError_t launch_dequantize2(const uint8_t* codes, const uint8_t* region2,
                                int bits, const float* m, const float* p1, const float* p2,
                                float* y, int layout, cudaStream_t stream);
 
+// Bias correction: folded scale xi and offset beta per row; dequantize that applies them; dense
+// (b+1)-bit storage of code and region bit.
+size_t bias_workspace_bytes(int64_t C, int64_t max_n);
+cudaError_t launch_bias_correction(const float* x, const int64_t* row_offsets, int64_t C,
+                                   int64_t n, int64_t max_n, int bits, const float* m,
+                                   const float* p, float* xi_out, float* beta_out, void* workspace,
+                                   cudaStream_t stream);
+cudaError_t launch_dequantize_bc(const uint8_t* codes, const uint8_t* mask,
+                                 const int64_t* row_offsets, int64_t C, int64_t n, int64_t total,
+                                 int bits, const float* m, const float* p, const float* xi,
+                                 const float* beta, float* y, int layout, cudaStream_t stream);
+cudaError_t launch_pack_dense(const uint8_t* codes, const uint8_t* mask, int64_t total, int bits,
+                              uint8_t* out, cudaStream_t stream);
+cudaError_t launch_unpack_dense(const uint8_t* in, int64_t total, int bits, uint8_t* codes,
+                                uint8_t* mask, cudaStream_t stream);
+
 size_t select_workspace_bytes(int64_t C, int64_t max_n);
 cudaError_t launch_select_analytic(const float* x, const int64_t* row_offsets, int64_t C,
                                    int64_t n, int64_t max_n, const float* m, int model,

@@ -1,6 +1,8 @@
-"""Timing of the two-breakpoint calls (pair search, quantize, dequantize) on ResNet-50 weight shapes.
+"""Timing of the calls beyond the one-breakpoint path on ResNet-50 weight shapes: the two-breakpoint
+pair search with its quantize / dequantize, bias correction with the corrected dequantize, and the
+dense (b+1)-bit stream.
 
-    python -m paper_2002_00104_b200.pair_bench [--K 32] [--bits 4] [--reps 5]
+    python -m paper_2002_00104_b200.extras_bench [--K 32] [--bits 4] [--reps 5]
 
 Prints milliseconds per call and, for the search, value-pair evaluations per second: every value
 of a row is quantized once under each of the K (K - 1) / 2 breakpoint pairs.  The kernel reaches
@@ -61,6 +63,25 @@ def main():
     print(f"quantize2               {tq:8.3f} ms  {nbytes / tq / 1e6:8.0f} GB/s")
     print(f"dequantize2             {td:8.3f} ms  {nbytes / td / 1e6:8.0f} GB/s")
     print(f"summed squared error, one breakpoint / two breakpoints: {gain:.2f}")
+    # bias correction on the one-breakpoint result; dense stream of its codes
+    ws = torch.empty(max(256, int(pwlq.load_library().pwlq_bias_workspace_bytes(w.C, max_n))),
+                     dtype=torch.uint8, device="cuda")
+    xi, beta = pwlq.bias_correction(x, args.bits, m, one["p"], row_offsets=ro, max_n=max_n,
+                                    workspace=ws)
+    c8, k8, _ = pwlq.quantize(x, args.bits, m, one["p"], layout=0, row_offsets=ro)
+    dense = pwlq.pack_dense(c8, k8, args.bits)
+    tb = timed(lambda: pwlq.bias_correction(x, args.bits, m, one["p"], row_offsets=ro, max_n=max_n,
+                                            workspace=ws))
+    tdb = timed(lambda: pwlq.dequantize_bc(c8, k8, args.bits, m, one["p"], xi, beta,
+                                           row_offsets=ro, out=y))
+    tp = timed(lambda: pwlq.pack_dense(c8, k8, args.bits, out=dense))
+    tu = timed(lambda: pwlq.unpack_dense(dense, w.total, args.bits))
+    b8 = w.total * 4 + c8.numel() + k8.numel()
+    bp = c8.numel() + k8.numel() + dense.numel()
+    print(f"bias_correction         {tb:8.3f} ms  {w.total * 4 / tb / 1e6:8.0f} GB/s")
+    print(f"dequantize_bc           {tdb:8.3f} ms  {b8 / tdb / 1e6:8.0f} GB/s")
+    print(f"pack_dense              {tp:8.3f} ms  {bp / tp / 1e6:8.0f} GB/s")
+    print(f"unpack_dense            {tu:8.3f} ms  {bp / tu / 1e6:8.0f} GB/s")
     assert pwlq.device_status() == 0
 
 

@@ -57,6 +57,16 @@ _SIGNATURES = {
     "pwlq_quantize2_ragged": (_INT, [_P, _P, _I64, _I64, _INT, _P, _P, _P, _P, _P, _P, _INT, _P]),
     "pwlq_dequantize2": (_INT, [_P, _P, _I64, _I64, _INT, _P, _P, _P, _P, _INT, _P]),
     "pwlq_dequantize2_ragged": (_INT, [_P, _P, _P, _I64, _I64, _INT, _P, _P, _P, _P, _INT, _P]),
+    "pwlq_bias_workspace_bytes": (_SZ, [_I64, _I64]),
+    "pwlq_bias_correction": (_INT, [_P, _I64, _I64, _INT, _P, _P, _P, _P, _P, _SZ, _P]),
+    "pwlq_bias_correction_ragged": (_INT, [_P, _P, _I64, _I64, _I64, _INT, _P, _P, _P, _P, _P, _SZ,
+                                           _P]),
+    "pwlq_dequantize_bc": (_INT, [_P, _P, _I64, _I64, _INT, _P, _P, _P, _P, _P, _INT, _P]),
+    "pwlq_dequantize_bc_ragged": (_INT, [_P, _P, _P, _I64, _I64, _INT, _P, _P, _P, _P, _P, _INT,
+                                         _P]),
+    "pwlq_dense_bytes": (_SZ, [_I64, _INT]),
+    "pwlq_pack_dense": (_INT, [_P, _P, _I64, _INT, _P, _P]),
+    "pwlq_unpack_dense": (_INT, [_P, _I64, _INT, _P, _P, _P]),
     "pwlq_encode_host_scratch_bytes": (_SZ, [_I64, _I64, _I64, _INT]),
     "pwlq_encode_host": (_INT, [_P, _P, _I64, _I64, _I64, _INT, _P, _INT, _P, _P, _P, _P, _P, _P,
                                 _INT, _P, _SZ, _P, _P]),
@@ -472,6 +482,79 @@ def dequantize2(codes, region, bits, m, p1, p2, C=None, n=None, layout=CODES_U8,
                                          *tail)
     _check(rc, "pwlq_dequantize2")
     return y
+
+
+# ---- bias correction and dense (b+1)-bit storage
+def bias_correction(x, bits, m, p, row_offsets=None, max_n=None, workspace=None, stream=None):
+    """Returns (xi, beta): the folded scale and offset of every row."""
+    lib = load_library()
+    C, n, total = _shape(x, row_offsets)
+    longest = n if row_offsets is None else int(max_n)
+    need = int(lib.pwlq_bias_workspace_bytes(C, longest))
+    if workspace is None:
+        workspace = torch.empty(max(need, 256), dtype=torch.uint8, device=x.device)
+    xi = torch.empty(C, dtype=torch.float32, device=x.device)
+    beta = torch.empty(C, dtype=torch.float32, device=x.device)
+    tail = (int(bits), _dev(m, torch.float32, "m"), _dev(p, torch.float32, "p"),
+            _dev(xi, torch.float32, "xi"), _dev(beta, torch.float32, "beta"),
+            _dev(workspace, torch.uint8, "workspace"), workspace.numel(), _stream(stream))
+    if row_offsets is None:
+        rc = lib.pwlq_bias_correction(_dev(x, torch.float32, "x"), C, n, *tail)
+    else:
+        rc = lib.pwlq_bias_correction_ragged(_dev(x, torch.float32, "x"),
+                                             _dev(row_offsets, torch.int64, "row_offsets"), C,
+                                             total, longest, *tail)
+    _check(rc, "pwlq_bias_correction")
+    return xi, beta
+
+
+def dequantize_bc(codes, mask, bits, m, p, xi, beta, C=None, n=None, layout=CODES_U8,
+                  row_offsets=None, out=None, stream=None):
+    lib = load_library()
+    if row_offsets is None:
+        total = int(C) * int(n)
+    else:
+        C = row_offsets.numel() - 1
+        total = int(out.numel()) if out is not None else int(row_offsets[-1].item())
+    y = out if out is not None else torch.empty(total, dtype=torch.float32, device=codes.device)
+    tail = (int(bits), _dev(m, torch.float32, "m"), _dev(p, torch.float32, "p"),
+            _dev(xi, torch.float32, "xi"), _dev(beta, torch.float32, "beta"),
+            _dev(y, torch.float32, "y"), int(layout), _stream(stream))
+    if row_offsets is None:
+        rc = lib.pwlq_dequantize_bc(_dev(codes, torch.uint8, "codes"),
+                                    _dev(mask, torch.uint8, "mask"), int(C), int(n), *tail)
+    else:
+        rc = lib.pwlq_dequantize_bc_ragged(_dev(codes, torch.uint8, "codes"),
+                                           _dev(mask, torch.uint8, "mask"),
+                                           _dev(row_offsets, torch.int64, "row_offsets"), C, total,
+                                           *tail)
+    _check(rc, "pwlq_dequantize_bc")
+    return y
+
+
+def dense_bytes(total: int, bits: int) -> int:
+    return int(load_library().pwlq_dense_bytes(total, bits))
+
+
+def pack_dense(codes_u8, mask, bits, out=None, stream=None):
+    lib = load_library()
+    total = codes_u8.numel()
+    if out is None:
+        out = torch.empty(dense_bytes(total, bits), dtype=torch.uint8, device=codes_u8.device)
+    _check(lib.pwlq_pack_dense(_dev(codes_u8, torch.uint8, "codes"), _dev(mask, torch.uint8, "mask"),
+                               total, int(bits), _dev(out, torch.uint8, "out"), _stream(stream)),
+           "pwlq_pack_dense")
+    return out
+
+
+def unpack_dense(stream_bytes, total, bits, stream=None):
+    lib = load_library()
+    codes = torch.empty(total, dtype=torch.uint8, device=stream_bytes.device)
+    mask = torch.empty((total + 7) // 8, dtype=torch.uint8, device=stream_bytes.device)
+    _check(lib.pwlq_unpack_dense(_dev(stream_bytes, torch.uint8, "stream"), int(total), int(bits),
+                                 _dev(codes, torch.uint8, "codes"), _dev(mask, torch.uint8, "mask"),
+                                 _stream(stream)), "pwlq_unpack_dense")
+    return codes, mask
 
 
 def encode_host_scratch_bytes(C: int, total: int, max_n: int, K: int) -> int:
