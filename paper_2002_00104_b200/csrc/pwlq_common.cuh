@@ -53,6 +53,24 @@ __device__ __forceinline__ void quantize_mag(float a, const PieceParams& P, floa
     v_out = v;
 }
 
+// ---------------------------------------------------------------------------- packed fp32x2
+// Two binary32 lanes in one 64-bit register; fma.rn.f32x2 / add.rn.f32x2 take one issue slot for
+// both lanes.  (The assembler contracts a packed multiply followed by a packed add into one packed
+// FMA, so code that needs the product's own rounding uses the scalar __f*_rn intrinsics instead.)
+typedef unsigned long long u64;
+__device__ __forceinline__ u64 pack2(float lo, float hi) {
+    u64 r; asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi)); return r;
+}
+__device__ __forceinline__ void unpack2(u64 v, float& lo, float& hi) {
+    asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+}
+__device__ __forceinline__ u64 fma2(u64 a, u64 b, u64 c) {
+    u64 d; asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c)); return d;
+}
+__device__ __forceinline__ u64 add2(u64 a, u64 b) {
+    u64 d; asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b)); return d;
+}
+
 // Row lookup: dense rows have length n, ragged rows are given by ascending offsets.
 struct Rows {
     const int64_t* offsets;  // [C + 1] or nullptr (dense)

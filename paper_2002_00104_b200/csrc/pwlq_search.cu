@@ -58,20 +58,6 @@ struct SearchArgs {
     int* status;
 };
 
-// ---------------------------------------------------------------------------- packed fp32x2
-typedef unsigned long long u64;
-__device__ __forceinline__ u64 pack2(float lo, float hi) {
-    u64 r; asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi)); return r;
-}
-__device__ __forceinline__ void unpack2(u64 v, float& lo, float& hi) {
-    asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
-}
-__device__ __forceinline__ u64 fma2(u64 a, u64 b, u64 c) {
-    u64 d; asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c)); return d;
-}
-__device__ __forceinline__ u64 add2(u64 a, u64 b) {
-    u64 d; asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b)); return d;
-}
 // Unfused reconstruction error of a pair of values: e = ((q * s) + z) - a, one rounding per
 // operation.  Done with scalar intrinsics: the assembler contracts a packed mul.rn.f32x2 followed
 // by add.rn.f32x2 into one packed FMA (observed on the device: the pair loses the product's

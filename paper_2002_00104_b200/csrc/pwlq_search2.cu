@@ -7,7 +7,7 @@
 //     M_ij = error of the values p_i < a <= p_j  quantized on [p_i, p_j]
 //     T_j  = error of the values a > p_j         quantized on [p_j, m]
 // One CTA per row: the row's magnitudes are counting-sorted by candidate interval into shared
-// memory (deterministic placement), after which every term is a sum over a contiguous range of
+// memory (deterministic placement, per-warp counts and in-warp ranks), after which every term is a sum over a contiguous range of
 // the sorted tile.  A warp takes one term at a time, its lanes stride over the range (per value
 // the operation-by-operation sequence of Eq. 1, no fused multiply-add), and the lane sums are
 // added in binary64 in a fixed order.  Work per row: the honest evaluation of every (value, pair)
@@ -21,7 +21,6 @@ namespace pwlq {
 
 constexpr int kS2Threads = 256;
 constexpr int kS2Warps = kS2Threads / 32;
-constexpr int kS2HistStride = 258;          // u16 entries per bucket row (256 threads + padding)
 constexpr float kMagic2 = 12582912.0f;      // 1.5 * 2^23
 
 struct Search2Args {
@@ -44,14 +43,14 @@ struct Search2Args {
 __host__ __device__ inline size_t s2_align(size_t v) { return (v + 15) & ~(size_t)15; }
 
 // Shared-memory layout: sorted tile | bucket+rank per value | breakpoints | bucket starts |
-// per-thread bucket counts | C, T | M (triangular).
+// per-warp bucket counts | C, T | M (triangular).
 __host__ __device__ inline size_t search2_smem(int cap, int K, size_t* off) {
     size_t o = 0;
     off[0] = o; o = s2_align(o + sizeof(float) * (size_t)cap);
-    off[1] = o; o = s2_align(o + sizeof(uint16_t) * (size_t)cap);
+    off[1] = o; o = s2_align(o + sizeof(uint32_t) * (size_t)cap);
     off[2] = o; o = s2_align(o + sizeof(float) * (size_t)K);
     off[3] = o; o = s2_align(o + sizeof(int) * (size_t)(K + 2));
-    off[4] = o; o = s2_align(o + sizeof(uint16_t) * (size_t)(K + 1) * kS2HistStride);
+    off[4] = o; o = s2_align(o + sizeof(uint16_t) * (size_t)(K + 1) * kS2Warps);
     off[5] = o; o = s2_align(o + sizeof(double) * (size_t)(2 * K));
     off[6] = o; o = s2_align(o + sizeof(double) * (size_t)(K * (K - 1) / 2));
     return o;
@@ -93,6 +92,125 @@ __device__ __forceinline__ double range_error(const float* tile, int beg, int en
     return d;
 }
 
+// Squared error of Eq. 1 for one value on the range [z, z + delta] (s = delta / L, inv = L / delta),
+// added to acc; operation by operation, no fused multiply-add except the final square-and-add.
+// (No saturation needed: a - z <= delta, so the level cannot exceed L.)
+__device__ __forceinline__ float add_sq_err(float a, float z, float inv, float s, float acc) {
+    const float r = __fadd_rn(__fmul_rn(__fsub_rn(a, z), inv), kMagic2);
+    const float q = __fsub_rn(r, kMagic2);
+    const float e = __fsub_rn(__fadd_rn(__fmul_rn(q, s), z), a);
+    return __fmaf_rn(e, e, acc);
+}
+
+// Constants of one (i, j) middle region, replicated in both lanes of a packed register.
+struct MidConst {
+    float pi, pj, inv, s;
+    u64 npi2, inv2, magic2, nmagic2, ns2;
+};
+
+// Error of two values, fused form: u = a - p_i, r = fma(u, inv, magic), q = r - magic,
+// e = fma(q, -s, u).  It differs from the operation-by-operation form only in rounding.
+__device__ __forceinline__ u64 fused_err2(u64 a, const MidConst& c) {
+    const u64 u = add2(a, c.npi2);
+    const u64 r = fma2(u, c.inv2, c.magic2);
+    const u64 q = add2(r, c.nmagic2);
+    return fma2(q, c.ns2, u);
+}
+
+// Middle terms M_ij for one first breakpoint i and eight consecutive second breakpoints
+// j = jb .. jb + 7, by one warp: lane = (phase, sub) with sub = lane & 7 the candidate and
+// phase = lane >> 3 taking every fourth 128-bit vector of the sorted tile (shared-memory
+// broadcast reads: the eight candidates of a phase read the same vector).  All eight candidates
+// need the values between B_i and the smallest B_j; only the vectors around B_i and between the
+// smallest and the largest B_j need the per-value test p_i < a <= p_j.
+// EXACT: the oracle's operation-by-operation arithmetic (short rows, where the rounding of the
+// fused form would show in the sums); otherwise the fused form on packed pairs of values.
+template <bool EXACT>
+__device__ __forceinline__ void middle_terms(const float* tile, const int* start, const float* ps,
+                                             int K, int i, int jb, float Lf, double* M) {
+    const int lane = threadIdx.x & 31, sub = lane & 7, phase = lane >> 3;
+    const int j = jb + sub;
+    MidConst c;
+    c.pi = ps[i];
+    c.pj = (j < K) ? ps[j] : c.pi;                   // j >= K: empty range, contributes nothing
+    const float delta = __fsub_rn(c.pj, c.pi);
+    c.s = 0.0f; c.inv = 0.0f;
+    if (delta > 0.0f) { c.s = __fdiv_rn(delta, Lf); c.inv = __fdiv_rn(Lf, delta); }
+    c.npi2 = pack2(-c.pi, -c.pi);
+    c.inv2 = pack2(c.inv, c.inv);
+    c.magic2 = pack2(kMagic2, kMagic2);
+    c.nmagic2 = pack2(-kMagic2, -kMagic2);
+    c.ns2 = pack2(-c.s, -c.s);
+    const int b_i = start[i + 1], b_first = start[jb + 1], b_last = start[min(jb + 7, K - 1) + 1];
+    const int v_lo = b_i >> 2, v_in0 = (b_i + 3) >> 2, v_in1 = max(b_first >> 2, v_in0);
+    const int v_hi = (b_last + 3) >> 2;
+    const float4* t4 = reinterpret_cast<const float4*>(tile);
+    const ulonglong2* t2 = reinterpret_cast<const ulonglong2*>(tile);
+    double total = 0.0;
+    float acc = 0.0f;                                 // EXACT, and the tested vectors
+    u64 acc2a = 0, acc2b = 0;                         // fused interior: two packed accumulators
+    // vectors that hold B_i (at most one) and those from the smallest B_j on: tested per value
+    auto tested = [&](int v0, int v1) {
+        int run = 0;
+        for (int v = v0 + phase; v < v1; v += 4) {
+            const float4 q = t4[v];
+            const float a4[4] = {q.x, q.y, q.z, q.w};
+            if (EXACT) {
+#pragma unroll
+                for (int t = 0; t < 4; ++t) {
+                    const float with = add_sq_err(a4[t], c.pi, c.inv, c.s, acc);
+                    acc = (a4[t] > c.pi && a4[t] <= c.pj) ? with : acc;
+                }
+            } else {
+                float e[4];
+                unpack2(fused_err2(pack2(q.x, q.y), c), e[0], e[1]);
+                unpack2(fused_err2(pack2(q.z, q.w), c), e[2], e[3]);
+#pragma unroll
+                for (int t = 0; t < 4; ++t) {
+                    const float et = (a4[t] > c.pi && a4[t] <= c.pj) ? e[t] : 0.0f;
+                    acc = __fmaf_rn(et, et, acc);
+                }
+            }
+            if (++run == 128) { total += (double)acc; acc = 0.0f; run = 0; }
+        }
+    };
+    tested(v_lo, v_in0);
+    {
+        int run = 0;
+        for (int v = v_in0 + phase; v < v_in1; v += 4) {
+            if (EXACT) {
+                const float4 q = t4[v];
+                acc = add_sq_err(q.x, c.pi, c.inv, c.s, acc);
+                acc = add_sq_err(q.y, c.pi, c.inv, c.s, acc);
+                acc = add_sq_err(q.z, c.pi, c.inv, c.s, acc);
+                acc = add_sq_err(q.w, c.pi, c.inv, c.s, acc);
+            } else {
+                const ulonglong2 q = t2[v];
+                const u64 e0 = fused_err2(q.x, c), e1 = fused_err2(q.y, c);
+                acc2a = fma2(e0, e0, acc2a);
+                acc2b = fma2(e1, e1, acc2b);
+            }
+            if (++run == 128) {
+                float f0, f1, f2, f3;
+                unpack2(acc2a, f0, f1);
+                unpack2(acc2b, f2, f3);
+                total += (double)acc + ((double)f0 + (double)f1) + ((double)f2 + (double)f3);
+                acc = 0.0f; acc2a = 0; acc2b = 0; run = 0;
+            }
+        }
+    }
+    tested(v_in1, v_hi);
+    {
+        float f0, f1, f2, f3;
+        unpack2(acc2a, f0, f1);
+        unpack2(acc2b, f2, f3);
+        total += (double)acc + ((double)f0 + (double)f1) + ((double)f2 + (double)f3);
+    }
+    total += __shfl_xor_sync(0xffffffffu, total, 8);
+    total += __shfl_xor_sync(0xffffffffu, total, 16);
+    if (phase == 0 && j < K) M[pair_index(i, j, K)] = total;
+}
+
 __device__ __forceinline__ void write_degenerate2(const Search2Args& a, int64_t row) {
     if (threadIdx.x == 0) {
         a.idx1_out[row] = 0;
@@ -126,7 +244,7 @@ search2_kernel(Search2Args a) {
     size_t off[7];
     search2_smem(a.cap, K, off);
     float* tile = reinterpret_cast<float*>(smem_raw + off[0]);
-    uint16_t* jr = reinterpret_cast<uint16_t*>(smem_raw + off[1]);
+    uint32_t* jr = reinterpret_cast<uint32_t*>(smem_raw + off[1]);
     float* ps = reinterpret_cast<float*>(smem_raw + off[2]);
     int* start = reinterpret_cast<int*>(smem_raw + off[3]);
     uint16_t* hist = reinterpret_cast<uint16_t*>(smem_raw + off[4]);
@@ -140,30 +258,47 @@ search2_kernel(Search2Args a) {
         if (k > 0) unordered |= (rk < __ldg(a.ratios + k - 1));
         ps[k] = __fmul_rn(m, rk);
     }
-    for (int t = tid; t < (K + 1) * kS2HistStride; t += kS2Threads) hist[t] = 0;
+    for (int t = tid; t < (K + 1) * kS2Warps; t += kS2Threads) hist[t] = 0;
     if (__syncthreads_or(unordered)) {               // the pair search needs an ascending grid
         if (tid == 0) atomicOr(a.status, kStatusBadGrid);
         write_degenerate2(a, row);
         return;
     }
 
-    // pass 1: bucket j = #{k : p_k < a} and the value's rank among this thread's values of the
-    // bucket (a thread takes values tid, tid + 256, ...: at most 32 of them)
-    for (int i = tid; i < cnt; i += kS2Threads) {
-        const float v = fminf(fabsf(__ldg(a.x + beg + i)), m);
-        int lo = 0, hi = K;                           // p_k < v for k < lo; p_k >= v for k >= hi
-        while (lo < hi) {
-            const int mid = (lo + hi) >> 1;
-            if (ps[mid] < v) lo = mid + 1; else hi = mid;
+    // pass 1: bucket j = #{k : p_k < a} of every value and its rank among the earlier values of
+    // the same bucket in this warp's segment (each warp owns a contiguous segment of the row and
+    // walks it 32 values at a time; ranks inside a group of 32 come from match.any)
+    const unsigned full = 0xffffffffu;
+    const int seg = (((cnt + kS2Warps - 1) / kS2Warps) + 31) & ~31;
+    const int w_beg = min(warp * seg, cnt), w_end = min(w_beg + seg, cnt);
+    uint16_t* myhist = hist + warp * (K + 1);
+    for (int base = w_beg; base < w_end; base += 32) {
+        const int i = base + lane;
+        int j = K + 1;                                // "no value"
+        if (i < w_end) {
+            const float v = fminf(fabsf(__ldg(a.x + beg + i)), m);
+            int lo = 0, hi = K;                       // p_k < v for k < lo; p_k >= v for k >= hi
+            while (lo < hi) {
+                const int mid = (lo + hi) >> 1;
+                if (ps[mid] < v) lo = mid + 1; else hi = mid;
+            }
+            j = lo;
         }
-        const int rank = hist[lo * kS2HistStride + tid]++;
-        jr[i] = (uint16_t)(lo | (rank << 7));
+        const unsigned peers = __match_any_sync(full, j);
+        int before = 0;
+        if (j <= K) before = myhist[j];
+        __syncwarp();
+        if (j <= K) {
+            if (lane == __ffs(peers) - 1) myhist[j] = (uint16_t)(before + __popc(peers));
+            jr[i] = (uint32_t)j | ((uint32_t)(before + __popc(peers & ((1u << lane) - 1u))) << 7);
+        }
+        __syncwarp();
     }
     __syncthreads();
-    // bucket totals, exclusive scan over buckets, then per (bucket, thread) start positions
+    // exclusive scan over buckets, then over the warps inside a bucket
     if (tid <= K) {
         int tot = 0;
-        for (int t = 0; t < kS2Threads; ++t) tot += hist[tid * kS2HistStride + t];
+        for (int w = 0; w < kS2Warps; ++w) tot += hist[w * (K + 1) + tid];
         start[tid] = tot;
     }
     __syncthreads();
@@ -175,18 +310,19 @@ search2_kernel(Search2Args a) {
     __syncthreads();
     if (tid <= K) {
         int run = start[tid];
-        for (int t = 0; t < kS2Threads; ++t) {
-            const int c = hist[tid * kS2HistStride + t];
-            hist[tid * kS2HistStride + t] = (uint16_t)run;
+        for (int w = 0; w < kS2Warps; ++w) {
+            const int c = hist[w * (K + 1) + tid];
+            hist[w * (K + 1) + tid] = (uint16_t)run;
             run += c;
         }
     }
     __syncthreads();
-    // pass 2: placement (bucket, then thread, then the thread's own order): deterministic
-    for (int i = tid; i < cnt; i += kS2Threads) {
-        const int j = jr[i] & 0x7f, rank = jr[i] >> 7;
-        tile[hist[j * kS2HistStride + tid] + rank] = fminf(fabsf(__ldg(a.x + beg + i)), m);
+    // pass 2: placement (bucket, then warp segment, then order inside the segment): deterministic
+    for (int i = w_beg + lane; i < w_end; i += 32) {
+        const uint32_t e = jr[i];
+        tile[myhist[e & 0x7fu] + (e >> 7)] = fminf(fabsf(__ldg(a.x + beg + i)), m);
     }
+    if (tid < ((4 - (cnt & 3)) & 3)) tile[cnt + tid] = 0.0f;     // whole vectors: zeros pass no test
     __syncthreads();
 
     // evaluation: values <= p_k are the first B_k = start[k + 1] entries of the sorted tile
@@ -196,13 +332,17 @@ search2_kernel(Search2Args a) {
         else       d = range_error(tile, start[k - K + 1], cnt, ps[k - K], __fsub_rn(m, ps[k - K]), Lf);
         if (lane == 0) CT[k] = d;
     }
-    for (int i = 0; i < K - 1; ++i) {
-        const float pi = ps[i];
-        const int bi = start[i + 1];
-        for (int j = i + 1 + warp; j < K; j += kS2Warps) {
-            const double d = range_error(tile, bi, start[j + 1], pi, __fsub_rn(ps[j], pi), Lf);
-            if (lane == 0) M[pair_index(i, j, K)] = d;
-        }
+    // The fused form's rounding shows in the sums of short rows (it grows like L / sqrt(n)); rows
+    // shorter than L^2 / 2 use the operation-by-operation form.
+    const bool fused = 2 * (int64_t)cnt >= (int64_t)a.levels * a.levels;
+    {
+        int item = 0;                                  // (i, group of eight j) in a fixed order
+        for (int i = 0; i < K - 1; ++i)
+            for (int jb = i + 1; jb < K; jb += 8, ++item)
+                if ((item & (kS2Warps - 1)) == warp) {
+                    if (fused) middle_terms<false>(tile, start, ps, K, i, jb, Lf, M);
+                    else       middle_terms<true>(tile, start, ps, K, i, jb, Lf, M);
+                }
     }
     __syncthreads();
 
