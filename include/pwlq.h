@@ -282,7 +282,12 @@ int pwlq_select_analytic_ragged(const float* x, const int64_t* row_offsets, int6
  * row_offsets_host means dense [C, n] with n = total / C.  dev_scratch is device memory of at
  * least pwlq_encode_host_scratch_bytes(...) bytes, 256-byte aligned.  The call returns after
  * enqueueing; the host outputs are valid once `stream` is synchronised.  The dequantized tensor
- * stays in dev_scratch (offset reported through y_dev_out when non-NULL). */
+ * stays in dev_scratch (offset reported through y_dev_out when non-NULL).
+ * Rows are independent, so large tensors are cut into up to eight runs of whole rows whose input
+ * copy, kernels and output copies overlap: the copies run on two internal streams (created once
+ * per device, the only resources this library ever creates) chained to `stream` by events; work
+ * queued on `stream` before the call is finished before any of it starts, and `stream` ends the
+ * call.  The results are those of the four device calls run one after another. */
 size_t pwlq_encode_host_scratch_bytes(int64_t C, int64_t total, int64_t max_n, int K);
 int pwlq_encode_host(const float* x_host, const int64_t* row_offsets_host, int64_t C,
                      int64_t total, int64_t max_n, int bits, const float* ratios_host, int K,

@@ -278,7 +278,8 @@ __global__ void minmax_finalize_kernel(uint32_t* __restrict__ lo_bits,
 // MINMAX = true folds ordered keys of the maxima into out_a and of the minima into out_b.
 template <bool MINMAX>
 static cudaError_t launch_fold(const float* x, const int64_t* row_offsets, int64_t C, int64_t n,
-                               int64_t total, float* out_a, float* out_b, cudaStream_t stream) {
+                               int64_t total, float* out_a, float* out_b, cudaStream_t stream,
+                               int64_t shift) {
     cudaError_t e = cudaMemsetAsync(out_a, 0, sizeof(float) * (size_t)C, stream);
     if (e != cudaSuccess) return e;
     if (MINMAX) {
@@ -286,7 +287,7 @@ static cudaError_t launch_fold(const float* x, const int64_t* row_offsets, int64
         if (e != cudaSuccess) return e;
     }
     if (total == 0) return cudaSuccess;
-    Rows rows{row_offsets, C, n, n > 0 ? 1.0 / (double)n : 0.0};
+    Rows rows{row_offsets, C, n, n > 0 ? 1.0 / (double)n : 0.0, row_offsets ? shift : 0};
     const int64_t nspans = (total + kAbsSpan - 1) / kAbsSpan;
     static int cached[64] = {0};                       // CTAs that fit the device at once
     int dev = 0;
@@ -319,13 +320,13 @@ static cudaError_t launch_fold(const float* x, const int64_t* row_offsets, int64
 }
 
 cudaError_t launch_absmax(const float* x, const int64_t* row_offsets, int64_t C, int64_t n,
-                          int64_t total, float* m_out, cudaStream_t stream) {
-    return launch_fold<false>(x, row_offsets, C, n, total, m_out, nullptr, stream);
+                          int64_t total, float* m_out, cudaStream_t stream, int64_t shift) {
+    return launch_fold<false>(x, row_offsets, C, n, total, m_out, nullptr, stream, shift);
 }
 
 cudaError_t launch_minmax(const float* x, const int64_t* row_offsets, int64_t C, int64_t n,
                           int64_t total, float* lo_out, float* hi_out, cudaStream_t stream) {
-    cudaError_t e = launch_fold<true>(x, row_offsets, C, n, total, hi_out, lo_out, stream);
+    cudaError_t e = launch_fold<true>(x, row_offsets, C, n, total, hi_out, lo_out, stream, 0);
     if (e != cudaSuccess) return e;
     minmax_finalize_kernel<<<(unsigned)((C + 255) / 256), 256, 0, stream>>>(
         reinterpret_cast<uint32_t*>(lo_out), reinterpret_cast<uint32_t*>(hi_out), C);

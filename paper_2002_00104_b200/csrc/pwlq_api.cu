@@ -1,4 +1,7 @@
 // C ABI of the PWLQ library: argument checks and kernel launches, nothing else.
+#include <algorithm>
+#include <mutex>
+
 #include "../../include/pwlq.h"
 #include "pwlq_kernels.h"
 
@@ -117,6 +120,62 @@ HostPlan plan_host(int64_t C, int64_t total, int64_t max_n, int K) {
     h.ws = take(h.sp.bytes);
     h.bytes = o;
     return h;
+}
+
+// ---- pipelining of pwlq_encode_host
+constexpr int kHostChunks = 8;
+constexpr int64_t kHostChunkMin = 1 << 20;     // values: below this a run is not worth its launches
+
+// Internal streams and events of the host-buffer entry point, created once per device.
+struct HostPipe {
+    std::mutex mu;
+    cudaStream_t copy_in = nullptr, copy_out = nullptr;
+    cudaEvent_t start = nullptr, finished = nullptr;
+    cudaEvent_t in_done[kHostChunks] = {}, out_ready[kHostChunks] = {};
+    bool ready = false;
+};
+HostPipe* host_pipe() {
+    static HostPipe pipes[64];
+    static std::mutex create_mu;
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
+    HostPipe& p = pipes[dev];
+    std::lock_guard<std::mutex> lock(create_mu);
+    if (!p.ready) {
+        bool ok = cudaStreamCreateWithFlags(&p.copy_in, cudaStreamNonBlocking) == cudaSuccess &&
+                  cudaStreamCreateWithFlags(&p.copy_out, cudaStreamNonBlocking) == cudaSuccess &&
+                  cudaEventCreateWithFlags(&p.start, cudaEventDisableTiming) == cudaSuccess &&
+                  cudaEventCreateWithFlags(&p.finished, cudaEventDisableTiming) == cudaSuccess;
+        for (int k = 0; ok && k < kHostChunks; ++k)
+            ok = cudaEventCreateWithFlags(&p.in_done[k], cudaEventDisableTiming) == cudaSuccess &&
+                 cudaEventCreateWithFlags(&p.out_ready[k], cudaEventDisableTiming) == cudaSuccess;
+        if (!ok) return nullptr;
+        p.ready = true;
+    }
+    return &p;
+}
+
+// Cuts rows [0, C) into at most kHostChunks runs of about equal size whose first flat index is a
+// multiple of 8; row_b[0 .. runs] receives the run boundaries.  Returns the number of runs.
+int split_rows(const int64_t* ro, int64_t C, int64_t n, int64_t total, int64_t* row_b) {
+    auto flat = [&](int64_t c) { return ro ? ro[c] : c * n; };
+    int runs = 0;
+    row_b[0] = 0;
+    const int want = (int)std::min<int64_t>(kHostChunks, std::max<int64_t>(1, total / kHostChunkMin));
+    for (int k = 1; k < want; ++k) {
+        const int64_t target = total / want * k;
+        int64_t lo = row_b[runs], hi = C;               // first row with flat(row) >= target
+        while (lo < hi) {
+            const int64_t mid = (lo + hi) / 2;
+            if (flat(mid) < target) lo = mid + 1; else hi = mid;
+        }
+        int64_t r = lo;
+        for (int step = 0; r < C && (flat(r) & 7) != 0 && step < 4096; ++step) ++r;
+        if (r >= C || (flat(r) & 7) != 0 || r <= row_b[runs]) continue;
+        row_b[++runs] = r;
+    }
+    row_b[++runs] = C;
+    return runs;
 }
 
 }  // namespace
@@ -509,29 +568,72 @@ int pwlq_encode_host(const float* x_host, const int64_t* row_offsets_host, int64
     uint8_t* dc = d + h.codes;
     uint8_t* dk = d + h.mask;
     float* dy = reinterpret_cast<float*>(d + h.y);
-    const size_t cb = code_bytes(total, bits, code_layout), mb = (size_t)((total + 7) / 8);
+
+    // The rows are independent, so the tensor is cut into up to kHostChunks runs of whole rows
+    // and the three phases of a run -- copy in, compute, copy out -- overlap with those of its
+    // neighbours: the input copies queue on one internal stream, the kernels on the caller's
+    // stream, the output copies on a second internal stream, chained by events.  A run starts
+    // at a multiple of 8 values so that its slices of every buffer are vector- and byte-aligned.
+    int64_t row_b[kHostChunks + 1];
+    const int nchunks = split_rows(row_offsets_host, C, n, total, row_b);
+    auto flat = [&](int64_t c) { return row_offsets_host ? row_offsets_host[c] : c * n; };
+    HostPipe* hp = host_pipe();
+    if (!hp) return PWLQ_ERR_CUDA;
+    std::lock_guard<std::mutex> lock(hp->mu);
 
     cudaError_t e;
 #define PWLQ_TRY(call) do { e = (call); if (e != cudaSuccess) return PWLQ_ERR_CUDA; } while (0)
-    PWLQ_TRY(cudaMemcpyAsync(dx, x_host, sizeof(float) * (size_t)total, cudaMemcpyHostToDevice, st));
+    PWLQ_TRY(cudaEventRecord(hp->start, st));
+    PWLQ_TRY(cudaStreamWaitEvent(hp->copy_in, hp->start, 0));
+    PWLQ_TRY(cudaStreamWaitEvent(hp->copy_out, hp->start, 0));
     if (dro)
         PWLQ_TRY(cudaMemcpyAsync(dro, row_offsets_host, sizeof(int64_t) * (size_t)(C + 1),
-                                 cudaMemcpyHostToDevice, st));
-    PWLQ_TRY(cudaMemcpyAsync(dr, ratios_host, sizeof(float) * (size_t)K, cudaMemcpyHostToDevice, st));
-    PWLQ_TRY(pwlq::launch_absmax(dx, dro, C, n, total, dm, st));
-    PWLQ_TRY(pwlq::launch_search(dx, dro, C, n, total, bits, dr, K, dm, nullptr, dp, de, di,
-                                 nullptr, d + h.ws, h.sp, st));
-    PWLQ_TRY(pwlq::launch_quantize(dx, dro, C, n, total, bits, dm, nullptr, dp, dc, dk, nullptr,
-                                   code_layout, st));
-    PWLQ_TRY(pwlq::launch_dequantize(dc, dk, dro, C, n, total, bits, dm, nullptr, dp, dy,
-                                     code_layout, st));
-    PWLQ_TRY(cudaMemcpyAsync(m_host, dm, sizeof(float) * (size_t)C, cudaMemcpyDeviceToHost, st));
-    PWLQ_TRY(cudaMemcpyAsync(p_host, dp, sizeof(float) * (size_t)C, cudaMemcpyDeviceToHost, st));
+                                 cudaMemcpyHostToDevice, hp->copy_in));
+    PWLQ_TRY(cudaMemcpyAsync(dr, ratios_host, sizeof(float) * (size_t)K, cudaMemcpyHostToDevice,
+                             hp->copy_in));
+    const bool packed = (code_layout == PWLQ_CODES_PACKED && bits <= 4);
+    for (int k = 0; k < nchunks; ++k) {
+        const int64_t c0 = row_b[k], c1 = row_b[k + 1], f0 = flat(c0), f1 = flat(c1);
+        const int64_t Ck = c1 - c0, tk = f1 - f0;
+        const int64_t* rok = dro ? dro + c0 : nullptr;
+        PWLQ_TRY(cudaMemcpyAsync(dx + f0, x_host + f0, sizeof(float) * (size_t)tk,
+                                 cudaMemcpyHostToDevice, hp->copy_in));
+        PWLQ_TRY(cudaEventRecord(hp->in_done[k], hp->copy_in));
+        PWLQ_TRY(cudaStreamWaitEvent(st, hp->in_done[k], 0));
+        uint8_t* dck = dc + (packed ? f0 / 2 : f0);
+        uint8_t* dkk = dk + f0 / 8;
+        if (tk > 0) {
+            PWLQ_TRY(pwlq::launch_absmax(dx + f0, rok, Ck, n, tk, dm + c0, st, f0));
+            PWLQ_TRY(pwlq::launch_search(dx + f0, rok, Ck, n, tk, bits, dr, K, dm + c0, nullptr,
+                                         dp + c0, de + c0, di + c0, nullptr, d + h.ws, h.sp, st, f0,
+                                         k == 0));
+            PWLQ_TRY(pwlq::launch_quantize(dx + f0, rok, Ck, n, tk, bits, dm + c0, nullptr, dp + c0,
+                                           dck, dkk, nullptr, code_layout, st, f0));
+            PWLQ_TRY(pwlq::launch_dequantize(dck, dkk, rok, Ck, n, tk, bits, dm + c0, nullptr,
+                                             dp + c0, dy + f0, code_layout, st, f0));
+        }
+        PWLQ_TRY(cudaEventRecord(hp->out_ready[k], st));
+        PWLQ_TRY(cudaStreamWaitEvent(hp->copy_out, hp->out_ready[k], 0));
+        const size_t cbk = code_bytes(f1, bits, code_layout) - code_bytes(f0, bits, code_layout);
+        const size_t mbk = (size_t)((f1 + 7) / 8 - f0 / 8);
+        if (tk > 0) {
+            PWLQ_TRY(cudaMemcpyAsync(codes_host + (dck - dc), dck, cbk, cudaMemcpyDeviceToHost,
+                                     hp->copy_out));
+            PWLQ_TRY(cudaMemcpyAsync(region_mask_host + f0 / 8, dkk, mbk, cudaMemcpyDeviceToHost,
+                                     hp->copy_out));
+        }
+    }
+    PWLQ_TRY(cudaMemcpyAsync(m_host, dm, sizeof(float) * (size_t)C, cudaMemcpyDeviceToHost,
+                             hp->copy_out));
+    PWLQ_TRY(cudaMemcpyAsync(p_host, dp, sizeof(float) * (size_t)C, cudaMemcpyDeviceToHost,
+                             hp->copy_out));
     if (err_host)
-        PWLQ_TRY(cudaMemcpyAsync(err_host, de, sizeof(float) * (size_t)C, cudaMemcpyDeviceToHost, st));
-    PWLQ_TRY(cudaMemcpyAsync(idx_host, di, sizeof(int32_t) * (size_t)C, cudaMemcpyDeviceToHost, st));
-    PWLQ_TRY(cudaMemcpyAsync(codes_host, dc, cb, cudaMemcpyDeviceToHost, st));
-    PWLQ_TRY(cudaMemcpyAsync(region_mask_host, dk, mb, cudaMemcpyDeviceToHost, st));
+        PWLQ_TRY(cudaMemcpyAsync(err_host, de, sizeof(float) * (size_t)C, cudaMemcpyDeviceToHost,
+                                 hp->copy_out));
+    PWLQ_TRY(cudaMemcpyAsync(idx_host, di, sizeof(int32_t) * (size_t)C, cudaMemcpyDeviceToHost,
+                             hp->copy_out));
+    PWLQ_TRY(cudaEventRecord(hp->finished, hp->copy_out));
+    PWLQ_TRY(cudaStreamWaitEvent(st, hp->finished, 0));    // the caller's stream ends the call
 #undef PWLQ_TRY
     if (y_dev_out) *y_dev_out = dy;
     return PWLQ_OK;

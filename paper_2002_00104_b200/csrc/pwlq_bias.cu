@@ -124,7 +124,7 @@ cudaError_t launch_bias_correction(const float* x, const int64_t* row_offsets, i
                                    int64_t n, int64_t max_n, int bits, const float* m,
                                    const float* p, float* xi_out, float* beta_out, void* workspace,
                                    cudaStream_t stream) {
-    Rows rows{row_offsets, C, n, n > 0 ? 1.0 / (double)n : 0.0};
+    Rows rows{row_offsets, C, n, n > 0 ? 1.0 / (double)n : 0.0, 0};
     const int64_t tiles = std::max<int64_t>(1, (max_n + kBcTile - 1) / kBcTile);
     double* partial = static_cast<double*>(workspace);
     bias_moments_kernel<<<(unsigned)(C * tiles), kBcThreads, 0, stream>>>(
@@ -184,7 +184,7 @@ cudaError_t launch_dequantize_bc(const uint8_t* codes, const uint8_t* mask,
                                  int bits, const float* m, const float* p, const float* xi,
                                  const float* beta, float* y, int layout, cudaStream_t stream) {
     if (total == 0) return cudaSuccess;
-    Rows rows{row_offsets, C, n, n > 0 ? 1.0 / (double)n : 0.0};
+    Rows rows{row_offsets, C, n, n > 0 ? 1.0 / (double)n : 0.0, 0};
     const bool packed = (layout == 1 && bits <= 4);
     const int64_t per_cta = (int64_t)kDbThreads * kDbPerThread;
     const unsigned grid = (unsigned)((total + per_cta - 1) / per_cta);

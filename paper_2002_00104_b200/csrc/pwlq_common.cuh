@@ -77,6 +77,8 @@ struct Rows {
     int64_t C;
     int64_t n;               // dense row length (unused when ragged)
     double inv_n;            // 1 / n (dense), so that i / n costs a multiply and a correction
+    int64_t shift;           // ragged: subtracted from every offset (a slice of a longer list of
+                             // rows whose data pointer was advanced by `shift` values); else 0
 
     // i / n for dense rows without a 64-bit integer division (exact for i < 2^52).
     __device__ __forceinline__ int64_t dense_row(int64_t i) const {
@@ -87,15 +89,16 @@ struct Rows {
     }
 
     __device__ __forceinline__ int64_t begin(int64_t c) const {
-        return offsets ? offsets[c] : c * n;
+        return offsets ? offsets[c] - shift : c * n;
     }
     // Row that contains flat index i (0 <= i < total); empty rows are skipped.
     __device__ __forceinline__ int64_t row_of(int64_t i) const {
         if (!offsets) return dense_row(i);
-        int64_t lo = 0, hi = C;                      // offsets[lo] <= i < offsets[hi]
+        const int64_t key = i + shift;
+        int64_t lo = 0, hi = C;                      // offsets[lo] <= key < offsets[hi]
         while (hi - lo > 1) {
             const int64_t mid = (lo + hi) >> 1;
-            if (offsets[mid] <= i) lo = mid; else hi = mid;
+            if (offsets[mid] <= key) lo = mid; else hi = mid;
         }
         return lo;
     }
@@ -113,7 +116,7 @@ __device__ __forceinline__ int64_t warp_row_of(const Rows& rows, int64_t i) {
     while (hi - lo > 1) {
         const int64_t step = (hi - lo + 31) / 32;
         const int64_t q = lo + (int64_t)(lane + 1) * step;
-        const bool le = (q < hi) && (rows.offsets[q] <= i);     // true for a prefix of the lanes
+        const bool le = (q < hi) && (rows.offsets[q] - rows.shift <= i);   // true for a prefix of the lanes
         const int cnt = __popc(__ballot_sync(0xffffffffu, le));
         const int64_t new_lo = lo + (int64_t)cnt * step;
         hi = min(hi, new_lo + step);
@@ -133,7 +136,7 @@ __device__ __forceinline__ int64_t cta_row_near(const Rows& rows, int64_t i) {
     while (hi - lo > 4) {
         const int64_t step = (hi - lo + T - 1) / T;
         const int64_t q = lo + (int64_t)(threadIdx.x + 1) * step;
-        const int le = (q < hi) && (rows.offsets[q] <= i);       // true for a prefix of the threads
+        const int le = (q < hi) && (rows.offsets[q] - rows.shift <= i);    // true for a prefix of the threads
         const int cnt = __syncthreads_count(le);
         const int64_t new_lo = lo + (int64_t)cnt * step;
         hi = min(hi, new_lo + step);

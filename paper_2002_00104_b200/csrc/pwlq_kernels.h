@@ -11,8 +11,11 @@ namespace pwlq {
 // into tiles whose partial sums are combined in a fixed order by a second kernel.
 constexpr int kSearchTile = 8192;
 
+// shift (here and below): for a slice of a longer list of ragged rows -- row_offsets points at the
+// slice's first offset, the data pointers were advanced by `shift` values, `total` counts the
+// slice's values; every offset read is reduced by `shift`.  0 for whole tensors.
 cudaError_t launch_absmax(const float* x, const int64_t* row_offsets, int64_t C, int64_t n,
-                          int64_t total, float* m_out, cudaStream_t stream);
+                          int64_t total, float* m_out, cudaStream_t stream, int64_t shift = 0);
 
 // Per-row minimum and maximum (the range [m1, m2] of a one-sided / asymmetric tensor).
 cudaError_t launch_minmax(const float* x, const int64_t* row_offsets, int64_t C, int64_t n,
@@ -31,7 +34,8 @@ SearchPlan plan_search(int64_t C, int64_t max_n, int K);
 cudaError_t launch_search(const float* x, const int64_t* row_offsets, int64_t C, int64_t n,
                           int64_t total, int bits, const float* ratios, int K, const float* m,
                           const float* lo, float* p_out, float* err_out, int32_t* idx_out, float* sse_all,
-                          void* workspace, const SearchPlan& plan, cudaStream_t stream);
+                          void* workspace, const SearchPlan& plan, cudaStream_t stream,
+                          int64_t shift = 0, bool clear_status = true);
 
 // lo == nullptr: signed scheme with m = abs-max; lo != nullptr: one-sided ranges [lo, m] (m = upper
 // bounds), unsigned b-bit levels.  The same convention holds for launch_dequantize and
@@ -39,12 +43,12 @@ cudaError_t launch_search(const float* x, const int64_t* row_offsets, int64_t C,
 cudaError_t launch_quantize(const float* x, const int64_t* row_offsets, int64_t C, int64_t n,
                             int64_t total, int bits, const float* m, const float* lo,
                             const float* p, uint8_t* codes, uint8_t* mask, float* fake, int layout,
-                            cudaStream_t stream);
+                            cudaStream_t stream, int64_t shift = 0);
 
 cudaError_t launch_dequantize(const uint8_t* codes, const uint8_t* mask,
                               const int64_t* row_offsets, int64_t C, int64_t n, int64_t total,
                               int bits, const float* m, const float* lo, const float* p, float* y,
-                              int layout, cudaStream_t stream);
+                              int layout, cudaStream_t stream, int64_t shift = 0);
 
 // Two breakpoints (three regions): pair search over a grid of K <= kSearch2MaxK ascending ratios
 // for rows of at most kSearchTile values; quantize / dequantize with a two-bit region index.

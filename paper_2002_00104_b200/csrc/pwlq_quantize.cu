@@ -645,9 +645,9 @@ int quantize_timeout_flag() {
 cudaError_t launch_quantize(const float* x, const int64_t* row_offsets, int64_t C, int64_t n,
                             int64_t total, int bits, const float* m, const float* lo,
                             const float* p, uint8_t* codes, uint8_t* mask, float* fake, int layout,
-                            cudaStream_t stream) {
+                            cudaStream_t stream, int64_t shift) {
     if (total == 0) return cudaSuccess;
-    Rows rows{row_offsets, C, n, n > 0 ? 1.0 / (double)n : 0.0};
+    Rows rows{row_offsets, C, n, n > 0 ? 1.0 / (double)n : 0.0, row_offsets ? shift : 0};
     const RowArrays A{m, lo, p};
     const bool packed = (layout == 1 && bits <= 4);
     const int64_t nspans = (total + kQSpan - 1) / kQSpan;
@@ -677,9 +677,9 @@ cudaError_t launch_quantize(const float* x, const int64_t* row_offsets, int64_t 
 cudaError_t launch_dequantize(const uint8_t* codes, const uint8_t* mask,
                               const int64_t* row_offsets, int64_t C, int64_t n, int64_t total,
                               int bits, const float* m, const float* lo, const float* p, float* y,
-                              int layout, cudaStream_t stream) {
+                              int layout, cudaStream_t stream, int64_t shift) {
     if (total == 0) return cudaSuccess;
-    Rows rows{row_offsets, C, n, n > 0 ? 1.0 / (double)n : 0.0};
+    Rows rows{row_offsets, C, n, n > 0 ? 1.0 / (double)n : 0.0, row_offsets ? shift : 0};
     const RowArrays A{m, lo, p};
     const bool packed = (layout == 1 && bits <= 4);
     const int64_t nspans = (total + kQSpan - 1) / kQSpan;

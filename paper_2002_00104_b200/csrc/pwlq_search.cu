@@ -703,19 +703,20 @@ cudaError_t launch_search(const float* x, const int64_t* row_offsets, int64_t C,
                           int64_t total, int bits, const float* ratios, int K, const float* m,
                           const float* lo, float* p_out, float* err_out, int32_t* idx_out,
                           float* sse_all, void* workspace, const SearchPlan& plan,
-                          cudaStream_t stream) {
+                          cudaStream_t stream, int64_t shift, bool clear_status) {
     unsigned char* ws = static_cast<unsigned char*>(workspace);
-    cudaError_t e = cudaMemsetAsync(ws, 0, 256, stream);          // status word
+    cudaError_t e = cudaSuccess;
+    if (clear_status) e = cudaMemsetAsync(ws, 0, 256, stream);    // status word
     if (e != cudaSuccess) return e;
     if (!m && !lo) {
         float* m_ws = reinterpret_cast<float*>(ws + plan.off_m);
-        e = launch_absmax(x, row_offsets, C, n, total, m_ws, stream);
+        e = launch_absmax(x, row_offsets, C, n, total, m_ws, stream, shift);
         if (e != cudaSuccess) return e;
         m = m_ws;
     }
     SearchArgs a;
     a.x = x;
-    a.rows = Rows{row_offsets, C, n, n > 0 ? 1.0 / (double)n : 0.0};
+    a.rows = Rows{row_offsets, C, n, n > 0 ? 1.0 / (double)n : 0.0, row_offsets ? shift : 0};
     a.m = m;
     a.ratios = ratios;
     a.K = K;

@@ -405,7 +405,7 @@ cudaError_t launch_search2(const float* x, const int64_t* row_offsets, int64_t C
     if (e != cudaSuccess) return e;
     Search2Args a;
     a.x = x;
-    a.rows = Rows{row_offsets, C, n, n > 0 ? 1.0 / (double)n : 0.0};
+    a.rows = Rows{row_offsets, C, n, n > 0 ? 1.0 / (double)n : 0.0, 0};
     a.m = m;
     a.ratios = ratios;
     a.K = K;
@@ -553,7 +553,7 @@ cudaError_t launch_quantize2(const float* x, const int64_t* row_offsets, int64_t
                              const float* p2, uint8_t* codes, uint8_t* region2, float* fake,
                              int layout, cudaStream_t stream) {
     if (total == 0) return cudaSuccess;
-    Rows rows{row_offsets, C, n, n > 0 ? 1.0 / (double)n : 0.0};
+    Rows rows{row_offsets, C, n, n > 0 ? 1.0 / (double)n : 0.0, 0};
     const bool packed = (layout == 1 && bits <= 4);
     const int64_t per_cta = (int64_t)kQ2Threads * kQ2PerThread;
     const unsigned grid = (unsigned)((total + per_cta - 1) / per_cta);
@@ -572,7 +572,7 @@ cudaError_t launch_dequantize2(const uint8_t* codes, const uint8_t* region2,
                                int bits, const float* m, const float* p1, const float* p2,
                                float* y, int layout, cudaStream_t stream) {
     if (total == 0) return cudaSuccess;
-    Rows rows{row_offsets, C, n, n > 0 ? 1.0 / (double)n : 0.0};
+    Rows rows{row_offsets, C, n, n > 0 ? 1.0 / (double)n : 0.0, 0};
     const bool packed = (layout == 1 && bits <= 4);
     const int64_t per_cta = (int64_t)kQ2Threads * kQ2PerThread;
     const unsigned grid = (unsigned)((total + per_cta - 1) / per_cta);

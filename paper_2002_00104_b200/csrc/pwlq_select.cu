@@ -120,7 +120,7 @@ cudaError_t launch_select_analytic(const float* x, const int64_t* row_offsets, i
                                    int64_t n, int64_t max_n, const float* m, int model,
                                    float* p_out, float* scale_out, void* workspace,
                                    cudaStream_t stream) {
-    Rows rows{row_offsets, C, n, n > 0 ? 1.0 / (double)n : 0.0};
+    Rows rows{row_offsets, C, n, n > 0 ? 1.0 / (double)n : 0.0, 0};
     const int64_t tiles = std::max<int64_t>(1, (max_n + kSelTile - 1) / kSelTile);
     double* partial = static_cast<double*>(workspace);
     moments_kernel<<<(unsigned)(C * tiles), kSelThreads, 0, stream>>>(x, rows, tiles, partial, m,

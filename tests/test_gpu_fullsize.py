@@ -130,3 +130,53 @@ def test_laplace_matrix_sweep(pwlq, oracle, bits, K):
     g = run_path(pwlq, w, bits=bits, K=K)
     m = check_all_rows(oracle, w, g)
     check_sampled_rows(oracle, w, g, np.arange(5, w.C, 512), m)
+
+
+# ------------------------------------------------------------ host-buffer entry point, pipelined
+@pytest.mark.parametrize("layout,bits", [(1, 4), (0, 6)])
+def test_encode_host_in_several_runs_equals_the_resident_path(pwlq, oracle, layout, bits):
+    """A tensor large enough to be cut into runs of rows whose copies and kernels overlap, with row
+    lengths that put most row starts off a multiple of 8: the outputs must equal those of the four
+    device calls on the whole tensor, and sampled rows must equal the oracle."""
+    rng = np.random.default_rng(77)
+    lengths = np.tile(np.array([147, 1001, 64, 4608, 9, 2304, 33], np.int64), 1800)
+    ro = np.concatenate([[0], np.cumsum(lengths)]).astype(np.int64)
+    total, C, max_n, K = int(ro[-1]), lengths.size, int(lengths.max()), 32
+    assert total > 8 * (1 << 20)
+    x = rng.laplace(0, 0.03, total).astype(np.float32)
+    ratios = W.ratio_grid(K)
+    hx, hro = torch.from_numpy(x).pin_memory(), torch.from_numpy(ro).pin_memory()
+    cb = (total + 1) // 2 if (layout == 1 and bits <= 4) else total
+    out = {"m": torch.empty(C, dtype=torch.float32).pin_memory(),
+           "p": torch.empty(C, dtype=torch.float32).pin_memory(),
+           "err": torch.empty(C, dtype=torch.float32).pin_memory(),
+           "idx": torch.empty(C, dtype=torch.int32).pin_memory(),
+           "codes": torch.empty(cb, dtype=torch.uint8).pin_memory(),
+           "mask": torch.empty((total + 7) // 8, dtype=torch.uint8).pin_memory()}
+    scratch = torch.empty(pwlq.encode_host_scratch_bytes(C, total, max_n, K), dtype=torch.uint8,
+                          device="cuda")
+    for _ in range(2):                                # the second call reuses streams and scratch
+        pwlq.encode_host(hx, hro, C, max_n, bits, torch.from_numpy(ratios).pin_memory(), out,
+                         layout, scratch)
+    torch.cuda.synchronize()
+    xd, rod = hx.cuda(), hro.cuda()
+    m = pwlq.absmax(xd, row_offsets=rod)
+    s = pwlq.search(xd, bits, torch.from_numpy(ratios).cuda(), m=m, row_offsets=rod, max_n=max_n)
+    codes, mask, _ = pwlq.quantize(xd, bits, m, s["p"], layout=layout, row_offsets=rod)
+    torch.cuda.synchronize()
+    assert torch.equal(out["m"], m.cpu()) and torch.equal(out["idx"], s["idx"].cpu())
+    assert torch.equal(out["p"], s["p"].cpu()) and torch.equal(out["err"], s["err"].cpu())
+    assert torch.equal(out["codes"], codes.cpu()) and torch.equal(out["mask"], mask.cpu())
+    assert pwlq.device_status() == 0
+    for c in rng.choice(C, 40, replace=False):
+        xr = x[ro[c]:ro[c + 1]]
+        om = oracle.absmax(xr)
+        assert out["m"][c].item() == om[0]
+        oc, _, _ = oracle.quantize(xr, bits, om, [out["p"][c].item()], layout=0)
+        got = codes.cpu().numpy()
+        if layout == 1 and bits <= 4:
+            idx = np.arange(ro[c], ro[c + 1])
+            got_row = (got[idx >> 1] >> ((idx & 1) * 4)) & 0xF
+        else:
+            got_row = got[ro[c]:ro[c + 1]]
+        assert np.array_equal(got_row, oc)
