@@ -95,7 +95,7 @@ absmax_kernel(const float* __restrict__ x, Rows rows, int64_t total, uint32_t* _
     if (use_table && s0 < s1) {
         row0 = cta_row_near(rows, s0 * kAbsSpan);
         S.T.fetch(rows, nullptr, nullptr, nullptr, row0, nf);
-        S.T.commit(nf, 0.0f);
+        S.T.commit(nf, 0, 0.0f);
         __syncthreads();
     }
 
@@ -241,7 +241,7 @@ absmax_kernel(const float* __restrict__ x, Rows rows, int64_t total, uint32_t* _
             if (threadIdx.x == 0) atomicExch(&g_absmax_timeout, 1);
             return;
         }
-        if (has_next) { S.T.commit(nf, 0.0f); row0 = next_row0; }
+        if (has_next) { S.T.commit(nf, 0, 0.0f); row0 = next_row0; }
         if (span + kAbsStages < s1)
             S.ring.issue(it + kAbsStages, x + (span + kAbsStages) * kAbsSpan,
                          abs_bulk_bytes(span + kAbsStages, total, vec_ok));

@@ -198,7 +198,8 @@ struct SpanTable {
         return lo;
     }
     // Requests the window that starts at row r0 (no barrier; the values stay in registers).
-    // lo_arr != nullptr: one-sided ranges, m_arr holds the upper bounds.
+    // lo_arr != nullptr: one-sided ranges, m_arr holds the upper bounds.  (All loads are
+    // independent of each other, so that none of them is waited for here.)
     __device__ __forceinline__ void fetch(const Rows& rows, const float* __restrict__ m_arr,
                                           const float* __restrict__ p_arr,
                                           const float* __restrict__ lo_arr, int64_t r0,
@@ -220,14 +221,16 @@ struct SpanTable {
         f.off[kPerThread] = (threadIdx.x == 0 && r0 + CAP <= rows.C) ? rows.begin(r0 + CAP)
                                                                      : INT64_MAX;
     }
-    // Writes what fetch() requested, with the rows' constants; call between the barrier that
-    // retires the previous window and the barrier that publishes this one.
-    __device__ __forceinline__ void commit(const RowFetch<CAP>& f, float Lf) {
+    // Writes what fetch() requested, with the constants of the rows that start before `limit`
+    // (the end of the CTA's share of the storage; later rows are staged with their offsets
+    // alone); call between the barrier that retires the previous window and the barrier that
+    // publishes this one.
+    __device__ __forceinline__ void commit(const RowFetch<CAP>& f, int64_t limit, float Lf) {
 #pragma unroll
         for (int u = 0; u < kPerThread; ++u) {
             const int r = (int)threadIdx.x + u * kTableThreads;
             off[r] = f.off[u];
-            if (PARAMS) {
+            if (PARAMS && f.off[u] < limit) {
                 m[r] = f.m[u];
                 lo[r] = f.lo[u];
                 P[r] = make_params(f.m[u], f.p[u], Lf);

@@ -152,12 +152,14 @@ __device__ __forceinline__ void quantize8(const float (&xv)[8], int split, float
         const float xi = xv[t];
         const float a = UNS ? fminf(fmaxf(__fsub_rn(xi, lo), 0.0f), m) : fminf(fabsf(xi), m);
         const bool tail = a > p;
-        const float z = tail ? p : 0.0f;
-        const float inv = tail ? inv2 : inv1;
-        const float r = __fadd_rn(__fmul_rn(__fsub_rn(a, z), inv), 12582912.0f);
-        const uint32_t q = (uint32_t)min(__float_as_int(r) - 0x4B400000, Li);
-        const uint32_t xs0 = UNS ? 0u : __float_as_uint(__fadd_rn(xi, 0.0f));   // sign bit = (x < 0)
-        const uint32_t code = UNS ? q : (((xs0 >> sign_shift) & sign_unit) | q);
+        // Both pieces are evaluated and one result is kept: two more operations on the FP32 pipe
+        // instead of two selects on the (half-rate) ALU pipe.  t + 1.5 * 2^23 leaves the level in
+        // the low mantissa bits; it never exceeds L (a - z <= Delta), so no saturation is needed.
+        const float rc = __fadd_rn(__fmul_rn(a, inv1), 12582912.0f);
+        const float rt = __fadd_rn(__fmul_rn(__fsub_rn(a, p), inv2), 12582912.0f);
+        const float r = tail ? rt : rc;
+        const uint32_t q = __float_as_uint(r) & 0xFFu;
+        const uint32_t code = (UNS || !(xi < 0.0f)) ? q : (q | sign_unit);
         if (PACKED) w0 += code << (4 * t);
         else if (t < 4) w0 += code << (8 * t);
         else w1 += code << (8 * (t - 4));
@@ -166,9 +168,9 @@ __device__ __forceinline__ void quantize8(const float (&xv)[8], int split, float
             const float s1 = second ? B.s1 : A.s1;
             const float s2 = second ? B.s2 : A.s2;
             const float s = tail ? s2 : s1;
-            const float qf = fminf(__fsub_rn(r, 12582912.0f), Lf);
-            const float v = __fadd_rn(__fmul_rn(qf, s), z);
-            yv[t] = UNS ? __fadd_rn(v, lo) : __uint_as_float(__float_as_uint(v) | (xs0 & 0x80000000u));
+            const float qf = __fsub_rn(r, 12582912.0f);
+            const float v = __fadd_rn(__fmul_rn(qf, s), tail ? p : 0.0f);
+            yv[t] = UNS ? __fadd_rn(v, lo) : ((xi < 0.0f) ? -v : v);
         }
     }
 }
@@ -201,6 +203,7 @@ quantize_kernel(const float* __restrict__ x, Rows rows, int64_t total, int bits,
     const int64_t first = TABLE ? blockIdx.x * spans_per_cta : blockIdx.x;
     const int64_t stride = TABLE ? 1 : gridDim.x;
     const int64_t last = TABLE ? min(first + spans_per_cta, nspans) : nspans;        // exclusive
+    const int64_t block_end = min(last * kQSpan, total);   // rows that start later are not this CTA's
     if (threadIdx.x == 0) s_abort = 0;
     Q.ring.init();
     for (int it = 0; it < kQStages; ++it) {
@@ -212,7 +215,7 @@ quantize_kernel(const float* __restrict__ x, Rows rows, int64_t total, int bits,
     if (TABLE && first < last) {
         row0 = cta_row_near(rows, first * kQSpan);
         S.fetch(rows, A.m, A.p, A.lo, row0, nf);
-        S.commit(nf, Lf);
+        S.commit(nf, block_end, Lf);
         __syncthreads();
     }
     RowState ws;                                    // the row a warp's pass starts in (warp-uniform)
@@ -376,7 +379,7 @@ quantize_kernel(const float* __restrict__ x, Rows rows, int64_t total, int bits,
         if (ahead < last)
             Q.ring.issue(it + kQStages, x + ahead * kQSpan, q_bulk_bytes(ahead, total, vec_in));
         if (has_next) {
-            S.commit(nf, Lf);
+            S.commit(nf, block_end, Lf);
             row0 = next_row0;
             ws.beg = ws.end = 0;                     // indices into the window are stale
             __syncthreads();                        // the next window is published
@@ -468,6 +471,7 @@ dequantize_kernel(const uint8_t* __restrict__ codes, const uint8_t* __restrict__
     const int64_t first = TABLE ? blockIdx.x * spans_per_cta : blockIdx.x;
     const int64_t stride = TABLE ? 1 : gridDim.x;
     const int64_t last = TABLE ? min(first + spans_per_cta, nspans) : nspans;        // exclusive
+    const int64_t block_end = min(last * kQSpan, total);   // rows that start later are not this CTA's
     CodeRegs<PACKED> cur, nxt;
     RowState ws;                                    // the row a warp's pass starts in (warp-uniform)
     cur.load(codes, mask, first * kQSpan, total, vec_codes);
@@ -476,7 +480,7 @@ dequantize_kernel(const uint8_t* __restrict__ codes, const uint8_t* __restrict__
     if (TABLE && first < last) {
         row0 = cta_row_near(rows, first * kQSpan);
         S.fetch(rows, A.m, A.p, A.lo, row0, nf);
-        S.commit(nf, Lf);
+        S.commit(nf, block_end, Lf);
         __syncthreads();
     }
     for (int64_t span = first; span < last; span += stride) {
@@ -584,7 +588,7 @@ dequantize_kernel(const uint8_t* __restrict__ codes, const uint8_t* __restrict__
         }
         if (has_next) {
             __syncthreads();                        // the window is no longer read
-            S.commit(nf, Lf);
+            S.commit(nf, block_end, Lf);
             row0 = next_row0;
             ws.beg = ws.end = 0;                     // indices into the window are stale
             __syncthreads();                        // the next window is published
