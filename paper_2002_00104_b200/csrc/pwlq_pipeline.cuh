@@ -43,6 +43,15 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, unsigned parity) {
         if (mbar_try_wait(bar, parity)) return true;
     return false;
 }
+// The same with a pause between polls, for waits that are expected to last: the waiting warps
+// then leave the issue slots to the warps that have work.
+__device__ __forceinline__ bool mbar_wait_relaxed(uint64_t* bar, unsigned parity) {
+    for (int i = 0; i < kMaxSpins; ++i) {
+        if (mbar_try_wait(bar, parity)) return true;
+        __nanosleep(100);
+    }
+    return false;
+}
 // Makes the barrier initialisation visible to the asynchronous proxy.
 __device__ __forceinline__ void fence_barrier_init() {
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");

@@ -13,6 +13,7 @@
 #include "pwlq_common.cuh"
 #include "pwlq_kernels.h"
 #include "pwlq_pipeline.cuh"
+#include "pwlq_rowmap.cuh"
 
 namespace pwlq {
 
@@ -127,11 +128,28 @@ __device__ __forceinline__ unsigned q_bulk_bytes(int64_t span, int64_t total, in
     return (vec_in && (cnt & 3) == 0) ? (unsigned)(cnt * 4) : 0u;
 }
 
+// Bit t of x moved to bit 4 t (t < 8) resp. to bit 8 t (t < 4).
+__device__ __forceinline__ uint32_t spread_to_nibbles(uint32_t x) {
+    x = (x | (x << 12)) & 0x000F000Fu;
+    x = (x | (x << 6)) & 0x03030303u;
+    x = (x | (x << 3)) & 0x11111111u;
+    return x;
+}
+__device__ __forceinline__ uint32_t spread_to_bytes(uint32_t x) {
+    return ((x & 0xFu) * 0x00204081u) & 0x01010101u;
+}
+
 // Eight consecutive values, the first `split` of them in row A and the rest in row B (TWO = false:
-// all in row A), both rows with m > 0.  The sequence of quantize_mag with the per-row tests
-// hoisted, the level taken from the mantissa of t + 1.5 * 2^23, and the sign flag (x < 0, false
-// for -0.0) read off the sign bit of x + 0.0.  Codes are packed and region bits gathered on the
-// fly; there is no branch per value.
+// all in row A), both rows with m > 0.  The sequence of quantize_mag without a branch, a compare
+// or a select per value:
+//   - both pieces are evaluated, r_c = a L/p + 1.5 * 2^23 and r_t = (a - p) L/(m-p) + 1.5 * 2^23
+//     (the latter as (p - a) * -(L/(m-p)), the same value), and the one that applies is kept with
+//     a bitwise blend under the sign of p - a (negative exactly when a > p: p - a is never -0);
+//   - the level sits in the low mantissa bits of r (it never exceeds L, since a - z <= Delta), so
+//     r's bit patterns are summed at their code positions and the constant the eight exponent
+//     fields add up to is taken off once;
+//   - region bits and sign flags (x < 0, false for -0.0: the sign bit of x + 0.0) are gathered
+//     with one funnel shift each and spread to their positions once per eight values.
 // UNS: one-sided range, a = min(max(x - lo, 0), m), the code is the level itself and the delivered
 // value is v + lo.
 template <bool PACKED, bool WANT_FAKE, bool TWO, bool UNS>
@@ -140,39 +158,55 @@ __device__ __forceinline__ void quantize8(const float (&xv)[8], int split, float
                                           const PieceParams& B, float Lf, int Li,
                                           uint32_t sign_unit, int sign_shift, uint32_t& w0,
                                           uint32_t& w1, uint32_t& mb, float (&yv)[8]) {
-    w0 = w1 = mb = 0;
+    constexpr uint32_t kR = 0x4B400000u;                  // bit pattern of 1.5 * 2^23
+    uint32_t acc0 = 0, acc1 = 0, tails = 0, signs = 0;
 #pragma unroll
-    for (int t = 0; t < 8; ++t) {
+    for (int u = 0; u < 8; ++u) {
+        const int t = 7 - u;                              // descending: bit t of tails / signs
         const bool second = TWO && t >= split;
         const float m = second ? mB : mA;
         const float lo = second ? loB : loA;
         const float p = second ? B.p : A.p;
         const float inv1 = second ? B.inv1 : A.inv1;
-        const float inv2 = second ? B.inv2 : A.inv2;
+        const float ninv2 = -(second ? B.inv2 : A.inv2);
         const float xi = xv[t];
         const float a = UNS ? fminf(fmaxf(__fsub_rn(xi, lo), 0.0f), m) : fminf(fabsf(xi), m);
-        const bool tail = a > p;
-        // Both pieces are evaluated and one result is kept: two more operations on the FP32 pipe
-        // instead of two selects on the (half-rate) ALU pipe.  t + 1.5 * 2^23 leaves the level in
-        // the low mantissa bits; it never exceeds L (a - z <= Delta), so no saturation is needed.
-        const float rc = __fadd_rn(__fmul_rn(a, inv1), 12582912.0f);
-        const float rt = __fadd_rn(__fmul_rn(__fsub_rn(a, p), inv2), 12582912.0f);
-        const float r = tail ? rt : rc;
-        const uint32_t q = __float_as_uint(r) & 0xFFu;
-        const uint32_t code = (UNS || !(xi < 0.0f)) ? q : (q | sign_unit);
-        if (PACKED) w0 += code << (4 * t);
-        else if (t < 4) w0 += code << (8 * t);
-        else w1 += code << (8 * (t - 4));
-        mb += tail ? (1u << t) : 0u;
+        const float nu = __fsub_rn(p, a);                 // -(a - p); negative: tail piece
+        const uint32_t T = (uint32_t)((int32_t)__float_as_uint(nu) >> 31);   // all ones: tail
+        const uint32_t rc = __float_as_uint(__fadd_rn(__fmul_rn(a, inv1), 12582912.0f));
+        const uint32_t rt = __float_as_uint(__fadd_rn(__fmul_rn(nu, ninv2), 12582912.0f));
+        const uint32_t r = (rt & T) | (rc & ~T);
+        if (PACKED) acc0 += r << (4 * t);
+        else if (t < 4) acc0 += r << (8 * t);
+        else acc1 += r << (8 * (t - 4));
+        tails = __funnelshift_l(__float_as_uint(nu), tails, 1);
+        uint32_t sb = 0;
+        if (!UNS) {
+            sb = __float_as_uint(__fadd_rn(xi, 0.0f));
+            signs = __funnelshift_l(sb, signs, 1);
+        }
         if (WANT_FAKE) {
-            const float s1 = second ? B.s1 : A.s1;
-            const float s2 = second ? B.s2 : A.s2;
-            const float s = tail ? s2 : s1;
-            const float qf = __fsub_rn(r, 12582912.0f);
-            const float v = __fadd_rn(__fmul_rn(qf, s), tail ? p : 0.0f);
-            yv[t] = UNS ? __fadd_rn(v, lo) : ((xi < 0.0f) ? -v : v);
+            const uint32_t s1 = __float_as_uint(second ? B.s1 : A.s1);
+            const uint32_t s2 = __float_as_uint(second ? B.s2 : A.s2);
+            const float s = __uint_as_float((s2 & T) | (s1 & ~T));
+            const float z = __uint_as_float(__float_as_uint(p) & T);
+            const float qf = __fsub_rn(__uint_as_float(r), 12582912.0f);
+            const float v = __fadd_rn(__fmul_rn(qf, s), z);
+            yv[t] = UNS ? __fadd_rn(v, lo)
+                        : __uint_as_float(__float_as_uint(v) | (sb & 0x80000000u));
         }
     }
+    mb = tails;
+    if (PACKED) {
+        constexpr uint32_t kGarbage = (uint32_t)(0x4B400000ull * 0x11111111ull);
+        w0 = (acc0 - kGarbage) | (UNS ? 0u : spread_to_nibbles(signs) * sign_unit);
+        w1 = 0;
+    } else {
+        constexpr uint32_t kGarbage = (uint32_t)(0x4B400000ull * 0x01010101ull);
+        w0 = (acc0 - kGarbage) | (UNS ? 0u : spread_to_bytes(signs) * sign_unit);
+        w1 = (acc1 - kGarbage) | (UNS ? 0u : spread_to_bytes(signs >> 4) * sign_unit);
+    }
+    (void)kR;
 }
 
 // Persistent CTAs.  TABLE (ragged rows, or dense rows shorter than a span): each CTA walks a block
@@ -384,6 +418,243 @@ quantize_kernel(const float* __restrict__ x, Rows rows, int64_t total, int bits,
             ws.beg = ws.end = 0;                     // indices into the window are stale
             __syncthreads();                        // the next window is published
         }
+    }
+}
+
+// ------------------------------------------------------------------ several rows per span
+// Producer / consumer form of the quantizer for ragged rows and dense rows shorter than a span
+// (see pwlq_rowmap.cuh): warp kMapConsumers fills the stages (bulk copy of the span's values, row
+// map, row constants), the other warps quantize.  A consumer warp owns a contiguous eighth of the
+// span and walks it in passes of 256 values, a lane owns eight consecutive values of a pass.
+constexpr int kMapConsumers = 8;
+constexpr int kMapThreads = (kMapConsumers + 1) * 32;
+constexpr int kMapStages = 2;
+
+template <bool DATA, bool QB>
+struct MapStage {
+    alignas(128) float data[DATA ? kMapSpan : 4];
+    SpanRowMap map;
+    alignas(16) float4 qa[kMapSlots];
+    alignas(16) float4 qb[QB ? kMapSlots : 1];
+};
+
+// Row of value i and its constants straight from global memory (spans without a usable map).
+struct GlobalRow {
+    int64_t beg = 0, end = 0;
+    float m = 0.0f, lo = 0.0f;
+    PieceParams P;
+    __device__ __forceinline__ void seek(const Rows& rows, const RowArrays& A, float Lf, int64_t i) {
+        if (i >= beg && i < end) return;
+        const int64_t row = rows.row_of(i);
+        beg = rows.begin(row);
+        end = rows.begin(row + 1);
+        RowState::load_range(A, row, m, lo);
+        P = make_params(m, __ldg(A.p + row), Lf);
+    }
+};
+
+__device__ __forceinline__ PieceParams params_of(const float4 qa, const float4 qb) {
+    PieceParams P;
+    P.p = qa.y; P.inv1 = qa.z; P.inv2 = qa.w; P.s1 = qb.x; P.s2 = qb.y;
+    return P;
+}
+
+template <bool PACKED, bool WANT_FAKE, bool UNS>
+__global__ void __launch_bounds__(kMapThreads, (WANT_FAKE || UNS) ? 3 : 4)
+quantize_map_kernel(const float* __restrict__ x, Rows rows, int64_t total, int bits, RowArrays A,
+                    uint8_t* __restrict__ codes, uint8_t* __restrict__ mask,
+                    float* __restrict__ fake, int vec_in, int vec_fake, int vec_codes,
+                    int64_t spans_per_cta) {
+    constexpr bool QB = WANT_FAKE || UNS;
+    typedef MapStage<true, QB> Stage;
+    extern __shared__ __align__(128) unsigned char smem_raw[];
+    Stage* st = reinterpret_cast<Stage*>(smem_raw);
+    __shared__ uint64_t full_bar[kMapStages], empty_bar[kMapStages];
+    const unsigned full = 0xffffffffu;
+    const int Li = UNS ? (1 << bits) - 1 : (1 << (bits - 1)) - 1;    // largest level of a piece
+    const float Lf = (float)Li;
+    const uint32_t sign_unit = 1u << (bits - 1);
+    const int sign_shift = 32 - bits;
+    const int64_t nspans = (total + kMapSpan - 1) / kMapSpan;
+    const int64_t first = blockIdx.x * spans_per_cta, last = min(first + spans_per_cta, nspans);
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < kMapStages; ++s) {
+            mbar_init(&full_bar[s], 2);            // the data (or its stand-in) and the map
+            mbar_init(&empty_bar[s], kMapConsumers);
+        }
+        fence_barrier_init();
+    }
+    __syncthreads();
+    if (first >= last) return;
+
+    if (warp == kMapConsumers) {
+        // ---- producer
+        MapProducer<true, UNS> prod;
+        prod.rows = rows;
+        prod.in = RowInputs{A.m, A.lo, A.p};
+        prod.Lf = Lf;
+        prod.request(warp_row_of(rows, first * kMapSpan), true);
+        int64_t it = 0;
+        for (int64_t span = first; span < last; ++span, ++it) {
+            const int s = (int)(it % kMapStages);
+            const unsigned use = (unsigned)(it / kMapStages);
+            if (use > 0 && !mbar_wait(&empty_bar[s], (use - 1) & 1u)) {
+                if (lane == 0) atomicExch(&g_quantize_timeout, 1);
+                return;
+            }
+            const int64_t span_beg = span * kMapSpan, span_end = min(span_beg + kMapSpan, total);
+            const unsigned bytes = q_bulk_bytes(span, total, vec_in);
+            if (bytes != 0) {
+                if (lane == 0) {
+                    // the stage was last read (by the consumers, whose arrivals this warp has
+                    // waited for), not written, through the generic proxy: no proxy fence needed
+                    mbar_expect_tx(&full_bar[s], bytes);
+                    bulk_copy_g2s(st[s].data, x + span_beg, bytes, &full_bar[s]);
+                }
+            } else {                               // unaligned base or ragged tail: plain loads
+                for (int i = lane; i < (int)(span_end - span_beg); i += 32) st[s].data[i] = x[span_beg + i];
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&full_bar[s]);
+            }
+            prod.build(st[s].map, st[s].qa, QB ? st[s].qb : nullptr, span_beg, span_end,
+                       span + 1 < last);
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&full_bar[s]);
+        }
+        return;
+    }
+
+    // ---- consumers
+    int64_t it = 0;
+    for (int64_t span = first; span < last; ++span, ++it) {
+        const int s = (int)(it % kMapStages);
+        const unsigned use = (unsigned)(it / kMapStages);
+        if (!mbar_wait_relaxed(&full_bar[s], use & 1u)) {
+            if (lane == 0) atomicExch(&g_quantize_timeout, 1);
+            return;
+        }
+        const int64_t span_beg = span * kMapSpan;
+        const Stage& S = st[s];
+        const bool slow = S.map.slow != 0;
+#pragma unroll 1
+        for (int c = 0; c < 2; ++c) {
+            const int li = warp * (kMapSpan / kMapConsumers) + c * 256 + lane * 8;
+            const int64_t i0 = span_beg + li;
+            const int cnt = (int)max((int64_t)0, min((int64_t)8, total - i0));
+            const float4 xa = *reinterpret_cast<const float4*>(S.data + li);
+            const float4 xb = *reinterpret_cast<const float4*>(S.data + li + 4);
+            const float xv[8] = {xa.x, xa.y, xa.z, xa.w, xb.x, xb.y, xb.z, xb.w};
+            uint32_t w0 = 0, w1 = 0, mb = 0;
+            float yv[8];
+            if (!slow) {
+                uint32_t word;
+                const int l = map_slot(S.map, li, word);
+                const uint32_t inner = (word >> ((li & 31) + 1)) & 0x7Fu;   // starts at li+1 .. li+7
+                const float4 ca = S.qa[l];
+                const float4 cb = QB ? S.qb[l] : make_float4(0.0f, 0.0f, 0.0f, 0.0f);
+                const bool simple = inner == 0 && ca.x > 0.0f && cnt == 8;
+                if (__all_sync(full, simple)) {
+                    const PieceParams P = params_of(ca, cb);
+                    quantize8<PACKED, WANT_FAKE, false, UNS>(xv, 8, ca.x, cb.z, P, ca.x, cb.z, P, Lf,
+                                                             Li, sign_unit, sign_shift, w0, w1, mb, yv);
+                } else {
+                    const bool one = inner != 0 && (inner & (inner - 1)) == 0 && ca.x > 0.0f && cnt == 8;
+                    float4 da = ca, db = cb;
+                    int split = 8;
+                    if (one) {
+                        da = S.qa[l + 1];
+                        if (QB) db = S.qb[l + 1];
+                        split = __ffs(inner);
+                    }
+                    if (__all_sync(full, simple || (one && da.x > 0.0f))) {
+                        quantize8<PACKED, WANT_FAKE, true, UNS>(xv, split, ca.x, cb.z, params_of(ca, cb),
+                                                                da.x, db.z, params_of(da, db), Lf, Li,
+                                                                sign_unit, sign_shift, w0, w1, mb, yv);
+                    } else {
+#pragma unroll
+                        for (int t = 0; t < 8; ++t) {
+                            yv[t] = 0.0f;
+                            if (t < cnt) {
+                                const int lt = l + __popc(inner & ((1u << t) - 1u));
+                                const float4 ea = S.qa[lt];
+                                const float4 eb = QB ? S.qb[lt] : make_float4(0.0f, 0.0f, 0.0f, 0.0f);
+                                if (UNS) yv[t] = eb.z;                 // a constant row delivers lo
+                                if (ea.x > 0.0f) {
+                                    const float xi = xv[t];
+                                    const int neg = !UNS && xi < 0.0f;
+                                    int q, tail;
+                                    float v;
+                                    const float a = UNS ? fminf(fmaxf(__fsub_rn(xi, eb.z), 0.0f), ea.x)
+                                                        : fminf(fabsf(xi), ea.x);
+                                    quantize_mag(a, params_of(ea, eb), Lf, q, tail, v);
+                                    const uint32_t code = (uint32_t)((neg << (bits - 1)) | q);
+                                    if (PACKED) w0 |= code << (4 * t);
+                                    else if (t < 4) w0 |= code << (8 * t);
+                                    else w1 |= code << (8 * (t - 4));
+                                    mb |= (uint32_t)tail << t;
+                                    yv[t] = UNS ? __fadd_rn(v, eb.z) : (neg ? -v : v);
+                                }
+                            }
+                        }
+                    }
+                }
+            } else {
+                GlobalRow rs;
+#pragma unroll
+                for (int t = 0; t < 8; ++t) {
+                    yv[t] = 0.0f;
+                    if (t < cnt) {
+                        rs.seek(rows, A, Lf, i0 + t);
+                        if (UNS) yv[t] = rs.lo;
+                        if (rs.m > 0.0f) {
+                            const float xi = xv[t];
+                            const int neg = !UNS && xi < 0.0f;
+                            int q, tail;
+                            float v;
+                            const float a = UNS ? fminf(fmaxf(__fsub_rn(xi, rs.lo), 0.0f), rs.m)
+                                                : fminf(fabsf(xi), rs.m);
+                            quantize_mag(a, rs.P, Lf, q, tail, v);
+                            const uint32_t code = (uint32_t)((neg << (bits - 1)) | q);
+                            if (PACKED) w0 |= code << (4 * t);
+                            else if (t < 4) w0 |= code << (8 * t);
+                            else w1 |= code << (8 * (t - 4));
+                            mb |= (uint32_t)tail << t;
+                            yv[t] = UNS ? __fadd_rn(v, rs.lo) : (neg ? -v : v);
+                        }
+                    }
+                }
+            }
+            if (cnt == 0) continue;
+            mask[i0 >> 3] = (uint8_t)mb;
+            if (PACKED) {
+                uint8_t* dst = codes + (i0 >> 1);
+                if (vec_codes && cnt == 8) {
+                    *reinterpret_cast<uint32_t*>(dst) = w0;
+                } else {
+                    const int nb = (cnt + 1) >> 1;
+                    for (int b = 0; b < nb; ++b) dst[b] = (uint8_t)(w0 >> (8 * b));
+                }
+            } else {
+                uint8_t* dst = codes + i0;
+                if (vec_codes && cnt == 8) {
+                    *reinterpret_cast<uint2*>(dst) = make_uint2(w0, w1);
+                } else {
+                    for (int t = 0; t < cnt; ++t)
+                        dst[t] = (uint8_t)((t < 4 ? w0 : w1) >> (8 * (t & 3)));
+                }
+            }
+            if (WANT_FAKE) {
+                if (vec_fake && cnt == 8) {
+                    __stcs(reinterpret_cast<float4*>(fake + i0), make_float4(yv[0], yv[1], yv[2], yv[3]));
+                    __stcs(reinterpret_cast<float4*>(fake + i0 + 4), make_float4(yv[4], yv[5], yv[6], yv[7]));
+                } else {
+                    for (int t = 0; t < cnt; ++t) fake[i0 + t] = yv[t];
+                }
+            }
+        }
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&empty_bar[s]);
     }
 }
 
@@ -661,6 +932,15 @@ cudaError_t launch_quantize(const float* x, const int64_t* row_offsets, int64_t 
     const bool table = row_offsets != nullptr || n < kQSpan;    // several rows per span
 #define PWLQ_LAUNCH_QUANTIZE(PK, FK, RG, UN)                                                      \
     do {                                                                                          \
+        if (RG) {                                                                                 \
+            const size_t msmem = sizeof(MapStage<true, FK || UN>) * kMapStages;                   \
+            const SpanGrid g = span_grid((const void*)quantize_map_kernel<PK, FK, UN>,            \
+                                         kMapThreads, msmem, nspans, true);                       \
+            quantize_map_kernel<PK, FK, UN><<<g.grid, kMapThreads, msmem, stream>>>(              \
+                x, rows, total, bits, A, codes, mask, fake, vec_in, vec_fake, vec_codes,          \
+                g.per_cta);                                                                       \
+            break;                                                                                \
+        }                                                                                         \
         const SpanGrid g = span_grid((const void*)quantize_kernel<PK, FK, RG, UN>, kQThreads,     \
                                      smem, nspans, RG);                                           \
         quantize_kernel<PK, FK, RG, UN><<<g.grid, kQThreads, smem, stream>>>(                     \

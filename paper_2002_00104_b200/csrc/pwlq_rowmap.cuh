@@ -1,0 +1,204 @@
+// Row maps for the streaming kernels when a span of the flat storage holds several rows (ragged
+// rows, and dense rows shorter than a span).
+//
+// A CTA is one producer warp and a number of consumer warps.  For every span of kMapSpan values
+// the producer describes the rows that overlap it in a stage of shared memory: a bitmap with one
+// bit per position at which a row starts, the number of starts before every 32-bit word of the
+// bitmap, and the rows' constants in the order in which the rows appear ("slots"; slot 0 is the
+// row that holds the span's first value).  A consumer lane then finds the slot of any position
+// with two shared-memory reads and a population count, and sees the row starts among the values
+// it owns directly in the bitmap; it never searches and never touches the row arrays in global
+// memory.  The producer walks the spans in order, so the first row of a span is where the previous
+// span ended.  It keeps the offsets and inputs of the 33 to 64 rows from that row on in registers
+// (two chunks of 32 consecutive rows, one row per lane) and requests a new chunk as soon as the
+// walk has left an old one, so that with rows of a few hundred values or more its loads are
+// several spans ahead of their use.  Stages are handed over through mbarriers (full: producer ->
+// consumers, empty: consumers -> producer), which keeps the producer's global round trips off the
+// consumers' path.
+//
+// Spans the map cannot describe (more than kMapSlots rows, or empty rows inside the span) are
+// marked `slow`; consumers then look every value's row up in global memory.
+#pragma once
+
+#include "pwlq_common.cuh"
+#include "pwlq_pipeline.cuh"
+
+namespace pwlq {
+
+constexpr int kMapSpan = 4096;                 // values per span
+constexpr int kMapWords = kMapSpan / 32;
+constexpr int kMapRounds = 17;                 // rounds of 32 rows the producer looks at per span
+constexpr int kMapSlots = kMapRounds * 32;     // rows a map can describe (rows of >= 8 values fit)
+
+struct SpanRowMap {
+    uint32_t bits[kMapWords];     // bit i: a row starts at position i of the span (i > 0)
+    uint16_t before[kMapWords];   // number of set bits in the words before this one
+    int64_t first_row;            // row of slot 0
+    int32_t slow;                 // 1: the map does not describe the span
+    int32_t pad;
+};
+
+// Slot of the row that holds position li of the span; `word` returns the bitmap word of li.
+__device__ __forceinline__ int map_slot(const SpanRowMap& M, int li, uint32_t& word) {
+    word = M.bits[li >> 5];
+    return (int)M.before[li >> 5] + __popc(word & (0xFFFFFFFFu >> (31 - (li & 31))));
+}
+
+__device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_addr(bar)) : "memory");
+}
+
+// Per-row inputs of the quantizer: m = abs-max and lo = nullptr (signed scheme), or m = upper and
+// lo = lower bound of a one-sided range; p = breakpoint.
+struct RowInputs {
+    const float* __restrict__ m;
+    const float* __restrict__ lo;
+    const float* __restrict__ p;
+};
+
+// Constants of one row as the consumers read them: qa = (m, p, L/p, L/(m-p)),
+// qb = (p/L, (m-p)/L, lo, 0); m is the range width (abs-max, or upper - lower bound).
+__device__ __forceinline__ void store_row_consts(float4* qa, float4* qb, int slot, float m, float p,
+                                                 float lo, float Lf) {
+    const PieceParams P = make_params(m, p, Lf);
+    qa[slot] = make_float4(m, P.p, P.inv1, P.inv2);
+    if (qb) qb[slot] = make_float4(P.s1, P.s2, lo, 0.0f);
+}
+
+// The producer warp's view of the rows.  Rows are looked at in chunks of 32 consecutive rows
+// (chunk c = rows 32 c .. 32 c + 31, lane = row % 32); the two chunks from the current first row
+// on are held in registers.  Every member function is called by all 32 lanes.
+template <bool PARAMS, bool UNS>
+struct MapProducer {
+    Rows rows;
+    RowInputs in;
+    float Lf;
+    int64_t rf;                 // row that holds the first value of the next span
+    int64_t ch0, ch1;           // chunk held in (o0, m0, p0, lo0): even chunks; (o1, ...): odd chunks
+    int64_t o0, o1;             // offset of row 32 ch + lane (INT64_MAX past the last offset)
+    float m0, p0, lo0, m1, p1, lo1;
+
+    __device__ __forceinline__ void load_inputs(int64_t r, float& mv, float& pv, float& lov) const {
+        mv = __ldg(in.m + r);
+        pv = __ldg(in.p + r);
+        lov = 0.0f;
+        if (UNS) lov = __ldg(in.lo + r);            // m stays the upper bound until it is used
+    }
+    __device__ __forceinline__ void load_chunk(int64_t c, int64_t& o, float& mv, float& pv,
+                                               float& lov) const {
+        const int64_t r = 32 * c + (threadIdx.x & 31);
+        // as stored (ragged: before the slice's shift is taken off), so that nothing here waits
+        // for the load
+        o = (r <= rows.C) ? (rows.offsets ? __ldg(rows.offsets + r) : r * rows.n) : INT64_MAX;
+        mv = pv = lov = 0.0f;
+        if (PARAMS && r < rows.C) load_inputs(r, mv, pv, lov);
+    }
+    // Makes the registers hold the two chunks from row `first_row` on; chunks already held are
+    // kept, nothing is waited for.
+    __device__ __forceinline__ void request(int64_t first_row, bool fresh) {
+        rf = first_row;
+        const int64_t c = rf >> 5;
+        const int64_t want0 = (c & 1) ? c + 1 : c, want1 = (c & 1) ? c : c + 1;
+        if (fresh || ch0 != want0) { ch0 = want0; load_chunk(want0, o0, m0, p0, lo0); }
+        if (fresh || ch1 != want1) { ch1 = want1; load_chunk(want1, o1, m1, p1, lo1); }
+    }
+    // Writes the map of the span [span_beg, span_end), whose first value lies in row rf, and the
+    // constants of its rows; then moves on to the first row of the next span (more == true).
+    __device__ __forceinline__ void build(SpanRowMap& M, float4* qa, float4* qb, int64_t span_beg,
+                                          int64_t span_end, bool more) {
+        const unsigned full = 0xffffffffu;
+        const int lane = threadIdx.x & 31;
+        reinterpret_cast<uint4*>(M.bits)[lane] = make_uint4(0u, 0u, 0u, 0u);
+        __syncwarp();
+        const int64_t this_rf = rf;
+        const int64_t c0 = this_rf >> 5;
+        const int l0 = (int)(this_rf & 31);        // slot s = 32 k + lane - l0 in round k
+        int total_in = 0;
+        bool open = true;                          // every row seen so far starts in the span
+        // offsets of the first two rows that do not start inside the span
+        int64_t os = 0, os1 = 0;
+        bool have_os = false, have_os1 = false;
+        for (int k = 0; open && k < kMapRounds; ++k) {
+            const int64_t c = c0 + k;
+            const int s = 32 * k + lane - l0;
+            const int64_t r = 32 * c + lane;
+            int64_t off;
+            float mv, pv, lov;
+            if (k < 2) {                           // held in registers
+                const bool odd = (c & 1) != 0;
+                off = odd ? o1 : o0;
+                mv = odd ? m1 : m0; pv = odd ? p1 : p0; lov = odd ? lo1 : lo0;
+            } else {                               // short rows: fetched now
+                off = (r <= rows.C) ? (rows.offsets ? __ldg(rows.offsets + r) : r * rows.n) : INT64_MAX;
+                mv = pv = lov = 0.0f;
+            }
+            if (off != INT64_MAX) off -= rows.shift;
+            const bool inside = s >= 0 && r < rows.C && (s == 0 || off < span_end);
+            if (inside) {
+                if (s > 0) {
+                    const int pos = (int)(off - span_beg);
+                    const uint32_t bit = 1u << (pos & 31);
+                    atomicOr(&M.bits[pos >> 5], bit);
+                }
+                if (PARAMS) {
+                    if (k >= 2) load_inputs(r, mv, pv, lov);
+                    if (UNS) mv = __fsub_rn(mv, lov);              // range width
+                    store_row_consts(qa, qb, s, mv, pv, lov, Lf);
+                }
+            }
+            const unsigned in_mask = __ballot_sync(full, inside);
+            const int cnt = __popc(in_mask);
+            total_in += cnt;
+            // the rows inside are the lanes from (k == 0 ? l0 : 0) up to some lane
+            const int first_out = (k == 0 ? l0 : 0) + cnt;
+            open = first_out == 32;
+            if (!open) {
+                os = __shfl_sync(full, off, first_out);
+                have_os = true;
+                if (first_out < 31) {
+                    os1 = __shfl_sync(full, off, first_out + 1);
+                    have_os1 = true;
+                }
+            }
+        }
+        const bool overflow = open;                // all rounds full: there may be more rows
+        if (more) {
+            // the row that holds position span_end (the last row that starts at or before it)
+            int64_t rn;
+            if (overflow) {
+                rn = warp_row_of(rows, span_end);
+            } else {
+                const int64_t rs = this_rf + total_in;              // first row not inside, <= C
+                if (!have_os) os = rows.begin(rs);
+                if (rs < rows.C && os == span_end) {
+                    if (!have_os1) os1 = (rs + 1 <= rows.C) ? rows.begin(rs + 1) : INT64_MAX;
+                    const bool empty_next = rs + 1 < rows.C && os1 == span_end;
+                    rn = empty_next ? warp_row_of(rows, span_end) : rs;
+                } else {
+                    rn = rs - 1;
+                }
+            }
+            request(rn, false);
+        }
+        __syncwarp();
+        const uint4 w = reinterpret_cast<const uint4*>(M.bits)[lane];
+        const int c0b = __popc(w.x), c1b = __popc(w.y), c2b = __popc(w.z), c3b = __popc(w.w);
+        const int tot = c0b + c1b + c2b + c3b;
+        int incl = tot;
+#pragma unroll
+        for (int d = 1; d < 32; d <<= 1) {
+            const int t = __shfl_up_sync(full, incl, d);
+            if (lane >= d) incl += t;
+        }
+        const uint32_t e0 = (uint32_t)(incl - tot), e1 = e0 + c0b, e2 = e1 + c1b, e3 = e2 + c2b;
+        reinterpret_cast<uint2*>(M.before)[lane] = make_uint2(e0 | (e1 << 16), e2 | (e3 << 16));
+        // rows that start at the same position (empty rows) set one bit between them
+        const bool dup = __shfl_sync(full, incl, 31) != total_in - 1;
+        if (lane == 0) {
+            M.first_row = this_rf;
+            M.slow = (dup || overflow) ? 1 : 0;
+        }
+    }
+};
+
+}  // namespace pwlq
