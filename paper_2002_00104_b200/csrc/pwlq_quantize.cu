@@ -459,7 +459,7 @@ __device__ __forceinline__ PieceParams params_of(const float4 qa, const float4 q
     return P;
 }
 
-template <bool PACKED, bool WANT_FAKE, bool UNS>
+template <bool PACKED, bool WANT_FAKE, bool UNS, bool LONG>
 __global__ void __launch_bounds__(kMapThreads, (WANT_FAKE || UNS) ? 3 : 4)
 quantize_map_kernel(const float* __restrict__ x, Rows rows, int64_t total, int bits, RowArrays A,
                     uint8_t* __restrict__ codes, uint8_t* __restrict__ mask,
@@ -494,7 +494,10 @@ quantize_map_kernel(const float* __restrict__ x, Rows rows, int64_t total, int b
         prod.rows = rows;
         prod.in = RowInputs{A.m, A.lo, A.p};
         prod.Lf = Lf;
-        prod.request(warp_row_of(rows, first * kMapSpan), true);
+        // LONG: dense rows of at least a span, the map follows from the row length
+        constexpr bool long_rows = LONG;
+        if (long_rows) prod.request_long(rows.dense_row(first * kMapSpan));
+        else prod.request(warp_row_of(rows, first * kMapSpan), true);
         int64_t it = 0;
         for (int64_t span = first; span < last; ++span, ++it) {
             const int s = (int)(it % kMapStages);
@@ -517,8 +520,12 @@ quantize_map_kernel(const float* __restrict__ x, Rows rows, int64_t total, int b
                 __syncwarp();
                 if (lane == 0) mbar_arrive(&full_bar[s]);
             }
-            prod.build(st[s].map, st[s].qa, QB ? st[s].qb : nullptr, span_beg, span_end,
-                       span + 1 < last);
+            if (long_rows)
+                prod.build_long(st[s].map, st[s].qa, QB ? st[s].qb : nullptr, s, span_beg, span_end,
+                                span + 1 < last);
+            else
+                prod.build(st[s].map, st[s].qa, QB ? st[s].qb : nullptr, span_beg, span_end,
+                           span + 1 < last);
             __syncwarp();
             if (lane == 0) mbar_arrive(&full_bar[s]);
         }
@@ -929,16 +936,25 @@ cudaError_t launch_quantize(const float* x, const int64_t* row_offsets, int64_t 
     const int vec_in = aligned(x, 16), vec_fake = fake ? aligned(fake, 16) : 0;
     const size_t smem = sizeof(QuantizeSmem);
     const int vec_codes = packed ? aligned(codes, 4) : aligned(codes, 8);
-    const bool table = row_offsets != nullptr || n < kQSpan;    // several rows per span
+    const bool table = true;
+    const bool long_rows = row_offsets == nullptr && n >= kMapSpan;   // the map follows from n
 #define PWLQ_LAUNCH_QUANTIZE(PK, FK, RG, UN)                                                      \
     do {                                                                                          \
         if (RG) {                                                                                 \
             const size_t msmem = sizeof(MapStage<true, FK || UN>) * kMapStages;                   \
-            const SpanGrid g = span_grid((const void*)quantize_map_kernel<PK, FK, UN>,            \
-                                         kMapThreads, msmem, nspans, true);                       \
-            quantize_map_kernel<PK, FK, UN><<<g.grid, kMapThreads, msmem, stream>>>(              \
-                x, rows, total, bits, A, codes, mask, fake, vec_in, vec_fake, vec_codes,          \
-                g.per_cta);                                                                       \
+            if (long_rows) {                                                                      \
+                const SpanGrid g = span_grid((const void*)quantize_map_kernel<PK, FK, UN, true>,  \
+                                             kMapThreads, msmem, nspans, true);                   \
+                quantize_map_kernel<PK, FK, UN, true><<<g.grid, kMapThreads, msmem, stream>>>(    \
+                    x, rows, total, bits, A, codes, mask, fake, vec_in, vec_fake, vec_codes,      \
+                    g.per_cta);                                                                   \
+            } else {                                                                              \
+                const SpanGrid g = span_grid((const void*)quantize_map_kernel<PK, FK, UN, false>, \
+                                             kMapThreads, msmem, nspans, true);                   \
+                quantize_map_kernel<PK, FK, UN, false><<<g.grid, kMapThreads, msmem, stream>>>(   \
+                    x, rows, total, bits, A, codes, mask, fake, vec_in, vec_fake, vec_codes,      \
+                    g.per_cta);                                                                   \
+            }                                                                                     \
             break;                                                                                \
         }                                                                                         \
         const SpanGrid g = span_grid((const void*)quantize_kernel<PK, FK, RG, UN>, kQThreads,     \

@@ -199,6 +199,59 @@ struct MapProducer {
             M.slow = (dup || overflow) ? 1 : 0;
         }
     }
+
+    // ---- dense rows of at least kMapSpan values: a span holds one row, or the end of one and
+    // the beginning of the next.  Everything follows from the row length; the inputs of the
+    // current and the next row are held in registers (every lane the same), and a stage whose
+    // slot 0 already belongs to the row is left as it is.
+    int64_t long_end;           // end of row rf
+    int64_t stage_first[2];     // per stage: the row its slot 0 was written for, or -1
+    bool stage_plain[2];        // per stage: the map says "one row, no start"
+
+    __device__ __forceinline__ void request_long(int64_t first_row) {
+        rf = first_row;
+        long_end = (rf + 1) * rows.n;
+        m0 = p0 = lo0 = m1 = p1 = lo1 = 0.0f;
+        if (PARAMS) {
+            load_inputs(rf, m0, p0, lo0);
+            if (rf + 1 < rows.C) load_inputs(rf + 1, m1, p1, lo1);
+        }
+        stage_first[0] = stage_first[1] = -1;
+        stage_plain[0] = stage_plain[1] = false;
+    }
+    __device__ __forceinline__ void build_long(SpanRowMap& M, float4* qa, float4* qb, int stage,
+                                               int64_t span_beg, int64_t span_end, bool more) {
+        const int lane = threadIdx.x & 31;
+        const bool starts = long_end < span_end;          // row rf + 1 begins inside the span
+        const bool have_first = (stage == 0 ? stage_first[0] : stage_first[1]) == rf;
+        const bool plain = stage == 0 ? stage_plain[0] : stage_plain[1];
+        if (PARAMS && !have_first && lane == 0)
+            store_row_consts(qa, qb, 0, UNS ? __fsub_rn(m0, lo0) : m0, p0, lo0, Lf);
+        if (PARAMS && starts && lane == 1)
+            store_row_consts(qa, qb, 1, UNS ? __fsub_rn(m1, lo1) : m1, p1, lo1, Lf);
+        if (starts || !plain || !have_first) {
+            const int pos = starts ? (int)(long_end - span_beg) : -1;      // > 0 when it exists
+            const int wpos = pos >> 5;                                     // -1: no start
+            uint32_t w[4], e[4];
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                const int wi = 4 * lane + j;
+                w[j] = (wi == wpos) ? (1u << (pos & 31)) : 0u;
+                e[j] = (starts && wi > wpos) ? 1u : 0u;
+            }
+            reinterpret_cast<uint4*>(M.bits)[lane] = make_uint4(w[0], w[1], w[2], w[3]);
+            reinterpret_cast<uint2*>(M.before)[lane] = make_uint2(e[0] | (e[1] << 16), e[2] | (e[3] << 16));
+            if (lane == 0) { M.first_row = rf; M.slow = 0; }
+        }
+        if (stage == 0) { stage_first[0] = rf; stage_plain[0] = !starts; }
+        else            { stage_first[1] = rf; stage_plain[1] = !starts; }
+        if (more && long_end <= span_end) {               // the next span begins in row rf + 1
+            rf += 1;
+            long_end += rows.n;
+            m0 = m1; p0 = p1; lo0 = lo1;
+            if (PARAMS && rf + 1 < rows.C) load_inputs(rf + 1, m1, p1, lo1);
+        }
+    }
 };
 
 }  // namespace pwlq
