@@ -875,6 +875,169 @@ dequantize_kernel(const uint8_t* __restrict__ codes, const uint8_t* __restrict__
     }
 }
 
+// ------------------------------------------------------------------ several rows per span
+// Producer / consumer form of the inverse (see quantize_map_kernel and pwlq_rowmap.cuh).  The
+// producer writes row maps and constants only; the consumers request the codes and region bits
+// of the next span into registers before they wait for the current span's map.
+template <bool PACKED, bool UNS, bool LONG>
+__global__ void __launch_bounds__(kMapThreads, 4)
+dequantize_map_kernel(const uint8_t* __restrict__ codes, const uint8_t* __restrict__ mask, Rows rows,
+                      int64_t total, int bits, RowArrays A, float* __restrict__ y, int vec_codes,
+                      int vec_out, int64_t spans_per_cta) {
+    typedef MapStage<false, UNS> Stage;
+    extern __shared__ __align__(128) unsigned char smem_raw[];
+    Stage* st = reinterpret_cast<Stage*>(smem_raw);
+    __shared__ uint64_t full_bar[kMapStages], empty_bar[kMapStages];
+    const unsigned full = 0xffffffffu;
+    const int qmask = UNS ? (1 << bits) - 1 : (1 << (bits - 1)) - 1;   // the level inside a code
+    const float Lf = (float)qmask;
+    const int sign_shift = 32 - bits;                 // moves a code's sign bit to bit 31
+    const int64_t nspans = (total + kMapSpan - 1) / kMapSpan;
+    const int64_t first = blockIdx.x * spans_per_cta, last = min(first + spans_per_cta, nspans);
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < kMapStages; ++s) {
+            mbar_init(&full_bar[s], 1);
+            mbar_init(&empty_bar[s], kMapConsumers);
+        }
+        fence_barrier_init();
+    }
+    __syncthreads();
+    if (first >= last) return;
+
+    if (warp == kMapConsumers) {
+        // ---- producer
+        MapProducer<true, UNS, true> prod;
+        prod.rows = rows;
+        prod.in = RowInputs{A.m, A.lo, A.p};
+        prod.Lf = Lf;
+        if (LONG) prod.request_long(rows.dense_row(first * kMapSpan));
+        else prod.request(warp_row_of(rows, first * kMapSpan), true);
+        int64_t it = 0;
+        for (int64_t span = first; span < last; ++span, ++it) {
+            const int s = (int)(it % kMapStages);
+            const unsigned use = (unsigned)(it / kMapStages);
+            if (use > 0 && !mbar_wait(&empty_bar[s], (use - 1) & 1u)) {
+                if (lane == 0) atomicExch(&g_quantize_timeout, 1);
+                return;
+            }
+            const int64_t span_beg = span * kMapSpan, span_end = min(span_beg + kMapSpan, total);
+            if (LONG)
+                prod.build_long(st[s].map, st[s].qa, UNS ? st[s].qb : nullptr, s, span_beg, span_end,
+                                span + 1 < last);
+            else
+                prod.build(st[s].map, st[s].qa, UNS ? st[s].qb : nullptr, span_beg, span_end,
+                           span + 1 < last);
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&full_bar[s]);
+        }
+        return;
+    }
+
+    // ---- consumers
+    CodeRegs<PACKED> cur, nxt;
+    cur.load(codes, mask, first * kMapSpan, total, vec_codes);
+    int64_t it = 0;
+    for (int64_t span = first; span < last; ++span, ++it) {
+        const int s = (int)(it % kMapStages);
+        const unsigned use = (unsigned)(it / kMapStages);
+        if (span + 1 < last) nxt.load(codes, mask, (span + 1) * kMapSpan, total, vec_codes);
+        if (!mbar_wait_relaxed(&full_bar[s], use & 1u)) {
+            if (lane == 0) atomicExch(&g_quantize_timeout, 1);
+            return;
+        }
+        const int64_t span_beg = span * kMapSpan;
+        const Stage& S = st[s];
+        const bool slow = S.map.slow != 0;
+#pragma unroll
+        for (int c = 0; c < kQChunks; ++c) {
+            const int li = chunk_offset(c);
+            const int64_t i0 = span_beg + li;
+            const int cnt = (int)max((int64_t)0, min((int64_t)8, total - i0));
+            float yv[8];
+            if (!slow) {
+                uint32_t word;
+                const int l = map_slot(S.map, li, word);
+                const uint32_t inner = (word >> ((li & 31) + 1)) & 0x7Fu;   // starts at li+1 .. li+7
+                const float4 ca = S.qa[l];
+                const float loA = UNS ? S.qb[l].x : 0.0f;
+                const bool simple = inner == 0 && ca.x > 0.0f && cnt == 8;
+                PieceParams PA;
+                PA.p = ca.y; PA.s1 = ca.z; PA.s2 = ca.w; PA.inv1 = PA.inv2 = 0.0f;
+                if (__all_sync(full, simple)) {
+                    dequantize8<PACKED, false, UNS>(cur.w0[c], cur.w1[c], cur.mb[c], 8, PA, loA, PA, loA,
+                                                    qmask, sign_shift, yv);
+                } else {
+                    const bool one = inner != 0 && (inner & (inner - 1)) == 0 && ca.x > 0.0f && cnt == 8;
+                    float4 da = ca;
+                    float loB = loA;
+                    int split = 8;
+                    if (one) {
+                        da = S.qa[l + 1];
+                        if (UNS) loB = S.qb[l + 1].x;
+                        split = __ffs(inner);
+                    }
+                    if (__all_sync(full, simple || (one && da.x > 0.0f))) {
+                        PieceParams PB;
+                        PB.p = da.y; PB.s1 = da.z; PB.s2 = da.w; PB.inv1 = PB.inv2 = 0.0f;
+                        dequantize8<PACKED, true, UNS>(cur.w0[c], cur.w1[c], cur.mb[c], split, PA, loA,
+                                                       PB, loB, qmask, sign_shift, yv);
+                    } else {
+#pragma unroll
+                        for (int t = 0; t < 8; ++t) {
+                            yv[t] = 0.0f;
+                            if (t < cnt) {
+                                const int lt = l + __popc(inner & ((1u << t) - 1u));
+                                const float4 ea = S.qa[lt];
+                                const float loE = UNS ? S.qb[lt].x : 0.0f;
+                                if (UNS) yv[t] = loE;                  // a constant row delivers lo
+                                if (ea.x > 0.0f) {
+                                    const uint32_t code = code_of<PACKED>(cur.w0[c], cur.w1[c], t);
+                                    const int tail = (cur.mb[c] >> t) & 1;
+                                    const int neg = !UNS && ((code >> (bits - 1)) & 1);
+                                    const float q = (float)(code & qmask);
+                                    float v = __fmul_rn(q, tail ? ea.w : ea.z);
+                                    v = __fadd_rn(v, tail ? ea.y : 0.0f);
+                                    yv[t] = UNS ? __fadd_rn(v, loE) : (neg ? -v : v);
+                                }
+                            }
+                        }
+                    }
+                }
+            } else {
+                GlobalRow rs;
+#pragma unroll
+                for (int t = 0; t < 8; ++t) {
+                    yv[t] = 0.0f;
+                    if (t < cnt) {
+                        rs.seek(rows, A, Lf, i0 + t);
+                        if (UNS) yv[t] = rs.lo;
+                        if (rs.m > 0.0f) {
+                            const uint32_t code = code_of<PACKED>(cur.w0[c], cur.w1[c], t);
+                            const int tail = (cur.mb[c] >> t) & 1;
+                            const int neg = !UNS && ((code >> (bits - 1)) & 1);
+                            const float q = (float)(code & qmask);
+                            float v = __fmul_rn(q, tail ? rs.P.s2 : rs.P.s1);
+                            v = __fadd_rn(v, tail ? rs.P.p : 0.0f);
+                            yv[t] = UNS ? __fadd_rn(v, rs.lo) : (neg ? -v : v);
+                        }
+                    }
+                }
+            }
+            if (cnt == 0) continue;
+            if (vec_out && cnt == 8) {
+                __stcs(reinterpret_cast<float4*>(y + i0), make_float4(yv[0], yv[1], yv[2], yv[3]));
+                __stcs(reinterpret_cast<float4*>(y + i0 + 4), make_float4(yv[4], yv[5], yv[6], yv[7]));
+            } else {
+                for (int t = 0; t < cnt; ++t) y[i0 + t] = yv[t];
+            }
+        }
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&empty_bar[s]);
+        cur = nxt;
+    }
+}
+
 static inline bool aligned(const void* p, size_t a) {
     return (reinterpret_cast<uintptr_t>(p) & (a - 1)) == 0;
 }
@@ -985,6 +1148,22 @@ cudaError_t launch_dequantize(const uint8_t* codes, const uint8_t* mask,
     const int64_t nspans = (total + kQSpan - 1) / kQSpan;
 #define PWLQ_LAUNCH_DEQUANTIZE(PK, RG, UN)                                                        \
     do {                                                                                          \
+        if (RG) {                                                                                 \
+            const size_t msmem = sizeof(MapStage<false, UN>) * kMapStages;                        \
+            const int vc = aligned(codes, PK ? 4 : 8), vo = aligned(y, 16);                       \
+            if (long_rows) {                                                                      \
+                const SpanGrid g = span_grid((const void*)dequantize_map_kernel<PK, UN, true>,    \
+                                             kMapThreads, msmem, nspans, true);                   \
+                dequantize_map_kernel<PK, UN, true><<<g.grid, kMapThreads, msmem, stream>>>(      \
+                    codes, mask, rows, total, bits, A, y, vc, vo, g.per_cta);                     \
+            } else {                                                                              \
+                const SpanGrid g = span_grid((const void*)dequantize_map_kernel<PK, UN, false>,   \
+                                             kMapThreads, msmem, nspans, true);                   \
+                dequantize_map_kernel<PK, UN, false><<<g.grid, kMapThreads, msmem, stream>>>(     \
+                    codes, mask, rows, total, bits, A, y, vc, vo, g.per_cta);                     \
+            }                                                                                     \
+            break;                                                                                \
+        }                                                                                         \
         const SpanGrid g = span_grid((const void*)dequantize_kernel<PK, RG, UN>, kQThreads, 0,    \
                                      nspans, RG);                                                 \
         dequantize_kernel<PK, RG, UN><<<g.grid, kQThreads, 0, stream>>>(                          \
@@ -993,7 +1172,10 @@ cudaError_t launch_dequantize(const uint8_t* codes, const uint8_t* mask,
     } while (0)
 #define PWLQ_LAUNCH_DEQUANTIZE_UN(PK, RG) \
     do { if (lo) PWLQ_LAUNCH_DEQUANTIZE(PK, RG, true); else PWLQ_LAUNCH_DEQUANTIZE(PK, RG, false); } while (0)
-    const bool table = row_offsets != nullptr || n < kQSpan;    // several rows per span
+    // Dense rows of many spans stream through the register-only kernel (no row lookups worth
+    // speaking of); everything else goes through the producer / consumer kernel.
+    const bool table = row_offsets != nullptr || n < 16 * (int64_t)kMapSpan;
+    const bool long_rows = row_offsets == nullptr && n >= kMapSpan;   // the map follows from n
     if (packed) { if (table) PWLQ_LAUNCH_DEQUANTIZE_UN(true, true); else PWLQ_LAUNCH_DEQUANTIZE_UN(true, false); }
     else        { if (table) PWLQ_LAUNCH_DEQUANTIZE_UN(false, true); else PWLQ_LAUNCH_DEQUANTIZE_UN(false, false); }
 #undef PWLQ_LAUNCH_DEQUANTIZE_UN

@@ -56,19 +56,26 @@ struct RowInputs {
     const float* __restrict__ p;
 };
 
-// Constants of one row as the consumers read them: qa = (m, p, L/p, L/(m-p)),
-// qb = (p/L, (m-p)/L, lo, 0); m is the range width (abs-max, or upper - lower bound).
+// Constants of one row as the consumers read them; m is the range width (abs-max, or upper -
+// lower bound).  Quantize (DEQ = false): qa = (m, p, L/p, L/(m-p)), qb = (p/L, (m-p)/L, lo, 0).
+// Dequantize (DEQ = true): qa = (m, p, p/L, (m-p)/L), qb = (lo, 0, 0, 0).
+template <bool DEQ>
 __device__ __forceinline__ void store_row_consts(float4* qa, float4* qb, int slot, float m, float p,
                                                  float lo, float Lf) {
     const PieceParams P = make_params(m, p, Lf);
-    qa[slot] = make_float4(m, P.p, P.inv1, P.inv2);
-    if (qb) qb[slot] = make_float4(P.s1, P.s2, lo, 0.0f);
+    if (DEQ) {
+        qa[slot] = make_float4(m, P.p, P.s1, P.s2);
+        if (qb) qb[slot] = make_float4(lo, 0.0f, 0.0f, 0.0f);
+    } else {
+        qa[slot] = make_float4(m, P.p, P.inv1, P.inv2);
+        if (qb) qb[slot] = make_float4(P.s1, P.s2, lo, 0.0f);
+    }
 }
 
 // The producer warp's view of the rows.  Rows are looked at in chunks of 32 consecutive rows
 // (chunk c = rows 32 c .. 32 c + 31, lane = row % 32); the two chunks from the current first row
 // on are held in registers.  Every member function is called by all 32 lanes.
-template <bool PARAMS, bool UNS>
+template <bool PARAMS, bool UNS, bool DEQ = false>
 struct MapProducer {
     Rows rows;
     RowInputs in;
@@ -143,7 +150,7 @@ struct MapProducer {
                 if (PARAMS) {
                     if (k >= 2) load_inputs(r, mv, pv, lov);
                     if (UNS) mv = __fsub_rn(mv, lov);              // range width
-                    store_row_consts(qa, qb, s, mv, pv, lov, Lf);
+                    store_row_consts<DEQ>(qa, qb, s, mv, pv, lov, Lf);
                 }
             }
             const unsigned in_mask = __ballot_sync(full, inside);
@@ -226,9 +233,9 @@ struct MapProducer {
         const bool have_first = (stage == 0 ? stage_first[0] : stage_first[1]) == rf;
         const bool plain = stage == 0 ? stage_plain[0] : stage_plain[1];
         if (PARAMS && !have_first && lane == 0)
-            store_row_consts(qa, qb, 0, UNS ? __fsub_rn(m0, lo0) : m0, p0, lo0, Lf);
+            store_row_consts<DEQ>(qa, qb, 0, UNS ? __fsub_rn(m0, lo0) : m0, p0, lo0, Lf);
         if (PARAMS && starts && lane == 1)
-            store_row_consts(qa, qb, 1, UNS ? __fsub_rn(m1, lo1) : m1, p1, lo1, Lf);
+            store_row_consts<DEQ>(qa, qb, 1, UNS ? __fsub_rn(m1, lo1) : m1, p1, lo1, Lf);
         if (starts || !plain || !have_first) {
             const int pos = starts ? (int)(long_end - span_beg) : -1;      // > 0 when it exists
             const int wpos = pos >> 5;                                     // -1: no start
