@@ -1,26 +1,22 @@
 // Range m of every row: m_c = max_i |x_{c,i}|  (Sec. 3.2: quantization range [-m, m]).
 //
 // HBM-bound streaming reduction, 4 bytes read per value.  The flat storage is cut into spans of
-// kAbsSpan values that persistent CTAs walk; the spans arrive in a ring of shared-memory slots
-// filled by bulk asynchronous copies, three spans ahead.
-// Magnitude bit patterns are folded with an integer maximum (exact and order-free).  A span that
-// lies inside one row is folded into per-thread registers that live on from span to span (one
-// atomic per warp when the row ends); a span that holds several rows is cut into one slice per
-// warp, and the warp walks the rows overlapping its slice (offsets staged in shared memory) with
-// a strided read, a shuffle reduction and one atomicMax per piece.
+// kMapSpan values; a CTA walks consecutive spans, which arrive in a ring of shared-memory stages
+// filled by bulk asynchronous copies together with a map of the rows that start in them.
+// Magnitude bit patterns are folded with an integer maximum (exact and order-free).
 #include <algorithm>
 
 #include "pwlq_common.cuh"
 #include "pwlq_kernels.h"
 #include "pwlq_pipeline.cuh"
+#include "pwlq_rowmap.cuh"
 
 namespace pwlq {
 
-constexpr int kAbsThreads = 256;
-constexpr int kAbsUnroll = 4;
-constexpr int kAbsSpan = kAbsThreads * 4 * kAbsUnroll;  // values per span
+constexpr int kAbsConsumers = 8;                         // folding warps per CTA
+constexpr int kAbsThreads = (kAbsConsumers + 1) * 32;    // + the producer warp
 constexpr int kAbsStages = 3;                            // spans in flight per CTA
-constexpr int kAbsTableRows = 512;                       // staged rows per span (rows of >= 8 values fit)
+static_assert(kAbsStages <= 4, "MapProducer tracks at most four stages");
 
 static __device__ int g_absmax_timeout;                  // set when a bounded wait expired
 
@@ -50,6 +46,12 @@ struct Fold {
         }
     }
     __device__ __forceinline__ void add4(const float4 v) { add(v.x); add(v.y); add(v.z); add(v.w); }
+    // keys as add() forms them (0: nothing)
+    __device__ __forceinline__ void add_keys(uint32_t ka, uint32_t kb) {
+        a = max(a, ka);
+        if (MINMAX) b = max(b, kb);
+    }
+    __device__ __forceinline__ void merge(const Fold& o) { add_keys(o.a, o.b); }
     __device__ __forceinline__ void reduce_warp() {
         a = __reduce_max_sync(0xffffffffu, a);
         if (MINMAX) b = __reduce_max_sync(0xffffffffu, b);
@@ -61,193 +63,228 @@ struct Fold {
     __device__ __forceinline__ void clear() { a = b = 0; }
 };
 
-struct AbsSmem {
-    BulkRing<kAbsStages, kAbsSpan * 4> ring;
-    SpanTable<false, kAbsTableRows> T;
+// One stage of the producer / consumer pipeline: a span's values and its row map.
+struct AbsStage {
+    alignas(128) float data[kMapSpan];
+    SpanRowMap map;
 };
 
 // Bytes of span `span` if it can be fetched by a bulk copy (aligned base, whole 16-byte units).
 __device__ __forceinline__ unsigned abs_bulk_bytes(int64_t span, int64_t total, int vec_ok) {
-    const int64_t beg = span * kAbsSpan;
-    const int64_t cnt = min((int64_t)kAbsSpan, total - beg);
+    const int64_t beg = span * kMapSpan;
+    const int64_t cnt = min((int64_t)kMapSpan, total - beg);
     return (vec_ok && (cnt & 3) == 0) ? (unsigned)(cnt * 4) : 0u;
 }
 
-template <bool MINMAX>
+// Warp kAbsConsumers produces (bulk copy of the span's values + row map, see pwlq_rowmap.cuh);
+// the other warps fold.  A consumer warp owns a contiguous eighth of the span and walks it in
+// windows of 256 values, eight consecutive values per lane.  The fold of the row the warp is in
+// stays in per-lane registers from window to window and from span to span (a long row costs one
+// atomic per warp for the whole kernel).  A window in which rows start is handled without a
+// loop over the rows: every lane splits its values at its start, a segmented scan over the lanes
+// joins the pieces of every row, and the lane in which a row ends issues the row's atomic.
+// LONG: dense rows of at least a span (the maps follow from the row length).
+template <bool MINMAX, bool LONG>
 __global__ void __launch_bounds__(kAbsThreads)
 absmax_kernel(const float* __restrict__ x, Rows rows, int64_t total, uint32_t* __restrict__ m_bits,
               uint32_t* __restrict__ lo_bits, int vec_ok, int64_t spans_per_cta) {
     extern __shared__ __align__(128) unsigned char smem_raw[];
-    AbsSmem& S = *reinterpret_cast<AbsSmem*>(smem_raw);
-    __shared__ int s_abort;
-    const int64_t nspans = (total + kAbsSpan - 1) / kAbsSpan;
-    // this CTA's consecutive spans
-    const int64_t s0 = blockIdx.x * spans_per_cta, s1 = min(s0 + spans_per_cta, nspans);
-    const bool use_table = rows.offsets != nullptr || rows.n < kAbsSpan;   // several rows per span
-    if (threadIdx.x == 0) s_abort = 0;
-    S.ring.init();
-    for (int it = 0; it < kAbsStages; ++it)
-        if (s0 + it < s1)
-            S.ring.issue(it, x + (s0 + it) * kAbsSpan, abs_bulk_bytes(s0 + it, total, vec_ok));
+    AbsStage* st = reinterpret_cast<AbsStage*>(smem_raw);
+    __shared__ uint64_t full_bar[kAbsStages], empty_bar[kAbsStages];
+    const unsigned full = 0xffffffffu;
+    const int64_t nspans = (total + kMapSpan - 1) / kMapSpan;
+    const int64_t first = blockIdx.x * spans_per_cta, last = min(first + spans_per_cta, nspans);
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < kAbsStages; ++s) {
+            mbar_init(&full_bar[s], 2);            // the data (or its stand-in) and the map
+            mbar_init(&empty_bar[s], kAbsConsumers);
+        }
+        fence_barrier_init();
+    }
+    __syncthreads();
+    if (first >= last) return;
 
-    int64_t row0 = 0;                                  // first staged row of the current span
-    RowFetch<kAbsTableRows> nf;
-    if (use_table && s0 < s1) {
-        row0 = cta_row_near(rows, s0 * kAbsSpan);
-        S.T.fetch(rows, nullptr, nullptr, nullptr, row0, nf);
-        S.T.commit(nf, 0, 0.0f);
-        __syncthreads();
+    if (warp == kAbsConsumers) {
+        // ---- producer
+        MapProducer<false, false> prod;
+        prod.rows = rows;
+        prod.in = RowInputs{nullptr, nullptr, nullptr};
+        prod.Lf = 0.0f;
+        if (LONG) prod.request_long(rows.dense_row(first * kMapSpan));
+        else prod.request(warp_row_of(rows, first * kMapSpan), true);
+        int64_t it = 0;
+        for (int64_t span = first; span < last; ++span, ++it) {
+            const int s = (int)(it % kAbsStages);
+            const unsigned use = (unsigned)(it / kAbsStages);
+            if (use > 0 && !mbar_wait(&empty_bar[s], (use - 1) & 1u)) {
+                if (lane == 0) atomicExch(&g_absmax_timeout, 1);
+                return;
+            }
+            const int64_t span_beg = span * kMapSpan, span_end = min(span_beg + kMapSpan, total);
+            const unsigned bytes = abs_bulk_bytes(span, total, vec_ok);
+            if (bytes != 0) {
+                if (lane == 0) {
+                    // the stage was last read (by the consumers, whose arrivals this warp has
+                    // waited for), not written, through the generic proxy: no proxy fence needed
+                    mbar_expect_tx(&full_bar[s], bytes);
+                    bulk_copy_g2s(st[s].data, x + span_beg, bytes, &full_bar[s]);
+                }
+            } else {                               // unaligned base or ragged tail: plain loads
+                for (int i = lane; i < (int)(span_end - span_beg); i += 32) st[s].data[i] = x[span_beg + i];
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&full_bar[s]);
+            }
+            if (LONG) prod.build_long(st[s].map, nullptr, nullptr, s, span_beg, span_end, span + 1 < last);
+            else prod.build(st[s].map, nullptr, nullptr, span_beg, span_end, span + 1 < last);
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&full_bar[s]);
+        }
+        return;
     }
 
-    // The long row the CTA is inside of (the same for all of its threads) and this thread's
-    // maximum over it; both survive from span to span, so a long row costs one atomic per warp
-    // for the whole kernel.
-    int64_t grow = -1;
-    Fold<MINMAX> mx;
-    auto flush_merged = [&]() {                        // every lane of the warp calls this
-        mx.reduce_warp();
-        if ((threadIdx.x & 31) == 0 && grow >= 0) mx.store(m_bits, lo_bits, grow);
-        mx.clear();
+    // ---- consumers
+    Fold<MINMAX> acc;                              // this lane's share of the row the warp is in
+    int64_t acc_row = -1;                          // that row (the same for all lanes)
+    auto flush_acc = [&]() {                       // every lane of the warp calls this
+        acc.reduce_warp();
+        if (lane == 0 && acc_row >= 0) acc.store(m_bits, lo_bits, acc_row);
+        acc.clear();
     };
-
-    for (int64_t span = s0; span < s1; ++span) {
-        const int64_t it = span - s0;
-        const int64_t span_beg = span * kAbsSpan;
-        const int64_t span_end = min(span_beg + kAbsSpan, total);
-        // Does the span lie inside one row?
-        bool single;
-        int64_t first_row;
-        if (use_table) {
-            const int l0 = S.T.find(span_beg);          // -1: more rows than the window holds
-            first_row = row0 + l0;
-            single = l0 >= 0 && S.T.off[l0 + 1] >= span_end;
-        } else {
-            first_row = rows.dense_row(span_beg);
-            single = (first_row + 1) * rows.n >= span_end;
-        }
-        // the staged rows end before the next span does: request the window that starts in the
-        // row in which this span ends
-        int64_t next_row0 = 0;
-        const bool has_next = use_table && span + 1 < s1 &&
-                              !S.T.covers(min(span_end + kAbsSpan, total));
-        if (has_next) {
-            const int l = S.T.find(span_end);
-            next_row0 = (l >= 0) ? row0 + l : warp_row_of(rows, span_end);
-            S.T.fetch(rows, nullptr, nullptr, nullptr, next_row0, nf);
-        }
-        if (!single) {                                 // several rows: nothing is carried across
-            flush_merged();
-            grow = -1;
-        } else if (grow != first_row) {                // a new long row begins
-            flush_merged();
-            grow = first_row;
-        }
-
-        float* xs = reinterpret_cast<float*>(S.ring.slot(it));
-        if (abs_bulk_bytes(span, total, vec_ok) != 0) {
-            if (!S.ring.wait(it, (unsigned)(it / kAbsStages))) s_abort = 1;   // never expected
-        } else {                                       // unaligned base or ragged tail: plain loads
-            for (int i = threadIdx.x; i < (int)(span_end - span_beg); i += kAbsThreads)
-                xs[i] = x[span_beg + i];
-            __syncthreads();
-        }
-        if (single) {
-            // the whole span belongs to the carried row: registers only
-#pragma unroll
-            for (int j = 0; j < kAbsUnroll; ++j) {
-                const int li = (j * kAbsThreads + threadIdx.x) * 4;
-                if (span_beg + li + 4 <= span_end) {
-                    mx.add4(*reinterpret_cast<const float4*>(xs + li));
-                } else {
-                    for (int t = 0; t < 4; ++t)
-                        if (span_beg + li + t < span_end) mx.add(xs[li + t]);
-                }
-            }
-        } else {
-            // several rows: every warp takes a contiguous slice of the span and walks it in
-            // windows of 128 values (one 128-bit read per lane).  The maximum of the row the warp
-            // is in stays in per-lane registers from window to window; when the row ends inside a
-            // window the lanes' values are split at the boundary, the finished row is reduced with
-            // one warp-wide maximum and one atomic, and the next row starts.  All control flow is
-            // warp-uniform.
-            const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-            constexpr int kSlice = kAbsSpan / (kAbsThreads / 32);
-            const int sl_beg = warp * kSlice;                              // relative to the span
-            const int sl_end = min(sl_beg + kSlice, (int)(span_end - span_beg));
-            if (sl_beg < sl_end) {
-                int l = use_table ? S.T.find(span_beg + sl_beg) : -1;
-                int64_t r_glob = 0;
-                int r_end = 0;                                             // relative to the span
-                auto enter_row = [&](int pos) {            // the row that contains / follows pos
-                    int64_t e;
-                    if (l >= 0 && l < kAbsTableRows) {     // staged row
-                        r_glob = row0 + l;
-                        e = S.T.off[l + 1];
-                        ++l;
-                    } else {                               // long dense rows, or beyond the table
-                        r_glob = rows.row_of(span_beg + pos);
-                        e = rows.begin(r_glob + 1);
-                        l = -1;
-                    }
-                    r_end = (int)min(e - span_beg, (int64_t)kAbsSpan);
-                };
-                enter_row(sl_beg);
-                Fold<MINMAX> v;
-                for (int wb = sl_beg; wb < sl_end; wb += 128) {
-                    const int we = min(wb + 128, sl_end);
-                    const int i0 = wb + 4 * lane;
-                    float f[4] = {0.0f, 0.0f, 0.0f, 0.0f};
-                    const bool whole = i0 + 4 <= we;       // all four values lie inside the window
-                    if (whole) {
-                        const float4 q = *reinterpret_cast<const float4*>(xs + i0);
-                        f[0] = q.x; f[1] = q.y; f[2] = q.z; f[3] = q.w;
-                    } else {
-#pragma unroll
-                        for (int t = 0; t < 4; ++t)
-                            if (i0 + t < we) f[t] = xs[i0 + t];
-                    }
-                    if (r_end >= we) {                     // the window lies inside the current row
-                        if (whole) {
-                            v.add4(make_float4(f[0], f[1], f[2], f[3]));
-                        } else {
-#pragma unroll
-                            for (int t = 0; t < 4; ++t)
-                                if (i0 + t < we) v.add(f[t]);
-                        }
-                        continue;
-                    }
-                    int pos = wb;                          // values before pos are accounted for
-                    while (true) {
-                        const int e = min(r_end, we);
-#pragma unroll
-                        for (int t = 0; t < 4; ++t)
-                            if (i0 + t >= pos && i0 + t < e) v.add(f[t]);
-                        if (r_end > we) break;             // the row continues in the next window
-                        v.reduce_warp();
-                        if (lane == 0) v.store(m_bits, lo_bits, r_glob);
-                        v.clear();
-                        pos = e;
-                        if (pos >= sl_end) break;          // the slice ends with this row
-                        enter_row(pos);
-                        if (pos >= we) break;              // the new row starts with the next window
-                    }
-                }
-                v.reduce_warp();                           // the row the slice ends in
-                if (lane == 0) v.store(m_bits, lo_bits, r_glob);
-            }
-        }
-        __syncthreads();                              // slot and table are no longer read
-        if (s_abort) {                                 // a wait ran out: report and leave
-            if (threadIdx.x == 0) atomicExch(&g_absmax_timeout, 1);
+    constexpr int kSlice = kMapSpan / kAbsConsumers;
+    int64_t it = 0;
+    for (int64_t span = first; span < last; ++span, ++it) {
+        const int s = (int)(it % kAbsStages);
+        const unsigned use = (unsigned)(it / kAbsStages);
+        if (!mbar_wait_relaxed(&full_bar[s], use & 1u)) {
+            if (lane == 0) atomicExch(&g_absmax_timeout, 1);
             return;
         }
-        if (has_next) { S.T.commit(nf, 0, 0.0f); row0 = next_row0; }
-        if (span + kAbsStages < s1)
-            S.ring.issue(it + kAbsStages, x + (span + kAbsStages) * kAbsSpan,
-                         abs_bulk_bytes(span + kAbsStages, total, vec_ok));
-        if (has_next) __syncthreads();                // the next window is published
+        const int64_t span_beg = span * kMapSpan;
+        const int span_len = (int)min((int64_t)kMapSpan, total - span_beg);
+        const AbsStage& S = st[s];
+        const float* xs = S.data;
+        const int sl_beg = warp * kSlice;
+        if (sl_beg < span_len) {
+            const bool slow = S.map.slow != 0;
+            const int64_t first_row = S.map.first_row;
+            if (!slow) {
+                // the row that is open where the slice begins (a row that starts exactly there
+                // is opened by the window below)
+                uint32_t w0;
+                const int sl_slot = map_slot(S.map, sl_beg, w0);
+                const int64_t r_open = first_row + sl_slot - (int)((w0 >> (sl_beg & 31)) & 1u);
+                if (r_open != acc_row) { flush_acc(); acc_row = r_open; }
+            } else {
+                flush_acc();
+                acc_row = -1;
+            }
+#pragma unroll 1
+            for (int win = 0; win < kSlice / 256; ++win) {
+                const int li = sl_beg + win * 256 + lane * 8;
+                const int cnt = max(0, min(8, span_len - li));
+                uint32_t ka[8], kb[8];
+                if (cnt == 8) {
+                    const float4 xa = *reinterpret_cast<const float4*>(xs + li);
+                    const float4 xb = *reinterpret_cast<const float4*>(xs + li + 4);
+                    const float v[8] = {xa.x, xa.y, xa.z, xa.w, xb.x, xb.y, xb.z, xb.w};
+#pragma unroll
+                    for (int j = 0; j < 8; ++j) {
+                        ka[j] = MINMAX ? ordered_key(v[j]) : abs_bits(v[j]);
+                        kb[j] = MINMAX ? ~ka[j] : 0u;
+                    }
+                } else {
+#pragma unroll
+                    for (int j = 0; j < 8; ++j) {
+                        ka[j] = kb[j] = 0u;                      // 0: nothing
+                        if (j < cnt) {
+                            ka[j] = MINMAX ? ordered_key(xs[li + j]) : abs_bits(xs[li + j]);
+                            kb[j] = MINMAX ? ~ka[j] : 0u;
+                        }
+                    }
+                }
+                if (slow) {
+                    // no usable map: every value finds its row in global memory
+                    for (int j = 0; j < cnt; ++j) {
+                        Fold<MINMAX> one;
+                        one.a = ka[j]; one.b = kb[j];
+                        one.store(m_bits, lo_bits, rows.row_of(span_beg + li + j));
+                    }
+                    continue;
+                }
+                uint32_t word;
+                const int slot0 = map_slot(S.map, li, word);     // row of my first value
+                const uint32_t nib = (word >> (li & 31)) & 0xFFu;   // bit j: a row starts at li + j
+                const unsigned starts = __ballot_sync(full, nib != 0);
+                if (starts == 0) {                               // the window lies inside the open row
+#pragma unroll
+                    for (int j = 0; j < 8; ++j) acc.add_keys(ka[j], kb[j]);
+                    continue;
+                }
+                if (__any_sync(full, (nib & (nib - 1)) != 0)) {
+                    // a lane holds more than one start (rows of fewer than eight values): every
+                    // lane walks its values on its own
+                    flush_acc();
+                    Fold<MINMAX> cur;
+                    int cur_slot = slot0 - (int)(nib & 1u);
+#pragma unroll
+                    for (int j = 0; j < 8; ++j) {
+                        if ((nib >> j) & 1u) {
+                            cur.store(m_bits, lo_bits, first_row + cur_slot);
+                            cur.clear();
+                            ++cur_slot;
+                        }
+                        cur.add_keys(ka[j], kb[j]);
+                    }
+                    cur.store(m_bits, lo_bits, first_row + cur_slot);
+                    acc_row = first_row + __shfl_sync(full, cur_slot, 31);
+                    continue;
+                }
+                // at most one start per lane: split my values at it
+                const bool flag = nib != 0;
+                const int fpos = flag ? __ffs(nib) - 1 : 8;
+                const uint32_t low = (1u << fpos) - 1u;          // bit j: value j lies before my start
+                Fold<MINMAX> h, t;
+#pragma unroll
+                for (int j = 0; j < 8; ++j) {
+                    const uint32_t hm = 0u - ((low >> j) & 1u);
+                    h.add_keys(ka[j] & hm, kb[j] & hm);
+                    t.add_keys(ka[j] & ~hm, kb[j] & ~hm);
+                }
+                // inclusive scan over the lanes, restarted at every lane with a start
+                Fold<MINMAX> sc = flag ? t : h;
+                const unsigned below = starts & (0xFFFFFFFFu >> (31 - lane));
+                const int ss = below ? 31 - __clz(below) : 0;
+#pragma unroll
+                for (int d = 1; d < 32; d <<= 1) {
+                    Fold<MINMAX> y;
+                    y.a = __shfl_up_sync(full, sc.a, d);
+                    y.b = MINMAX ? __shfl_up_sync(full, sc.b, d) : 0u;
+                    if (lane - d >= ss) sc.merge(y);
+                }
+                Fold<MINMAX> left;                               // the lanes between the previous start and me
+                left.a = __shfl_up_sync(full, sc.a, 1);
+                left.b = MINMAX ? __shfl_up_sync(full, sc.b, 1) : 0u;
+                if (lane == 0) left.clear();
+                Fold<MINMAX> carry = acc;                        // the open row so far
+                carry.reduce_warp();
+                if (flag) {                                      // a row ends before my start
+                    Fold<MINMAX> closed = h;
+                    closed.merge(left);
+                    if ((starts & ((1u << lane) - 1u)) == 0) closed.merge(carry);
+                    closed.store(m_bits, lo_bits, first_row + slot0 - (int)(nib & 1u));
+                }
+                const int last_flag = 31 - __clz(starts);
+                acc.clear();
+                if (lane > last_flag) acc = h;
+                else if (lane == last_flag) acc = t;
+                acc_row = first_row + __shfl_sync(full, slot0 + __popc(nib >> 1), last_flag);
+            }
+        }
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&empty_bar[s]);
     }
-    flush_merged();                                   // what is still carried at the end
+    flush_acc();                                      // what is still carried at the end
 }
 
 int absmax_timeout_flag() {
@@ -288,34 +325,39 @@ static cudaError_t launch_fold(const float* x, const int64_t* row_offsets, int64
     }
     if (total == 0) return cudaSuccess;
     Rows rows{row_offsets, C, n, n > 0 ? 1.0 / (double)n : 0.0, row_offsets ? shift : 0};
-    const int64_t nspans = (total + kAbsSpan - 1) / kAbsSpan;
-    static int cached[64] = {0};                       // CTAs that fit the device at once
+    const int64_t nspans = (total + kMapSpan - 1) / kMapSpan;
+    const bool long_rows = row_offsets == nullptr && n >= kMapSpan;   // the maps follow from n
+    const size_t smem = sizeof(AbsStage) * kAbsStages;
+    const void* kernel = long_rows ? (const void*)absmax_kernel<MINMAX, true>
+                                   : (const void*)absmax_kernel<MINMAX, false>;
+    static int cached[2][64] = {{0}};                  // CTAs that fit the device at once
     int dev = 0;
     cudaGetDevice(&dev);
     if (dev < 0 || dev >= 64) dev = 0;
-    if (cached[dev] == 0) {
-        e = cudaFuncSetAttribute(absmax_kernel<MINMAX>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                 (int)sizeof(AbsSmem));
+    int& slots_dev = cached[long_rows ? 1 : 0][dev];
+    if (slots_dev == 0) {
+        e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (e != cudaSuccess) return e;
         int sms = 0, per_sm = 0;
         cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-        cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, absmax_kernel<MINMAX>, kAbsThreads,
-                                                      sizeof(AbsSmem));
-        cached[dev] = (sms > 0 && per_sm > 0) ? sms * per_sm : 148;
+        cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kernel, kAbsThreads, smem);
+        slots_dev = (sms > 0 && per_sm > 0) ? sms * per_sm : 148;
     }
-    // Long dense rows cost the same everywhere: one CTA per slot of the device, equal shares.
-    // Where spans hold several rows the cost per span depends on the row lengths, so the spans are
-    // handed out in small blocks (about four per slot) and the hardware scheduler balances them.
-    const int64_t slots = cached[dev];
-    const bool several_rows = row_offsets != nullptr || n < kAbsSpan;
-    int64_t per_cta = (nspans + slots - 1) / slots;
-    if (several_rows)
-        per_cta = std::min<int64_t>(std::max<int64_t>((nspans + 4 * slots - 1) / (4 * slots), 4), 32);
+    // Consecutive spans are handed out in blocks, about four per slot of the device, so that the
+    // hardware scheduler evens out what differs between them (row starts per span).
+    const int64_t slots = slots_dev;
+    const int64_t per_cta =
+        std::min<int64_t>(std::max<int64_t>((nspans + 4 * slots - 1) / (4 * slots), 4), 64);
     const unsigned grid = (unsigned)((nspans + per_cta - 1) / per_cta);
     const int vec_ok = (reinterpret_cast<uintptr_t>(x) & 15u) == 0;
-    absmax_kernel<MINMAX><<<grid, kAbsThreads, sizeof(AbsSmem), stream>>>(
-        x, rows, total, reinterpret_cast<uint32_t*>(out_a), reinterpret_cast<uint32_t*>(out_b),
-        vec_ok, per_cta);
+    if (long_rows)
+        absmax_kernel<MINMAX, true><<<grid, kAbsThreads, smem, stream>>>(
+            x, rows, total, reinterpret_cast<uint32_t*>(out_a), reinterpret_cast<uint32_t*>(out_b),
+            vec_ok, per_cta);
+    else
+        absmax_kernel<MINMAX, false><<<grid, kAbsThreads, smem, stream>>>(
+            x, rows, total, reinterpret_cast<uint32_t*>(out_a), reinterpret_cast<uint32_t*>(out_b),
+            vec_ok, per_cta);
     return cudaGetLastError();
 }
 

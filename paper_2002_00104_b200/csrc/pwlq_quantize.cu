@@ -429,6 +429,7 @@ quantize_kernel(const float* __restrict__ x, Rows rows, int64_t total, int bits,
 constexpr int kMapConsumers = 8;
 constexpr int kMapThreads = (kMapConsumers + 1) * 32;
 constexpr int kMapStages = 2;
+static_assert(kMapStages <= 4, "MapProducer tracks at most four stages");
 
 template <bool DATA, bool QB>
 struct MapStage {

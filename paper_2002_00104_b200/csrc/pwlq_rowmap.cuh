@@ -211,9 +211,10 @@ struct MapProducer {
     // the beginning of the next.  Everything follows from the row length; the inputs of the
     // current and the next row are held in registers (every lane the same), and a stage whose
     // slot 0 already belongs to the row is left as it is.
-    int64_t long_end;           // end of row rf
-    int64_t stage_first[2];     // per stage: the row its slot 0 was written for, or -1
-    bool stage_plain[2];        // per stage: the map says "one row, no start"
+    static constexpr int kMaxStages = 4;
+    int64_t long_end;                    // end of row rf
+    int64_t stage_first[kMaxStages];     // per stage: the row its slot 0 was written for, or -1
+    bool stage_plain[kMaxStages];        // per stage: the map says "one row, no start"
 
     __device__ __forceinline__ void request_long(int64_t first_row) {
         rf = first_row;
@@ -223,15 +224,18 @@ struct MapProducer {
             load_inputs(rf, m0, p0, lo0);
             if (rf + 1 < rows.C) load_inputs(rf + 1, m1, p1, lo1);
         }
-        stage_first[0] = stage_first[1] = -1;
-        stage_plain[0] = stage_plain[1] = false;
+#pragma unroll
+        for (int i = 0; i < kMaxStages; ++i) { stage_first[i] = -1; stage_plain[i] = false; }
     }
     __device__ __forceinline__ void build_long(SpanRowMap& M, float4* qa, float4* qb, int stage,
                                                int64_t span_beg, int64_t span_end, bool more) {
         const int lane = threadIdx.x & 31;
         const bool starts = long_end < span_end;          // row rf + 1 begins inside the span
-        const bool have_first = (stage == 0 ? stage_first[0] : stage_first[1]) == rf;
-        const bool plain = stage == 0 ? stage_plain[0] : stage_plain[1];
+        // (selected with constant indices: the arrays stay in registers; stage < kMaxStages)
+        bool have_first = false, plain = false;
+#pragma unroll
+        for (int i = 0; i < kMaxStages; ++i)
+            if (stage == i) { have_first = stage_first[i] == rf; plain = stage_plain[i]; }
         if (PARAMS && !have_first && lane == 0)
             store_row_consts<DEQ>(qa, qb, 0, UNS ? __fsub_rn(m0, lo0) : m0, p0, lo0, Lf);
         if (PARAMS && starts && lane == 1)
@@ -250,8 +254,9 @@ struct MapProducer {
             reinterpret_cast<uint2*>(M.before)[lane] = make_uint2(e[0] | (e[1] << 16), e[2] | (e[3] << 16));
             if (lane == 0) { M.first_row = rf; M.slow = 0; }
         }
-        if (stage == 0) { stage_first[0] = rf; stage_plain[0] = !starts; }
-        else            { stage_first[1] = rf; stage_plain[1] = !starts; }
+#pragma unroll
+        for (int i = 0; i < kMaxStages; ++i)
+            if (stage == i) { stage_first[i] = rf; stage_plain[i] = !starts; }
         if (more && long_end <= span_end) {               // the next span begins in row rf + 1
             rf += 1;
             long_end += rows.n;
