@@ -111,6 +111,14 @@ absmax_kernel(const float* __restrict__ x, Rows rows, int64_t total, uint32_t* _
         prod.rows = rows;
         prod.in = RowInputs{nullptr, nullptr, nullptr};
         prod.Lf = 0.0f;
+        // the values of the first spans do not depend on the rows: request them before the search
+        for (int64_t span = first; span < last && span < first + kAbsStages; ++span) {
+            const unsigned bytes = abs_bulk_bytes(span, total, vec_ok);
+            if (bytes != 0 && lane == 0) {
+                mbar_expect_tx(&full_bar[span - first], bytes);
+                bulk_copy_g2s(st[span - first].data, x + span * kMapSpan, bytes, &full_bar[span - first]);
+            }
+        }
         if (LONG) prod.request_long(rows.dense_row(first * kMapSpan));
         else prod.request(warp_row_of(rows, first * kMapSpan), true);
         int64_t it = 0;
@@ -124,7 +132,7 @@ absmax_kernel(const float* __restrict__ x, Rows rows, int64_t total, uint32_t* _
             const int64_t span_beg = span * kMapSpan, span_end = min(span_beg + kMapSpan, total);
             const unsigned bytes = abs_bulk_bytes(span, total, vec_ok);
             if (bytes != 0) {
-                if (lane == 0) {
+                if (lane == 0 && use > 0) {        // (first round: requested above)
                     // the stage was last read (by the consumers, whose arrivals this warp has
                     // waited for), not written, through the generic proxy: no proxy fence needed
                     mbar_expect_tx(&full_bar[s], bytes);
@@ -343,11 +351,12 @@ static cudaError_t launch_fold(const float* x, const int64_t* row_offsets, int64
         cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kernel, kAbsThreads, smem);
         slots_dev = (sms > 0 && per_sm > 0) ? sms * per_sm : 148;
     }
-    // Consecutive spans are handed out in blocks, about four per slot of the device, so that the
-    // hardware scheduler evens out what differs between them (row starts per span).
+    // Consecutive spans are handed out in blocks of at most 32, about four per slot of the device:
+    // long enough to pay for the producer's start, short enough for the hardware scheduler to even
+    // out what differs between spans (row starts per span).
     const int64_t slots = slots_dev;
     const int64_t per_cta =
-        std::min<int64_t>(std::max<int64_t>((nspans + 4 * slots - 1) / (4 * slots), 4), 64);
+        std::min<int64_t>(std::max<int64_t>((nspans + 4 * slots - 1) / (4 * slots), 1), 32);
     const unsigned grid = (unsigned)((nspans + per_cta - 1) / per_cta);
     const int vec_ok = (reinterpret_cast<uintptr_t>(x) & 15u) == 0;
     if (long_rows)

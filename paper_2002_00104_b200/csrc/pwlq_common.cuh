@@ -125,119 +125,4 @@ __device__ __forceinline__ int64_t warp_row_of(const Rows& rows, int64_t i) {
     return lo;
 }
 
-// A row at or shortly before the row that contains flat index i (at most three rows before it),
-// found by a whole CTA together in rounds of blockDim.x-way search: two dependent rounds of loads
-// for up to 65536 rows with 256 threads.  Every thread calls it with the same i (it contains CTA
-// barriers) and gets the same answer.
-__device__ __forceinline__ int64_t cta_row_near(const Rows& rows, int64_t i) {
-    if (!rows.offsets) return rows.dense_row(i);
-    const int64_t T = blockDim.x;
-    int64_t lo = 0, hi = rows.C;                     // offsets[lo] <= i < offsets[hi]
-    while (hi - lo > 4) {
-        const int64_t step = (hi - lo + T - 1) / T;
-        const int64_t q = lo + (int64_t)(threadIdx.x + 1) * step;
-        const int le = (q < hi) && (rows.offsets[q] - rows.shift <= i);    // true for a prefix of the threads
-        const int cnt = __syncthreads_count(le);
-        const int64_t new_lo = lo + (int64_t)cnt * step;
-        hi = min(hi, new_lo + step);
-        lo = new_lo;
-    }
-    return lo;
-}
-
-// A window of CAP consecutive rows of the flat storage, staged in shared memory so that the
-// per-thread row lookups of a CTA never touch global memory.  The CTA walks consecutive spans and
-// keeps the window for as long as it reaches to the end of the next span: with long
-// rows it is filled once per CTA.  When the next span will run past it, the window that starts at
-// the row in which the current span ends is requested into registers before the current span is
-// processed and written to shared memory after it, which keeps the global round trip off the
-// critical path.  Values that lie beyond the last staged row (spans with more than CAP rows) use
-// the global search.
-constexpr int kTableThreads = 256;        // CTA size the fetch / commit pattern is written for
-
-template <int CAP>
-struct RowFetch {                          // what one thread holds of the next window
-    static constexpr int kPerThread = CAP / kTableThreads;
-    int64_t off[kPerThread + 1];           // rows tid + u * 256, and (thread 0) the entry CAP
-    float m[kPerThread], p[kPerThread], lo[kPerThread];
-};
-
-template <bool PARAMS, int CAP>
-struct SpanTable {
-    static constexpr int kPerThread = CAP / kTableThreads;
-    static_assert(CAP % kTableThreads == 0, "whole rounds of the CTA");
-    int64_t off[CAP + 1];     // off[r] = first flat index of row row0 + r (INT64_MAX past the last row)
-    float m[PARAMS ? CAP : 1];    // range width: abs-max, or hi - lo for one-sided ranges
-    float lo[PARAMS ? CAP : 1];   // lower bound of a one-sided range (0 otherwise)
-    PieceParams P[PARAMS ? CAP : 1];
-
-    // True when every flat index below `end` lies in a staged row (or past the last row).
-    __device__ __forceinline__ bool covers(int64_t end) const { return off[CAP] >= end; }
-
-    // Local index of the staged row containing i, or -1 when i lies beyond the staged rows.
-    // Neighbouring rows are mostly equally long (one layer), so a proportional guess is tried
-    // first and corrected by a few neighbour steps; irregular windows fall back to bisection.
-    __device__ __forceinline__ int find(int64_t i) const {
-        const int64_t last = off[CAP];
-        if (i >= last) return -1;
-        int lo = 0, hi = CAP;                         // off[lo] <= i < off[hi]
-        if (last != INT64_MAX) {
-            const float scale = (float)CAP / (float)(last - off[0]);
-            int g = min(max((int)((float)(i - off[0]) * scale), 0), CAP - 1);
-#pragma unroll
-            for (int t = 0; t < 4; ++t) {
-                if (off[g] > i) { hi = g; g = max(g - 1, 0); }
-                else if (off[g + 1] <= i) { lo = g + 1; g = min(g + 1, CAP - 1); }
-                else return g;
-            }
-        }
-        while (hi - lo > 1) {
-            const int mid = (lo + hi) >> 1;
-            if (off[mid] <= i) lo = mid; else hi = mid;
-        }
-        return lo;
-    }
-    // Requests the window that starts at row r0 (no barrier; the values stay in registers).
-    // lo_arr != nullptr: one-sided ranges, m_arr holds the upper bounds.  (All loads are
-    // independent of each other, so that none of them is waited for here.)
-    __device__ __forceinline__ void fetch(const Rows& rows, const float* __restrict__ m_arr,
-                                          const float* __restrict__ p_arr,
-                                          const float* __restrict__ lo_arr, int64_t r0,
-                                          RowFetch<CAP>& f) const {
-#pragma unroll
-        for (int u = 0; u < kPerThread; ++u) {
-            const int64_t row = r0 + (int)threadIdx.x + u * kTableThreads;
-            f.off[u] = (row <= rows.C) ? rows.begin(row) : INT64_MAX;
-            f.m[u] = f.p[u] = f.lo[u] = 0.0f;
-            if (PARAMS && row < rows.C) {
-                f.m[u] = __ldg(m_arr + row);
-                f.p[u] = __ldg(p_arr + row);
-                if (lo_arr) {
-                    f.lo[u] = __ldg(lo_arr + row);
-                    f.m[u] = __fsub_rn(f.m[u], f.lo[u]);
-                }
-            }
-        }
-        f.off[kPerThread] = (threadIdx.x == 0 && r0 + CAP <= rows.C) ? rows.begin(r0 + CAP)
-                                                                     : INT64_MAX;
-    }
-    // Writes what fetch() requested, with the constants of the rows that start before `limit`
-    // (the end of the CTA's share of the storage; later rows are staged with their offsets
-    // alone); call between the barrier that retires the previous window and the barrier that
-    // publishes this one.
-    __device__ __forceinline__ void commit(const RowFetch<CAP>& f, int64_t limit, float Lf) {
-#pragma unroll
-        for (int u = 0; u < kPerThread; ++u) {
-            const int r = (int)threadIdx.x + u * kTableThreads;
-            off[r] = f.off[u];
-            if (PARAMS && f.off[u] < limit) {
-                m[r] = f.m[u];
-                lo[r] = f.lo[u];
-                P[r] = make_params(f.m[u], f.p[u], Lf);
-            }
-        }
-        if (threadIdx.x == 0) off[CAP] = f.off[kPerThread];
-    }
-};
-
 }  // namespace pwlq

@@ -1,7 +1,7 @@
-// A ring of shared-memory slots filled by bulk asynchronous copies (the TMA engine's untiled
-// cp.async.bulk, global -> shared, completion counted in bytes on an mbarrier), for the
-// HBM-bound streaming kernels: a persistent CTA keeps the copies of its next spans in flight
-// while it works on the current one, without spending registers on them.
+// Bulk asynchronous copies (the TMA engine's untiled cp.async.bulk, global -> shared, completion
+// counted in bytes on an mbarrier) and mbarrier helpers for the HBM-bound streaming kernels: a CTA
+// keeps the copies of its next spans in flight while it works on the current one, without
+// spending registers on them.
 //
 // Rules kept here: source and destination 16-byte aligned, size a multiple of 16 bytes (spans
 // that do not qualify are staged with ordinary loads instead); no multicast, no cluster; every
@@ -66,40 +66,5 @@ __device__ __forceinline__ void bulk_copy_g2s(void* dst_smem, const void* src_gm
         "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
         ::"r"(smem_addr(dst_smem)), "l"(src_gmem), "r"(bytes), "r"(smem_addr(bar)) : "memory");
 }
-
-// Ring of kStages slots of kSlotBytes each.  One thread (thread 0) issues the copies; everybody
-// waits on the slot's barrier.  Use by a persistent CTA that consumes items 0, 1, 2, ... in order:
-//     ring.init();  for the first kStages items: ring.issue(item, src, bytes)
-//     loop item:    ok = ring.wait(item);  ... read ring.slot(item) ...;  __syncthreads();
-//                   ring.issue(item + kStages, src, bytes)
-// bytes == 0 means "not eligible for a bulk copy": nothing is issued, wait() returns at once, and
-// the caller fills the slot itself.
-template <int kStages, int kSlotBytes>
-struct BulkRing {
-    alignas(128) unsigned char data[kStages][kSlotBytes];
-    alignas(8) uint64_t bar[kStages];
-
-    __device__ __forceinline__ void init() {
-        if (threadIdx.x == 0) {
-            for (int s = 0; s < kStages; ++s) mbar_init(&bar[s], 1);
-            fence_barrier_init();
-        }
-        __syncthreads();
-    }
-    __device__ __forceinline__ unsigned char* slot(int64_t item) { return data[item % kStages]; }
-    // Called by every thread after the barrier that ends the slot's previous use; thread 0 acts.
-    __device__ __forceinline__ void issue(int64_t item, const void* src, unsigned bytes) {
-        if (threadIdx.x == 0 && bytes != 0) {
-            const int s = (int)(item % kStages);
-            fence_proxy_async();
-            mbar_expect_tx(&bar[s], bytes);
-            bulk_copy_g2s(data[s], src, bytes, &bar[s]);
-        }
-    }
-    // use_index = how many bulk copies this slot has completed before this one (parity source).
-    __device__ __forceinline__ bool wait(int64_t item, unsigned use_index) {
-        return mbar_wait(&bar[item % kStages], use_index & 1u);
-    }
-};
 
 }  // namespace pwlq

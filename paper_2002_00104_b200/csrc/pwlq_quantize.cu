@@ -1,12 +1,11 @@
 // Quantizer of Eq. 3 (integer code + region bit, Sec. 4) and its inverse (Eq. 1, first line).
 //
 // Both are single streaming passes bound by HBM.  A thread owns 8 consecutive values: two
-// 128-bit loads of x, then one 64-bit store of byte codes (or one 32-bit store of nibble-packed
+// 128-bit reads of x, then one 64-bit store of byte codes (or one 32-bit store of nibble-packed
 // codes) and one region-mask byte, so that a warp writes contiguous 256 / 128 / 32-byte runs.
-// CTAs are persistent and walk spans of 8192 values; the rows that overlap a span are staged in
-// shared memory with their constants (four divisions per row, done once per span), so a thread's
-// row lookups and constant fetches stay on chip, and the next span's loads are already in flight
-// while the current one is staged and computed.
+// The flat storage is cut into spans of 4096 values.  A CTA is a producer warp, which requests
+// the spans' values with bulk asynchronous copies and describes the rows of every span (row map
+// and row constants, see pwlq_rowmap.cuh), and eight consumer warps, which quantize.
 #include <algorithm>
 #include <mutex>
 
@@ -20,8 +19,8 @@ namespace pwlq {
 constexpr int kQThreads = 256;
 constexpr int kQChunk = kQThreads * 8;           // values one pass of the CTA covers
 constexpr int kQChunks = 2;                      // passes per span
-constexpr int kQSpan = kQChunk * kQChunks;       // values per span (one staged row table)
-constexpr int kQStages = 2;                      // spans in flight per CTA (quantize)
+constexpr int kQSpan = kQChunk * kQChunks;       // values per span
+static_assert(kQSpan == kMapSpan, "the spans of the row maps");
 
 static __device__ int g_quantize_timeout;        // set when a bounded wait expired
 
@@ -33,12 +32,6 @@ __device__ __forceinline__ int chunk_offset(int c) {
     return ((int)threadIdx.x >> 5) * (kQSpan / (kQThreads / 32)) + c * 256 + ((int)threadIdx.x & 31) * 8;
 }
 
-// The rows overlapping the CTA's current span, with their constants (ragged rows, and dense rows
-// shorter than a span).
-constexpr int kQTableRows = 512;                 // rows of >= 8 values always fit
-typedef SpanTable<true, kQTableRows> QuantSmem;
-typedef RowFetch<kQTableRows> QuantFetch;
-
 // Per-row inputs: m = abs-max and lo = nullptr (signed scheme), or m = upper and lo = lower
 // bound of a one-sided range; p = breakpoint.
 struct RowArrays {
@@ -47,13 +40,13 @@ struct RowArrays {
     const float* __restrict__ p;
 };
 
-// The row a thread is currently in: constants in registers, refreshed when it crosses a boundary.
+// The row a thread is currently in, with its constants in registers, looked up in global memory
+// (long dense rows: the register-only dequantize kernel; and spans without a usable row map).
 struct RowState {
     int64_t beg = 0, end = 0;
     float m = 0.0f;                                // range width (abs-max, or hi - lo)
     float lo = 0.0f;                               // lower bound of a one-sided range, else 0
     PieceParams P;
-    int loc = -1;                                  // index in the staged table (-1: not from it)
 
     // Range width and lower bound of `row` straight from global memory.
     static __device__ __forceinline__ void load_range(const RowArrays& A, int64_t row, float& m,
@@ -62,40 +55,18 @@ struct RowState {
         lo = 0.0f;
         if (A.lo) { lo = __ldg(A.lo + row); m = __fsub_rn(m, lo); }
     }
-    template <bool TABLE>
-    __device__ __forceinline__ void seek(const QuantSmem& S, const Rows& rows, const RowArrays& A,
-                                         float Lf, int64_t i) {
+    __device__ __forceinline__ void seek(const Rows& rows, const RowArrays& A, float Lf, int64_t i) {
         if (i >= beg && i < end) return;
-        loc = TABLE ? S.find(i) : -1;
-        if (loc >= 0) {
-            beg = S.off[loc];
-            end = S.off[loc + 1];
-            m = S.m[loc];
-            lo = S.lo[loc];
-            P = S.P[loc];
-        } else {                                   // long dense rows, or beyond the staged rows
-            const int64_t row = rows.row_of(i);
-            beg = rows.begin(row);
-            end = rows.begin(row + 1);
-            load_range(A, row, m, lo);
-            P = make_params(m, __ldg(A.p + row), Lf);
-        }
+        const int64_t row = rows.row_of(i);
+        beg = rows.begin(row);
+        end = rows.begin(row + 1);
+        load_range(A, row, m, lo);
+        P = make_params(m, __ldg(A.p + row), Lf);
     }
-    // Constants of the row that follows, if that row reaches at least to need_end.
-    template <bool TABLE>
-    __device__ __forceinline__ bool next_row(const QuantSmem& S, const Rows& rows,
-                                             const RowArrays& A, float Lf, int64_t need_end,
-                                             float& mB, float& loB, PieceParams& PB,
-                                             int64_t& endB) const {
-        if (TABLE) {
-            if (loc < 0 || loc + 1 >= kQTableRows) return false;
-            endB = S.off[loc + 2];
-            if (endB < need_end) return false;
-            mB = S.m[loc + 1];
-            loB = S.lo[loc + 1];
-            PB = S.P[loc + 1];
-            return true;
-        }
+    // Constants of the row that follows (dense rows), if that row reaches at least to need_end.
+    __device__ __forceinline__ bool next_row(const Rows& rows, const RowArrays& A, float Lf,
+                                             int64_t need_end, float& mB, float& loB,
+                                             PieceParams& PB, int64_t& endB) const {
         if (rows.offsets || rows.n < need_end - end) return false;
         const int64_t row = rows.dense_row(end);
         if (row >= rows.C) return false;
@@ -112,13 +83,7 @@ struct RowState {
         m = mB;
         lo = loB;
         P = PB;
-        if (loc >= 0) ++loc;
     }
-};
-
-struct QuantizeSmem {
-    BulkRing<kQStages, kQSpan * 4> ring;
-    QuantSmem rows;
 };
 
 // Bytes of span `span` if it can be fetched by a bulk copy (aligned base, whole 16-byte units).
@@ -209,218 +174,6 @@ __device__ __forceinline__ void quantize8(const float (&xv)[8], int split, float
     (void)kR;
 }
 
-// Persistent CTAs.  TABLE (ragged rows, or dense rows shorter than a span): each CTA walks a block
-// of consecutive spans, so the next span's first row is the row this span ends in and its row
-// table can be requested without a search.  Otherwise every gridDim.x-th span.  The values of
-// the next spans are already on their way into a ring of shared-memory slots (bulk asynchronous
-// copies) while the current span is quantized.
-//
-// A warp's 256 values of one pass are handled by one of three warp-uniform variants: all lanes
-// have their eight values inside one row; some lanes have them in two rows (per-value selects
-// between the two rows' constants); anything else (the tensor's tail, rows with m = 0, more than
-// two rows in eight values) takes the per-value path.
-template <bool PACKED, bool WANT_FAKE, bool TABLE, bool UNS>
-__global__ void __launch_bounds__(kQThreads)
-quantize_kernel(const float* __restrict__ x, Rows rows, int64_t total, int bits, RowArrays A,
-                uint8_t* __restrict__ codes, uint8_t* __restrict__ mask, float* __restrict__ fake,
-                int vec_in, int vec_fake, int vec_codes, int64_t spans_per_cta) {
-    extern __shared__ __align__(128) unsigned char smem_raw[];
-    QuantizeSmem& Q = *reinterpret_cast<QuantizeSmem*>(smem_raw);
-    QuantSmem& S = Q.rows;
-    __shared__ int s_abort;
-    const unsigned full = 0xffffffffu;
-    const int Li = UNS ? (1 << bits) - 1 : (1 << (bits - 1)) - 1;    // largest level of a piece
-    const float Lf = (float)Li;
-    const uint32_t sign_unit = 1u << (bits - 1);      // value of the sign bit inside a code
-    const int sign_shift = 32 - bits;                 // moves bit 31 onto the code's sign bit
-    const int64_t nspans = (total + kQSpan - 1) / kQSpan;
-    const int64_t first = TABLE ? blockIdx.x * spans_per_cta : blockIdx.x;
-    const int64_t stride = TABLE ? 1 : gridDim.x;
-    const int64_t last = TABLE ? min(first + spans_per_cta, nspans) : nspans;        // exclusive
-    const int64_t block_end = min(last * kQSpan, total);   // rows that start later are not this CTA's
-    if (threadIdx.x == 0) s_abort = 0;
-    Q.ring.init();
-    for (int it = 0; it < kQStages; ++it) {
-        const int64_t span = first + (int64_t)it * stride;
-        if (span < last) Q.ring.issue(it, x + span * kQSpan, q_bulk_bytes(span, total, vec_in));
-    }
-    int64_t row0 = 0;                               // first staged row of the current span
-    QuantFetch nf;
-    if (TABLE && first < last) {
-        row0 = cta_row_near(rows, first * kQSpan);
-        S.fetch(rows, A.m, A.p, A.lo, row0, nf);
-        S.commit(nf, block_end, Lf);
-        __syncthreads();
-    }
-    RowState ws;                                    // the row a warp's pass starts in (warp-uniform)
-    int64_t it = 0;
-    for (int64_t span = first; span < last; span += stride, ++it) {
-        const int64_t span_beg = span * kQSpan;
-        const int64_t span_end = min(span_beg + kQSpan, total);
-        // the staged rows end before the next span does: request the window that starts in the
-        // row in which this span ends now, write it when this span is done
-        int64_t next_row0 = 0;
-        const bool has_next = TABLE && span + 1 < last && !S.covers(min(span_end + kQSpan, total));
-        if (has_next) {
-            const int l = S.find(span_end);
-            next_row0 = (l >= 0) ? row0 + l : warp_row_of(rows, span_end);
-            S.fetch(rows, A.m, A.p, A.lo, next_row0, nf);
-        }
-        float* xs = reinterpret_cast<float*>(Q.ring.slot(it));
-        if (q_bulk_bytes(span, total, vec_in) != 0) {
-            if (!Q.ring.wait(it, (unsigned)(it / kQStages))) s_abort = 1;   // never expected
-        } else {                                       // unaligned base or ragged tail: plain loads
-            for (int i = threadIdx.x; i < (int)(span_end - span_beg); i += kQThreads)
-                xs[i] = x[span_beg + i];
-            __syncthreads();
-        }
-#pragma unroll 1
-        for (int c = 0; c < kQChunks; ++c) {
-            const int li = chunk_offset(c);
-            const int64_t i0 = span_beg + li;
-            const int cnt = (int)max((int64_t)0, min((int64_t)8, total - i0));
-            const float4 xa = *reinterpret_cast<const float4*>(xs + li);
-            const float4 xb = *reinterpret_cast<const float4*>(xs + li + 4);
-            const float xv[8] = {xa.x, xa.y, xa.z, xa.w, xb.x, xb.y, xb.z, xb.w};
-            uint32_t w0 = 0, w1 = 0, mb = 0;
-            float yv[8];
-            // Warp-uniform part: the pass starts in row A (kept in ws from pass to pass); if the
-            // row ends inside the pass, row B follows and must reach to the end of the pass.
-            const int64_t pass_beg = i0 - ((int)threadIdx.x & 31) * 8, pass_end = pass_beg + 256;
-            bool done = false;
-            if (pass_end <= total) {
-                ws.seek<TABLE>(S, rows, A, Lf, pass_beg);
-                if (ws.m > 0.0f) {
-                    if (ws.end >= pass_end) {
-                        quantize8<PACKED, WANT_FAKE, false, UNS>(xv, 8, ws.m, ws.lo, ws.P, ws.m, ws.lo,
-                                                                 ws.P, Lf, Li, sign_unit, sign_shift,
-                                                                 w0, w1, mb, yv);
-                        done = true;
-                    } else {
-                        float mB = 0.0f, loB = 0.0f;
-                        PieceParams PB = ws.P;
-                        int64_t endB = 0;
-                        if (ws.next_row<TABLE>(S, rows, A, Lf, pass_end, mB, loB, PB, endB) &&
-                            mB > 0.0f) {
-                            const int split = (int)max((int64_t)0, min((int64_t)8, ws.end - i0));
-                            if (__any_sync(full, split > 0 && split < 8)) {   // a lane holds both rows
-                                quantize8<PACKED, WANT_FAKE, true, UNS>(xv, split, ws.m, ws.lo, ws.P, mB,
-                                                                        loB, PB, Lf, Li, sign_unit,
-                                                                        sign_shift, w0, w1, mb, yv);
-                            } else {
-                                const bool second = split == 0;
-                                PieceParams PL;
-                                PL.p = second ? PB.p : ws.P.p;
-                                PL.s1 = second ? PB.s1 : ws.P.s1;
-                                PL.inv1 = second ? PB.inv1 : ws.P.inv1;
-                                PL.s2 = second ? PB.s2 : ws.P.s2;
-                                PL.inv2 = second ? PB.inv2 : ws.P.inv2;
-                                const float mL = second ? mB : ws.m;
-                                const float loL = second ? loB : ws.lo;
-                                quantize8<PACKED, WANT_FAKE, false, UNS>(xv, 8, mL, loL, PL, mL, loL,
-                                                                         PL, Lf, Li, sign_unit,
-                                                                         sign_shift, w0, w1, mb, yv);
-                            }
-                            ws.advance(mB, loB, PB, endB);
-                            done = true;
-                        }
-                    }
-                }
-            }
-            if (!done) {
-                // Per-thread part (short rows, rows with m = 0, the tensor's tail): every lane
-                // looks up its own row; lanes whose eight values lie in two rows select between
-                // the two rows' constants per value; anything else takes the per-value path.
-                RowState rs;
-                int split = 8;
-                bool simple = true, two = false;
-                float mB = 0.0f, loB = 0.0f;
-                PieceParams PB = ws.P;
-                int64_t endB = 0;
-                if (cnt > 0) {
-                    rs.seek<TABLE>(S, rows, A, Lf, i0);
-                    split = (int)min((int64_t)8, rs.end - i0);
-                    simple = cnt == 8 && split == 8 && rs.m > 0.0f;
-                    if (cnt == 8 && split < 8 && rs.m > 0.0f)
-                        two = rs.next_row<TABLE>(S, rows, A, Lf, i0 + 8, mB, loB, PB, endB) &&
-                              mB > 0.0f;
-                }
-                if (__all_sync(full, simple || two)) {
-                    if (!two) { mB = rs.m; loB = rs.lo; PB = rs.P; split = 8; }
-                    quantize8<PACKED, WANT_FAKE, true, UNS>(xv, split, rs.m, rs.lo, rs.P, mB, loB, PB,
-                                                            Lf, Li, sign_unit, sign_shift, w0, w1, mb,
-                                                            yv);
-                } else {
-#pragma unroll
-                    for (int t = 0; t < 8; ++t) {
-                        yv[t] = 0.0f;
-                        if (t < cnt) {
-                            rs.seek<TABLE>(S, rows, A, Lf, i0 + t);
-                            if (UNS) yv[t] = rs.lo;                // a constant row delivers lo
-                            if (rs.m > 0.0f) {
-                                const float xi = xv[t];
-                                const int neg = !UNS && xi < 0.0f;
-                                int q, tail;
-                                float v;
-                                const float a = UNS ? fminf(fmaxf(__fsub_rn(xi, rs.lo), 0.0f), rs.m)
-                                                    : fminf(fabsf(xi), rs.m);
-                                quantize_mag(a, rs.P, Lf, q, tail, v);
-                                const uint32_t code = (uint32_t)((neg << (bits - 1)) | q);
-                                if (PACKED) w0 |= code << (4 * t);
-                                else if (t < 4) w0 |= code << (8 * t);
-                                else w1 |= code << (8 * (t - 4));
-                                mb |= (uint32_t)tail << t;
-                                yv[t] = UNS ? __fadd_rn(v, rs.lo) : (neg ? -v : v);
-                            }
-                        }
-                    }
-                }
-            }
-            if (cnt == 0) continue;
-            mask[i0 >> 3] = (uint8_t)mb;
-            if (PACKED) {
-                uint8_t* dst = codes + (i0 >> 1);
-                if (vec_codes && cnt == 8) {
-                    *reinterpret_cast<uint32_t*>(dst) = w0;
-                } else {
-                    const int nb = (cnt + 1) >> 1;
-                    for (int b = 0; b < nb; ++b) dst[b] = (uint8_t)(w0 >> (8 * b));
-                }
-            } else {
-                uint8_t* dst = codes + i0;
-                if (vec_codes && cnt == 8) {
-                    *reinterpret_cast<uint2*>(dst) = make_uint2(w0, w1);
-                } else {
-                    for (int t = 0; t < cnt; ++t)
-                        dst[t] = (uint8_t)((t < 4 ? w0 : w1) >> (8 * (t & 3)));
-                }
-            }
-            if (WANT_FAKE) {
-                if (vec_fake && cnt == 8) {
-                    __stcs(reinterpret_cast<float4*>(fake + i0), make_float4(yv[0], yv[1], yv[2], yv[3]));
-                    __stcs(reinterpret_cast<float4*>(fake + i0 + 4), make_float4(yv[4], yv[5], yv[6], yv[7]));
-                } else {
-                    for (int t = 0; t < cnt; ++t) fake[i0 + t] = yv[t];
-                }
-            }
-        }
-        __syncthreads();                            // slot and row table are free again
-        if (s_abort) {                               // a wait ran out: report and leave
-            if (threadIdx.x == 0) atomicExch(&g_quantize_timeout, 1);
-            return;
-        }
-        const int64_t ahead = span + (int64_t)kQStages * stride;
-        if (ahead < last)
-            Q.ring.issue(it + kQStages, x + ahead * kQSpan, q_bulk_bytes(ahead, total, vec_in));
-        if (has_next) {
-            S.commit(nf, block_end, Lf);
-            row0 = next_row0;
-            ws.beg = ws.end = 0;                     // indices into the window are stale
-            __syncthreads();                        // the next window is published
-        }
-    }
-}
-
 // ------------------------------------------------------------------ several rows per span
 // Producer / consumer form of the quantizer for ragged rows and dense rows shorter than a span
 // (see pwlq_rowmap.cuh): warp kMapConsumers fills the stages (bulk copy of the span's values, row
@@ -437,21 +190,6 @@ struct MapStage {
     SpanRowMap map;
     alignas(16) float4 qa[kMapSlots];
     alignas(16) float4 qb[QB ? kMapSlots : 1];
-};
-
-// Row of value i and its constants straight from global memory (spans without a usable map).
-struct GlobalRow {
-    int64_t beg = 0, end = 0;
-    float m = 0.0f, lo = 0.0f;
-    PieceParams P;
-    __device__ __forceinline__ void seek(const Rows& rows, const RowArrays& A, float Lf, int64_t i) {
-        if (i >= beg && i < end) return;
-        const int64_t row = rows.row_of(i);
-        beg = rows.begin(row);
-        end = rows.begin(row + 1);
-        RowState::load_range(A, row, m, lo);
-        P = make_params(m, __ldg(A.p + row), Lf);
-    }
 };
 
 __device__ __forceinline__ PieceParams params_of(const float4 qa, const float4 qb) {
@@ -497,6 +235,14 @@ quantize_map_kernel(const float* __restrict__ x, Rows rows, int64_t total, int b
         prod.Lf = Lf;
         // LONG: dense rows of at least a span, the map follows from the row length
         constexpr bool long_rows = LONG;
+        // the values of the first spans do not depend on the rows: request them before the search
+        for (int64_t span = first; span < last && span < first + kMapStages; ++span) {
+            const unsigned bytes = q_bulk_bytes(span, total, vec_in);
+            if (bytes != 0 && lane == 0) {
+                mbar_expect_tx(&full_bar[span - first], bytes);
+                bulk_copy_g2s(st[span - first].data, x + span * kMapSpan, bytes, &full_bar[span - first]);
+            }
+        }
         if (long_rows) prod.request_long(rows.dense_row(first * kMapSpan));
         else prod.request(warp_row_of(rows, first * kMapSpan), true);
         int64_t it = 0;
@@ -510,7 +256,7 @@ quantize_map_kernel(const float* __restrict__ x, Rows rows, int64_t total, int b
             const int64_t span_beg = span * kMapSpan, span_end = min(span_beg + kMapSpan, total);
             const unsigned bytes = q_bulk_bytes(span, total, vec_in);
             if (bytes != 0) {
-                if (lane == 0) {
+                if (lane == 0 && use > 0) {        // (first round: requested above)
                     // the stage was last read (by the consumers, whose arrivals this warp has
                     // waited for), not written, through the generic proxy: no proxy fence needed
                     mbar_expect_tx(&full_bar[s], bytes);
@@ -608,7 +354,7 @@ quantize_map_kernel(const float* __restrict__ x, Rows rows, int64_t total, int b
                     }
                 }
             } else {
-                GlobalRow rs;
+                RowState rs;
 #pragma unroll
                 for (int t = 0; t < 8; ++t) {
                     yv[t] = 0.0f;
@@ -735,54 +481,37 @@ __device__ __forceinline__ void dequantize8(uint32_t w0, uint32_t w1, uint32_t m
     }
 }
 
-template <bool PACKED, bool TABLE, bool UNS>
+// Register-only form for dense rows of many spans: a persistent grid, one CTA per slot of the
+// device, walks the spans with a stride; the codes and region bits of a thread's next span are
+// requested before the current one is expanded.  A warp's 256 values of one pass lie in one row
+// (constants kept in registers from pass to pass) or in two (the row that follows is looked up
+// when the first one ends); the tensor's tail and rows with m = 0 go value by value.
+template <bool PACKED, bool UNS>
 __global__ void __launch_bounds__(kQThreads)
-dequantize_kernel(const uint8_t* __restrict__ codes, const uint8_t* __restrict__ mask, Rows rows,
-                  int64_t total, int bits, RowArrays A, float* __restrict__ y, int vec_codes,
-                  int vec_out, int64_t spans_per_cta) {
-    __shared__ QuantSmem S;
+dequantize_long_kernel(const uint8_t* __restrict__ codes, const uint8_t* __restrict__ mask, Rows rows,
+                       int64_t total, int bits, RowArrays A, float* __restrict__ y, int vec_codes,
+                       int vec_out) {
     const unsigned full = 0xffffffffu;
     const int qmask = UNS ? (1 << bits) - 1 : (1 << (bits - 1)) - 1;   // the level inside a code
     const float Lf = (float)qmask;
     const int sign_shift = 32 - bits;                 // moves a code's sign bit to bit 31
     const int64_t nspans = (total + kQSpan - 1) / kQSpan;
-    // the CTA's spans: consecutive with a row table (chained tables), strided otherwise
-    const int64_t first = TABLE ? blockIdx.x * spans_per_cta : blockIdx.x;
-    const int64_t stride = TABLE ? 1 : gridDim.x;
-    const int64_t last = TABLE ? min(first + spans_per_cta, nspans) : nspans;        // exclusive
-    const int64_t block_end = min(last * kQSpan, total);   // rows that start later are not this CTA's
+    const int64_t first = blockIdx.x, stride = gridDim.x;
     CodeRegs<PACKED> cur, nxt;
     RowState ws;                                    // the row a warp's pass starts in (warp-uniform)
     cur.load(codes, mask, first * kQSpan, total, vec_codes);
-    int64_t row0 = 0;                               // first staged row of the current span
-    QuantFetch nf;
-    if (TABLE && first < last) {
-        row0 = cta_row_near(rows, first * kQSpan);
-        S.fetch(rows, A.m, A.p, A.lo, row0, nf);
-        S.commit(nf, block_end, Lf);
-        __syncthreads();
-    }
-    for (int64_t span = first; span < last; span += stride) {
+    for (int64_t span = first; span < nspans; span += stride) {
         const int64_t span_beg = span * kQSpan;
-        const int64_t span_end = min(span_beg + kQSpan, total);
-        if (span + stride < last) nxt.load(codes, mask, (span + stride) * kQSpan, total, vec_codes);
-        int64_t next_row0 = 0;
-        const bool has_next = TABLE && span + 1 < last && !S.covers(min(span_end + kQSpan, total));
-        if (has_next) {
-            const int l = S.find(span_end);
-            next_row0 = (l >= 0) ? row0 + l : warp_row_of(rows, span_end);
-            S.fetch(rows, A.m, A.p, A.lo, next_row0, nf);
-        }
+        if (span + stride < nspans) nxt.load(codes, mask, (span + stride) * kQSpan, total, vec_codes);
 #pragma unroll
         for (int c = 0; c < kQChunks; ++c) {
             const int64_t i0 = span_beg + chunk_offset(c);
             const int cnt = (int)max((int64_t)0, min((int64_t)8, total - i0));
             float yv[8];
-            // warp-uniform part and per-thread part as in quantize_kernel
             const int64_t pass_beg = i0 - ((int)threadIdx.x & 31) * 8, pass_end = pass_beg + 256;
             bool done = false;
             if (pass_end <= total) {
-                ws.seek<TABLE>(S, rows, A, Lf, pass_beg);
+                ws.seek(rows, A, Lf, pass_beg);
                 if (ws.m > 0.0f) {
                     if (ws.end >= pass_end) {
                         dequantize8<PACKED, false, UNS>(cur.w0[c], cur.w1[c], cur.mb[c], 8, ws.P, ws.lo,
@@ -792,67 +521,32 @@ dequantize_kernel(const uint8_t* __restrict__ codes, const uint8_t* __restrict__
                         float mB = 0.0f, loB = 0.0f;
                         PieceParams PB = ws.P;
                         int64_t endB = 0;
-                        if (ws.next_row<TABLE>(S, rows, A, Lf, pass_end, mB, loB, PB, endB) &&
-                            mB > 0.0f) {
+                        if (ws.next_row(rows, A, Lf, pass_end, mB, loB, PB, endB) && mB > 0.0f) {
                             const int split = (int)max((int64_t)0, min((int64_t)8, ws.end - i0));
-                            if (__any_sync(full, split > 0 && split < 8)) {   // a lane holds both rows
-                                dequantize8<PACKED, true, UNS>(cur.w0[c], cur.w1[c], cur.mb[c], split,
-                                                               ws.P, ws.lo, PB, loB, qmask,
-                                                               sign_shift, yv);
-                            } else {
-                                const bool second = split == 0;
-                                PieceParams PL;
-                                PL.p = second ? PB.p : ws.P.p;
-                                PL.s1 = second ? PB.s1 : ws.P.s1;
-                                PL.s2 = second ? PB.s2 : ws.P.s2;
-                                PL.inv1 = PL.inv2 = 0.0f;
-                                const float loL = second ? loB : ws.lo;
-                                dequantize8<PACKED, false, UNS>(cur.w0[c], cur.w1[c], cur.mb[c], 8, PL,
-                                                                loL, PL, loL, qmask, sign_shift, yv);
-                            }
+                            dequantize8<PACKED, true, UNS>(cur.w0[c], cur.w1[c], cur.mb[c], split, ws.P,
+                                                           ws.lo, PB, loB, qmask, sign_shift, yv);
                             ws.advance(mB, loB, PB, endB);
                             done = true;
                         }
                     }
                 }
             }
-            if (!done) {
+            if (!__all_sync(full, done)) {
                 RowState rs;
-                int split = 8;
-                bool simple = true, two = false;
-                float mB = 0.0f, loB = 0.0f;
-                PieceParams PB = ws.P;
-                int64_t endB = 0;
-                if (cnt > 0) {
-                    rs.seek<TABLE>(S, rows, A, Lf, i0);
-                    split = (int)min((int64_t)8, rs.end - i0);
-                    simple = cnt == 8 && split == 8 && rs.m > 0.0f;
-                    if (cnt == 8 && split < 8 && rs.m > 0.0f)
-                        two = rs.next_row<TABLE>(S, rows, A, Lf, i0 + 8, mB, loB, PB, endB) &&
-                              mB > 0.0f;
-                }
-                if (__all_sync(full, simple || two)) {
-                    if (!two) { PB = rs.P; loB = rs.lo; split = 8; }
-                    dequantize8<PACKED, true, UNS>(cur.w0[c], cur.w1[c], cur.mb[c], split, rs.P, rs.lo,
-                                                   PB, loB, qmask, sign_shift, yv);
-                } else {
 #pragma unroll
-                    for (int t = 0; t < 8; ++t) {
-                        yv[t] = 0.0f;
-                        if (t < cnt) {
-                            rs.seek<TABLE>(S, rows, A, Lf, i0 + t);
-                            if (UNS) yv[t] = rs.lo;                // a constant row delivers lo
-                            if (rs.m > 0.0f) {
-                                const uint32_t code = code_of<PACKED>(cur.w0[c], cur.w1[c], t);
-                                const int tail = (cur.mb[c] >> t) & 1;
-                                const int neg = !UNS && ((code >> (bits - 1)) & 1);
-                                const float q = (float)(code & qmask);
-                                const float s = tail ? rs.P.s2 : rs.P.s1;
-                                const float z = tail ? rs.P.p : 0.0f;
-                                float v = __fmul_rn(q, s);
-                                v = __fadd_rn(v, z);
-                                yv[t] = UNS ? __fadd_rn(v, rs.lo) : (neg ? -v : v);
-                            }
+                for (int t = 0; t < 8; ++t) {
+                    yv[t] = 0.0f;
+                    if (t < cnt) {
+                        rs.seek(rows, A, Lf, i0 + t);
+                        if (UNS) yv[t] = rs.lo;                    // a constant row delivers lo
+                        if (rs.m > 0.0f) {
+                            const uint32_t code = code_of<PACKED>(cur.w0[c], cur.w1[c], t);
+                            const int tail = (cur.mb[c] >> t) & 1;
+                            const int neg = !UNS && ((code >> (bits - 1)) & 1);
+                            const float q = (float)(code & qmask);
+                            float v = __fmul_rn(q, tail ? rs.P.s2 : rs.P.s1);
+                            v = __fadd_rn(v, tail ? rs.P.p : 0.0f);
+                            yv[t] = UNS ? __fadd_rn(v, rs.lo) : (neg ? -v : v);
                         }
                     }
                 }
@@ -864,13 +558,6 @@ dequantize_kernel(const uint8_t* __restrict__ codes, const uint8_t* __restrict__
             } else {
                 for (int t = 0; t < cnt; ++t) y[i0 + t] = yv[t];
             }
-        }
-        if (has_next) {
-            __syncthreads();                        // the window is no longer read
-            S.commit(nf, block_end, Lf);
-            row0 = next_row0;
-            ws.beg = ws.end = 0;                     // indices into the window are stale
-            __syncthreads();                        // the next window is published
         }
         cur = nxt;
     }
@@ -1006,7 +693,7 @@ dequantize_map_kernel(const uint8_t* __restrict__ codes, const uint8_t* __restri
                     }
                 }
             } else {
-                GlobalRow rs;
+                RowState rs;
 #pragma unroll
                 for (int t = 0; t < 8; ++t) {
                     yv[t] = 0.0f;
@@ -1068,16 +755,17 @@ static int64_t device_slots(const void* kernel, int threads, size_t smem) {
     return ctas;
 }
 
-// Grid and spans per CTA.  Without a row table (long dense rows) the cost per span is the same
-// everywhere: a persistent grid, one CTA per slot, walks the spans with a stride.  With a row
-// table the cost per span depends on the row lengths, so consecutive spans are handed out in
-// small blocks (about four per slot) and the hardware scheduler balances them.
+// Grid and spans per CTA.  The register-only dequantize kernel for very long dense rows runs a
+// persistent grid, one CTA per slot of the device, that walks the spans with a stride.  The
+// producer / consumer kernels walk consecutive spans, handed out in blocks of at most 32, about
+// four per slot: a block should be long enough to pay for the producer's start (finding its first
+// row), and short enough for the hardware scheduler to even out what differs between spans.
 struct SpanGrid { unsigned grid; int64_t per_cta; };
 static SpanGrid span_grid(const void* kernel, int threads, size_t smem, int64_t nspans, bool table) {
     const int64_t slots = device_slots(kernel, threads, smem);
     if (!table) return SpanGrid{(unsigned)std::min(nspans, slots), 0};
     const int64_t per_cta =
-        std::min<int64_t>(std::max<int64_t>((nspans + 4 * slots - 1) / (4 * slots), 4), 32);
+        std::min<int64_t>(std::max<int64_t>((nspans + 4 * slots - 1) / (4 * slots), 1), 32);
     return SpanGrid{(unsigned)((nspans + per_cta - 1) / per_cta), per_cta};
 }
 
@@ -1098,41 +786,29 @@ cudaError_t launch_quantize(const float* x, const int64_t* row_offsets, int64_t 
     const bool packed = (layout == 1 && bits <= 4);
     const int64_t nspans = (total + kQSpan - 1) / kQSpan;
     const int vec_in = aligned(x, 16), vec_fake = fake ? aligned(fake, 16) : 0;
-    const size_t smem = sizeof(QuantizeSmem);
     const int vec_codes = packed ? aligned(codes, 4) : aligned(codes, 8);
-    const bool table = true;
     const bool long_rows = row_offsets == nullptr && n >= kMapSpan;   // the map follows from n
-#define PWLQ_LAUNCH_QUANTIZE(PK, FK, RG, UN)                                                      \
+#define PWLQ_LAUNCH_QUANTIZE(PK, FK, UN)                                                          \
     do {                                                                                          \
-        if (RG) {                                                                                 \
-            const size_t msmem = sizeof(MapStage<true, FK || UN>) * kMapStages;                   \
-            if (long_rows) {                                                                      \
-                const SpanGrid g = span_grid((const void*)quantize_map_kernel<PK, FK, UN, true>,  \
-                                             kMapThreads, msmem, nspans, true);                   \
-                quantize_map_kernel<PK, FK, UN, true><<<g.grid, kMapThreads, msmem, stream>>>(    \
-                    x, rows, total, bits, A, codes, mask, fake, vec_in, vec_fake, vec_codes,      \
-                    g.per_cta);                                                                   \
-            } else {                                                                              \
-                const SpanGrid g = span_grid((const void*)quantize_map_kernel<PK, FK, UN, false>, \
-                                             kMapThreads, msmem, nspans, true);                   \
-                quantize_map_kernel<PK, FK, UN, false><<<g.grid, kMapThreads, msmem, stream>>>(   \
-                    x, rows, total, bits, A, codes, mask, fake, vec_in, vec_fake, vec_codes,      \
-                    g.per_cta);                                                                   \
-            }                                                                                     \
-            break;                                                                                \
+        const size_t msmem = sizeof(MapStage<true, FK || UN>) * kMapStages;                       \
+        if (long_rows) {                                                                          \
+            const SpanGrid g = span_grid((const void*)quantize_map_kernel<PK, FK, UN, true>,      \
+                                         kMapThreads, msmem, nspans, true);                       \
+            quantize_map_kernel<PK, FK, UN, true><<<g.grid, kMapThreads, msmem, stream>>>(        \
+                x, rows, total, bits, A, codes, mask, fake, vec_in, vec_fake, vec_codes,          \
+                g.per_cta);                                                                       \
+        } else {                                                                                  \
+            const SpanGrid g = span_grid((const void*)quantize_map_kernel<PK, FK, UN, false>,     \
+                                         kMapThreads, msmem, nspans, true);                       \
+            quantize_map_kernel<PK, FK, UN, false><<<g.grid, kMapThreads, msmem, stream>>>(       \
+                x, rows, total, bits, A, codes, mask, fake, vec_in, vec_fake, vec_codes,          \
+                g.per_cta);                                                                       \
         }                                                                                         \
-        const SpanGrid g = span_grid((const void*)quantize_kernel<PK, FK, RG, UN>, kQThreads,     \
-                                     smem, nspans, RG);                                           \
-        quantize_kernel<PK, FK, RG, UN><<<g.grid, kQThreads, smem, stream>>>(                     \
-            x, rows, total, bits, A, codes, mask, fake, vec_in, vec_fake, vec_codes, g.per_cta);  \
     } while (0)
-#define PWLQ_LAUNCH_QUANTIZE_UN(PK, FK, RG) \
-    do { if (lo) PWLQ_LAUNCH_QUANTIZE(PK, FK, RG, true); else PWLQ_LAUNCH_QUANTIZE(PK, FK, RG, false); } while (0)
-#define PWLQ_LAUNCH_QUANTIZE_RG(PK, FK) \
-    do { if (table) PWLQ_LAUNCH_QUANTIZE_UN(PK, FK, true); else PWLQ_LAUNCH_QUANTIZE_UN(PK, FK, false); } while (0)
-    if (packed) { if (fake) PWLQ_LAUNCH_QUANTIZE_RG(true, true); else PWLQ_LAUNCH_QUANTIZE_RG(true, false); }
-    else        { if (fake) PWLQ_LAUNCH_QUANTIZE_RG(false, true); else PWLQ_LAUNCH_QUANTIZE_RG(false, false); }
-#undef PWLQ_LAUNCH_QUANTIZE_RG
+#define PWLQ_LAUNCH_QUANTIZE_UN(PK, FK) \
+    do { if (lo) PWLQ_LAUNCH_QUANTIZE(PK, FK, true); else PWLQ_LAUNCH_QUANTIZE(PK, FK, false); } while (0)
+    if (packed) { if (fake) PWLQ_LAUNCH_QUANTIZE_UN(true, true); else PWLQ_LAUNCH_QUANTIZE_UN(true, false); }
+    else        { if (fake) PWLQ_LAUNCH_QUANTIZE_UN(false, true); else PWLQ_LAUNCH_QUANTIZE_UN(false, false); }
 #undef PWLQ_LAUNCH_QUANTIZE_UN
 #undef PWLQ_LAUNCH_QUANTIZE
     return cudaGetLastError();
@@ -1147,11 +823,16 @@ cudaError_t launch_dequantize(const uint8_t* codes, const uint8_t* mask,
     const RowArrays A{m, lo, p};
     const bool packed = (layout == 1 && bits <= 4);
     const int64_t nspans = (total + kQSpan - 1) / kQSpan;
-#define PWLQ_LAUNCH_DEQUANTIZE(PK, RG, UN)                                                        \
+#define PWLQ_LAUNCH_DEQUANTIZE(PK, UN)                                                            \
     do {                                                                                          \
-        if (RG) {                                                                                 \
+        const int vc = aligned(codes, PK ? 4 : 8), vo = aligned(y, 16);                           \
+        if (very_long) {                                                                          \
+            const SpanGrid g = span_grid((const void*)dequantize_long_kernel<PK, UN>, kQThreads,  \
+                                         0, nspans, false);                                       \
+            dequantize_long_kernel<PK, UN><<<g.grid, kQThreads, 0, stream>>>(                     \
+                codes, mask, rows, total, bits, A, y, vc, vo);                                    \
+        } else {                                                                                  \
             const size_t msmem = sizeof(MapStage<false, UN>) * kMapStages;                        \
-            const int vc = aligned(codes, PK ? 4 : 8), vo = aligned(y, 16);                       \
             if (long_rows) {                                                                      \
                 const SpanGrid g = span_grid((const void*)dequantize_map_kernel<PK, UN, true>,    \
                                              kMapThreads, msmem, nspans, true);                   \
@@ -1163,22 +844,15 @@ cudaError_t launch_dequantize(const uint8_t* codes, const uint8_t* mask,
                 dequantize_map_kernel<PK, UN, false><<<g.grid, kMapThreads, msmem, stream>>>(     \
                     codes, mask, rows, total, bits, A, y, vc, vo, g.per_cta);                     \
             }                                                                                     \
-            break;                                                                                \
         }                                                                                         \
-        const SpanGrid g = span_grid((const void*)dequantize_kernel<PK, RG, UN>, kQThreads, 0,    \
-                                     nspans, RG);                                                 \
-        dequantize_kernel<PK, RG, UN><<<g.grid, kQThreads, 0, stream>>>(                          \
-            codes, mask, rows, total, bits, A, y, aligned(codes, PK ? 4 : 8), aligned(y, 16),     \
-            g.per_cta);                                                                           \
     } while (0)
-#define PWLQ_LAUNCH_DEQUANTIZE_UN(PK, RG) \
-    do { if (lo) PWLQ_LAUNCH_DEQUANTIZE(PK, RG, true); else PWLQ_LAUNCH_DEQUANTIZE(PK, RG, false); } while (0)
+#define PWLQ_LAUNCH_DEQUANTIZE_UN(PK) \
+    do { if (lo) PWLQ_LAUNCH_DEQUANTIZE(PK, true); else PWLQ_LAUNCH_DEQUANTIZE(PK, false); } while (0)
     // Dense rows of many spans stream through the register-only kernel (no row lookups worth
     // speaking of); everything else goes through the producer / consumer kernel.
-    const bool table = row_offsets != nullptr || n < 16 * (int64_t)kMapSpan;
+    const bool very_long = row_offsets == nullptr && n >= 16 * (int64_t)kMapSpan;
     const bool long_rows = row_offsets == nullptr && n >= kMapSpan;   // the map follows from n
-    if (packed) { if (table) PWLQ_LAUNCH_DEQUANTIZE_UN(true, true); else PWLQ_LAUNCH_DEQUANTIZE_UN(true, false); }
-    else        { if (table) PWLQ_LAUNCH_DEQUANTIZE_UN(false, true); else PWLQ_LAUNCH_DEQUANTIZE_UN(false, false); }
+    if (packed) PWLQ_LAUNCH_DEQUANTIZE_UN(true); else PWLQ_LAUNCH_DEQUANTIZE_UN(false);
 #undef PWLQ_LAUNCH_DEQUANTIZE_UN
 #undef PWLQ_LAUNCH_DEQUANTIZE
     return cudaGetLastError();
