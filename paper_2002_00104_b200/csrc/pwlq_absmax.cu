@@ -253,11 +253,19 @@ absmax_kernel(const float* __restrict__ x, Rows rows, int64_t total, uint32_t* _
                 const int fpos = flag ? __ffs(nib) - 1 : 8;
                 const uint32_t low = (1u << fpos) - 1u;          // bit j: value j lies before my start
                 Fold<MINMAX> h, t;
+                if (!__any_sync(full, (nib & 0xFEu) != 0)) {
+                    // every start is at a lane's first value (row lengths that are multiples of
+                    // eight): a lane's values all go one way
 #pragma unroll
-                for (int j = 0; j < 8; ++j) {
-                    const uint32_t hm = 0u - ((low >> j) & 1u);
-                    h.add_keys(ka[j] & hm, kb[j] & hm);
-                    t.add_keys(ka[j] & ~hm, kb[j] & ~hm);
+                    for (int j = 0; j < 8; ++j) t.add_keys(ka[j], kb[j]);
+                    if (!flag) { h = t; t.clear(); }
+                } else {
+#pragma unroll
+                    for (int j = 0; j < 8; ++j) {
+                        const uint32_t hm = 0u - ((low >> j) & 1u);
+                        h.add_keys(ka[j] & hm, kb[j] & hm);
+                        t.add_keys(ka[j] & ~hm, kb[j] & ~hm);
+                    }
                 }
                 // inclusive scan over the lanes, restarted at every lane with a start
                 Fold<MINMAX> sc = flag ? t : h;

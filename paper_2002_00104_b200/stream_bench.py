@@ -1,7 +1,7 @@
 """Back-to-back timing of the HBM-bound kernels (abs-max, quantize, dequantize) on inputs larger
 than the 126 MB L2, so that every launch streams from HBM without an eviction pass in between.
 
-    python -m paper_2002_00104_b200.stream_bench [--values N] [--reps R]
+    python -m paper_2002_00104_b200.stream_bench [--values N] [--reps R] [--only LAYOUT]
 
 Prints one line per (layout, kernel): microseconds per launch and algorithmic GB/s (abs-max:
 4 B/value read; quantize and dequantize with packed 4-bit codes: 4 + 0.5 + 0.125 B/value), next to
@@ -58,18 +58,32 @@ def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--values", type=int, default=1 << 27, help="values per dense tensor (512 MB)")
     ap.add_argument("--reps", type=int, default=10)
+    ap.add_argument("--only", default=None,
+                    help="run only the layouts whose name contains this text (e.g. 'resnet50')")
     args = ap.parse_args()
     N = args.values
-    g = torch.Generator(device="cuda")
-    g.manual_seed(0)
-    x = torch.randn(N, device="cuda", generator=g) * 0.02
-    run("dense, 1 row", x.view(1, N), None, 1, N, args.reps)
-    run("dense, rows of 4096", x.view(N // 4096, 4096), None, N // 4096, 4096, args.reps)
-    run("dense, rows of 147", x[:147 * (N // 147)].view(N // 147, 147), None, N // 147, 147, args.reps)
-    xr, ro = tiled(W.resnet50(), 5)
-    run("ragged, resnet50 x5", xr, ro, None, None, args.reps)
-    xr, ro = tiled(W.mobilenetv2(), 30)
-    run("ragged, mobilenetv2 x30", xr, ro, None, None, args.reps, bits=3)
+
+    def wanted(name):
+        return args.only is None or args.only in name
+
+    if wanted("dense"):
+        g = torch.Generator(device="cuda")
+        g.manual_seed(0)
+        x = torch.randn(N, device="cuda", generator=g) * 0.02
+        if wanted("dense, 1 row"):
+            run("dense, 1 row", x.view(1, N), None, 1, N, args.reps)
+        if wanted("dense, rows of 4096"):
+            run("dense, rows of 4096", x.view(N // 4096, 4096), None, N // 4096, 4096, args.reps)
+        if wanted("dense, rows of 147"):
+            run("dense, rows of 147", x[:147 * (N // 147)].view(N // 147, 147), None, N // 147, 147,
+                args.reps)
+        del x
+    if wanted("ragged, resnet50 x5"):
+        xr, ro = tiled(W.resnet50(), 5)
+        run("ragged, resnet50 x5", xr, ro, None, None, args.reps)
+    if wanted("ragged, mobilenetv2 x30"):
+        xr, ro = tiled(W.mobilenetv2(), 30)
+        run("ragged, mobilenetv2 x30", xr, ro, None, None, args.reps, bits=3)
 
 
 if __name__ == "__main__":
