@@ -1,0 +1,116 @@
+"""GPU parity of the streaming kernels (abs-max, min/max, quantize, dequantize) on row layouts
+chosen around the limits of their row maps: a span of the flat storage is 4096 values, a map
+describes up to about 510 rows of a span, rows may start exactly at span boundaries, be empty, be
+shorter than the eight values a lane owns, or change length from span to span.  Everything is
+compared with the CPU oracle bit for bit."""
+import numpy as np
+import pytest
+import torch
+
+from gpu_util import dev
+
+pytestmark = [pytest.mark.gpu,
+              pytest.mark.skipif(not torch.cuda.is_available(), reason="needs a CUDA device")]
+
+SPAN = 4096
+
+
+@pytest.fixture(scope="module")
+def pwlq():
+    from paper_2002_00104_b200 import pwlq as _p
+    _p.load_library()
+    return _p
+
+
+def np_(t):
+    return t.cpu().numpy()
+
+
+def layouts():
+    """name -> list of row lengths."""
+    rng = np.random.default_rng(11)
+    out = {
+        # more rows per span than a map describes, then long rows again (slow spans and back)
+        "tiny_then_long": [1] * 3000 + [2, 3] * 900 + [5000, 3, 4096, 8192, 1],
+        # 455 / 512 / 585 rows per span: below, at and above the limit
+        "rows_of_9": [9] * 2000,
+        "rows_of_8": [8] * 2100,
+        "rows_of_7": [7] * 2400,
+        # starts exactly at span boundaries, with and without empty rows there
+        "span_aligned": [SPAN, SPAN, 0, SPAN, 2 * SPAN, 0, 0, SPAN - 1, 1, SPAN + 1, SPAN - 1],
+        # empty rows inside spans, in front and at the end
+        "empties": [0, 0, 100, 0, 200, 0, 0, 0, 3000, 0, 5000, 0, 17, 0],
+        # lengths that change between chunks of 32 rows (the producer's register chunks)
+        "mixed": list(rng.integers(1, 700, 400)),
+        # one start per lane group and odd lengths
+        "odd": [147] * 300 + [27] * 500 + [1153] * 20,
+        # more than 64 rows per span for many spans (rows beyond the two register chunks)
+        "rows_of_24": [24] * 3000,
+    }
+    return out
+
+
+def make(lengths, seed):
+    rng = np.random.default_rng(seed)
+    lengths = [int(v) for v in lengths]
+    total = int(sum(lengths))
+    x = rng.laplace(0, 0.05, total).astype(np.float32)
+    scale = np.repeat(10.0 ** rng.uniform(-2, 1, len(lengths)), lengths).astype(np.float32)
+    x *= scale
+    ro = np.concatenate([[0], np.cumsum(lengths)]).astype(np.int64)
+    return x, ro
+
+
+@pytest.mark.parametrize("name", sorted(layouts()))
+def test_absmax_and_minmax(pwlq, oracle, name):
+    x, ro = make(layouts()[name], 5)
+    m = pwlq.absmax(dev(x), row_offsets=dev(ro))
+    assert np.array_equal(np_(m), oracle.absmax(x, ro))
+    y = x + np.float32(0.125)
+    lo, hi = pwlq.minmax(dev(y), row_offsets=dev(ro))
+    olo, ohi = oracle.minmax(y, ro)
+    assert np.array_equal(np_(lo), olo) and np.array_equal(np_(hi), ohi)
+    assert pwlq.device_status() == 0
+
+
+@pytest.mark.parametrize("bits,layout", [(3, 1), (4, 1), (8, 0)])
+@pytest.mark.parametrize("name", sorted(layouts()))
+def test_quantize_dequantize(pwlq, oracle, name, bits, layout):
+    x, ro = make(layouts()[name], 7)
+    total = x.size
+    om = oracle.absmax(x, ro)
+    rng = np.random.default_rng(3)
+    p = (om * rng.uniform(0.05, 1.0, om.size)).astype(np.float32)
+    p[::7] = om[::7]                                   # p = m: empty tail
+    codes, mask, fake = pwlq.quantize(dev(x), bits, dev(om), dev(p), layout=layout,
+                                      row_offsets=dev(ro), want_fake=True)
+    oc, ok, of = oracle.quantize(x, bits, om, p, layout=layout, row_offsets=ro)
+    assert np.array_equal(np_(codes), oc) and np.array_equal(np_(mask), ok)
+    assert np_(fake).tobytes() == of.tobytes()
+    codes2, mask2, none = pwlq.quantize(dev(x), bits, dev(om), dev(p), layout=layout,
+                                        row_offsets=dev(ro), want_fake=False)
+    assert none is None
+    assert np.array_equal(np_(codes2), oc) and np.array_equal(np_(mask2), ok)
+    y = pwlq.dequantize(codes, mask, bits, dev(om), dev(p), layout=layout, row_offsets=dev(ro))
+    assert np_(y).tobytes() == of.tobytes()
+    assert total == y.numel()
+    assert pwlq.device_status() == 0
+
+
+@pytest.mark.parametrize("C,n", [(5000, 1), (700, 7), (600, 8), (520, 9), (3, 4095), (3, 4096),
+                                 (3, 4097), (2, 65535), (2, 65536), (2, 65537), (1, 300001)])
+def test_dense_rows_around_the_span(pwlq, oracle, C, n):
+    """Dense rows below, at and above one span and sixteen spans (where dequantize changes kernel)."""
+    rng = np.random.default_rng(C + n)
+    x = (rng.standard_normal((C, n)) * rng.uniform(0.01, 3.0, (C, 1))).astype(np.float32)
+    m = pwlq.absmax(dev(x))
+    om = oracle.absmax(x)
+    assert np.array_equal(np_(m), om)
+    p = (om * np.float32(0.3)).astype(np.float32)
+    codes, mask, fake = pwlq.quantize(dev(x), 4, m, dev(p), layout=1, want_fake=True)
+    oc, ok, of = oracle.quantize(x, 4, om, p, layout=1)
+    assert np.array_equal(np_(codes), oc) and np.array_equal(np_(mask), ok)
+    assert np_(fake).tobytes() == of.tobytes()
+    y = pwlq.dequantize(codes, mask, 4, m, dev(p), C=C, n=n, layout=1)
+    assert np_(y).tobytes() == of.tobytes()
+    assert pwlq.device_status() == 0
