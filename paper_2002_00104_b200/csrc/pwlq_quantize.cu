@@ -457,13 +457,20 @@ __device__ __forceinline__ uint32_t code_of(uint32_t w0, uint32_t w1, int t) {
 }
 
 // Eight consecutive codes, the first `split` of them in row A and the rest in row B (TWO = false:
-// all in row A), both rows with m > 0.  The level becomes a float through the mantissa of
-// 1.5 * 2^23 (exact for q < 2^22) instead of an integer conversion.
+// all in row A), both rows with m > 0.  The levels are masked out of the code words once per
+// eight values and spread to one byte each; a byte permute then puts a level straight under the
+// exponent of 1.5 * 2^23, whose subtraction leaves the level as a float (exact for q < 2^22)
+// without an integer conversion.  The sign bit is shifted from its place in the code word to
+// bit 31.
 // UNS: one-sided range, the code is the level and the delivered value is v + lo.
 template <bool PACKED, bool TWO, bool UNS>
 __device__ __forceinline__ void dequantize8(uint32_t w0, uint32_t w1, uint32_t mb, int split,
                                             const PieceParams& A, float loA, const PieceParams& B,
                                             float loB, int qmask, int sign_shift, float (&yv)[8]) {
+    // byte j of e0 / e1: level of value 2j / 2j + 1 (packed nibbles), or of value j / 4 + j
+    const uint32_t rep = (uint32_t)qmask * 0x01010101u;
+    const uint32_t e0 = w0 & rep;
+    const uint32_t e1 = (PACKED ? (w0 >> 4) : w1) & rep;
 #pragma unroll
     for (int t = 0; t < 8; ++t) {
         const bool second = TWO && t >= split;
@@ -471,13 +478,17 @@ __device__ __forceinline__ void dequantize8(uint32_t w0, uint32_t w1, uint32_t m
         const float p = second ? B.p : A.p;
         const float s1 = second ? B.s1 : A.s1;
         const float s2 = second ? B.s2 : A.s2;
-        const uint32_t code = code_of<PACKED>(w0, w1, t);
+        const uint32_t src = PACKED ? ((t & 1) ? e1 : e0) : (t < 4 ? e0 : e1);
+        const uint32_t sel = 0x7650u | (uint32_t)(PACKED ? (t >> 1) : (t & 3));
         const bool tail = (mb & (1u << t)) != 0;
-        const float q = __fsub_rn(__uint_as_float(0x4B400000u | (code & (uint32_t)qmask)), 12582912.0f);
+        const float q = __fsub_rn(__uint_as_float(__byte_perm(src, 0x4B400000u, sel)), 12582912.0f);
         const float v = __fadd_rn(__fmul_rn(q, tail ? s2 : s1), tail ? p : 0.0f);
-        // signed scheme: the code's sign bit moved to bit 31
+        // signed scheme: the code's sign bit, at bit 4 t + b - 1 (8 (t mod 4) + b - 1 for byte
+        // codes) of its word, moved to bit 31
+        const uint32_t word = PACKED ? w0 : (t < 4 ? w0 : w1);
+        const int up = sign_shift - (PACKED ? 4 * t : 8 * (t & 3));
         yv[t] = UNS ? __fadd_rn(v, lo)
-                    : __uint_as_float(__float_as_uint(v) | ((code << sign_shift) & 0x80000000u));
+                    : __uint_as_float(__float_as_uint(v) | ((word << up) & 0x80000000u));
     }
 }
 
