@@ -137,60 +137,14 @@ cudaError_t launch_bias_correction(const float* x, const int64_t* row_offsets, i
 }
 
 // ---------------------------------------------------------------- dequantize with the correction
-constexpr int kDbThreads = 256;
-constexpr int kDbPerThread = 16;
-
-// y' = xi * y + beta with y the value pwlq_dequantize delivers (one multiply, one add).
-template <bool PACKED>
-__global__ void __launch_bounds__(kDbThreads)
-dequantize_bc_kernel(const uint8_t* __restrict__ codes, const uint8_t* __restrict__ mask, Rows rows,
-                     int64_t total, int bits, const float* __restrict__ m_arr,
-                     const float* __restrict__ p_arr, const float* __restrict__ xi_arr,
-                     const float* __restrict__ beta_arr, float* __restrict__ y) {
-    const int64_t i0 = ((int64_t)blockIdx.x * kDbThreads + threadIdx.x) * kDbPerThread;
-    if (i0 >= total) return;
-    const float Lf = (float)((1 << (bits - 1)) - 1);
-    const int qmask = (1 << (bits - 1)) - 1;
-    const int cnt = (int)min((int64_t)kDbPerThread, total - i0);
-    int64_t row = -1, end = 0;
-    float m = 0.0f, xi = 1.0f, beta = 0.0f;
-    PieceParams P = {};
-#pragma unroll
-    for (int t = 0; t < kDbPerThread; ++t) {
-        if (t < cnt) {
-            const int64_t i = i0 + t;
-            if (row < 0 || i >= end) {
-                row = (row < 0) ? rows.row_of(i) : row + 1;
-                while (rows.begin(row + 1) <= i) ++row;          // skips empty rows
-                end = rows.begin(row + 1);
-                m = __ldg(m_arr + row);
-                P = make_params(m, __ldg(p_arr + row), Lf);
-                xi = __ldg(xi_arr + row);
-                beta = __ldg(beta_arr + row);
-            }
-            const int code = PACKED ? ((codes[i >> 1] >> ((i & 1) * 4)) & 0xF) : codes[i];
-            const int tail = (mask[i >> 3] >> (i & 7)) & 1;
-            float v = __fadd_rn(__fmul_rn((float)(code & qmask), tail ? P.s2 : P.s1),
-                                tail ? P.p : 0.0f);
-            int neg = (code >> (bits - 1)) & 1;
-            if (!(m > 0.0f)) { v = 0.0f; neg = 0; }
-            y[i] = __fadd_rn(__fmul_rn(xi, neg ? -v : v), beta);
-        }
-    }
-}
-
+// y' = xi * y + beta with y the value pwlq_dequantize delivers (one multiply, one add): the
+// dequantize kernel with the two per-row constants added to its row maps.
 cudaError_t launch_dequantize_bc(const uint8_t* codes, const uint8_t* mask,
                                  const int64_t* row_offsets, int64_t C, int64_t n, int64_t total,
                                  int bits, const float* m, const float* p, const float* xi,
                                  const float* beta, float* y, int layout, cudaStream_t stream) {
-    if (total == 0) return cudaSuccess;
-    Rows rows{row_offsets, C, n, n > 0 ? 1.0 / (double)n : 0.0, 0};
-    const bool packed = (layout == 1 && bits <= 4);
-    const int64_t per_cta = (int64_t)kDbThreads * kDbPerThread;
-    const unsigned grid = (unsigned)((total + per_cta - 1) / per_cta);
-    if (packed) dequantize_bc_kernel<true><<<grid, kDbThreads, 0, stream>>>(codes, mask, rows, total, bits, m, p, xi, beta, y);
-    else        dequantize_bc_kernel<false><<<grid, kDbThreads, 0, stream>>>(codes, mask, rows, total, bits, m, p, xi, beta, y);
-    return cudaGetLastError();
+    return launch_dequantize(codes, mask, row_offsets, C, n, total, bits, m, nullptr, p, y, layout,
+                             stream, 0, xi, beta);
 }
 
 // ------------------------------------------------------------------------- dense bit stream

@@ -39,7 +39,8 @@ cudaError_t launch_search(const float* x, const int64_t* row_offsets, int64_t C,
 
 // lo == nullptr: signed scheme with m = abs-max; lo != nullptr: one-sided ranges [lo, m] (m = upper
 // bounds), unsigned b-bit levels.  The same convention holds for launch_dequantize and
-// launch_search.
+// launch_search.  launch_dequantize with xi and beta (signed scheme only) delivers the
+// bias-corrected values xi[row] * y + beta[row].
 cudaError_t launch_quantize(const float* x, const int64_t* row_offsets, int64_t C, int64_t n,
                             int64_t total, int bits, const float* m, const float* lo,
                             const float* p, uint8_t* codes, uint8_t* mask, float* fake, int layout,
@@ -48,7 +49,8 @@ cudaError_t launch_quantize(const float* x, const int64_t* row_offsets, int64_t 
 cudaError_t launch_dequantize(const uint8_t* codes, const uint8_t* mask,
                               const int64_t* row_offsets, int64_t C, int64_t n, int64_t total,
                               int bits, const float* m, const float* lo, const float* p, float* y,
-                              int layout, cudaStream_t stream, int64_t shift = 0);
+                              int layout, cudaStream_t stream, int64_t shift = 0,
+                              const float* xi = nullptr, const float* beta = nullptr);
 
 // Two breakpoints (three regions): pair search over a grid of K <= kSearch2MaxK ascending ratios
 // for rows of at most kSearchTile values; quantize / dequantize with a two-bit region index.

@@ -38,6 +38,8 @@ struct RowArrays {
     const float* __restrict__ m;
     const float* __restrict__ lo;
     const float* __restrict__ p;
+    const float* __restrict__ xi;      // bias correction (dequantize): per-row scale and offset,
+    const float* __restrict__ beta;    // or nullptr
 };
 
 // The row a thread is currently in, with its constants in registers, looked up in global memory
@@ -47,6 +49,7 @@ struct RowState {
     float m = 0.0f;                                // range width (abs-max, or hi - lo)
     float lo = 0.0f;                               // lower bound of a one-sided range, else 0
     PieceParams P;
+    int64_t row = -1;
 
     // Range width and lower bound of `row` straight from global memory.
     static __device__ __forceinline__ void load_range(const RowArrays& A, int64_t row, float& m,
@@ -57,7 +60,7 @@ struct RowState {
     }
     __device__ __forceinline__ void seek(const Rows& rows, const RowArrays& A, float Lf, int64_t i) {
         if (i >= beg && i < end) return;
-        const int64_t row = rows.row_of(i);
+        row = rows.row_of(i);
         beg = rows.begin(row);
         end = rows.begin(row + 1);
         load_range(A, row, m, lo);
@@ -231,7 +234,7 @@ quantize_map_kernel(const float* __restrict__ x, Rows rows, int64_t total, int b
         // ---- producer
         MapProducer<true, UNS> prod;
         prod.rows = rows;
-        prod.in = RowInputs{A.m, A.lo, A.p};
+        prod.in = RowInputs{A.m, A.lo, A.p, A.xi, A.beta};
         prod.Lf = Lf;
         // LONG: dense rows of at least a span, the map follows from the row length
         constexpr bool long_rows = LONG;
@@ -578,12 +581,14 @@ dequantize_long_kernel(const uint8_t* __restrict__ codes, const uint8_t* __restr
 // Producer / consumer form of the inverse (see quantize_map_kernel and pwlq_rowmap.cuh).  The
 // producer writes row maps and constants only; the consumers request the codes and region bits
 // of the next span into registers before they wait for the current span's map.
-template <bool PACKED, bool UNS, bool LONG>
+// BC: the bias-corrected value xi * y + beta (one multiply, one add) instead of y.
+template <bool PACKED, bool UNS, bool LONG, bool BC>
 __global__ void __launch_bounds__(kMapThreads, 4)
 dequantize_map_kernel(const uint8_t* __restrict__ codes, const uint8_t* __restrict__ mask, Rows rows,
                       int64_t total, int bits, RowArrays A, float* __restrict__ y, int vec_codes,
                       int vec_out, int64_t spans_per_cta) {
-    typedef MapStage<false, UNS> Stage;
+    constexpr bool QB = UNS || BC;                    // the stages hold the second half of the constants
+    typedef MapStage<false, QB> Stage;
     extern __shared__ __align__(128) unsigned char smem_raw[];
     Stage* st = reinterpret_cast<Stage*>(smem_raw);
     __shared__ uint64_t full_bar[kMapStages], empty_bar[kMapStages];
@@ -606,9 +611,9 @@ dequantize_map_kernel(const uint8_t* __restrict__ codes, const uint8_t* __restri
 
     if (warp == kMapConsumers) {
         // ---- producer
-        MapProducer<true, UNS, true> prod;
+        MapProducer<true, UNS, true, BC> prod;
         prod.rows = rows;
-        prod.in = RowInputs{A.m, A.lo, A.p};
+        prod.in = RowInputs{A.m, A.lo, A.p, A.xi, A.beta};
         prod.Lf = Lf;
         if (LONG) prod.request_long(rows.dense_row(first * kMapSpan));
         else prod.request(warp_row_of(rows, first * kMapSpan), true);
@@ -622,10 +627,10 @@ dequantize_map_kernel(const uint8_t* __restrict__ codes, const uint8_t* __restri
             }
             const int64_t span_beg = span * kMapSpan, span_end = min(span_beg + kMapSpan, total);
             if (LONG)
-                prod.build_long(st[s].map, st[s].qa, UNS ? st[s].qb : nullptr, s, span_beg, span_end,
+                prod.build_long(st[s].map, st[s].qa, QB ? st[s].qb : nullptr, s, span_beg, span_end,
                                 span + 1 < last);
             else
-                prod.build(st[s].map, st[s].qa, UNS ? st[s].qb : nullptr, span_beg, span_end,
+                prod.build(st[s].map, st[s].qa, QB ? st[s].qb : nullptr, span_beg, span_end,
                            span + 1 < last);
             __syncwarp();
             if (lane == 0) mbar_arrive(&full_bar[s]);
@@ -666,6 +671,11 @@ dequantize_map_kernel(const uint8_t* __restrict__ codes, const uint8_t* __restri
                 if (__all_sync(full, simple)) {
                     dequantize8<PACKED, false, UNS>(cur.w0[c], cur.w1[c], cur.mb[c], 8, PA, loA, PA, loA,
                                                     qmask, sign_shift, yv);
+                    if (BC) {
+                        const float4 ba = S.qb[l];
+#pragma unroll
+                        for (int t = 0; t < 8; ++t) yv[t] = __fadd_rn(__fmul_rn(ba.y, yv[t]), ba.z);
+                    }
                 } else {
                     const bool one = inner != 0 && (inner & (inner - 1)) == 0 && ca.x > 0.0f && cnt == 8;
                     float4 da = ca;
@@ -681,6 +691,13 @@ dequantize_map_kernel(const uint8_t* __restrict__ codes, const uint8_t* __restri
                         PB.p = da.y; PB.s1 = da.z; PB.s2 = da.w; PB.inv1 = PB.inv2 = 0.0f;
                         dequantize8<PACKED, true, UNS>(cur.w0[c], cur.w1[c], cur.mb[c], split, PA, loA,
                                                        PB, loB, qmask, sign_shift, yv);
+                        if (BC) {
+                            const float4 ba = S.qb[l], bb = S.qb[one ? l + 1 : l];
+#pragma unroll
+                            for (int t = 0; t < 8; ++t)
+                                yv[t] = __fadd_rn(__fmul_rn(t < split ? ba.y : bb.y, yv[t]),
+                                                  t < split ? ba.z : bb.z);
+                        }
                     } else {
 #pragma unroll
                         for (int t = 0; t < 8; ++t) {
@@ -698,6 +715,10 @@ dequantize_map_kernel(const uint8_t* __restrict__ codes, const uint8_t* __restri
                                     float v = __fmul_rn(q, tail ? ea.w : ea.z);
                                     v = __fadd_rn(v, tail ? ea.y : 0.0f);
                                     yv[t] = UNS ? __fadd_rn(v, loE) : (neg ? -v : v);
+                                }
+                                if (BC) {
+                                    const float4 eb = S.qb[lt];
+                                    yv[t] = __fadd_rn(__fmul_rn(eb.y, yv[t]), eb.z);
                                 }
                             }
                         }
@@ -720,6 +741,7 @@ dequantize_map_kernel(const uint8_t* __restrict__ codes, const uint8_t* __restri
                             v = __fadd_rn(v, tail ? rs.P.p : 0.0f);
                             yv[t] = UNS ? __fadd_rn(v, rs.lo) : (neg ? -v : v);
                         }
+                        if (BC) yv[t] = __fadd_rn(__fmul_rn(__ldg(A.xi + rs.row), yv[t]), __ldg(A.beta + rs.row));
                     }
                 }
             }
@@ -791,9 +813,11 @@ cudaError_t launch_quantize(const float* x, const int64_t* row_offsets, int64_t 
                             int64_t total, int bits, const float* m, const float* lo,
                             const float* p, uint8_t* codes, uint8_t* mask, float* fake, int layout,
                             cudaStream_t stream, int64_t shift) {
+    const float* xi = nullptr;
+    const float* beta = nullptr;
     if (total == 0) return cudaSuccess;
     Rows rows{row_offsets, C, n, n > 0 ? 1.0 / (double)n : 0.0, row_offsets ? shift : 0};
-    const RowArrays A{m, lo, p};
+    const RowArrays A{m, lo, p, xi, beta};
     const bool packed = (layout == 1 && bits <= 4);
     const int64_t nspans = (total + kQSpan - 1) / kQSpan;
     const int vec_in = aligned(x, 16), vec_fake = fake ? aligned(fake, 16) : 0;
@@ -828,43 +852,53 @@ cudaError_t launch_quantize(const float* x, const int64_t* row_offsets, int64_t 
 cudaError_t launch_dequantize(const uint8_t* codes, const uint8_t* mask,
                               const int64_t* row_offsets, int64_t C, int64_t n, int64_t total,
                               int bits, const float* m, const float* lo, const float* p, float* y,
-                              int layout, cudaStream_t stream, int64_t shift) {
+                              int layout, cudaStream_t stream, int64_t shift, const float* xi,
+                              const float* beta) {
     if (total == 0) return cudaSuccess;
     Rows rows{row_offsets, C, n, n > 0 ? 1.0 / (double)n : 0.0, row_offsets ? shift : 0};
-    const RowArrays A{m, lo, p};
+    const RowArrays A{m, lo, p, xi, beta};
     const bool packed = (layout == 1 && bits <= 4);
     const int64_t nspans = (total + kQSpan - 1) / kQSpan;
-#define PWLQ_LAUNCH_DEQUANTIZE(PK, UN)                                                            \
+#define PWLQ_LAUNCH_DEQUANTIZE(PK, UN, BCF)                                                       \
     do {                                                                                          \
         const int vc = aligned(codes, PK ? 4 : 8), vo = aligned(y, 16);                           \
-        if (very_long) {                                                                          \
-            const SpanGrid g = span_grid((const void*)dequantize_long_kernel<PK, UN>, kQThreads,  \
-                                         0, nspans, false);                                       \
-            dequantize_long_kernel<PK, UN><<<g.grid, kQThreads, 0, stream>>>(                     \
-                codes, mask, rows, total, bits, A, y, vc, vo);                                    \
+        const size_t msmem = sizeof(MapStage<false, UN || BCF>) * kMapStages;                     \
+        if (long_rows) {                                                                          \
+            const SpanGrid g = span_grid((const void*)dequantize_map_kernel<PK, UN, true, BCF>,   \
+                                         kMapThreads, msmem, nspans, true);                       \
+            dequantize_map_kernel<PK, UN, true, BCF><<<g.grid, kMapThreads, msmem, stream>>>(     \
+                codes, mask, rows, total, bits, A, y, vc, vo, g.per_cta);                         \
         } else {                                                                                  \
-            const size_t msmem = sizeof(MapStage<false, UN>) * kMapStages;                        \
-            if (long_rows) {                                                                      \
-                const SpanGrid g = span_grid((const void*)dequantize_map_kernel<PK, UN, true>,    \
-                                             kMapThreads, msmem, nspans, true);                   \
-                dequantize_map_kernel<PK, UN, true><<<g.grid, kMapThreads, msmem, stream>>>(      \
-                    codes, mask, rows, total, bits, A, y, vc, vo, g.per_cta);                     \
-            } else {                                                                              \
-                const SpanGrid g = span_grid((const void*)dequantize_map_kernel<PK, UN, false>,   \
-                                             kMapThreads, msmem, nspans, true);                   \
-                dequantize_map_kernel<PK, UN, false><<<g.grid, kMapThreads, msmem, stream>>>(     \
-                    codes, mask, rows, total, bits, A, y, vc, vo, g.per_cta);                     \
-            }                                                                                     \
+            const SpanGrid g = span_grid((const void*)dequantize_map_kernel<PK, UN, false, BCF>,  \
+                                         kMapThreads, msmem, nspans, true);                       \
+            dequantize_map_kernel<PK, UN, false, BCF><<<g.grid, kMapThreads, msmem, stream>>>(    \
+                codes, mask, rows, total, bits, A, y, vc, vo, g.per_cta);                         \
         }                                                                                         \
     } while (0)
-#define PWLQ_LAUNCH_DEQUANTIZE_UN(PK) \
-    do { if (lo) PWLQ_LAUNCH_DEQUANTIZE(PK, true); else PWLQ_LAUNCH_DEQUANTIZE(PK, false); } while (0)
+#define PWLQ_LAUNCH_DEQUANTIZE_LONG(PK, UN)                                                       \
+    do {                                                                                          \
+        const SpanGrid g = span_grid((const void*)dequantize_long_kernel<PK, UN>, kQThreads, 0,   \
+                                     nspans, false);                                              \
+        dequantize_long_kernel<PK, UN><<<g.grid, kQThreads, 0, stream>>>(                         \
+            codes, mask, rows, total, bits, A, y, aligned(codes, PK ? 4 : 8), aligned(y, 16));    \
+    } while (0)
     // Dense rows of many spans stream through the register-only kernel (no row lookups worth
-    // speaking of); everything else goes through the producer / consumer kernel.
-    const bool very_long = row_offsets == nullptr && n >= 16 * (int64_t)kMapSpan;
+    // speaking of); everything else, and every bias-corrected call, goes through the producer /
+    // consumer kernel.
+    const bool bc = xi != nullptr;
+    const bool very_long = !bc && row_offsets == nullptr && n >= 16 * (int64_t)kMapSpan;
     const bool long_rows = row_offsets == nullptr && n >= kMapSpan;   // the map follows from n
-    if (packed) PWLQ_LAUNCH_DEQUANTIZE_UN(true); else PWLQ_LAUNCH_DEQUANTIZE_UN(false);
-#undef PWLQ_LAUNCH_DEQUANTIZE_UN
+    if (very_long) {
+        if (packed) { if (lo) PWLQ_LAUNCH_DEQUANTIZE_LONG(true, true); else PWLQ_LAUNCH_DEQUANTIZE_LONG(true, false); }
+        else        { if (lo) PWLQ_LAUNCH_DEQUANTIZE_LONG(false, true); else PWLQ_LAUNCH_DEQUANTIZE_LONG(false, false); }
+    } else if (bc) {
+        if (packed) PWLQ_LAUNCH_DEQUANTIZE(true, false, true); else PWLQ_LAUNCH_DEQUANTIZE(false, false, true);
+    } else if (lo) {
+        if (packed) PWLQ_LAUNCH_DEQUANTIZE(true, true, false); else PWLQ_LAUNCH_DEQUANTIZE(false, true, false);
+    } else {
+        if (packed) PWLQ_LAUNCH_DEQUANTIZE(true, false, false); else PWLQ_LAUNCH_DEQUANTIZE(false, false, false);
+    }
+#undef PWLQ_LAUNCH_DEQUANTIZE_LONG
 #undef PWLQ_LAUNCH_DEQUANTIZE
     return cudaGetLastError();
 }

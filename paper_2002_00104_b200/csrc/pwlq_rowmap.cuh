@@ -54,18 +54,21 @@ struct RowInputs {
     const float* __restrict__ m;
     const float* __restrict__ lo;
     const float* __restrict__ p;
+    const float* __restrict__ xi;      // bias correction (dequantize only): scale and offset
+    const float* __restrict__ beta;    // per row, or nullptr
 };
 
 // Constants of one row as the consumers read them; m is the range width (abs-max, or upper -
 // lower bound).  Quantize (DEQ = false): qa = (m, p, L/p, L/(m-p)), qb = (p/L, (m-p)/L, lo, 0).
-// Dequantize (DEQ = true): qa = (m, p, p/L, (m-p)/L), qb = (lo, 0, 0, 0).
+// Dequantize (DEQ = true): qa = (m, p, p/L, (m-p)/L), qb = (lo, xi, beta, 0) with the scale and
+// offset of the bias correction (1 and 0 without it).
 template <bool DEQ>
 __device__ __forceinline__ void store_row_consts(float4* qa, float4* qb, int slot, float m, float p,
-                                                 float lo, float Lf) {
+                                                 float lo, float xi, float beta, float Lf) {
     const PieceParams P = make_params(m, p, Lf);
     if (DEQ) {
         qa[slot] = make_float4(m, P.p, P.s1, P.s2);
-        if (qb) qb[slot] = make_float4(lo, 0.0f, 0.0f, 0.0f);
+        if (qb) qb[slot] = make_float4(lo, xi, beta, 0.0f);
     } else {
         qa[slot] = make_float4(m, P.p, P.inv1, P.inv2);
         if (qb) qb[slot] = make_float4(P.s1, P.s2, lo, 0.0f);
@@ -75,7 +78,7 @@ __device__ __forceinline__ void store_row_consts(float4* qa, float4* qb, int slo
 // The producer warp's view of the rows.  Rows are looked at in chunks of 32 consecutive rows
 // (chunk c = rows 32 c .. 32 c + 31, lane = row % 32); the two chunks from the current first row
 // on are held in registers.  Every member function is called by all 32 lanes.
-template <bool PARAMS, bool UNS, bool DEQ = false>
+template <bool PARAMS, bool UNS, bool DEQ = false, bool BC = false>
 struct MapProducer {
     Rows rows;
     RowInputs in;
@@ -84,21 +87,27 @@ struct MapProducer {
     int64_t ch0, ch1;           // chunk held in (o0, m0, p0, lo0): even chunks; (o1, ...): odd chunks
     int64_t o0, o1;             // offset of row 32 ch + lane (INT64_MAX past the last offset)
     float m0, p0, lo0, m1, p1, lo1;
+    float x0, b0, x1, b1;       // BC: scale and offset of the bias correction
 
-    __device__ __forceinline__ void load_inputs(int64_t r, float& mv, float& pv, float& lov) const {
+    __device__ __forceinline__ void load_inputs(int64_t r, float& mv, float& pv, float& lov,
+                                                float& xv, float& bv) const {
         mv = __ldg(in.m + r);
         pv = __ldg(in.p + r);
         lov = 0.0f;
         if (UNS) lov = __ldg(in.lo + r);            // m stays the upper bound until it is used
+        xv = 1.0f;
+        bv = 0.0f;
+        if (BC) { xv = __ldg(in.xi + r); bv = __ldg(in.beta + r); }
     }
     __device__ __forceinline__ void load_chunk(int64_t c, int64_t& o, float& mv, float& pv,
-                                               float& lov) const {
+                                               float& lov, float& xv, float& bv) const {
         const int64_t r = 32 * c + (threadIdx.x & 31);
         // as stored (ragged: before the slice's shift is taken off), so that nothing here waits
         // for the load
         o = (r <= rows.C) ? (rows.offsets ? __ldg(rows.offsets + r) : r * rows.n) : INT64_MAX;
-        mv = pv = lov = 0.0f;
-        if (PARAMS && r < rows.C) load_inputs(r, mv, pv, lov);
+        mv = pv = lov = bv = 0.0f;
+        xv = 1.0f;
+        if (PARAMS && r < rows.C) load_inputs(r, mv, pv, lov, xv, bv);
     }
     // Makes the registers hold the two chunks from row `first_row` on; chunks already held are
     // kept, nothing is waited for.
@@ -106,8 +115,8 @@ struct MapProducer {
         rf = first_row;
         const int64_t c = rf >> 5;
         const int64_t want0 = (c & 1) ? c + 1 : c, want1 = (c & 1) ? c : c + 1;
-        if (fresh || ch0 != want0) { ch0 = want0; load_chunk(want0, o0, m0, p0, lo0); }
-        if (fresh || ch1 != want1) { ch1 = want1; load_chunk(want1, o1, m1, p1, lo1); }
+        if (fresh || ch0 != want0) { ch0 = want0; load_chunk(want0, o0, m0, p0, lo0, x0, b0); }
+        if (fresh || ch1 != want1) { ch1 = want1; load_chunk(want1, o1, m1, p1, lo1, x1, b1); }
     }
     // Writes the map of the span [span_beg, span_end), whose first value lies in row rf, and the
     // constants of its rows; then moves on to the first row of the next span (more == true).
@@ -130,14 +139,16 @@ struct MapProducer {
             const int s = 32 * k + lane - l0;
             const int64_t r = 32 * c + lane;
             int64_t off;
-            float mv, pv, lov;
+            float mv, pv, lov, xv, bv;
             if (k < 2) {                           // held in registers
                 const bool odd = (c & 1) != 0;
                 off = odd ? o1 : o0;
                 mv = odd ? m1 : m0; pv = odd ? p1 : p0; lov = odd ? lo1 : lo0;
+                xv = odd ? x1 : x0; bv = odd ? b1 : b0;
             } else {                               // short rows: fetched now
                 off = (r <= rows.C) ? (rows.offsets ? __ldg(rows.offsets + r) : r * rows.n) : INT64_MAX;
-                mv = pv = lov = 0.0f;
+                mv = pv = lov = bv = 0.0f;
+                xv = 1.0f;
             }
             if (off != INT64_MAX) off -= rows.shift;
             const bool inside = s >= 0 && r < rows.C && (s == 0 || off < span_end);
@@ -148,9 +159,9 @@ struct MapProducer {
                     atomicOr(&M.bits[pos >> 5], bit);
                 }
                 if (PARAMS) {
-                    if (k >= 2) load_inputs(r, mv, pv, lov);
+                    if (k >= 2) load_inputs(r, mv, pv, lov, xv, bv);
                     if (UNS) mv = __fsub_rn(mv, lov);              // range width
-                    store_row_consts<DEQ>(qa, qb, s, mv, pv, lov, Lf);
+                    store_row_consts<DEQ>(qa, qb, s, mv, pv, lov, xv, bv, Lf);
                 }
             }
             const unsigned in_mask = __ballot_sync(full, inside);
@@ -219,10 +230,11 @@ struct MapProducer {
     __device__ __forceinline__ void request_long(int64_t first_row) {
         rf = first_row;
         long_end = (rf + 1) * rows.n;
-        m0 = p0 = lo0 = m1 = p1 = lo1 = 0.0f;
+        m0 = p0 = lo0 = m1 = p1 = lo1 = b0 = b1 = 0.0f;
+        x0 = x1 = 1.0f;
         if (PARAMS) {
-            load_inputs(rf, m0, p0, lo0);
-            if (rf + 1 < rows.C) load_inputs(rf + 1, m1, p1, lo1);
+            load_inputs(rf, m0, p0, lo0, x0, b0);
+            if (rf + 1 < rows.C) load_inputs(rf + 1, m1, p1, lo1, x1, b1);
         }
 #pragma unroll
         for (int i = 0; i < kMaxStages; ++i) { stage_first[i] = -1; stage_plain[i] = false; }
@@ -237,9 +249,9 @@ struct MapProducer {
         for (int i = 0; i < kMaxStages; ++i)
             if (stage == i) { have_first = stage_first[i] == rf; plain = stage_plain[i]; }
         if (PARAMS && !have_first && lane == 0)
-            store_row_consts<DEQ>(qa, qb, 0, UNS ? __fsub_rn(m0, lo0) : m0, p0, lo0, Lf);
+            store_row_consts<DEQ>(qa, qb, 0, UNS ? __fsub_rn(m0, lo0) : m0, p0, lo0, x0, b0, Lf);
         if (PARAMS && starts && lane == 1)
-            store_row_consts<DEQ>(qa, qb, 1, UNS ? __fsub_rn(m1, lo1) : m1, p1, lo1, Lf);
+            store_row_consts<DEQ>(qa, qb, 1, UNS ? __fsub_rn(m1, lo1) : m1, p1, lo1, x1, b1, Lf);
         if (starts || !plain || !have_first) {
             const int pos = starts ? (int)(long_end - span_beg) : -1;      // > 0 when it exists
             const int wpos = pos >> 5;                                     // -1: no start
@@ -260,8 +272,8 @@ struct MapProducer {
         if (more && long_end <= span_end) {               // the next span begins in row rf + 1
             rf += 1;
             long_end += rows.n;
-            m0 = m1; p0 = p1; lo0 = lo1;
-            if (PARAMS && rf + 1 < rows.C) load_inputs(rf + 1, m1, p1, lo1);
+            m0 = m1; p0 = p1; lo0 = lo1; x0 = x1; b0 = b1;
+            if (PARAMS && rf + 1 < rows.C) load_inputs(rf + 1, m1, p1, lo1, x1, b1);
         }
     }
 };
