@@ -379,7 +379,7 @@ def run_ours(args, rank, world, local_rank):
     # (plus the two combine launches when a row exceeds one tile), quantize, dequantize
     lens = np.diff(w.row_offsets)
     classes = sum(bool(np.any((lens >= lo) & (lens <= hi)))
-                  for lo, hi in ((0, 256), (257, 1152), (1153, 1 << 62))) if w.K <= 1024 else 1
+                  for lo, hi in ((0, 64), (65, 256), (257, 1152), (1153, 1 << 62))) if w.K <= 1024 else 1
     per_step = 1 + classes + (2 if max_n > 8192 else 0) + 2
     if rank == 0:
         peaks, peak_kind = measured_peaks()

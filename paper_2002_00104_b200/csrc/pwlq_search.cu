@@ -597,6 +597,101 @@ search_sorted_kernel(SearchArgs a) {
     finish_tile(a, row, tile, m, S.part, E, red_val, red_idx);
 }
 
+// --------------------------------------------------------------------------- tiny rows
+// Rows of at most kTinyMax values (depthwise 3x3 channels have 9): one warp per row, eight rows
+// per CTA.  The row's magnitudes sit in two registers per lane and are broadcast with shuffles;
+// a lane owns kTinyBatch candidates at a time (candidate k0 + 32 j + lane, so that a warp's
+// stores of the sums are contiguous) and evaluates the region select for every value -- with a
+// handful of values there is nothing to sort, and no cross-lane reduction exists.  Sums: binary32
+// over the row's at most kTinyMax terms, compared in binary64; first minimum.
+constexpr int kTinyMax = 64;
+constexpr int kTinyBatch = 4;
+constexpr int kTinyWarps = 8;
+
+template <bool EXACT_V>
+__device__ __forceinline__ void tiny_row(const SearchArgs& a, int64_t row, int cnt, float m,
+                                         float a0, float a1) {
+    const unsigned full = 0xffffffffu;
+    const int lane = threadIdx.x & 31;
+    const int K = a.K;
+    const float Lf = (float)a.levels;
+    double best = 0.0;
+    int bk = 0x7fffffff;
+    for (int k0 = 0; k0 < K; k0 += 32 * kTinyBatch) {
+        PieceParams P[kTinyBatch];
+        float acc[kTinyBatch];
+#pragma unroll
+        for (int j = 0; j < kTinyBatch; ++j) {
+            const int k = min(k0 + 32 * j + lane, K - 1);
+            P[j] = make_params(m, __fmul_rn(m, __ldg(a.ratios + k)), Lf);
+            acc[j] = 0.0f;
+        }
+        for (int i = 0; i < cnt; ++i) {
+            const float v = __shfl_sync(full, i < 32 ? a0 : a1, i & 31);
+#pragma unroll
+            for (int j = 0; j < kTinyBatch; ++j) acc[j] = sq_err_select<EXACT_V>(v, P[j], acc[j]);
+        }
+#pragma unroll
+        for (int j = 0; j < kTinyBatch; ++j) {
+            const int k = k0 + 32 * j + lane;
+            if (k < K) {
+                const double tot = (double)acc[j];
+                if (a.tiles > 1) {
+                    a.partials[((size_t)row * a.tiles) * K + k] = tot;    // tile 0 of the row
+                } else {
+                    if (a.sse_all) a.sse_all[row * K + k] = (float)tot;
+                    if (bk == 0x7fffffff || tot < best) { best = tot; bk = k; }   // k ascends
+                }
+            }
+        }
+    }
+    if (a.tiles > 1) return;                          // the combine kernels finish the row
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        const double ov = __shfl_xor_sync(full, best, o);
+        const int ok = __shfl_xor_sync(full, bk, o);
+        if (ok != 0x7fffffff && (bk == 0x7fffffff || ov < best || (ov == best && ok < bk))) {
+            best = ov; bk = ok;
+        }
+    }
+    if (lane == 0) write_row_result(a, row, m, best, bk);
+}
+
+__global__ void __launch_bounds__(kTinyWarps * 32)
+search_tiny_kernel(SearchArgs a) {
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int64_t row = (int64_t)blockIdx.x * kTinyWarps + warp;
+    if (row >= a.rows.C) return;
+    const int64_t beg = a.rows.begin(row), end = a.rows.begin(row + 1);
+    if (end - beg > a.n_max || end - beg < a.n_min) return;          // another launch's row
+    const int cnt = (int)(end - beg);
+    float lo;
+    const float m = row_range(a, row, lo);
+    const bool finite = (__float_as_uint(m) & 0x7fffffffu) < 0x7f800000u &&
+                        (__float_as_uint(lo) & 0x7fffffffu) < 0x7f800000u;
+    if (!finite || !(m > 0.0f) || cnt <= 0) {
+        // m == 0 (or not finite): nothing to search; with several tiles per row the combine
+        // kernels write the row
+        if (!finite && lane == 0) atomicOr(a.status, kStatusNonFinite);
+        if (a.tiles == 1) {
+            if (lane == 0) {
+                a.idx_out[row] = 0;
+                a.p_out[row] = 0.0f;
+                if (a.err_out) a.err_out[row] = 0.0f;
+            }
+            if (a.sse_all)
+                for (int k = lane; k < a.K; k += 32) a.sse_all[row * a.K + k] = 0.0f;
+        }
+        return;
+    }
+    const float a0 = lane < cnt ? mag_of(a, __ldg(a.x + beg + lane), m, lo) : 0.0f;
+    const float a1 = lane + 32 < cnt ? mag_of(a, __ldg(a.x + beg + lane + 32), m, lo) : 0.0f;
+    const int64_t L = a.levels;
+    if (2 * (int64_t)cnt >= L * L) tiny_row<false>(a, row, cnt, m, a0, a1);
+    else tiny_row<true>(a, row, cnt, m, a0, a1);
+}
+
 // ------------------------------------------------------------------------ generic kernel
 // More than kSortMaxK candidates: region select for every (value, candidate).
 __global__ void __launch_bounds__(kSThreads)
@@ -737,7 +832,8 @@ cudaError_t launch_search(const float* x, const int64_t* row_offsets, int64_t C,
         // more small CTAs per SM.  One launch per class; a CTA whose row belongs to another
         // class exits at once.  A dense tensor has one class.
         struct RowClass { int64_t n_min, n_max; int threads; };
-        const RowClass classes[3] = {{1153, INT64_MAX, 256}, {257, 1152, 128}, {0, 256, 64}};
+        const RowClass classes[4] = {{1153, INT64_MAX, 256}, {257, 1152, 128},
+                                     {kTinyMax + 1, 256, 64}, {0, kTinyMax, 0}};   // 0: tiny rows
         size_t off[7];
         const size_t smem_max = sorted_smem_layout(a.cap, K, kSWarps, off);
         if (smem_max > 48 * 1024) {  // above the default limit: opt in (idempotent, per device)
@@ -756,13 +852,15 @@ cudaError_t launch_search(const float* x, const int64_t* row_offsets, int64_t C,
             a.grid_tiles = longest ? plan.tiles : 1;
             a.cap = longest ? full_cap
                             : (int)((std::min<int64_t>(plan.max_n, rc.n_max) + 3) / 4 * 4);
-            const size_t smem = sorted_smem_layout(a.cap, K, rc.threads / 32, off);
+            const bool tiny = rc.threads == 0;            // one warp per row, no shared memory
+            const size_t smem = tiny ? 0 : sorted_smem_layout(a.cap, K, rc.threads / 32, off);
             // Launches after the first may overlap the tail of the one before (they are
             // independent of each other; all of them were ordered after the abs-max above by the
             // first, ordinary launch).
             cudaLaunchConfig_t cfg = {};
-            cfg.gridDim = dim3((unsigned)(C * a.grid_tiles));
-            cfg.blockDim = dim3((unsigned)rc.threads);
+            cfg.gridDim = dim3(tiny ? (unsigned)((C + kTinyWarps - 1) / kTinyWarps)
+                                    : (unsigned)(C * a.grid_tiles));
+            cfg.blockDim = dim3(tiny ? (unsigned)(kTinyWarps * 32) : (unsigned)rc.threads);
             cfg.dynamicSmemBytes = smem;
             cfg.stream = stream;
             cudaLaunchAttribute attr[1];
@@ -770,7 +868,8 @@ cudaError_t launch_search(const float* x, const int64_t* row_offsets, int64_t C,
             attr[0].val.programmaticStreamSerializationAllowed = 1;
             cfg.attrs = attr;
             cfg.numAttrs = launched > 0 ? 1 : 0;
-            e = cudaLaunchKernelEx(&cfg, search_sorted_kernel, a);
+            e = tiny ? cudaLaunchKernelEx(&cfg, search_tiny_kernel, a)
+                     : cudaLaunchKernelEx(&cfg, search_sorted_kernel, a);
             if (e != cudaSuccess) return e;
             ++launched;
         }

@@ -169,6 +169,35 @@ def test_search_dense_tiles_and_tails(pwlq, oracle, C, n, bits, K):
     check_search(gpu, ora, ratios, oracle.absmax(x), n)
 
 
+@pytest.mark.parametrize("n", [1, 2, 9, 31, 32, 33, 63, 64, 65])
+@pytest.mark.parametrize("bits,K", [(3, 256), (4, 100), (8, 300), (2, 1), (4, 1024)])
+def test_search_tiny_rows(pwlq, oracle, n, bits, K):
+    """Rows around the limit of the one-warp-per-row kernel (64 values), with candidate counts that
+    are not multiples of its batch, bit-widths on both sides of the fused / unfused switch, a zero
+    row and an exact-tie row."""
+    rng = np.random.default_rng(n * 100 + K)
+    x = (rng.laplace(0, 0.02, (37, n)) * 10.0 ** rng.uniform(-2, 1, (37, 1))).astype(np.float32)
+    x[5] = 0.0
+    x[6] = np.float32(0.75) * np.where(np.arange(n) % 2, -1, 1)      # all |x| = m
+    ratios = W.ratio_grid(K)
+    ora = oracle.search(x, bits, ratios)
+    gpu, status = run_search(pwlq, x, bits, ratios)
+    assert status == 0
+    check_search(gpu, ora, ratios, oracle.absmax(x), n)
+    assert gpu["idx"][5] == 0 and gpu["p"][5] == 0.0 and gpu["err"][5] == 0.0
+
+
+def test_search_tiny_rows_unsorted_grid_and_ties(pwlq, oracle):
+    rng = np.random.default_rng(8)
+    x = rng.standard_normal((50, 9)).astype(np.float32)
+    ratios = np.array([0.5, 0.2, 0.2, 0.9, 0.35, 1.0, 0.05, 0.2], dtype=np.float32)
+    ora = oracle.search(x, 4, ratios)
+    gpu, _ = run_search(pwlq, x, 4, ratios)
+    check_search(gpu, ora, ratios, oracle.absmax(x), 9)
+    assert np.all(gpu["idx"] != 2) and np.all(gpu["idx"] != 7)        # duplicates: lowest index wins
+    assert np.array_equal(gpu["sse"][:, 1], gpu["sse"][:, 2])
+
+
 def test_search_with_given_range_and_unsorted_grid(pwlq, oracle):
     rng = np.random.default_rng(77)
     x = rng.standard_normal((6, 700)).astype(np.float32)
