@@ -43,9 +43,9 @@ ALU_PEAK_TLANEOPS = SM_COUNT * FP32_LANES_PER_SM * SM_MAX_GHZ / 1e3     # 37.2 T
 LANE_OPS_PER_ELEM_CAND = 6      # sub, mul, 2 adds (round to nearest even), fma, fma
 L2_FLUSH_BYTES = 256 << 20
 # dram__bytes_read.sum + dram__bytes_write.sum of the search kernels of ONE step, from the ncu
-# capture summarised in profiles/search_sorted_kernel_resnet50.md (103.08 MB read, 0.75 MB
+# capture summarised in profiles/search_sorted_kernel_resnet50.md (103.31 MB read, 0.33 MB
 # written; the values themselves are 102.0 MB).  Keyed by (workload, bits, K); None elsewhere.
-SEARCH_DRAM_BYTES = {("resnet50", 4, 256): 103.83e6}
+SEARCH_DRAM_BYTES = {("resnet50", 4, 256): 103.64e6}
 
 WORKLOADS = {
     "resnet50": W.resnet50,
@@ -379,7 +379,7 @@ def run_ours(args, rank, world, local_rank):
     # (plus the two combine launches when a row exceeds one tile), quantize, dequantize
     lens = np.diff(w.row_offsets)
     classes = sum(bool(np.any((lens >= lo) & (lens <= hi)))
-                  for lo, hi in ((0, 64), (65, 256), (257, 1152), (1153, 1 << 62))) if w.K <= 1024 else 1
+                  for lo, hi in ((0, 64), (65, 512), (513, 2304), (2305, 1 << 62))) if w.K <= 1024 else 1
     per_step = 1 + classes + (2 if max_n > 8192 else 0) + 2
     if rank == 0:
         peaks, peak_kind = measured_peaks()

@@ -832,8 +832,10 @@ cudaError_t launch_search(const float* x, const int64_t* row_offsets, int64_t C,
         // more small CTAs per SM.  One launch per class; a CTA whose row belongs to another
         // class exits at once.  A dense tensor has one class.
         struct RowClass { int64_t n_min, n_max; int threads; };
-        const RowClass classes[4] = {{1153, INT64_MAX, 256}, {257, 1152, 128},
-                                     {kTinyMax + 1, 256, 64}, {0, kTinyMax, 0}};   // 0: tiny rows
+        // (boundaries measured on B200: 128-thread CTAs beat 256-thread ones up to rows of about
+        // 2300 values, 64-thread CTAs beat 128-thread ones up to about 500)
+        const RowClass classes[4] = {{2305, INT64_MAX, 256}, {513, 2304, 128},
+                                     {kTinyMax + 1, 512, 64}, {0, kTinyMax, 0}};   // 0: tiny rows
         size_t off[7];
         const size_t smem_max = sorted_smem_layout(a.cap, K, kSWarps, off);
         if (smem_max > 48 * 1024) {  // above the default limit: opt in (idempotent, per device)
