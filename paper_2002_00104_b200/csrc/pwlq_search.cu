@@ -340,11 +340,14 @@ __host__ __device__ inline int group_width(int cnt) {
     return cnt >= kLongTileMin ? kCwLongTile : (cnt >= kMidTileMin ? kCwMidTile : kCwShortTile);
 }
 
-// Element slices per candidate group: enough (group, slice) work items to keep eight warps
-// busy.  Sized for the narrowest group so that one shared-memory layout serves every width.
+// Element slices per candidate group: enough (group, slice) work items to keep the warps busy.
+// Sized for the narrowest group so that one shared-memory layout serves every width.
+// (two work items per warp: every item recomputes its candidates' constants, so more, smaller
+// items cost more than the better balance gains -- measured at K = 64)
+constexpr int kItemsPerWarp = 2;
 __host__ __device__ inline int slices_sorted(int K, int cw, int warps) {
     const int G = (K + cw - 1) / cw;
-    const int E = (4 * warps + G - 1) / G;
+    const int E = (kItemsPerWarp * warps + G - 1) / G;
     return E < 1 ? 1 : (E > 8 ? 8 : E);
 }
 __host__ __device__ inline int max_slices_sorted(int K, int warps) {
