@@ -375,11 +375,14 @@ def run_ours(args, rank, world, local_rank):
     else:
         stage_tot = stage_ms.sum(axis=0).tolist()
 
-    # kernels of this library per step: abs-max, one search launch per row-length class present
-    # (plus the two combine launches when a row exceeds one tile), quantize, dequantize
-    lens = np.diff(w.row_offsets)
-    classes = sum(bool(np.any((lens >= lo) & (lens <= hi)))
-                  for lo, hi in ((0, 64), (65, 512), (513, 2304), (2305, 1 << 62))) if w.K <= 1024 else 1
+    # kernels of this library per step: abs-max, the search launches (a dense matrix: the one for
+    # its row length; ragged rows: one per row-length class that begins at or below the longest
+    # row -- the library does not look at the lengths), the two combine launches when a row exceeds
+    # one tile, quantize, dequantize
+    if w.K > 1024 or dense_n is not None:
+        classes = 1
+    else:
+        classes = sum(max_n >= lo for lo in (0, 65, 513, 2305))
     per_step = 1 + classes + (2 if max_n > 8192 else 0) + 2
     if rank == 0:
         peaks, peak_kind = measured_peaks()
