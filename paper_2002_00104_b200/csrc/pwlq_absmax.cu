@@ -15,7 +15,7 @@ namespace pwlq {
 
 constexpr int kAbsConsumers = 8;                         // folding warps per CTA
 constexpr int kAbsThreads = (kAbsConsumers + 1) * 32;    // + the producer warp
-constexpr int kAbsStages = 3;                            // spans in flight per CTA
+constexpr int kAbsStages = 2;                            // spans in flight per CTA
 static_assert(kAbsStages <= 4, "MapProducer tracks at most four stages");
 
 static __device__ int g_absmax_timeout;                  // set when a bounded wait expired
