@@ -66,7 +66,7 @@ def main():
     def wanted(name):
         return args.only is None or args.only in name
 
-    if wanted("dense"):
+    if any(wanted(name) for name in ("dense, 1 row", "dense, rows of 4096", "dense, rows of 147")):
         g = torch.Generator(device="cuda")
         g.manual_seed(0)
         x = torch.randn(N, device="cuda", generator=g) * 0.02
