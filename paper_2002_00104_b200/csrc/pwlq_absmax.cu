@@ -126,7 +126,11 @@ absmax_kernel(const float* __restrict__ x, Rows rows, int64_t total, uint32_t* _
             const int s = (int)(it % kAbsStages);
             const unsigned use = (unsigned)(it / kAbsStages);
             if (use > 0 && !mbar_wait(&empty_bar[s], (use - 1) & 1u)) {
+                // never expected: report, let the copies of the earlier spans land (their stages'
+                // barriers have this warp's arrivals already), and leave
                 if (lane == 0) atomicExch(&g_absmax_timeout, 1);
+                for (int64_t j = it - 1; j >= 0 && j > it - 1 - kAbsStages; --j)
+                    mbar_wait(&full_bar[j % kAbsStages], (unsigned)(j / kAbsStages) & 1u);
                 return;
             }
             const int64_t span_beg = span * kMapSpan, span_end = min(span_beg + kMapSpan, total);
