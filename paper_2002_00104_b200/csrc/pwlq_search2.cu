@@ -470,19 +470,30 @@ __global__ void __launch_bounds__(kQ2Threads)
 quantize2_kernel(const float* __restrict__ x, Rows rows, int64_t total, int bits,
                  const float* __restrict__ m_arr, const float* __restrict__ p1_arr,
                  const float* __restrict__ p2_arr, uint8_t* __restrict__ codes,
-                 uint8_t* __restrict__ region2, float* __restrict__ fake) {
+                 uint8_t* __restrict__ region2, float* __restrict__ fake, int vec_ok) {
     const int64_t i0 = ((int64_t)blockIdx.x * kQ2Threads + threadIdx.x) * kQ2PerThread;
     if (i0 >= total) return;
     const float Lf = (float)((1 << (bits - 1)) - 1);
     const int cnt = (int)min((int64_t)kQ2PerThread, total - i0);
     Row3 rs;
     uint32_t code[kQ2PerThread], reg[kQ2PerThread];
+    // whole groups of 16 with aligned buffers: 128-bit loads, one store per output
+    const bool vec = cnt == kQ2PerThread && vec_ok;
+    float xv[kQ2PerThread], yv[kQ2PerThread];
+    if (vec) {
+#pragma unroll
+        for (int v = 0; v < kQ2PerThread / 4; ++v) {
+            const float4 q = __ldcs(reinterpret_cast<const float4*>(x + i0) + v);
+            xv[4 * v] = q.x; xv[4 * v + 1] = q.y; xv[4 * v + 2] = q.z; xv[4 * v + 3] = q.w;
+        }
+    }
 #pragma unroll
     for (int t = 0; t < kQ2PerThread; ++t) {
         code[t] = reg[t] = 0;
+        yv[t] = 0.0f;
         if (t < cnt) {
             rs.seek(rows, m_arr, p1_arr, p2_arr, Lf, i0 + t);
-            const float xi = x[i0 + t];
+            const float xi = vec ? xv[t] : x[i0 + t];
             float y = 0.0f;
             if (rs.m > 0.0f) {
                 const float a = fminf(fabsf(xi), rs.m);
@@ -498,10 +509,35 @@ quantize2_kernel(const float* __restrict__ x, Rows rows, int64_t total, int bits
                 reg[t] = (uint32_t)r;
                 y = neg ? -v : v;
             }
-            if (WANT_FAKE) fake[i0 + t] = y;
+            yv[t] = y;
+            if (WANT_FAKE && !vec) fake[i0 + t] = y;
         }
     }
     // i0 is a multiple of 16: region bytes i0/4 .. i0/4 + 3, code bytes i0 .. (or i0/2 ..)
+    if (vec) {
+        uint32_t rw = 0;
+#pragma unroll
+        for (int t = 0; t < kQ2PerThread; ++t) rw |= reg[t] << (2 * t);
+        *reinterpret_cast<uint32_t*>(region2 + (i0 >> 2)) = rw;
+        if (PACKED) {
+            uint32_t w0 = 0, w1 = 0;
+#pragma unroll
+            for (int t = 0; t < 8; ++t) { w0 |= code[t] << (4 * t); w1 |= code[8 + t] << (4 * t); }
+            *reinterpret_cast<uint2*>(codes + (i0 >> 1)) = make_uint2(w0, w1);
+        } else {
+            uint32_t w[4] = {0, 0, 0, 0};
+#pragma unroll
+            for (int t = 0; t < kQ2PerThread; ++t) w[t >> 2] |= code[t] << (8 * (t & 3));
+            *reinterpret_cast<uint4*>(codes + i0) = make_uint4(w[0], w[1], w[2], w[3]);
+        }
+        if (WANT_FAKE) {
+#pragma unroll
+            for (int v = 0; v < kQ2PerThread / 4; ++v)
+                __stcs(reinterpret_cast<float4*>(fake + i0) + v,
+                       make_float4(yv[4 * v], yv[4 * v + 1], yv[4 * v + 2], yv[4 * v + 3]));
+        }
+        return;
+    }
 #pragma unroll
     for (int b = 0; b < 4; ++b)
         if (4 * b < cnt)
@@ -523,28 +559,57 @@ __global__ void __launch_bounds__(kQ2Threads)
 dequantize2_kernel(const uint8_t* __restrict__ codes, const uint8_t* __restrict__ region2,
                    Rows rows, int64_t total, int bits, const float* __restrict__ m_arr,
                    const float* __restrict__ p1_arr, const float* __restrict__ p2_arr,
-                   float* __restrict__ y) {
+                   float* __restrict__ y, int vec_ok) {
     const int64_t i0 = ((int64_t)blockIdx.x * kQ2Threads + threadIdx.x) * kQ2PerThread;
     if (i0 >= total) return;
     const float Lf = (float)((1 << (bits - 1)) - 1);
     const int qmask = (1 << (bits - 1)) - 1;
     const int cnt = (int)min((int64_t)kQ2PerThread, total - i0);
     Row3 rs;
+    // whole groups of 16 with aligned buffers: one load per input, 128-bit stores
+    const bool vec = cnt == kQ2PerThread && vec_ok;
+    uint32_t cw[4] = {0, 0, 0, 0}, rw = 0;
+    float yv[kQ2PerThread];
+    if (vec) {
+        rw = __ldcs(reinterpret_cast<const unsigned int*>(region2 + (i0 >> 2)));
+        if (PACKED) {
+            const uint2 q = __ldcs(reinterpret_cast<const uint2*>(codes + (i0 >> 1)));
+            cw[0] = q.x; cw[1] = q.y;
+        } else {
+            const uint4 q = __ldcs(reinterpret_cast<const uint4*>(codes + i0));
+            cw[0] = q.x; cw[1] = q.y; cw[2] = q.z; cw[3] = q.w;
+        }
+    }
 #pragma unroll
     for (int t = 0; t < kQ2PerThread; ++t) {
+        yv[t] = 0.0f;
         if (t < cnt) {
             rs.seek(rows, m_arr, p1_arr, p2_arr, Lf, i0 + t);
             const int64_t i = i0 + t;
-            const int code = PACKED ? ((codes[i >> 1] >> ((i & 1) * 4)) & 0xF) : codes[i];
-            int r = (region2[i >> 2] >> ((i & 3) * 2)) & 3;
+            int code, r;
+            if (vec) {
+                code = PACKED ? (int)((cw[t >> 3] >> (4 * (t & 7))) & 0xFu)
+                              : (int)((cw[t >> 2] >> (8 * (t & 3))) & 0xFFu);
+                r = (int)((rw >> (2 * t)) & 3u);
+            } else {
+                code = PACKED ? ((codes[i >> 1] >> ((i & 1) * 4)) & 0xF) : codes[i];
+                r = (region2[i >> 2] >> ((i & 3) * 2)) & 3;
+            }
             r = min(r, 2);
             const float s = r == 0 ? rs.P.s[0] : (r == 1 ? rs.P.s[1] : rs.P.s[2]);
             const float z = r == 0 ? 0.0f : (r == 1 ? rs.P.z[1] : rs.P.z[2]);
             float v = __fadd_rn(__fmul_rn((float)(code & qmask), s), z);
             int neg = (code >> (bits - 1)) & 1;
             if (!(rs.m > 0.0f)) { v = 0.0f; neg = 0; }
-            y[i] = neg ? -v : v;
+            yv[t] = neg ? -v : v;
+            if (!vec) y[i] = yv[t];
         }
+    }
+    if (vec) {
+#pragma unroll
+        for (int v = 0; v < kQ2PerThread / 4; ++v)
+            __stcs(reinterpret_cast<float4*>(y + i0) + v,
+                   make_float4(yv[4 * v], yv[4 * v + 1], yv[4 * v + 2], yv[4 * v + 3]));
     }
 }
 
@@ -557,12 +622,14 @@ cudaError_t launch_quantize2(const float* x, const int64_t* row_offsets, int64_t
     const bool packed = (layout == 1 && bits <= 4);
     const int64_t per_cta = (int64_t)kQ2Threads * kQ2PerThread;
     const unsigned grid = (unsigned)((total + per_cta - 1) / per_cta);
+    auto al = [](const void* q, size_t a) { return (reinterpret_cast<uintptr_t>(q) & (a - 1)) == 0; };
+    const int vec_ok = al(x, 16) && al(codes, 16) && al(region2, 4) && (!fake || al(fake, 16));
     if (packed) {
-        if (fake) quantize2_kernel<true, true><<<grid, kQ2Threads, 0, stream>>>(x, rows, total, bits, m, p1, p2, codes, region2, fake);
-        else      quantize2_kernel<true, false><<<grid, kQ2Threads, 0, stream>>>(x, rows, total, bits, m, p1, p2, codes, region2, fake);
+        if (fake) quantize2_kernel<true, true><<<grid, kQ2Threads, 0, stream>>>(x, rows, total, bits, m, p1, p2, codes, region2, fake, vec_ok);
+        else      quantize2_kernel<true, false><<<grid, kQ2Threads, 0, stream>>>(x, rows, total, bits, m, p1, p2, codes, region2, fake, vec_ok);
     } else {
-        if (fake) quantize2_kernel<false, true><<<grid, kQ2Threads, 0, stream>>>(x, rows, total, bits, m, p1, p2, codes, region2, fake);
-        else      quantize2_kernel<false, false><<<grid, kQ2Threads, 0, stream>>>(x, rows, total, bits, m, p1, p2, codes, region2, fake);
+        if (fake) quantize2_kernel<false, true><<<grid, kQ2Threads, 0, stream>>>(x, rows, total, bits, m, p1, p2, codes, region2, fake, vec_ok);
+        else      quantize2_kernel<false, false><<<grid, kQ2Threads, 0, stream>>>(x, rows, total, bits, m, p1, p2, codes, region2, fake, vec_ok);
     }
     return cudaGetLastError();
 }
@@ -576,8 +643,10 @@ cudaError_t launch_dequantize2(const uint8_t* codes, const uint8_t* region2,
     const bool packed = (layout == 1 && bits <= 4);
     const int64_t per_cta = (int64_t)kQ2Threads * kQ2PerThread;
     const unsigned grid = (unsigned)((total + per_cta - 1) / per_cta);
-    if (packed) dequantize2_kernel<true><<<grid, kQ2Threads, 0, stream>>>(codes, region2, rows, total, bits, m, p1, p2, y);
-    else        dequantize2_kernel<false><<<grid, kQ2Threads, 0, stream>>>(codes, region2, rows, total, bits, m, p1, p2, y);
+    auto al = [](const void* q, size_t a) { return (reinterpret_cast<uintptr_t>(q) & (a - 1)) == 0; };
+    const int vec_ok = al(y, 16) && al(codes, 16) && al(region2, 4);
+    if (packed) dequantize2_kernel<true><<<grid, kQ2Threads, 0, stream>>>(codes, region2, rows, total, bits, m, p1, p2, y, vec_ok);
+    else        dequantize2_kernel<false><<<grid, kQ2Threads, 0, stream>>>(codes, region2, rows, total, bits, m, p1, p2, y, vec_ok);
     return cudaGetLastError();
 }
 
