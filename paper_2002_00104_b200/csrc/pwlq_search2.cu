@@ -452,12 +452,30 @@ constexpr int kQ2PerThread = 16;      // consecutive values per thread: four reg
 // Row state of a thread that walks consecutive values.
 struct Row3 {
     int64_t row = -1, end = 0;
+    int64_t first = 0, last = 0;       // the rows of the warp's values: bounds of the first lookup
     float m = 0.0f;
     Params3 P;
+    // The rows that hold the first and the last value of the warp's 32 x kQ2PerThread values,
+    // found by the warp together (a few dependent loads instead of a bisection over all rows per
+    // thread).  Every lane of the warp calls this, before any lane leaves.
+    __device__ __forceinline__ void bracket(const Rows& rows, int64_t warp_beg, int64_t total) {
+        if (warp_beg >= total) return;
+        first = warp_row_of(rows, warp_beg);
+        last = warp_row_of(rows, min(warp_beg + 32 * (int64_t)kQ2PerThread, total) - 1);
+    }
     __device__ __forceinline__ void seek(const Rows& rows, const float* m_arr, const float* p1,
                                          const float* p2, float Lf, int64_t i) {
         if (row >= 0 && i < end) return;
-        row = (row < 0) ? rows.row_of(i) : row + 1;
+        if (row < 0) {                                    // last row of [first, last] that begins at or before i
+            int64_t lo = first, hi = last;
+            while (hi > lo) {
+                const int64_t mid = (lo + hi + 1) >> 1;
+                if (rows.begin(mid) <= i) lo = mid; else hi = mid - 1;
+            }
+            row = lo;
+        } else {
+            row = row + 1;
+        }
         while (rows.begin(row + 1) <= i) ++row;              // skips empty rows
         end = rows.begin(row + 1);
         m = __ldg(m_arr + row);
@@ -472,10 +490,11 @@ quantize2_kernel(const float* __restrict__ x, Rows rows, int64_t total, int bits
                  const float* __restrict__ p2_arr, uint8_t* __restrict__ codes,
                  uint8_t* __restrict__ region2, float* __restrict__ fake, int vec_ok) {
     const int64_t i0 = ((int64_t)blockIdx.x * kQ2Threads + threadIdx.x) * kQ2PerThread;
+    Row3 rs;
+    rs.bracket(rows, i0 - (int64_t)(threadIdx.x & 31) * kQ2PerThread, total);
     if (i0 >= total) return;
     const float Lf = (float)((1 << (bits - 1)) - 1);
     const int cnt = (int)min((int64_t)kQ2PerThread, total - i0);
-    Row3 rs;
     uint32_t code[kQ2PerThread], reg[kQ2PerThread];
     // whole groups of 16 with aligned buffers: 128-bit loads, one store per output
     const bool vec = cnt == kQ2PerThread && vec_ok;
@@ -561,11 +580,12 @@ dequantize2_kernel(const uint8_t* __restrict__ codes, const uint8_t* __restrict_
                    const float* __restrict__ p1_arr, const float* __restrict__ p2_arr,
                    float* __restrict__ y, int vec_ok) {
     const int64_t i0 = ((int64_t)blockIdx.x * kQ2Threads + threadIdx.x) * kQ2PerThread;
+    Row3 rs;
+    rs.bracket(rows, i0 - (int64_t)(threadIdx.x & 31) * kQ2PerThread, total);
     if (i0 >= total) return;
     const float Lf = (float)((1 << (bits - 1)) - 1);
     const int qmask = (1 << (bits - 1)) - 1;
     const int cnt = (int)min((int64_t)kQ2PerThread, total - i0);
-    Row3 rs;
     // whole groups of 16 with aligned buffers: one load per input, 128-bit stores
     const bool vec = cnt == kQ2PerThread && vec_ok;
     uint32_t cw[4] = {0, 0, 0, 0}, rw = 0;
