@@ -379,11 +379,14 @@ def run_ours(args, rank, world, local_rank):
     # its row length; ragged rows: one per row-length class that begins at or below the longest
     # row -- the library does not look at the lengths), the two combine launches when a row exceeds
     # one tile, quantize, dequantize
+    tiled = max_n > 8192 or (max_n > 1024 and w.C * -(-max_n // 8192) < 296)   # several tiles per row
     if w.K > 1024 or dense_n is not None:
         classes = 1
+    elif tiled and max_n <= 8192:
+        classes = 2                                     # one launch for all rows above 64 values
     else:
         classes = sum(max_n >= lo for lo in (0, 65, 513, 2305))
-    per_step = 1 + classes + (2 if max_n > 8192 else 0) + 2
+    per_step = 1 + classes + (2 if tiled else 0) + 2
     if rank == 0:
         peaks, peak_kind = measured_peaks()
         ec = w.elem_cand

@@ -24,6 +24,7 @@ cudaError_t launch_minmax(const float* x, const int64_t* row_offsets, int64_t C,
 struct SearchPlan {
     int64_t max_n;         // longest row
     int64_t tiles;         // tiles per row (by the longest row)
+    int64_t tile;          // values per tile when a row has several (<= kSearchTile)
     size_t off_m;          // workspace offset of the internally computed ranges [C] floats
     size_t off_partials;   // workspace offset of the partial sums [C * tiles * K] doubles (tiles > 1)
     size_t off_sums;       // workspace offset of the combined sums [C * K] doubles (tiles > 1)

@@ -789,8 +789,20 @@ static inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; 
 SearchPlan plan_search(int64_t C, int64_t max_n, int K) {
     SearchPlan p;
     p.max_n = max_n;
+    p.tile = kSearchTile;
     p.tiles = (max_n + kSearchTile - 1) / kSearchTile;
     if (p.tiles < 1) p.tiles = 1;
+    // A few long rows (a per-tensor search) give few CTAs at full tiles: cut them finer, down to
+    // kMinSplitTile values, until there are about two CTAs per SM.  (The extra tiles cost a
+    // sort each, but they run side by side.)
+    constexpr int64_t kMinSplitTile = 1024, kWantCtas = 2 * 148;
+    if (max_n > kMinSplitTile && C * p.tiles < kWantCtas) {
+        const int64_t per_row = (kWantCtas + C - 1) / C;                    // tiles wanted per row
+        int64_t tile = (max_n + per_row - 1) / per_row;
+        tile = std::min<int64_t>(std::max<int64_t>((tile + 255) / 256 * 256, kMinSplitTile), kSearchTile);
+        const int64_t tiles = (max_n + tile - 1) / tile;
+        if (tiles > 1) { p.tile = tile; p.tiles = tiles; }
+    }
     p.off_m = 256;
     p.off_partials = align_up(p.off_m + sizeof(float) * (size_t)C, 256);
     p.off_sums = p.off_partials;
@@ -828,7 +840,7 @@ cudaError_t launch_search(const float* x, const int64_t* row_offsets, int64_t C,
     a.lo = lo;
     a.levels = lo ? (1 << bits) - 1 : (1 << (bits - 1)) - 1;
     a.tiles = plan.tiles;
-    a.cap = (plan.tiles > 1) ? kSearchTile : (int)((plan.max_n + 3) / 4 * 4);
+    a.cap = (plan.tiles > 1) ? (int)plan.tile : (int)((plan.max_n + 3) / 4 * 4);
     a.partials = reinterpret_cast<double*>(ws + plan.off_partials);
     a.p_out = p_out;
     a.err_out = err_out;
@@ -844,8 +856,15 @@ cudaError_t launch_search(const float* x, const int64_t* row_offsets, int64_t C,
         struct RowClass { int64_t n_min, n_max; int threads; };
         // (boundaries measured on B200: 128-thread CTAs beat 256-thread ones up to rows of about
         // 2300 values, 64-thread CTAs beat 128-thread ones up to about 500)
-        const RowClass classes[4] = {{2305, INT64_MAX, 256}, {513, 2304, 128},
-                                     {kTinyMax + 1, 512, 64}, {0, kTinyMax, 0}};   // 0: tiny rows
+        RowClass classes[4] = {{2305, INT64_MAX, 256}, {513, 2304, 128},
+                               {kTinyMax + 1, 512, 64}, {0, kTinyMax, 0}};   // 0: tiny rows
+        if (plan.tile < kSearchTile) {
+            // a few long rows cut into finer tiles (plan_search): every row longer than the tiny
+            // ones is tiled the same way, in one launch, so that the combine kernel finds the
+            // partial sums of all its tiles
+            classes[0] = RowClass{kTinyMax + 1, INT64_MAX, plan.tile <= 2304 ? 128 : 256};
+            classes[1] = classes[2] = RowClass{INT64_MAX, INT64_MAX, 64};   // never launched
+        }
         size_t off[7];
         const size_t smem_max = sorted_smem_layout(a.cap, K, kSWarps, off);
         if (smem_max > 48 * 1024) {  // above the default limit: opt in (idempotent, per device)
