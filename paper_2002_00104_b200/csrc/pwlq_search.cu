@@ -726,11 +726,12 @@ search_generic_kernel(SearchArgs a) {
 }
 
 // Long rows, step 1: sums the tiles' partial sums of 32 candidates of one row.  The tiles are cut
-// into eight consecutive segments, one per warp, each summed in ascending tile order; the eight
+// into kCombineWarps consecutive segments, one per warp, each summed in ascending tile order; the
 // segment sums are then added in ascending order.  Fixed order, hence reproducible.
-__global__ void __launch_bounds__(kSThreads)
+constexpr int kCombineWarps = 32;
+__global__ void __launch_bounds__(kCombineWarps * 32)
 search_combine_kernel(SearchArgs a, double* __restrict__ sums) {
-    __shared__ double seg[kSWarps][32];
+    __shared__ double seg[kCombineWarps][32];
     const int chunks = (a.K + 31) / 32;
     const int64_t row = blockIdx.x / chunks;
     const int chunk = (int)(blockIdx.x - row * chunks);
@@ -743,7 +744,7 @@ search_combine_kernel(SearchArgs a, double* __restrict__ sums) {
                         (__float_as_uint(lo) & 0x7fffffffu) < 0x7f800000u;
     const bool degenerate = !finite || !(m > 0.0f) || n_row <= 0;
     const int64_t nt = degenerate ? 0 : (n_row + a.cap - 1) / a.cap;
-    const int64_t t0 = nt * warp / kSWarps, t1 = nt * (warp + 1) / kSWarps;
+    const int64_t t0 = nt * warp / kCombineWarps, t1 = nt * (warp + 1) / kCombineWarps;
     double tot = 0.0;
     if (k < a.K) {
         const double* src = a.partials + (size_t)row * a.tiles * a.K + k;
@@ -753,7 +754,7 @@ search_combine_kernel(SearchArgs a, double* __restrict__ sums) {
     __syncthreads();
     if (warp == 0 && k < a.K) {
         double v = seg[0][lane];
-        for (int w = 1; w < kSWarps; ++w) v += seg[w][lane];
+        for (int w = 1; w < kCombineWarps; ++w) v += seg[w][lane];
         sums[row * a.K + k] = v;
         if (a.sse_all) a.sse_all[row * a.K + k] = (float)v;
     }
@@ -924,7 +925,7 @@ cudaError_t launch_search(const float* x, const int64_t* row_offsets, int64_t C,
     if (plan.tiles > 1) {
         double* sums = reinterpret_cast<double*>(ws + plan.off_sums);
         const int64_t chunks = (K + 31) / 32;
-        search_combine_kernel<<<(unsigned)(C * chunks), kSThreads, 0, stream>>>(a, sums);
+        search_combine_kernel<<<(unsigned)(C * chunks), kCombineWarps * 32, 0, stream>>>(a, sums);
         e = cudaGetLastError();
         if (e != cudaSuccess) return e;
         search_argmin_kernel<<<(unsigned)C, kSThreads, 0, stream>>>(a, sums);
