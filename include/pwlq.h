@@ -29,8 +29,13 @@
  * Pointers.  Unless a parameter says "host", every pointer is a DEVICE pointer
  * owned by the caller, valid on the device that is current at the call; fp32 and
  * int32 arrays need 4-byte alignment, int64 and workspace 8 / 256 bytes.  The
- * library keeps no state between calls and allocates no memory (the *_host
- * call included: it works in caller-provided device scratch).
+ * library allocates no device memory (the *_host call included: it works in
+ * caller-provided device scratch).  What it keeps per device, for the life of
+ * the process: the occupancy figures of its kernels (looked up at a kernel's first
+ * launch), two streams and a few events of pwlq_encode_host (created at its first
+ * call), the device address of the built-in scratch of pwlq_search_noalloc, and
+ * the two expiry flags that pwlq_device_status reads and clears.  The tables are
+ * guarded by mutexes; calls may come from several host threads.
  *
  * Execution.  Every call only enqueues work on `stream` (a cudaStream_t passed
  * as void*, NULL = default stream) and returns; results are valid after the
@@ -259,7 +264,7 @@ int pwlq_unpack_dense(const uint8_t* stream_in, int64_t total, int bits, uint8_t
  * O(n) per row instead of O(n K); the result can be fed to pwlq_quantize directly.
  *   model      PWLQ_MODEL_GAUSS_APPROX   p = sigma ln(0.8614 m / sigma + 0.6079)  (Sec. 5.1, m and p
  *                                        in units of sigma)
- *              PWLQ_MODEL_GAUSS_ROOT     Gaussian, root of Eq. 9 (80 bisection steps, binary64)
+ *              PWLQ_MODEL_GAUSS_ROOT     Gaussian, root of Eq. 9 (bracketed Newton iteration, binary64)
  *              PWLQ_MODEL_LAPLACE        Laplacian, root of Eq. 9
  *   scale fit  sigma = sqrt(mean x^2) (Gaussian), b = mean |x| (Laplacian), binary64 sums in a
  *              fixed order
@@ -319,11 +324,13 @@ int pwlq_search_noalloc(const float* x, int64_t C, int64_t n, int bits, const fl
                         float* sse_all, int32_t* status_out, void* stream);
 size_t pwlq_search_noalloc_max_bytes(void);
 
-/* The streaming kernels (abs-max, quantize) receive their inputs through asynchronous bulk copies
- * whose completion they await with a bounded number of polls; a wait that runs out makes the
- * kernel stop early and sets a flag on the device.  This call reads the flags (it synchronises
- * with the device) and returns 0, or 1 << PWLQ_ERR_TIMEOUT if any wait has expired since the
- * library was loaded, in which case the outputs of that call are not valid. */
+/* The streaming kernels (abs-max, quantize, dequantize) hand their data over through shared-memory
+ * barriers that they await with a bounded number of polls; a wait that runs out makes the kernel
+ * stop early and sets a flag on the current device.  This call reads the flags (it synchronises
+ * with the device) and returns 0, or 1 << PWLQ_ERR_TIMEOUT if a wait has expired on the current
+ * device since the previous call of pwlq_device_status -- the outputs of the streaming calls made
+ * in between are then not valid -- or 1 << PWLQ_ERR_CUDA if the flags could not be read.  Reading
+ * clears the flags: call it after synchronising the work it is meant to vouch for. */
 int pwlq_device_status(void);
 
 /* Text for a status value (static storage). */

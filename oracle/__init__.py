@@ -3,10 +3,10 @@
 Only the tests, the smoke check and the benchmark's CPU-baseline leg import
 this package.  It shares no code with the CUDA path.
 """
-from .pwlq_oracle import (  # noqa: F401
-    OracleError, OracleLib, absmax, analytic_p, bias_correction, build, code_bytes, dequantize,
-    dequantize2, dequantize_bc, pack_dense, unpack_dense,
-    dequantize_u, elem,
-    elem_u, minmax, params, quantize, quantize2, quantize_u, search, search2, search_u,
-    select_analytic,
-)
+from . import pwlq_oracle as _impl
+from .pwlq_oracle import OracleError, OracleLib, build, code_bytes  # noqa: F401
+
+
+def __getattr__(name):
+    """``oracle.search(...)`` and the like: methods of one shared ``OracleLib``."""
+    return getattr(_impl, name)

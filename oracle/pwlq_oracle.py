@@ -377,81 +377,9 @@ def _get() -> OracleLib:
     return _default
 
 
-def absmax(*a, **k):
-    return _get().absmax(*a, **k)
-
-
-def search(*a, **k):
-    return _get().search(*a, **k)
-
-
-def quantize(*a, **k):
-    return _get().quantize(*a, **k)
-
-
-def dequantize(*a, **k):
-    return _get().dequantize(*a, **k)
-
-
-def elem(*a, **k):
-    return _get().elem(*a, **k)
-
-
-def analytic_p(*a, **k):
-    return _get().analytic_p(*a, **k)
-
-
-def select_analytic(*a, **k):
-    return _get().select_analytic(*a, **k)
-
-
-def params(*a, **k):
-    return _get().params(*a, **k)
-
-
-def minmax(*a, **k):
-    return _get().minmax(*a, **k)
-
-
-def search_u(*a, **k):
-    return _get().search_u(*a, **k)
-
-
-def quantize_u(*a, **k):
-    return _get().quantize_u(*a, **k)
-
-
-def dequantize_u(*a, **k):
-    return _get().dequantize_u(*a, **k)
-
-
-def elem_u(*a, **k):
-    return _get().elem_u(*a, **k)
-
-
-def search2(*a, **k):
-    return _get().search2(*a, **k)
-
-
-def quantize2(*a, **k):
-    return _get().quantize2(*a, **k)
-
-
-def dequantize2(*a, **k):
-    return _get().dequantize2(*a, **k)
-
-
-def bias_correction(*a, **k):
-    return _get().bias_correction(*a, **k)
-
-
-def dequantize_bc(*a, **k):
-    return _get().dequantize_bc(*a, **k)
-
-
-def pack_dense(*a, **k):
-    return _get().pack_dense(*a, **k)
-
-
-def unpack_dense(*a, **k):
-    return _get().unpack_dense(*a, **k)
+def __getattr__(name):
+    """Module-level access to the default oracle's methods: ``pwlq_oracle.search(...)`` is
+    ``OracleLib().search(...)`` on one shared instance."""
+    if not name.startswith("_") and callable(getattr(OracleLib, name, None)):
+        return getattr(_get(), name)
+    raise AttributeError(name)

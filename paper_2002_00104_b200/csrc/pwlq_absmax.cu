@@ -5,6 +5,7 @@
 // filled by bulk asynchronous copies together with a map of the rows that start in them.
 // Magnitude bit patterns are folded with an integer maximum (exact and order-free).
 #include <algorithm>
+#include <mutex>
 
 #include "pwlq_common.cuh"
 #include "pwlq_kernels.h"
@@ -307,9 +308,11 @@ absmax_kernel(const float* __restrict__ x, Rows rows, int64_t total, uint32_t* _
     flush_acc();                                      // what is still carried at the end
 }
 
-int absmax_timeout_flag() {
+int take_absmax_timeout_flag() {
     int v = 0;
-    cudaMemcpyFromSymbol(&v, g_absmax_timeout, sizeof(int));
+    const int zero = 0;
+    if (cudaMemcpyFromSymbol(&v, g_absmax_timeout, sizeof(int)) != cudaSuccess) return -1;
+    if (v != 0 && cudaMemcpyToSymbol(g_absmax_timeout, &zero, sizeof(int)) != cudaSuccess) return -1;
     return v;
 }
 
@@ -350,11 +353,13 @@ static cudaError_t launch_fold(const float* x, const int64_t* row_offsets, int64
     const size_t smem = sizeof(AbsStage) * kAbsStages;
     const void* kernel = long_rows ? (const void*)absmax_kernel<MINMAX, true>
                                    : (const void*)absmax_kernel<MINMAX, false>;
-    static int cached[2][64] = {{0}};                  // CTAs that fit the device at once
+    static int cached[2][2][64] = {{{0}}};             // CTAs that fit the device at once
+    static std::mutex cached_mu;
     int dev = 0;
     cudaGetDevice(&dev);
     if (dev < 0 || dev >= 64) dev = 0;
-    int& slots_dev = cached[long_rows ? 1 : 0][dev];
+    std::lock_guard<std::mutex> lock(cached_mu);
+    int& slots_dev = cached[MINMAX ? 1 : 0][long_rows ? 1 : 0][dev];
     if (slots_dev == 0) {
         e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (e != cudaSuccess) return e;

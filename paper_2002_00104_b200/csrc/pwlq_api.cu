@@ -680,8 +680,17 @@ int pwlq_select_analytic_ragged(const float* x, const int64_t* row_offsets, int6
 }
 
 int pwlq_device_status(void) {
-    const int expired = pwlq::absmax_timeout_flag() | pwlq::quantize_timeout_flag();
-    return expired ? (1 << PWLQ_ERR_TIMEOUT) : 0;
+    const int a = pwlq::take_absmax_timeout_flag(), q = pwlq::take_quantize_timeout_flag();
+    if (a < 0 || q < 0) return 1 << PWLQ_ERR_CUDA;
+    return (a | q) ? (1 << PWLQ_ERR_TIMEOUT) : 0;
+}
+
+// Not part of the public interface (include/pwlq.h does not declare it): lets the test suite see
+// a bounded device wait run out.  A one-warp kernel waits `polls` times (1 .. 1024) on a barrier
+// nobody arrives on, sets the flag pwlq_device_status() reports, and returns.
+int pwlq_selftest_expire_wait(int polls, void* stream) {
+    if (polls < 1 || polls > 1024) return PWLQ_ERR_INVALID_ARG;
+    return from_cuda(pwlq::launch_expire_wait(polls, as_stream(stream)));
 }
 
 const char* pwlq_status_string(int status) {

@@ -92,9 +92,12 @@ cudaError_t launch_select_analytic(const float* x, const int64_t* row_offsets, i
                                    float* p_out, float* scale_out, void* workspace,
                                    cudaStream_t stream);
 
-// 1 when a bounded wait of the kernel family expired since the library was loaded (reads a
-// device flag: synchronises with the device).
-int absmax_timeout_flag();
-int quantize_timeout_flag();
+// 1 when a bounded wait of the kernel family expired on the current device since the last call
+// of the same function, which also clears the flag (reads a device flag: synchronises with the
+// device); -1 when the flag could not be read.
+int take_absmax_timeout_flag();
+int take_quantize_timeout_flag();
+// Runs a bounded wait that is certain to expire after `polls` polls (self-test of the reporting).
+cudaError_t launch_expire_wait(int polls, cudaStream_t stream);
 
 }  // namespace pwlq

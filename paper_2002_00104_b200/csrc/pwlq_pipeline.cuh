@@ -38,8 +38,8 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, unsigned parity) {
 // Bounded wait: false after kMaxSpins unsuccessful polls, i.e. after about half a second, far
 // longer than any copy can take.
 constexpr int kMaxSpins = 1 << 18;
-__device__ __forceinline__ bool mbar_wait(uint64_t* bar, unsigned parity) {
-    for (int i = 0; i < kMaxSpins; ++i)
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, unsigned parity, int max_spins = kMaxSpins) {
+    for (int i = 0; i < max_spins; ++i)
         if (mbar_try_wait(bar, parity)) return true;
     return false;
 }

@@ -341,13 +341,14 @@ quantize_map_kernel(const float* __restrict__ x, Rows rows, int64_t total, int b
                                 const float4 ea = S.qa[lt];
                                 const float4 eb = QB ? S.qb[lt] : make_float4(0.0f, 0.0f, 0.0f, 0.0f);
                                 if (UNS) yv[t] = eb.z;                 // a constant row delivers lo
-                                if (ea.x > 0.0f) {
+                                const float em = fabsf(ea.x);          // (-m marks a row kept off the fast paths)
+                                if (em > 0.0f) {
                                     const float xi = xv[t];
                                     const int neg = !UNS && xi < 0.0f;
                                     int q, tail;
                                     float v;
-                                    const float a = UNS ? fminf(fmaxf(__fsub_rn(xi, eb.z), 0.0f), ea.x)
-                                                        : fminf(fabsf(xi), ea.x);
+                                    const float a = UNS ? fminf(fmaxf(__fsub_rn(xi, eb.z), 0.0f), em)
+                                                        : fminf(fabsf(xi), em);
                                     quantize_mag(a, params_of(ea, eb), Lf, q, tail, v);
                                     const uint32_t code = (uint32_t)((neg << (bits - 1)) | q);
                                     if (PACKED) w0 |= code << (4 * t);
@@ -806,10 +807,29 @@ static SpanGrid span_grid(const void* kernel, int threads, size_t smem, int64_t 
     return SpanGrid{(unsigned)((nspans + per_cta - 1) / per_cta), per_cta};
 }
 
-int quantize_timeout_flag() {
+int take_quantize_timeout_flag() {
     int v = 0;
-    cudaMemcpyFromSymbol(&v, g_quantize_timeout, sizeof(int));
+    const int zero = 0;
+    if (cudaMemcpyFromSymbol(&v, g_quantize_timeout, sizeof(int)) != cudaSuccess) return -1;
+    if (v != 0 && cudaMemcpyToSymbol(g_quantize_timeout, &zero, sizeof(int)) != cudaSuccess) return -1;
     return v;
+}
+
+// Self-test of the expiry path: one warp initialises a barrier that expects one arrival which
+// nobody makes, polls it `polls` times through the helper the streaming kernels use, reports the
+// expiry exactly as they do, and returns.  No copy is in flight and nothing is left waiting.
+__global__ void expire_wait_kernel(int polls) {
+    __shared__ uint64_t bar;
+    if (threadIdx.x == 0) {
+        mbar_init(&bar, 1);
+        fence_barrier_init();
+    }
+    __syncwarp();
+    if (!mbar_wait(&bar, 0u, polls) && threadIdx.x == 0) atomicExch(&g_quantize_timeout, 1);
+}
+cudaError_t launch_expire_wait(int polls, cudaStream_t stream) {
+    expire_wait_kernel<<<1, 32, 0, stream>>>(polls);
+    return cudaGetLastError();
 }
 
 // lo == nullptr: signed scheme, m = abs-max.  lo != nullptr: one-sided ranges [lo, m].

@@ -59,7 +59,10 @@ struct RowInputs {
 };
 
 // Constants of one row as the consumers read them; m is the range width (abs-max, or upper -
-// lower bound).  Quantize (DEQ = false): qa = (m, p, L/p, L/(m-p)), qb = (p/L, (m-p)/L, lo, 0).
+// lower bound).  Quantize (DEQ = false): qa = (m, p, L/p, L/(m-p)), qb = (p/L, (m-p)/L, lo, 0);
+// a row whose L/p or L/(m-p) is not finite (a breakpoint or tail range near the smallest binary32
+// magnitudes) is stored with -m: the branch-free quantizer, which has no saturation, must not see
+// it, and the consumers send every row with m <= 0 to the value-by-value path.
 // Dequantize (DEQ = true): qa = (m, p, p/L, (m-p)/L), qb = (lo, xi, beta, 0) with the scale and
 // offset of the bias correction (1 and 0 without it).
 template <bool DEQ>
@@ -70,7 +73,8 @@ __device__ __forceinline__ void store_row_consts(float4* qa, float4* qb, int slo
         qa[slot] = make_float4(m, P.p, P.s1, P.s2);
         if (qb) qb[slot] = make_float4(lo, xi, beta, 0.0f);
     } else {
-        qa[slot] = make_float4(m, P.p, P.inv1, P.inv2);
+        const bool finite = P.inv1 <= 3.402823466e38f && P.inv2 <= 3.402823466e38f;
+        qa[slot] = make_float4(m > 0.0f ? (finite ? m : -m) : 0.0f, P.p, P.inv1, P.inv2);
         if (qb) qb[slot] = make_float4(P.s1, P.s2, lo, 0.0f);
     }
 }

@@ -15,36 +15,62 @@ namespace pwlq {
 constexpr int kSelThreads = 128;
 constexpr int kSelTile = 8192;
 
-__device__ __forceinline__ double model_cdf(int model, double scale, double p) {
-    if (model == 2) return 1.0 - 0.5 * exp(-p / scale);             // Laplace, p >= 0
-    return 0.5 * erfc(-p / (scale * 1.4142135623730951));           // Gaussian
+// Eq. 9 in units of the density's scale: with t = p / scale and M = m / scale, and F0, f0 the CDF
+// and PDF of the unit-scale density,
+//     h(t) = 2 M F0(t) - 2 M + t - M (M - 2 t) f0(t),       h < 0 left of the root,
+//     h'(t) = 1 + 4 M f0(t) - M (M - 2 t) f0'(t),           f0' = -t f0 (Gaussian), -f0 (Laplacian).
+struct Eq9 {
+    double M;
+    bool laplace;
+    __device__ __forceinline__ void eval(double t, double& h, double& dh) const {
+        double F0, f0, df0;
+        if (laplace) {
+            const double e = exp(-t);
+            F0 = 1.0 - 0.5 * e;
+            f0 = 0.5 * e;
+            df0 = -f0;
+        } else {
+            F0 = 0.5 * erfc(t * -0.70710678118654752);          // -t / sqrt(2)
+            f0 = 0.39894228040143268 * exp(-0.5 * t * t);         // 1 / sqrt(2 pi)
+            df0 = -t * f0;
+        }
+        const double w = M * (M - 2.0 * t);
+        h = 2.0 * M * (F0 - 1.0) + t - w * f0;
+        dh = 1.0 + 4.0 * M * f0 - w * df0;
+    }
+};
+
+// Root of Eq. 9 on (0, M/2) by Newton's iteration kept inside a shrinking bracket (a step that
+// leaves the bracket, or does not at least halve it, is replaced by the bracket's midpoint).
+// Returns M/2 when h(M/2) <= 0 (no sign change inside: the row is flatter than the model).
+__device__ double eq9_root(double M, bool laplace) {
+    const Eq9 g{M, laplace};
+    double a = 0.0, b = 0.5 * M, h, dh;
+    g.eval(b, h, dh);
+    if (!(h > 0.0)) return b;
+    double t = 0.5 * b, width = b - a;
+    for (int it = 0; it < 200; ++it) {
+        g.eval(t, h, dh);
+        if (h < 0.0) a = t; else b = t;
+        if (h == 0.0) break;
+        double next = t - h / dh;
+        const double new_width = b - a;
+        if (!(next > a && next < b) || 2.0 * new_width > width) next = 0.5 * (a + b);
+        width = new_width;
+        if (fabs(next - t) <= 4e-16 * t || new_width <= 4e-16 * b) { t = next; break; }
+        t = next;
+    }
+    return t;
 }
-__device__ __forceinline__ double model_pdf(int model, double scale, double p) {
-    if (model == 2) return 0.5 / scale * exp(-p / scale);
-    const double t = p / scale;
-    return exp(-0.5 * t * t) / (scale * 2.5066282746310002);
-}
-// Eq. 9 as g(p) = 2 m F(p) - [2 m - p + m (m - 2 p) f(p)]; negative left of the root.
-__device__ __forceinline__ double eq9_residual(int model, double scale, double m, double p) {
-    return 2.0 * m * model_cdf(model, scale, p) -
-           (2.0 * m - p + m * (m - 2.0 * p) * model_pdf(model, scale, p));
-}
-// model 0: Gaussian closed form p = sigma ln(0.8614 m / sigma + 0.6079); 1: Gaussian root of
-// Eq. 9; 2: Laplacian root of Eq. 9.  Result in (0, m/2]; m/2 when Eq. 9 has no root there.
+
+// model 0: Gaussian closed form p = sigma ln(0.8614 m / sigma + 0.6079) (Sec. 5.1, m and p in units
+// of sigma); 1: Gaussian root of Eq. 9; 2: Laplacian root of Eq. 9.  Result in (0, m/2]: m/2 when
+// Eq. 9 has no root there, and m/2 * 1e-6 when the closed form's logarithm is not positive.
 __device__ double analytic_breakpoint(double m, double scale, int model) {
     if (!(m > 0.0) || !(scale > 0.0)) return 0.0;
-    double p;
-    if (model == 0) {
-        p = scale * log(0.8614 * (m / scale) + 0.6079);
-    } else {
-        double lo = 0.0, hi = 0.5 * m;
-        if (!(eq9_residual(model, scale, m, hi) > 0.0)) return 0.5 * m;
-        for (int it = 0; it < 80; ++it) {
-            const double mid = 0.5 * (lo + hi);
-            if (eq9_residual(model, scale, m, mid) < 0.0) lo = mid; else hi = mid;
-        }
-        p = 0.5 * (lo + hi);
-    }
+    const double M = m / scale;
+    const double t = (model == 0) ? log(0.8614 * M + 0.6079) : eq9_root(M, model == 2);
+    double p = t * scale;
     if (!(p > 0.0)) p = 0.5 * m * 1e-6;
     if (p > 0.5 * m) p = 0.5 * m;
     return p;

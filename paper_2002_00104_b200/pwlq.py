@@ -79,6 +79,10 @@ _SIGNATURES = {
     "pwlq_status_string": (ctypes.c_char_p, [_INT]),
     "pwlq_version": (ctypes.c_char_p, []),
 }
+# exported by the library but not declared in the public header: hooks for the test suite
+_TEST_HOOKS = {
+    "pwlq_selftest_expire_wait": (_INT, [_INT, _P]),
+}
 
 
 class PwlqError(RuntimeError):
@@ -97,7 +101,7 @@ def load_library(path: Optional[str] = None) -> ctypes.CDLL:
                 f"{path} is missing: build it with `python -m paper_2002_00104_b200.build` "
                 "(nvcc, sm_100a); this package has no CPU or PyTorch fallback")
         lib = ctypes.CDLL(path)
-        for name, (res, args) in _SIGNATURES.items():
+        for name, (res, args) in {**_SIGNATURES, **_TEST_HOOKS}.items():
             fn = getattr(lib, name)
             fn.restype, fn.argtypes = res, args
         _lib = lib
@@ -109,8 +113,15 @@ def exported_symbols():
 
 
 def device_status() -> int:
-    """0, or 1 << ERR_TIMEOUT if a bounded device wait has expired (synchronises)."""
+    """0, or 1 << ERR_TIMEOUT if a bounded device wait has expired on the current device since
+    the previous call (synchronises; reading clears the flag)."""
     return int(load_library().pwlq_device_status())
+
+
+def selftest_expire_wait(polls: int = 48, stream=None) -> None:
+    """Runs a one-warp kernel whose bounded wait is certain to run out (test hook)."""
+    _check(load_library().pwlq_selftest_expire_wait(int(polls), _stream(stream)),
+           "pwlq_selftest_expire_wait")
 
 
 def status_string(status: int) -> str:

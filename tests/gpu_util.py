@@ -1,4 +1,7 @@
 """Helpers shared by the GPU parity tests."""
+import os
+from concurrent.futures import ThreadPoolExecutor
+
 import numpy as np
 import torch
 
@@ -42,3 +45,16 @@ def check_search(gpu, ora, ratios, m, row_len, want_sse=True):
     d = np.abs(gpu["err"].astype(np.float64) - sse_o[rows, gi])
     assert np.all(d <= SSE_RTOL * sse_o[rows, gi] + atol + 2.0 ** -23 * sse_o[rows, gi])
     return int(differ.sum())
+
+
+def oracle_sse_over_candidates(oracle, x, bits, ratios, m, threads=None):
+    """Binary64 sums of ONE long row for every candidate, the single-threaded oracle run on
+    slices of the candidate grid by host threads (the C call releases the interpreter lock)."""
+    threads = threads or max(1, min(os.cpu_count() or 1, 32))
+    chunks = [c for c in np.array_split(np.arange(ratios.size), 4 * threads) if c.size]
+
+    def one(ks):
+        return oracle.search(x, bits, np.ascontiguousarray(ratios[ks]), m=m)["sse64"][0]
+
+    with ThreadPoolExecutor(threads) as ex:
+        return np.concatenate(list(ex.map(one, chunks)))

@@ -7,7 +7,7 @@ import numpy as np
 import pytest
 import torch
 
-from gpu_util import check_search, dev
+from gpu_util import check_search, dev, oracle_sse_over_candidates
 from paper_2002_00104_b200 import workloads as W
 
 pytestmark = [pytest.mark.gpu,
@@ -108,19 +108,17 @@ def test_mobilenetv2_full(pwlq, oracle):
 
 
 def test_relu_activation_full(pwlq, oracle):
+    """One row of 25.7 M values, K = 1024: every one of the 1024 per-candidate sums against the
+    oracle's binary64 sums (the sum over 25.7 M terms with a range of 10^5 .. 10^6 is where
+    accumulation error would show), the oracle fanned over the candidates on the host threads."""
     w = W.relu_activation()
     g = run_path(pwlq, w)
     m = check_all_rows(oracle, w, g)
-    idx = int(g["idx"][0])
-    ks = sorted({0, 1, 7, 100, 511, 1023, max(idx - 1, 0), idx, min(idx + 1, w.K - 1)})
-    ora = oracle.search(w.x, w.bits, g["ratios"][ks], m=m)
-    sse_o = ora["sse64"][0]
-    got = g["sse"][0, ks].astype(np.float64)
-    tol = 1e-5 * sse_o + w.total * (2.0 ** -23 * m[0]) ** 2 + 2.0 ** -23 * sse_o
-    assert np.all(np.abs(got - sse_o) <= tol), (got, sse_o)
-    # the chosen candidate beats its neighbours in the oracle's own sums (up to a near-tie)
-    best = sse_o[ks.index(idx)]
-    assert np.all(sse_o >= best * (1 - 1e-5))
+    sse_o = oracle_sse_over_candidates(oracle, w.x, w.bits, g["ratios"], m)
+    assert sse_o.shape == (w.K,)
+    ora = {"sse64": sse_o[None, :], "idx": np.array([int(np.argmin(sse_o))])}
+    sub = {k: g[k][:1] for k in ("p", "err", "idx", "sse")}
+    check_search(sub, ora, g["ratios"], m[:1], w.total)
 
 
 @pytest.mark.parametrize("bits", [3, 4, 6, 8])
@@ -129,7 +127,7 @@ def test_laplace_matrix_sweep(pwlq, oracle, bits, K):
     w = W.laplace_matrix()
     g = run_path(pwlq, w, bits=bits, K=K)
     m = check_all_rows(oracle, w, g)
-    check_sampled_rows(oracle, w, g, np.arange(5, w.C, 512), m)
+    check_sampled_rows(oracle, w, g, np.arange(5, w.C, 64), m)          # 64 rows per (b, K)
 
 
 # ------------------------------------------------------------ host-buffer entry point, pipelined

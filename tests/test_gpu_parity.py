@@ -340,3 +340,77 @@ def test_encode_host_matches_oracle(pwlq, oracle, ragged):
     assert np.all(gap <= 1e-5 * ora["sse64"][rows, ora["idx"]] + 1e-30)
     oc, ok, _ = oracle.quantize(xo, 4, om, out["p"].numpy(), layout=1, row_offsets=ro)
     assert np.array_equal(out["codes"].numpy(), oc) and np.array_equal(out["mask"].numpy(), ok)
+
+
+def test_a_bounded_wait_that_runs_out_is_reported_once(pwlq):
+    """Failure detection without a fault: a one-warp kernel polls a barrier that nobody arrives on
+    through the streaming kernels' own wait helper, with a limit of a few dozen polls; the wait
+    runs out, the kernel sets the expiry flag and returns.  pwlq_device_status reports it once
+    (reading clears it), and the library works as before afterwards."""
+    torch.cuda.synchronize()
+    assert pwlq.device_status() == 0
+    pwlq.selftest_expire_wait(48)
+    torch.cuda.synchronize()
+    assert pwlq.device_status() == 1 << pwlq.ERR_TIMEOUT
+    assert pwlq.device_status() == 0
+    x = torch.arange(-2000, 2000, dtype=torch.float32, device="cuda").reshape(4, 1000)
+    m = pwlq.absmax(x)
+    torch.cuda.synchronize()
+    assert m.cpu().tolist() == [2000.0, 1000.0, 999.0, 1999.0]
+    assert pwlq.device_status() == 0
+
+
+@pytest.mark.parametrize("layout,bits", [(1, 4), (0, 8), (1, 3)])
+def test_quantize_nan_values_and_ranges_near_the_smallest_magnitudes(pwlq, oracle, layout, bits):
+    """Values outside the precondition (NaN of either sign: quantized like +m by both sides) and
+    rows whose range is so small that L / p or L / (m - p) overflows: every path of the kernel
+    (whole passes inside a row, passes with row starts, the tensor's tail) must give the oracle's
+    bytes."""
+    rng = np.random.default_rng(5 + bits)
+    lengths = np.array([512, 147, 40, 1024, 9, 300, 4096 + 24, 77], np.int64)
+    ro = np.concatenate([[0], np.cumsum(lengths)]).astype(np.int64)
+    x = rng.laplace(0, 0.03, int(ro[-1])).astype(np.float32)
+    tiny = [1, 3, 6]                                         # rows scaled into the subnormal range
+    for c, scale in zip(tiny, (1e-38, 3e-39, 1e-41)):
+        x[ro[c]:ro[c + 1]] *= np.float32(scale) / np.float32(0.03)
+    m = oracle.absmax(x, ro)
+    p = (m * rng.uniform(0.2, 0.9, lengths.size).astype(np.float32)).astype(np.float32)
+    p[6] = m[6] * np.float32(1 - 2.0 ** -20)                 # a tail range of a few subnormal steps
+    nan_pos = np.frombuffer(np.array([0x7FC00000], np.uint32).tobytes(), np.float32)[0]
+    nan_neg = np.frombuffer(np.array([0xFFC00000], np.uint32).tobytes(), np.float32)[0]
+    for c in (0, 2, 3, 5):
+        b, e = int(ro[c]), int(ro[c + 1])
+        x[b] = nan_pos; x[b + 1] = nan_neg; x[e - 1] = nan_neg; x[(b + e) // 2] = nan_pos
+    oc, om, of = oracle.quantize(x, bits, m, p, layout=layout, row_offsets=ro)
+    codes, mask, fake = pwlq.quantize(dev(x), bits, dev(m), dev(p), layout=layout,
+                                      row_offsets=dev(ro), want_fake=True)
+    y = pwlq.dequantize(codes, mask, bits, dev(m), dev(p), layout=layout, row_offsets=dev(ro))
+    torch.cuda.synchronize()
+    assert np.array_equal(np_(codes), oc) and np.array_equal(np_(mask), om)
+    assert np_(fake).tobytes() == of.tobytes() and np_(y).tobytes() == of.tobytes()
+
+
+@pytest.mark.parametrize("K", [64, 256])
+def test_search_many_ragged_rows_of_every_class_with_full_tiles(pwlq, oracle, K):
+    """Enough rows that long rows keep full tiles (no finer cut), rows of every row-length class
+    and rows of several tiles in one call: every class launch writes its rows' partial sums and
+    the combine kernels read them all.  Repeated: the result must not change from run to run."""
+    rng = np.random.default_rng(K)
+    lengths = np.concatenate([rng.integers(1, 3001, 400), [9001, 20000, 8192, 8193, 64, 65, 512,
+                                                           513, 2304, 2305]]).astype(np.int64)
+    rng.shuffle(lengths)
+    ro = np.concatenate([[0], np.cumsum(lengths)]).astype(np.int64)
+    x = (rng.standard_normal(int(ro[-1])) * rng.choice([0.01, 1.0, 30.0], 1)).astype(np.float32)
+    ratios = W.ratio_grid(K)
+    first = None
+    for rep in range(3):
+        out, status = run_search(pwlq, x, 4, ratios, row_offsets=ro, max_n=int(lengths.max()))
+        assert status == 0
+        if first is None:
+            first = out
+            m = oracle.absmax(x, ro)
+            ora = oracle.search(x, 4, ratios, m=m, row_offsets=ro)
+            check_search(out, ora, ratios, m, lengths)
+        else:
+            for k in ("p", "err", "idx", "sse"):
+                assert out[k].tobytes() == first[k].tobytes(), (rep, k)

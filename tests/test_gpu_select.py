@@ -33,6 +33,44 @@ def compare(pwlq, oracle, x, model, row_offsets=None, max_n=None):
 
 
 @pytest.mark.parametrize("model", [0, 1, 2])
+def test_select_against_scipy_and_the_closed_form(pwlq, model):
+    """The GPU's breakpoints against solvers that share nothing with it or with the oracle: SciPy's
+    Brent root finder on Eq. 9 written with SciPy's CDF / PDF (models 1, 2), math.log for the
+    Sec. 5.1 closed form (model 0); the scale against NumPy's binary64 moments."""
+    import math
+    from scipy.optimize import brentq
+    from scipy.stats import laplace, norm
+    rng = np.random.default_rng(91 + model)
+    scales = np.array([0.003, 0.02, 0.05, 0.4, 1.0, 1.3, 7.0, 0.05])
+    n = 6000
+    gen = rng.laplace if model == 2 else rng.normal
+    x = np.stack([gen(0, s, n) for s in scales]).astype(np.float32)
+    x[-1] = rng.uniform(-1, 1, n).astype(np.float32)        # flatter than either model
+    x64 = x.astype(np.float64)
+    m = np.abs(x).max(axis=1)
+    p, scale = pwlq.select_analytic(dev(x), dev(m), model, want_scale=True)
+    torch.cuda.synchronize()
+    p, scale = p.cpu().numpy().astype(np.float64), scale.cpu().numpy().astype(np.float64)
+    fit = np.mean(np.abs(x64), axis=1) if model == 2 else np.sqrt(np.mean(x64 ** 2, axis=1))
+    assert np.allclose(scale, fit, rtol=2e-7, atol=0)
+    inside = 0
+    for c in range(len(scales)):
+        mc, sc = float(m[c]), float(fit[c])
+        if model == 0:
+            want = min(sc * math.log(0.8614 * mc / sc + 0.6079), 0.5 * mc)
+        else:
+            d = (laplace if model == 2 else norm)(0, sc)
+            g = lambda t: 2 * mc * d.cdf(t) - (2 * mc - t + mc * (mc - 2 * t) * d.pdf(t))
+            if g(0.5 * mc) <= 0:
+                want = 0.5 * mc
+            else:
+                want = brentq(g, 1e-12 * mc, 0.5 * mc, xtol=1e-15, rtol=1e-14)
+                inside += 1
+        assert math.isclose(p[c], want, rel_tol=1e-6), (c, p[c], want)
+    assert model == 0 or inside >= 5                        # real roots were compared, not only bounds
+
+
+@pytest.mark.parametrize("model", [0, 1, 2])
 def test_select_ragged_rows(pwlq, oracle, model):
     w = W.small_mixed(seed=31 + model)
     compare(pwlq, oracle, w.x, model, w.row_offsets, int(np.diff(w.row_offsets).max()))
