@@ -104,6 +104,30 @@ int pwlq_search_ragged(const float* x, const int64_t* row_offsets, int64_t C, in
                        float* p_out, float* err_out, int32_t* idx_out, float* sse_all,
                        void* workspace, size_t workspace_bytes, void* stream);
 
+/* The search of a row that is cut into pieces -- one tensor quantized per layer (Sec. 5:
+ * activations) whose elements are spread over several GPUs, or fed in several calls.  The squared
+ * error of Eq. 3 is a sum over values, so every piece contributes its own per-candidate sums under
+ * the row's common range; the pieces' sums are added in a fixed order and the first minimum is
+ * taken (grid form of Eq. 6), exactly as pwlq_search does for the tiles of a long row.
+ *
+ * pwlq_search_partial: x is this piece, [C, n] (n values of each of the C rows); m [C] is the
+ * range of the WHOLE row (e.g. the maximum over the pieces' pwlq_absmax results), required; lo is
+ * NULL for the signed scheme or [C] lower bounds of one-sided ranges [lo, m] as in
+ * pwlq_search_unsigned.  sums_out [C, K] receives the binary64 sums of this piece, 8-byte aligned.
+ * workspace as for pwlq_search (pwlq_search_workspace_bytes(C, n, K); status word in its first
+ * 4 bytes).  No p, error or index is produced.
+ * pwlq_search_finish: sums is [parts, C, K] (the pieces' sums_out stacked in a fixed order, e.g. by
+ * rank); for every row the parts are added in ascending order in binary64, then idx_out = first
+ * minimum, p_out = m * ratios[idx] ((m - lo) * ratios[idx] for one-sided ranges), err_out (may be
+ * NULL) = the minimum, sse_all ([C, K] or NULL) = the totals in binary32.  status_out (4 bytes,
+ * may be NULL) receives the status word (non-finite range).  All pointers are device pointers. */
+int pwlq_search_partial(const float* x, int64_t C, int64_t n, int bits, const float* ratios,
+                        int K, const float* m, const float* lo, double* sums_out, void* workspace,
+                        size_t workspace_bytes, void* stream);
+int pwlq_search_finish(const double* sums, int parts, int64_t C, int K, const float* m,
+                       const float* lo, const float* ratios, float* p_out, float* err_out,
+                       int32_t* idx_out, float* sse_all, int32_t* status_out, void* stream);
+
 /* Quantizer of Eq. 3 with the chosen (m[c], p[c]) of each row, 0 < p <= m.
  *   codes        PWLQ_CODES_U8: total bytes; PWLQ_CODES_PACKED and bits <= 4: (total+1)/2 bytes
  *   region_mask  (total+7)/8 bytes; value i is bit (i & 7) of byte (i >> 3); 1 = tail region

@@ -217,6 +217,40 @@ int pwlq_search_ragged(const float* x, const int64_t* row_offsets, int64_t C, in
                        err_out, idx_out, sse_all, workspace, workspace_bytes, stream);
 }
 
+int pwlq_search_partial(const float* x, int64_t C, int64_t n, int bits, const float* ratios,
+                        int K, const float* m, const float* lo, double* sums_out, void* workspace,
+                        size_t workspace_bytes, void* stream) {
+    if (int rc = check_rows(C, n)) return rc;
+    if (!x || !ratios || !m || !sums_out || bits < 2 || bits > 8 || K < 1)
+        return PWLQ_ERR_INVALID_ARG;
+    if (misaligned(x, 4) || misaligned(ratios, 4) || misaligned(m, 4) || misaligned(lo, 4) ||
+        misaligned(sums_out, 8))
+        return PWLQ_ERR_INVALID_ARG;
+    if (K > PWLQ_MAX_K || C * n > kMaxTotal) return PWLQ_ERR_UNSUPPORTED;
+    const pwlq::SearchPlan plan = pwlq::plan_search(C, n, K);
+    if (C * plan.tiles > ((int64_t)1 << 31) - 1 || C * ((K + 31) / 32) > ((int64_t)1 << 31) - 1)
+        return PWLQ_ERR_UNSUPPORTED;
+    if (!workspace || workspace_bytes < plan.bytes) return PWLQ_ERR_WORKSPACE;
+    if (misaligned(workspace, 256)) return PWLQ_ERR_INVALID_ARG;
+    return from_cuda(pwlq::launch_search(x, nullptr, C, n, C * n, bits, ratios, K, m, lo, nullptr,
+                                         nullptr, nullptr, nullptr, workspace, plan,
+                                         as_stream(stream), 0, true, sums_out));
+}
+
+int pwlq_search_finish(const double* sums, int parts, int64_t C, int K, const float* m,
+                       const float* lo, const float* ratios, float* p_out, float* err_out,
+                       int32_t* idx_out, float* sse_all, int32_t* status_out, void* stream) {
+    if (!sums || !m || !ratios || !p_out || !idx_out || parts < 1 || C < 1 || K < 1)
+        return PWLQ_ERR_INVALID_ARG;
+    if (misaligned(sums, 8) || misaligned(m, 4) || misaligned(lo, 4) || misaligned(ratios, 4) ||
+        misaligned(p_out, 4) || misaligned(err_out, 4) || misaligned(idx_out, 4) ||
+        misaligned(sse_all, 4) || misaligned(status_out, 4))
+        return PWLQ_ERR_INVALID_ARG;
+    if (K > PWLQ_MAX_K || C > ((int64_t)1 << 31) - 1) return PWLQ_ERR_UNSUPPORTED;
+    return from_cuda(pwlq::launch_search_finish(sums, parts, C, K, m, lo, ratios, p_out, err_out,
+                                                idx_out, sse_all, status_out, as_stream(stream)));
+}
+
 int pwlq_quantize(const float* x, int64_t C, int64_t n, int bits, const float* m, const float* p,
                   uint8_t* codes, uint8_t* region_mask, float* fake_out, int code_layout,
                   void* stream) {

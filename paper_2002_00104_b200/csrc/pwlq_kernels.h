@@ -36,7 +36,14 @@ cudaError_t launch_search(const float* x, const int64_t* row_offsets, int64_t C,
                           int64_t total, int bits, const float* ratios, int K, const float* m,
                           const float* lo, float* p_out, float* err_out, int32_t* idx_out, float* sse_all,
                           void* workspace, const SearchPlan& plan, cudaStream_t stream,
-                          int64_t shift = 0, bool clear_status = true);
+                          int64_t shift = 0, bool clear_status = true, double* sums64 = nullptr);
+// sums64 != nullptr: only the binary64 per-candidate sums [C][K] are delivered (p_out, err_out,
+// idx_out, sse_all are not touched and may be null).  launch_search_finish adds `parts` such sets
+// ([parts][C][K]) in ascending order and takes the first minimum of every row.
+cudaError_t launch_search_finish(const double* sums, int parts, int64_t C, int K, const float* m,
+                                 const float* lo, const float* ratios, float* p_out, float* err_out,
+                                 int32_t* idx_out, float* sse_all, int* status,
+                                 cudaStream_t stream);
 
 // lo == nullptr: signed scheme with m = abs-max; lo != nullptr: one-sided ranges [lo, m] (m = upper
 // bounds), unsigned b-bit levels.  The same convention holds for launch_dequantize and

@@ -62,6 +62,7 @@ struct SearchArgs {
     float* err_out;
     int32_t* idx_out;
     float* sse_all;
+    double* sums64;     // not null: deliver the binary64 sums [C][K] only (no argmin, no p / err / idx)
     int* status;
 };
 
@@ -117,6 +118,10 @@ __device__ __forceinline__ void block_argmin(const double* sse, int K, double* r
 
 __device__ __forceinline__ void write_degenerate_row(const SearchArgs& a, int64_t row) {
     // m == 0 (or not finite): nothing to search.
+    if (a.sums64) {
+        for (int k = threadIdx.x; k < a.K; k += blockDim.x) a.sums64[row * a.K + k] = 0.0;
+        return;
+    }
     if (threadIdx.x == 0) {
         a.idx_out[row] = 0;
         a.p_out[row] = 0.0f;
@@ -144,12 +149,14 @@ __device__ __forceinline__ void finish_tile(const SearchArgs& a, int64_t row, in
         for (int e = 1; e < E; ++e) tot += part[e * K + k];
         if (a.tiles > 1) {
             a.partials[((size_t)row * a.tiles + tile) * K + k] = tot;
+        } else if (a.sums64) {
+            a.sums64[row * K + k] = tot;
         } else {
             if (E > 1) part[k] = tot;
             if (a.sse_all) a.sse_all[row * K + k] = (float)tot;
         }
     }
-    if (a.tiles > 1) return;
+    if (a.tiles > 1 || a.sums64) return;
     if (E > 1) __syncthreads();                      // E == 1: part[] already holds the sums
     double best; int idx;
     block_argmin(part, K, red_val, red_idx, best, idx);
@@ -648,6 +655,8 @@ __device__ __forceinline__ void tiny_row(const SearchArgs& a, int64_t row, int c
                 const double tot = (double)acc[j];
                 if (a.tiles > 1) {
                     a.partials[((size_t)row * a.tiles) * K + k] = tot;    // tile 0 of the row
+                } else if (a.sums64) {
+                    a.sums64[row * K + k] = tot;
                 } else {
                     if (a.sse_all) a.sse_all[row * K + k] = (float)tot;
                     if (bk == 0x7fffffff || tot < best) { best = tot; bk = k; }   // k ascends
@@ -655,7 +664,7 @@ __device__ __forceinline__ void tiny_row(const SearchArgs& a, int64_t row, int c
             }
         }
     }
-    if (a.tiles > 1) return;                          // the combine kernels finish the row
+    if (a.tiles > 1 || a.sums64) return;              // the combine kernels finish the row
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) {
         const double ov = __shfl_xor_sync(full, best, o);
@@ -684,7 +693,9 @@ search_tiny_kernel(SearchArgs a) {
         // m == 0 (or not finite): nothing to search; with several tiles per row the combine
         // kernels write the row
         if (!finite && lane == 0) atomicOr(a.status, kStatusNonFinite);
-        if (a.tiles == 1) {
+        if (a.tiles == 1 && a.sums64) {
+            for (int k = lane; k < a.K; k += 32) a.sums64[row * a.K + k] = 0.0;
+        } else if (a.tiles == 1) {
             if (lane == 0) {
                 a.idx_out[row] = 0;
                 a.p_out[row] = 0.0f;
@@ -821,7 +832,7 @@ cudaError_t launch_search(const float* x, const int64_t* row_offsets, int64_t C,
                           int64_t total, int bits, const float* ratios, int K, const float* m,
                           const float* lo, float* p_out, float* err_out, int32_t* idx_out,
                           float* sse_all, void* workspace, const SearchPlan& plan,
-                          cudaStream_t stream, int64_t shift, bool clear_status) {
+                          cudaStream_t stream, int64_t shift, bool clear_status, double* sums64) {
     unsigned char* ws = static_cast<unsigned char*>(workspace);
     cudaError_t e = cudaSuccess;
     if (clear_status) e = cudaMemsetAsync(ws, 0, 256, stream);    // status word
@@ -847,6 +858,7 @@ cudaError_t launch_search(const float* x, const int64_t* row_offsets, int64_t C,
     a.err_out = err_out;
     a.idx_out = idx_out;
     a.sse_all = sse_all;
+    a.sums64 = sums64;
     a.status = reinterpret_cast<int*>(ws);
 
     if (K <= kSortMaxK) {
@@ -923,15 +935,72 @@ cudaError_t launch_search(const float* x, const int64_t* row_offsets, int64_t C,
     e = cudaGetLastError();
     if (e != cudaSuccess) return e;
     if (plan.tiles > 1) {
-        double* sums = reinterpret_cast<double*>(ws + plan.off_sums);
+        double* sums = sums64 ? sums64 : reinterpret_cast<double*>(ws + plan.off_sums);
         const int64_t chunks = (K + 31) / 32;
         search_combine_kernel<<<(unsigned)(C * chunks), kCombineWarps * 32, 0, stream>>>(a, sums);
         e = cudaGetLastError();
-        if (e != cudaSuccess) return e;
+        if (e != cudaSuccess || sums64) return e;
         search_argmin_kernel<<<(unsigned)C, kSThreads, 0, stream>>>(a, sums);
         e = cudaGetLastError();
     }
     return e;
+}
+
+// Rows cut across several devices or calls: adds the `parts` sets of per-candidate sums of every
+// row in ascending part order (fixed order: reproducible), then takes the first minimum.
+__global__ void __launch_bounds__(kSThreads)
+search_finish_kernel(const double* __restrict__ sums, int parts, int64_t C, int K,
+                     const float* __restrict__ m_in, const float* __restrict__ lo_in,
+                     const float* __restrict__ ratios, float* __restrict__ p_out,
+                     float* __restrict__ err_out, int32_t* __restrict__ idx_out,
+                     float* __restrict__ sse_all, int* __restrict__ status) {
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    __shared__ double red_val[kSWarps];
+    __shared__ int red_idx[kSWarps];
+    double* tot = reinterpret_cast<double*>(smem_raw);
+    const int64_t row = blockIdx.x;
+    float m = m_in[row];
+    const float lo = lo_in ? lo_in[row] : 0.0f;
+    if (lo_in) m = __fsub_rn(m, lo);
+    const bool finite = (__float_as_uint(m) & 0x7fffffffu) < 0x7f800000u &&
+                        (__float_as_uint(lo) & 0x7fffffffu) < 0x7f800000u;
+    if (!finite || !(m > 0.0f)) {
+        if (!finite && threadIdx.x == 0 && status) atomicOr(status, kStatusNonFinite);
+        if (threadIdx.x == 0) {
+            idx_out[row] = 0;
+            p_out[row] = 0.0f;
+            if (err_out) err_out[row] = 0.0f;
+        }
+        if (sse_all)
+            for (int k = threadIdx.x; k < K; k += blockDim.x) sse_all[row * K + k] = 0.0f;
+        return;
+    }
+    for (int k = threadIdx.x; k < K; k += blockDim.x) {
+        double v = sums[(size_t)row * K + k];
+        for (int part = 1; part < parts; ++part) v += sums[((size_t)part * C + row) * K + k];
+        tot[k] = v;
+        if (sse_all) sse_all[row * K + k] = (float)v;
+    }
+    __syncthreads();
+    double best; int idx;
+    block_argmin(tot, K, red_val, red_idx, best, idx);
+    if (threadIdx.x == 0) {
+        idx_out[row] = idx;
+        p_out[row] = __fmul_rn(m, ratios[idx]);
+        if (err_out) err_out[row] = (float)best;
+    }
+}
+
+cudaError_t launch_search_finish(const double* sums, int parts, int64_t C, int K, const float* m,
+                                 const float* lo, const float* ratios, float* p_out, float* err_out,
+                                 int32_t* idx_out, float* sse_all, int* status,
+                                 cudaStream_t stream) {
+    cudaError_t e = cudaSuccess;
+    if (status) e = cudaMemsetAsync(status, 0, sizeof(int), stream);
+    if (e != cudaSuccess) return e;
+    search_finish_kernel<<<(unsigned)C, kSThreads, sizeof(double) * (size_t)K, stream>>>(
+        sums, parts, C, K, m, lo, ratios, p_out, err_out, idx_out, sse_all, status);
+    return cudaGetLastError();
 }
 
 }  // namespace pwlq

@@ -33,6 +33,8 @@ _SIGNATURES = {
     "pwlq_search": (_INT, [_P, _I64, _I64, _INT, _P, _INT, _P, _P, _P, _P, _P, _P, _SZ, _P]),
     "pwlq_search_ragged": (_INT, [_P, _P, _I64, _I64, _I64, _INT, _P, _INT, _P, _P, _P, _P, _P, _P,
                                   _SZ, _P]),
+    "pwlq_search_partial": (_INT, [_P, _I64, _I64, _INT, _P, _INT, _P, _P, _P, _P, _SZ, _P]),
+    "pwlq_search_finish": (_INT, [_P, _INT, _I64, _INT, _P, _P, _P, _P, _P, _P, _P, _P, _P]),
     "pwlq_quantize": (_INT, [_P, _I64, _I64, _INT, _P, _P, _P, _P, _P, _INT, _P]),
     "pwlq_quantize_ragged": (_INT, [_P, _P, _I64, _I64, _INT, _P, _P, _P, _P, _P, _INT, _P]),
     "pwlq_dequantize": (_INT, [_P, _P, _I64, _I64, _INT, _P, _P, _P, _INT, _P]),
@@ -211,6 +213,47 @@ def search(x, bits, ratios, m=None, row_offsets=None, max_n=None, want_sse=False
     _check(rc, "pwlq_search")
     out = dict(out)
     out["workspace"] = workspace
+    return out
+
+
+def search_partial(x, bits, ratios, m, lo=None, workspace=None, out=None, stream=None):
+    """Binary64 per-candidate sums ``[C, K]`` of one piece ``x`` ``[C, n]`` of rows whose common
+    ranges are ``m`` (see ``pwlq_search_partial``).  Returns (sums, workspace)."""
+    lib = load_library()
+    C, n, _ = _shape(x, None)
+    K = ratios.numel()
+    if workspace is None:
+        workspace = torch.empty(max(search_workspace_bytes(C, n, K), 256), dtype=torch.uint8,
+                                device=x.device)
+    sums = out if out is not None else torch.empty((C, K), dtype=torch.float64, device=x.device)
+    _check(lib.pwlq_search_partial(_dev(x, torch.float32, "x"), C, n, int(bits),
+                                   _dev(ratios, torch.float32, "ratios"), K,
+                                   _dev(m, torch.float32, "m"), _dev(lo, torch.float32, "lo"),
+                                   _dev(sums, torch.float64, "sums"),
+                                   _dev(workspace, torch.uint8, "workspace"), workspace.numel(),
+                                   _stream(stream)), "pwlq_search_partial")
+    return sums, workspace
+
+
+def search_finish(sums, m, ratios, lo=None, want_sse=False, stream=None):
+    """Adds the stacked pieces' sums ``[parts, C, K]`` in order and takes the first minimum of
+    every row.  Returns dict(p, err, idx, sse or None, status)."""
+    lib = load_library()
+    parts, C, K = sums.shape
+    out = {"p": torch.empty(C, dtype=torch.float32, device=sums.device),
+           "err": torch.empty(C, dtype=torch.float32, device=sums.device),
+           "idx": torch.empty(C, dtype=torch.int32, device=sums.device),
+           "sse": torch.empty((C, K), dtype=torch.float32, device=sums.device) if want_sse else None,
+           "status": torch.zeros(1, dtype=torch.int32, device=sums.device)}
+    _check(lib.pwlq_search_finish(_dev(sums, torch.float64, "sums"), int(parts), C, K,
+                                  _dev(m, torch.float32, "m"), _dev(lo, torch.float32, "lo"),
+                                  _dev(ratios, torch.float32, "ratios"),
+                                  _dev(out["p"], torch.float32, "p"),
+                                  _dev(out["err"], torch.float32, "err"),
+                                  _dev(out["idx"], torch.int32, "idx"),
+                                  _dev(out["sse"], torch.float32, "sse"),
+                                  _dev(out["status"], torch.int32, "status"), _stream(stream)),
+           "pwlq_search_finish")
     return out
 
 

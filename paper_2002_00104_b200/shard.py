@@ -40,3 +40,40 @@ def gather_rows(local: dict, ranges, dist, rank: int, world_size: int):
     out = [None] * world_size
     dist.all_gather_object(out, {k: np.asarray(v) for k, v in local.items()})
     return {k: np.concatenate([out[r][k] for r in range(world_size)]) for k in local}
+
+
+# ---------------------------------------------------------------------------- one row, many ranks
+# A tensor quantized per layer is ONE row; it does not shard by rows.  Its elements are cut into
+# contiguous slices instead.  The range needs one exchange (maximum of the ranks' abs-max values),
+# the search a second one (the ranks' per-candidate sums, K binary64 values per row, added in rank
+# order so that every rank gets the same bits), after which every rank takes the same argmin.
+# Quantize and dequantize are element-wise and need nothing.  The functions below are the two
+# exchanges; the arithmetic between them is the library's (pwlq_absmax, pwlq_search_partial,
+# pwlq_search_finish).
+
+def partition_elements(n: int, world_size: int, align: int = 8):
+    """Contiguous element ranges [(b, e)] * world_size of a row of n values, cut at multiples of
+    `align` (so that every slice keeps the vector and byte alignment of codes and region bits)."""
+    cuts = [0]
+    for k in range(1, world_size):
+        c = (n * k // world_size) // align * align
+        cuts.append(min(max(c, cuts[-1]), n))
+    cuts.append(n)
+    return [(cuts[k], cuts[k + 1]) for k in range(world_size)]
+
+
+def allreduce_range(m_local, dist, group=None):
+    """Range of the whole rows from the ranks' ranges of their slices: element-wise maximum
+    (exact and order-free).  m_local: float32 tensor [C] on the backend's device; in place."""
+    dist.all_reduce(m_local, op=dist.ReduceOp.MAX, group=group)
+    return m_local
+
+
+def gather_partial_sums(sums_local, dist, world_size: int, group=None):
+    """All ranks' per-candidate sums stacked in rank order, [world_size, C, K] binary64 -- the
+    layout pwlq_search_finish adds up in a fixed order.  (An all-reduce would leave the order of
+    the additions to the backend; K doubles per row make the gather just as cheap.)"""
+    import torch
+    parts = [torch.empty_like(sums_local) for _ in range(world_size)]
+    dist.all_gather(parts, sums_local.contiguous(), group=group)
+    return torch.stack(parts, dim=0)
