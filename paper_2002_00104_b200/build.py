@@ -8,6 +8,8 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libpwlq.so")
+PEAK_LIB = os.path.join(HERE, "libpwlq_peak.so")     # FP32 micro-benchmark, loaded by bench.py only
+PEAK_SOURCES = ["fp32_peak.cu"]
 SOURCES = ["pwlq_api.cu", "pwlq_absmax.cu", "pwlq_search.cu", "pwlq_quantize.cu",
            "pwlq_noalloc.cu", "pwlq_select.cu", "pwlq_search2.cu", "pwlq_bias.cu"]
 NVCC_FLAGS = [
@@ -17,26 +19,32 @@ NVCC_FLAGS = [
 ]
 
 
-def _stale() -> bool:
-    if not os.path.exists(LIB):
+def _stale(lib: str) -> bool:
+    if not os.path.exists(lib):
         return True
-    t = os.path.getmtime(LIB)
+    t = os.path.getmtime(lib)
     deps = [os.path.join(CSRC, f) for f in os.listdir(CSRC)]
     deps += [os.path.join(HERE, "..", "include", "pwlq.h"), os.path.abspath(__file__)]
     return any(os.path.getmtime(d) > t for d in deps)
 
 
-def build(force: bool = False, verbose: bool = False) -> str:
-    if not force and not _stale():
-        return LIB
+def _nvcc(sources, lib: str, verbose: bool) -> None:
     nvcc = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
     cmd = [nvcc] + NVCC_FLAGS + (["-Xptxas", "-v"] if verbose else []) + \
-          [os.path.join(CSRC, s) for s in SOURCES] + ["-o", LIB]
+          [os.path.join(CSRC, s) for s in sources] + ["-o", lib]
     res = subprocess.run(cmd, capture_output=True, text=True)
     if res.returncode != 0:
         raise RuntimeError("nvcc failed:\n" + res.stdout + res.stderr)
     if verbose:
         print(res.stderr)
+
+
+def build(force: bool = False, verbose: bool = False) -> str:
+    """Compiles the library (and the benchmark's FP32 micro-benchmark) if a source is newer."""
+    if force or _stale(LIB):
+        _nvcc(SOURCES, LIB, verbose)
+    if force or _stale(PEAK_LIB):
+        _nvcc(PEAK_SOURCES, PEAK_LIB, verbose)
     return LIB
 
 
