@@ -455,6 +455,85 @@ class DevicePath:
         return 1 + int(self.unsigned) + classes + (2 if tiled else 0) + 2
 
 
+def timed_call(torch, fn, flush, reps=5):
+    """Median ms of single cold launches (L2 evicted before each)."""
+    ts = []
+    st = torch.cuda.current_stream()
+    for _ in range(reps + 2):
+        flush.fill_(1)
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record(st); fn(); b.record(st)
+        torch.cuda.synchronize()
+        ts.append(a.elapsed_time(b))
+    return float(np.median(ts[2:]))
+
+
+def extras(torch, pwlq, path: DevicePath, flush, hbm, K2=32):
+    """The calls beyond the four-call path, on the headline workload's rows (single cold launches):
+    two-breakpoint pair search with its quantize / dequantize, analytic selection, bias correction
+    with the corrected dequantize, dense (b+1)-bit stream; and the streaming kernels on dense rows
+    of 147 values (row starts off every vector boundary)."""
+    w, x, ro, m, bits = path.w, path.x, path.ro, path.m, path.bits
+    kw = dict(row_offsets=ro)
+    r2 = torch.from_numpy(W.ratio_grid(K2)).to(path.dev)
+    out = {}
+    ws2 = None
+    try:
+        s2 = pwlq.search2(x, bits, r2, m, max_n=path.max_n, **kw)
+        ws2 = s2["workspace"]
+        pairs = K2 * (K2 - 1) // 2
+        t = timed_call(torch, lambda: pwlq.search2(x, bits, r2, m, max_n=path.max_n, workspace=ws2,
+                                                   **kw), flush)
+        one = pwlq.search(x, bits, r2, m=m, max_n=path.max_n, **kw)
+        gain = float((one["err"].double().sum() / s2["err"].double().sum()).item())
+        out["search2"] = {"K": K2, "pairs": pairs, "ms": t,
+                          "t_value_pairs_per_s": w.total * pairs / (t * 1e-3) / 1e12,
+                          "sse_one_over_two_breakpoints": gain}
+        codes, region, _ = pwlq.quantize2(x, bits, m, s2["p1"], s2["p2"], layout=1, **kw)
+        nb = w.total * 4 + codes.numel() + region.numel()
+        t = timed_call(torch, lambda: pwlq.quantize2(x, bits, m, s2["p1"], s2["p2"], layout=1,
+                                                     out=(codes, region, None), **kw), flush)
+        out["quantize2"] = {"ms": t, "hbm_cold_frac": nb / (t * 1e-3) / 1e9 / hbm}
+        y = path.y
+        t = timed_call(torch, lambda: pwlq.dequantize2(codes, region, bits, m, s2["p1"], s2["p2"],
+                                                       C=w.C, n=path.dense_n, layout=1, out=y, **kw),
+                       flush)
+        out["dequantize2"] = {"ms": t, "hbm_cold_frac": nb / (t * 1e-3) / 1e9 / hbm}
+    except pwlq.PwlqError as e:                   # e.g. rows beyond the pair search's limit
+        out["search2"] = {"skipped": str(e)}
+    p = path.sout["p"]
+    t = timed_call(torch, lambda: pwlq.select_analytic(x, m, pwlq.MODEL_GAUSS_ROOT,
+                                                       max_n=path.max_n, **kw), flush)
+    out["select_analytic"] = {"ms": t, "hbm_cold_frac": w.total * 4 / (t * 1e-3) / 1e9 / hbm}
+    t = timed_call(torch, lambda: pwlq.bias_correction(x, bits, m, p, max_n=path.max_n, **kw), flush)
+    out["bias_correction"] = {"ms": t, "hbm_cold_frac": w.total * 4 / (t * 1e-3) / 1e9 / hbm}
+    xi, beta = pwlq.bias_correction(x, bits, m, p, max_n=path.max_n, **kw)
+    c8, k8, _ = pwlq.quantize(x, bits, m, p, layout=0, **kw)
+    b8 = w.total * 4 + c8.numel() + k8.numel()
+    t = timed_call(torch, lambda: pwlq.dequantize_bc(c8, k8, bits, m, p, xi, beta, C=w.C,
+                                                     n=path.dense_n, out=path.y, **kw), flush)
+    out["dequantize_bc"] = {"ms": t, "hbm_cold_frac": b8 / (t * 1e-3) / 1e9 / hbm}
+    dense = pwlq.pack_dense(c8, k8, bits)
+    bp = c8.numel() + k8.numel() + dense.numel()
+    t = timed_call(torch, lambda: pwlq.pack_dense(c8, k8, bits, out=dense), flush)
+    out["pack_dense"] = {"ms": t, "hbm_cold_frac": bp / (t * 1e-3) / 1e9 / hbm}
+    t = timed_call(torch, lambda: pwlq.unpack_dense(dense, w.total, bits), flush)
+    out["unpack_dense"] = {"ms": t, "hbm_cold_frac": bp / (t * 1e-3) / 1e9 / hbm}
+    del c8, k8, dense
+    # streaming kernels on dense rows of 147 values, 512 MB
+    n147 = (1 << 27) // 147
+    rng = np.random.default_rng(147)
+    w147 = W.Workload("dense_rows_of_147", (rng.standard_normal(n147 * 147) * 0.02).astype(np.float32),
+                      np.arange(n147 + 1, dtype=np.int64) * 147, 4, 16)
+    p147 = DevicePath(torch, pwlq, w147, path.dev)
+    pwlq.absmax(p147.x, out=p147.m)
+    p147.sout["p"].copy_(p147.m * 0.3)
+    s = p147.streaming(reps=5)
+    out["hbm_streaming_frac_rows_of_147"] = {k: s[k]["gbs"] / hbm for k in
+                                             ("absmax", "quantize", "quantize_fused", "dequantize")}
+    return out
+
+
 def summarize(path: DevicePath, stage_ms, hbm, peak_measured, issued=None):
     """Per-workload figures from stage times [steps, 4]."""
     mean = stage_ms.mean(axis=0)
@@ -504,6 +583,17 @@ def run_ours(args, rank, world, local_rank):
 
     w = make_workload(args, None if world == 1 else 1000 + 17 * rank)
     path = DevicePath(torch, pwlq, w, dev, args.scheme)
+    if args.leg == "streaming":
+        # only the HBM-bound kernels back to back (a small case for a profiler: few launches)
+        pwlq.absmax(path.x, row_offsets=path.ro, out=path.m)
+        path.sout["p"].copy_(path.m * 0.3)
+        s = path.streaming(reps=args.reps)
+        s["workload"] = w.name
+        for k in ("absmax", "quantize", "quantize_fused", "dequantize"):
+            s[k]["frac"] = s[k]["gbs"] / hbm
+        s["device_status"] = pwlq.device_status()
+        print(json.dumps({"leg": "streaming", "hbm_streaming": s}), flush=True)
+        return
     unsigned = path.unsigned
     flush = torch.empty(L2_FLUSH_BYTES, dtype=torch.uint8, device=dev)
     warmup = max(3, args.warmup)
@@ -555,7 +645,7 @@ def run_ours(args, rank, world, local_rank):
     del scratch
 
     # ---- rank 0, one GPU: the side measurements
-    streaming = sustained = others = None
+    streaming = sustained = others = extra = None
     peak_measured = peak_detail = None
     if rank == 0 and world == 1 and not args.quick:
         fp = FP32Peak()
@@ -578,6 +668,8 @@ def run_ours(args, rank, world, local_rank):
                      "search_frac_at_sampled_clock":
                          LANE_OPS_PER_ELEM_CAND * sus_search /
                          (SM_COUNT * FP32_LANES_PER_SM * mhz * 1e6)}
+        if not unsigned:
+            extra = extras(torch, pwlq, path, flush, hbm)
         # the other benchmark configurations
         if args.workload == "resnet50" and not (args.bits or args.K) and not unsigned:
             others = {}
@@ -671,6 +763,8 @@ def run_ours(args, rank, world, local_rank):
             line["sustained"] = sustained
         if others is not None:
             line["workloads"] = others
+        if extra is not None:
+            line["extras"] = extra
         if unsigned:
             line["e2e"]["scheme"] = "signed (the host-buffer entry point has no one-sided form)"
         if world == 1 and not args.no_cpu_baseline and not unsigned:
@@ -689,6 +783,10 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="resnet50", choices=sorted(WORKLOADS))
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--leg", default="all", choices=["all", "streaming"],
+                    help="streaming: only the three HBM-bound kernels back to back on the "
+                         "workload's rows repeated beyond L2 (--reps launches each after 3 warm-ups)")
+    ap.add_argument("--reps", type=int, default=10)
     ap.add_argument("--quick", action="store_true",
                     help="only the timed steps and the end-to-end leg (no micro-benchmark, "
                          "streaming, sustained or other-workload legs)")
