@@ -184,7 +184,13 @@ __device__ __forceinline__ void quantize8(const float (&xv)[8], int split, float
 // span and walks it in passes of 256 values, a lane owns eight consecutive values of a pass.
 constexpr int kMapConsumers = 8;
 constexpr int kMapThreads = (kMapConsumers + 1) * 32;
-constexpr int kMapStages = 2;
+#ifndef PWLQ_MAP_STAGES
+#define PWLQ_MAP_STAGES 2
+#endif
+#ifndef PWLQ_Q_MINBLOCKS
+#define PWLQ_Q_MINBLOCKS 4
+#endif
+constexpr int kMapStages = PWLQ_MAP_STAGES;
 static_assert(kMapStages <= 4, "MapProducer tracks at most four stages");
 
 template <bool DATA, bool QB>
@@ -201,8 +207,164 @@ __device__ __forceinline__ PieceParams params_of(const float4 qa, const float4 q
     return P;
 }
 
+// What a consumer's pass needs besides the stage.
+template <bool UNS>
+struct QuantizeCtx {
+    Rows rows;
+    RowArrays A;
+    int64_t total;
+    int bits, Li;
+    float Lf;
+    uint32_t sign_unit;
+    int sign_shift;
+    uint8_t* __restrict__ codes;
+    uint8_t* __restrict__ mask;
+    float* __restrict__ fake;
+    int vec_fake, vec_codes;
+};
+
+// One pass of a consumer lane: the eight values at offset li of the span that begins at flat
+// index span_beg.  FULL: the span is complete, its map is usable and every output can be stored
+// with vector stores (the common case: no value counts, no 64-bit indices, no byte-wise stores).
+template <bool PACKED, bool WANT_FAKE, bool UNS, bool QB, bool FULL>
+__device__ __forceinline__ void quantize_pass(const QuantizeCtx<UNS>& g, const float* data,
+                                              const SpanRowMap& M, const float4* qa,
+                                              const float4* qb, int64_t span_beg, int li) {
+    const unsigned full = 0xffffffffu;
+    const int64_t i0 = span_beg + li;
+    const int cnt = FULL ? 8 : (int)max((int64_t)0, min((int64_t)8, g.total - i0));
+    const float4 xa = *reinterpret_cast<const float4*>(data + li);
+    const float4 xb = *reinterpret_cast<const float4*>(data + li + 4);
+    const float xv[8] = {xa.x, xa.y, xa.z, xa.w, xb.x, xb.y, xb.z, xb.w};
+    uint32_t w0 = 0, w1 = 0, mb = 0;
+    float yv[8];
+    if (FULL || M.slow == 0) {
+        uint32_t word;
+        const int l = map_slot(M, li, word);
+        const uint32_t inner = (word >> ((li & 31) + 1)) & 0x7Fu;   // starts at li+1 .. li+7
+        const float4 ca = qa[l];
+        const float4 cb = QB ? qb[l] : make_float4(0.0f, 0.0f, 0.0f, 0.0f);
+        const bool simple = inner == 0 && ca.x > 0.0f && cnt == 8;
+        if (__all_sync(full, simple)) {
+            const PieceParams P = params_of(ca, cb);
+            quantize8<PACKED, WANT_FAKE, false, UNS>(xv, 8, ca.x, cb.z, P, ca.x, cb.z, P, g.Lf, g.Li,
+                                                     g.sign_unit, g.sign_shift, w0, w1, mb, yv);
+        } else {
+            const bool one = inner != 0 && (inner & (inner - 1)) == 0 && ca.x > 0.0f && cnt == 8;
+            float4 da = ca, db = cb;
+            int split = 8;
+            if (one) {
+                da = qa[l + 1];
+                if (QB) db = qb[l + 1];
+                split = __ffs(inner);
+            }
+            if (__all_sync(full, simple || (one && da.x > 0.0f))) {
+                quantize8<PACKED, WANT_FAKE, true, UNS>(xv, split, ca.x, cb.z, params_of(ca, cb), da.x,
+                                                        db.z, params_of(da, db), g.Lf, g.Li, g.sign_unit,
+                                                        g.sign_shift, w0, w1, mb, yv);
+            } else {
+#pragma unroll
+                for (int t = 0; t < 8; ++t) {
+                    yv[t] = 0.0f;
+                    if (t < cnt) {
+                        const int lt = l + __popc(inner & ((1u << t) - 1u));
+                        const float4 ea = qa[lt];
+                        const float4 eb = QB ? qb[lt] : make_float4(0.0f, 0.0f, 0.0f, 0.0f);
+                        if (UNS) yv[t] = eb.z;                 // a constant row delivers lo
+                        const float em = fabsf(ea.x);          // (-m marks a row kept off the fast paths)
+                        if (em > 0.0f) {
+                            const float xi = xv[t];
+                            const int neg = !UNS && xi < 0.0f;
+                            int q, tail;
+                            float v;
+                            const float a = UNS ? fminf(fmaxf(__fsub_rn(xi, eb.z), 0.0f), em)
+                                                : fminf(fabsf(xi), em);
+                            quantize_mag(a, params_of(ea, eb), g.Lf, q, tail, v);
+                            const uint32_t code = (uint32_t)((neg << (g.bits - 1)) | q);
+                            if (PACKED) w0 |= code << (4 * t);
+                            else if (t < 4) w0 |= code << (8 * t);
+                            else w1 |= code << (8 * (t - 4));
+                            mb |= (uint32_t)tail << t;
+                            yv[t] = UNS ? __fadd_rn(v, eb.z) : (neg ? -v : v);
+                        }
+                    }
+                }
+            }
+        }
+    } else {
+        RowState rs;
+#pragma unroll
+        for (int t = 0; t < 8; ++t) {
+            yv[t] = 0.0f;
+            if (t < cnt) {
+                rs.seek(g.rows, g.A, g.Lf, i0 + t);
+                if (UNS) yv[t] = rs.lo;
+                if (rs.m > 0.0f) {
+                    const float xi = xv[t];
+                    const int neg = !UNS && xi < 0.0f;
+                    int q, tail;
+                    float v;
+                    const float a = UNS ? fminf(fmaxf(__fsub_rn(xi, rs.lo), 0.0f), rs.m)
+                                        : fminf(fabsf(xi), rs.m);
+                    quantize_mag(a, rs.P, g.Lf, q, tail, v);
+                    const uint32_t code = (uint32_t)((neg << (g.bits - 1)) | q);
+                    if (PACKED) w0 |= code << (4 * t);
+                    else if (t < 4) w0 |= code << (8 * t);
+                    else w1 |= code << (8 * (t - 4));
+                    mb |= (uint32_t)tail << t;
+                    yv[t] = UNS ? __fadd_rn(v, rs.lo) : (neg ? -v : v);
+                }
+            }
+        }
+    }
+    if (FULL) {
+        // span_beg is a multiple of the span: the span's slices of the outputs start at
+        // multiples of 512 / 2048 / 4096 bytes, so 32-bit offsets inside them suffice
+        uint8_t* mask_s = g.mask + (span_beg >> 3);
+        mask_s[li >> 3] = (uint8_t)mb;
+        if (PACKED) {
+            reinterpret_cast<uint32_t*>(g.codes + (span_beg >> 1))[li >> 3] = w0;
+        } else {
+            reinterpret_cast<uint2*>(g.codes + span_beg)[li >> 3] = make_uint2(w0, w1);
+        }
+        if (WANT_FAKE) {
+            float4* f = reinterpret_cast<float4*>(g.fake + span_beg) + (li >> 2);
+            __stcs(f, make_float4(yv[0], yv[1], yv[2], yv[3]));
+            __stcs(f + 1, make_float4(yv[4], yv[5], yv[6], yv[7]));
+        }
+        return;
+    }
+    if (cnt == 0) return;
+    g.mask[i0 >> 3] = (uint8_t)mb;
+    if (PACKED) {
+        uint8_t* dst = g.codes + (i0 >> 1);
+        if (g.vec_codes && cnt == 8) {
+            *reinterpret_cast<uint32_t*>(dst) = w0;
+        } else {
+            const int nb = (cnt + 1) >> 1;
+            for (int b = 0; b < nb; ++b) dst[b] = (uint8_t)(w0 >> (8 * b));
+        }
+    } else {
+        uint8_t* dst = g.codes + i0;
+        if (g.vec_codes && cnt == 8) {
+            *reinterpret_cast<uint2*>(dst) = make_uint2(w0, w1);
+        } else {
+            for (int t = 0; t < cnt; ++t)
+                dst[t] = (uint8_t)((t < 4 ? w0 : w1) >> (8 * (t & 3)));
+        }
+    }
+    if (WANT_FAKE) {
+        if (g.vec_fake && cnt == 8) {
+            __stcs(reinterpret_cast<float4*>(g.fake + i0), make_float4(yv[0], yv[1], yv[2], yv[3]));
+            __stcs(reinterpret_cast<float4*>(g.fake + i0 + 4), make_float4(yv[4], yv[5], yv[6], yv[7]));
+        } else {
+            for (int t = 0; t < cnt; ++t) g.fake[i0 + t] = yv[t];
+        }
+    }
+}
+
 template <bool PACKED, bool WANT_FAKE, bool UNS, bool LONG>
-__global__ void __launch_bounds__(kMapThreads, (WANT_FAKE || UNS) ? 3 : 4)
+__global__ void __launch_bounds__(kMapThreads, (WANT_FAKE || UNS) ? (PWLQ_Q_MINBLOCKS > 3 ? 3 : PWLQ_Q_MINBLOCKS) : PWLQ_Q_MINBLOCKS)
 quantize_map_kernel(const float* __restrict__ x, Rows rows, int64_t total, int bits, RowArrays A,
                     uint8_t* __restrict__ codes, uint8_t* __restrict__ mask,
                     float* __restrict__ fake, int vec_in, int vec_fake, int vec_codes,
@@ -287,6 +449,10 @@ quantize_map_kernel(const float* __restrict__ x, Rows rows, int64_t total, int b
     }
 
     // ---- consumers
+    QuantizeCtx<UNS> ctx{rows, A, total, bits, Li, Lf, sign_unit, sign_shift, codes, mask, fake,
+                         vec_fake, vec_codes};
+    const int li0 = warp * (kMapSpan / kMapConsumers) + lane * 8;     // pass c: li0 + 256 c
+    const bool vec_all = vec_codes && (!WANT_FAKE || vec_fake);
     int64_t it = 0;
     for (int64_t span = first; span < last; ++span, ++it) {
         const int s = (int)(it % kMapStages);
@@ -297,123 +463,18 @@ quantize_map_kernel(const float* __restrict__ x, Rows rows, int64_t total, int b
         }
         const int64_t span_beg = span * kMapSpan;
         const Stage& S = st[s];
-        const bool slow = S.map.slow != 0;
+        // a whole span with a usable map and vector-aligned outputs: no counts, no 64-bit
+        // indices, no byte-wise stores in the passes
+        if (S.map.slow == 0 && span_beg + kMapSpan <= total && vec_all) {
+#pragma unroll
+            for (int c = 0; c < 2; ++c)
+                quantize_pass<PACKED, WANT_FAKE, UNS, QB, true>(ctx, S.data, S.map, S.qa, S.qb,
+                                                                span_beg, li0 + c * 256);
+        } else {
 #pragma unroll 1
-        for (int c = 0; c < 2; ++c) {
-            const int li = warp * (kMapSpan / kMapConsumers) + c * 256 + lane * 8;
-            const int64_t i0 = span_beg + li;
-            const int cnt = (int)max((int64_t)0, min((int64_t)8, total - i0));
-            const float4 xa = *reinterpret_cast<const float4*>(S.data + li);
-            const float4 xb = *reinterpret_cast<const float4*>(S.data + li + 4);
-            const float xv[8] = {xa.x, xa.y, xa.z, xa.w, xb.x, xb.y, xb.z, xb.w};
-            uint32_t w0 = 0, w1 = 0, mb = 0;
-            float yv[8];
-            if (!slow) {
-                uint32_t word;
-                const int l = map_slot(S.map, li, word);
-                const uint32_t inner = (word >> ((li & 31) + 1)) & 0x7Fu;   // starts at li+1 .. li+7
-                const float4 ca = S.qa[l];
-                const float4 cb = QB ? S.qb[l] : make_float4(0.0f, 0.0f, 0.0f, 0.0f);
-                const bool simple = inner == 0 && ca.x > 0.0f && cnt == 8;
-                if (__all_sync(full, simple)) {
-                    const PieceParams P = params_of(ca, cb);
-                    quantize8<PACKED, WANT_FAKE, false, UNS>(xv, 8, ca.x, cb.z, P, ca.x, cb.z, P, Lf,
-                                                             Li, sign_unit, sign_shift, w0, w1, mb, yv);
-                } else {
-                    const bool one = inner != 0 && (inner & (inner - 1)) == 0 && ca.x > 0.0f && cnt == 8;
-                    float4 da = ca, db = cb;
-                    int split = 8;
-                    if (one) {
-                        da = S.qa[l + 1];
-                        if (QB) db = S.qb[l + 1];
-                        split = __ffs(inner);
-                    }
-                    if (__all_sync(full, simple || (one && da.x > 0.0f))) {
-                        quantize8<PACKED, WANT_FAKE, true, UNS>(xv, split, ca.x, cb.z, params_of(ca, cb),
-                                                                da.x, db.z, params_of(da, db), Lf, Li,
-                                                                sign_unit, sign_shift, w0, w1, mb, yv);
-                    } else {
-#pragma unroll
-                        for (int t = 0; t < 8; ++t) {
-                            yv[t] = 0.0f;
-                            if (t < cnt) {
-                                const int lt = l + __popc(inner & ((1u << t) - 1u));
-                                const float4 ea = S.qa[lt];
-                                const float4 eb = QB ? S.qb[lt] : make_float4(0.0f, 0.0f, 0.0f, 0.0f);
-                                if (UNS) yv[t] = eb.z;                 // a constant row delivers lo
-                                const float em = fabsf(ea.x);          // (-m marks a row kept off the fast paths)
-                                if (em > 0.0f) {
-                                    const float xi = xv[t];
-                                    const int neg = !UNS && xi < 0.0f;
-                                    int q, tail;
-                                    float v;
-                                    const float a = UNS ? fminf(fmaxf(__fsub_rn(xi, eb.z), 0.0f), em)
-                                                        : fminf(fabsf(xi), em);
-                                    quantize_mag(a, params_of(ea, eb), Lf, q, tail, v);
-                                    const uint32_t code = (uint32_t)((neg << (bits - 1)) | q);
-                                    if (PACKED) w0 |= code << (4 * t);
-                                    else if (t < 4) w0 |= code << (8 * t);
-                                    else w1 |= code << (8 * (t - 4));
-                                    mb |= (uint32_t)tail << t;
-                                    yv[t] = UNS ? __fadd_rn(v, eb.z) : (neg ? -v : v);
-                                }
-                            }
-                        }
-                    }
-                }
-            } else {
-                RowState rs;
-#pragma unroll
-                for (int t = 0; t < 8; ++t) {
-                    yv[t] = 0.0f;
-                    if (t < cnt) {
-                        rs.seek(rows, A, Lf, i0 + t);
-                        if (UNS) yv[t] = rs.lo;
-                        if (rs.m > 0.0f) {
-                            const float xi = xv[t];
-                            const int neg = !UNS && xi < 0.0f;
-                            int q, tail;
-                            float v;
-                            const float a = UNS ? fminf(fmaxf(__fsub_rn(xi, rs.lo), 0.0f), rs.m)
-                                                : fminf(fabsf(xi), rs.m);
-                            quantize_mag(a, rs.P, Lf, q, tail, v);
-                            const uint32_t code = (uint32_t)((neg << (bits - 1)) | q);
-                            if (PACKED) w0 |= code << (4 * t);
-                            else if (t < 4) w0 |= code << (8 * t);
-                            else w1 |= code << (8 * (t - 4));
-                            mb |= (uint32_t)tail << t;
-                            yv[t] = UNS ? __fadd_rn(v, rs.lo) : (neg ? -v : v);
-                        }
-                    }
-                }
-            }
-            if (cnt == 0) continue;
-            mask[i0 >> 3] = (uint8_t)mb;
-            if (PACKED) {
-                uint8_t* dst = codes + (i0 >> 1);
-                if (vec_codes && cnt == 8) {
-                    *reinterpret_cast<uint32_t*>(dst) = w0;
-                } else {
-                    const int nb = (cnt + 1) >> 1;
-                    for (int b = 0; b < nb; ++b) dst[b] = (uint8_t)(w0 >> (8 * b));
-                }
-            } else {
-                uint8_t* dst = codes + i0;
-                if (vec_codes && cnt == 8) {
-                    *reinterpret_cast<uint2*>(dst) = make_uint2(w0, w1);
-                } else {
-                    for (int t = 0; t < cnt; ++t)
-                        dst[t] = (uint8_t)((t < 4 ? w0 : w1) >> (8 * (t & 3)));
-                }
-            }
-            if (WANT_FAKE) {
-                if (vec_fake && cnt == 8) {
-                    __stcs(reinterpret_cast<float4*>(fake + i0), make_float4(yv[0], yv[1], yv[2], yv[3]));
-                    __stcs(reinterpret_cast<float4*>(fake + i0 + 4), make_float4(yv[4], yv[5], yv[6], yv[7]));
-                } else {
-                    for (int t = 0; t < cnt; ++t) fake[i0 + t] = yv[t];
-                }
-            }
+            for (int c = 0; c < 2; ++c)
+                quantize_pass<PACKED, WANT_FAKE, UNS, QB, false>(ctx, S.data, S.map, S.qa, S.qb,
+                                                                 span_beg, li0 + c * 256);
         }
         __syncwarp();
         if (lane == 0) mbar_arrive(&empty_bar[s]);
@@ -588,7 +649,7 @@ dequantize_long_kernel(const uint8_t* __restrict__ codes, const uint8_t* __restr
 // of the next span into registers before they wait for the current span's map.
 // BC: the bias-corrected value xi * y + beta (one multiply, one add) instead of y.
 template <bool PACKED, bool UNS, bool LONG, bool BC>
-__global__ void __launch_bounds__(kMapThreads, 4)
+__global__ void __launch_bounds__(kMapThreads, PWLQ_Q_MINBLOCKS)
 dequantize_map_kernel(const uint8_t* __restrict__ codes, const uint8_t* __restrict__ mask, Rows rows,
                       int64_t total, int bits, RowArrays A, float* __restrict__ y, int vec_codes,
                       int vec_out, int64_t spans_per_cta) {
