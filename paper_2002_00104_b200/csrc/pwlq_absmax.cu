@@ -16,10 +16,7 @@ namespace pwlq {
 
 constexpr int kAbsConsumers = 8;                         // folding warps per CTA
 constexpr int kAbsThreads = (kAbsConsumers + 1) * 32;    // + the producer warp
-#ifndef PWLQ_ABS_STAGES
-#define PWLQ_ABS_STAGES 2
-#endif
-constexpr int kAbsStages = PWLQ_ABS_STAGES;                            // spans in flight per CTA
+constexpr int kAbsStages = 2;                            // spans in flight per CTA
 static_assert(kAbsStages <= 4, "MapProducer tracks at most four stages");
 
 static __device__ int g_absmax_timeout;                  // set when a bounded wait expired

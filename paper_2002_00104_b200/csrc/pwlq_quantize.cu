@@ -184,13 +184,7 @@ __device__ __forceinline__ void quantize8(const float (&xv)[8], int split, float
 // span and walks it in passes of 256 values, a lane owns eight consecutive values of a pass.
 constexpr int kMapConsumers = 8;
 constexpr int kMapThreads = (kMapConsumers + 1) * 32;
-#ifndef PWLQ_MAP_STAGES
-#define PWLQ_MAP_STAGES 2
-#endif
-#ifndef PWLQ_Q_MINBLOCKS
-#define PWLQ_Q_MINBLOCKS 4
-#endif
-constexpr int kMapStages = PWLQ_MAP_STAGES;
+constexpr int kMapStages = 2;
 static_assert(kMapStages <= 4, "MapProducer tracks at most four stages");
 
 template <bool DATA, bool QB>
@@ -364,7 +358,7 @@ __device__ __forceinline__ void quantize_pass(const QuantizeCtx<UNS>& g, const f
 }
 
 template <bool PACKED, bool WANT_FAKE, bool UNS, bool LONG>
-__global__ void __launch_bounds__(kMapThreads, (WANT_FAKE || UNS) ? (PWLQ_Q_MINBLOCKS > 3 ? 3 : PWLQ_Q_MINBLOCKS) : PWLQ_Q_MINBLOCKS)
+__global__ void __launch_bounds__(kMapThreads, (WANT_FAKE || UNS) ? 3 : 4)
 quantize_map_kernel(const float* __restrict__ x, Rows rows, int64_t total, int bits, RowArrays A,
                     uint8_t* __restrict__ codes, uint8_t* __restrict__ mask,
                     float* __restrict__ fake, int vec_in, int vec_fake, int vec_codes,
@@ -644,12 +638,157 @@ dequantize_long_kernel(const uint8_t* __restrict__ codes, const uint8_t* __restr
 }
 
 // ------------------------------------------------------------------ several rows per span
+// What a consumer's pass of the inverse needs besides the stage.
+struct DequantizeCtx {
+    Rows rows;
+    RowArrays A;
+    int64_t total;
+    int bits, qmask, sign_shift;
+    float Lf;
+    float* __restrict__ y;
+    int vec_out;
+};
+
+// One pass of a consumer lane of the inverse: the eight codes (w0, w1) and region bits (mb) at
+// offset li of the span that begins at flat index span_beg.  FULL: the span is complete, its map
+// is usable and y can be stored with vector stores (no value counts, no 64-bit indices).
+template <bool PACKED, bool UNS, bool BC, bool FULL>
+__device__ __forceinline__ void dequantize_pass(const DequantizeCtx& g, uint32_t w0, uint32_t w1,
+                                                uint32_t mb, const SpanRowMap& M, const float4* qa,
+                                                const float4* qb, int64_t span_beg, int li) {
+    constexpr bool QB = UNS || BC;
+    const unsigned full = 0xffffffffu;
+    const int64_t i0 = span_beg + li;
+    const int cnt = FULL ? 8 : (int)max((int64_t)0, min((int64_t)8, g.total - i0));
+    float yv[8];
+    if (FULL || M.slow == 0) {
+        uint32_t word;
+        const int l = map_slot(M, li, word);
+        const uint32_t inner = (word >> ((li & 31) + 1)) & 0x7Fu;   // starts at li+1 .. li+7
+        const float4 ca = qa[l];
+        const float4 ba = QB ? qb[l] : make_float4(0.0f, 1.0f, 0.0f, 0.0f);
+        const float loA = UNS ? ba.x : 0.0f;
+        const bool simple = inner == 0 && ca.x > 0.0f && cnt == 8;
+        PieceParams PA;
+        PA.p = ca.y; PA.s1 = ca.z; PA.s2 = ca.w; PA.inv1 = PA.inv2 = 0.0f;
+        if (__all_sync(full, simple)) {
+            dequantize8<PACKED, false, UNS>(w0, w1, mb, 8, PA, loA, PA, loA, g.qmask, g.sign_shift, yv);
+            if (BC) {
+#pragma unroll
+                for (int t = 0; t < 8; ++t) yv[t] = __fadd_rn(__fmul_rn(ba.y, yv[t]), ba.z);
+            }
+        } else {
+            const bool one = inner != 0 && (inner & (inner - 1)) == 0 && ca.x > 0.0f && cnt == 8;
+            float4 da = ca, bb = ba;
+            int split = 8;
+            if (one) {
+                da = qa[l + 1];
+                if (QB) bb = qb[l + 1];
+                split = __ffs(inner);
+            }
+            const float loB = UNS ? bb.x : 0.0f;
+            if (__all_sync(full, simple || (one && da.x > 0.0f))) {
+                PieceParams PB;
+                PB.p = da.y; PB.s1 = da.z; PB.s2 = da.w; PB.inv1 = PB.inv2 = 0.0f;
+                dequantize8<PACKED, true, UNS>(w0, w1, mb, split, PA, loA, PB, loB, g.qmask,
+                                               g.sign_shift, yv);
+                if (BC) {
+#pragma unroll
+                    for (int t = 0; t < 8; ++t)
+                        yv[t] = __fadd_rn(__fmul_rn(t < split ? ba.y : bb.y, yv[t]),
+                                          t < split ? ba.z : bb.z);
+                }
+            } else {
+#pragma unroll
+                for (int t = 0; t < 8; ++t) {
+                    yv[t] = 0.0f;
+                    if (t < cnt) {
+                        const int lt = l + __popc(inner & ((1u << t) - 1u));
+                        const float4 ea = qa[lt];
+                        const float4 eb = QB ? qb[lt] : make_float4(0.0f, 1.0f, 0.0f, 0.0f);
+                        const float loE = UNS ? eb.x : 0.0f;
+                        if (UNS) yv[t] = loE;                  // a constant row delivers lo
+                        if (ea.x > 0.0f) {
+                            const uint32_t code = code_of<PACKED>(w0, w1, t);
+                            const int tail = (mb >> t) & 1;
+                            const int neg = !UNS && ((code >> (g.bits - 1)) & 1);
+                            const float q = (float)(code & g.qmask);
+                            float v = __fmul_rn(q, tail ? ea.w : ea.z);
+                            v = __fadd_rn(v, tail ? ea.y : 0.0f);
+                            yv[t] = UNS ? __fadd_rn(v, loE) : (neg ? -v : v);
+                        }
+                        if (BC) yv[t] = __fadd_rn(__fmul_rn(eb.y, yv[t]), eb.z);
+                    }
+                }
+            }
+        }
+    } else {
+        RowState rs;
+#pragma unroll
+        for (int t = 0; t < 8; ++t) {
+            yv[t] = 0.0f;
+            if (t < cnt) {
+                rs.seek(g.rows, g.A, g.Lf, i0 + t);
+                if (UNS) yv[t] = rs.lo;
+                if (rs.m > 0.0f) {
+                    const uint32_t code = code_of<PACKED>(w0, w1, t);
+                    const int tail = (mb >> t) & 1;
+                    const int neg = !UNS && ((code >> (g.bits - 1)) & 1);
+                    const float q = (float)(code & g.qmask);
+                    float v = __fmul_rn(q, tail ? rs.P.s2 : rs.P.s1);
+                    v = __fadd_rn(v, tail ? rs.P.p : 0.0f);
+                    yv[t] = UNS ? __fadd_rn(v, rs.lo) : (neg ? -v : v);
+                }
+                if (BC) yv[t] = __fadd_rn(__fmul_rn(__ldg(g.A.xi + rs.row), yv[t]), __ldg(g.A.beta + rs.row));
+            }
+        }
+    }
+    if (FULL) {
+        float4* dst = reinterpret_cast<float4*>(g.y + span_beg) + (li >> 2);
+        __stcs(dst, make_float4(yv[0], yv[1], yv[2], yv[3]));
+        __stcs(dst + 1, make_float4(yv[4], yv[5], yv[6], yv[7]));
+        return;
+    }
+    if (cnt == 0) return;
+    if (g.vec_out && cnt == 8) {
+        __stcs(reinterpret_cast<float4*>(g.y + i0), make_float4(yv[0], yv[1], yv[2], yv[3]));
+        __stcs(reinterpret_cast<float4*>(g.y + i0 + 4), make_float4(yv[4], yv[5], yv[6], yv[7]));
+    } else {
+        for (int t = 0; t < cnt; ++t) g.y[i0 + t] = yv[t];
+    }
+}
+
+// A thread's codes and region bits of one span, requested ahead of use.  A complete span whose
+// code words can be read whole takes 32-bit offsets from the span's slices of the two streams.
+template <bool PACKED>
+__device__ __forceinline__ void load_codes(CodeRegs<PACKED>& r, const uint8_t* __restrict__ codes,
+                                           const uint8_t* __restrict__ mask, int64_t span_beg,
+                                           int64_t total, int vec_codes, int li0) {
+    if (vec_codes && span_beg + kMapSpan <= total) {
+        const uint8_t* ms = mask + (span_beg >> 3);
+#pragma unroll
+        for (int c = 0; c < kQChunks; ++c) {
+            const int g8 = (li0 + c * 256) >> 3;
+            if (PACKED) {
+                r.w0[c] = __ldcs(reinterpret_cast<const unsigned int*>(codes + (span_beg >> 1)) + g8);
+                r.w1[c] = 0;
+            } else {
+                const uint2 w = __ldcs(reinterpret_cast<const uint2*>(codes + span_beg) + g8);
+                r.w0[c] = w.x; r.w1[c] = w.y;
+            }
+            r.mb[c] = ms[g8];
+        }
+    } else {
+        r.load(codes, mask, span_beg, total, vec_codes);
+    }
+}
+
 // Producer / consumer form of the inverse (see quantize_map_kernel and pwlq_rowmap.cuh).  The
 // producer writes row maps and constants only; the consumers request the codes and region bits
 // of the next span into registers before they wait for the current span's map.
 // BC: the bias-corrected value xi * y + beta (one multiply, one add) instead of y.
 template <bool PACKED, bool UNS, bool LONG, bool BC>
-__global__ void __launch_bounds__(kMapThreads, PWLQ_Q_MINBLOCKS)
+__global__ void __launch_bounds__(kMapThreads, 4)
 dequantize_map_kernel(const uint8_t* __restrict__ codes, const uint8_t* __restrict__ mask, Rows rows,
                       int64_t total, int bits, RowArrays A, float* __restrict__ y, int vec_codes,
                       int vec_out, int64_t spans_per_cta) {
@@ -658,7 +797,6 @@ dequantize_map_kernel(const uint8_t* __restrict__ codes, const uint8_t* __restri
     extern __shared__ __align__(128) unsigned char smem_raw[];
     Stage* st = reinterpret_cast<Stage*>(smem_raw);
     __shared__ uint64_t full_bar[kMapStages], empty_bar[kMapStages];
-    const unsigned full = 0xffffffffu;
     const int qmask = UNS ? (1 << bits) - 1 : (1 << (bits - 1)) - 1;   // the level inside a code
     const float Lf = (float)qmask;
     const int sign_shift = 32 - bits;                 // moves a code's sign bit to bit 31
@@ -705,119 +843,31 @@ dequantize_map_kernel(const uint8_t* __restrict__ codes, const uint8_t* __restri
     }
 
     // ---- consumers
+    const DequantizeCtx ctx{rows, A, total, bits, qmask, sign_shift, Lf, y, vec_out};
+    const int li0 = warp * (kMapSpan / kMapConsumers) + lane * 8;     // pass c: li0 + 256 c
     CodeRegs<PACKED> cur, nxt;
-    cur.load(codes, mask, first * kMapSpan, total, vec_codes);
+    load_codes<PACKED>(cur, codes, mask, first * kMapSpan, total, vec_codes, li0);
     int64_t it = 0;
     for (int64_t span = first; span < last; ++span, ++it) {
         const int s = (int)(it % kMapStages);
         const unsigned use = (unsigned)(it / kMapStages);
-        if (span + 1 < last) nxt.load(codes, mask, (span + 1) * kMapSpan, total, vec_codes);
+        const int64_t span_beg = span * kMapSpan;
+        if (span + 1 < last) load_codes<PACKED>(nxt, codes, mask, span_beg + kMapSpan, total, vec_codes, li0);
         if (!mbar_wait_relaxed(&full_bar[s], use & 1u)) {
             if (lane == 0) atomicExch(&g_quantize_timeout, 1);
             return;
         }
-        const int64_t span_beg = span * kMapSpan;
         const Stage& S = st[s];
-        const bool slow = S.map.slow != 0;
+        if (S.map.slow == 0 && span_beg + kMapSpan <= total && vec_out) {
 #pragma unroll
-        for (int c = 0; c < kQChunks; ++c) {
-            const int li = chunk_offset(c);
-            const int64_t i0 = span_beg + li;
-            const int cnt = (int)max((int64_t)0, min((int64_t)8, total - i0));
-            float yv[8];
-            if (!slow) {
-                uint32_t word;
-                const int l = map_slot(S.map, li, word);
-                const uint32_t inner = (word >> ((li & 31) + 1)) & 0x7Fu;   // starts at li+1 .. li+7
-                const float4 ca = S.qa[l];
-                const float loA = UNS ? S.qb[l].x : 0.0f;
-                const bool simple = inner == 0 && ca.x > 0.0f && cnt == 8;
-                PieceParams PA;
-                PA.p = ca.y; PA.s1 = ca.z; PA.s2 = ca.w; PA.inv1 = PA.inv2 = 0.0f;
-                if (__all_sync(full, simple)) {
-                    dequantize8<PACKED, false, UNS>(cur.w0[c], cur.w1[c], cur.mb[c], 8, PA, loA, PA, loA,
-                                                    qmask, sign_shift, yv);
-                    if (BC) {
-                        const float4 ba = S.qb[l];
+            for (int c = 0; c < kQChunks; ++c)
+                dequantize_pass<PACKED, UNS, BC, true>(ctx, cur.w0[c], cur.w1[c], cur.mb[c], S.map, S.qa,
+                                                       S.qb, span_beg, li0 + c * 256);
+        } else {
 #pragma unroll
-                        for (int t = 0; t < 8; ++t) yv[t] = __fadd_rn(__fmul_rn(ba.y, yv[t]), ba.z);
-                    }
-                } else {
-                    const bool one = inner != 0 && (inner & (inner - 1)) == 0 && ca.x > 0.0f && cnt == 8;
-                    float4 da = ca;
-                    float loB = loA;
-                    int split = 8;
-                    if (one) {
-                        da = S.qa[l + 1];
-                        if (UNS) loB = S.qb[l + 1].x;
-                        split = __ffs(inner);
-                    }
-                    if (__all_sync(full, simple || (one && da.x > 0.0f))) {
-                        PieceParams PB;
-                        PB.p = da.y; PB.s1 = da.z; PB.s2 = da.w; PB.inv1 = PB.inv2 = 0.0f;
-                        dequantize8<PACKED, true, UNS>(cur.w0[c], cur.w1[c], cur.mb[c], split, PA, loA,
-                                                       PB, loB, qmask, sign_shift, yv);
-                        if (BC) {
-                            const float4 ba = S.qb[l], bb = S.qb[one ? l + 1 : l];
-#pragma unroll
-                            for (int t = 0; t < 8; ++t)
-                                yv[t] = __fadd_rn(__fmul_rn(t < split ? ba.y : bb.y, yv[t]),
-                                                  t < split ? ba.z : bb.z);
-                        }
-                    } else {
-#pragma unroll
-                        for (int t = 0; t < 8; ++t) {
-                            yv[t] = 0.0f;
-                            if (t < cnt) {
-                                const int lt = l + __popc(inner & ((1u << t) - 1u));
-                                const float4 ea = S.qa[lt];
-                                const float loE = UNS ? S.qb[lt].x : 0.0f;
-                                if (UNS) yv[t] = loE;                  // a constant row delivers lo
-                                if (ea.x > 0.0f) {
-                                    const uint32_t code = code_of<PACKED>(cur.w0[c], cur.w1[c], t);
-                                    const int tail = (cur.mb[c] >> t) & 1;
-                                    const int neg = !UNS && ((code >> (bits - 1)) & 1);
-                                    const float q = (float)(code & qmask);
-                                    float v = __fmul_rn(q, tail ? ea.w : ea.z);
-                                    v = __fadd_rn(v, tail ? ea.y : 0.0f);
-                                    yv[t] = UNS ? __fadd_rn(v, loE) : (neg ? -v : v);
-                                }
-                                if (BC) {
-                                    const float4 eb = S.qb[lt];
-                                    yv[t] = __fadd_rn(__fmul_rn(eb.y, yv[t]), eb.z);
-                                }
-                            }
-                        }
-                    }
-                }
-            } else {
-                RowState rs;
-#pragma unroll
-                for (int t = 0; t < 8; ++t) {
-                    yv[t] = 0.0f;
-                    if (t < cnt) {
-                        rs.seek(rows, A, Lf, i0 + t);
-                        if (UNS) yv[t] = rs.lo;
-                        if (rs.m > 0.0f) {
-                            const uint32_t code = code_of<PACKED>(cur.w0[c], cur.w1[c], t);
-                            const int tail = (cur.mb[c] >> t) & 1;
-                            const int neg = !UNS && ((code >> (bits - 1)) & 1);
-                            const float q = (float)(code & qmask);
-                            float v = __fmul_rn(q, tail ? rs.P.s2 : rs.P.s1);
-                            v = __fadd_rn(v, tail ? rs.P.p : 0.0f);
-                            yv[t] = UNS ? __fadd_rn(v, rs.lo) : (neg ? -v : v);
-                        }
-                        if (BC) yv[t] = __fadd_rn(__fmul_rn(__ldg(A.xi + rs.row), yv[t]), __ldg(A.beta + rs.row));
-                    }
-                }
-            }
-            if (cnt == 0) continue;
-            if (vec_out && cnt == 8) {
-                __stcs(reinterpret_cast<float4*>(y + i0), make_float4(yv[0], yv[1], yv[2], yv[3]));
-                __stcs(reinterpret_cast<float4*>(y + i0 + 4), make_float4(yv[4], yv[5], yv[6], yv[7]));
-            } else {
-                for (int t = 0; t < cnt; ++t) y[i0 + t] = yv[t];
-            }
+            for (int c = 0; c < kQChunks; ++c)
+                dequantize_pass<PACKED, UNS, BC, false>(ctx, cur.w0[c], cur.w1[c], cur.mb[c], S.map, S.qa,
+                                                        S.qb, span_beg, li0 + c * 256);
         }
         __syncwarp();
         if (lane == 0) mbar_arrive(&empty_bar[s]);
@@ -910,7 +960,7 @@ cudaError_t launch_quantize(const float* x, const int64_t* row_offsets, int64_t 
     const bool long_rows = row_offsets == nullptr && n >= kMapSpan;   // the map follows from n
 #define PWLQ_LAUNCH_QUANTIZE(PK, FK, UN)                                                          \
     do {                                                                                          \
-        const size_t msmem = sizeof(MapStage<true, FK || UN>) * kMapStages;                       \
+        const size_t msmem = sizeof(MapStage<true, FK || UN>) * kMapStages;                     \
         if (long_rows) {                                                                          \
             const SpanGrid g = span_grid((const void*)quantize_map_kernel<PK, FK, UN, true>,      \
                                          kMapThreads, msmem, nspans, true);                       \

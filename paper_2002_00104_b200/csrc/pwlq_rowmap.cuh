@@ -27,10 +27,7 @@ namespace pwlq {
 
 constexpr int kMapSpan = 4096;                 // values per span
 constexpr int kMapWords = kMapSpan / 32;
-#ifndef PWLQ_MAP_ROUNDS
-#define PWLQ_MAP_ROUNDS 17
-#endif
-constexpr int kMapRounds = PWLQ_MAP_ROUNDS;                 // rounds of 32 rows the producer looks at per span
+constexpr int kMapRounds = 17;                 // rounds of 32 rows the producer looks at per span
 constexpr int kMapSlots = kMapRounds * 32;     // rows a map can describe (rows of >= 8 values fit)
 
 struct SpanRowMap {
