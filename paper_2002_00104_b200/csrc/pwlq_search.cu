@@ -343,7 +343,14 @@ __device__ __forceinline__ bool row_setup(const SearchArgs& a, int64_t& row, int
 // the constants, closing the sums) that a handful of vectors per lane cannot amortise.
 constexpr int kCwLongTile = 8, kCwMidTile = 16, kCwShortTile = 32;
 constexpr int kLongTileMin = 3072, kMidTileMin = 768;     // values per tile
-__host__ __device__ inline int group_width(int cnt) {
+// Few candidates on a long tile: groups of four keep as many (group, slice) items as there are
+// warps without slicing the tile, and halve the entries between a group's boundaries.
+constexpr int kCwFewCand = 4;
+#ifndef PWLQ_FEW_CAND_K
+#define PWLQ_FEW_CAND_K 64
+#endif
+__host__ __device__ inline int group_width(int cnt, int K) {
+    if (cnt >= kLongTileMin && K <= PWLQ_FEW_CAND_K) return kCwFewCand;
     return cnt >= kLongTileMin ? kCwLongTile : (cnt >= kMidTileMin ? kCwMidTile : kCwShortTile);
 }
 
@@ -468,7 +475,7 @@ search_sorted_kernel(SearchArgs a) {
 
     const int K = a.K;
     const int nwarps = (int)(blockDim.x >> 5), nthreads = (int)blockDim.x;
-    const int cw = group_width(cnt);
+    const int cw = group_width(cnt, K);
     const int E = min(slices_sorted(K, cw, nwarps), max(1, cnt / 512));   // a slice is worth >= 128 vectors
     size_t off[7];
     sorted_smem_layout(a.cap, K, nwarps, off);
@@ -600,7 +607,10 @@ search_sorted_kernel(SearchArgs a) {
     const int64_t n_row = a.rows.begin(row + 1) - a.rows.begin(row);
     const int64_t L = a.levels;
     const bool fused = fused_ok(n_row, L);
-    if (cw == kCwLongTile) {
+    if (cw == kCwFewCand) {
+        if (fused) eval_sorted<kCwFewCand, false>(a, S, m, n4, pad, E, &next_item);
+        else       eval_sorted<kCwFewCand, true>(a, S, m, n4, pad, E, &next_item);
+    } else if (cw == kCwLongTile) {
         if (fused) eval_sorted<kCwLongTile, false>(a, S, m, n4, pad, E, &next_item);
         else       eval_sorted<kCwLongTile, true>(a, S, m, n4, pad, E, &next_item);
     } else if (cw == kCwMidTile) {
