@@ -151,6 +151,38 @@ int pwlq_dequantize_ragged(const uint8_t* codes, const uint8_t* region_mask,
                            const float* m, const float* p, float* y, int code_layout,
                            void* stream);
 
+/* Row maps built once per layout.  The three streaming calls above (abs-max, quantize,
+ * dequantize) work on spans of 4096 consecutive values and must know, for every span, which rows
+ * overlap it (Sec. 5: weights are quantized per output channel, so a network's weights are many
+ * short rows).  That description depends on the row layout only -- not on the values, m or p --
+ * and without help every call rebuilds it inside the kernel.  A caller that runs several calls over
+ * one layout builds it once:
+ *   pwlq_rowmap_bytes(total)   size of the map buffer (0 if total is out of range)
+ *   pwlq_rowmap_build          fills `rowmap` (device memory of the caller, 16-byte aligned,
+ *                              rowmap_bytes >= pwlq_rowmap_bytes(total), else PWLQ_ERR_WORKSPACE)
+ *                              for ragged rows (row_offsets != NULL; n ignored) or for dense rows
+ *                              of n values (row_offsets == NULL, total = C * n)
+ *   pwlq_*_mapped              the same operation and bit-identical results as pwlq_absmax /
+ *                              pwlq_quantize / pwlq_dequantize (and their _ragged forms), given the
+ *                              maps of this very layout.  The maps are only read: any number of
+ *                              calls, on any streams, may share them once the build has finished.
+ * Maps built for another layout (other C, total or n) are detected on the device: the call then
+ * writes nothing and pwlq_device_status() reports 1 << PWLQ_ERR_INVALID_ARG.  Offsets that were
+ * changed after the build while C and total stayed the same are not detected. */
+size_t pwlq_rowmap_bytes(int64_t total);
+int pwlq_rowmap_build(const int64_t* row_offsets, int64_t C, int64_t n, int64_t total,
+                      void* rowmap, size_t rowmap_bytes, void* stream);
+int pwlq_absmax_mapped(const float* x, const int64_t* row_offsets, int64_t C, int64_t n,
+                       int64_t total, const void* rowmap, float* m_out, void* stream);
+int pwlq_quantize_mapped(const float* x, const int64_t* row_offsets, int64_t C, int64_t n,
+                         int64_t total, const void* rowmap, int bits, const float* m,
+                         const float* p, uint8_t* codes, uint8_t* region_mask, float* fake_out,
+                         int code_layout, void* stream);
+int pwlq_dequantize_mapped(const uint8_t* codes, const uint8_t* region_mask,
+                           const int64_t* row_offsets, int64_t C, int64_t n, int64_t total,
+                           const void* rowmap, int bits, const float* m, const float* p, float* y,
+                           int code_layout, void* stream);
+
 /* One-sided ranges: unsigned tensors such as ReLU activations, or any asymmetric range [m1, m2]
  * (Sec. 3.2, footnote to the range; Eq. 1 with z = r_l and the unsigned integer domain
  * {0, ..., 2^b - 1} for one-sided distributions).  The paper does not spell the piecewise form
@@ -352,7 +384,8 @@ size_t pwlq_search_noalloc_max_bytes(void);
  * barriers that they await with a bounded number of polls; a wait that runs out makes the kernel
  * stop early and sets a flag on the current device.  This call reads the flags (it synchronises
  * with the device) and returns 0, or 1 << PWLQ_ERR_TIMEOUT if a wait has expired on the current
- * device since the previous call of pwlq_device_status -- the outputs of the streaming calls made
+ * device since the previous call of pwlq_device_status, OR-ed with 1 << PWLQ_ERR_INVALID_ARG if a
+ * *_mapped call was given row maps of another layout -- the outputs of the streaming calls made
  * in between are then not valid -- or 1 << PWLQ_ERR_CUDA if the flags could not be read.  Reading
  * clears the flags: call it after synchronising the work it is meant to vouch for. */
 int pwlq_device_status(void);

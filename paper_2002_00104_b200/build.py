@@ -11,7 +11,7 @@ LIB = os.path.join(HERE, "libpwlq.so")
 PEAK_LIB = os.path.join(HERE, "libpwlq_peak.so")     # FP32 micro-benchmark, loaded by bench.py only
 PEAK_SOURCES = ["fp32_peak.cu"]
 SOURCES = ["pwlq_api.cu", "pwlq_absmax.cu", "pwlq_search.cu", "pwlq_quantize.cu",
-           "pwlq_noalloc.cu", "pwlq_select.cu", "pwlq_search2.cu", "pwlq_bias.cu"]
+           "pwlq_noalloc.cu", "pwlq_select.cu", "pwlq_search2.cu", "pwlq_bias.cu", "pwlq_rowmap.cu"]
 NVCC_FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a", "-O3", "-std=c++17", "-lineinfo",
     "-fmad=false",            # no implicit FMA contraction: every fused op is an explicit fmaf

@@ -19,7 +19,7 @@ constexpr int kAbsThreads = (kAbsConsumers + 1) * 32;    // + the producer warp
 constexpr int kAbsStages = 2;                            // spans in flight per CTA
 static_assert(kAbsStages <= 4, "MapProducer tracks at most four stages");
 
-static __device__ int g_absmax_timeout;                  // set when a bounded wait expired
+static __device__ int g_absmax_timeout;   // bit 0: a bounded wait expired; bit 1: row maps of another layout
 
 // Order-preserving map of binary32 values onto unsigned integers (and back), so that minima and
 // maxima of signed values can use integer atomics.
@@ -85,11 +85,18 @@ __device__ __forceinline__ unsigned abs_bulk_bytes(int64_t span, int64_t total, 
 // loop over the rows: every lane splits its values at its start, a segmented scan over the lanes
 // joins the pieces of every row, and the lane in which a row ends issues the row's atomic.
 // LONG: dense rows of at least a span (the maps follow from the row length).
-template <bool MINMAX, bool LONG>
+// PRE: the maps were built ahead of time (premap: header, then one map per span); the producer
+// only requests copies.
+template <bool MINMAX, bool LONG, bool PRE>
 __global__ void __launch_bounds__(kAbsThreads)
 absmax_kernel(const float* __restrict__ x, Rows rows, int64_t total, uint32_t* __restrict__ m_bits,
-              uint32_t* __restrict__ lo_bits, int vec_ok, int64_t spans_per_cta) {
+              uint32_t* __restrict__ lo_bits, int vec_ok, int64_t spans_per_cta,
+              const unsigned char* __restrict__ premap) {
     extern __shared__ __align__(128) unsigned char smem_raw[];
+    if (PRE && !rowmap_matches(premap, rows, total)) {        // maps of another layout: no work
+        if (threadIdx.x == 0) atomicOr(&g_absmax_timeout, 2);
+        return;
+    }
     AbsStage* st = reinterpret_cast<AbsStage*>(smem_raw);
     __shared__ uint64_t full_bar[kAbsStages], empty_bar[kAbsStages];
     const unsigned full = 0xffffffffu;
@@ -106,6 +113,38 @@ absmax_kernel(const float* __restrict__ x, Rows rows, int64_t total, uint32_t* _
     __syncthreads();
     if (first >= last) return;
 
+    if (PRE && warp == kAbsConsumers) {
+        // ---- producer, maps built ahead of time: two bulk copies per span
+        const SpanRowMap* maps = reinterpret_cast<const SpanRowMap*>(premap + kRowMapHeaderBytes);
+        int64_t it = 0;
+        for (int64_t span = first; span < last; ++span, ++it) {
+            const int s = (int)(it % kAbsStages);
+            const unsigned use = (unsigned)(it / kAbsStages);
+            if (use > 0 && !mbar_wait(&empty_bar[s], (use - 1) & 1u)) {
+                if (lane == 0) atomicOr(&g_absmax_timeout, 1);
+                for (int64_t j = it - 1; j >= 0 && j > it - 1 - kAbsStages; --j)
+                    mbar_wait(&full_bar[j % kAbsStages], (unsigned)(j / kAbsStages) & 1u);
+                return;
+            }
+            const int64_t span_beg = span * kMapSpan, span_end = min(span_beg + kMapSpan, total);
+            const unsigned bytes = abs_bulk_bytes(span, total, vec_ok);
+            if (bytes != 0) {
+                if (lane == 0) {
+                    mbar_expect_tx(&full_bar[s], bytes);
+                    bulk_copy_g2s(st[s].data, x + span_beg, bytes, &full_bar[s]);
+                }
+            } else {                               // unaligned base or ragged tail: plain loads
+                for (int i = lane; i < (int)(span_end - span_beg); i += 32) st[s].data[i] = x[span_beg + i];
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&full_bar[s]);
+            }
+            if (lane == 0) {
+                mbar_expect_tx(&full_bar[s], (unsigned)sizeof(SpanRowMap));
+                bulk_copy_g2s(&st[s].map, maps + span, (unsigned)sizeof(SpanRowMap), &full_bar[s]);
+            }
+        }
+        return;
+    }
     if (warp == kAbsConsumers) {
         // ---- producer
         MapProducer<false, false> prod;
@@ -129,7 +168,7 @@ absmax_kernel(const float* __restrict__ x, Rows rows, int64_t total, uint32_t* _
             if (use > 0 && !mbar_wait(&empty_bar[s], (use - 1) & 1u)) {
                 // never expected: report, let the copies of the earlier spans land (their stages'
                 // barriers have this warp's arrivals already), and leave
-                if (lane == 0) atomicExch(&g_absmax_timeout, 1);
+                if (lane == 0) atomicOr(&g_absmax_timeout, 1);
                 for (int64_t j = it - 1; j >= 0 && j > it - 1 - kAbsStages; --j)
                     mbar_wait(&full_bar[j % kAbsStages], (unsigned)(j / kAbsStages) & 1u);
                 return;
@@ -170,7 +209,7 @@ absmax_kernel(const float* __restrict__ x, Rows rows, int64_t total, uint32_t* _
         const int s = (int)(it % kAbsStages);
         const unsigned use = (unsigned)(it / kAbsStages);
         if (!mbar_wait_relaxed(&full_bar[s], use & 1u)) {
-            if (lane == 0) atomicExch(&g_absmax_timeout, 1);
+            if (lane == 0) atomicOr(&g_absmax_timeout, 1);
             return;
         }
         const int64_t span_beg = span * kMapSpan;
@@ -339,7 +378,7 @@ __global__ void minmax_finalize_kernel(uint32_t* __restrict__ lo_bits,
 template <bool MINMAX>
 static cudaError_t launch_fold(const float* x, const int64_t* row_offsets, int64_t C, int64_t n,
                                int64_t total, float* out_a, float* out_b, cudaStream_t stream,
-                               int64_t shift) {
+                               int64_t shift, const void* rowmap) {
     cudaError_t e = cudaMemsetAsync(out_a, 0, sizeof(float) * (size_t)C, stream);
     if (e != cudaSuccess) return e;
     if (MINMAX) {
@@ -351,15 +390,18 @@ static cudaError_t launch_fold(const float* x, const int64_t* row_offsets, int64
     const int64_t nspans = (total + kMapSpan - 1) / kMapSpan;
     const bool long_rows = row_offsets == nullptr && n >= kMapSpan;   // the maps follow from n
     const size_t smem = sizeof(AbsStage) * kAbsStages;
-    const void* kernel = long_rows ? (const void*)absmax_kernel<MINMAX, true>
-                                   : (const void*)absmax_kernel<MINMAX, false>;
-    static int cached[2][2][64] = {{{0}}};             // CTAs that fit the device at once
+    // (maps built ahead of time are of no use where the map follows from the row length)
+    const unsigned char* premap = long_rows ? nullptr : static_cast<const unsigned char*>(rowmap);
+    const void* kernel = long_rows ? (const void*)absmax_kernel<MINMAX, true, false>
+                         : premap  ? (const void*)absmax_kernel<MINMAX, false, true>
+                                   : (const void*)absmax_kernel<MINMAX, false, false>;
+    static int cached[2][3][64] = {{{0}}};             // CTAs that fit the device at once
     static std::mutex cached_mu;
     int dev = 0;
     cudaGetDevice(&dev);
     if (dev < 0 || dev >= 64) dev = 0;
     std::lock_guard<std::mutex> lock(cached_mu);
-    int& slots_dev = cached[MINMAX ? 1 : 0][long_rows ? 1 : 0][dev];
+    int& slots_dev = cached[MINMAX ? 1 : 0][long_rows ? 1 : (premap ? 2 : 0)][dev];
     if (slots_dev == 0) {
         e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (e != cudaSuccess) return e;
@@ -376,25 +418,29 @@ static cudaError_t launch_fold(const float* x, const int64_t* row_offsets, int64
         std::min<int64_t>(std::max<int64_t>((nspans + 4 * slots - 1) / (4 * slots), 1), 32);
     const unsigned grid = (unsigned)((nspans + per_cta - 1) / per_cta);
     const int vec_ok = (reinterpret_cast<uintptr_t>(x) & 15u) == 0;
+    uint32_t* a_bits = reinterpret_cast<uint32_t*>(out_a);
+    uint32_t* b_bits = reinterpret_cast<uint32_t*>(out_b);
     if (long_rows)
-        absmax_kernel<MINMAX, true><<<grid, kAbsThreads, smem, stream>>>(
-            x, rows, total, reinterpret_cast<uint32_t*>(out_a), reinterpret_cast<uint32_t*>(out_b),
-            vec_ok, per_cta);
+        absmax_kernel<MINMAX, true, false><<<grid, kAbsThreads, smem, stream>>>(
+            x, rows, total, a_bits, b_bits, vec_ok, per_cta, nullptr);
+    else if (premap)
+        absmax_kernel<MINMAX, false, true><<<grid, kAbsThreads, smem, stream>>>(
+            x, rows, total, a_bits, b_bits, vec_ok, per_cta, premap);
     else
-        absmax_kernel<MINMAX, false><<<grid, kAbsThreads, smem, stream>>>(
-            x, rows, total, reinterpret_cast<uint32_t*>(out_a), reinterpret_cast<uint32_t*>(out_b),
-            vec_ok, per_cta);
+        absmax_kernel<MINMAX, false, false><<<grid, kAbsThreads, smem, stream>>>(
+            x, rows, total, a_bits, b_bits, vec_ok, per_cta, nullptr);
     return cudaGetLastError();
 }
 
 cudaError_t launch_absmax(const float* x, const int64_t* row_offsets, int64_t C, int64_t n,
-                          int64_t total, float* m_out, cudaStream_t stream, int64_t shift) {
-    return launch_fold<false>(x, row_offsets, C, n, total, m_out, nullptr, stream, shift);
+                          int64_t total, float* m_out, cudaStream_t stream, int64_t shift,
+                          const void* rowmap) {
+    return launch_fold<false>(x, row_offsets, C, n, total, m_out, nullptr, stream, shift, rowmap);
 }
 
 cudaError_t launch_minmax(const float* x, const int64_t* row_offsets, int64_t C, int64_t n,
                           int64_t total, float* lo_out, float* hi_out, cudaStream_t stream) {
-    cudaError_t e = launch_fold<true>(x, row_offsets, C, n, total, hi_out, lo_out, stream, 0);
+    cudaError_t e = launch_fold<true>(x, row_offsets, C, n, total, hi_out, lo_out, stream, 0, nullptr);
     if (e != cudaSuccess) return e;
     minmax_finalize_kernel<<<(unsigned)((C + 255) / 256), 256, 0, stream>>>(
         reinterpret_cast<uint32_t*>(lo_out), reinterpret_cast<uint32_t*>(hi_out), C);

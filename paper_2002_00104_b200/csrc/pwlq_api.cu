@@ -24,11 +24,22 @@ int check_rows(int64_t C, int64_t n_or_total) {
 }
 
 int absmax_impl(const float* x, const int64_t* ro, int64_t C, int64_t n, int64_t total,
-                float* m_out, void* stream) {
-    if (!x || !m_out || misaligned(x, 4) || misaligned(m_out, 4) || misaligned(ro, 8))
+                float* m_out, void* stream, const void* rowmap = nullptr) {
+    if (!x || !m_out || misaligned(x, 4) || misaligned(m_out, 4) || misaligned(ro, 8) ||
+        misaligned(rowmap, 16))
         return PWLQ_ERR_INVALID_ARG;
     if (total > kMaxTotal) return PWLQ_ERR_UNSUPPORTED;
-    return from_cuda(pwlq::launch_absmax(x, ro, C, n, total, m_out, as_stream(stream)));
+    return from_cuda(pwlq::launch_absmax(x, ro, C, n, total, m_out, as_stream(stream), 0, rowmap));
+}
+
+// Arguments of the *_mapped entry points that describe the layout: ragged rows (row_offsets, n
+// ignored) or dense rows of n values with total = C * n.
+int check_layout(const int64_t* ro, int64_t C, int64_t& n, int64_t total, const void* rowmap) {
+    if (int rc = check_rows(C, total)) return rc;
+    if (!rowmap) return PWLQ_ERR_INVALID_ARG;
+    if (ro) { n = 0; return PWLQ_OK; }
+    if (n < 1 || C * n != total) return PWLQ_ERR_INVALID_ARG;
+    return PWLQ_OK;
 }
 
 int minmax_impl(const float* x, const int64_t* ro, int64_t C, int64_t n, int64_t total,
@@ -67,8 +78,9 @@ int search_impl(const float* x, const int64_t* ro, int64_t C, int64_t n, int64_t
 
 int quantize_impl(const float* x, const int64_t* ro, int64_t C, int64_t n, int64_t total,
                   int bits, const float* m, const float* lo, const float* p, uint8_t* codes,
-                  uint8_t* mask, float* fake, int layout, void* stream) {
-    if (!x || !m || !p || !codes || !mask || bits < 2 || bits > 8 ||
+                  uint8_t* mask, float* fake, int layout, void* stream,
+                  const void* rowmap = nullptr) {
+    if (!x || !m || !p || !codes || !mask || bits < 2 || bits > 8 || misaligned(rowmap, 16) ||
         (layout != PWLQ_CODES_U8 && layout != PWLQ_CODES_PACKED))
         return PWLQ_ERR_INVALID_ARG;
     if (misaligned(x, 4) || misaligned(m, 4) || misaligned(lo, 4) || misaligned(p, 4) ||
@@ -76,13 +88,14 @@ int quantize_impl(const float* x, const int64_t* ro, int64_t C, int64_t n, int64
         return PWLQ_ERR_INVALID_ARG;
     if (total > kMaxTotal) return PWLQ_ERR_UNSUPPORTED;
     return from_cuda(pwlq::launch_quantize(x, ro, C, n, total, bits, m, lo, p, codes, mask, fake,
-                                           layout, as_stream(stream)));
+                                           layout, as_stream(stream), 0, rowmap));
 }
 
 int dequantize_impl(const uint8_t* codes, const uint8_t* mask, const int64_t* ro, int64_t C,
                     int64_t n, int64_t total, int bits, const float* m, const float* lo,
-                    const float* p, float* y, int layout, void* stream) {
-    if (!codes || !mask || !m || !p || !y || bits < 2 || bits > 8 ||
+                    const float* p, float* y, int layout, void* stream,
+                    const void* rowmap = nullptr) {
+    if (!codes || !mask || !m || !p || !y || bits < 2 || bits > 8 || misaligned(rowmap, 16) ||
         (layout != PWLQ_CODES_U8 && layout != PWLQ_CODES_PACKED))
         return PWLQ_ERR_INVALID_ARG;
     if (misaligned(m, 4) || misaligned(lo, 4) || misaligned(p, 4) || misaligned(y, 4) ||
@@ -90,7 +103,8 @@ int dequantize_impl(const uint8_t* codes, const uint8_t* mask, const int64_t* ro
         return PWLQ_ERR_INVALID_ARG;
     if (total > kMaxTotal) return PWLQ_ERR_UNSUPPORTED;
     return from_cuda(pwlq::launch_dequantize(codes, mask, ro, C, n, total, bits, m, lo, p, y,
-                                             layout, as_stream(stream)));
+                                             layout, as_stream(stream), 0, nullptr, nullptr,
+                                             rowmap));
 }
 
 inline size_t code_bytes(int64_t total, int bits, int layout) {
@@ -284,6 +298,44 @@ int pwlq_dequantize_ragged(const uint8_t* codes, const uint8_t* region_mask,
     if (!row_offsets) return PWLQ_ERR_INVALID_ARG;
     return dequantize_impl(codes, region_mask, row_offsets, C, 0, total, bits, m, nullptr, p, y,
                            code_layout, stream);
+}
+
+size_t pwlq_rowmap_bytes(int64_t total) {
+    if (total < 1 || total > kMaxTotal) return 0;
+    return pwlq::rowmap_bytes(total);
+}
+
+int pwlq_rowmap_build(const int64_t* row_offsets, int64_t C, int64_t n, int64_t total,
+                      void* rowmap, size_t rowmap_bytes, void* stream) {
+    if (int rc = check_layout(row_offsets, C, n, total, rowmap)) return rc;
+    if (misaligned(rowmap, 16) || misaligned(row_offsets, 8)) return PWLQ_ERR_INVALID_ARG;
+    if (total > kMaxTotal) return PWLQ_ERR_UNSUPPORTED;
+    if (rowmap_bytes < pwlq::rowmap_bytes(total)) return PWLQ_ERR_WORKSPACE;
+    return from_cuda(pwlq::launch_rowmap_build(row_offsets, C, n, total, rowmap, as_stream(stream)));
+}
+
+int pwlq_absmax_mapped(const float* x, const int64_t* row_offsets, int64_t C, int64_t n,
+                       int64_t total, const void* rowmap, float* m_out, void* stream) {
+    if (int rc = check_layout(row_offsets, C, n, total, rowmap)) return rc;
+    return absmax_impl(x, row_offsets, C, n, total, m_out, stream, rowmap);
+}
+
+int pwlq_quantize_mapped(const float* x, const int64_t* row_offsets, int64_t C, int64_t n,
+                         int64_t total, const void* rowmap, int bits, const float* m,
+                         const float* p, uint8_t* codes, uint8_t* region_mask, float* fake_out,
+                         int code_layout, void* stream) {
+    if (int rc = check_layout(row_offsets, C, n, total, rowmap)) return rc;
+    return quantize_impl(x, row_offsets, C, n, total, bits, m, nullptr, p, codes, region_mask,
+                         fake_out, code_layout, stream, rowmap);
+}
+
+int pwlq_dequantize_mapped(const uint8_t* codes, const uint8_t* region_mask,
+                           const int64_t* row_offsets, int64_t C, int64_t n, int64_t total,
+                           const void* rowmap, int bits, const float* m, const float* p, float* y,
+                           int code_layout, void* stream) {
+    if (int rc = check_layout(row_offsets, C, n, total, rowmap)) return rc;
+    return dequantize_impl(codes, region_mask, row_offsets, C, n, total, bits, m, nullptr, p, y,
+                           code_layout, stream, rowmap);
 }
 
 int pwlq_minmax(const float* x, int64_t C, int64_t n, float* lo_out, float* hi_out,
@@ -716,7 +768,8 @@ int pwlq_select_analytic_ragged(const float* x, const int64_t* row_offsets, int6
 int pwlq_device_status(void) {
     const int a = pwlq::take_absmax_timeout_flag(), q = pwlq::take_quantize_timeout_flag();
     if (a < 0 || q < 0) return 1 << PWLQ_ERR_CUDA;
-    return (a | q) ? (1 << PWLQ_ERR_TIMEOUT) : 0;
+    return (((a | q) & 1) ? (1 << PWLQ_ERR_TIMEOUT) : 0) |
+           (((a | q) & 2) ? (1 << PWLQ_ERR_INVALID_ARG) : 0);
 }
 
 // Not part of the public interface (include/pwlq.h does not declare it): lets the test suite see

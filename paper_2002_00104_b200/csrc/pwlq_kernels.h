@@ -14,8 +14,17 @@ constexpr int kSearchTile = 8192;
 // shift (here and below): for a slice of a longer list of ragged rows -- row_offsets points at the
 // slice's first offset, the data pointers were advanced by `shift` values, `total` counts the
 // slice's values; every offset read is reduced by `shift`.  0 for whole tensors.
+// rowmap (here and in launch_quantize / launch_dequantize): nullptr, or row maps of this layout
+// built by launch_rowmap_build, which spare the kernel's producer warps the map building.
 cudaError_t launch_absmax(const float* x, const int64_t* row_offsets, int64_t C, int64_t n,
-                          int64_t total, float* m_out, cudaStream_t stream, int64_t shift = 0);
+                          int64_t total, float* m_out, cudaStream_t stream, int64_t shift = 0,
+                          const void* rowmap = nullptr);
+
+// Row maps of a layout (ragged rows, or dense rows of n values), built once into `rowmap`
+// (rowmap_bytes(total) bytes, 16-byte aligned) for any number of streaming calls.
+size_t rowmap_bytes(int64_t total);
+cudaError_t launch_rowmap_build(const int64_t* row_offsets, int64_t C, int64_t n, int64_t total,
+                                void* rowmap, cudaStream_t stream);
 
 // Per-row minimum and maximum (the range [m1, m2] of a one-sided / asymmetric tensor).
 cudaError_t launch_minmax(const float* x, const int64_t* row_offsets, int64_t C, int64_t n,
@@ -52,13 +61,14 @@ cudaError_t launch_search_finish(const double* sums, int parts, int64_t C, int K
 cudaError_t launch_quantize(const float* x, const int64_t* row_offsets, int64_t C, int64_t n,
                             int64_t total, int bits, const float* m, const float* lo,
                             const float* p, uint8_t* codes, uint8_t* mask, float* fake, int layout,
-                            cudaStream_t stream, int64_t shift = 0);
+                            cudaStream_t stream, int64_t shift = 0, const void* rowmap = nullptr);
 
 cudaError_t launch_dequantize(const uint8_t* codes, const uint8_t* mask,
                               const int64_t* row_offsets, int64_t C, int64_t n, int64_t total,
                               int bits, const float* m, const float* lo, const float* p, float* y,
                               int layout, cudaStream_t stream, int64_t shift = 0,
-                              const float* xi = nullptr, const float* beta = nullptr);
+                              const float* xi = nullptr, const float* beta = nullptr,
+                              const void* rowmap = nullptr);
 
 // Two breakpoints (three regions): pair search over a grid of K <= kSearch2MaxK ascending ratios
 // for rows of at most kSearchTile values; quantize / dequantize with a two-bit region index.
@@ -99,9 +109,10 @@ cudaError_t launch_select_analytic(const float* x, const int64_t* row_offsets, i
                                    float* p_out, float* scale_out, void* workspace,
                                    cudaStream_t stream);
 
-// 1 when a bounded wait of the kernel family expired on the current device since the last call
-// of the same function, which also clears the flag (reads a device flag: synchronises with the
-// device); -1 when the flag could not be read.
+// Conditions the kernel family met on the current device since the last call of the same
+// function, which also clears them (reads a device flag: synchronises with the device): bit 0, a
+// bounded wait expired; bit 1, a call was given row maps of another layout.  -1 when the flag
+// could not be read.
 int take_absmax_timeout_flag();
 int take_quantize_timeout_flag();
 // Runs a bounded wait that is certain to expire after `polls` polls (self-test of the reporting).

@@ -22,7 +22,7 @@ constexpr int kQChunks = 2;                      // passes per span
 constexpr int kQSpan = kQChunk * kQChunks;       // values per span
 static_assert(kQSpan == kMapSpan, "the spans of the row maps");
 
-static __device__ int g_quantize_timeout;        // set when a bounded wait expired
+static __device__ int g_quantize_timeout;   // bit 0: a bounded wait expired; bit 1: row maps of another layout
 
 // Offset inside the span of the eight values a thread handles in pass c.  A warp owns one
 // contiguous eighth of the span and walks it in passes of 256 values, so that a thread's
@@ -357,15 +357,20 @@ __device__ __forceinline__ void quantize_pass(const QuantizeCtx<UNS>& g, const f
     }
 }
 
-template <bool PACKED, bool WANT_FAKE, bool UNS, bool LONG>
+// PRE: the row maps were built ahead of time (premap: header, then one map per span).
+template <bool PACKED, bool WANT_FAKE, bool UNS, bool LONG, bool PRE>
 __global__ void __launch_bounds__(kMapThreads, (WANT_FAKE || UNS) ? 3 : 4)
 quantize_map_kernel(const float* __restrict__ x, Rows rows, int64_t total, int bits, RowArrays A,
                     uint8_t* __restrict__ codes, uint8_t* __restrict__ mask,
                     float* __restrict__ fake, int vec_in, int vec_fake, int vec_codes,
-                    int64_t spans_per_cta) {
+                    int64_t spans_per_cta, const unsigned char* __restrict__ premap) {
     constexpr bool QB = WANT_FAKE || UNS;
     typedef MapStage<true, QB> Stage;
     extern __shared__ __align__(128) unsigned char smem_raw[];
+    if (PRE && !rowmap_matches(premap, rows, total)) {        // maps of another layout: no work
+        if (threadIdx.x == 0) atomicOr(&g_quantize_timeout, 2);
+        return;
+    }
     Stage* st = reinterpret_cast<Stage*>(smem_raw);
     __shared__ uint64_t full_bar[kMapStages], empty_bar[kMapStages];
     const unsigned full = 0xffffffffu;
@@ -386,6 +391,45 @@ quantize_map_kernel(const float* __restrict__ x, Rows rows, int64_t total, int b
     __syncthreads();
     if (first >= last) return;
 
+    if (PRE && warp == kMapConsumers) {
+        // ---- producer, maps built ahead of time: the values and the map of a span arrive by
+        // bulk copies; the warp computes the constants of the span's rows
+        const SpanRowMap* maps = reinterpret_cast<const SpanRowMap*>(premap + kRowMapHeaderBytes);
+        PreProducer<true, UNS> prod;
+        prod.in = RowInputs{A.m, A.lo, A.p, A.xi, A.beta};
+        prod.Lf = Lf;
+        prod.begin(maps, first, last);
+        int64_t it = 0;
+        for (int64_t span = first; span < last; ++span, ++it) {
+            const int s = (int)(it % kMapStages);
+            const unsigned use = (unsigned)(it / kMapStages);
+            if (use > 0 && !mbar_wait(&empty_bar[s], (use - 1) & 1u)) {
+                if (lane == 0) atomicOr(&g_quantize_timeout, 1);
+                for (int64_t j = it - 1; j >= 0 && j > it - 1 - kMapStages; --j)
+                    mbar_wait(&full_bar[j % kMapStages], (unsigned)(j / kMapStages) & 1u);
+                return;
+            }
+            const int64_t span_beg = span * kMapSpan, span_end = min(span_beg + kMapSpan, total);
+            const unsigned bytes = q_bulk_bytes(span, total, vec_in);
+            if (bytes != 0) {
+                if (lane == 0) {
+                    mbar_expect_tx(&full_bar[s], bytes);
+                    bulk_copy_g2s(st[s].data, x + span_beg, bytes, &full_bar[s]);
+                }
+            } else {                               // unaligned base or ragged tail: plain loads
+                for (int i = lane; i < (int)(span_end - span_beg); i += 32) st[s].data[i] = x[span_beg + i];
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&full_bar[s]);
+            }
+            prod.build(st[s].qa, QB ? st[s].qb : nullptr, span, last);
+            __syncwarp();
+            if (lane == 0) {
+                mbar_expect_tx(&full_bar[s], (unsigned)sizeof(SpanRowMap));
+                bulk_copy_g2s(&st[s].map, maps + span, (unsigned)sizeof(SpanRowMap), &full_bar[s]);
+            }
+        }
+        return;
+    }
     if (warp == kMapConsumers) {
         // ---- producer
         MapProducer<true, UNS> prod;
@@ -411,7 +455,7 @@ quantize_map_kernel(const float* __restrict__ x, Rows rows, int64_t total, int b
             if (use > 0 && !mbar_wait(&empty_bar[s], (use - 1) & 1u)) {
                 // never expected: report, let the copies of the earlier spans land (their stages'
                 // barriers have this warp's arrivals already), and leave
-                if (lane == 0) atomicExch(&g_quantize_timeout, 1);
+                if (lane == 0) atomicOr(&g_quantize_timeout, 1);
                 for (int64_t j = it - 1; j >= 0 && j > it - 1 - kMapStages; --j)
                     mbar_wait(&full_bar[j % kMapStages], (unsigned)(j / kMapStages) & 1u);
                 return;
@@ -452,7 +496,7 @@ quantize_map_kernel(const float* __restrict__ x, Rows rows, int64_t total, int b
         const int s = (int)(it % kMapStages);
         const unsigned use = (unsigned)(it / kMapStages);
         if (!mbar_wait_relaxed(&full_bar[s], use & 1u)) {
-            if (lane == 0) atomicExch(&g_quantize_timeout, 1);
+            if (lane == 0) atomicOr(&g_quantize_timeout, 1);
             return;
         }
         const int64_t span_beg = span * kMapSpan;
@@ -787,14 +831,19 @@ __device__ __forceinline__ void load_codes(CodeRegs<PACKED>& r, const uint8_t* _
 // producer writes row maps and constants only; the consumers request the codes and region bits
 // of the next span into registers before they wait for the current span's map.
 // BC: the bias-corrected value xi * y + beta (one multiply, one add) instead of y.
-template <bool PACKED, bool UNS, bool LONG, bool BC>
+// PRE: the row maps were built ahead of time (premap: header, then one map per span).
+template <bool PACKED, bool UNS, bool LONG, bool BC, bool PRE>
 __global__ void __launch_bounds__(kMapThreads, 4)
 dequantize_map_kernel(const uint8_t* __restrict__ codes, const uint8_t* __restrict__ mask, Rows rows,
                       int64_t total, int bits, RowArrays A, float* __restrict__ y, int vec_codes,
-                      int vec_out, int64_t spans_per_cta) {
+                      int vec_out, int64_t spans_per_cta, const unsigned char* __restrict__ premap) {
     constexpr bool QB = UNS || BC;                    // the stages hold the second half of the constants
     typedef MapStage<false, QB> Stage;
     extern __shared__ __align__(128) unsigned char smem_raw[];
+    if (PRE && !rowmap_matches(premap, rows, total)) {        // maps of another layout: no work
+        if (threadIdx.x == 0) atomicOr(&g_quantize_timeout, 2);
+        return;
+    }
     Stage* st = reinterpret_cast<Stage*>(smem_raw);
     __shared__ uint64_t full_bar[kMapStages], empty_bar[kMapStages];
     const int qmask = UNS ? (1 << bits) - 1 : (1 << (bits - 1)) - 1;   // the level inside a code
@@ -813,6 +862,33 @@ dequantize_map_kernel(const uint8_t* __restrict__ codes, const uint8_t* __restri
     __syncthreads();
     if (first >= last) return;
 
+    if (PRE && warp == kMapConsumers) {
+        // ---- producer, maps built ahead of time: the map arrives by a bulk copy, the warp
+        // computes the constants of the span's rows
+        const SpanRowMap* maps = reinterpret_cast<const SpanRowMap*>(premap + kRowMapHeaderBytes);
+        PreProducer<true, UNS, true, BC> prod;
+        prod.in = RowInputs{A.m, A.lo, A.p, A.xi, A.beta};
+        prod.Lf = Lf;
+        prod.begin(maps, first, last);
+        int64_t it = 0;
+        for (int64_t span = first; span < last; ++span, ++it) {
+            const int s = (int)(it % kMapStages);
+            const unsigned use = (unsigned)(it / kMapStages);
+            if (use > 0 && !mbar_wait(&empty_bar[s], (use - 1) & 1u)) {
+                if (lane == 0) atomicOr(&g_quantize_timeout, 1);
+                for (int64_t j = it - 1; j >= 0 && j > it - 1 - kMapStages; --j)
+                    mbar_wait(&full_bar[j % kMapStages], (unsigned)(j / kMapStages) & 1u);
+                return;
+            }
+            prod.build(st[s].qa, QB ? st[s].qb : nullptr, span, last);
+            __syncwarp();
+            if (lane == 0) {
+                mbar_expect_tx(&full_bar[s], (unsigned)sizeof(SpanRowMap));
+                bulk_copy_g2s(&st[s].map, maps + span, (unsigned)sizeof(SpanRowMap), &full_bar[s]);
+            }
+        }
+        return;
+    }
     if (warp == kMapConsumers) {
         // ---- producer
         MapProducer<true, UNS, true, BC> prod;
@@ -826,7 +902,7 @@ dequantize_map_kernel(const uint8_t* __restrict__ codes, const uint8_t* __restri
             const int s = (int)(it % kMapStages);
             const unsigned use = (unsigned)(it / kMapStages);
             if (use > 0 && !mbar_wait(&empty_bar[s], (use - 1) & 1u)) {
-                if (lane == 0) atomicExch(&g_quantize_timeout, 1);
+                if (lane == 0) atomicOr(&g_quantize_timeout, 1);
                 return;
             }
             const int64_t span_beg = span * kMapSpan, span_end = min(span_beg + kMapSpan, total);
@@ -854,7 +930,7 @@ dequantize_map_kernel(const uint8_t* __restrict__ codes, const uint8_t* __restri
         const int64_t span_beg = span * kMapSpan;
         if (span + 1 < last) load_codes<PACKED>(nxt, codes, mask, span_beg + kMapSpan, total, vec_codes, li0);
         if (!mbar_wait_relaxed(&full_bar[s], use & 1u)) {
-            if (lane == 0) atomicExch(&g_quantize_timeout, 1);
+            if (lane == 0) atomicOr(&g_quantize_timeout, 1);
             return;
         }
         const Stage& S = st[s];
@@ -936,7 +1012,7 @@ __global__ void expire_wait_kernel(int polls) {
         fence_barrier_init();
     }
     __syncwarp();
-    if (!mbar_wait(&bar, 0u, polls) && threadIdx.x == 0) atomicExch(&g_quantize_timeout, 1);
+    if (!mbar_wait(&bar, 0u, polls) && threadIdx.x == 0) atomicOr(&g_quantize_timeout, 1);
 }
 cudaError_t launch_expire_wait(int polls, cudaStream_t stream) {
     expire_wait_kernel<<<1, 32, 0, stream>>>(polls);
@@ -947,7 +1023,7 @@ cudaError_t launch_expire_wait(int polls, cudaStream_t stream) {
 cudaError_t launch_quantize(const float* x, const int64_t* row_offsets, int64_t C, int64_t n,
                             int64_t total, int bits, const float* m, const float* lo,
                             const float* p, uint8_t* codes, uint8_t* mask, float* fake, int layout,
-                            cudaStream_t stream, int64_t shift) {
+                            cudaStream_t stream, int64_t shift, const void* rowmap) {
     const float* xi = nullptr;
     const float* beta = nullptr;
     if (total == 0) return cudaSuccess;
@@ -958,22 +1034,22 @@ cudaError_t launch_quantize(const float* x, const int64_t* row_offsets, int64_t 
     const int vec_in = aligned(x, 16), vec_fake = fake ? aligned(fake, 16) : 0;
     const int vec_codes = packed ? aligned(codes, 4) : aligned(codes, 8);
     const bool long_rows = row_offsets == nullptr && n >= kMapSpan;   // the map follows from n
+    // (maps built ahead of time are of no use where the map follows from the row length)
+    const unsigned char* premap = long_rows ? nullptr : static_cast<const unsigned char*>(rowmap);
+#define PWLQ_LAUNCH_QUANTIZE_AS(PK, FK, UN, LG, PR)                                                \
+    do {                                                                                          \
+        const size_t msmem = sizeof(MapStage<true, FK || UN>) * kMapStages;                       \
+        const SpanGrid g = span_grid((const void*)quantize_map_kernel<PK, FK, UN, LG, PR>,        \
+                                     kMapThreads, msmem, nspans, true);                           \
+        quantize_map_kernel<PK, FK, UN, LG, PR><<<g.grid, kMapThreads, msmem, stream>>>(          \
+            x, rows, total, bits, A, codes, mask, fake, vec_in, vec_fake, vec_codes, g.per_cta,   \
+            premap);                                                                              \
+    } while (0)
 #define PWLQ_LAUNCH_QUANTIZE(PK, FK, UN)                                                          \
     do {                                                                                          \
-        const size_t msmem = sizeof(MapStage<true, FK || UN>) * kMapStages;                     \
-        if (long_rows) {                                                                          \
-            const SpanGrid g = span_grid((const void*)quantize_map_kernel<PK, FK, UN, true>,      \
-                                         kMapThreads, msmem, nspans, true);                       \
-            quantize_map_kernel<PK, FK, UN, true><<<g.grid, kMapThreads, msmem, stream>>>(        \
-                x, rows, total, bits, A, codes, mask, fake, vec_in, vec_fake, vec_codes,          \
-                g.per_cta);                                                                       \
-        } else {                                                                                  \
-            const SpanGrid g = span_grid((const void*)quantize_map_kernel<PK, FK, UN, false>,     \
-                                         kMapThreads, msmem, nspans, true);                       \
-            quantize_map_kernel<PK, FK, UN, false><<<g.grid, kMapThreads, msmem, stream>>>(       \
-                x, rows, total, bits, A, codes, mask, fake, vec_in, vec_fake, vec_codes,          \
-                g.per_cta);                                                                       \
-        }                                                                                         \
+        if (long_rows)   PWLQ_LAUNCH_QUANTIZE_AS(PK, FK, UN, true, false);                        \
+        else if (premap) PWLQ_LAUNCH_QUANTIZE_AS(PK, FK, UN, false, true);                        \
+        else             PWLQ_LAUNCH_QUANTIZE_AS(PK, FK, UN, false, false);                       \
     } while (0)
 #define PWLQ_LAUNCH_QUANTIZE_UN(PK, FK) \
     do { if (lo) PWLQ_LAUNCH_QUANTIZE(PK, FK, true); else PWLQ_LAUNCH_QUANTIZE(PK, FK, false); } while (0)
@@ -981,6 +1057,7 @@ cudaError_t launch_quantize(const float* x, const int64_t* row_offsets, int64_t 
     else        { if (fake) PWLQ_LAUNCH_QUANTIZE_UN(false, true); else PWLQ_LAUNCH_QUANTIZE_UN(false, false); }
 #undef PWLQ_LAUNCH_QUANTIZE_UN
 #undef PWLQ_LAUNCH_QUANTIZE
+#undef PWLQ_LAUNCH_QUANTIZE_AS
     return cudaGetLastError();
 }
 
@@ -988,27 +1065,26 @@ cudaError_t launch_dequantize(const uint8_t* codes, const uint8_t* mask,
                               const int64_t* row_offsets, int64_t C, int64_t n, int64_t total,
                               int bits, const float* m, const float* lo, const float* p, float* y,
                               int layout, cudaStream_t stream, int64_t shift, const float* xi,
-                              const float* beta) {
+                              const float* beta, const void* rowmap) {
     if (total == 0) return cudaSuccess;
     Rows rows{row_offsets, C, n, n > 0 ? 1.0 / (double)n : 0.0, row_offsets ? shift : 0};
     const RowArrays A{m, lo, p, xi, beta};
     const bool packed = (layout == 1 && bits <= 4);
     const int64_t nspans = (total + kQSpan - 1) / kQSpan;
-#define PWLQ_LAUNCH_DEQUANTIZE(PK, UN, BCF)                                                       \
+#define PWLQ_LAUNCH_DEQUANTIZE_AS(PK, UN, LG, BCF, PR)                                             \
     do {                                                                                          \
         const int vc = aligned(codes, PK ? 4 : 8), vo = aligned(y, 16);                           \
         const size_t msmem = sizeof(MapStage<false, UN || BCF>) * kMapStages;                     \
-        if (long_rows) {                                                                          \
-            const SpanGrid g = span_grid((const void*)dequantize_map_kernel<PK, UN, true, BCF>,   \
-                                         kMapThreads, msmem, nspans, true);                       \
-            dequantize_map_kernel<PK, UN, true, BCF><<<g.grid, kMapThreads, msmem, stream>>>(     \
-                codes, mask, rows, total, bits, A, y, vc, vo, g.per_cta);                         \
-        } else {                                                                                  \
-            const SpanGrid g = span_grid((const void*)dequantize_map_kernel<PK, UN, false, BCF>,  \
-                                         kMapThreads, msmem, nspans, true);                       \
-            dequantize_map_kernel<PK, UN, false, BCF><<<g.grid, kMapThreads, msmem, stream>>>(    \
-                codes, mask, rows, total, bits, A, y, vc, vo, g.per_cta);                         \
-        }                                                                                         \
+        const SpanGrid g = span_grid((const void*)dequantize_map_kernel<PK, UN, LG, BCF, PR>,     \
+                                     kMapThreads, msmem, nspans, true);                           \
+        dequantize_map_kernel<PK, UN, LG, BCF, PR><<<g.grid, kMapThreads, msmem, stream>>>(       \
+            codes, mask, rows, total, bits, A, y, vc, vo, g.per_cta, premap);                     \
+    } while (0)
+#define PWLQ_LAUNCH_DEQUANTIZE(PK, UN, BCF)                                                       \
+    do {                                                                                          \
+        if (long_rows)   PWLQ_LAUNCH_DEQUANTIZE_AS(PK, UN, true, BCF, false);                     \
+        else if (premap) PWLQ_LAUNCH_DEQUANTIZE_AS(PK, UN, false, BCF, true);                     \
+        else             PWLQ_LAUNCH_DEQUANTIZE_AS(PK, UN, false, BCF, false);                    \
     } while (0)
 #define PWLQ_LAUNCH_DEQUANTIZE_LONG(PK, UN)                                                       \
     do {                                                                                          \
@@ -1023,6 +1099,7 @@ cudaError_t launch_dequantize(const uint8_t* codes, const uint8_t* mask,
     const bool bc = xi != nullptr;
     const bool very_long = !bc && row_offsets == nullptr && n >= 16 * (int64_t)kMapSpan;
     const bool long_rows = row_offsets == nullptr && n >= kMapSpan;   // the map follows from n
+    const unsigned char* premap = long_rows ? nullptr : static_cast<const unsigned char*>(rowmap);
     if (very_long) {
         if (packed) { if (lo) PWLQ_LAUNCH_DEQUANTIZE_LONG(true, true); else PWLQ_LAUNCH_DEQUANTIZE_LONG(true, false); }
         else        { if (lo) PWLQ_LAUNCH_DEQUANTIZE_LONG(false, true); else PWLQ_LAUNCH_DEQUANTIZE_LONG(false, false); }
@@ -1035,6 +1112,7 @@ cudaError_t launch_dequantize(const uint8_t* codes, const uint8_t* mask,
     }
 #undef PWLQ_LAUNCH_DEQUANTIZE_LONG
 #undef PWLQ_LAUNCH_DEQUANTIZE
+#undef PWLQ_LAUNCH_DEQUANTIZE_AS
     return cudaGetLastError();
 }
 

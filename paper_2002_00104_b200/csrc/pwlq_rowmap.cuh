@@ -18,6 +18,12 @@
 //
 // Spans the map cannot describe (more than kMapSlots rows, or empty rows inside the span) are
 // marked `slow`; consumers then look every value's row up in global memory.
+//
+// The maps depend on the row layout only, not on the values or on the rows' inputs.  A caller
+// that runs several streaming calls over one layout can have them built once, into memory of its
+// own (rowmap_build_kernel, RowMapHeader); the producer of a kernel that is given such maps
+// fetches each span's map with one more bulk copy and only computes the rows' constants, from
+// inputs it requested a span earlier.
 #pragma once
 
 #include "pwlq_common.cuh"
@@ -35,8 +41,26 @@ struct SpanRowMap {
     uint16_t before[kMapWords];   // number of set bits in the words before this one
     int64_t first_row;            // row of slot 0
     int32_t slow;                 // 1: the map does not describe the span
-    int32_t pad;
+    int32_t nrows;                // rows (slots) the map describes; 0 when slow
 };
+static_assert(sizeof(SpanRowMap) % 16 == 0, "maps are moved with bulk copies");
+
+// Maps built ahead of time: a header, then one SpanRowMap per span.
+constexpr uint64_t kRowMapMagic = 0x70776c7170616d31ull;
+constexpr size_t kRowMapHeaderBytes = 256;
+struct RowMapHeader {
+    uint64_t magic;
+    int64_t C, total, n;          // the layout the maps describe (n = 0: ragged rows)
+};
+
+// Whether maps built ahead of time describe this layout (every thread of a CTA asks before it
+// does anything else; the header is 32 bytes that stay in L2).
+__device__ __forceinline__ bool rowmap_matches(const unsigned char* premap, const Rows& rows,
+                                               int64_t total) {
+    const RowMapHeader* h = reinterpret_cast<const RowMapHeader*>(premap);
+    return __ldg(&h->magic) == kRowMapMagic && __ldg(&h->C) == rows.C &&
+           __ldg(&h->total) == total && __ldg(&h->n) == (rows.offsets ? 0 : rows.n);
+}
 
 // Slot of the row that holds position li of the span; `word` returns the bitmap word of li.
 __device__ __forceinline__ int map_slot(const SpanRowMap& M, int li, uint32_t& word) {
@@ -219,6 +243,7 @@ struct MapProducer {
         if (lane == 0) {
             M.first_row = this_rf;
             M.slow = (dup || overflow) ? 1 : 0;
+            M.nrows = (dup || overflow) ? 0 : total_in;
         }
     }
 
@@ -278,6 +303,76 @@ struct MapProducer {
             long_end += rows.n;
             m0 = m1; p0 = p1; lo0 = lo1; x0 = x1; b0 = b1;
             if (PARAMS && rf + 1 < rows.C) load_inputs(rf + 1, m1, p1, lo1, x1, b1);
+        }
+    }
+};
+
+// The producer warp's work when the maps were built ahead of time: it fetches each span's map
+// with a bulk copy (issued by the kernel) and computes the constants of the span's rows.  Lane l
+// holds the first row and the row count of span pre_batch + l; (mn, pn, ...) are the inputs of
+// row (first row of the span that is built next) + lane, requested while the span before it was
+// being built.  Every member function is called by all 32 lanes.
+template <bool PARAMS, bool UNS, bool DEQ = false, bool BC = false>
+struct PreProducer {
+    RowInputs in;
+    float Lf;
+    const SpanRowMap* pre;
+    int64_t pre_batch, pre_first;
+    int pre_rows;
+    float mn, pn, lon, xn, bn;
+
+    __device__ __forceinline__ void load_inputs(int64_t r, float& mv, float& pv, float& lov,
+                                                float& xv, float& bv) const {
+        mv = __ldg(in.m + r);
+        pv = __ldg(in.p + r);
+        lov = 0.0f;
+        if (UNS) lov = __ldg(in.lo + r);
+        xv = 1.0f;
+        bv = 0.0f;
+        if (BC) { xv = __ldg(in.xi + r); bv = __ldg(in.beta + r); }
+    }
+    __device__ __forceinline__ void load_batch(int64_t span0, int64_t last) {
+        const int64_t sp = span0 + (threadIdx.x & 31);
+        pre_batch = span0;
+        pre_first = 0;
+        pre_rows = 0;
+        if (PARAMS && sp < last) {
+            pre_first = __ldg(&pre[sp].first_row);
+            pre_rows = __ldg(&pre[sp].nrows);
+        }
+    }
+    __device__ __forceinline__ void fetch(int64_t span) {
+        if (!PARAMS) return;
+        const int j = (int)(span - pre_batch);
+        const int64_t fr = __shfl_sync(0xffffffffu, pre_first, j);
+        const int nr = __shfl_sync(0xffffffffu, pre_rows, j);
+        const int lane = threadIdx.x & 31;
+        mn = pn = lon = bn = 0.0f;
+        xn = 1.0f;
+        if (lane < nr) load_inputs(fr + lane, mn, pn, lon, xn, bn);
+    }
+    __device__ __forceinline__ void begin(const SpanRowMap* maps, int64_t first, int64_t last) {
+        pre = maps;
+        load_batch(first, last);
+        fetch(first);
+    }
+    // Constants of the rows of `span`; then the inputs of the next span's rows are requested.
+    __device__ __forceinline__ void build(float4* qa, float4* qb, int64_t span, int64_t last) {
+        if (!PARAMS) return;
+        const int lane = threadIdx.x & 31;
+        const int j = (int)(span - pre_batch);
+        const int64_t fr = __shfl_sync(0xffffffffu, pre_first, j);
+        const int nr = __shfl_sync(0xffffffffu, pre_rows, j);
+        if (lane < nr)
+            store_row_consts<DEQ>(qa, qb, lane, UNS ? __fsub_rn(mn, lon) : mn, pn, lon, xn, bn, Lf);
+        for (int k = 32 + lane; k < nr; k += 32) {          // many short rows: fetched now
+            float mv, pv, lov, xv, bv;
+            load_inputs(fr + k, mv, pv, lov, xv, bv);
+            store_row_consts<DEQ>(qa, qb, k, UNS ? __fsub_rn(mv, lov) : mv, pv, lov, xv, bv, Lf);
+        }
+        if (span + 1 < last) {
+            if (span + 1 - pre_batch == 32) load_batch(span + 1, last);
+            fetch(span + 1);
         }
     }
 };

@@ -39,6 +39,11 @@ _SIGNATURES = {
     "pwlq_quantize_ragged": (_INT, [_P, _P, _I64, _I64, _INT, _P, _P, _P, _P, _P, _INT, _P]),
     "pwlq_dequantize": (_INT, [_P, _P, _I64, _I64, _INT, _P, _P, _P, _INT, _P]),
     "pwlq_dequantize_ragged": (_INT, [_P, _P, _P, _I64, _I64, _INT, _P, _P, _P, _INT, _P]),
+    "pwlq_rowmap_bytes": (_SZ, [_I64]),
+    "pwlq_rowmap_build": (_INT, [_P, _I64, _I64, _I64, _P, _SZ, _P]),
+    "pwlq_absmax_mapped": (_INT, [_P, _P, _I64, _I64, _I64, _P, _P, _P]),
+    "pwlq_quantize_mapped": (_INT, [_P, _P, _I64, _I64, _I64, _P, _INT, _P, _P, _P, _P, _P, _INT, _P]),
+    "pwlq_dequantize_mapped": (_INT, [_P, _P, _P, _I64, _I64, _I64, _P, _INT, _P, _P, _P, _INT, _P]),
     "pwlq_minmax": (_INT, [_P, _I64, _I64, _P, _P, _P]),
     "pwlq_minmax_ragged": (_INT, [_P, _P, _I64, _I64, _P, _P, _P]),
     "pwlq_search_unsigned": (_INT, [_P, _I64, _I64, _INT, _P, _INT, _P, _P, _P, _P, _P, _P, _P, _SZ,
@@ -116,7 +121,8 @@ def exported_symbols():
 
 def device_status() -> int:
     """0, or 1 << ERR_TIMEOUT if a bounded device wait has expired on the current device since
-    the previous call (synchronises; reading clears the flag)."""
+    the previous call, 1 << ERR_INVALID_ARG if a call was given row maps of another layout
+    (synchronises; reading clears the flags)."""
     return int(load_library().pwlq_device_status())
 
 
@@ -166,11 +172,36 @@ def code_bytes(total: int, bits: int, layout: int) -> int:
     return (total + 1) // 2 if (layout == CODES_PACKED and bits <= 4) else total
 
 
-def absmax(x, row_offsets=None, out=None, stream=None):
+def rowmap_bytes(total: int) -> int:
+    return int(load_library().pwlq_rowmap_bytes(int(total)))
+
+
+def rowmap_build(C, total, row_offsets=None, n=0, device=None, out=None, stream=None):
+    """Row maps of a layout (``pwlq_rowmap_build``) in a uint8 tensor, for the ``rowmap=``
+    argument of ``absmax`` / ``quantize`` / ``dequantize``."""
+    lib = load_library()
+    need = rowmap_bytes(total)
+    if out is None:
+        dev = device if device is not None else row_offsets.device
+        out = torch.empty(max(need, 16), dtype=torch.uint8, device=dev)
+    rc = lib.pwlq_rowmap_build(_dev(row_offsets, torch.int64, "row_offsets"), int(C), int(n),
+                               int(total), _dev(out, torch.uint8, "rowmap"), out.numel(),
+                               _stream(stream))
+    _check(rc, "pwlq_rowmap_build")
+    return out
+
+
+def absmax(x, row_offsets=None, out=None, stream=None, rowmap=None):
     lib = load_library()
     C, n, total = _shape(x, row_offsets)
     m = out if out is not None else torch.empty(C, dtype=torch.float32, device=x.device)
-    if row_offsets is None:
+    if rowmap is not None:
+        rc = lib.pwlq_absmax_mapped(_dev(x, torch.float32, "x"),
+                                    _dev(row_offsets, torch.int64, "row_offsets"), C,
+                                    0 if row_offsets is not None else n, total,
+                                    _dev(rowmap, torch.uint8, "rowmap"),
+                                    _dev(m, torch.float32, "out"), _stream(stream))
+    elif row_offsets is None:
         rc = lib.pwlq_absmax(_dev(x, torch.float32, "x"), C, n, _dev(m, torch.float32, "out"),
                              _stream(stream))
     else:
@@ -315,7 +346,7 @@ def search_status(workspace) -> int:
 
 
 def quantize(x, bits, m, p, layout=CODES_U8, row_offsets=None, want_fake=False, out=None,
-             stream=None):
+             stream=None, rowmap=None):
     """Returns (codes uint8, region_mask uint8, fake fp32 or None)."""
     lib = load_library()
     C, n, total = _shape(x, row_offsets)
@@ -328,7 +359,12 @@ def quantize(x, bits, m, p, layout=CODES_U8, row_offsets=None, want_fake=False, 
     tail = (int(bits), _dev(m, torch.float32, "m"), _dev(p, torch.float32, "p"),
             _dev(codes, torch.uint8, "codes"), _dev(mask, torch.uint8, "mask"),
             _dev(fake, torch.float32, "fake"), int(layout), _stream(stream))
-    if row_offsets is None:
+    if rowmap is not None:
+        rc = lib.pwlq_quantize_mapped(_dev(x, torch.float32, "x"),
+                                      _dev(row_offsets, torch.int64, "row_offsets"), C,
+                                      0 if row_offsets is not None else n, total,
+                                      _dev(rowmap, torch.uint8, "rowmap"), *tail)
+    elif row_offsets is None:
         rc = lib.pwlq_quantize(_dev(x, torch.float32, "x"), C, n, *tail)
     else:
         rc = lib.pwlq_quantize_ragged(_dev(x, torch.float32, "x"),
@@ -338,7 +374,7 @@ def quantize(x, bits, m, p, layout=CODES_U8, row_offsets=None, want_fake=False, 
 
 
 def dequantize(codes, mask, bits, m, p, C=None, n=None, layout=CODES_U8, row_offsets=None,
-               out=None, stream=None):
+               out=None, stream=None, rowmap=None):
     lib = load_library()
     if row_offsets is None:
         total = int(C) * int(n)
@@ -348,7 +384,13 @@ def dequantize(codes, mask, bits, m, p, C=None, n=None, layout=CODES_U8, row_off
     y = out if out is not None else torch.empty(total, dtype=torch.float32, device=codes.device)
     tail = (int(bits), _dev(m, torch.float32, "m"), _dev(p, torch.float32, "p"),
             _dev(y, torch.float32, "y"), int(layout), _stream(stream))
-    if row_offsets is None:
+    if rowmap is not None:
+        rc = lib.pwlq_dequantize_mapped(_dev(codes, torch.uint8, "codes"),
+                                        _dev(mask, torch.uint8, "mask"),
+                                        _dev(row_offsets, torch.int64, "row_offsets"), int(C),
+                                        0 if row_offsets is not None else int(n), total,
+                                        _dev(rowmap, torch.uint8, "rowmap"), *tail)
+    elif row_offsets is None:
         rc = lib.pwlq_dequantize(_dev(codes, torch.uint8, "codes"), _dev(mask, torch.uint8, "mask"),
                                  int(C), int(n), *tail)
     else:

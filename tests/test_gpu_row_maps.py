@@ -114,3 +114,68 @@ def test_dense_rows_around_the_span(pwlq, oracle, C, n):
     y = pwlq.dequantize(codes, mask, 4, m, dev(p), C=C, n=n, layout=1)
     assert np_(y).tobytes() == of.tobytes()
     assert pwlq.device_status() == 0
+
+
+# ---------------------------------------------------------------- maps built once per layout
+@pytest.mark.parametrize("bits,layout", [(3, 1), (8, 0)])
+@pytest.mark.parametrize("name", sorted(layouts()))
+def test_calls_with_prebuilt_maps_match_the_oracle(pwlq, oracle, name, bits, layout):
+    """pwlq_rowmap_build once, then abs-max, quantize (with and without the reconstructed
+    values) and dequantize through the *_mapped entry points: bit for bit the oracle's results."""
+    x, ro = make(layouts()[name], 9)
+    total, C = x.size, ro.size - 1
+    dro = dev(ro)
+    rowmap = pwlq.rowmap_build(C, total, row_offsets=dro)
+    assert rowmap.numel() >= pwlq.rowmap_bytes(total)
+    m = pwlq.absmax(dev(x), row_offsets=dro, rowmap=rowmap)
+    om = oracle.absmax(x, ro)
+    assert np.array_equal(np_(m), om)
+    rng = np.random.default_rng(4)
+    p = (om * rng.uniform(0.05, 1.0, om.size)).astype(np.float32)
+    p[::5] = om[::5]
+    oc, ok, of = oracle.quantize(x, bits, om, p, layout=layout, row_offsets=ro)
+    for want_fake in (True, False):
+        codes, mask, fake = pwlq.quantize(dev(x), bits, m, dev(p), layout=layout, row_offsets=dro,
+                                          want_fake=want_fake, rowmap=rowmap)
+        assert np.array_equal(np_(codes), oc) and np.array_equal(np_(mask), ok)
+        if want_fake:
+            assert np_(fake).tobytes() == of.tobytes()
+    y = pwlq.dequantize(codes, mask, bits, m, dev(p), layout=layout, row_offsets=dro, rowmap=rowmap)
+    assert np_(y).tobytes() == of.tobytes()
+    assert pwlq.device_status() == 0
+
+
+@pytest.mark.parametrize("C,n", [(5000, 1), (700, 7), (520, 9), (300, 147), (3, 4095), (3, 4097)])
+def test_prebuilt_maps_of_dense_rows(pwlq, oracle, C, n):
+    rng = np.random.default_rng(C + n)
+    x = (rng.standard_normal((C, n)) * rng.uniform(0.01, 3.0, (C, 1))).astype(np.float32)
+    dx = dev(x)
+    rowmap = pwlq.rowmap_build(C, C * n, n=n, device=dx.device)
+    m = pwlq.absmax(dx, rowmap=rowmap)
+    om = oracle.absmax(x)
+    assert np.array_equal(np_(m), om)
+    p = (om * np.float32(0.3)).astype(np.float32)
+    codes, mask, fake = pwlq.quantize(dx, 4, m, dev(p), layout=1, want_fake=True, rowmap=rowmap)
+    oc, ok, of = oracle.quantize(x, 4, om, p, layout=1)
+    assert np.array_equal(np_(codes), oc) and np.array_equal(np_(mask), ok)
+    assert np_(fake).tobytes() == of.tobytes()
+    y = pwlq.dequantize(codes, mask, 4, m, dev(p), C=C, n=n, layout=1, rowmap=rowmap)
+    assert np_(y).tobytes() == of.tobytes()
+    assert pwlq.device_status() == 0
+
+
+def test_maps_of_another_layout_are_reported(pwlq):
+    """Maps built for other rows make the call a no-op that the device status names."""
+    x, ro = make([300] * 40, 1)
+    other = np.concatenate([[0], np.cumsum([200] * 40)]).astype(np.int64)
+    rowmap = pwlq.rowmap_build(40, int(other[-1]), row_offsets=dev(other))
+    assert pwlq.device_status() == 0
+    m = torch.full((40,), -1.0, dtype=torch.float32, device="cuda")
+    pwlq.absmax(dev(x), row_offsets=dev(ro), rowmap=rowmap, out=m)
+    torch.cuda.synchronize()
+    assert pwlq.device_status() == 1 << pwlq.ERR_INVALID_ARG
+    assert pwlq.device_status() == 0                    # read and cleared
+    # too small a buffer is refused on the host
+    small = torch.empty(64, dtype=torch.uint8, device="cuda")
+    with pytest.raises(Exception):
+        pwlq.rowmap_build(40, x.size, row_offsets=dev(ro), out=small)
