@@ -356,6 +356,15 @@ int pwlq_encode_host(const float* x_host, const int64_t* row_offsets_host, int64
                      uint8_t* codes_host, uint8_t* region_mask_host, int code_layout,
                      void* dev_scratch, size_t dev_scratch_bytes, float** y_dev_out,
                      void* stream);
+/* The same for one-sided ranges (pwlq_minmax, pwlq_search_unsigned, pwlq_quantize_unsigned,
+ * pwlq_dequantize_unsigned): lo_host / hi_host [C] receive the rows' lower and upper bounds;
+ * everything else as in pwlq_encode_host (same scratch size). */
+int pwlq_encode_host_unsigned(const float* x_host, const int64_t* row_offsets_host, int64_t C,
+                              int64_t total, int64_t max_n, int bits, const float* ratios_host,
+                              int K, float* lo_host, float* hi_host, float* p_host,
+                              float* err_host, int32_t* idx_host, uint8_t* codes_host,
+                              uint8_t* region_mask_host, int code_layout, void* dev_scratch,
+                              size_t dev_scratch_bytes, float** y_dev_out, void* stream);
 
 /* No counterpart in the paper: a packaging variant of pwlq_search for callers that cannot
  * allocate device memory -- for example a plugin inside an application whose own memory pool

@@ -439,8 +439,9 @@ cudaError_t launch_absmax(const float* x, const int64_t* row_offsets, int64_t C,
 }
 
 cudaError_t launch_minmax(const float* x, const int64_t* row_offsets, int64_t C, int64_t n,
-                          int64_t total, float* lo_out, float* hi_out, cudaStream_t stream) {
-    cudaError_t e = launch_fold<true>(x, row_offsets, C, n, total, hi_out, lo_out, stream, 0, nullptr);
+                          int64_t total, float* lo_out, float* hi_out, cudaStream_t stream,
+                          int64_t shift) {
+    cudaError_t e = launch_fold<true>(x, row_offsets, C, n, total, hi_out, lo_out, stream, shift, nullptr);
     if (e != cudaSuccess) return e;
     minmax_finalize_kernel<<<(unsigned)((C + 255) / 256), 256, 0, stream>>>(
         reinterpret_cast<uint32_t*>(lo_out), reinterpret_cast<uint32_t*>(hi_out), C);

@@ -113,7 +113,7 @@ inline size_t code_bytes(int64_t total, int bits, int layout) {
 
 // Layout of the device scratch of pwlq_encode_host (every block 256-byte aligned).
 struct HostPlan {
-    size_t x, ro, ratios, m, p, err, idx, codes, mask, y, ws, bytes;
+    size_t x, ro, ratios, m, lo, p, err, idx, codes, mask, y, ws, bytes;
     pwlq::SearchPlan sp;
 };
 HostPlan plan_host(int64_t C, int64_t total, int64_t max_n, int K) {
@@ -124,6 +124,7 @@ HostPlan plan_host(int64_t C, int64_t total, int64_t max_n, int K) {
     h.ro = take(sizeof(int64_t) * (size_t)(C + 1));
     h.ratios = take(sizeof(float) * (size_t)K);
     h.m = take(sizeof(float) * (size_t)C);
+    h.lo = take(sizeof(float) * (size_t)C);            // lower bounds (one-sided form only)
     h.p = take(sizeof(float) * (size_t)C);
     h.err = take(sizeof(float) * (size_t)C);
     h.idx = take(sizeof(int32_t) * (size_t)C);
@@ -622,12 +623,14 @@ size_t pwlq_encode_host_scratch_bytes(int64_t C, int64_t total, int64_t max_n, i
     return plan_host(C, total, max_n, K).bytes;
 }
 
-int pwlq_encode_host(const float* x_host, const int64_t* row_offsets_host, int64_t C,
-                     int64_t total, int64_t max_n, int bits, const float* ratios_host, int K,
-                     float* m_host, float* p_host, float* err_host, int32_t* idx_host,
-                     uint8_t* codes_host, uint8_t* region_mask_host, int code_layout,
-                     void* dev_scratch, size_t dev_scratch_bytes, float** y_dev_out,
-                     void* stream) {
+// lo_host == nullptr: signed scheme, m_host receives the abs-max values; otherwise one-sided ranges,
+// lo_host / m_host receive the rows' lower / upper bounds.
+static int encode_host_impl(const float* x_host, const int64_t* row_offsets_host, int64_t C,
+                            int64_t total, int64_t max_n, int bits, const float* ratios_host,
+                            int K, float* lo_host, float* m_host, float* p_host, float* err_host,
+                            int32_t* idx_host, uint8_t* codes_host, uint8_t* region_mask_host,
+                            int code_layout, void* dev_scratch, size_t dev_scratch_bytes,
+                            float** y_dev_out, void* stream) {
     if (int rc = check_rows(C, total)) return rc;
     if (!x_host || !ratios_host || !m_host || !p_host || !idx_host || !codes_host ||
         !region_mask_host || bits < 2 || bits > 8 || K < 1 || max_n < 1 || max_n > total ||
@@ -648,6 +651,7 @@ int pwlq_encode_host(const float* x_host, const int64_t* row_offsets_host, int64
     int64_t* dro = row_offsets_host ? reinterpret_cast<int64_t*>(d + h.ro) : nullptr;
     float* dr = reinterpret_cast<float*>(d + h.ratios);
     float* dm = reinterpret_cast<float*>(d + h.m);
+    float* dlo = lo_host ? reinterpret_cast<float*>(d + h.lo) : nullptr;
     float* dp = reinterpret_cast<float*>(d + h.p);
     float* de = reinterpret_cast<float*>(d + h.err);
     int32_t* di = reinterpret_cast<int32_t*>(d + h.idx);
@@ -689,13 +693,15 @@ int pwlq_encode_host(const float* x_host, const int64_t* row_offsets_host, int64
         uint8_t* dck = dc + (packed ? f0 / 2 : f0);
         uint8_t* dkk = dk + f0 / 8;
         if (tk > 0) {
-            PWLQ_TRY(pwlq::launch_absmax(dx + f0, rok, Ck, n, tk, dm + c0, st, f0));
-            PWLQ_TRY(pwlq::launch_search(dx + f0, rok, Ck, n, tk, bits, dr, K, dm + c0, nullptr,
+            float* lok = dlo ? dlo + c0 : nullptr;
+            if (dlo) PWLQ_TRY(pwlq::launch_minmax(dx + f0, rok, Ck, n, tk, lok, dm + c0, st, f0));
+            else     PWLQ_TRY(pwlq::launch_absmax(dx + f0, rok, Ck, n, tk, dm + c0, st, f0));
+            PWLQ_TRY(pwlq::launch_search(dx + f0, rok, Ck, n, tk, bits, dr, K, dm + c0, lok,
                                          dp + c0, de + c0, di + c0, nullptr, d + h.ws, h.sp, st, f0,
                                          k == 0));
-            PWLQ_TRY(pwlq::launch_quantize(dx + f0, rok, Ck, n, tk, bits, dm + c0, nullptr, dp + c0,
+            PWLQ_TRY(pwlq::launch_quantize(dx + f0, rok, Ck, n, tk, bits, dm + c0, lok, dp + c0,
                                            dck, dkk, nullptr, code_layout, st, f0));
-            PWLQ_TRY(pwlq::launch_dequantize(dck, dkk, rok, Ck, n, tk, bits, dm + c0, nullptr,
+            PWLQ_TRY(pwlq::launch_dequantize(dck, dkk, rok, Ck, n, tk, bits, dm + c0, lok,
                                              dp + c0, dy + f0, code_layout, st, f0));
         }
         PWLQ_TRY(cudaEventRecord(hp->out_ready[k], st));
@@ -711,6 +717,9 @@ int pwlq_encode_host(const float* x_host, const int64_t* row_offsets_host, int64
     }
     PWLQ_TRY(cudaMemcpyAsync(m_host, dm, sizeof(float) * (size_t)C, cudaMemcpyDeviceToHost,
                              hp->copy_out));
+    if (lo_host)
+        PWLQ_TRY(cudaMemcpyAsync(lo_host, dlo, sizeof(float) * (size_t)C, cudaMemcpyDeviceToHost,
+                                 hp->copy_out));
     PWLQ_TRY(cudaMemcpyAsync(p_host, dp, sizeof(float) * (size_t)C, cudaMemcpyDeviceToHost,
                              hp->copy_out));
     if (err_host)
@@ -723,6 +732,31 @@ int pwlq_encode_host(const float* x_host, const int64_t* row_offsets_host, int64
 #undef PWLQ_TRY
     if (y_dev_out) *y_dev_out = dy;
     return PWLQ_OK;
+}
+
+int pwlq_encode_host(const float* x_host, const int64_t* row_offsets_host, int64_t C,
+                     int64_t total, int64_t max_n, int bits, const float* ratios_host, int K,
+                     float* m_host, float* p_host, float* err_host, int32_t* idx_host,
+                     uint8_t* codes_host, uint8_t* region_mask_host, int code_layout,
+                     void* dev_scratch, size_t dev_scratch_bytes, float** y_dev_out,
+                     void* stream) {
+    return encode_host_impl(x_host, row_offsets_host, C, total, max_n, bits, ratios_host, K,
+                            nullptr, m_host, p_host, err_host, idx_host, codes_host,
+                            region_mask_host, code_layout, dev_scratch, dev_scratch_bytes,
+                            y_dev_out, stream);
+}
+
+int pwlq_encode_host_unsigned(const float* x_host, const int64_t* row_offsets_host, int64_t C,
+                              int64_t total, int64_t max_n, int bits, const float* ratios_host,
+                              int K, float* lo_host, float* hi_host, float* p_host,
+                              float* err_host, int32_t* idx_host, uint8_t* codes_host,
+                              uint8_t* region_mask_host, int code_layout, void* dev_scratch,
+                              size_t dev_scratch_bytes, float** y_dev_out, void* stream) {
+    if (!lo_host) return PWLQ_ERR_INVALID_ARG;
+    return encode_host_impl(x_host, row_offsets_host, C, total, max_n, bits, ratios_host, K,
+                            lo_host, hi_host, p_host, err_host, idx_host, codes_host,
+                            region_mask_host, code_layout, dev_scratch, dev_scratch_bytes,
+                            y_dev_out, stream);
 }
 
 size_t pwlq_select_workspace_bytes(int64_t C, int64_t n) {

@@ -28,7 +28,8 @@ cudaError_t launch_rowmap_build(const int64_t* row_offsets, int64_t C, int64_t n
 
 // Per-row minimum and maximum (the range [m1, m2] of a one-sided / asymmetric tensor).
 cudaError_t launch_minmax(const float* x, const int64_t* row_offsets, int64_t C, int64_t n,
-                          int64_t total, float* lo_out, float* hi_out, cudaStream_t stream);
+                          int64_t total, float* lo_out, float* hi_out, cudaStream_t stream,
+                          int64_t shift = 0);
 
 struct SearchPlan {
     int64_t max_n;         // longest row

@@ -77,6 +77,8 @@ _SIGNATURES = {
     "pwlq_encode_host_scratch_bytes": (_SZ, [_I64, _I64, _I64, _INT]),
     "pwlq_encode_host": (_INT, [_P, _P, _I64, _I64, _I64, _INT, _P, _INT, _P, _P, _P, _P, _P, _P,
                                 _INT, _P, _SZ, _P, _P]),
+    "pwlq_encode_host_unsigned": (_INT, [_P, _P, _I64, _I64, _I64, _INT, _P, _INT, _P, _P, _P, _P, _P,
+                                         _P, _P, _INT, _P, _SZ, _P, _P]),
     "pwlq_search_noalloc": (_INT, [_P, _I64, _I64, _INT, _P, _INT, _P, _P, _P, _P, _P, _P, _P]),
     "pwlq_search_noalloc_max_bytes": (_SZ, []),
     "pwlq_select_workspace_bytes": (_SZ, [_I64, _I64]),
@@ -680,3 +682,20 @@ def encode_host(x_host, row_offsets_host, C, max_n, bits, ratios_host, out_host,
         _host(out_host["mask"], torch.uint8, "mask"), int(layout),
         _dev(dev_scratch, torch.uint8, "dev_scratch"), dev_scratch.numel(), None, _stream(stream))
     _check(rc, "pwlq_encode_host")
+
+
+def encode_host_unsigned(x_host, row_offsets_host, C, max_n, bits, ratios_host, out_host, layout,
+                         dev_scratch, stream=None):
+    """One-sided form of ``encode_host``; ``out_host`` = dict(lo, hi, p, err, idx, codes, mask)."""
+    lib = load_library()
+    total = x_host.numel()
+    rc = lib.pwlq_encode_host_unsigned(
+        _host(x_host, torch.float32, "x_host"), _host(row_offsets_host, torch.int64, "row_offsets"),
+        int(C), total, int(max_n), int(bits), _host(ratios_host, torch.float32, "ratios"),
+        ratios_host.numel(), _host(out_host["lo"], torch.float32, "lo"),
+        _host(out_host["hi"], torch.float32, "hi"), _host(out_host["p"], torch.float32, "p"),
+        _host(out_host.get("err"), torch.float32, "err"), _host(out_host["idx"], torch.int32, "idx"),
+        _host(out_host["codes"], torch.uint8, "codes"), _host(out_host["mask"], torch.uint8, "mask"),
+        int(layout), _dev(dev_scratch, torch.uint8, "dev_scratch"), dev_scratch.numel(), None,
+        _stream(stream))
+    _check(rc, "pwlq_encode_host_unsigned")

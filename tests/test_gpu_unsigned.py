@@ -183,3 +183,43 @@ def test_unsigned_argument_errors(pwlq):
         pwlq.search_unsigned(x, 4, dev(W.ratio_grid(4)), None, hi)
     with pytest.raises(pwlq.PwlqError):
         pwlq.quantize_unsigned(x, 4, None, hi, hi)
+
+
+@pytest.mark.parametrize("ragged", [False, True])
+def test_encode_host_unsigned_matches_oracle(pwlq, oracle, ragged):
+    """The one-sided form of the host-buffer entry point: min/max, search, quantize and
+    dequantize from pinned host buffers, against the oracle run step by step."""
+    rng = np.random.default_rng(77)
+    if ragged:
+        w = W.small_mixed(seed=29, bits=4, K=64)
+        x = (np.abs(w.x) + np.float32(0.25)).astype(np.float32)
+        ro, C = w.row_offsets, w.C
+    else:
+        x = relu_like(rng, (9, 500), offset=-0.5).reshape(-1)
+        ro, C = None, 9
+    total = x.size
+    max_n = int(np.diff(ro).max()) if ragged else 500
+    ratios = W.ratio_grid(64)
+    hx = torch.from_numpy(x).pin_memory()
+    hro = torch.from_numpy(ro).pin_memory() if ragged else None
+    f32 = lambda n: torch.empty(n, dtype=torch.float32).pin_memory()
+    out = {"lo": f32(C), "hi": f32(C), "p": f32(C), "err": f32(C),
+           "idx": torch.empty(C, dtype=torch.int32).pin_memory(),
+           "codes": torch.empty((total + 1) // 2, dtype=torch.uint8).pin_memory(),
+           "mask": torch.empty((total + 7) // 8, dtype=torch.uint8).pin_memory()}
+    scratch = torch.empty(pwlq.encode_host_scratch_bytes(C, total, max_n, 64), dtype=torch.uint8,
+                          device="cuda")
+    pwlq.encode_host_unsigned(hx, hro, C, max_n, 4, torch.from_numpy(ratios).pin_memory(), out,
+                              pwlq.CODES_PACKED, scratch)
+    torch.cuda.synchronize()
+    xo = x if ragged else x.reshape(C, -1)
+    olo, ohi = oracle.minmax(xo, ro)
+    assert np.array_equal(out["lo"].numpy(), olo) and np.array_equal(out["hi"].numpy(), ohi)
+    ora = oracle.search_u(xo, 4, ratios, olo, ohi, row_offsets=ro)
+    rows = np.arange(C)
+    gi = out["idx"].numpy()
+    gap = np.abs(ora["sse64"][rows, gi] - ora["sse64"][rows, ora["idx"]])
+    assert np.all(gap <= 1e-5 * ora["sse64"][rows, ora["idx"]] + 1e-30)
+    oc, ok, _ = oracle.quantize_u(xo, 4, olo, ohi, out["p"].numpy(), layout=1, row_offsets=ro)
+    assert np.array_equal(out["codes"].numpy(), oc) and np.array_equal(out["mask"].numpy(), ok)
+    assert pwlq.device_status() == 0
