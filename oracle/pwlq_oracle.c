@@ -638,6 +638,152 @@ int pwlq_oracle_dequantize2(const uint8_t *codes, const uint8_t *region2,
 }
 
 /* ------------------------------------------------------------------------------------------
+ * Three breakpoints (Sec. 5.1, "Multiple Breakpoints"; Table 1 of the paper lists one, two and
+ * three).  The reading is the two-breakpoint one with one more region: 0 < p1 < p2 < p3 <= m,
+ * R1 = [0, p1], R2 = (p1, p2], R3 = (p2, p3], R4 = (p3, m]; inside every region (and sign) Eq. 1
+ * with b-1 bits, range [z, z + Delta], offset z = the region's lower end.  Sign-magnitude code as
+ * before; the region index (0..3) fills the two bits per value of the region stream.  The search
+ * takes all triples i < j < k of the K candidate ratios; the first minimal triple in the order
+ * (i, j, k) wins.  With p3 = m the scheme is the two-breakpoint scheme, which is what the tests
+ * pin it to first.
+ */
+typedef struct { float z[4], s[4], inv[4], Lf; } pw3_params;
+
+static pw3_params make_params3(float m, float p1, float p2, float p3, int bits)
+{
+    pw3_params P;
+    float d[4];
+    int r;
+    P.Lf = (float)((1 << (bits - 1)) - 1);
+    P.z[0] = 0.0f; P.z[1] = p1; P.z[2] = p2; P.z[3] = p3;
+    d[0] = p1; d[1] = p2 - p1; d[2] = p3 - p2; d[3] = m - p3;
+    for (r = 0; r < 4; ++r) {
+        if (d[r] > 0.0f) { P.s[r] = d[r] / P.Lf; P.inv[r] = P.Lf / d[r]; }
+        else             { P.s[r] = 0.0f;        P.inv[r] = 0.0f; }
+    }
+    return P;
+}
+
+static float pw3_elem(float x, float m, const pw3_params *P, int *q_out, int *region_out,
+                      float *a_out)
+{
+    float a = fminf(fabsf(x), m);
+    int r = (a > P->z[1]) + (a > P->z[2]) + (a > P->z[3]);
+    float u = a - P->z[r];
+    float t = u * P->inv[r];
+    float q = fminf(rintf(t), P->Lf);
+    float v = q * P->s[r];
+    v = v + P->z[r];
+    *q_out = (int)q;
+    *region_out = r;
+    *a_out = a;
+    return v;
+}
+
+/* sse_f64 (may be NULL): [C, K, K, K], entry (i, j, k) valid for i < j < k, others 0. */
+int pwlq_oracle_search3(const float *x, const int64_t *row_offsets, int64_t C, int64_t n,
+                        int bits, const float *ratios, int K, const float *m_in,
+                        float *p_out /* [C, 3] */, float *err_out, int32_t *idx_out /* [C, 3] */,
+                        double *sse_f64)
+{
+    int64_t c, e, b, t;
+    int i, j, k;
+    if (!x || !ratios || !m_in || C < 1 || K < 3 || bits < 2 || bits > 8) return ORACLE_ERR_ARG;
+    for (c = 0; c < C; ++c) {
+        float m = m_in[c];
+        double best = 0.0;
+        int bi = 0, bj = 1, bk = 2, first = 1;
+        b = row_begin(row_offsets, n, c);
+        e = row_begin(row_offsets, n, c + 1);
+        if (!(m <= 3.402823466e+38f)) return ORACLE_ERR_NONFINITE;
+        for (i = 0; i < K; ++i) for (j = 0; j < K; ++j) for (k = 0; k < K; ++k) {
+            double sse = 0.0;
+            int valid = (i < j && j < k);
+            if (valid && m > 0.0f) {
+                pw3_params P = make_params3(m, m * ratios[i], m * ratios[j], m * ratios[k], bits);
+                for (t = b; t < e; ++t) {
+                    int q, r; float a;
+                    float v = pw3_elem(x[t], m, &P, &q, &r, &a);
+                    double d = (double)v - (double)a;
+                    sse += d * d;
+                }
+            }
+            if (sse_f64) sse_f64[((c * (int64_t)K + i) * K + j) * K + k] = sse;
+            if (valid && (first || sse < best)) { best = sse; bi = i; bj = j; bk = k; first = 0; }
+        }
+        if (idx_out) { idx_out[3 * c] = bi; idx_out[3 * c + 1] = bj; idx_out[3 * c + 2] = bk; }
+        if (p_out) {
+            p_out[3 * c]     = (m > 0.0f) ? m * ratios[bi] : 0.0f;
+            p_out[3 * c + 1] = (m > 0.0f) ? m * ratios[bj] : 0.0f;
+            p_out[3 * c + 2] = (m > 0.0f) ? m * ratios[bk] : 0.0f;
+        }
+        if (err_out) err_out[c] = (float)best;
+    }
+    return ORACLE_OK;
+}
+
+/* p_in: [C, 3] breakpoints p1 <= p2 <= p3 <= m of every row. */
+int pwlq_oracle_quantize3(const float *x, const int64_t *row_offsets, int64_t C, int64_t n,
+                          int bits, const float *m_in, const float *p_in, uint8_t *codes,
+                          uint8_t *region2, float *fake_out, int layout)
+{
+    int64_t c, i, total;
+    int packed = (layout == 1 && bits <= 4);
+    if (!x || !m_in || !p_in || C < 1 || bits < 2 || bits > 8) return ORACLE_ERR_ARG;
+    total = row_begin(row_offsets, n, C);
+    if (codes)   for (i = 0; i < (packed ? (total + 1) / 2 : total); ++i) codes[i] = 0;
+    if (region2) for (i = 0; i < (total + 3) / 4; ++i) region2[i] = 0;
+    for (c = 0; c < C; ++c) {
+        int64_t b = row_begin(row_offsets, n, c), e = row_begin(row_offsets, n, c + 1);
+        float m = m_in[c];
+        pw3_params P = make_params3(m, p_in[3 * c], p_in[3 * c + 1], p_in[3 * c + 2], bits);
+        for (i = b; i < e; ++i) {
+            int q = 0, r = 0, neg = 0, code;
+            float a, v = 0.0f;
+            if (m > 0.0f) {
+                neg = (x[i] < 0.0f);
+                v = pw3_elem(x[i], m, &P, &q, &r, &a);
+            }
+            code = (neg << (bits - 1)) | q;
+            if (codes) {
+                if (packed) codes[i >> 1] |= (uint8_t)(code << ((i & 1) * 4));
+                else        codes[i] = (uint8_t)code;
+            }
+            if (region2) region2[i >> 2] |= (uint8_t)(r << ((i & 3) * 2));
+            if (fake_out) fake_out[i] = neg ? -v : v;
+        }
+    }
+    return ORACLE_OK;
+}
+
+int pwlq_oracle_dequantize3(const uint8_t *codes, const uint8_t *region2,
+                            const int64_t *row_offsets, int64_t C, int64_t n, int bits,
+                            const float *m_in, const float *p_in, float *y, int layout)
+{
+    int64_t c, i;
+    int packed = (layout == 1 && bits <= 4);
+    int qmask = (1 << (bits - 1)) - 1;
+    if (!codes || !region2 || !m_in || !p_in || !y || C < 1 || bits < 2 || bits > 8)
+        return ORACLE_ERR_ARG;
+    for (c = 0; c < C; ++c) {
+        int64_t b = row_begin(row_offsets, n, c), e = row_begin(row_offsets, n, c + 1);
+        float m = m_in[c];
+        pw3_params P = make_params3(m, p_in[3 * c], p_in[3 * c + 1], p_in[3 * c + 2], bits);
+        for (i = b; i < e; ++i) {
+            int code = packed ? ((codes[i >> 1] >> ((i & 1) * 4)) & 0xF) : codes[i];
+            int r = (region2[i >> 2] >> ((i & 3) * 2)) & 3;
+            int neg = (code >> (bits - 1)) & 1;
+            float q = (float)(code & qmask);
+            float v = q * P.s[r];
+            v = v + P.z[r];
+            if (!(m > 0.0f)) { v = 0.0f; neg = 0; }
+            y[i] = neg ? -v : v;
+        }
+    }
+    return ORACLE_OK;
+}
+
+/* ------------------------------------------------------------------------------------------
  * Bias correction (Sec. 5.1, "Bias Correction"): quantization shifts the mean and the variance of
  * a row; the paper compensates this by folding correction terms into the scale and the offset,
  * citing earlier work, and prints no formula.  Reading taken here: with y_i = pw(x_i) the

@@ -101,6 +101,12 @@ class OracleLib:
                                             P, P, P, P, P]
         lib.pwlq_oracle_quantize2.argtypes = [P, P, I64, I64, ctypes.c_int, P, P, P, P, P, P,
                                               ctypes.c_int]
+        lib.pwlq_oracle_search3.argtypes = [P, P, I64, I64, ctypes.c_int, P, ctypes.c_int, P, P, P,
+                                            P, P]
+        lib.pwlq_oracle_quantize3.argtypes = [P, P, I64, I64, ctypes.c_int, P, P, P, P, P,
+                                              ctypes.c_int]
+        lib.pwlq_oracle_dequantize3.argtypes = [P, P, P, I64, I64, ctypes.c_int, P, P, P,
+                                                ctypes.c_int]
         lib.pwlq_oracle_dequantize2.argtypes = [P, P, P, I64, I64, ctypes.c_int, P, P, P, P,
                                                 ctypes.c_int]
         lib.pwlq_oracle_bias_correction.argtypes = [P, P, I64, I64, ctypes.c_int, P, P, P, P]
@@ -309,6 +315,55 @@ class OracleLib:
         _check(self._lib.pwlq_oracle_dequantize2(_ptr(codes), _ptr(region), _ptr(ro), C, n,
                                                  int(bits), _ptr(m), _ptr(p1), _ptr(p2), _ptr(y),
                                                  int(layout)), "dequantize2")
+        return y
+
+    # ---- three breakpoints: four regions, region index 0..3 in the two bits per value
+    def search3(self, x, bits, ratios, m, row_offsets=None, want_sse=True):
+        """Returns dict(p [C,3], err, idx [C,3], sse64 [C,K,K,K] (entries i < j < k valid))."""
+        flat, ro, C, n = _rows(x, row_offsets)
+        ratios = np.ascontiguousarray(ratios, dtype=np.float32)
+        K = int(ratios.size)
+        m = np.ascontiguousarray(m, dtype=np.float32)
+        assert m.size == C
+        p = np.empty((C, 3), dtype=np.float32)
+        err = np.empty(C, dtype=np.float32)
+        idx = np.empty((C, 3), dtype=np.int32)
+        sse64 = np.empty((C, K, K, K), dtype=np.float64) if want_sse else None
+        _check(self._lib.pwlq_oracle_search3(_ptr(flat), _ptr(ro), C, n, int(bits), _ptr(ratios),
+                                             K, _ptr(m), _ptr(p), _ptr(err), _ptr(idx),
+                                             _ptr(sse64)), "search3")
+        return {"p": p, "err": err, "idx": idx, "sse64": sse64}
+
+    def quantize3(self, x, bits, m, p, layout=0, row_offsets=None, want_fake=True):
+        """p: [C, 3].  Returns (codes uint8, region2 uint8 (two bits per value), fake or None)."""
+        flat, ro, C, n = _rows(x, row_offsets)
+        total = flat.size
+        m = np.ascontiguousarray(m, dtype=np.float32)
+        p = np.ascontiguousarray(p, dtype=np.float32).reshape(-1, 3)
+        assert m.size == C and p.shape[0] == C
+        codes = np.empty(code_bytes(total, bits, layout), dtype=np.uint8)
+        region = np.empty((total + 3) // 4, dtype=np.uint8)
+        fake = np.empty(total, dtype=np.float32) if want_fake else None
+        _check(self._lib.pwlq_oracle_quantize3(_ptr(flat), _ptr(ro), C, n, int(bits), _ptr(m),
+                                               _ptr(p), _ptr(codes), _ptr(region), _ptr(fake),
+                                               int(layout)), "quantize3")
+        return codes, region, fake
+
+    def dequantize3(self, codes, region, bits, m, p, C=None, n=None, layout=0, row_offsets=None):
+        codes = np.ascontiguousarray(codes, dtype=np.uint8)
+        region = np.ascontiguousarray(region, dtype=np.uint8)
+        m = np.ascontiguousarray(m, dtype=np.float32)
+        p = np.ascontiguousarray(p, dtype=np.float32).reshape(-1, 3)
+        if row_offsets is not None:
+            ro = np.ascontiguousarray(row_offsets, dtype=np.int64)
+            C, n, total = ro.size - 1, 0, int(ro[-1])
+        else:
+            ro, total = None, int(C) * int(n)
+        assert m.size == C and p.shape[0] == C
+        y = np.empty(total, dtype=np.float32)
+        _check(self._lib.pwlq_oracle_dequantize3(_ptr(codes), _ptr(region), _ptr(ro), C, n,
+                                                 int(bits), _ptr(m), _ptr(p), _ptr(y),
+                                                 int(layout)), "dequantize3")
         return y
 
     # ---- bias correction (folded scale xi and offset beta per row) and dense (b+1)-bit storage

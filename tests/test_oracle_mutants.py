@@ -8,6 +8,7 @@ import pytest
 import test_oracle_pins as pins
 import test_oracle_bias_and_packing_pins as bpins
 import test_oracle_two_breakpoints_pins as tpins
+import test_oracle_three_breakpoints_pins as t3pins
 import test_oracle_unsigned_pins as upins
 
 ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
@@ -60,6 +61,19 @@ MUTANTS = {
     "two_bp_region_bit_order": ("region2[i >> 2] |= (uint8_t)(r << ((i & 3) * 2));",
                                 "region2[i >> 2] |= (uint8_t)(r << ((3 - (i & 3)) * 2));"),
     "two_bp_pairs_not_ordered": ("if (i < j && m > 0.0f) {", "if (i != j && m > 0.0f) {"),
+    "three_bp_region_closed_at_p3": ("int r = (a > P->z[1]) + (a > P->z[2]) + (a > P->z[3]);",
+                                     "int r = (a > P->z[1]) + (a > P->z[2]) + (a >= P->z[3]);"),
+    "three_bp_third_range": ("d[0] = p1; d[1] = p2 - p1; d[2] = p3 - p2; d[3] = m - p3;",
+                             "d[0] = p1; d[1] = p2 - p1; d[2] = p3 - p1; d[3] = m - p3;"),
+    "three_bp_fourth_offset": ("P.z[0] = 0.0f; P.z[1] = p1; P.z[2] = p2; P.z[3] = p3;",
+                               "P.z[0] = 0.0f; P.z[1] = p1; P.z[2] = p2; P.z[3] = p2;"),
+    "three_bp_last_triple_on_ties": ("if (valid && (first || sse < best))",
+                                     "if (valid && (first || sse <= best))"),
+    "three_bp_triples_not_ordered": ("int valid = (i < j && j < k);", "int valid = (i < j && i < k && j != k);"),
+    "three_bp_breakpoints_swapped": ("make_params3(m, m * ratios[i], m * ratios[j], m * ratios[k], bits);",
+                                     "make_params3(m, m * ratios[i], m * ratios[k], m * ratios[j], bits);"),
+    "three_bp_dequant_region_capped": ("            float v = q * P.s[r];\n            v = v + P.z[r];\n            if (!(m > 0.0f)) { v = 0.0f; neg = 0; }\n            y[i] = neg ? -v : v;\n        }\n    }\n    return ORACLE_OK;\n}\n\n/* ------------------------------------------------------------------------------------------\n * Bias",
+                                       "            float v = q * P.s[r > 2 ? 2 : r];\n            v = v + P.z[r > 2 ? 2 : r];\n            if (!(m > 0.0f)) { v = 0.0f; neg = 0; }\n            y[i] = neg ? -v : v;\n        }\n    }\n    return ORACLE_OK;\n}\n\n/* ------------------------------------------------------------------------------------------\n * Bias"),
     "bc_ratio_inverted": ("xi = sqrt(vx / vy);", "xi = sqrt(vy / vx);"),
     "bc_variance_ratio_without_sqrt": ("xi = sqrt(vx / vy);", "xi = (vx / vy);"),
     "bc_offset_sign": ("beta_out[c] = (float)(mx - xi * my);", "beta_out[c] = (float)(mx + xi * my);"),
@@ -99,6 +113,10 @@ PIN_CALLS = [
     lambda o: tpins.test_second_breakpoint_at_m_is_the_one_breakpoint_scheme(o, 3),
     lambda o: tpins.test_pair_order_and_degenerate_rows(o),
     lambda o: tpins.test_half_step_bound_per_region(o, 4),
+    lambda o: t3pins.test_worked_example_three_breakpoints(o),
+    lambda o: t3pins.test_third_breakpoint_at_m_is_the_two_breakpoint_scheme(o, 3),
+    lambda o: t3pins.test_triple_order_and_degenerate_rows(o),
+    lambda o: t3pins.test_half_step_bound_per_region_three_breakpoints(o, 4),
     lambda o: bpins.test_corrected_rows_keep_mean_and_centred_norm(o, 4),
     lambda o: bpins.test_hand_computed_row(o),
     lambda o: bpins.test_dequantize_with_correction_applies_scale_then_offset(o),
