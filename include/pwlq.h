@@ -240,8 +240,9 @@ int pwlq_dequantize_unsigned_ragged(const uint8_t* codes, const uint8_t* region_
  *
  * pwlq_search2: for every row, all pairs i < j of the K candidate ratios (ascending, K in
  * [2, PWLQ_MAX_K2]), p1 = m * ratios[i], p2 = m * ratios[j]; squared error summed as in
- * pwlq_search; the first minimal pair in the order (i, j) wins.  Rows are limited to 8192 values
- * (PWLQ_ERR_UNSUPPORTED beyond).  m (device, [C]) is required.
+ * pwlq_search; the first minimal pair in the order (i, j) wins.  Rows of more than 8192 values are
+ * cut into tiles whose terms are added in ascending tile order (reproducible).  m (device, [C]) is
+ * required.
  *   p1_out, p2_out, idx1_out, idx2_out   device, [C]; err_out device [C] or NULL
  *   sse_pairs   device, [C, K, K] or NULL; entry (i, j) is written with the sum for i < j, 0 otherwise
  *   workspace   device, 256-byte aligned, pwlq_search2_workspace_bytes(...) bytes; its first word
@@ -274,6 +275,44 @@ int pwlq_dequantize2_ragged(const uint8_t* codes, const uint8_t* region2,
                             const int64_t* row_offsets, int64_t C, int64_t total, int bits,
                             const float* m, const float* p1, const float* p2, float* y,
                             int code_layout, void* stream);
+
+/* Three breakpoints (Sec. 5.1 "Multiple Breakpoints"; Table 1 of the paper compares one, two and
+ * three).  The same reading with one more region: 0 < p1 < p2 < p3 <= m, regions [0, p1],
+ * (p1, p2], (p2, p3], (p3, m], each quantized by Eq. 1 with b-1 bits and offset z = its lower
+ * end; the region index 0..3 fills the two bits per value of region2.  With p3 = m the scheme is
+ * the two-breakpoint one.
+ *
+ * pwlq_search3: all triples i < j < k of the K candidate ratios (ascending, K in [3, PWLQ_MAX_K2]);
+ * the first minimal triple in the order (i, j, k) wins.  The error of a triple is the sum of its
+ * four regions' errors, which share their terms with the pair search: the cost is that of
+ * pwlq_search2 plus O(K^2) per row, not K^3 / 6 evaluations.
+ *   p_out, idx_out   device, [C, 3] (the three breakpoints / grid indices of a row side by side)
+ *   err_out          device [C] or NULL
+ *   sse_triples      device, [C, K, K, K] or NULL; entry (i, j, k) holds the sum for i < j < k,
+ *                    0 otherwise (meant for small K: K^3 floats per row)
+ *   workspace        as for pwlq_search2 (pwlq_search2_workspace_bytes)
+ * A row with m = 0 or no values gets indices (0, 1, 2), p = 0, error 0.
+ * pwlq_quantize3 / pwlq_dequantize3 take the breakpoints as one [C, 3] array p. */
+int pwlq_search3(const float* x, int64_t C, int64_t n, int bits, const float* ratios, int K,
+                 const float* m, float* p_out, float* err_out, int32_t* idx_out,
+                 float* sse_triples, void* workspace, size_t workspace_bytes, void* stream);
+int pwlq_search3_ragged(const float* x, const int64_t* row_offsets, int64_t C, int64_t total,
+                        int64_t max_n, int bits, const float* ratios, int K, const float* m,
+                        float* p_out, float* err_out, int32_t* idx_out, float* sse_triples,
+                        void* workspace, size_t workspace_bytes, void* stream);
+int pwlq_quantize3(const float* x, int64_t C, int64_t n, int bits, const float* m, const float* p,
+                   uint8_t* codes, uint8_t* region2, float* fake_out, int code_layout,
+                   void* stream);
+int pwlq_quantize3_ragged(const float* x, const int64_t* row_offsets, int64_t C, int64_t total,
+                          int bits, const float* m, const float* p, uint8_t* codes,
+                          uint8_t* region2, float* fake_out, int code_layout, void* stream);
+int pwlq_dequantize3(const uint8_t* codes, const uint8_t* region2, int64_t C, int64_t n,
+                     int bits, const float* m, const float* p, float* y, int code_layout,
+                     void* stream);
+int pwlq_dequantize3_ragged(const uint8_t* codes, const uint8_t* region2,
+                            const int64_t* row_offsets, int64_t C, int64_t total, int bits,
+                            const float* m, const float* p, float* y, int code_layout,
+                            void* stream);
 
 /* Bias correction (Sec. 5.1, "Bias Correction"): quantization shifts the mean and the variance of
  * a row; the paper compensates this by folding correction terms into the scale and the offset and

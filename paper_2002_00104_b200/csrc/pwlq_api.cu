@@ -412,27 +412,30 @@ int pwlq_dequantize_unsigned_ragged(const uint8_t* codes, const uint8_t* region_
 }
 
 size_t pwlq_search2_workspace_bytes(int64_t C, int64_t max_n, int K) {
-    if (C < 1 || max_n < 1 || max_n > pwlq::kSearchTile || K < 2 || K > PWLQ_MAX_K2) return 0;
-    return 256;
+    if (C < 1 || max_n < 1 || K < 2 || K > PWLQ_MAX_K2) return 0;
+    return pwlq::search2_workspace_bytes(C, max_n, K);
 }
 
-static int search2_impl(const float* x, const int64_t* ro, int64_t C, int64_t n, int64_t total,
-                        int64_t max_n, int bits, const float* ratios, int K, const float* m,
-                        float* p1_out, float* p2_out, float* err_out, int32_t* idx1_out,
-                        int32_t* idx2_out, float* sse_pairs, void* ws, size_t ws_bytes,
-                        void* stream) {
-    if (!x || !ratios || !m || !p1_out || !p2_out || !idx1_out || !idx2_out || bits < 2 ||
-        bits > 8 || K < 2 || max_n < 1)
+// nbp = 2: p_out / idx_out are {p1, p2} / {idx1, idx2} arrays of [C]; nbp = 3: one [C, 3] array each.
+static int search23_impl(const float* x, const int64_t* ro, int64_t C, int64_t n, int64_t total,
+                         int64_t max_n, int bits, const float* ratios, int K, const float* m,
+                         int nbp, float* const* p_out, int32_t* const* idx_out, int out_stride,
+                         float* err_out, float* sse_out, void* ws, size_t ws_bytes, void* stream) {
+    if (!x || !ratios || !m || bits < 2 || bits > 8 || K < nbp || max_n < 1)
         return PWLQ_ERR_INVALID_ARG;
-    if (misaligned(x, 4) || misaligned(ratios, 4) || misaligned(m, 4) || misaligned(p1_out, 4) ||
-        misaligned(p2_out, 4) || misaligned(err_out, 4) || misaligned(idx1_out, 4) ||
-        misaligned(idx2_out, 4) || misaligned(sse_pairs, 4) || misaligned(ro, 8))
+    for (int t = 0; t < nbp; ++t)
+        if (!p_out[t] || !idx_out[t] || misaligned(p_out[t], 4) || misaligned(idx_out[t], 4))
+            return PWLQ_ERR_INVALID_ARG;
+    if (misaligned(x, 4) || misaligned(ratios, 4) || misaligned(m, 4) || misaligned(err_out, 4) ||
+        misaligned(sse_out, 4) || misaligned(ro, 8))
         return PWLQ_ERR_INVALID_ARG;
-    if (K > PWLQ_MAX_K2 || max_n > pwlq::kSearchTile || total > kMaxTotal) return PWLQ_ERR_UNSUPPORTED;
-    if (!ws || ws_bytes < 256) return PWLQ_ERR_WORKSPACE;
+    if (K > PWLQ_MAX_K2 || total > kMaxTotal) return PWLQ_ERR_UNSUPPORTED;
+    const int64_t tiles = (max_n + pwlq::kSearchTile - 1) / pwlq::kSearchTile;
+    if (C * tiles > ((int64_t)1 << 31) - 1) return PWLQ_ERR_UNSUPPORTED;
+    if (!ws || ws_bytes < pwlq::search2_workspace_bytes(C, max_n, K)) return PWLQ_ERR_WORKSPACE;
     if (misaligned(ws, 256)) return PWLQ_ERR_INVALID_ARG;
-    return from_cuda(pwlq::launch_search2(x, ro, C, n, max_n, bits, ratios, K, m, p1_out, p2_out,
-                                          err_out, idx1_out, idx2_out, sse_pairs, ws,
+    return from_cuda(pwlq::launch_search2(x, ro, C, n, max_n, bits, ratios, K, m, nbp, p_out,
+                                          idx_out, out_stride, err_out, sse_out, ws,
                                           as_stream(stream)));
 }
 
@@ -441,8 +444,10 @@ int pwlq_search2(const float* x, int64_t C, int64_t n, int bits, const float* ra
                  int32_t* idx2_out, float* sse_pairs, void* workspace, size_t workspace_bytes,
                  void* stream) {
     if (int rc = check_rows(C, n)) return rc;
-    return search2_impl(x, nullptr, C, n, C * n, n, bits, ratios, K, m, p1_out, p2_out, err_out,
-                        idx1_out, idx2_out, sse_pairs, workspace, workspace_bytes, stream);
+    float* const p[3] = {p1_out, p2_out, nullptr};
+    int32_t* const idx[3] = {idx1_out, idx2_out, nullptr};
+    return search23_impl(x, nullptr, C, n, C * n, n, bits, ratios, K, m, 2, p, idx, 1, err_out,
+                         sse_pairs, workspace, workspace_bytes, stream);
 }
 
 int pwlq_search2_ragged(const float* x, const int64_t* row_offsets, int64_t C, int64_t total,
@@ -452,14 +457,41 @@ int pwlq_search2_ragged(const float* x, const int64_t* row_offsets, int64_t C, i
                         size_t workspace_bytes, void* stream) {
     if (int rc = check_rows(C, total)) return rc;
     if (!row_offsets || max_n > total) return PWLQ_ERR_INVALID_ARG;
-    return search2_impl(x, row_offsets, C, 0, total, max_n, bits, ratios, K, m, p1_out, p2_out,
-                        err_out, idx1_out, idx2_out, sse_pairs, workspace, workspace_bytes, stream);
+    float* const p[3] = {p1_out, p2_out, nullptr};
+    int32_t* const idx[3] = {idx1_out, idx2_out, nullptr};
+    return search23_impl(x, row_offsets, C, 0, total, max_n, bits, ratios, K, m, 2, p, idx, 1,
+                         err_out, sse_pairs, workspace, workspace_bytes, stream);
 }
 
-static int quantize2_impl(const float* x, const int64_t* ro, int64_t C, int64_t n, int64_t total,
-                          int bits, const float* m, const float* p1, const float* p2,
-                          uint8_t* codes, uint8_t* region2, float* fake, int layout,
-                          void* stream) {
+int pwlq_search3(const float* x, int64_t C, int64_t n, int bits, const float* ratios, int K,
+                 const float* m, float* p_out, float* err_out, int32_t* idx_out,
+                 float* sse_triples, void* workspace, size_t workspace_bytes, void* stream) {
+    if (int rc = check_rows(C, n)) return rc;
+    if (!p_out || !idx_out) return PWLQ_ERR_INVALID_ARG;
+    float* const p[3] = {p_out, p_out + 1, p_out + 2};
+    int32_t* const idx[3] = {idx_out, idx_out + 1, idx_out + 2};
+    return search23_impl(x, nullptr, C, n, C * n, n, bits, ratios, K, m, 3, p, idx, 3, err_out,
+                         sse_triples, workspace, workspace_bytes, stream);
+}
+
+int pwlq_search3_ragged(const float* x, const int64_t* row_offsets, int64_t C, int64_t total,
+                        int64_t max_n, int bits, const float* ratios, int K, const float* m,
+                        float* p_out, float* err_out, int32_t* idx_out, float* sse_triples,
+                        void* workspace, size_t workspace_bytes, void* stream) {
+    if (int rc = check_rows(C, total)) return rc;
+    if (!row_offsets || max_n > total || !p_out || !idx_out) return PWLQ_ERR_INVALID_ARG;
+    float* const p[3] = {p_out, p_out + 1, p_out + 2};
+    int32_t* const idx[3] = {idx_out, idx_out + 1, idx_out + 2};
+    return search23_impl(x, row_offsets, C, 0, total, max_n, bits, ratios, K, m, 3, p, idx, 3,
+                         err_out, sse_triples, workspace, workspace_bytes, stream);
+}
+
+// p3 == nullptr: two breakpoints in separate arrays (stride 1); otherwise p1 = p, p2 = p + 1,
+// p3 = p + 2 of one [C, 3] array (stride 3).
+static int quantize23_impl(const float* x, const int64_t* ro, int64_t C, int64_t n, int64_t total,
+                           int bits, const float* m, const float* p1, const float* p2,
+                           const float* p3, int p_stride, uint8_t* codes, uint8_t* region2,
+                           float* fake, int layout, void* stream) {
     if (!x || !m || !p1 || !p2 || !codes || !region2 || bits < 2 || bits > 8 ||
         (layout != PWLQ_CODES_U8 && layout != PWLQ_CODES_PACKED))
         return PWLQ_ERR_INVALID_ARG;
@@ -467,16 +499,16 @@ static int quantize2_impl(const float* x, const int64_t* ro, int64_t C, int64_t 
         misaligned(fake, 4) || misaligned(ro, 8))
         return PWLQ_ERR_INVALID_ARG;
     if (total > kMaxTotal) return PWLQ_ERR_UNSUPPORTED;
-    return from_cuda(pwlq::launch_quantize2(x, ro, C, n, total, bits, m, p1, p2, codes, region2,
-                                            fake, layout, as_stream(stream)));
+    return from_cuda(pwlq::launch_quantize2(x, ro, C, n, total, bits, m, p1, p2, p3, p_stride,
+                                            codes, region2, fake, layout, as_stream(stream)));
 }
 
 int pwlq_quantize2(const float* x, int64_t C, int64_t n, int bits, const float* m,
                    const float* p1, const float* p2, uint8_t* codes, uint8_t* region2,
                    float* fake_out, int code_layout, void* stream) {
     if (int rc = check_rows(C, n)) return rc;
-    return quantize2_impl(x, nullptr, C, n, C * n, bits, m, p1, p2, codes, region2, fake_out,
-                          code_layout, stream);
+    return quantize23_impl(x, nullptr, C, n, C * n, bits, m, p1, p2, nullptr, 1, codes, region2,
+                           fake_out, code_layout, stream);
 }
 
 int pwlq_quantize2_ragged(const float* x, const int64_t* row_offsets, int64_t C, int64_t total,
@@ -485,14 +517,32 @@ int pwlq_quantize2_ragged(const float* x, const int64_t* row_offsets, int64_t C,
                           void* stream) {
     if (int rc = check_rows(C, total)) return rc;
     if (!row_offsets) return PWLQ_ERR_INVALID_ARG;
-    return quantize2_impl(x, row_offsets, C, 0, total, bits, m, p1, p2, codes, region2, fake_out,
-                          code_layout, stream);
+    return quantize23_impl(x, row_offsets, C, 0, total, bits, m, p1, p2, nullptr, 1, codes,
+                           region2, fake_out, code_layout, stream);
 }
 
-static int dequantize2_impl(const uint8_t* codes, const uint8_t* region2, const int64_t* ro,
-                            int64_t C, int64_t n, int64_t total, int bits, const float* m,
-                            const float* p1, const float* p2, float* y, int layout,
-                            void* stream) {
+int pwlq_quantize3(const float* x, int64_t C, int64_t n, int bits, const float* m, const float* p,
+                   uint8_t* codes, uint8_t* region2, float* fake_out, int code_layout,
+                   void* stream) {
+    if (int rc = check_rows(C, n)) return rc;
+    if (!p) return PWLQ_ERR_INVALID_ARG;
+    return quantize23_impl(x, nullptr, C, n, C * n, bits, m, p, p + 1, p + 2, 3, codes, region2,
+                           fake_out, code_layout, stream);
+}
+
+int pwlq_quantize3_ragged(const float* x, const int64_t* row_offsets, int64_t C, int64_t total,
+                          int bits, const float* m, const float* p, uint8_t* codes,
+                          uint8_t* region2, float* fake_out, int code_layout, void* stream) {
+    if (int rc = check_rows(C, total)) return rc;
+    if (!row_offsets || !p) return PWLQ_ERR_INVALID_ARG;
+    return quantize23_impl(x, row_offsets, C, 0, total, bits, m, p, p + 1, p + 2, 3, codes,
+                           region2, fake_out, code_layout, stream);
+}
+
+static int dequantize23_impl(const uint8_t* codes, const uint8_t* region2, const int64_t* ro,
+                             int64_t C, int64_t n, int64_t total, int bits, const float* m,
+                             const float* p1, const float* p2, const float* p3, int p_stride,
+                             float* y, int layout, void* stream) {
     if (!codes || !region2 || !m || !p1 || !p2 || !y || bits < 2 || bits > 8 ||
         (layout != PWLQ_CODES_U8 && layout != PWLQ_CODES_PACKED))
         return PWLQ_ERR_INVALID_ARG;
@@ -500,16 +550,16 @@ static int dequantize2_impl(const uint8_t* codes, const uint8_t* region2, const 
         misaligned(ro, 8))
         return PWLQ_ERR_INVALID_ARG;
     if (total > kMaxTotal) return PWLQ_ERR_UNSUPPORTED;
-    return from_cuda(pwlq::launch_dequantize2(codes, region2, ro, C, n, total, bits, m, p1, p2, y,
-                                              layout, as_stream(stream)));
+    return from_cuda(pwlq::launch_dequantize2(codes, region2, ro, C, n, total, bits, m, p1, p2, p3,
+                                              p_stride, y, layout, as_stream(stream)));
 }
 
 int pwlq_dequantize2(const uint8_t* codes, const uint8_t* region2, int64_t C, int64_t n,
                      int bits, const float* m, const float* p1, const float* p2, float* y,
                      int code_layout, void* stream) {
     if (int rc = check_rows(C, n)) return rc;
-    return dequantize2_impl(codes, region2, nullptr, C, n, C * n, bits, m, p1, p2, y, code_layout,
-                            stream);
+    return dequantize23_impl(codes, region2, nullptr, C, n, C * n, bits, m, p1, p2, nullptr, 1, y,
+                             code_layout, stream);
 }
 
 int pwlq_dequantize2_ragged(const uint8_t* codes, const uint8_t* region2,
@@ -518,8 +568,27 @@ int pwlq_dequantize2_ragged(const uint8_t* codes, const uint8_t* region2,
                             int code_layout, void* stream) {
     if (int rc = check_rows(C, total)) return rc;
     if (!row_offsets) return PWLQ_ERR_INVALID_ARG;
-    return dequantize2_impl(codes, region2, row_offsets, C, 0, total, bits, m, p1, p2, y,
-                            code_layout, stream);
+    return dequantize23_impl(codes, region2, row_offsets, C, 0, total, bits, m, p1, p2, nullptr, 1,
+                             y, code_layout, stream);
+}
+
+int pwlq_dequantize3(const uint8_t* codes, const uint8_t* region2, int64_t C, int64_t n,
+                     int bits, const float* m, const float* p, float* y, int code_layout,
+                     void* stream) {
+    if (int rc = check_rows(C, n)) return rc;
+    if (!p) return PWLQ_ERR_INVALID_ARG;
+    return dequantize23_impl(codes, region2, nullptr, C, n, C * n, bits, m, p, p + 1, p + 2, 3, y,
+                             code_layout, stream);
+}
+
+int pwlq_dequantize3_ragged(const uint8_t* codes, const uint8_t* region2,
+                            const int64_t* row_offsets, int64_t C, int64_t total, int bits,
+                            const float* m, const float* p, float* y, int code_layout,
+                            void* stream) {
+    if (int rc = check_rows(C, total)) return rc;
+    if (!row_offsets || !p) return PWLQ_ERR_INVALID_ARG;
+    return dequantize23_impl(codes, region2, row_offsets, C, 0, total, bits, m, p, p + 1, p + 2, 3,
+                             y, code_layout, stream);
 }
 
 size_t pwlq_bias_workspace_bytes(int64_t C, int64_t max_n) {

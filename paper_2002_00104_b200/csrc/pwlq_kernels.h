@@ -71,22 +71,28 @@ cudaError_t launch_dequantize(const uint8_t* codes, const uint8_t* mask,
                               const float* xi = nullptr, const float* beta = nullptr,
                               const void* rowmap = nullptr);
 
-// Two breakpoints (three regions): pair search over a grid of K <= kSearch2MaxK ascending ratios
-// for rows of at most kSearchTile values; quantize / dequantize with a two-bit region index.
+// Two or three breakpoints (three or four regions): search over all pairs (nbp = 2) or triples
+// (nbp = 3) of a grid of K <= kSearch2MaxK ascending ratios; rows longer than kSearchTile values
+// are cut into tiles whose terms a second kernel adds in a fixed order (workspace:
+// search2_workspace_bytes).  Breakpoint t of row c is delivered to p_out[t][c * out_stride] (and
+// its grid index to idx_out[t][...]).  sse_out: [C, K, K] (pairs) or [C, K, K, K] (triples) or
+// nullptr.  Quantize / dequantize with a two-bit region index; p3 == nullptr: two breakpoints;
+// breakpoint arrays are read with stride p_stride.
 constexpr int kSearch2MaxK = 64;
+size_t search2_workspace_bytes(int64_t C, int64_t max_n, int K);
 cudaError_t launch_search2(const float* x, const int64_t* row_offsets, int64_t C, int64_t n,
                            int64_t max_n, int bits, const float* ratios, int K, const float* m,
-                           float* p1_out, float* p2_out, float* err_out, int32_t* idx1_out,
-                           int32_t* idx2_out, float* sse_pairs, void* workspace,
-                           cudaStream_t stream);
+                           int nbp, float* const* p_out, int32_t* const* idx_out, int out_stride,
+                           float* err_out, float* sse_out, void* workspace, cudaStream_t stream);
 cudaError_t launch_quantize2(const float* x, const int64_t* row_offsets, int64_t C, int64_t n,
                              int64_t total, int bits, const float* m, const float* p1,
-                             const float* p2, uint8_t* codes, uint8_t* region2, float* fake,
-                             int layout, cudaStream_t stream);
+                             const float* p2, const float* p3, int p_stride, uint8_t* codes,
+                             uint8_t* region2, float* fake, int layout, cudaStream_t stream);
 cudaError_t launch_dequantize2(const uint8_t* codes, const uint8_t* region2,
                                const int64_t* row_offsets, int64_t C, int64_t n, int64_t total,
                                int bits, const float* m, const float* p1, const float* p2,
-                               float* y, int layout, cudaStream_t stream);
+                               const float* p3, int p_stride, float* y, int layout,
+                               cudaStream_t stream);
 
 // Bias correction: folded scale xi and offset beta per row; dequantize that applies them; dense
 // (b+1)-bit storage of code and region bit.

@@ -31,19 +31,21 @@ struct Search2Args {
     int K;
     int levels;
     int cap;              // tile capacity in values
-    float* p1_out;
-    float* p2_out;
+    int nbp;              // breakpoints searched: 2 (pairs) or 3 (triples)
+    int64_t tiles;        // tiles per row (by the longest row); > 1: partial terms go to `partials`
+    double* partials;     // [C, tiles, 2 K + K (K - 1) / 2]: C_i, T_j, M_ij of every tile
+    float* p_out[3];      // breakpoint t of row c: p_out[t][c * out_stride]
+    int32_t* idx_out[3];
+    int out_stride;
     float* err_out;
-    int32_t* idx1_out;
-    int32_t* idx2_out;
-    float* sse_pairs;     // [C, K, K] or nullptr
+    float* sse_out;       // pairs: [C, K, K]; triples: [C, K, K, K]; or nullptr
     int* status;
 };
 
 __host__ __device__ inline size_t s2_align(size_t v) { return (v + 15) & ~(size_t)15; }
 
 // Shared-memory layout: sorted tile | bucket+rank per value | breakpoints | bucket starts |
-// per-warp bucket counts | C, T | M (triangular).
+// per-warp bucket counts | C, T | M (triangular) | best left / right parts of the triple search.
 __host__ __device__ inline size_t search2_smem(int cap, int K, size_t* off) {
     size_t o = 0;
     off[0] = o; o = s2_align(o + sizeof(float) * (size_t)cap);
@@ -53,6 +55,8 @@ __host__ __device__ inline size_t search2_smem(int cap, int K, size_t* off) {
     off[4] = o; o = s2_align(o + sizeof(uint16_t) * (size_t)(K + 1) * kS2Warps);
     off[5] = o; o = s2_align(o + sizeof(double) * (size_t)(2 * K));
     off[6] = o; o = s2_align(o + sizeof(double) * (size_t)(K * (K - 1) / 2));
+    off[7] = o; o = s2_align(o + sizeof(double) * (size_t)(2 * K));      // triples: best left / right parts
+    off[8] = o; o = s2_align(o + sizeof(int) * (size_t)(2 * K));
     return o;
 }
 
@@ -213,35 +217,175 @@ __device__ __forceinline__ void middle_terms(const float* tile, const int* start
 
 __device__ __forceinline__ void write_degenerate2(const Search2Args& a, int64_t row) {
     if (threadIdx.x == 0) {
-        a.idx1_out[row] = 0;
-        a.idx2_out[row] = 1;
-        a.p1_out[row] = 0.0f;
-        a.p2_out[row] = 0.0f;
+        for (int t = 0; t < a.nbp; ++t) {
+            a.idx_out[t][row * a.out_stride] = t;
+            a.p_out[t][row * a.out_stride] = 0.0f;
+        }
         if (a.err_out) a.err_out[row] = 0.0f;
     }
-    if (a.sse_pairs)
-        for (int t = threadIdx.x; t < a.K * a.K; t += kS2Threads)
-            a.sse_pairs[row * a.K * a.K + t] = 0.0f;
+    if (a.sse_out) {
+        const int64_t per_row = (int64_t)a.K * a.K * (a.nbp == 3 ? a.K : 1);
+        for (int64_t t = threadIdx.x; t < per_row; t += kS2Threads) a.sse_out[row * per_row + t] = 0.0f;
+    }
 }
 
+// First minimum of (value, index) pairs over the CTA; the result is valid in thread 0.
+__device__ __forceinline__ void cta_first_min(double& best, int& best_idx, double* red_val,
+                                              int* red_idx) {
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        const double ov = __shfl_xor_sync(0xffffffffu, best, o);
+        const int oi = __shfl_xor_sync(0xffffffffu, best_idx, o);
+        if (oi != 0x7fffffff && (best_idx == 0x7fffffff || ov < best || (ov == best && oi < best_idx))) {
+            best = ov; best_idx = oi;
+        }
+    }
+    if (lane == 0) { red_val[warp] = best; red_idx[warp] = best_idx; }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        for (int w = 1; w < kS2Warps; ++w) {
+            const double ov = red_val[w];
+            const int oi = red_idx[w];
+            if (oi != 0x7fffffff && (best_idx == 0x7fffffff || ov < best || (ov == best && oi < best_idx))) {
+                best = ov; best_idx = oi;
+            }
+        }
+    }
+}
+
+// Totals and the first minimal pair in the order (i, j), from the terms of one row in shared
+// memory (CT = C[0..K), T[K..2K); M triangular; ps = the row's breakpoints).  All threads call.
+__device__ __forceinline__ void finish_pairs(const Search2Args& a, int64_t row, const float* ps,
+                                             double* CT, double* M, double* red_val, int* red_idx) {
+    const int K = a.K, tid = threadIdx.x;
+    const int npairs = K * (K - 1) / 2;
+    double best = 0.0;
+    int best_idx = 0x7fffffff;
+    {
+        int i = 0, base = 0;                          // base = pair_index(i, i + 1)
+        for (int t = tid; t < npairs; t += kS2Threads) {
+            while (t >= base + (K - 1 - i)) { base += K - 1 - i; ++i; }
+            const int j = i + 1 + (t - base);
+            const double v = CT[i] + M[t] + CT[K + j];
+            M[t] = v;
+            if (best_idx == 0x7fffffff || v < best) { best = v; best_idx = t; }
+        }
+    }
+    cta_first_min(best, best_idx, red_val, red_idx);
+    if (tid == 0) {
+        int i = 0, base = 0;
+        while (best_idx >= base + (K - 1 - i)) { base += K - 1 - i; ++i; }
+        const int j = i + 1 + (best_idx - base);
+        a.idx_out[0][row * a.out_stride] = i;
+        a.idx_out[1][row * a.out_stride] = j;
+        a.p_out[0][row * a.out_stride] = ps[i];
+        a.p_out[1][row * a.out_stride] = ps[j];
+        if (a.err_out) a.err_out[row] = (float)best;
+    }
+    if (a.sse_out) {
+        float* dst = a.sse_out + row * K * K;
+        for (int t = tid; t < K * K; t += kS2Threads) {
+            const int i = t / K, j = t - i * K;
+            dst[t] = (i < j) ? (float)M[pair_index(i, j, K)] : 0.0f;
+        }
+    }
+}
+
+// Three breakpoints: SSE(i, j, k) = (C_i + M_ij) + (M_jk + T_k), the regions' errors being sums
+// over disjoint sets of values.  For every middle breakpoint j the best left part (over i < j) and
+// the best right part (over k > j) are independent, so the first minimal triple in the order
+// (i, j, k) follows from K - 2 pairs of scans over the terms the pair search already has --
+// O(K^2) per row instead of K^3 / 6 evaluations.  left / right: 2 K doubles and 2 K ints of
+// shared memory.
+__device__ __forceinline__ void finish_triples(const Search2Args& a, int64_t row, const float* ps,
+                                               const double* CT, const double* M, double* lr_val,
+                                               int* lr_idx, double* red_val, int* red_idx) {
+    const int K = a.K, tid = threadIdx.x;
+    for (int t = tid; t < 2 * K; t += kS2Threads) {
+        const bool left = t < K;
+        const int j = left ? t : t - K;
+        double best = 0.0;
+        int arg = -1;
+        if (left) {
+            for (int i = 0; i < j; ++i) {             // ascending i: the first minimum stays
+                const double v = CT[i] + M[pair_index(i, j, K)];
+                if (arg < 0 || v < best) { best = v; arg = i; }
+            }
+        } else {
+            for (int k = j + 1; k < K; ++k) {
+                const double v = M[pair_index(j, k, K)] + CT[K + k];
+                if (arg < 0 || v < best) { best = v; arg = k; }
+            }
+        }
+        lr_val[t] = best;
+        lr_idx[t] = arg;
+    }
+    __syncthreads();
+    // the triples of two middle breakpoints differ in j, so (total, i, j) orders them completely
+    double best = 0.0;
+    int best_idx = 0x7fffffff;
+    for (int j = 1 + tid; j < K - 1; j += kS2Threads) {
+        const double v = lr_val[j] + lr_val[K + j];
+        const int key = lr_idx[j] * K + j;            // order (i, j)
+        if (best_idx == 0x7fffffff || v < best || (v == best && key < best_idx)) { best = v; best_idx = key; }
+    }
+    cta_first_min(best, best_idx, red_val, red_idx);
+    if (tid == 0) {
+        const int i = best_idx / K, j = best_idx - i * K, k = lr_idx[K + j];
+        const int idx[3] = {i, j, k};
+        for (int t = 0; t < 3; ++t) {
+            a.idx_out[t][row * a.out_stride] = idx[t];
+            a.p_out[t][row * a.out_stride] = ps[idx[t]];
+        }
+        if (a.err_out) a.err_out[row] = (float)best;
+    }
+    if (a.sse_out) {
+        float* dst = a.sse_out + row * (int64_t)K * K * K;
+        for (int t = tid; t < K * K * K; t += kS2Threads) {
+            const int i = t / (K * K), j = (t / K) % K, k = t % K;
+            dst[t] = (i < j && j < k)
+                         ? (float)((CT[i] + M[pair_index(i, j, K)]) + (M[pair_index(j, k, K)] + CT[K + k]))
+                         : 0.0f;
+        }
+    }
+}
+
+// Shared memory of the row-closing step: breakpoints | C, T | M | best left / right parts.
+__host__ __device__ inline size_t finish2_smem(int K, size_t* off) {
+    size_t o = 0;
+    off[0] = o; o = s2_align(o + sizeof(float) * (size_t)K);
+    off[1] = o; o = s2_align(o + sizeof(double) * (size_t)(2 * K));
+    off[2] = o; o = s2_align(o + sizeof(double) * (size_t)(K * (K - 1) / 2));
+    off[3] = o; o = s2_align(o + sizeof(double) * (size_t)(2 * K));
+    off[4] = o; o = s2_align(o + sizeof(int) * (size_t)(2 * K));
+    return o;
+}
+
+// One CTA per (row, tile of at most a.cap values).  A row of one tile is closed here; the terms
+// of a longer row's tiles go to a.partials and search2_finish_kernel closes the row.
 __global__ void __launch_bounds__(kS2Threads)
 search2_kernel(Search2Args a) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
     __shared__ double red_val[kS2Warps];
     __shared__ int red_idx[kS2Warps];
-    const int64_t row = blockIdx.x;
-    const int64_t beg = a.rows.begin(row), end = a.rows.begin(row + 1);
-    const int cnt = (int)(end - beg);
+    const int64_t row = blockIdx.x / a.tiles, tile_no = blockIdx.x - row * a.tiles;
+    const int64_t row_beg = a.rows.begin(row), end = a.rows.begin(row + 1);
+    const int64_t n_row = end - row_beg;
+    const int64_t beg = row_beg + tile_no * (int64_t)a.cap;
+    if (tile_no > 0 && beg >= end) return;            // this row has fewer tiles than the longest
+    const int cnt = (int)min((int64_t)a.cap, end - beg);
     const int K = a.K;
     const float m = a.m[row];
     const float Lf = (float)a.levels;
     const bool finite = (__float_as_uint(m) & 0x7fffffffu) < 0x7f800000u;
     if (!finite || !(m > 0.0f) || cnt <= 0) {
+        if (a.tiles > 1) return;                      // the row-closing kernel writes the row
         if (!finite && threadIdx.x == 0) atomicOr(a.status, kStatusNonFinite);
         write_degenerate2(a, row);
         return;
     }
-    size_t off[7];
+    size_t off[9];
     search2_smem(a.cap, K, off);
     float* tile = reinterpret_cast<float*>(smem_raw + off[0]);
     uint32_t* jr = reinterpret_cast<uint32_t*>(smem_raw + off[1]);
@@ -259,14 +403,15 @@ search2_kernel(Search2Args a) {
         ps[k] = __fmul_rn(m, rk);
     }
     for (int t = tid; t < (K + 1) * kS2Warps; t += kS2Threads) hist[t] = 0;
-    if (__syncthreads_or(unordered)) {               // the pair search needs an ascending grid
+    if (__syncthreads_or(unordered)) {               // the search needs an ascending grid
+        if (a.tiles > 1) return;
         if (tid == 0) atomicOr(a.status, kStatusBadGrid);
         write_degenerate2(a, row);
         return;
     }
 
     // pass 1: bucket j = #{k : p_k < a} of every value and its rank among the earlier values of
-    // the same bucket in this warp's segment (each warp owns a contiguous segment of the row and
+    // the same bucket in this warp's segment (each warp owns a contiguous segment of the tile and
     // walks it 32 values at a time; ranks inside a group of 32 come from match.any)
     const unsigned full = 0xffffffffu;
     const int seg = (((cnt + kS2Warps - 1) / kS2Warps) + 31) & ~31;
@@ -334,7 +479,7 @@ search2_kernel(Search2Args a) {
     }
     // The fused form's rounding shows in the sums of short rows (it grows like L / sqrt(n)); rows
     // shorter than L^2 / 2 use the operation-by-operation form.
-    const bool fused = 2 * (int64_t)cnt >= (int64_t)a.levels * a.levels;
+    const bool fused = 2 * n_row >= (int64_t)a.levels * a.levels;
     {
         int item = 0;                                  // (i, group of eight j) in a fixed order
         for (int i = 0; i < K - 1; ++i)
@@ -346,61 +491,81 @@ search2_kernel(Search2Args a) {
     }
     __syncthreads();
 
-    // totals and the first minimal pair in the order (i, j)
     const int npairs = K * (K - 1) / 2;
-    double best = 0.0;
-    int best_idx = 0x7fffffff;
-    {
-        int i = 0, base = 0;                          // base = pair_index(i, i + 1)
-        for (int t = tid; t < npairs; t += kS2Threads) {
-            while (t >= base + (K - 1 - i)) { base += K - 1 - i; ++i; }
-            const int j = i + 1 + (t - base);
-            const double v = CT[i] + M[t] + CT[K + j];
-            M[t] = v;
-            if (best_idx == 0x7fffffff || v < best) { best = v; best_idx = t; }
-        }
+    if (a.tiles > 1) {
+        double* dst = a.partials + ((size_t)row * a.tiles + tile_no) * (size_t)(2 * K + npairs);
+        for (int t = tid; t < 2 * K; t += kS2Threads) dst[t] = CT[t];
+        for (int t = tid; t < npairs; t += kS2Threads) dst[2 * K + t] = M[t];
+        return;
     }
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) {
-        const double ov = __shfl_xor_sync(0xffffffffu, best, o);
-        const int oi = __shfl_xor_sync(0xffffffffu, best_idx, o);
-        if (oi != 0x7fffffff && (best_idx == 0x7fffffff || ov < best || (ov == best && oi < best_idx))) {
-            best = ov; best_idx = oi;
-        }
+    if (a.nbp == 3)
+        finish_triples(a, row, ps, CT, M, reinterpret_cast<double*>(smem_raw + off[7]),
+                       reinterpret_cast<int*>(smem_raw + off[8]), red_val, red_idx);
+    else
+        finish_pairs(a, row, ps, CT, M, red_val, red_idx);
+}
+
+// Closes the rows that were cut into tiles: adds the tiles' terms in ascending tile order (fixed
+// order: reproducible) and takes the first minimal pair or triple.  One CTA per row.
+__global__ void __launch_bounds__(kS2Threads)
+search2_finish_kernel(Search2Args a) {
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    __shared__ double red_val[kS2Warps];
+    __shared__ int red_idx[kS2Warps];
+    const int64_t row = blockIdx.x;
+    const int64_t n_row = a.rows.begin(row + 1) - a.rows.begin(row);
+    const int K = a.K, tid = threadIdx.x;
+    const float m = a.m[row];
+    const bool finite = (__float_as_uint(m) & 0x7fffffffu) < 0x7f800000u;
+    if (!finite || !(m > 0.0f) || n_row <= 0) {
+        if (!finite && tid == 0) atomicOr(a.status, kStatusNonFinite);
+        write_degenerate2(a, row);
+        return;
     }
-    if (lane == 0) { red_val[warp] = best; red_idx[warp] = best_idx; }
+    size_t off[5];
+    finish2_smem(K, off);
+    float* ps = reinterpret_cast<float*>(smem_raw + off[0]);
+    double* CT = reinterpret_cast<double*>(smem_raw + off[1]);
+    double* M = reinterpret_cast<double*>(smem_raw + off[2]);
+    int unordered = 0;
+    for (int k = tid; k < K; k += kS2Threads) {
+        const float rk = __ldg(a.ratios + k);
+        if (k > 0) unordered |= (rk < __ldg(a.ratios + k - 1));
+        ps[k] = __fmul_rn(m, rk);
+    }
+    if (__syncthreads_or(unordered)) {
+        if (tid == 0) atomicOr(a.status, kStatusBadGrid);
+        write_degenerate2(a, row);
+        return;
+    }
+    const int npairs = K * (K - 1) / 2, nterms = 2 * K + npairs;
+    const int64_t nt = (n_row + a.cap - 1) / a.cap;
+    const double* src = a.partials + (size_t)row * a.tiles * (size_t)nterms;
+    for (int t = tid; t < nterms; t += kS2Threads) {
+        double v = 0.0;
+        for (int64_t u = 0; u < nt; ++u) v += src[(size_t)u * nterms + t];
+        if (t < 2 * K) CT[t] = v; else M[t - 2 * K] = v;
+    }
     __syncthreads();
-    if (tid == 0) {
-        for (int w = 1; w < kS2Warps; ++w) {
-            const double ov = red_val[w];
-            const int oi = red_idx[w];
-            if (oi != 0x7fffffff && (best_idx == 0x7fffffff || ov < best || (ov == best && oi < best_idx))) {
-                best = ov; best_idx = oi;
-            }
-        }
-        int i = 0, base = 0;
-        while (best_idx >= base + (K - 1 - i)) { base += K - 1 - i; ++i; }
-        const int j = i + 1 + (best_idx - base);
-        a.idx1_out[row] = i;
-        a.idx2_out[row] = j;
-        a.p1_out[row] = ps[i];
-        a.p2_out[row] = ps[j];
-        if (a.err_out) a.err_out[row] = (float)best;
-    }
-    if (a.sse_pairs) {
-        float* dst = a.sse_pairs + row * K * K;
-        for (int t = tid; t < K * K; t += kS2Threads) {
-            const int i = t / K, j = t - i * K;
-            dst[t] = (i < j) ? (float)M[pair_index(i, j, K)] : 0.0f;
-        }
-    }
+    if (a.nbp == 3)
+        finish_triples(a, row, ps, CT, M, reinterpret_cast<double*>(smem_raw + off[3]),
+                       reinterpret_cast<int*>(smem_raw + off[4]), red_val, red_idx);
+    else
+        finish_pairs(a, row, ps, CT, M, red_val, red_idx);
+}
+
+size_t search2_workspace_bytes(int64_t C, int64_t max_n, int K) {
+    const int64_t tiles = (max_n + kSearchTile - 1) / kSearchTile;
+    size_t bytes = 256;
+    if (tiles > 1)
+        bytes += sizeof(double) * (size_t)C * (size_t)tiles * (size_t)(2 * K + K * (K - 1) / 2);
+    return (bytes + 255) / 256 * 256;
 }
 
 cudaError_t launch_search2(const float* x, const int64_t* row_offsets, int64_t C, int64_t n,
                            int64_t max_n, int bits, const float* ratios, int K, const float* m,
-                           float* p1_out, float* p2_out, float* err_out, int32_t* idx1_out,
-                           int32_t* idx2_out, float* sse_pairs, void* workspace,
-                           cudaStream_t stream) {
+                           int nbp, float* const* p_out, int32_t* const* idx_out, int out_stride,
+                           float* err_out, float* sse_out, void* workspace, cudaStream_t stream) {
     cudaError_t e = cudaMemsetAsync(workspace, 0, 256, stream);          // status word
     if (e != cudaSuccess) return e;
     Search2Args a;
@@ -410,36 +575,53 @@ cudaError_t launch_search2(const float* x, const int64_t* row_offsets, int64_t C
     a.ratios = ratios;
     a.K = K;
     a.levels = (1 << (bits - 1)) - 1;
-    a.cap = (int)((max_n + 3) / 4 * 4);
-    a.p1_out = p1_out;
-    a.p2_out = p2_out;
+    a.nbp = nbp;
+    a.tiles = (max_n + kSearchTile - 1) / kSearchTile;
+    a.cap = a.tiles > 1 ? kSearchTile : (int)((max_n + 3) / 4 * 4);
+    a.partials = reinterpret_cast<double*>(static_cast<unsigned char*>(workspace) + 256);
+    for (int t = 0; t < 3; ++t) {
+        a.p_out[t] = t < nbp ? p_out[t] : nullptr;
+        a.idx_out[t] = t < nbp ? idx_out[t] : nullptr;
+    }
+    a.out_stride = out_stride;
     a.err_out = err_out;
-    a.idx1_out = idx1_out;
-    a.idx2_out = idx2_out;
-    a.sse_pairs = sse_pairs;
+    a.sse_out = sse_out;
     a.status = static_cast<int*>(workspace);
-    size_t off[7];
+    size_t off[9];
     const size_t smem = search2_smem(a.cap, K, off);
     if (smem > 48 * 1024) {
         e = cudaFuncSetAttribute(search2_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                  (int)smem);
         if (e != cudaSuccess) return e;
     }
-    search2_kernel<<<(unsigned)C, kS2Threads, smem, stream>>>(a);
+    search2_kernel<<<(unsigned)(C * a.tiles), kS2Threads, smem, stream>>>(a);
+    e = cudaGetLastError();
+    if (e != cudaSuccess || a.tiles == 1) return e;
+    size_t foff[5];
+    search2_finish_kernel<<<(unsigned)C, kS2Threads, finish2_smem(K, foff), stream>>>(a);
     return cudaGetLastError();
 }
 
-// ------------------------------------------------------------- quantize / dequantize, 3 regions
-// Constants of the three regions of one row.
-struct Params3 {
-    float z[3], s[3], inv[3];
+// ------------------------------------------------ quantize / dequantize, three or four regions
+// Breakpoints of the rows: two arrays (p3 == nullptr: three regions) or three, read with a stride
+// (1 for separate arrays, 3 for one [C, 3] array).
+struct BreakPts {
+    const float* p1;
+    const float* p2;
+    const float* p3;
+    int stride;
 };
-__device__ __forceinline__ Params3 make_params3(float m, float p1, float p2, float Lf) {
+// Constants of the regions of one row.  Without a third breakpoint the fourth region starts at m
+// and is never entered (a <= m).
+struct Params3 {
+    float z[4], s[4], inv[4];
+};
+__device__ __forceinline__ Params3 make_params3(float m, float p1, float p2, float p3, float Lf) {
     Params3 P;
-    P.z[0] = 0.0f; P.z[1] = p1; P.z[2] = p2;
-    const float d[3] = {p1, __fsub_rn(p2, p1), __fsub_rn(m, p2)};
+    P.z[0] = 0.0f; P.z[1] = p1; P.z[2] = p2; P.z[3] = p3;
+    const float d[4] = {p1, __fsub_rn(p2, p1), __fsub_rn(p3, p2), __fsub_rn(m, p3)};
 #pragma unroll
-    for (int r = 0; r < 3; ++r) {
+    for (int r = 0; r < 4; ++r) {
         if (d[r] > 0.0f) { P.s[r] = __fdiv_rn(d[r], Lf); P.inv[r] = __fdiv_rn(Lf, d[r]); }
         else             { P.s[r] = 0.0f;                P.inv[r] = 0.0f; }
     }
@@ -463,8 +645,8 @@ struct Row3 {
         first = warp_row_of(rows, warp_beg);
         last = warp_row_of(rows, min(warp_beg + 32 * (int64_t)kQ2PerThread, total) - 1);
     }
-    __device__ __forceinline__ void seek(const Rows& rows, const float* m_arr, const float* p1,
-                                         const float* p2, float Lf, int64_t i) {
+    __device__ __forceinline__ void seek(const Rows& rows, const float* m_arr, const BreakPts& bp,
+                                         float Lf, int64_t i) {
         if (row >= 0 && i < end) return;
         if (row < 0) {                                    // last row of [first, last] that begins at or before i
             int64_t lo = first, hi = last;
@@ -479,15 +661,15 @@ struct Row3 {
         while (rows.begin(row + 1) <= i) ++row;              // skips empty rows
         end = rows.begin(row + 1);
         m = __ldg(m_arr + row);
-        P = make_params3(m, __ldg(p1 + row), __ldg(p2 + row), Lf);
+        P = make_params3(m, __ldg(bp.p1 + row * bp.stride), __ldg(bp.p2 + row * bp.stride),
+                         bp.p3 ? __ldg(bp.p3 + row * bp.stride) : m, Lf);
     }
 };
 
 template <bool PACKED, bool WANT_FAKE>
 __global__ void __launch_bounds__(kQ2Threads)
 quantize2_kernel(const float* __restrict__ x, Rows rows, int64_t total, int bits,
-                 const float* __restrict__ m_arr, const float* __restrict__ p1_arr,
-                 const float* __restrict__ p2_arr, uint8_t* __restrict__ codes,
+                 const float* __restrict__ m_arr, BreakPts bp, uint8_t* __restrict__ codes,
                  uint8_t* __restrict__ region2, float* __restrict__ fake, int vec_ok) {
     const int64_t i0 = ((int64_t)blockIdx.x * kQ2Threads + threadIdx.x) * kQ2PerThread;
     Row3 rs;
@@ -511,15 +693,15 @@ quantize2_kernel(const float* __restrict__ x, Rows rows, int64_t total, int bits
         code[t] = reg[t] = 0;
         yv[t] = 0.0f;
         if (t < cnt) {
-            rs.seek(rows, m_arr, p1_arr, p2_arr, Lf, i0 + t);
+            rs.seek(rows, m_arr, bp, Lf, i0 + t);
             const float xi = vec ? xv[t] : x[i0 + t];
             float y = 0.0f;
             if (rs.m > 0.0f) {
                 const float a = fminf(fabsf(xi), rs.m);
-                const int r = (a > rs.P.z[1]) + (a > rs.P.z[2]);
-                const float z = r == 0 ? 0.0f : (r == 1 ? rs.P.z[1] : rs.P.z[2]);
-                const float inv = r == 0 ? rs.P.inv[0] : (r == 1 ? rs.P.inv[1] : rs.P.inv[2]);
-                const float s = r == 0 ? rs.P.s[0] : (r == 1 ? rs.P.s[1] : rs.P.s[2]);
+                const int r = (a > rs.P.z[1]) + (a > rs.P.z[2]) + (a > rs.P.z[3]);
+                const float z = r == 0 ? 0.0f : (r == 1 ? rs.P.z[1] : (r == 2 ? rs.P.z[2] : rs.P.z[3]));
+                const float inv = r == 0 ? rs.P.inv[0] : (r == 1 ? rs.P.inv[1] : (r == 2 ? rs.P.inv[2] : rs.P.inv[3]));
+                const float s = r == 0 ? rs.P.s[0] : (r == 1 ? rs.P.s[1] : (r == 2 ? rs.P.s[2] : rs.P.s[3]));
                 const float rr = __fadd_rn(__fmul_rn(__fsub_rn(a, z), inv), kMagic2);
                 const float q = fminf(__fsub_rn(rr, kMagic2), Lf);
                 const float v = __fadd_rn(__fmul_rn(q, s), z);
@@ -577,8 +759,7 @@ template <bool PACKED>
 __global__ void __launch_bounds__(kQ2Threads)
 dequantize2_kernel(const uint8_t* __restrict__ codes, const uint8_t* __restrict__ region2,
                    Rows rows, int64_t total, int bits, const float* __restrict__ m_arr,
-                   const float* __restrict__ p1_arr, const float* __restrict__ p2_arr,
-                   float* __restrict__ y, int vec_ok) {
+                   BreakPts bp, float* __restrict__ y, int vec_ok) {
     const int64_t i0 = ((int64_t)blockIdx.x * kQ2Threads + threadIdx.x) * kQ2PerThread;
     Row3 rs;
     rs.bracket(rows, i0 - (int64_t)(threadIdx.x & 31) * kQ2PerThread, total);
@@ -604,7 +785,7 @@ dequantize2_kernel(const uint8_t* __restrict__ codes, const uint8_t* __restrict_
     for (int t = 0; t < kQ2PerThread; ++t) {
         yv[t] = 0.0f;
         if (t < cnt) {
-            rs.seek(rows, m_arr, p1_arr, p2_arr, Lf, i0 + t);
+            rs.seek(rows, m_arr, bp, Lf, i0 + t);
             const int64_t i = i0 + t;
             int code, r;
             if (vec) {
@@ -615,9 +796,9 @@ dequantize2_kernel(const uint8_t* __restrict__ codes, const uint8_t* __restrict_
                 code = PACKED ? ((codes[i >> 1] >> ((i & 1) * 4)) & 0xF) : codes[i];
                 r = (region2[i >> 2] >> ((i & 3) * 2)) & 3;
             }
-            r = min(r, 2);
-            const float s = r == 0 ? rs.P.s[0] : (r == 1 ? rs.P.s[1] : rs.P.s[2]);
-            const float z = r == 0 ? 0.0f : (r == 1 ? rs.P.z[1] : rs.P.z[2]);
+            r = min(r, bp.p3 ? 3 : 2);
+            const float s = r == 0 ? rs.P.s[0] : (r == 1 ? rs.P.s[1] : (r == 2 ? rs.P.s[2] : rs.P.s[3]));
+            const float z = r == 0 ? 0.0f : (r == 1 ? rs.P.z[1] : (r == 2 ? rs.P.z[2] : rs.P.z[3]));
             float v = __fadd_rn(__fmul_rn((float)(code & qmask), s), z);
             int neg = (code >> (bits - 1)) & 1;
             if (!(rs.m > 0.0f)) { v = 0.0f; neg = 0; }
@@ -635,9 +816,10 @@ dequantize2_kernel(const uint8_t* __restrict__ codes, const uint8_t* __restrict_
 
 cudaError_t launch_quantize2(const float* x, const int64_t* row_offsets, int64_t C, int64_t n,
                              int64_t total, int bits, const float* m, const float* p1,
-                             const float* p2, uint8_t* codes, uint8_t* region2, float* fake,
-                             int layout, cudaStream_t stream) {
+                             const float* p2, const float* p3, int p_stride, uint8_t* codes,
+                             uint8_t* region2, float* fake, int layout, cudaStream_t stream) {
     if (total == 0) return cudaSuccess;
+    const BreakPts bp{p1, p2, p3, p_stride};
     Rows rows{row_offsets, C, n, n > 0 ? 1.0 / (double)n : 0.0, 0};
     const bool packed = (layout == 1 && bits <= 4);
     const int64_t per_cta = (int64_t)kQ2Threads * kQ2PerThread;
@@ -645,11 +827,11 @@ cudaError_t launch_quantize2(const float* x, const int64_t* row_offsets, int64_t
     auto al = [](const void* q, size_t a) { return (reinterpret_cast<uintptr_t>(q) & (a - 1)) == 0; };
     const int vec_ok = al(x, 16) && al(codes, 16) && al(region2, 4) && (!fake || al(fake, 16));
     if (packed) {
-        if (fake) quantize2_kernel<true, true><<<grid, kQ2Threads, 0, stream>>>(x, rows, total, bits, m, p1, p2, codes, region2, fake, vec_ok);
-        else      quantize2_kernel<true, false><<<grid, kQ2Threads, 0, stream>>>(x, rows, total, bits, m, p1, p2, codes, region2, fake, vec_ok);
+        if (fake) quantize2_kernel<true, true><<<grid, kQ2Threads, 0, stream>>>(x, rows, total, bits, m, bp, codes, region2, fake, vec_ok);
+        else      quantize2_kernel<true, false><<<grid, kQ2Threads, 0, stream>>>(x, rows, total, bits, m, bp, codes, region2, fake, vec_ok);
     } else {
-        if (fake) quantize2_kernel<false, true><<<grid, kQ2Threads, 0, stream>>>(x, rows, total, bits, m, p1, p2, codes, region2, fake, vec_ok);
-        else      quantize2_kernel<false, false><<<grid, kQ2Threads, 0, stream>>>(x, rows, total, bits, m, p1, p2, codes, region2, fake, vec_ok);
+        if (fake) quantize2_kernel<false, true><<<grid, kQ2Threads, 0, stream>>>(x, rows, total, bits, m, bp, codes, region2, fake, vec_ok);
+        else      quantize2_kernel<false, false><<<grid, kQ2Threads, 0, stream>>>(x, rows, total, bits, m, bp, codes, region2, fake, vec_ok);
     }
     return cudaGetLastError();
 }
@@ -657,16 +839,18 @@ cudaError_t launch_quantize2(const float* x, const int64_t* row_offsets, int64_t
 cudaError_t launch_dequantize2(const uint8_t* codes, const uint8_t* region2,
                                const int64_t* row_offsets, int64_t C, int64_t n, int64_t total,
                                int bits, const float* m, const float* p1, const float* p2,
-                               float* y, int layout, cudaStream_t stream) {
+                               const float* p3, int p_stride, float* y, int layout,
+                               cudaStream_t stream) {
     if (total == 0) return cudaSuccess;
+    const BreakPts bp{p1, p2, p3, p_stride};
     Rows rows{row_offsets, C, n, n > 0 ? 1.0 / (double)n : 0.0, 0};
     const bool packed = (layout == 1 && bits <= 4);
     const int64_t per_cta = (int64_t)kQ2Threads * kQ2PerThread;
     const unsigned grid = (unsigned)((total + per_cta - 1) / per_cta);
     auto al = [](const void* q, size_t a) { return (reinterpret_cast<uintptr_t>(q) & (a - 1)) == 0; };
     const int vec_ok = al(y, 16) && al(codes, 16) && al(region2, 4);
-    if (packed) dequantize2_kernel<true><<<grid, kQ2Threads, 0, stream>>>(codes, region2, rows, total, bits, m, p1, p2, y, vec_ok);
-    else        dequantize2_kernel<false><<<grid, kQ2Threads, 0, stream>>>(codes, region2, rows, total, bits, m, p1, p2, y, vec_ok);
+    if (packed) dequantize2_kernel<true><<<grid, kQ2Threads, 0, stream>>>(codes, region2, rows, total, bits, m, bp, y, vec_ok);
+    else        dequantize2_kernel<false><<<grid, kQ2Threads, 0, stream>>>(codes, region2, rows, total, bits, m, bp, y, vec_ok);
     return cudaGetLastError();
 }
 

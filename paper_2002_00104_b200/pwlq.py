@@ -60,6 +60,13 @@ _SIGNATURES = {
     "pwlq_search2": (_INT, [_P, _I64, _I64, _INT, _P, _INT, _P, _P, _P, _P, _P, _P, _P, _P, _SZ, _P]),
     "pwlq_search2_ragged": (_INT, [_P, _P, _I64, _I64, _I64, _INT, _P, _INT, _P, _P, _P, _P, _P,
                                    _P, _P, _P, _SZ, _P]),
+    "pwlq_search3": (_INT, [_P, _I64, _I64, _INT, _P, _INT, _P, _P, _P, _P, _P, _P, _SZ, _P]),
+    "pwlq_search3_ragged": (_INT, [_P, _P, _I64, _I64, _I64, _INT, _P, _INT, _P, _P, _P, _P, _P,
+                                   _P, _SZ, _P]),
+    "pwlq_quantize3": (_INT, [_P, _I64, _I64, _INT, _P, _P, _P, _P, _P, _INT, _P]),
+    "pwlq_quantize3_ragged": (_INT, [_P, _P, _I64, _I64, _INT, _P, _P, _P, _P, _P, _INT, _P]),
+    "pwlq_dequantize3": (_INT, [_P, _P, _I64, _I64, _INT, _P, _P, _P, _INT, _P]),
+    "pwlq_dequantize3_ragged": (_INT, [_P, _P, _P, _I64, _I64, _INT, _P, _P, _P, _INT, _P]),
     "pwlq_quantize2": (_INT, [_P, _I64, _I64, _INT, _P, _P, _P, _P, _P, _P, _INT, _P]),
     "pwlq_quantize2_ragged": (_INT, [_P, _P, _I64, _I64, _INT, _P, _P, _P, _P, _P, _P, _INT, _P]),
     "pwlq_dequantize2": (_INT, [_P, _P, _I64, _I64, _INT, _P, _P, _P, _P, _INT, _P]),
@@ -504,6 +511,10 @@ def dequantize_unsigned(codes, mask, bits, lo, hi, p, C=None, n=None, layout=COD
 
 
 # ---- two breakpoints: regions [0, p1], (p1, p2], (p2, m]; two-bit region index per value
+def search2_workspace_bytes(C: int, max_n: int, K: int) -> int:
+    return int(load_library().pwlq_search2_workspace_bytes(int(C), int(max_n), int(K)))
+
+
 def search2(x, bits, ratios, m, row_offsets=None, max_n=None, want_sse=False, workspace=None,
             stream=None):
     """Pair search; returns dict(p1, p2, err, idx1, idx2, sse ([C, K, K] or None), workspace)."""
@@ -512,7 +523,8 @@ def search2(x, bits, ratios, m, row_offsets=None, max_n=None, want_sse=False, wo
     K = ratios.numel()
     longest = n if row_offsets is None else int(max_n)
     if workspace is None:
-        workspace = torch.empty(256, dtype=torch.uint8, device=x.device)
+        workspace = torch.empty(search2_workspace_bytes(C, longest, K), dtype=torch.uint8,
+                                device=x.device)
     f32 = lambda: torch.empty(C, dtype=torch.float32, device=x.device)
     i32 = lambda: torch.empty(C, dtype=torch.int32, device=x.device)
     out = {"p1": f32(), "p2": f32(), "err": f32(), "idx1": i32(), "idx2": i32(),
@@ -579,6 +591,84 @@ def dequantize2(codes, region, bits, m, p1, p2, C=None, n=None, layout=CODES_U8,
                                          _dev(row_offsets, torch.int64, "row_offsets"), C, total,
                                          *tail)
     _check(rc, "pwlq_dequantize2")
+    return y
+
+
+# ---- three breakpoints: the breakpoints of a row side by side, [C, 3]
+def search3(x, bits, ratios, m, row_offsets=None, max_n=None, want_sse=False, workspace=None,
+            stream=None):
+    """Triple search; returns dict(p [C, 3], err, idx [C, 3], sse ([C, K, K, K] or None),
+    workspace)."""
+    lib = load_library()
+    C, n, total = _shape(x, row_offsets)
+    K = ratios.numel()
+    longest = n if row_offsets is None else int(max_n)
+    if workspace is None:
+        workspace = torch.empty(search2_workspace_bytes(C, longest, K), dtype=torch.uint8,
+                                device=x.device)
+    out = {"p": torch.empty((C, 3), dtype=torch.float32, device=x.device),
+           "err": torch.empty(C, dtype=torch.float32, device=x.device),
+           "idx": torch.empty((C, 3), dtype=torch.int32, device=x.device),
+           "sse": torch.empty((C, K, K, K), dtype=torch.float32, device=x.device) if want_sse else None}
+    tail = (int(bits), _dev(ratios, torch.float32, "ratios"), K, _dev(m, torch.float32, "m"),
+            _dev(out["p"], torch.float32, "p"), _dev(out["err"], torch.float32, "err"),
+            _dev(out["idx"], torch.int32, "idx"), _dev(out["sse"], torch.float32, "sse"),
+            _dev(workspace, torch.uint8, "workspace"), workspace.numel(), _stream(stream))
+    if row_offsets is None:
+        rc = lib.pwlq_search3(_dev(x, torch.float32, "x"), C, n, *tail)
+    else:
+        rc = lib.pwlq_search3_ragged(_dev(x, torch.float32, "x"),
+                                     _dev(row_offsets, torch.int64, "row_offsets"), C, total,
+                                     longest, *tail)
+    _check(rc, "pwlq_search3")
+    out["workspace"] = workspace
+    return out
+
+
+def quantize3(x, bits, m, p, layout=CODES_U8, row_offsets=None, want_fake=False, out=None,
+              stream=None):
+    """p: [C, 3].  Returns (codes uint8, region2 uint8 (two bits per value), fake fp32 or None)."""
+    lib = load_library()
+    C, n, total = _shape(x, row_offsets)
+    if out is None:
+        codes = torch.empty(code_bytes(total, bits, layout), dtype=torch.uint8, device=x.device)
+        region = torch.empty((total + 3) // 4, dtype=torch.uint8, device=x.device)
+        fake = torch.empty(total, dtype=torch.float32, device=x.device) if want_fake else None
+    else:
+        codes, region, fake = out
+    tail = (int(bits), _dev(m, torch.float32, "m"), _dev(p, torch.float32, "p"),
+            _dev(codes, torch.uint8, "codes"), _dev(region, torch.uint8, "region2"),
+            _dev(fake, torch.float32, "fake"), int(layout), _stream(stream))
+    if row_offsets is None:
+        rc = lib.pwlq_quantize3(_dev(x, torch.float32, "x"), C, n, *tail)
+    else:
+        rc = lib.pwlq_quantize3_ragged(_dev(x, torch.float32, "x"),
+                                       _dev(row_offsets, torch.int64, "row_offsets"), C, total,
+                                       *tail)
+    _check(rc, "pwlq_quantize3")
+    return codes, region, fake
+
+
+def dequantize3(codes, region, bits, m, p, C=None, n=None, layout=CODES_U8, row_offsets=None,
+                out=None, stream=None):
+    lib = load_library()
+    if row_offsets is None:
+        total = int(C) * int(n)
+    else:
+        C = row_offsets.numel() - 1
+        total = int(out.numel()) if out is not None else int(row_offsets[-1].item())
+    y = out if out is not None else torch.empty(total, dtype=torch.float32, device=codes.device)
+    tail = (int(bits), _dev(m, torch.float32, "m"), _dev(p, torch.float32, "p"),
+            _dev(y, torch.float32, "y"), int(layout), _stream(stream))
+    if row_offsets is None:
+        rc = lib.pwlq_dequantize3(_dev(codes, torch.uint8, "codes"),
+                                  _dev(region, torch.uint8, "region2"), int(C), int(n), *tail)
+    else:
+        rc = lib.pwlq_dequantize3_ragged(_dev(codes, torch.uint8, "codes"),
+                                         _dev(region, torch.uint8, "region2"),
+                                         _dev(row_offsets, torch.int64, "row_offsets"), C, total,
+                                         *tail)
+    _check(rc, "pwlq_dequantize3")
     return y
 
 

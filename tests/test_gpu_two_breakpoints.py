@@ -86,6 +86,35 @@ def test_search2_ragged_mixed_rows(pwlq, oracle):
     assert (got["idx1"][4], got["idx2"][4], got["p2"][4]) == (0, 1, 0.0)
 
 
+@pytest.mark.parametrize("bits,K,C,n", [(4, 16, 3, 8193), (3, 12, 2, 20000), (8, 8, 1, 70001)])
+def test_search2_rows_longer_than_a_tile(pwlq, oracle, bits, K, C, n):
+    """Rows cut into tiles of 8192 values: the tiles' terms are added by the row-closing kernel."""
+    rng = np.random.default_rng(n + K)
+    x = rng.laplace(0, 0.02, (C, n)).astype(np.float32)
+    m = oracle.absmax(x)
+    ratios = W.ratio_grid(K)
+    got, status = run_search2(pwlq, x, bits, ratios, m)
+    assert status == 0
+    check_pairs(got, oracle.search2(x, bits, ratios, m), ratios, m, n)
+    again, _ = run_search2(pwlq, x, bits, ratios, m)
+    assert all(np.array_equal(got[k], again[k]) for k in got)           # fixed order of the tiles
+
+
+def test_search2_ragged_rows_with_and_without_tiles(pwlq, oracle):
+    rng = np.random.default_rng(5)
+    lengths = [9001, 0, 300, 8192, 16385, 1, 12000]
+    x = rng.standard_normal(sum(lengths)).astype(np.float32)
+    ro = np.concatenate([[0], np.cumsum(lengths)]).astype(np.int64)
+    x[ro[2]:ro[3]] = 0.0                                        # a row of zeros among tiled rows
+    m = oracle.absmax(x, ro)
+    ratios = W.ratio_grid(10)
+    got, status = run_search2(pwlq, x, 4, ratios, m, row_offsets=ro, max_n=max(lengths))
+    assert status == 0
+    check_pairs(got, oracle.search2(x, 4, ratios, m, row_offsets=ro), ratios, m, np.diff(ro))
+    assert (got["idx1"][1], got["idx2"][1], got["err"][1]) == (0, 1, 0.0)
+    assert (got["idx1"][2], got["idx2"][2], got["p2"][2]) == (0, 1, 0.0)
+
+
 def test_search2_with_p2_at_m_contains_the_one_breakpoint_search(pwlq):
     """Pairs (i, K-1) with ratios[K-1] = 1 are the one-breakpoint candidates i (same arithmetic up
     to the summation order)."""
@@ -106,9 +135,11 @@ def test_search2_limits_and_bad_grid(pwlq):
     with pytest.raises(pwlq.PwlqError) as e:
         pwlq.search2(x, 4, dev(W.ratio_grid(65)), m)
     assert e.value.status == pwlq.ERR_UNSUPPORTED
+    small = torch.empty(256, dtype=torch.uint8, device="cuda")           # a long row needs more
     with pytest.raises(pwlq.PwlqError) as e:
-        pwlq.search2(torch.zeros(1, 8200, device="cuda"), 4, dev(W.ratio_grid(8)), m[:1])
-    assert e.value.status == pwlq.ERR_UNSUPPORTED
+        pwlq.search2(torch.zeros(1, 8200, device="cuda"), 4, dev(W.ratio_grid(8)), m[:1],
+                     workspace=small)
+    assert e.value.status == pwlq.ERR_WORKSPACE
     with pytest.raises(pwlq.PwlqError):
         pwlq.search2(x, 4, dev(W.ratio_grid(1)), m)
     out = pwlq.search2(x, 4, dev(np.array([0.5, 0.25, 1.0], np.float32)), m)   # not ascending
