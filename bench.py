@@ -545,7 +545,30 @@ def extras(torch, pwlq, path: DevicePath, flush, hbm, K2=32):
                                                        C=w.C, n=path.dense_n, layout=1, out=y, **kw),
                        flush)
         out["dequantize2"] = {"ms": t, "hbm_cold_frac": nb / (t * 1e-3) / 1e9 / hbm}
-    except pwlq.PwlqError as e:                   # e.g. rows beyond the pair search's limit
+        # three breakpoints: the pair search's terms plus O(K^2) per row
+        s3 = pwlq.search3(x, bits, r2, m, max_n=path.max_n, workspace=ws2, **kw)
+        t = timed_call(torch, lambda: pwlq.search3(x, bits, r2, m, max_n=path.max_n, workspace=ws2,
+                                                   **kw), flush)
+        triples = K2 * (K2 - 1) * (K2 - 2) // 6
+        out["search3"] = {"K": K2, "triples": triples, "ms": t,
+                          "sse_two_over_three_breakpoints":
+                              float((s2["err"].double().sum() / s3["err"].double().sum()).item())}
+        c3, g3, _ = pwlq.quantize3(x, bits, m, s3["p"], layout=1, **kw)
+        t = timed_call(torch, lambda: pwlq.quantize3(x, bits, m, s3["p"], layout=1,
+                                                     out=(c3, g3, None), **kw), flush)
+        out["quantize3"] = {"ms": t, "hbm_cold_frac": nb / (t * 1e-3) / 1e9 / hbm}
+        del c3, g3
+        # the pair search on one long row (a tensor quantized per layer): tiles of 8192 values
+        wl = W.relu_activation()
+        xl = torch.from_numpy(wl.x).to(path.dev).view(1, -1)
+        ml = pwlq.absmax(xl)
+        sl = pwlq.search2(xl, bits, r2, ml)
+        t = timed_call(torch, lambda: pwlq.search2(xl, bits, r2, ml, workspace=sl["workspace"]),
+                       flush, reps=3)
+        out["search2_one_row_of_25.7M"] = {"K": K2, "pairs": pairs, "ms": t,
+                                           "t_value_pairs_per_s": wl.total * pairs / (t * 1e-3) / 1e12}
+        del xl, sl, wl
+    except pwlq.PwlqError as e:
         out["search2"] = {"skipped": str(e)}
     p = path.sout["p"]
     t = timed_call(torch, lambda: pwlq.select_analytic(x, m, pwlq.MODEL_GAUSS_ROOT,
