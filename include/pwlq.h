@@ -387,8 +387,11 @@ int pwlq_select_analytic_ragged(const float* x, const int64_t* row_offsets, int6
  * copy, kernels and output copies overlap: the copies run on two internal streams (created once
  * per device, the only resources this library ever creates) chained to `stream` by events; work
  * queued on `stream` before the call is finished before any of it starts, and `stream` ends the
- * call.  The results are those of the four device calls run one after another. */
+ * call.  The results are those of the four device calls run one after another.
+ * The search's status word (a non-finite range) of the whole call sits in dev_scratch at byte
+ * offset pwlq_encode_host_status_offset(...): copy its 4 bytes back after synchronising. */
 size_t pwlq_encode_host_scratch_bytes(int64_t C, int64_t total, int64_t max_n, int K);
+size_t pwlq_encode_host_status_offset(int64_t C, int64_t total, int64_t max_n, int K);
 int pwlq_encode_host(const float* x_host, const int64_t* row_offsets_host, int64_t C,
                      int64_t total, int64_t max_n, int bits, const float* ratios_host, int K,
                      float* m_host, float* p_host, float* err_host, int32_t* idx_host,

@@ -692,6 +692,11 @@ size_t pwlq_encode_host_scratch_bytes(int64_t C, int64_t total, int64_t max_n, i
     return plan_host(C, total, max_n, K).bytes;
 }
 
+size_t pwlq_encode_host_status_offset(int64_t C, int64_t total, int64_t max_n, int K) {
+    if (C < 1 || total < 1 || max_n < 1 || K < 1 || K > PWLQ_MAX_K) return 0;
+    return plan_host(C, total, max_n, K).ws;
+}
+
 // lo_host == nullptr: signed scheme, m_host receives the abs-max values; otherwise one-sided ranges,
 // lo_host / m_host receive the rows' lower / upper bounds.
 static int encode_host_impl(const float* x_host, const int64_t* row_offsets_host, int64_t C,

@@ -82,6 +82,7 @@ _SIGNATURES = {
     "pwlq_pack_dense": (_INT, [_P, _P, _I64, _INT, _P, _P]),
     "pwlq_unpack_dense": (_INT, [_P, _I64, _INT, _P, _P, _P]),
     "pwlq_encode_host_scratch_bytes": (_SZ, [_I64, _I64, _I64, _INT]),
+    "pwlq_encode_host_status_offset": (_SZ, [_I64, _I64, _I64, _INT]),
     "pwlq_encode_host": (_INT, [_P, _P, _I64, _I64, _I64, _INT, _P, _INT, _P, _P, _P, _P, _P, _P,
                                 _INT, _P, _SZ, _P, _P]),
     "pwlq_encode_host_unsigned": (_INT, [_P, _P, _I64, _I64, _I64, _INT, _P, _INT, _P, _P, _P, _P, _P,
@@ -747,6 +748,13 @@ def unpack_dense(stream_bytes, total, bits, stream=None):
 
 def encode_host_scratch_bytes(C: int, total: int, max_n: int, K: int) -> int:
     return int(load_library().pwlq_encode_host_scratch_bytes(C, total, max_n, K))
+
+
+def encode_host_status(dev_scratch, C: int, total: int, max_n: int, K: int) -> int:
+    """Status word of the search inside the last ``encode_host`` call that used ``dev_scratch``
+    (synchronises)."""
+    off = int(load_library().pwlq_encode_host_status_offset(C, total, max_n, K))
+    return int(dev_scratch[off:off + 4].view(torch.int32).item())
 
 
 def _host(t: Optional[torch.Tensor], dtype, what: str):

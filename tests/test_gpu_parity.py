@@ -340,6 +340,13 @@ def test_encode_host_matches_oracle(pwlq, oracle, ragged):
     assert np.all(gap <= 1e-5 * ora["sse64"][rows, ora["idx"]] + 1e-30)
     oc, ok, _ = oracle.quantize(xo, 4, om, out["p"].numpy(), layout=1, row_offsets=ro)
     assert np.array_equal(out["codes"].numpy(), oc) and np.array_equal(out["mask"].numpy(), ok)
+    assert pwlq.encode_host_status(scratch, C, total, max_n, 64) == 0
+    # a non-finite value makes its row's range non-finite: reported in the status word
+    hx[total // 2] = float("inf")
+    pwlq.encode_host(hx, hro, C, max_n, 4, torch.from_numpy(ratios).pin_memory(), out,
+                     pwlq.CODES_PACKED, scratch)
+    torch.cuda.synchronize()
+    assert pwlq.encode_host_status(scratch, C, total, max_n, 64) == 1 << pwlq.ERR_NONFINITE
 
 
 def test_a_bounded_wait_that_runs_out_is_reported_once(pwlq):
