@@ -895,6 +895,13 @@ cudaError_t launch_search(const float* x, const int64_t* row_offsets, int64_t C,
                                      cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_max);
             if (e != cudaSuccess) return e;
         }
+        if (plan.tile == kSearchTile && total / C < 512) {
+            // Mostly short rows (the library sees the mean length only): the small-CTA classes
+            // hold the bulk of the work and go first, so that the stream does not end with their
+            // long tail of half-empty SMs (MobileNetV2 shapes: 244 -> 236 us; with the longest
+            // class first the ResNet-50 shapes are 0.5 % faster, hence the two orders).
+            std::swap(classes[0], classes[2]);
+        }
         const int full_cap = a.cap;
         int launched = 0;
         for (const RowClass& rc : classes) {
