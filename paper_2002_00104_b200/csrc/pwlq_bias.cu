@@ -205,21 +205,113 @@ unpack_dense_kernel(const uint8_t* __restrict__ in, int64_t total, int bits,
     mask[i0 >> 3] = (uint8_t)mb;
 }
 
+// Whole groups of 32 values with aligned buffers: a thread reads its 32 codes and 32 region bits
+// as two 128-bit words and one 32-bit word and writes b + 1 whole 32-bit words of the stream
+// (every shift is a compile-time constant).
+template <int BITS>
+__global__ void __launch_bounds__(kPkThreads)
+pack_dense32_kernel(const uint8_t* __restrict__ codes, const uint8_t* __restrict__ mask,
+                    int64_t groups32, uint8_t* __restrict__ out) {
+    constexpr int W = BITS + 1;
+    const int64_t g = (int64_t)blockIdx.x * kPkThreads + threadIdx.x;
+    if (g >= groups32) return;
+    const uint4 c0 = __ldcs(reinterpret_cast<const uint4*>(codes) + 2 * g);
+    const uint4 c1 = __ldcs(reinterpret_cast<const uint4*>(codes) + 2 * g + 1);
+    const uint32_t mb = __ldcs(reinterpret_cast<const uint32_t*>(mask) + g);
+    const uint32_t cw[8] = {c0.x, c0.y, c0.z, c0.w, c1.x, c1.y, c1.z, c1.w};
+    uint32_t ow[W + 1];
+#pragma unroll
+    for (int j = 0; j <= W; ++j) ow[j] = 0u;
+#pragma unroll
+    for (int t = 0; t < 32; ++t) {
+        const uint32_t field = ((cw[t >> 2] >> (8 * (t & 3))) & ((1u << BITS) - 1u)) |
+                               (((mb >> t) & 1u) << BITS);
+        const int word = (t * W) >> 5, sh = (t * W) & 31;
+        ow[word] |= field << sh;
+        if (sh + W > 32) ow[word + 1] |= field >> (32 - sh);
+    }
+    uint32_t* dst = reinterpret_cast<uint32_t*>(out) + g * W;
+#pragma unroll
+    for (int j = 0; j < W; ++j) __stcs(dst + j, ow[j]);
+}
+
+template <int BITS>
+__global__ void __launch_bounds__(kPkThreads)
+unpack_dense32_kernel(const uint8_t* __restrict__ in, int64_t groups32,
+                      uint8_t* __restrict__ codes, uint8_t* __restrict__ mask) {
+    constexpr int W = BITS + 1;
+    const int64_t g = (int64_t)blockIdx.x * kPkThreads + threadIdx.x;
+    if (g >= groups32) return;
+    const uint32_t* src = reinterpret_cast<const uint32_t*>(in) + g * W;
+    uint32_t iw[W + 1];
+#pragma unroll
+    for (int j = 0; j < W; ++j) iw[j] = __ldcs(src + j);
+    iw[W] = 0u;
+    uint32_t cw[8] = {0u, 0u, 0u, 0u, 0u, 0u, 0u, 0u}, mb = 0u;
+#pragma unroll
+    for (int t = 0; t < 32; ++t) {
+        const int word = (t * W) >> 5, sh = (t * W) & 31;
+        uint32_t field = iw[word] >> sh;
+        if (sh + W > 32) field |= iw[word + 1] << (32 - sh);
+        cw[t >> 2] |= (field & ((1u << BITS) - 1u)) << (8 * (t & 3));
+        mb |= ((field >> BITS) & 1u) << t;
+    }
+    __stcs(reinterpret_cast<uint4*>(codes) + 2 * g, make_uint4(cw[0], cw[1], cw[2], cw[3]));
+    __stcs(reinterpret_cast<uint4*>(codes) + 2 * g + 1, make_uint4(cw[4], cw[5], cw[6], cw[7]));
+    __stcs(reinterpret_cast<uint32_t*>(mask) + g, mb);
+}
+
+static inline bool pk_aligned(const void* p, size_t a) {
+    return (reinterpret_cast<uintptr_t>(p) & (a - 1)) == 0;
+}
+
 cudaError_t launch_pack_dense(const uint8_t* codes, const uint8_t* mask, int64_t total, int bits,
                               uint8_t* out, cudaStream_t stream) {
     if (total == 0) return cudaSuccess;
-    const int64_t groups = (total + 7) / 8;
-    pack_dense_kernel<<<(unsigned)((groups + kPkThreads - 1) / kPkThreads), kPkThreads, 0, stream>>>(
-        codes, mask, total, bits, out);
+    // whole groups of 32 values through the word-wise kernel, the rest (and everything, when a
+    // buffer is not aligned) through the byte-wise one
+    int64_t done = 0;
+    if (pk_aligned(codes, 16) && pk_aligned(mask, 4) && pk_aligned(out, 4) && total >= 32) {
+        const int64_t g32 = total / 32;
+        const unsigned grid = (unsigned)((g32 + kPkThreads - 1) / kPkThreads);
+        switch (bits) {
+#define PWLQ_PACK_CASE(B) case B: pack_dense32_kernel<B><<<grid, kPkThreads, 0, stream>>>(codes, mask, g32, out); break;
+            PWLQ_PACK_CASE(2) PWLQ_PACK_CASE(3) PWLQ_PACK_CASE(4) PWLQ_PACK_CASE(5)
+            PWLQ_PACK_CASE(6) PWLQ_PACK_CASE(7) PWLQ_PACK_CASE(8)
+#undef PWLQ_PACK_CASE
+            default: return cudaErrorInvalidValue;
+        }
+        done = g32 * 32;
+    }
+    if (done < total) {
+        const int64_t groups = (total - done + 7) / 8;
+        pack_dense_kernel<<<(unsigned)((groups + kPkThreads - 1) / kPkThreads), kPkThreads, 0, stream>>>(
+            codes + done, mask + done / 8, total - done, bits, out + done / 8 * (bits + 1));
+    }
     return cudaGetLastError();
 }
 
 cudaError_t launch_unpack_dense(const uint8_t* in, int64_t total, int bits, uint8_t* codes,
                                 uint8_t* mask, cudaStream_t stream) {
     if (total == 0) return cudaSuccess;
-    const int64_t groups = (total + 7) / 8;
-    unpack_dense_kernel<<<(unsigned)((groups + kPkThreads - 1) / kPkThreads), kPkThreads, 0, stream>>>(
-        in, total, bits, codes, mask);
+    int64_t done = 0;
+    if (pk_aligned(codes, 16) && pk_aligned(mask, 4) && pk_aligned(in, 4) && total >= 32) {
+        const int64_t g32 = total / 32;
+        const unsigned grid = (unsigned)((g32 + kPkThreads - 1) / kPkThreads);
+        switch (bits) {
+#define PWLQ_UNPACK_CASE(B) case B: unpack_dense32_kernel<B><<<grid, kPkThreads, 0, stream>>>(in, g32, codes, mask); break;
+            PWLQ_UNPACK_CASE(2) PWLQ_UNPACK_CASE(3) PWLQ_UNPACK_CASE(4) PWLQ_UNPACK_CASE(5)
+            PWLQ_UNPACK_CASE(6) PWLQ_UNPACK_CASE(7) PWLQ_UNPACK_CASE(8)
+#undef PWLQ_UNPACK_CASE
+            default: return cudaErrorInvalidValue;
+        }
+        done = g32 * 32;
+    }
+    if (done < total) {
+        const int64_t groups = (total - done + 7) / 8;
+        unpack_dense_kernel<<<(unsigned)((groups + kPkThreads - 1) / kPkThreads), kPkThreads, 0, stream>>>(
+            in + done / 8 * (bits + 1), total - done, bits, codes + done, mask + done / 8);
+    }
     return cudaGetLastError();
 }
 

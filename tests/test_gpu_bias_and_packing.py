@@ -99,8 +99,8 @@ def test_corrected_rows_keep_mean_and_norm_on_the_device(pwlq):
     assert torch.allclose(ny, nx, rtol=1e-5)
 
 
-@pytest.mark.parametrize("bits", [2, 3, 4, 6, 7, 8])
-@pytest.mark.parametrize("total", [1, 8, 1003, 65536 + 5])
+@pytest.mark.parametrize("bits", [2, 3, 4, 5, 6, 7, 8])
+@pytest.mark.parametrize("total", [1, 8, 31, 32, 1003, 65536 + 5])
 def test_dense_stream_pack_and_unpack(pwlq, oracle, bits, total):
     rng = np.random.default_rng(bits * 7 + total)
     codes = rng.integers(0, 2 ** bits, total).astype(np.uint8)
@@ -110,6 +110,26 @@ def test_dense_stream_pack_and_unpack(pwlq, oracle, bits, total):
     assert s.numel() == pwlq.dense_bytes(total, bits) == want.size
     assert np.array_equal(np_(s), want)
     c2, m2 = pwlq.unpack_dense(s, total, bits)
+    assert np.array_equal(np_(c2), codes) and np.array_equal(np_(m2), mask)
+
+
+@pytest.mark.parametrize("bits", [3, 4, 8])
+def test_dense_stream_from_unaligned_buffers(pwlq, oracle, bits):
+    """Buffers that start off the word boundaries take the byte-wise kernels: same stream."""
+    total = 5000
+    rng = np.random.default_rng(bits)
+    codes = rng.integers(0, 2 ** bits, total).astype(np.uint8)
+    mask = np.packbits(rng.integers(0, 2, total).astype(np.uint8), bitorder="little")
+    cbuf = torch.zeros(total + 16, dtype=torch.uint8, device="cuda")
+    mbuf = torch.zeros(mask.size + 16, dtype=torch.uint8, device="cuda")
+    cbuf[3:3 + total] = dev(codes)
+    mbuf[1:1 + mask.size] = dev(mask)
+    want = oracle.pack_dense(codes, mask, bits)
+    s = pwlq.pack_dense(cbuf[3:3 + total], mbuf[1:1 + mask.size], bits)
+    assert np.array_equal(np_(s), want)
+    sbuf = torch.zeros(want.size + 8, dtype=torch.uint8, device="cuda")
+    sbuf[1:1 + want.size] = s
+    c2, m2 = pwlq.unpack_dense(sbuf[1:1 + want.size], total, bits)
     assert np.array_equal(np_(c2), codes) and np.array_equal(np_(m2), mask)
 
 
