@@ -18,9 +18,12 @@ Prints ONE JSON line.
                  a packed-FMA micro-benchmark run here
   hbm_stages     the three HBM-bound kernels as timed inside the step (one cold launch each after
                  the L2 eviction); hbm_streaming: the same kernels back to back on the workload's
-                 rows repeated until they exceed L2
+                 rows repeated until they exceed L2, and under `mapped` the same calls given row
+                 maps built once per layout (pwlq_rowmap_build) where several rows share a span
   sustained      at least two seconds of back-to-back steps with the SM clock sampled meanwhile
   workloads      the other benchmark configurations, each with its stage times and fractions
+  extras         the calls beyond the four-call path (two / three breakpoints, analytic selection,
+                 bias correction, dense packing) as single cold launches
   cpu_baseline   the CPU oracle on the host cores (all cores, and one thread)
 With N > 1 (torchrun) every rank processes its own batch (rows are independent: no collective on
 the data path) and the slowest rank's time counts.  `--impl reference` times the CPU oracle on a

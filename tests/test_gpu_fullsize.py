@@ -178,3 +178,32 @@ def test_encode_host_in_several_runs_equals_the_resident_path(pwlq, oracle, layo
         else:
             got_row = got[ro[c]:ro[c + 1]]
         assert np.array_equal(got_row, oc)
+
+
+@pytest.mark.parametrize("name", ["resnet50", "mobilenetv2"])
+def test_prebuilt_row_maps_at_full_size(pwlq, oracle, name):
+    """The *_mapped calls on the benchmark's ragged layouts, repeated as the streaming leg of the
+    benchmark repeats them (two copies back to back): every range, code byte, region byte and
+    reconstructed value against the oracle."""
+    w = getattr(W, name)()
+    copies = 2
+    x = np.tile(w.x, copies)
+    ro = np.concatenate([w.row_offsets[:-1] + k * w.total for k in range(copies)] +
+                        [np.array([copies * w.total])]).astype(np.int64)
+    C, total = ro.size - 1, x.size
+    xd, rod = dev(x), dev(ro)
+    rowmap = pwlq.rowmap_build(C, total, row_offsets=rod)
+    m = pwlq.absmax(xd, row_offsets=rod, rowmap=rowmap)
+    om = oracle.absmax(x, ro)
+    assert np.array_equal(m.cpu().numpy(), om)
+    p = (om * np.float32(0.3)).astype(np.float32)
+    codes, mask, fake = pwlq.quantize(xd, w.bits, m, dev(p), layout=pwlq.CODES_PACKED,
+                                      row_offsets=rod, want_fake=True, rowmap=rowmap)
+    y = pwlq.dequantize(codes, mask, w.bits, m, dev(p), layout=pwlq.CODES_PACKED, row_offsets=rod,
+                        rowmap=rowmap)
+    torch.cuda.synchronize()
+    assert pwlq.device_status() == 0
+    oc, ok, of = oracle.quantize(x, w.bits, om, p, layout=1, row_offsets=ro)
+    assert np.array_equal(codes.cpu().numpy(), oc) and np.array_equal(mask.cpu().numpy(), ok)
+    assert fake.cpu().numpy().tobytes() == of.tobytes()
+    assert y.cpu().numpy().tobytes() == of.tobytes()
