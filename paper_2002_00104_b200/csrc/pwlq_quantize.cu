@@ -373,7 +373,6 @@ quantize_map_kernel(const float* __restrict__ x, Rows rows, int64_t total, int b
     }
     Stage* st = reinterpret_cast<Stage*>(smem_raw);
     __shared__ uint64_t full_bar[kMapStages], empty_bar[kMapStages];
-    const unsigned full = 0xffffffffu;
     const int Li = UNS ? (1 << bits) - 1 : (1 << (bits - 1)) - 1;    // largest level of a piece
     const float Lf = (float)Li;
     const uint32_t sign_unit = 1u << (bits - 1);
