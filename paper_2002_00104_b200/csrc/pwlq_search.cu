@@ -393,23 +393,23 @@ __host__ __device__ inline size_t sorted_smem_layout(int cap, int K, int warps, 
 }
 
 // j(a) = number of candidates with p_k < a, for ascending ps[0..K).  A linear-grid guess is
-// verified and corrected by up to three neighbour steps; grids far from linear fall back to a
-// binary search between the bounds found so far.  Exact for every ascending grid.
-__device__ __forceinline__ int bucket_of(const float* ps, int K, float a, float p_first,
-                                         float hint_scale) {
-    int j = min((int)ceilf(fmaxf((a - p_first) * hint_scale, 0.0f)), K);
+// verified against its two neighbours; a guess that is off (rounding at a boundary, a grid that
+// is not linear) is replaced by a binary search, kept out of line so that the common path stays
+// a dozen instructions without branches.  Exact for every ascending grid.
+__device__ __noinline__ int bucket_search(const float* ps, int K, float a) {
     int lo = 0, hi = K;                               // the answer lies in [lo, hi]
-#pragma unroll
-    for (int t = 0; t < 3; ++t) {
-        if (j > 0 && !(ps[j - 1] < a)) { hi = min(hi, j - 1); --j; }
-        else if (j < K && ps[j] < a)   { lo = max(lo, j + 1); ++j; }
-        else return j;
-    }
     while (lo < hi) {
         const int mid = (lo + hi) >> 1;
         if (ps[mid] < a) lo = mid + 1; else hi = mid;
     }
     return lo;
+}
+__device__ __forceinline__ int bucket_of(const float* ps, int K, float a, float p_first,
+                                         float hint_scale) {
+    const int j = min((int)ceilf(fmaxf((a - p_first) * hint_scale, 0.0f)), K);
+    const float below = ps[max(j - 1, 0)], at = ps[min(j, K - 1)];
+    const bool ok = (j == 0 || below < a) && (j == K || !(at < a));
+    return ok ? j : bucket_search(ps, K, a);
 }
 
 template <int kCW, bool EXACT_V>
