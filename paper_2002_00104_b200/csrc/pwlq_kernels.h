@@ -94,6 +94,17 @@ cudaError_t launch_dequantize2(const uint8_t* codes, const uint8_t* region2,
                                const float* p3, int p_stride, float* y, int layout,
                                cudaStream_t stream);
 
+// The element-wise forms (any alignment; what the two above fall back to).
+cudaError_t launch_quantize2_plain(const float* x, const int64_t* row_offsets, int64_t C, int64_t n,
+                             int64_t total, int bits, const float* m, const float* p1,
+                             const float* p2, const float* p3, int p_stride, uint8_t* codes,
+                             uint8_t* region2, float* fake, int layout, cudaStream_t stream);
+cudaError_t launch_dequantize2_plain(const uint8_t* codes, const uint8_t* region2,
+                               const int64_t* row_offsets, int64_t C, int64_t n, int64_t total,
+                               int bits, const float* m, const float* p1, const float* p2,
+                               const float* p3, int p_stride, float* y, int layout,
+                               cudaStream_t stream);
+
 // Bias correction: folded scale xi and offset beta per row; dequantize that applies them; dense
 // (b+1)-bit storage of code and region bit.
 size_t bias_workspace_bytes(int64_t C, int64_t max_n);

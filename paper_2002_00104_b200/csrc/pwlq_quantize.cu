@@ -12,6 +12,7 @@
 #include "pwlq_common.cuh"
 #include "pwlq_kernels.h"
 #include "pwlq_pipeline.cuh"
+#include "pwlq_multi.cuh"
 #include "pwlq_rowmap.cuh"
 
 namespace pwlq {
@@ -950,6 +951,425 @@ dequantize_map_kernel(const uint8_t* __restrict__ codes, const uint8_t* __restri
     }
 }
 
+// ------------------------------------------------ two or three breakpoints per row (Sec. 5.1)
+// The same producer / consumer structure for rows with three or four regions: the producer
+// describes the rows of every span (row map, and per row one record of constants per region, see
+// store_row_consts_multi), the consumers quantize or expand eight consecutive values per lane and
+// pass; a value's constants are one shared-memory read indexed by its region.  The region index 0..3 takes two bits per value (16 bits per lane and pass).
+// Whole spans with a usable map take the form below; the tensor's last, partial span and spans
+// the map cannot describe go value by value with a lookup in global memory.
+template <bool DATA>
+struct MultiStage {
+    alignas(128) float data[DATA ? kMapSpan : 4];
+    SpanRowMap map;
+    alignas(16) float4 q[4 * kMultiSlots];
+};
+
+// Region, offset, L / range and step of magnitude a in a row with breakpoints z = (p1, p2, p3, m).
+__device__ __forceinline__ int region_of(float a, const float4& z) {
+    return (a > z.x) + (a > z.y) + (a > z.z);
+}
+__device__ __forceinline__ float pick4(int r, float v0, const float4& v) {
+    return r == 0 ? v0 : (r == 1 ? v.x : (r == 2 ? v.y : v.z));
+}
+__device__ __forceinline__ float pick4(int r, const float4& v) {
+    return r == 0 ? v.x : (r == 1 ? v.y : (r == 2 ? v.z : v.w));
+}
+
+// One value of a row with constants (z, inv, s): code, region and delivered value; the sequence
+// of the element-wise kernel (every product and sum rounded on its own).  A row with m <= 0
+// delivers zeros.
+__device__ __forceinline__ void quantize_multi_value(float xi, const float4& z, const float4& inv,
+                                                     const float4& s, float Lf, int bits,
+                                                     uint32_t& code, uint32_t& reg, float& y) {
+    const float m = z.w;
+    const float a = fminf(fabsf(xi), m);
+    const int r = region_of(a, z);
+    const float zr = pick4(r, 0.0f, z);
+    const float rr = __fadd_rn(__fmul_rn(__fsub_rn(a, zr), pick4(r, inv)), 12582912.0f);
+    const float q = fminf(__fsub_rn(rr, 12582912.0f), Lf);
+    const float v = __fadd_rn(__fmul_rn(q, pick4(r, s)), zr);
+    const int neg = xi < 0.0f;
+    const bool ok = m > 0.0f;
+    code = ok ? (uint32_t)((neg << (bits - 1)) | (int)q) : 0u;
+    reg = ok ? (uint32_t)r : 0u;
+    y = ok ? (neg ? -v : v) : 0.0f;
+}
+
+struct QuantizeMultiCtx {
+    Rows rows;
+    const float* __restrict__ m;
+    BreakPts bp;
+    int64_t total;
+    int bits;
+    float Lf;
+    uint8_t* __restrict__ codes;
+    uint8_t* __restrict__ region2;
+    float* __restrict__ fake;
+};
+
+// The constants of the row in slot l that a lane keeps in registers: the three breakpoints, the
+// range and the sign mask (0 for a row that delivers zeros).
+struct MultiRow {
+    const float4* rec;
+    float p1, p2, p3, m;
+    uint32_t smask;
+    __device__ __forceinline__ void load(const float4* q, int l) {
+        rec = q + 4 * l;
+        const float4 c0 = rec[0], c1 = rec[1];
+        m = c0.w;
+        p1 = c1.x;
+        smask = __float_as_uint(c1.w);
+        p2 = rec[2].x;
+        p3 = rec[3].x;
+    }
+};
+
+// One pass of a consumer lane over the eight values at offset li of a whole span with a usable
+// map (all outputs vector-aligned).  Per value the sequence of the element-wise kernel, every
+// product and sum rounded on its own; the sign is the sign bit of x + 0.0 (so that -0.0 is not
+// negative) under the row's mask.
+template <bool PACKED, bool WANT_FAKE>
+__device__ __forceinline__ void quantize_multi_pass(const QuantizeMultiCtx& g, const float* data,
+                                                    const SpanRowMap& M, const float4* q,
+                                                    int64_t span_beg, int li) {
+    const float4 xa = *reinterpret_cast<const float4*>(data + li);
+    const float4 xb = *reinterpret_cast<const float4*>(data + li + 4);
+    const float xv[8] = {xa.x, xa.y, xa.z, xa.w, xb.x, xb.y, xb.z, xb.w};
+    uint32_t word;
+    const int l = map_slot(M, li, word);
+    const uint32_t inner = (word >> ((li & 31) + 1)) & 0x7Fu;       // starts at li+1 .. li+7
+    MultiRow R;
+    R.load(q, l);
+    const int sign_shift = 32 - g.bits;
+    uint32_t w0 = 0, w1 = 0, rw = 0;
+    float yv[8];
+#pragma unroll
+    for (int t = 0; t < 8; ++t) {
+        if (t > 0 && (inner & (1u << (t - 1))))                     // a row starts at this value
+            R.load(q, l + __popc(inner & ((1u << t) - 1u)));
+        const float xi = xv[t];
+        const float a = fminf(fabsf(xi), R.m);
+        const int r = (a > R.p1) + (a > R.p2) + (a > R.p3);
+        const float4 c = R.rec[r];                                  // (z, L / range, step, -)
+        const float rr = __fadd_rn(__fmul_rn(__fsub_rn(a, c.x), c.y), 12582912.0f);
+        const float qf = fminf(__fsub_rn(rr, 12582912.0f), g.Lf);
+        const float v = __fadd_rn(__fmul_rn(qf, c.z), c.x);
+        const uint32_t sign = __float_as_uint(__fadd_rn(xi, 0.0f)) & R.smask;
+        const uint32_t code = (sign >> sign_shift) | (uint32_t)(int)qf;
+        yv[t] = __uint_as_float(__float_as_uint(v) | sign);
+        if (PACKED) w0 |= code << (4 * t);
+        else if (t < 4) w0 |= code << (8 * t);
+        else w1 |= code << (8 * (t - 4));
+        rw |= (uint32_t)r << (2 * t);
+    }
+    // span_beg is a multiple of the span: 32-bit offsets inside the span's slices of the outputs
+    reinterpret_cast<uint16_t*>(g.region2 + (span_beg >> 2))[li >> 3] = (uint16_t)rw;
+    if (PACKED) reinterpret_cast<uint32_t*>(g.codes + (span_beg >> 1))[li >> 3] = w0;
+    else        reinterpret_cast<uint2*>(g.codes + span_beg)[li >> 3] = make_uint2(w0, w1);
+    if (WANT_FAKE) {
+        float4* f = reinterpret_cast<float4*>(g.fake + span_beg) + (li >> 2);
+        __stcs(f, make_float4(yv[0], yv[1], yv[2], yv[3]));
+        __stcs(f + 1, make_float4(yv[4], yv[5], yv[6], yv[7]));
+    }
+}
+
+// The same value by value, rows looked up in global memory: the tensor's last span, and spans
+// without a usable map.
+template <bool PACKED, bool WANT_FAKE>
+__device__ __forceinline__ void quantize_multi_slow(const QuantizeMultiCtx& g, const float* data,
+                                                    int64_t span_beg, int li) {
+    const int64_t i0 = span_beg + li;
+    const int cnt = (int)max((int64_t)0, min((int64_t)8, g.total - i0));
+    if (cnt == 0) return;
+    Row3 rs;
+    rs.whole(g.rows);
+    uint32_t code[8], reg[8];
+#pragma unroll
+    for (int t = 0; t < 8; ++t) {
+        code[t] = reg[t] = 0;
+        if (t < cnt) {
+            rs.seek(g.rows, g.m, g.bp, g.Lf, i0 + t);
+            const float4 z = make_float4(rs.P.z[1], rs.P.z[2], rs.P.z[3], rs.m);
+            const float4 inv = make_float4(rs.P.inv[0], rs.P.inv[1], rs.P.inv[2], rs.P.inv[3]);
+            const float4 s = make_float4(rs.P.s[0], rs.P.s[1], rs.P.s[2], rs.P.s[3]);
+            float y;
+            quantize_multi_value(data[li + t], z, inv, s, g.Lf, g.bits, code[t], reg[t], y);
+            if (WANT_FAKE) g.fake[i0 + t] = y;
+        }
+    }
+#pragma unroll
+    for (int b = 0; b < 2; ++b)
+        if (4 * b < cnt)
+            g.region2[(i0 >> 2) + b] = (uint8_t)(reg[4 * b] | (reg[4 * b + 1] << 2) |
+                                                 (reg[4 * b + 2] << 4) | (reg[4 * b + 3] << 6));
+    if (PACKED) {
+#pragma unroll
+        for (int b = 0; b < 4; ++b)
+            if (2 * b < cnt) g.codes[(i0 >> 1) + b] = (uint8_t)(code[2 * b] | (code[2 * b + 1] << 4));
+    } else {
+#pragma unroll
+        for (int t = 0; t < 8; ++t)
+            if (t < cnt) g.codes[i0 + t] = (uint8_t)code[t];
+    }
+}
+
+// P3: the rows have a third breakpoint.  x, codes, region2 and fake are vector-aligned (the
+// launcher sends everything else to the element-wise kernel).
+template <bool PACKED, bool WANT_FAKE, bool P3>
+__global__ void __launch_bounds__(kMapThreads, 3)
+quantize_multi_kernel(const float* __restrict__ x, Rows rows, int64_t total, int bits,
+                      const float* __restrict__ m, BreakPts bp, uint8_t* __restrict__ codes,
+                      uint8_t* __restrict__ region2, float* __restrict__ fake,
+                      int64_t spans_per_cta) {
+    typedef MultiStage<true> Stage;
+    extern __shared__ __align__(128) unsigned char smem_raw[];
+    Stage* st = reinterpret_cast<Stage*>(smem_raw);
+    __shared__ uint64_t full_bar[kMapStages], empty_bar[kMapStages];
+    const float Lf = (float)((1 << (bits - 1)) - 1);
+    const int64_t nspans = (total + kMapSpan - 1) / kMapSpan;
+    const int64_t first = blockIdx.x * spans_per_cta, last = min(first + spans_per_cta, nspans);
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < kMapStages; ++s) {
+            mbar_init(&full_bar[s], 2);            // the data (or its stand-in) and the map
+            mbar_init(&empty_bar[s], kMapConsumers);
+        }
+        fence_barrier_init();
+    }
+    __syncthreads();
+    if (first >= last) return;
+
+    if (warp == kMapConsumers) {
+        // ---- producer
+        MapProducer<true, false, false, P3, 2> prod;
+        prod.rows = rows;
+        prod.in = RowInputs{m, bp.p2, bp.p1, bp.p3, nullptr};
+        prod.Lf = Lf;
+        prod.pstride = bp.stride;
+        for (int64_t span = first; span < last && span < first + kMapStages; ++span) {
+            const unsigned bytes = q_bulk_bytes(span, total, 1);
+            if (bytes != 0 && lane == 0) {
+                mbar_expect_tx(&full_bar[span - first], bytes);
+                bulk_copy_g2s(st[span - first].data, x + span * kMapSpan, bytes, &full_bar[span - first]);
+            }
+        }
+        prod.request(warp_row_of(rows, first * kMapSpan), true);
+        int64_t it = 0;
+        for (int64_t span = first; span < last; ++span, ++it) {
+            const int s = (int)(it % kMapStages);
+            const unsigned use = (unsigned)(it / kMapStages);
+            if (use > 0 && !mbar_wait(&empty_bar[s], (use - 1) & 1u)) {
+                // never expected: report, let the copies of the earlier spans land, and leave
+                if (lane == 0) atomicOr(&g_quantize_timeout, 1);
+                for (int64_t j = it - 1; j >= 0 && j > it - 1 - kMapStages; --j)
+                    mbar_wait(&full_bar[j % kMapStages], (unsigned)(j / kMapStages) & 1u);
+                return;
+            }
+            const int64_t span_beg = span * kMapSpan, span_end = min(span_beg + kMapSpan, total);
+            const unsigned bytes = q_bulk_bytes(span, total, 1);
+            if (bytes != 0) {
+                if (lane == 0 && use > 0) {        // (first round: requested above)
+                    mbar_expect_tx(&full_bar[s], bytes);
+                    bulk_copy_g2s(st[s].data, x + span_beg, bytes, &full_bar[s]);
+                }
+            } else {                               // ragged tail: plain loads
+                for (int i = lane; i < (int)(span_end - span_beg); i += 32) st[s].data[i] = x[span_beg + i];
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&full_bar[s]);
+            }
+            prod.build(st[s].map, st[s].q, nullptr, span_beg, span_end, span + 1 < last);
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&full_bar[s]);
+        }
+        return;
+    }
+
+    // ---- consumers
+    const QuantizeMultiCtx ctx{rows, m, bp, total, bits, Lf, codes, region2, fake};
+    const int li0 = warp * (kMapSpan / kMapConsumers) + lane * 8;     // pass c: li0 + 256 c
+    int64_t it = 0;
+    for (int64_t span = first; span < last; ++span, ++it) {
+        const int s = (int)(it % kMapStages);
+        const unsigned use = (unsigned)(it / kMapStages);
+        if (!mbar_wait_relaxed(&full_bar[s], use & 1u)) {
+            if (lane == 0) atomicOr(&g_quantize_timeout, 1);
+            return;
+        }
+        const int64_t span_beg = span * kMapSpan;
+        const Stage& S = st[s];
+        if (S.map.slow == 0 && span_beg + kMapSpan <= total) {
+#pragma unroll
+            for (int c = 0; c < 2; ++c)
+                quantize_multi_pass<PACKED, WANT_FAKE>(ctx, S.data, S.map, S.q, span_beg, li0 + c * 256);
+        } else {
+#pragma unroll 1
+            for (int c = 0; c < 2; ++c)
+                quantize_multi_slow<PACKED, WANT_FAKE>(ctx, S.data, span_beg, li0 + c * 256);
+        }
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&empty_bar[s]);
+    }
+}
+
+// A thread's codes and region bits of one span, requested ahead of use (whole spans: one load
+// per stream and pass; the tensor's last span byte by byte).
+template <bool PACKED>
+struct MultiCodeRegs {
+    uint32_t w0[kQChunks], w1[kQChunks], rw[kQChunks];
+    __device__ __forceinline__ void load(const uint8_t* __restrict__ codes,
+                                         const uint8_t* __restrict__ region2, int64_t span_beg,
+                                         int64_t total, int li0) {
+#pragma unroll
+        for (int c = 0; c < kQChunks; ++c) {
+            const int li = li0 + c * 256;
+            w0[c] = w1[c] = rw[c] = 0;
+            if (span_beg + kMapSpan <= total) {
+                const int g8 = li >> 3;
+                rw[c] = __ldcs(reinterpret_cast<const unsigned short*>(region2 + (span_beg >> 2)) + g8);
+                if (PACKED) {
+                    w0[c] = __ldcs(reinterpret_cast<const unsigned int*>(codes + (span_beg >> 1)) + g8);
+                } else {
+                    const uint2 w = __ldcs(reinterpret_cast<const uint2*>(codes + span_beg) + g8);
+                    w0[c] = w.x; w1[c] = w.y;
+                }
+            } else {
+                const int64_t i0 = span_beg + li;
+                const int cnt = (int)max((int64_t)0, min((int64_t)8, total - i0));
+                for (int t = 0; t < cnt; ++t) {
+                    const int64_t i = i0 + t;
+                    const uint32_t code = PACKED ? ((codes[i >> 1] >> ((i & 1) * 4)) & 0xFu) : codes[i];
+                    if (PACKED) w0[c] |= code << (4 * t);
+                    else if (t < 4) w0[c] |= code << (8 * t);
+                    else w1[c] |= code << (8 * (t - 4));
+                    rw[c] |= (uint32_t)((region2[i >> 2] >> ((i & 3) * 2)) & 3u) << (2 * t);
+                }
+            }
+        }
+    }
+};
+
+// Delivered value of one code in a row with breakpoints z = (p1, p2, p3, m) and steps s.
+__device__ __forceinline__ float dequantize_multi_value(uint32_t code, int r, const float4& z,
+                                                        const float4& s, int bits, int qmask) {
+    const float v = __fadd_rn(__fmul_rn((float)(int)(code & (uint32_t)qmask), pick4(r, s)),
+                              pick4(r, 0.0f, z));
+    const bool neg = ((code >> (bits - 1)) & 1u) != 0;
+    return z.w > 0.0f ? (neg ? -v : v) : 0.0f;
+}
+
+template <bool PACKED, bool P3>
+__global__ void __launch_bounds__(kMapThreads, 3)
+dequantize_multi_kernel(const uint8_t* __restrict__ codes, const uint8_t* __restrict__ region2,
+                        Rows rows, int64_t total, int bits, const float* __restrict__ m,
+                        BreakPts bp, float* __restrict__ y, int64_t spans_per_cta) {
+    typedef MultiStage<false> Stage;
+    extern __shared__ __align__(128) unsigned char smem_raw[];
+    Stage* st = reinterpret_cast<Stage*>(smem_raw);
+    __shared__ uint64_t full_bar[kMapStages], empty_bar[kMapStages];
+    const int qmask = (1 << (bits - 1)) - 1;
+    const float Lf = (float)qmask;
+    const int rmax = P3 ? 3 : 2;
+    const int sign_shift = 32 - bits;                 // moves a code's sign bit to bit 31
+    const int64_t nspans = (total + kMapSpan - 1) / kMapSpan;
+    const int64_t first = blockIdx.x * spans_per_cta, last = min(first + spans_per_cta, nspans);
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < kMapStages; ++s) {
+            mbar_init(&full_bar[s], 1);
+            mbar_init(&empty_bar[s], kMapConsumers);
+        }
+        fence_barrier_init();
+    }
+    __syncthreads();
+    if (first >= last) return;
+
+    if (warp == kMapConsumers) {
+        // ---- producer: row maps and constants only
+        MapProducer<true, false, true, P3, 2> prod;
+        prod.rows = rows;
+        prod.in = RowInputs{m, bp.p2, bp.p1, bp.p3, nullptr};
+        prod.Lf = Lf;
+        prod.pstride = bp.stride;
+        prod.request(warp_row_of(rows, first * kMapSpan), true);
+        int64_t it = 0;
+        for (int64_t span = first; span < last; ++span, ++it) {
+            const int s = (int)(it % kMapStages);
+            const unsigned use = (unsigned)(it / kMapStages);
+            if (use > 0 && !mbar_wait(&empty_bar[s], (use - 1) & 1u)) {
+                if (lane == 0) atomicOr(&g_quantize_timeout, 1);
+                return;
+            }
+            const int64_t span_beg = span * kMapSpan, span_end = min(span_beg + kMapSpan, total);
+            prod.build(st[s].map, st[s].q, nullptr, span_beg, span_end, span + 1 < last);
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&full_bar[s]);
+        }
+        return;
+    }
+
+    // ---- consumers
+    const int li0 = warp * (kMapSpan / kMapConsumers) + lane * 8;     // pass c: li0 + 256 c
+    MultiCodeRegs<PACKED> cur, nxt;
+    cur.load(codes, region2, first * kMapSpan, total, li0);
+    int64_t it = 0;
+    for (int64_t span = first; span < last; ++span, ++it) {
+        const int s = (int)(it % kMapStages);
+        const unsigned use = (unsigned)(it / kMapStages);
+        const int64_t span_beg = span * kMapSpan;
+        if (span + 1 < last) nxt.load(codes, region2, span_beg + kMapSpan, total, li0);
+        if (!mbar_wait_relaxed(&full_bar[s], use & 1u)) {
+            if (lane == 0) atomicOr(&g_quantize_timeout, 1);
+            return;
+        }
+        const Stage& S = st[s];
+        const bool whole = S.map.slow == 0 && span_beg + kMapSpan <= total;
+#pragma unroll
+        for (int c = 0; c < kQChunks; ++c) {
+            const int li = li0 + c * 256;
+            const uint32_t w0 = cur.w0[c], w1 = cur.w1[c], rw = cur.rw[c];
+            if (whole) {
+                uint32_t word;
+                const int l = map_slot(S.map, li, word);
+                const uint32_t inner = (word >> ((li & 31) + 1)) & 0x7Fu;
+                const float4* rec = S.q + 4 * l;
+                uint32_t smask = __float_as_uint(rec[1].w);
+                float yv[8];
+#pragma unroll
+                for (int t = 0; t < 8; ++t) {
+                    if (t > 0 && (inner & (1u << (t - 1)))) {
+                        rec = S.q + 4 * (l + __popc(inner & ((1u << t) - 1u)));
+                        smask = __float_as_uint(rec[1].w);
+                    }
+                    const uint32_t code = code_of<PACKED>(w0, w1, t);
+                    const float4 c = rec[min((int)((rw >> (2 * t)) & 3u), rmax)];   // (z, -, step, -)
+                    const float v = __fadd_rn(__fmul_rn((float)(int)(code & (uint32_t)qmask), c.z), c.x);
+                    yv[t] = __uint_as_float(__float_as_uint(v) | ((code << sign_shift) & smask));
+                }
+                float4* f = reinterpret_cast<float4*>(y + span_beg) + (li >> 2);
+                __stcs(f, make_float4(yv[0], yv[1], yv[2], yv[3]));
+                __stcs(f + 1, make_float4(yv[4], yv[5], yv[6], yv[7]));
+            } else {
+                const int64_t i0 = span_beg + li;
+                const int cnt = (int)max((int64_t)0, min((int64_t)8, total - i0));
+                Row3 rs;
+                rs.whole(rows);
+                for (int t = 0; t < cnt; ++t) {
+                    rs.seek(rows, m, bp, Lf, i0 + t);
+                    const float4 z = make_float4(rs.P.z[1], rs.P.z[2], rs.P.z[3], rs.m);
+                    const float4 sv = make_float4(rs.P.s[0], rs.P.s[1], rs.P.s[2], rs.P.s[3]);
+                    y[i0 + t] = dequantize_multi_value(code_of<PACKED>(w0, w1, t),
+                                                       min((int)((rw >> (2 * t)) & 3u), rmax), z, sv,
+                                                       bits, qmask);
+                }
+            }
+        }
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&empty_bar[s]);
+        cur = nxt;
+    }
+}
+
 static inline bool aligned(const void* p, size_t a) {
     return (reinterpret_cast<uintptr_t>(p) & (a - 1)) == 0;
 }
@@ -1112,6 +1532,71 @@ cudaError_t launch_dequantize(const uint8_t* codes, const uint8_t* mask,
 #undef PWLQ_LAUNCH_DEQUANTIZE_LONG
 #undef PWLQ_LAUNCH_DEQUANTIZE
 #undef PWLQ_LAUNCH_DEQUANTIZE_AS
+    return cudaGetLastError();
+}
+
+// Two or three breakpoints per row (p3 == nullptr: two).  Vector-aligned buffers go through the
+// producer / consumer kernels; anything else, and layouts whose rows are so short that most spans
+// would have no usable map, through the element-wise kernels.
+static bool multi_by_maps(int64_t C, int64_t total, bool vec_ok) {
+    return vec_ok && total >= 16 * C;
+}
+cudaError_t launch_quantize2(const float* x, const int64_t* row_offsets, int64_t C, int64_t n,
+                             int64_t total, int bits, const float* m, const float* p1,
+                             const float* p2, const float* p3, int p_stride, uint8_t* codes,
+                             uint8_t* region2, float* fake, int layout, cudaStream_t stream) {
+    if (total == 0) return cudaSuccess;
+    const bool vec_ok = aligned(x, 16) && aligned(codes, 16) && aligned(region2, 4) &&
+                        (!fake || aligned(fake, 16));
+    if (!multi_by_maps(C, total, vec_ok))
+        return launch_quantize2_plain(x, row_offsets, C, n, total, bits, m, p1, p2, p3, p_stride,
+                                      codes, region2, fake, layout, stream);
+    const BreakPts bp{p1, p2, p3, p_stride};
+    Rows rows{row_offsets, C, n, n > 0 ? 1.0 / (double)n : 0.0, 0};
+    const bool packed = (layout == 1 && bits <= 4);
+    const int64_t nspans = (total + kQSpan - 1) / kQSpan;
+    const size_t msmem = sizeof(MultiStage<true>) * kMapStages;
+#define PWLQ_LAUNCH_QM(PK, FK, P3)                                                                \
+    do {                                                                                          \
+        const SpanGrid g = span_grid((const void*)quantize_multi_kernel<PK, FK, P3>, kMapThreads, \
+                                     msmem, nspans, true);                                        \
+        quantize_multi_kernel<PK, FK, P3><<<g.grid, kMapThreads, msmem, stream>>>(                \
+            x, rows, total, bits, m, bp, codes, region2, fake, g.per_cta);                        \
+    } while (0)
+#define PWLQ_LAUNCH_QM3(PK, FK) \
+    do { if (p3) PWLQ_LAUNCH_QM(PK, FK, true); else PWLQ_LAUNCH_QM(PK, FK, false); } while (0)
+    if (packed) { if (fake) PWLQ_LAUNCH_QM3(true, true); else PWLQ_LAUNCH_QM3(true, false); }
+    else        { if (fake) PWLQ_LAUNCH_QM3(false, true); else PWLQ_LAUNCH_QM3(false, false); }
+#undef PWLQ_LAUNCH_QM3
+#undef PWLQ_LAUNCH_QM
+    return cudaGetLastError();
+}
+
+cudaError_t launch_dequantize2(const uint8_t* codes, const uint8_t* region2,
+                               const int64_t* row_offsets, int64_t C, int64_t n, int64_t total,
+                               int bits, const float* m, const float* p1, const float* p2,
+                               const float* p3, int p_stride, float* y, int layout,
+                               cudaStream_t stream) {
+    if (total == 0) return cudaSuccess;
+    const bool vec_ok = aligned(y, 16) && aligned(codes, 16) && aligned(region2, 4);
+    if (!multi_by_maps(C, total, vec_ok))
+        return launch_dequantize2_plain(codes, region2, row_offsets, C, n, total, bits, m, p1, p2,
+                                        p3, p_stride, y, layout, stream);
+    const BreakPts bp{p1, p2, p3, p_stride};
+    Rows rows{row_offsets, C, n, n > 0 ? 1.0 / (double)n : 0.0, 0};
+    const bool packed = (layout == 1 && bits <= 4);
+    const int64_t nspans = (total + kQSpan - 1) / kQSpan;
+    const size_t msmem = sizeof(MultiStage<false>) * kMapStages;
+#define PWLQ_LAUNCH_DM(PK, P3)                                                                    \
+    do {                                                                                          \
+        const SpanGrid g = span_grid((const void*)dequantize_multi_kernel<PK, P3>, kMapThreads,   \
+                                     msmem, nspans, true);                                        \
+        dequantize_multi_kernel<PK, P3><<<g.grid, kMapThreads, msmem, stream>>>(                  \
+            codes, region2, rows, total, bits, m, bp, y, g.per_cta);                              \
+    } while (0)
+    if (packed) { if (p3) PWLQ_LAUNCH_DM(true, true); else PWLQ_LAUNCH_DM(true, false); }
+    else        { if (p3) PWLQ_LAUNCH_DM(false, true); else PWLQ_LAUNCH_DM(false, false); }
+#undef PWLQ_LAUNCH_DM
     return cudaGetLastError();
 }
 

@@ -27,6 +27,7 @@
 #pragma once
 
 #include "pwlq_common.cuh"
+#include "pwlq_multi.cuh"
 #include "pwlq_pipeline.cuh"
 
 namespace pwlq {
@@ -106,11 +107,15 @@ __device__ __forceinline__ void store_row_consts(float4* qa, float4* qb, int slo
 // The producer warp's view of the rows.  Rows are looked at in chunks of 32 consecutive rows
 // (chunk c = rows 32 c .. 32 c + 31, lane = row % 32); the two chunks from the current first row
 // on are held in registers.  Every member function is called by all 32 lanes.
-template <bool PARAMS, bool UNS, bool DEQ = false, bool BC = false>
+// NBP > 1: rows with two or three breakpoints.  in.p, in.lo and in.xi then point to p1, p2 and p3
+// (BC: a third breakpoint exists), read with stride pstride; the constants of a row are three
+// 128-bit words in qa (store_row_consts_multi), for at most kMultiSlots rows per span.
+template <bool PARAMS, bool UNS, bool DEQ = false, bool BC = false, int NBP = 1>
 struct MapProducer {
     Rows rows;
     RowInputs in;
     float Lf;
+    int pstride;                // NBP > 1 only
     int64_t rf;                 // row that holds the first value of the next span
     int64_t ch0, ch1;           // chunk held in (o0, m0, p0, lo0): even chunks; (o1, ...): odd chunks
     int64_t o0, o1;             // offset of row 32 ch + lane (INT64_MAX past the last offset)
@@ -120,6 +125,13 @@ struct MapProducer {
     __device__ __forceinline__ void load_inputs(int64_t r, float& mv, float& pv, float& lov,
                                                 float& xv, float& bv) const {
         mv = __ldg(in.m + r);
+        if (NBP > 1) {                              // (p1, p2, p3) in (pv, lov, xv); p3 = m without one
+            pv = __ldg(in.p + r * pstride);
+            lov = __ldg(in.lo + r * pstride);
+            xv = BC ? __ldg(in.xi + r * pstride) : mv;
+            bv = 0.0f;
+            return;
+        }
         pv = __ldg(in.p + r);
         lov = 0.0f;
         if (UNS) lov = __ldg(in.lo + r);            // m stays the upper bound until it is used
@@ -188,8 +200,12 @@ struct MapProducer {
                 }
                 if (PARAMS) {
                     if (k >= 2) load_inputs(r, mv, pv, lov, xv, bv);
-                    if (UNS) mv = __fsub_rn(mv, lov);              // range width
-                    store_row_consts<DEQ>(qa, qb, s, mv, pv, lov, xv, bv, Lf);
+                    if (NBP > 1) {
+                        if (s < kMultiSlots) store_row_consts_multi(qa, s, mv, pv, lov, xv, Lf);
+                    } else {
+                        if (UNS) mv = __fsub_rn(mv, lov);          // range width
+                        store_row_consts<DEQ>(qa, qb, s, mv, pv, lov, xv, bv, Lf);
+                    }
                 }
             }
             const unsigned in_mask = __ballot_sync(full, inside);
@@ -241,9 +257,10 @@ struct MapProducer {
         // rows that start at the same position (empty rows) set one bit between them
         const bool dup = __shfl_sync(full, incl, 31) != total_in - 1;
         if (lane == 0) {
+            const bool unusable = dup || overflow || (NBP > 1 && total_in > kMultiSlots);
             M.first_row = this_rf;
-            M.slow = (dup || overflow) ? 1 : 0;
-            M.nrows = (dup || overflow) ? 0 : total_in;
+            M.slow = unusable ? 1 : 0;
+            M.nrows = unusable ? 0 : total_in;
         }
     }
 

@@ -16,6 +16,7 @@
 
 #include "pwlq_common.cuh"
 #include "pwlq_kernels.h"
+#include "pwlq_multi.cuh"
 
 namespace pwlq {
 
@@ -603,68 +604,8 @@ cudaError_t launch_search2(const float* x, const int64_t* row_offsets, int64_t C
 }
 
 // ------------------------------------------------ quantize / dequantize, three or four regions
-// Breakpoints of the rows: two arrays (p3 == nullptr: three regions) or three, read with a stride
-// (1 for separate arrays, 3 for one [C, 3] array).
-struct BreakPts {
-    const float* p1;
-    const float* p2;
-    const float* p3;
-    int stride;
-};
-// Constants of the regions of one row.  Without a third breakpoint the fourth region starts at m
-// and is never entered (a <= m).
-struct Params3 {
-    float z[4], s[4], inv[4];
-};
-__device__ __forceinline__ Params3 make_params3(float m, float p1, float p2, float p3, float Lf) {
-    Params3 P;
-    P.z[0] = 0.0f; P.z[1] = p1; P.z[2] = p2; P.z[3] = p3;
-    const float d[4] = {p1, __fsub_rn(p2, p1), __fsub_rn(p3, p2), __fsub_rn(m, p3)};
-#pragma unroll
-    for (int r = 0; r < 4; ++r) {
-        if (d[r] > 0.0f) { P.s[r] = __fdiv_rn(d[r], Lf); P.inv[r] = __fdiv_rn(Lf, d[r]); }
-        else             { P.s[r] = 0.0f;                P.inv[r] = 0.0f; }
-    }
-    return P;
-}
-
 constexpr int kQ2Threads = 256;
 constexpr int kQ2PerThread = 16;      // consecutive values per thread: four region bytes
-
-// Row state of a thread that walks consecutive values.
-struct Row3 {
-    int64_t row = -1, end = 0;
-    int64_t first = 0, last = 0;       // the rows of the warp's values: bounds of the first lookup
-    float m = 0.0f;
-    Params3 P;
-    // The rows that hold the first and the last value of the warp's 32 x kQ2PerThread values,
-    // found by the warp together (a few dependent loads instead of a bisection over all rows per
-    // thread).  Every lane of the warp calls this, before any lane leaves.
-    __device__ __forceinline__ void bracket(const Rows& rows, int64_t warp_beg, int64_t total) {
-        if (warp_beg >= total) return;
-        first = warp_row_of(rows, warp_beg);
-        last = warp_row_of(rows, min(warp_beg + 32 * (int64_t)kQ2PerThread, total) - 1);
-    }
-    __device__ __forceinline__ void seek(const Rows& rows, const float* m_arr, const BreakPts& bp,
-                                         float Lf, int64_t i) {
-        if (row >= 0 && i < end) return;
-        if (row < 0) {                                    // last row of [first, last] that begins at or before i
-            int64_t lo = first, hi = last;
-            while (hi > lo) {
-                const int64_t mid = (lo + hi + 1) >> 1;
-                if (rows.begin(mid) <= i) lo = mid; else hi = mid - 1;
-            }
-            row = lo;
-        } else {
-            row = row + 1;
-        }
-        while (rows.begin(row + 1) <= i) ++row;              // skips empty rows
-        end = rows.begin(row + 1);
-        m = __ldg(m_arr + row);
-        P = make_params3(m, __ldg(bp.p1 + row * bp.stride), __ldg(bp.p2 + row * bp.stride),
-                         bp.p3 ? __ldg(bp.p3 + row * bp.stride) : m, Lf);
-    }
-};
 
 template <bool PACKED, bool WANT_FAKE>
 __global__ void __launch_bounds__(kQ2Threads)
@@ -673,7 +614,7 @@ quantize2_kernel(const float* __restrict__ x, Rows rows, int64_t total, int bits
                  uint8_t* __restrict__ region2, float* __restrict__ fake, int vec_ok) {
     const int64_t i0 = ((int64_t)blockIdx.x * kQ2Threads + threadIdx.x) * kQ2PerThread;
     Row3 rs;
-    rs.bracket(rows, i0 - (int64_t)(threadIdx.x & 31) * kQ2PerThread, total);
+    rs.bracket(rows, i0 - (int64_t)(threadIdx.x & 31) * kQ2PerThread, 32 * kQ2PerThread, total);
     if (i0 >= total) return;
     const float Lf = (float)((1 << (bits - 1)) - 1);
     const int cnt = (int)min((int64_t)kQ2PerThread, total - i0);
@@ -762,7 +703,7 @@ dequantize2_kernel(const uint8_t* __restrict__ codes, const uint8_t* __restrict_
                    BreakPts bp, float* __restrict__ y, int vec_ok) {
     const int64_t i0 = ((int64_t)blockIdx.x * kQ2Threads + threadIdx.x) * kQ2PerThread;
     Row3 rs;
-    rs.bracket(rows, i0 - (int64_t)(threadIdx.x & 31) * kQ2PerThread, total);
+    rs.bracket(rows, i0 - (int64_t)(threadIdx.x & 31) * kQ2PerThread, 32 * kQ2PerThread, total);
     if (i0 >= total) return;
     const float Lf = (float)((1 << (bits - 1)) - 1);
     const int qmask = (1 << (bits - 1)) - 1;
@@ -814,7 +755,7 @@ dequantize2_kernel(const uint8_t* __restrict__ codes, const uint8_t* __restrict_
     }
 }
 
-cudaError_t launch_quantize2(const float* x, const int64_t* row_offsets, int64_t C, int64_t n,
+cudaError_t launch_quantize2_plain(const float* x, const int64_t* row_offsets, int64_t C, int64_t n,
                              int64_t total, int bits, const float* m, const float* p1,
                              const float* p2, const float* p3, int p_stride, uint8_t* codes,
                              uint8_t* region2, float* fake, int layout, cudaStream_t stream) {
@@ -836,7 +777,7 @@ cudaError_t launch_quantize2(const float* x, const int64_t* row_offsets, int64_t
     return cudaGetLastError();
 }
 
-cudaError_t launch_dequantize2(const uint8_t* codes, const uint8_t* region2,
+cudaError_t launch_dequantize2_plain(const uint8_t* codes, const uint8_t* region2,
                                const int64_t* row_offsets, int64_t C, int64_t n, int64_t total,
                                int bits, const float* m, const float* p1, const float* p2,
                                const float* p3, int p_stride, float* y, int layout,

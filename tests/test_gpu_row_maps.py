@@ -179,3 +179,81 @@ def test_maps_of_another_layout_are_reported(pwlq):
     small = torch.empty(64, dtype=torch.uint8, device="cuda")
     with pytest.raises(Exception):
         pwlq.rowmap_build(40, x.size, row_offsets=dev(ro), out=small)
+
+
+# ------------------------------------------------- two and three breakpoints on the same layouts
+def multi_layouts():
+    out = dict(layouts())
+    # around the number of rows a span's stage holds constants for (384): 372 / 409 rows per span
+    out["rows_of_11"] = [11] * 1500
+    out["rows_of_10"] = [10] * 1700
+    # long rows with short ones in between, a tail that is not a multiple of anything
+    out["long_and_short"] = [9000, 13, 4096 * 3, 40, 41, 42, 12289, 5]
+    return out
+
+
+def breakpoints(om, nbp, seed):
+    rng = np.random.default_rng(seed)
+    r = np.sort(rng.uniform(0.03, 1.0, (om.size, nbp)), axis=1)
+    r[::4, nbp - 1] = 1.0                              # last breakpoint = m: the last region is empty
+    return (om[:, None] * r).astype(np.float32)
+
+
+@pytest.mark.parametrize("bits,layout", [(3, 1), (4, 0), (8, 0)])
+@pytest.mark.parametrize("name", sorted(multi_layouts()))
+def test_quantize2_dequantize2_layouts(pwlq, oracle, name, bits, layout):
+    x, ro = make(multi_layouts()[name], 21)
+    om = oracle.absmax(x, ro)
+    om[3::11] = 0.0                                    # rows delivered as zeros
+    p = breakpoints(om, 2, 5)
+    p1, p2 = np.ascontiguousarray(p[:, 0]), np.ascontiguousarray(p[:, 1])
+    oc, orr, of = oracle.quantize2(x, bits, om, p1, p2, layout=layout, row_offsets=ro)
+    for want_fake in (True, False):
+        codes, reg, fake = pwlq.quantize2(dev(x), bits, dev(om), dev(p1), dev(p2), layout=layout,
+                                          row_offsets=dev(ro), want_fake=want_fake)
+        assert np.array_equal(np_(codes), oc) and np.array_equal(np_(reg), orr)
+        assert (fake is None) if not want_fake else np_(fake).tobytes() == of.tobytes()
+    y = pwlq.dequantize2(codes, reg, bits, dev(om), dev(p1), dev(p2), layout=layout,
+                         row_offsets=dev(ro))
+    assert np_(y).tobytes() == of.tobytes()
+    assert pwlq.device_status() == 0
+
+
+@pytest.mark.parametrize("bits,layout", [(2, 1), (4, 1), (6, 0)])
+@pytest.mark.parametrize("name", sorted(multi_layouts()))
+def test_quantize3_dequantize3_layouts(pwlq, oracle, name, bits, layout):
+    x, ro = make(multi_layouts()[name], 22)
+    om = oracle.absmax(x, ro)
+    om[5::13] = 0.0
+    p = breakpoints(om, 3, 6)
+    oc, orr, of = oracle.quantize3(x, bits, om, p, layout=layout, row_offsets=ro)
+    for want_fake in (True, False):
+        codes, reg, fake = pwlq.quantize3(dev(x), bits, dev(om), dev(p), layout=layout,
+                                          row_offsets=dev(ro), want_fake=want_fake)
+        assert np.array_equal(np_(codes), oc) and np.array_equal(np_(reg), orr)
+        assert (fake is None) if not want_fake else np_(fake).tobytes() == of.tobytes()
+    y = pwlq.dequantize3(codes, reg, bits, dev(om), dev(p), layout=layout, row_offsets=dev(ro))
+    assert np_(y).tobytes() == of.tobytes()
+    assert pwlq.device_status() == 0
+
+
+@pytest.mark.parametrize("C,n", [(600, 8), (3, 4095), (3, 4097), (2, 65537), (1, 300001), (380, 11)])
+def test_multi_breakpoint_dense_rows_around_the_span(pwlq, oracle, C, n):
+    rng = np.random.default_rng(C + n)
+    x = (rng.standard_normal((C, n)) * rng.uniform(0.01, 3.0, (C, 1))).astype(np.float32)
+    om = oracle.absmax(x)
+    p = breakpoints(om, 3, 7)
+    oc, orr, of = oracle.quantize3(x, 4, om, p, layout=1)
+    codes, reg, fake = pwlq.quantize3(dev(x), 4, dev(om), dev(p), layout=1, want_fake=True)
+    assert np.array_equal(np_(codes), oc) and np.array_equal(np_(reg), orr)
+    assert np_(fake).tobytes() == of.tobytes()
+    y = pwlq.dequantize3(codes, reg, 4, dev(om), dev(p), C=C, n=n, layout=1)
+    assert np_(y).tobytes() == of.tobytes()
+    p1, p2 = np.ascontiguousarray(p[:, 0]), np.ascontiguousarray(p[:, 1])
+    oc, orr, of = oracle.quantize2(x, 4, om, p1, p2, layout=1)
+    codes, reg, fake = pwlq.quantize2(dev(x), 4, dev(om), dev(p1), dev(p2), layout=1, want_fake=True)
+    assert np.array_equal(np_(codes), oc) and np.array_equal(np_(reg), orr)
+    assert np_(fake).tobytes() == of.tobytes()
+    y = pwlq.dequantize2(codes, reg, 4, dev(om), dev(p1), dev(p2), C=C, n=n, layout=1)
+    assert np_(y).tobytes() == of.tobytes()
+    assert pwlq.device_status() == 0
