@@ -392,9 +392,11 @@ class DevicePath:
         else: torch.cuda.synchronize()
         return np.array([[ev[j].elapsed_time(ev[j + 1]) for j in range(4)] for ev in events])
 
-    def streaming(self, reps=10):
+    def streaming(self, reps=10, multi=False):
         """The three HBM-bound kernels back to back on the workload's rows repeated until they
-        exceed L2 three times over (no eviction pass needed, no cold first wave per launch)."""
+        exceed L2 three times over (no eviction pass needed, no cold first wave per launch).
+        multi: also the three-breakpoint quantize / dequantize (signed scheme) on the same rows,
+        with breakpoints at 0.2 / 0.45 / 0.75 of every row's range."""
         torch, pwlq, w = self.torch, self.pwlq, self.w
         copies = max(1, -(-(3 * L2_BYTES) // (w.total * 4)))
         ro_b = None                                  # equally long rows stay a dense matrix
@@ -443,6 +445,20 @@ class DevicePath:
 
         for name, (fn, nbytes) in calls.items():
             out[name] = {"gbs": nbytes / (timed(fn, reps) * 1e-3) / 1e9}
+        if multi and not self.unsigned:
+            p3_b = torch.stack([m_b * 0.2, m_b * 0.45, m_b * 0.75], dim=1).contiguous()
+            reg_b = torch.empty((tot_b + 3) // 4, dtype=torch.uint8, device=self.dev)
+            io3 = tot_b * 4 + codes_b.numel() + reg_b.numel()
+            tcalls = {
+                "quantize3": lambda: pwlq.quantize3(x_b, self.bits, m_b, p3_b, layout=self.layout,
+                                                    row_offsets=ro_b, out=(codes_b, reg_b, None)),
+                "dequantize3": lambda: pwlq.dequantize3(codes_b, reg_b, self.bits, m_b, p3_b,
+                                                        C=copies * w.C, n=self.dense_n,
+                                                        layout=self.layout, row_offsets=ro_b, out=y_b),
+            }
+            out["three_breakpoints"] = {
+                name: {"gbs": io3 / (timed(fn, reps) * 1e-3) / 1e9} for name, fn in tcalls.items()}
+            del p3_b, reg_b
         if self.dense_n is None or self.dense_n < 4096:
             # several rows per span of 4096 values: the same calls with the layout's row maps
             # built once (pwlq_rowmap_build) instead of inside every kernel
@@ -494,6 +510,8 @@ def add_fracs(s, hbm):
         for k in STREAM_KEYS:
             if k in d:
                 d[k]["frac"] = d[k]["gbs"] / hbm
+    for v in s.get("three_breakpoints", {}).values():
+        v["frac"] = v["gbs"] / hbm
     return s
 
 
@@ -560,6 +578,9 @@ def extras(torch, pwlq, path: DevicePath, flush, hbm, K2=32):
         t = timed_call(torch, lambda: pwlq.quantize3(x, bits, m, s3["p"], layout=1,
                                                      out=(c3, g3, None), **kw), flush)
         out["quantize3"] = {"ms": t, "hbm_cold_frac": nb / (t * 1e-3) / 1e9 / hbm}
+        t = timed_call(torch, lambda: pwlq.dequantize3(c3, g3, bits, m, s3["p"], C=w.C,
+                                                       n=path.dense_n, layout=1, out=y, **kw), flush)
+        out["dequantize3"] = {"ms": t, "hbm_cold_frac": nb / (t * 1e-3) / 1e9 / hbm}
         del c3, g3
         # the pair search on one long row (a tensor quantized per layer): tiles of 8192 values
         wl = W.relu_activation()
@@ -730,7 +751,7 @@ def run_ours(args, rank, world, local_rank):
                        "fma.rn.f32": fp.run(torch, 0)}
         peak_measured = peak_detail["fma.rn.f32x2"]
         if not unsigned:
-            streaming = path.streaming()
+            streaming = path.streaming(multi=True)
             if path.dense_n is None or path.dense_n < 4096:
                 # the step's three streaming calls as single cold launches, given row maps built
                 # once for the layout (the step itself uses the plain calls)

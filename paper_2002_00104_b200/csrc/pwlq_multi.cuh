@@ -33,12 +33,12 @@ __device__ __forceinline__ Params3 make_params3(float m, float p1, float p2, flo
 }
 
 // Rows a span's stage holds constants for in the producer / consumer kernels; spans with more
-// rows -- rows of fewer than 16 values on average -- are marked slow.  A row takes four 128-bit
+// rows -- rows of fewer than 26 values on average -- are marked slow.  A row takes four 128-bit
 // records, one per region r: (z_r, L / range_r, step_r, aux_r) with aux_0 = m and aux_1 = the
 // sign mask 0x80000000, so that a consumer fetches what a value needs with one shared-memory read
 // indexed by the value's region.  A row with m <= 0 (or a NaN) is stored as zeros: every value
 // then comes out as level 0 of region 0, magnitude 0, no sign -- the zeros such a row delivers.
-constexpr int kMultiSlots = 256;
+constexpr int kMultiSlots = 160;
 __device__ __forceinline__ void store_row_consts_multi(float4* q, int slot, float m, float p1,
                                                        float p2, float p3, float Lf) {
     const Params3 P = make_params3(m, p1, p2, p3, Lf);

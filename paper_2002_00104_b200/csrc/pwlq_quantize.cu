@@ -958,6 +958,10 @@ dequantize_map_kernel(const uint8_t* __restrict__ codes, const uint8_t* __restri
 // pass; a value's constants are one shared-memory read indexed by its region.  The region index 0..3 takes two bits per value (16 bits per lane and pass).
 // Whole spans with a usable map take the form below; the tensor's last, partial span and spans
 // the map cannot describe go value by value with a lookup in global memory.
+// Two stages and four CTAs per SM (three stages were no faster: 0.41 / 0.36 of the copy peak with
+// three / two CTAs per SM against 0.45).
+constexpr int kMultiStages = 2;
+constexpr int kMultiCtasPerSm = 4;
 template <bool DATA>
 struct MultiStage {
     alignas(128) float data[DATA ? kMapSpan : 4];
@@ -1117,7 +1121,7 @@ __device__ __forceinline__ void quantize_multi_slow(const QuantizeMultiCtx& g, c
 // P3: the rows have a third breakpoint.  x, codes, region2 and fake are vector-aligned (the
 // launcher sends everything else to the element-wise kernel).
 template <bool PACKED, bool WANT_FAKE, bool P3>
-__global__ void __launch_bounds__(kMapThreads, 3)
+__global__ void __launch_bounds__(kMapThreads, kMultiCtasPerSm)
 quantize_multi_kernel(const float* __restrict__ x, Rows rows, int64_t total, int bits,
                       const float* __restrict__ m, BreakPts bp, uint8_t* __restrict__ codes,
                       uint8_t* __restrict__ region2, float* __restrict__ fake,
@@ -1125,13 +1129,13 @@ quantize_multi_kernel(const float* __restrict__ x, Rows rows, int64_t total, int
     typedef MultiStage<true> Stage;
     extern __shared__ __align__(128) unsigned char smem_raw[];
     Stage* st = reinterpret_cast<Stage*>(smem_raw);
-    __shared__ uint64_t full_bar[kMapStages], empty_bar[kMapStages];
+    __shared__ uint64_t full_bar[kMultiStages], empty_bar[kMultiStages];
     const float Lf = (float)((1 << (bits - 1)) - 1);
     const int64_t nspans = (total + kMapSpan - 1) / kMapSpan;
     const int64_t first = blockIdx.x * spans_per_cta, last = min(first + spans_per_cta, nspans);
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     if (threadIdx.x == 0) {
-        for (int s = 0; s < kMapStages; ++s) {
+        for (int s = 0; s < kMultiStages; ++s) {
             mbar_init(&full_bar[s], 2);            // the data (or its stand-in) and the map
             mbar_init(&empty_bar[s], kMapConsumers);
         }
@@ -1147,7 +1151,7 @@ quantize_multi_kernel(const float* __restrict__ x, Rows rows, int64_t total, int
         prod.in = RowInputs{m, bp.p2, bp.p1, bp.p3, nullptr};
         prod.Lf = Lf;
         prod.pstride = bp.stride;
-        for (int64_t span = first; span < last && span < first + kMapStages; ++span) {
+        for (int64_t span = first; span < last && span < first + kMultiStages; ++span) {
             const unsigned bytes = q_bulk_bytes(span, total, 1);
             if (bytes != 0 && lane == 0) {
                 mbar_expect_tx(&full_bar[span - first], bytes);
@@ -1157,13 +1161,13 @@ quantize_multi_kernel(const float* __restrict__ x, Rows rows, int64_t total, int
         prod.request(warp_row_of(rows, first * kMapSpan), true);
         int64_t it = 0;
         for (int64_t span = first; span < last; ++span, ++it) {
-            const int s = (int)(it % kMapStages);
-            const unsigned use = (unsigned)(it / kMapStages);
+            const int s = (int)(it % kMultiStages);
+            const unsigned use = (unsigned)(it / kMultiStages);
             if (use > 0 && !mbar_wait(&empty_bar[s], (use - 1) & 1u)) {
                 // never expected: report, let the copies of the earlier spans land, and leave
                 if (lane == 0) atomicOr(&g_quantize_timeout, 1);
-                for (int64_t j = it - 1; j >= 0 && j > it - 1 - kMapStages; --j)
-                    mbar_wait(&full_bar[j % kMapStages], (unsigned)(j / kMapStages) & 1u);
+                for (int64_t j = it - 1; j >= 0 && j > it - 1 - kMultiStages; --j)
+                    mbar_wait(&full_bar[j % kMultiStages], (unsigned)(j / kMultiStages) & 1u);
                 return;
             }
             const int64_t span_beg = span * kMapSpan, span_end = min(span_beg + kMapSpan, total);
@@ -1190,8 +1194,8 @@ quantize_multi_kernel(const float* __restrict__ x, Rows rows, int64_t total, int
     const int li0 = warp * (kMapSpan / kMapConsumers) + lane * 8;     // pass c: li0 + 256 c
     int64_t it = 0;
     for (int64_t span = first; span < last; ++span, ++it) {
-        const int s = (int)(it % kMapStages);
-        const unsigned use = (unsigned)(it / kMapStages);
+        const int s = (int)(it % kMultiStages);
+        const unsigned use = (unsigned)(it / kMultiStages);
         if (!mbar_wait_relaxed(&full_bar[s], use & 1u)) {
             if (lane == 0) atomicOr(&g_quantize_timeout, 1);
             return;
@@ -1259,14 +1263,14 @@ __device__ __forceinline__ float dequantize_multi_value(uint32_t code, int r, co
 }
 
 template <bool PACKED, bool P3>
-__global__ void __launch_bounds__(kMapThreads, 3)
+__global__ void __launch_bounds__(kMapThreads, kMultiCtasPerSm)
 dequantize_multi_kernel(const uint8_t* __restrict__ codes, const uint8_t* __restrict__ region2,
                         Rows rows, int64_t total, int bits, const float* __restrict__ m,
                         BreakPts bp, float* __restrict__ y, int64_t spans_per_cta) {
     typedef MultiStage<false> Stage;
     extern __shared__ __align__(128) unsigned char smem_raw[];
     Stage* st = reinterpret_cast<Stage*>(smem_raw);
-    __shared__ uint64_t full_bar[kMapStages], empty_bar[kMapStages];
+    __shared__ uint64_t full_bar[kMultiStages], empty_bar[kMultiStages];
     const int qmask = (1 << (bits - 1)) - 1;
     const float Lf = (float)qmask;
     const int rmax = P3 ? 3 : 2;
@@ -1275,7 +1279,7 @@ dequantize_multi_kernel(const uint8_t* __restrict__ codes, const uint8_t* __rest
     const int64_t first = blockIdx.x * spans_per_cta, last = min(first + spans_per_cta, nspans);
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     if (threadIdx.x == 0) {
-        for (int s = 0; s < kMapStages; ++s) {
+        for (int s = 0; s < kMultiStages; ++s) {
             mbar_init(&full_bar[s], 1);
             mbar_init(&empty_bar[s], kMapConsumers);
         }
@@ -1294,8 +1298,8 @@ dequantize_multi_kernel(const uint8_t* __restrict__ codes, const uint8_t* __rest
         prod.request(warp_row_of(rows, first * kMapSpan), true);
         int64_t it = 0;
         for (int64_t span = first; span < last; ++span, ++it) {
-            const int s = (int)(it % kMapStages);
-            const unsigned use = (unsigned)(it / kMapStages);
+            const int s = (int)(it % kMultiStages);
+            const unsigned use = (unsigned)(it / kMultiStages);
             if (use > 0 && !mbar_wait(&empty_bar[s], (use - 1) & 1u)) {
                 if (lane == 0) atomicOr(&g_quantize_timeout, 1);
                 return;
@@ -1314,8 +1318,8 @@ dequantize_multi_kernel(const uint8_t* __restrict__ codes, const uint8_t* __rest
     cur.load(codes, region2, first * kMapSpan, total, li0);
     int64_t it = 0;
     for (int64_t span = first; span < last; ++span, ++it) {
-        const int s = (int)(it % kMapStages);
-        const unsigned use = (unsigned)(it / kMapStages);
+        const int s = (int)(it % kMultiStages);
+        const unsigned use = (unsigned)(it / kMultiStages);
         const int64_t span_beg = span * kMapSpan;
         if (span + 1 < last) nxt.load(codes, region2, span_beg + kMapSpan, total, li0);
         if (!mbar_wait_relaxed(&full_bar[s], use & 1u)) {
@@ -1539,7 +1543,7 @@ cudaError_t launch_dequantize(const uint8_t* codes, const uint8_t* mask,
 // producer / consumer kernels; anything else, and layouts whose rows are so short that most spans
 // would have no usable map, through the element-wise kernels.
 static bool multi_by_maps(int64_t C, int64_t total, bool vec_ok) {
-    return vec_ok && total >= 16 * C;
+    return vec_ok && total >= 32 * C;
 }
 cudaError_t launch_quantize2(const float* x, const int64_t* row_offsets, int64_t C, int64_t n,
                              int64_t total, int bits, const float* m, const float* p1,
@@ -1555,7 +1559,7 @@ cudaError_t launch_quantize2(const float* x, const int64_t* row_offsets, int64_t
     Rows rows{row_offsets, C, n, n > 0 ? 1.0 / (double)n : 0.0, 0};
     const bool packed = (layout == 1 && bits <= 4);
     const int64_t nspans = (total + kQSpan - 1) / kQSpan;
-    const size_t msmem = sizeof(MultiStage<true>) * kMapStages;
+    const size_t msmem = sizeof(MultiStage<true>) * kMultiStages;
 #define PWLQ_LAUNCH_QM(PK, FK, P3)                                                                \
     do {                                                                                          \
         const SpanGrid g = span_grid((const void*)quantize_multi_kernel<PK, FK, P3>, kMapThreads, \
@@ -1586,7 +1590,7 @@ cudaError_t launch_dequantize2(const uint8_t* codes, const uint8_t* region2,
     Rows rows{row_offsets, C, n, n > 0 ? 1.0 / (double)n : 0.0, 0};
     const bool packed = (layout == 1 && bits <= 4);
     const int64_t nspans = (total + kQSpan - 1) / kQSpan;
-    const size_t msmem = sizeof(MultiStage<false>) * kMapStages;
+    const size_t msmem = sizeof(MultiStage<false>) * kMultiStages;
 #define PWLQ_LAUNCH_DM(PK, P3)                                                                    \
     do {                                                                                          \
         const SpanGrid g = span_grid((const void*)dequantize_multi_kernel<PK, P3>, kMapThreads,   \

@@ -184,9 +184,13 @@ def test_maps_of_another_layout_are_reported(pwlq):
 # ------------------------------------------------- two and three breakpoints on the same layouts
 def multi_layouts():
     out = dict(layouts())
-    # around the number of rows a span's stage holds constants for (384): 372 / 409 rows per span
-    out["rows_of_11"] = [11] * 1500
-    out["rows_of_10"] = [10] * 1700
+    # (layouts whose rows average fewer than 32 values go through the element-wise kernels)
+    # around the number of rows a span's stage holds constants for (160): 157 / 163 rows per
+    # span, followed by long rows so that the producer / consumer kernels take the layout
+    out["rows_of_26_then_long"] = [26] * 700 + [6000] * 30
+    out["rows_of_25_then_long"] = [25] * 700 + [6000] * 30
+    # spans without a usable map (too many rows, empty rows) between long rows
+    out["slow_spans_between_long_rows"] = [1] * 300 + [9] * 400 + [4096 * 5] + [3] * 100 + [0, 0, 20000]
     # long rows with short ones in between, a tail that is not a multiple of anything
     out["long_and_short"] = [9000, 13, 4096 * 3, 40, 41, 42, 12289, 5]
     return out
