@@ -679,7 +679,7 @@ def run_ours(args, rank, world, local_rank):
         # only the HBM-bound kernels back to back (a small case for a profiler: few launches)
         pwlq.absmax(path.x, row_offsets=path.ro, out=path.m)
         path.sout["p"].copy_(path.m * 0.3)
-        s = path.streaming(reps=args.reps)
+        s = path.streaming(reps=args.reps, multi=True)
         s["workload"] = w.name
         add_fracs(s, hbm)
         s["device_status"] = pwlq.device_status()
