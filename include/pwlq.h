@@ -249,6 +249,10 @@ int pwlq_dequantize_unsigned_ragged(const uint8_t* codes, const uint8_t* region_
  *               is a status word as in pwlq_search (bit 1 << PWLQ_ERR_INVALID_ARG: the ratios do
  *               not ascend, results of the launch are zeros)
  * A row with m = 0 or no values gets indices (0, 1), p1 = p2 = 0, error 0.
+ * pwlq_quantize2 / pwlq_dequantize2 (and the three-breakpoint forms below): breakpoints
+ * p1 <= p2 (<= p3) <= m per row; any alignment of the buffers is accepted, the streaming kernels
+ * run when x, codes, fake_out and y are 16-byte and region2 4-byte aligned.  A row with m <= 0
+ * gets codes 0, region 0 and values +0.
  * Asynchrony, ownership and error behaviour as for the one-breakpoint calls. */
 #define PWLQ_MAX_K2 64
 size_t pwlq_search2_workspace_bytes(int64_t C, int64_t max_n, int K);

@@ -182,3 +182,36 @@ def test_quantize3_dequantize3_ragged_after_search(pwlq, oracle):
     oc, orr, of = oracle.quantize3(x, 3, np_(m), np_(out["p"]), layout=1, row_offsets=ro)
     assert np.array_equal(np_(codes), oc) and np.array_equal(np_(reg), orr)
     assert np_(fake).tobytes() == of.tobytes() and np_(y).tobytes() == of.tobytes()
+
+
+@pytest.mark.parametrize("misalign", [0, 1, 4])
+def test_quantize3_dequantize3_with_buffers_off_their_vector_alignment(pwlq, oracle, misalign):
+    """Aligned buffers take the producer / consumer kernels, anything else the element-wise ones:
+    the same bytes either way, and nothing written outside the outputs."""
+    rng = np.random.default_rng(31 + misalign)
+    lengths = [5000, 13, 4096, 700, 701, 702, 9000, 3]
+    ro = np.concatenate([[0], np.cumsum(lengths)]).astype(np.int64)
+    total = int(ro[-1])
+    x = rng.laplace(0, 0.05, total).astype(np.float32)
+    m = oracle.absmax(x, ro)
+    p = (m[:, None] * np.array([0.15, 0.4, 0.8], dtype=np.float32)[None, :]).astype(np.float32)
+    bits, layout = 4, 1
+    xb = dev(np.concatenate([np.zeros(misalign, np.float32), x]))[misalign:]
+    nbytes = pwlq.code_bytes(total, bits, layout)
+    nreg = (total + 3) // 4
+    cbuf = torch.zeros(nbytes + 32, dtype=torch.uint8, device="cuda")
+    rbuf = torch.zeros(nreg + 32, dtype=torch.uint8, device="cuda")
+    fbuf = torch.zeros(total + 32, dtype=torch.float32, device="cuda")
+    ybuf = torch.zeros(total + 32, dtype=torch.float32, device="cuda")
+    codes, reg = cbuf[misalign:misalign + nbytes], rbuf[misalign:misalign + nreg]
+    fake, y = fbuf[misalign:misalign + total], ybuf[misalign:misalign + total]
+    pwlq.quantize3(xb, bits, dev(m), dev(p), layout=layout, row_offsets=dev(ro), out=(codes, reg, fake))
+    pwlq.dequantize3(codes, reg, bits, dev(m), dev(p), layout=layout, row_offsets=dev(ro), out=y)
+    torch.cuda.synchronize()
+    oc, orr, of = oracle.quantize3(x, bits, m, p, layout=layout, row_offsets=ro)
+    assert np.array_equal(np_(codes), oc) and np.array_equal(np_(reg), orr)
+    assert np_(fake).tobytes() == of.tobytes() and np_(y).tobytes() == of.tobytes()
+    for buf, n in ((cbuf, nbytes), (rbuf, nreg), (fbuf, total), (ybuf, total)):
+        assert float(buf[:misalign].float().abs().sum()) == 0
+        assert float(buf[misalign + n:].float().abs().sum()) == 0
+    assert pwlq.device_status() == 0
