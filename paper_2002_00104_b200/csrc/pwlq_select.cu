@@ -85,11 +85,11 @@ __device__ __forceinline__ void finish_row(int64_t row, int64_t n_row, double s2
     p_out[row] = (float)analytic_breakpoint((double)m[row], scale, model);
 }
 
-// One CTA per (row, tile): sums of x^2 and |x| over the tile.
+// One CTA per (row, tile): sums of x^2 and |x| over the tile.  The breakpoint itself is left to
+// select_finish_kernel, one thread per row: a Newton iteration in binary64 run by one thread of a
+// CTA while the other 127 wait took ten times as long as the sums.
 __global__ void __launch_bounds__(kSelThreads)
-moments_kernel(const float* __restrict__ x, Rows rows, int64_t tiles, double* __restrict__ partial,
-               const float* __restrict__ m, int model, float* __restrict__ p_out,
-               float* __restrict__ scale_out) {
+moments_kernel(const float* __restrict__ x, Rows rows, int64_t tiles, double* __restrict__ partial) {
     __shared__ double red[2][kSelThreads / 32];
     const int64_t row = blockIdx.x / tiles, tile = blockIdx.x - row * tiles;
     const int64_t beg = rows.begin(row), end = rows.begin(row + 1);
@@ -112,16 +112,12 @@ moments_kernel(const float* __restrict__ x, Rows rows, int64_t tiles, double* __
     if (threadIdx.x == 0) {
         s2 = red[0][0]; s1 = red[1][0];
         for (int w = 1; w < kSelThreads / 32; ++w) { s2 += red[0][w]; s1 += red[1][w]; }
-        if (tiles == 1) {
-            finish_row(row, end - beg, s2, s1, m, model, p_out, scale_out);
-        } else {
-            partial[2 * blockIdx.x] = s2;
-            partial[2 * blockIdx.x + 1] = s1;
-        }
+        partial[2 * blockIdx.x] = s2;
+        partial[2 * blockIdx.x + 1] = s1;
     }
 }
 
-// Long rows: the tiles' sums in ascending order, then the breakpoint.
+// The tiles' sums of every row in ascending order, then the breakpoint.
 __global__ void select_finish_kernel(Rows rows, int64_t tiles, const double* __restrict__ partial,
                                      const float* __restrict__ m, int model,
                                      float* __restrict__ p_out, float* __restrict__ scale_out) {
@@ -139,7 +135,7 @@ __global__ void select_finish_kernel(Rows rows, int64_t tiles, const double* __r
 
 size_t select_workspace_bytes(int64_t C, int64_t max_n) {
     const int64_t tiles = (max_n + kSelTile - 1) / kSelTile;
-    return tiles > 1 ? (size_t)(16 * C * tiles + 255) / 256 * 256 : 256;
+    return (size_t)(16 * C * tiles + 255) / 256 * 256;
 }
 
 cudaError_t launch_select_analytic(const float* x, const int64_t* row_offsets, int64_t C,
@@ -149,10 +145,9 @@ cudaError_t launch_select_analytic(const float* x, const int64_t* row_offsets, i
     Rows rows{row_offsets, C, n, n > 0 ? 1.0 / (double)n : 0.0, 0};
     const int64_t tiles = std::max<int64_t>(1, (max_n + kSelTile - 1) / kSelTile);
     double* partial = static_cast<double*>(workspace);
-    moments_kernel<<<(unsigned)(C * tiles), kSelThreads, 0, stream>>>(x, rows, tiles, partial, m,
-                                                                      model, p_out, scale_out);
+    moments_kernel<<<(unsigned)(C * tiles), kSelThreads, 0, stream>>>(x, rows, tiles, partial);
     cudaError_t e = cudaGetLastError();
-    if (e != cudaSuccess || tiles == 1) return e;
+    if (e != cudaSuccess) return e;
     select_finish_kernel<<<(unsigned)((C + 127) / 128), 128, 0, stream>>>(rows, tiles, partial, m,
                                                                           model, p_out, scale_out);
     return cudaGetLastError();
