@@ -108,8 +108,8 @@ __device__ __forceinline__ void store_row_consts(float4* qa, float4* qb, int slo
 // (chunk c = rows 32 c .. 32 c + 31, lane = row % 32); the two chunks from the current first row
 // on are held in registers.  Every member function is called by all 32 lanes.
 // NBP > 1: rows with two or three breakpoints.  in.p, in.lo and in.xi then point to p1, p2 and p3
-// (BC: a third breakpoint exists), read with stride pstride; the constants of a row are three
-// 128-bit words in qa (store_row_consts_multi), for at most kMultiSlots rows per span.
+// (BC: a third breakpoint exists), read with stride pstride; the constants of a row are four
+// 128-bit records in qa (store_row_consts_multi), for at most kMultiSlots rows per span.
 template <bool PARAMS, bool UNS, bool DEQ = false, bool BC = false, int NBP = 1>
 struct MapProducer {
     Rows rows;
