@@ -382,10 +382,19 @@ struct PreProducer {
         const int nr = __shfl_sync(0xffffffffu, pre_rows, j);
         if (lane < nr)
             store_row_consts<DEQ>(qa, qb, lane, UNS ? __fsub_rn(mn, lon) : mn, pn, lon, xn, bn, Lf);
-        for (int k = 32 + lane; k < nr; k += 32) {          // many short rows: fetched now
-            float mv, pv, lov, xv, bv;
-            load_inputs(fr + k, mv, pv, lov, xv, bv);
-            store_row_consts<DEQ>(qa, qb, k, UNS ? __fsub_rn(mv, lov) : mv, pv, lov, xv, bv, Lf);
+        // many short rows: fetched now, four rows per lane in flight (one row at a time, every 32
+        // rows exposed a round trip: MobileNetV2 rows, quantize 0.61 -> 0.67 of the copy peak)
+        constexpr int kB = 4;
+        for (int k0 = 32 + lane; k0 < nr; k0 += 32 * kB) {
+            float mv[kB], pv[kB], lov[kB], xv[kB], bv[kB];
+#pragma unroll
+            for (int u = 0; u < kB; ++u)
+                if (k0 + 32 * u < nr) load_inputs(fr + k0 + 32 * u, mv[u], pv[u], lov[u], xv[u], bv[u]);
+#pragma unroll
+            for (int u = 0; u < kB; ++u)
+                if (k0 + 32 * u < nr)
+                    store_row_consts<DEQ>(qa, qb, k0 + 32 * u, UNS ? __fsub_rn(mv[u], lov[u]) : mv[u],
+                                          pv[u], lov[u], xv[u], bv[u], Lf);
         }
         if (span + 1 < last) {
             if (span + 1 - pre_batch == 32) load_batch(span + 1, last);
