@@ -860,7 +860,11 @@ def run_ours(args, rank, world, local_rank):
                          "frac_of_measured_peak": achieved / peak_measured if peak_measured else None,
                          "lane_ops_issued_per_eval": issued, "center_share": center_share,
                          "frac_issued": issued * ec / (search_ms * 1e-3) / 1e12 / ALU_PEAK_TLANEOPS,
-                         "search_gelem_cand_per_s": ec / (search_ms * 1e-3) / 1e9},
+                         "search_gelem_cand_per_s": ec / (search_ms * 1e-3) / 1e9,
+                         # the same with the abs-max launch counted into the search's time
+                         "frac_with_absmax": LANE_OPS_PER_ELEM_CAND * ec /
+                             ((search_ms + stage_tot[0] / args.steps) * 1e-3) / 1e12 /
+                             ALU_PEAK_TLANEOPS},
             "hbm_stages": {
                 "peak_gbs": hbm, "peak_source": peak_kind,
                 "absmax": {"gbs": gbs(w.total * 4, stage_tot[0])},
