@@ -25,9 +25,11 @@
 //     r = fma(u, inv, 1.5 * 2^23); q = r - 1.5 * 2^23      round-half-even of u * inv
 //     e = fma(q, -s, u)                                      u = a - z;  e = -(v - a) up to rounding
 // which differs from the operation-by-operation sequence of Eq. 1 only in rounding; the relative
-// effect on a sum is about 3 L 2^-23 / sqrt(n).  Rows shorter than L^2 / 4 (and, for L > 3, rows
-// of fewer than 32 values, where few terms average the effect out) therefore use the unfused
-// reconstruction v = (q * s) + z, e = v - a instead; measured against binary64 sums of the
+// effect on a sum is about 3 L 2^-23 / sqrt(n).  Rows shorter than L^2 / 4, and all rows of fewer
+// than 32 values (few terms average the effect out; and when most of a short row's values sit on
+// levels -- the zeros of a ReLU output -- the sum is carried by two or three small errors whose
+// own rounding then shows at 1e-5 and more) therefore use the unfused reconstruction
+// v = (q * s) + z, e = v - a instead; measured against binary64 sums of the
 // operation-by-operation values, the fused form then stays within 2e-6 relative.
 #include <algorithm>
 #include <cstdint>
@@ -45,7 +47,7 @@ constexpr float kMagic = 12582912.0f;   // 1.5 * 2^23: adding it rounds to the n
 
 // Rows for which the fused error is accurate enough (see the file comment).
 __host__ __device__ inline bool fused_ok(int64_t n_row, int64_t L) {
-    return 4 * n_row >= L * L && n_row >= (L <= 3 ? 5 : 32);
+    return 4 * n_row >= L * L && n_row >= 32;
 }
 
 struct SearchArgs {

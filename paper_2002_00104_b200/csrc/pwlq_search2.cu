@@ -479,8 +479,9 @@ search2_kernel(Search2Args a) {
         if (lane == 0) CT[k] = d;
     }
     // The fused form's rounding shows in the sums of short rows (it grows like L / sqrt(n)); rows
-    // shorter than L^2 / 2 use the operation-by-operation form.
-    const bool fused = 2 * n_row >= (int64_t)a.levels * a.levels;
+    // shorter than L^2 / 2, and all rows of fewer than 32 values, use the operation-by-operation
+    // form.
+    const bool fused = 2 * n_row >= (int64_t)a.levels * a.levels && n_row >= 32;
     {
         int item = 0;                                  // (i, group of eight j) in a fixed order
         for (int i = 0; i < K - 1; ++i)

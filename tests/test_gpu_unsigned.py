@@ -223,3 +223,22 @@ def test_encode_host_unsigned_matches_oracle(pwlq, oracle, ragged):
     oc, ok, _ = oracle.quantize_u(xo, 4, olo, ohi, out["p"].numpy(), layout=1, row_offsets=ro)
     assert np.array_equal(out["codes"].numpy(), oc) and np.array_equal(out["mask"].numpy(), ok)
     assert pwlq.device_status() == 0
+
+
+@pytest.mark.parametrize("bits", [2, 3])
+def test_search_unsigned_short_rows_whose_values_mostly_sit_on_levels(pwlq, oracle, bits):
+    """Thousands of rows of 5 ... 31 values of a ReLU output moved off zero: most values of a row
+    equal its lower bound (error 0 under every candidate), so a sum is carried by a few small
+    errors and shows any rounding the search adds to the operation-by-operation sequence."""
+    rng = np.random.default_rng(40 + bits)
+    lens = rng.integers(5, 32, 6000).astype(np.int64)
+    ro = np.concatenate([[0], np.cumsum(lens)]).astype(np.int64)
+    total = int(ro[-1])
+    off = np.repeat(rng.uniform(-0.5, 0.5, lens.size), lens)
+    x = (np.maximum(rng.standard_normal(total), 0.0) + off).astype(np.float32)
+    lo, hi = oracle.minmax(x, ro)
+    ratios = W.ratio_grid(64)
+    got, status = run_search_u(pwlq, x, bits, ratios, lo, hi, row_offsets=ro, max_n=int(lens.max()))
+    assert status == 0
+    ora = oracle.search_u(x, bits, ratios, lo, hi, row_offsets=ro)
+    check_search(got, ora, ratios, (hi - lo).astype(np.float32), lens)
