@@ -421,3 +421,42 @@ def test_search_many_ragged_rows_of_every_class_with_full_tiles(pwlq, oracle, K)
         else:
             for k in ("p", "err", "idx", "sse"):
                 assert out[k].tobytes() == first[k].tobytes(), (rep, k)
+
+
+@pytest.mark.parametrize("kind", ["sparse", "relu_sparse", "on_a_grid"])
+@pytest.mark.parametrize("bits", [3, 4, 7, 8])
+def test_search_sums_carried_by_a_few_small_errors(pwlq, oracle, kind, bits):
+    """Pruned, ReLU-ed or already quantized values: under some candidates almost every value sits
+    on a level, and a sum is then orders of magnitude below n * step^2 / 12 and made of a few
+    small errors e_i.  Each e_i is a difference of two binary32 numbers of the size of m, known
+    to about one ulp of m on either side (the oracle rounds q * s and + z, the search rounds the
+    fused form once), so two correct evaluations may differ by sum 2 |e_i| ulp(m) <=
+    2 sqrt(n * SSE) * 2^-23 m in first order.  The 1e-5 relative bar holds where the sums have
+    their usual size; this test holds the search to the first-order bound elsewhere."""
+    rng = np.random.default_rng(bits * 7 + len(kind))
+    lens = rng.choice([32, 40, 64, 147, 512, 1000, 4096, 4608, 9000], 120).astype(np.int64)
+    ro = np.concatenate([[0], np.cumsum(lens)]).astype(np.int64)
+    total = int(ro[-1])
+    x = rng.laplace(0, 0.05, total).astype(np.float32)
+    if kind == "relu_sparse":
+        x = np.maximum(x, 0)
+    if kind == "on_a_grid":
+        x = (np.round(x * 64) / 64).astype(np.float32)
+    else:
+        x[rng.random(total) < np.repeat(rng.choice([0.5, 0.9, 0.99], lens.size), lens)] = 0.0
+    om = oracle.absmax(x, ro)
+    ratios = W.ratio_grid(64)
+    s = pwlq.search(dev(x), bits, dev(ratios), m=dev(om), row_offsets=dev(ro), max_n=int(lens.max()),
+                    want_sse=True)
+    ora = oracle.search(x, bits, ratios, row_offsets=ro)
+    sse = np_(s["sse"]).astype(np.float64)
+    o = ora["sse64"]
+    ulp_m = 2.0 ** -23 * om.astype(np.float64)[:, None]
+    n = lens[:, None].astype(np.float64)
+    bound = 1e-5 * o + 2.0 * np.sqrt(n * o) * ulp_m + n * ulp_m ** 2 + 2.0 ** -23 * o
+    assert np.all(np.abs(sse - o) <= bound)
+    # the chosen candidate is the oracle's, or as good within the same bound
+    rows = np.arange(lens.size)
+    gi, oi = np_(s["idx"]).astype(np.int64), ora["idx"].astype(np.int64)
+    assert np.all(np.abs(o[rows, gi] - o[rows, oi]) <= bound[rows, oi])
+    assert pwlq.device_status() == 0
