@@ -108,3 +108,54 @@ def test_random_layout(pwlq, oracle, seed):
     tol = 1e-5 * ora["sse64"] + lens[:, None] * (2.0 ** -23 * om[:, None]) ** 2 + 2.0 ** -23 * ora["sse64"]
     assert np.all(np.abs(sse - ora["sse64"]) <= tol)
     assert pwlq.device_status() == 0
+
+
+@pytest.mark.parametrize("seed", range(8))
+def test_random_layout_from_host_buffers(pwlq, oracle, seed):
+    """The host-buffer entry points (signed and one-sided) cut the rows into runs of their own; the
+    results must not depend on where the cuts fall."""
+    rng = np.random.default_rng(2000 + seed)
+    lens = random_layout(rng)
+    while lens.sum() == 0 or lens.sum() > 3_000_000:
+        lens = random_layout(rng)
+    total, C, max_n = int(lens.sum()), lens.size, int(lens.max())
+    ro = np.concatenate([[0], np.cumsum(lens)]).astype(np.int64)
+    one_sided = bool(seed & 1)
+    x = rng.laplace(0, 0.05, total).astype(np.float32)
+    if one_sided:
+        x = (np.maximum(x, 0) + np.float32(0.1)).astype(np.float32)
+    bits, layout, K = int(rng.integers(2, 9)), int(rng.integers(0, 2)), int(rng.choice([7, 64, 100]))
+    ratios = W.ratio_grid(K)
+
+    def pin(a):
+        return torch.from_numpy(np.ascontiguousarray(a)).pin_memory()
+
+    out = {k: torch.empty(C, dtype=torch.float32).pin_memory() for k in ("m", "p", "err", "lo", "hi")}
+    out["idx"] = torch.empty(C, dtype=torch.int32).pin_memory()
+    out["codes"] = torch.empty(pwlq.code_bytes(total, bits, layout), dtype=torch.uint8).pin_memory()
+    out["mask"] = torch.empty((total + 7) // 8, dtype=torch.uint8).pin_memory()
+    scratch = torch.empty(pwlq.encode_host_scratch_bytes(C, total, max_n, K), dtype=torch.uint8,
+                          device="cuda")
+    call = pwlq.encode_host_unsigned if one_sided else pwlq.encode_host
+    call(pin(x), pin(ro), C, max_n, bits, pin(ratios), out, layout, scratch)
+    torch.cuda.synchronize()
+    p = out["p"].numpy()
+    if one_sided:
+        olo, ohi = oracle.minmax(x, ro)
+        assert np.array_equal(out["lo"].numpy(), olo) and np.array_equal(out["hi"].numpy(), ohi)
+        ora = oracle.search_u(x, bits, ratios, olo, ohi, row_offsets=ro)
+        width = (ohi - olo).astype(np.float64)
+        oc, ok, _ = oracle.quantize_u(x, bits, olo, ohi, p, layout=layout, row_offsets=ro)
+    else:
+        om = oracle.absmax(x, ro)
+        assert np.array_equal(out["m"].numpy(), om)
+        ora = oracle.search(x, bits, ratios, row_offsets=ro)
+        width = om.astype(np.float64)
+        oc, ok, _ = oracle.quantize(x, bits, om, p, layout=layout, row_offsets=ro)
+    o, rows = ora["sse64"], np.arange(C)
+    gi, oi = out["idx"].numpy().astype(np.int64), ora["idx"].astype(np.int64)
+    tol = 1e-5 * o[rows, oi] + lens * (2.0 ** -23 * width) ** 2
+    assert np.all(np.abs(o[rows, gi] - o[rows, oi]) <= tol)      # the oracle's choice, or a near-tie
+    assert np.array_equal(out["codes"].numpy(), oc) and np.array_equal(out["mask"].numpy(), ok)
+    assert pwlq.encode_host_status(scratch, C, total, max_n, K) == 0
+    assert pwlq.device_status() == 0
