@@ -16,6 +16,7 @@ NVCC_FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a", "-O3", "-std=c++17", "-lineinfo",
     "-fmad=false",            # no implicit FMA contraction: every fused op is an explicit fmaf
     "--shared", "-Xcompiler", "-fPIC", "-cudart", "static",
+    "--threads", "0",         # the source files are compiled side by side
 ]
 
 

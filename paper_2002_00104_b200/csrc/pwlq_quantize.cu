@@ -383,7 +383,8 @@ quantize_map_kernel(const float* __restrict__ x, Rows rows, int64_t total, int b
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     if (threadIdx.x == 0) {
         for (int s = 0; s < kMapStages; ++s) {
-            mbar_init(&full_bar[s], 2);            // the data (or its stand-in) and the map
+            // the data (or its stand-in) and the map; PRE: and the rows' constants
+            mbar_init(&full_bar[s], PRE ? 3 : 2);
             mbar_init(&empty_bar[s], kMapConsumers);
         }
         fence_barrier_init();
@@ -421,12 +422,14 @@ quantize_map_kernel(const float* __restrict__ x, Rows rows, int64_t total, int b
                 __syncwarp();
                 if (lane == 0) mbar_arrive(&full_bar[s]);
             }
-            prod.build(st[s].qa, QB ? st[s].qb : nullptr, span, last);
-            __syncwarp();
+            // the map travels while the constants are computed
             if (lane == 0) {
                 mbar_expect_tx(&full_bar[s], (unsigned)sizeof(SpanRowMap));
                 bulk_copy_g2s(&st[s].map, maps + span, (unsigned)sizeof(SpanRowMap), &full_bar[s]);
             }
+            prod.build(st[s].qa, QB ? st[s].qb : nullptr, span, last);
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&full_bar[s]);
         }
         return;
     }
@@ -854,7 +857,7 @@ dequantize_map_kernel(const uint8_t* __restrict__ codes, const uint8_t* __restri
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     if (threadIdx.x == 0) {
         for (int s = 0; s < kMapStages; ++s) {
-            mbar_init(&full_bar[s], 1);
+            mbar_init(&full_bar[s], PRE ? 2 : 1);  // PRE: the map and the rows' constants
             mbar_init(&empty_bar[s], kMapConsumers);
         }
         fence_barrier_init();
@@ -880,12 +883,13 @@ dequantize_map_kernel(const uint8_t* __restrict__ codes, const uint8_t* __restri
                     mbar_wait(&full_bar[j % kMapStages], (unsigned)(j / kMapStages) & 1u);
                 return;
             }
-            prod.build(st[s].qa, QB ? st[s].qb : nullptr, span, last);
-            __syncwarp();
-            if (lane == 0) {
+            if (lane == 0) {                       // the map travels while the constants are computed
                 mbar_expect_tx(&full_bar[s], (unsigned)sizeof(SpanRowMap));
                 bulk_copy_g2s(&st[s].map, maps + span, (unsigned)sizeof(SpanRowMap), &full_bar[s]);
             }
+            prod.build(st[s].qa, QB ? st[s].qb : nullptr, span, last);
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&full_bar[s]);
         }
         return;
     }
