@@ -1409,15 +1409,16 @@ static int64_t device_slots(const void* kernel, int threads, size_t smem) {
 
 // Grid and spans per CTA.  The register-only dequantize kernel for very long dense rows runs a
 // persistent grid, one CTA per slot of the device, that walks the spans with a stride.  The
-// producer / consumer kernels walk consecutive spans, handed out in blocks of at most 32, about
-// four per slot: a block should be long enough to pay for the producer's start (finding its first
-// row), and short enough for the hardware scheduler to even out what differs between spans.
+// producer / consumer kernels walk consecutive spans, handed out in blocks of at most
+// kSpansPerBlockMax, about two per slot when the input is small: a block should be long enough to
+// pay for the producer's start (finding its first row), and short enough for the hardware
+// scheduler to even out what differs between spans.
 struct SpanGrid { unsigned grid; int64_t per_cta; };
 static SpanGrid span_grid(const void* kernel, int threads, size_t smem, int64_t nspans, bool table) {
     const int64_t slots = device_slots(kernel, threads, smem);
     if (!table) return SpanGrid{(unsigned)std::min(nspans, slots), 0};
-    const int64_t per_cta =
-        std::min<int64_t>(std::max<int64_t>((nspans + 4 * slots - 1) / (4 * slots), 1), 32);
+    const int64_t per_cta = std::min<int64_t>(
+        std::max<int64_t>((nspans + 2 * slots - 1) / (2 * slots), 1), kSpansPerBlockMax);
     return SpanGrid{(unsigned)((nspans + per_cta - 1) / per_cta), per_cta};
 }
 

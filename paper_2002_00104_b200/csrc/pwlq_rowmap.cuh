@@ -33,6 +33,7 @@
 namespace pwlq {
 
 constexpr int kMapSpan = 4096;                 // values per span
+constexpr int kSpansPerBlockMax = 11;          // consecutive spans one CTA walks, at most
 constexpr int kMapWords = kMapSpan / 32;
 constexpr int kMapRounds = 17;                 // rounds of 32 rows the producer looks at per span
 constexpr int kMapSlots = kMapRounds * 32;     // rows a map can describe (rows of >= 8 values fit)
