@@ -581,6 +581,10 @@ __device__ __forceinline__ void dequantize8(uint32_t w0, uint32_t w1, uint32_t m
     const uint32_t rep = (uint32_t)qmask * 0x01010101u;
     const uint32_t e0 = w0 & rep;
     const uint32_t e1 = (PACKED ? (w0 >> 4) : w1) & rep;
+    // the sign bit of the word's last code moved to bit 31 (sign_shift >= 28 for nibble codes,
+    // >= 24 for byte codes)
+    const uint32_t sw0 = w0 << (sign_shift - (PACKED ? 28 : 24));
+    const uint32_t sw1 = w1 << (sign_shift - (PACKED ? 28 : 24));
 #pragma unroll
     for (int t = 0; t < 8; ++t) {
         const bool second = TWO && t >= split;
@@ -592,95 +596,18 @@ __device__ __forceinline__ void dequantize8(uint32_t w0, uint32_t w1, uint32_t m
         const uint32_t sel = 0x7650u | (uint32_t)(PACKED ? (t >> 1) : (t & 3));
         const bool tail = (mb & (1u << t)) != 0;
         const float q = __fsub_rn(__uint_as_float(__byte_perm(src, 0x4B400000u, sel)), 12582912.0f);
-        const float v = __fadd_rn(__fmul_rn(q, tail ? s2 : s1), tail ? p : 0.0f);
+        // both pieces, then one select (q s1 + 0 is q s1: nothing here is negative)
+        const float vt = __fadd_rn(__fmul_rn(q, s2), p);
+        const float v = tail ? vt : __fmul_rn(q, s1);
         // signed scheme: the code's sign bit, at bit 4 t + b - 1 (8 (t mod 4) + b - 1 for byte
         // codes) of its word, moved to bit 31
-        const uint32_t word = PACKED ? w0 : (t < 4 ? w0 : w1);
-        const int up = sign_shift - (PACKED ? 4 * t : 8 * (t & 3));
+        // (the run-time part of the shift is applied once per word, sw0 / sw1 below; what is left
+        // per value is a shift by a constant)
+        const uint32_t sw = PACKED ? sw0 : (t < 4 ? sw0 : sw1);
+        constexpr int kTop = PACKED ? 28 : 24;
+        const int up = kTop - (PACKED ? 4 * t : 8 * (t & 3));
         yv[t] = UNS ? __fadd_rn(v, lo)
-                    : __uint_as_float(__float_as_uint(v) | ((word << up) & 0x80000000u));
-    }
-}
-
-// Register-only form for dense rows of many spans: a persistent grid, one CTA per slot of the
-// device, walks the spans with a stride; the codes and region bits of a thread's next span are
-// requested before the current one is expanded.  A warp's 256 values of one pass lie in one row
-// (constants kept in registers from pass to pass) or in two (the row that follows is looked up
-// when the first one ends); the tensor's tail and rows with m = 0 go value by value.
-template <bool PACKED, bool UNS>
-__global__ void __launch_bounds__(kQThreads)
-dequantize_long_kernel(const uint8_t* __restrict__ codes, const uint8_t* __restrict__ mask, Rows rows,
-                       int64_t total, int bits, RowArrays A, float* __restrict__ y, int vec_codes,
-                       int vec_out) {
-    const unsigned full = 0xffffffffu;
-    const int qmask = UNS ? (1 << bits) - 1 : (1 << (bits - 1)) - 1;   // the level inside a code
-    const float Lf = (float)qmask;
-    const int sign_shift = 32 - bits;                 // moves a code's sign bit to bit 31
-    const int64_t nspans = (total + kQSpan - 1) / kQSpan;
-    const int64_t first = blockIdx.x, stride = gridDim.x;
-    CodeRegs<PACKED> cur, nxt;
-    RowState ws;                                    // the row a warp's pass starts in (warp-uniform)
-    cur.load(codes, mask, first * kQSpan, total, vec_codes);
-    for (int64_t span = first; span < nspans; span += stride) {
-        const int64_t span_beg = span * kQSpan;
-        if (span + stride < nspans) nxt.load(codes, mask, (span + stride) * kQSpan, total, vec_codes);
-#pragma unroll
-        for (int c = 0; c < kQChunks; ++c) {
-            const int64_t i0 = span_beg + chunk_offset(c);
-            const int cnt = (int)max((int64_t)0, min((int64_t)8, total - i0));
-            float yv[8];
-            const int64_t pass_beg = i0 - ((int)threadIdx.x & 31) * 8, pass_end = pass_beg + 256;
-            bool done = false;
-            if (pass_end <= total) {
-                ws.seek(rows, A, Lf, pass_beg);
-                if (ws.m > 0.0f) {
-                    if (ws.end >= pass_end) {
-                        dequantize8<PACKED, false, UNS>(cur.w0[c], cur.w1[c], cur.mb[c], 8, ws.P, ws.lo,
-                                                        ws.P, ws.lo, qmask, sign_shift, yv);
-                        done = true;
-                    } else {
-                        float mB = 0.0f, loB = 0.0f;
-                        PieceParams PB = ws.P;
-                        int64_t endB = 0;
-                        if (ws.next_row(rows, A, Lf, pass_end, mB, loB, PB, endB) && mB > 0.0f) {
-                            const int split = (int)max((int64_t)0, min((int64_t)8, ws.end - i0));
-                            dequantize8<PACKED, true, UNS>(cur.w0[c], cur.w1[c], cur.mb[c], split, ws.P,
-                                                           ws.lo, PB, loB, qmask, sign_shift, yv);
-                            ws.advance(mB, loB, PB, endB);
-                            done = true;
-                        }
-                    }
-                }
-            }
-            if (!__all_sync(full, done)) {
-                RowState rs;
-#pragma unroll
-                for (int t = 0; t < 8; ++t) {
-                    yv[t] = 0.0f;
-                    if (t < cnt) {
-                        rs.seek(rows, A, Lf, i0 + t);
-                        if (UNS) yv[t] = rs.lo;                    // a constant row delivers lo
-                        if (rs.m > 0.0f) {
-                            const uint32_t code = code_of<PACKED>(cur.w0[c], cur.w1[c], t);
-                            const int tail = (cur.mb[c] >> t) & 1;
-                            const int neg = !UNS && ((code >> (bits - 1)) & 1);
-                            const float q = (float)(code & qmask);
-                            float v = __fmul_rn(q, tail ? rs.P.s2 : rs.P.s1);
-                            v = __fadd_rn(v, tail ? rs.P.p : 0.0f);
-                            yv[t] = UNS ? __fadd_rn(v, rs.lo) : (neg ? -v : v);
-                        }
-                    }
-                }
-            }
-            if (cnt == 0) continue;
-            if (vec_out && cnt == 8) {
-                __stcs(reinterpret_cast<float4*>(y + i0), make_float4(yv[0], yv[1], yv[2], yv[3]));
-                __stcs(reinterpret_cast<float4*>(y + i0 + 4), make_float4(yv[4], yv[5], yv[6], yv[7]));
-            } else {
-                for (int t = 0; t < cnt; ++t) y[i0 + t] = yv[t];
-            }
-        }
-        cur = nxt;
+                    : __uint_as_float(__float_as_uint(v) | ((sw << up) & 0x80000000u));
     }
 }
 
@@ -1514,31 +1441,21 @@ cudaError_t launch_dequantize(const uint8_t* codes, const uint8_t* mask,
         else if (premap) PWLQ_LAUNCH_DEQUANTIZE_AS(PK, UN, false, BCF, true);                     \
         else             PWLQ_LAUNCH_DEQUANTIZE_AS(PK, UN, false, BCF, false);                    \
     } while (0)
-#define PWLQ_LAUNCH_DEQUANTIZE_LONG(PK, UN)                                                       \
-    do {                                                                                          \
-        const SpanGrid g = span_grid((const void*)dequantize_long_kernel<PK, UN>, kQThreads, 0,   \
-                                     nspans, false);                                              \
-        dequantize_long_kernel<PK, UN><<<g.grid, kQThreads, 0, stream>>>(                         \
-            codes, mask, rows, total, bits, A, y, aligned(codes, PK ? 4 : 8), aligned(y, 16));    \
-    } while (0)
-    // Dense rows of many spans stream through the register-only kernel (no row lookups worth
-    // speaking of); everything else, and every bias-corrected call, goes through the producer /
-    // consumer kernel.
+    // Every layout goes through the producer / consumer kernel; for dense rows of at least a span
+    // the map follows from the row length (LONG).  (A register-only kernel with a persistent grid
+    // used to take dense rows of 16 spans or more; once the per-value work of the inverse had
+    // shrunk, the producer / consumer kernel was faster there too: 0.89 against 0.73-0.82 of the
+    // copy peak on one row of 25.7 M values.)
     const bool bc = xi != nullptr;
-    const bool very_long = !bc && row_offsets == nullptr && n >= 16 * (int64_t)kMapSpan;
     const bool long_rows = row_offsets == nullptr && n >= kMapSpan;   // the map follows from n
     const unsigned char* premap = long_rows ? nullptr : static_cast<const unsigned char*>(rowmap);
-    if (very_long) {
-        if (packed) { if (lo) PWLQ_LAUNCH_DEQUANTIZE_LONG(true, true); else PWLQ_LAUNCH_DEQUANTIZE_LONG(true, false); }
-        else        { if (lo) PWLQ_LAUNCH_DEQUANTIZE_LONG(false, true); else PWLQ_LAUNCH_DEQUANTIZE_LONG(false, false); }
-    } else if (bc) {
+    if (bc) {
         if (packed) PWLQ_LAUNCH_DEQUANTIZE(true, false, true); else PWLQ_LAUNCH_DEQUANTIZE(false, false, true);
     } else if (lo) {
         if (packed) PWLQ_LAUNCH_DEQUANTIZE(true, true, false); else PWLQ_LAUNCH_DEQUANTIZE(false, true, false);
     } else {
         if (packed) PWLQ_LAUNCH_DEQUANTIZE(true, false, false); else PWLQ_LAUNCH_DEQUANTIZE(false, false, false);
     }
-#undef PWLQ_LAUNCH_DEQUANTIZE_LONG
 #undef PWLQ_LAUNCH_DEQUANTIZE
 #undef PWLQ_LAUNCH_DEQUANTIZE_AS
     return cudaGetLastError();
