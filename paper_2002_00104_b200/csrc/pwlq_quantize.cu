@@ -118,7 +118,9 @@ __device__ __forceinline__ uint32_t spread_to_bytes(uint32_t x) {
 //     r's bit patterns are summed at their code positions and the constant the eight exponent
 //     fields add up to is taken off once;
 //   - region bits and sign flags (x < 0, false for -0.0: the sign bit of x + 0.0) are gathered
-//     with one funnel shift each and spread to their positions once per eight values.
+//     with one funnel shift each and spread to their positions once per eight values;
+//   - the magnitude is formed negated (-a = max(-|x|, -m), one instruction), so that p - a and
+//     x + 0.0 are plain additions, done for two values at a time (add.rn.f32x2).
 // UNS: one-sided range, a = min(max(x - lo, 0), m), the code is the level itself and the delivered
 // value is v + lo.
 template <bool PACKED, bool WANT_FAKE, bool TWO, bool UNS>
@@ -129,40 +131,59 @@ __device__ __forceinline__ void quantize8(const float (&xv)[8], int split, float
                                           uint32_t& w1, uint32_t& mb, float (&yv)[8]) {
     constexpr uint32_t kR = 0x4B400000u;                  // bit pattern of 1.5 * 2^23
     uint32_t acc0 = 0, acc1 = 0, tails = 0, signs = 0;
+    // Two values at a time where only additions are involved: p - a as p + (-a) and x + 0.0 are
+    // packed additions (one issue slot for two values, each lane rounded as the scalar operation
+    // rounds); the products and the additions that follow them stay scalar, so that no product is
+    // ever fused with its addition.
 #pragma unroll
-    for (int u = 0; u < 8; ++u) {
-        const int t = 7 - u;                              // descending: bit t of tails / signs
-        const bool second = TWO && t >= split;
-        const float m = second ? mB : mA;
-        const float lo = second ? loB : loA;
-        const float p = second ? B.p : A.p;
-        const float inv1 = second ? B.inv1 : A.inv1;
-        const float ninv2 = -(second ? B.inv2 : A.inv2);
-        const float xi = xv[t];
-        const float a = UNS ? fminf(fmaxf(__fsub_rn(xi, lo), 0.0f), m) : fminf(fabsf(xi), m);
-        const float nu = __fsub_rn(p, a);                 // -(a - p); negative: tail piece
-        const uint32_t T = (uint32_t)((int32_t)__float_as_uint(nu) >> 31);   // all ones: tail
-        const uint32_t rc = __float_as_uint(__fadd_rn(__fmul_rn(a, inv1), 12582912.0f));
-        const uint32_t rt = __float_as_uint(__fadd_rn(__fmul_rn(nu, ninv2), 12582912.0f));
-        const uint32_t r = (rt & T) | (rc & ~T);
-        if (PACKED) acc0 += r << (4 * t);
-        else if (t < 4) acc0 += r << (8 * t);
-        else acc1 += r << (8 * (t - 4));
-        tails = __funnelshift_l(__float_as_uint(nu), tails, 1);
-        uint32_t sb = 0;
-        if (!UNS) {
-            sb = __float_as_uint(__fadd_rn(xi, 0.0f));
-            signs = __funnelshift_l(sb, signs, 1);
+    for (int u = 0; u < 8; u += 2) {
+        const int t1 = 7 - u, t0 = 6 - u;                 // descending: bit t of tails / signs
+        float na[2], pp[2], nuv[2], sbv[2] = {0.0f, 0.0f};
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+            const int t = h ? t1 : t0;
+            const bool second = TWO && t >= split;
+            const float m = second ? mB : mA;
+            const float lo = second ? loB : loA;
+            pp[h] = second ? B.p : A.p;
+            const float xi = xv[t];
+            // -a, a = min(|x|, m) resp. min(max(x - lo, 0), m)
+            na[h] = UNS ? -fminf(fmaxf(__fsub_rn(xi, lo), 0.0f), m) : fmaxf(-fabsf(xi), -m);
         }
-        if (WANT_FAKE) {
-            const uint32_t s1 = __float_as_uint(second ? B.s1 : A.s1);
-            const uint32_t s2 = __float_as_uint(second ? B.s2 : A.s2);
-            const float s = __uint_as_float((s2 & T) | (s1 & ~T));
-            const float z = __uint_as_float(__float_as_uint(p) & T);
-            const float qf = __fsub_rn(__uint_as_float(r), 12582912.0f);
-            const float v = __fadd_rn(__fmul_rn(qf, s), z);
-            yv[t] = UNS ? __fadd_rn(v, lo)
-                        : __uint_as_float(__float_as_uint(v) | (sb & 0x80000000u));
+        unpack2(add2(pack2(pp[0], pp[1]), pack2(na[0], na[1])), nuv[0], nuv[1]);   // -(a - p)
+        if (!UNS) unpack2(add2(pack2(xv[t0], xv[t1]), pack2(0.0f, 0.0f)), sbv[0], sbv[1]);
+#pragma unroll
+        for (int h = 1; h >= 0; --h) {
+            const int t = h ? t1 : t0;
+            const bool second = TWO && t >= split;
+            const float lo = second ? loB : loA;
+            const float p = pp[h];
+            const float ninv1 = -(second ? B.inv1 : A.inv1);
+            const float ninv2 = -(second ? B.inv2 : A.inv2);
+            const float nu = nuv[h];                      // negative: tail piece
+            const uint32_t T = (uint32_t)((int32_t)__float_as_uint(nu) >> 31);   // all ones: tail
+            const uint32_t rc = __float_as_uint(__fadd_rn(__fmul_rn(na[h], ninv1), 12582912.0f));
+            const uint32_t rt = __float_as_uint(__fadd_rn(__fmul_rn(nu, ninv2), 12582912.0f));
+            const uint32_t r = (rt & T) | (rc & ~T);
+            if (PACKED) acc0 += r << (4 * t);
+            else if (t < 4) acc0 += r << (8 * t);
+            else acc1 += r << (8 * (t - 4));
+            tails = __funnelshift_l(__float_as_uint(nu), tails, 1);
+            uint32_t sb = 0;
+            if (!UNS) {
+                sb = __float_as_uint(sbv[h]);
+                signs = __funnelshift_l(sb, signs, 1);
+            }
+            if (WANT_FAKE) {
+                const uint32_t s1 = __float_as_uint(second ? B.s1 : A.s1);
+                const uint32_t s2 = __float_as_uint(second ? B.s2 : A.s2);
+                const float s = __uint_as_float((s2 & T) | (s1 & ~T));
+                const float z = __uint_as_float(__float_as_uint(p) & T);
+                const float qf = __fsub_rn(__uint_as_float(r), 12582912.0f);
+                const float v = __fadd_rn(__fmul_rn(qf, s), z);
+                yv[t] = UNS ? __fadd_rn(v, lo)
+                            : __uint_as_float(__float_as_uint(v) | (sb & 0x80000000u));
+            }
         }
     }
     mb = tails;
