@@ -606,6 +606,20 @@ __device__ __forceinline__ void dequantize8(uint32_t w0, uint32_t w1, uint32_t m
     // >= 24 for byte codes)
     const uint32_t sw0 = w0 << (sign_shift - (PACKED ? 28 : 24));
     const uint32_t sw1 = w1 << (sign_shift - (PACKED ? 28 : 24));
+    // the levels as floats, two at a time (the subtraction of 1.5 * 2^23 is a packed addition)
+    float qv[8];
+#pragma unroll
+    for (int t = 0; t < 8; t += 2) {
+        float r[2];
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+            const int tt = t + h;
+            const uint32_t src = PACKED ? ((tt & 1) ? e1 : e0) : (tt < 4 ? e0 : e1);
+            const uint32_t sel = 0x7650u | (uint32_t)(PACKED ? (tt >> 1) : (tt & 3));
+            r[h] = __uint_as_float(__byte_perm(src, 0x4B400000u, sel));
+        }
+        unpack2(add2(pack2(r[0], r[1]), pack2(-12582912.0f, -12582912.0f)), qv[t], qv[t + 1]);
+    }
 #pragma unroll
     for (int t = 0; t < 8; ++t) {
         const bool second = TWO && t >= split;
@@ -613,10 +627,8 @@ __device__ __forceinline__ void dequantize8(uint32_t w0, uint32_t w1, uint32_t m
         const float p = second ? B.p : A.p;
         const float s1 = second ? B.s1 : A.s1;
         const float s2 = second ? B.s2 : A.s2;
-        const uint32_t src = PACKED ? ((t & 1) ? e1 : e0) : (t < 4 ? e0 : e1);
-        const uint32_t sel = 0x7650u | (uint32_t)(PACKED ? (t >> 1) : (t & 3));
         const bool tail = (mb & (1u << t)) != 0;
-        const float q = __fsub_rn(__uint_as_float(__byte_perm(src, 0x4B400000u, sel)), 12582912.0f);
+        const float q = qv[t];
         // both pieces, then one select (q s1 + 0 is q s1: nothing here is negative)
         const float vt = __fadd_rn(__fmul_rn(q, s2), p);
         const float v = tail ? vt : __fmul_rn(q, s1);
