@@ -1009,8 +1009,13 @@ __device__ __forceinline__ void quantize_multi_pass(const QuantizeMultiCtx& g, c
     const uint32_t inner = (word >> ((li & 31) + 1)) & 0x7Fu;       // starts at li+1 .. li+7
     MultiRow R;
     R.load(q, l);
-    const int sign_shift = 32 - g.bits;
-    uint32_t w0 = 0, w1 = 0, rw = 0;
+    // As in quantize8: the level sits in the low mantissa bits of rr (clamped to L as a float:
+    // 1.5 * 2^23 + L), so the rr patterns are summed at their code positions and the constant
+    // their exponent fields add up to is taken off once; the sign flags (sign bit of x + 0.0 under
+    // the row's mask) are gathered with one funnel shift each and spread to their positions once.
+    const uint32_t sign_unit = 1u << (g.bits - 1);
+    const float top = __fadd_rn(12582912.0f, g.Lf);                 // exact: L < 2^22
+    uint32_t acc0 = 0, acc1 = 0, rw = 0, signs = 0;
     float yv[8];
 #pragma unroll
     for (int t = 0; t < 8; ++t) {
@@ -1020,16 +1025,28 @@ __device__ __forceinline__ void quantize_multi_pass(const QuantizeMultiCtx& g, c
         const float a = fminf(fabsf(xi), R.m);
         const int r = (a > R.p1) + (a > R.p2) + (a > R.p3);
         const float4 c = R.rec[r];                                  // (z, L / range, step, -)
-        const float rr = __fadd_rn(__fmul_rn(__fsub_rn(a, c.x), c.y), 12582912.0f);
-        const float qf = fminf(__fsub_rn(rr, 12582912.0f), g.Lf);
-        const float v = __fadd_rn(__fmul_rn(qf, c.z), c.x);
+        const float rr = fminf(__fadd_rn(__fmul_rn(__fsub_rn(a, c.x), c.y), 12582912.0f), top);
         const uint32_t sign = __float_as_uint(__fadd_rn(xi, 0.0f)) & R.smask;
-        const uint32_t code = (sign >> sign_shift) | (uint32_t)(int)qf;
-        yv[t] = __uint_as_float(__float_as_uint(v) | sign);
-        if (PACKED) w0 |= code << (4 * t);
-        else if (t < 4) w0 |= code << (8 * t);
-        else w1 |= code << (8 * (t - 4));
+        signs = __funnelshift_l(sign, signs, 1);                    // value t ends up at bit 7 - t
+        if (PACKED) acc0 += __float_as_uint(rr) << (4 * t);
+        else if (t < 4) acc0 += __float_as_uint(rr) << (8 * t);
+        else acc1 += __float_as_uint(rr) << (8 * (t - 4));
+        if (WANT_FAKE) {
+            const float qf = __fsub_rn(rr, 12582912.0f);
+            const float v = __fadd_rn(__fmul_rn(qf, c.z), c.x);
+            yv[t] = __uint_as_float(__float_as_uint(v) | sign);
+        }
         rw |= (uint32_t)r << (2 * t);
+    }
+    signs = __brev(signs) >> 24;                                    // value t at bit t
+    uint32_t w0, w1 = 0;
+    if (PACKED) {
+        constexpr uint32_t kGarbage = (uint32_t)(0x4B400000ull * 0x11111111ull);
+        w0 = (acc0 - kGarbage) | spread_to_nibbles(signs) * sign_unit;
+    } else {
+        constexpr uint32_t kGarbage = (uint32_t)(0x4B400000ull * 0x01010101ull);
+        w0 = (acc0 - kGarbage) | spread_to_bytes(signs) * sign_unit;
+        w1 = (acc1 - kGarbage) | spread_to_bytes(signs >> 4) * sign_unit;
     }
     // span_beg is a multiple of the span: 32-bit offsets inside the span's slices of the outputs
     reinterpret_cast<uint16_t*>(g.region2 + (span_beg >> 2))[li >> 3] = (uint16_t)rw;
@@ -1303,16 +1320,37 @@ dequantize_multi_kernel(const uint8_t* __restrict__ codes, const uint8_t* __rest
                 const float4* rec = S.q + 4 * l;
                 uint32_t smask = __float_as_uint(rec[1].w);
                 float yv[8];
+                // the levels as floats without an integer conversion, two at a time, and the
+                // sign bits moved with one run-time shift per code word (as in dequantize8)
+                const uint32_t rep = (uint32_t)qmask * 0x01010101u;
+                const uint32_t e0 = w0 & rep;
+                const uint32_t e1 = (PACKED ? (w0 >> 4) : w1) & rep;
+                const uint32_t sw0 = w0 << (sign_shift - (PACKED ? 28 : 24));
+                const uint32_t sw1 = w1 << (sign_shift - (PACKED ? 28 : 24));
+                float qv[8];
+#pragma unroll
+                for (int t = 0; t < 8; t += 2) {
+                    float r[2];
+#pragma unroll
+                    for (int h = 0; h < 2; ++h) {
+                        const int tt = t + h;
+                        const uint32_t src = PACKED ? ((tt & 1) ? e1 : e0) : (tt < 4 ? e0 : e1);
+                        const uint32_t sel = 0x7650u | (uint32_t)(PACKED ? (tt >> 1) : (tt & 3));
+                        r[h] = __uint_as_float(__byte_perm(src, 0x4B400000u, sel));
+                    }
+                    unpack2(add2(pack2(r[0], r[1]), pack2(-12582912.0f, -12582912.0f)), qv[t], qv[t + 1]);
+                }
 #pragma unroll
                 for (int t = 0; t < 8; ++t) {
                     if (t > 0 && (inner & (1u << (t - 1)))) {
                         rec = S.q + 4 * (l + __popc(inner & ((1u << t) - 1u)));
                         smask = __float_as_uint(rec[1].w);
                     }
-                    const uint32_t code = code_of<PACKED>(w0, w1, t);
                     const float4 c = rec[min((int)((rw >> (2 * t)) & 3u), rmax)];   // (z, -, step, -)
-                    const float v = __fadd_rn(__fmul_rn((float)(int)(code & (uint32_t)qmask), c.z), c.x);
-                    yv[t] = __uint_as_float(__float_as_uint(v) | ((code << sign_shift) & smask));
+                    const float v = __fadd_rn(__fmul_rn(qv[t], c.z), c.x);
+                    const uint32_t sw = PACKED ? sw0 : (t < 4 ? sw0 : sw1);
+                    const int up = (PACKED ? 28 : 24) - (PACKED ? 4 * t : 8 * (t & 3));
+                    yv[t] = __uint_as_float(__float_as_uint(v) | ((sw << up) & smask));
                 }
                 float4* f = reinterpret_cast<float4*>(y + span_beg) + (li >> 2);
                 __stcs(f, make_float4(yv[0], yv[1], yv[2], yv[3]));
