@@ -77,6 +77,26 @@ def test_search_unsigned_dense(pwlq, oracle, bits, K, C, n):
     check_search(got, ora, ratios, (hi - lo).astype(np.float32), n)
 
 
+def test_search_unsigned_rows_of_a_hundred_values_at_eight_bits(pwlq, oracle):
+    """Many levels, few values: 255 levels per piece over rows of 65 .. 200 values.  Here a
+    single value that lands on the other of two neighbouring levels shows in the row's sum at the
+    1e-5 level, so the level has to be decided as Eq. 3 is evaluated operation by operation: the
+    product u * L / range rounded first, then rounded to the nearest level.  (A product that rounds
+    to an exact tie, x.5, while its unrounded value does not, goes to the other level when product
+    and rounding are fused; a randomized run met that case in a row of 116 values.)"""
+    rng = np.random.default_rng(424201)
+    lens = rng.integers(65, 201, 3000).astype(np.int64)
+    row_offsets = np.concatenate([[0], np.cumsum(lens)]).astype(np.int64)
+    x = (np.maximum(rng.standard_normal(int(lens.sum())), 0) + rng.uniform(-0.5, 0.5)).astype(np.float32)
+    lo, hi = oracle.minmax(x, row_offsets)
+    ratios = W.ratio_grid(64)
+    got, status = run_search_u(pwlq, x, 8, ratios, lo, hi, row_offsets=row_offsets,
+                               max_n=int(lens.max()))
+    assert status == 0
+    ora = oracle.search_u(x, 8, ratios, lo, hi, row_offsets=row_offsets)
+    check_search(got, ora, ratios, (hi - lo).astype(np.float32), lens)
+
+
 def test_search_unsigned_ragged_with_given_ranges(pwlq, oracle):
     w = W.small_mixed(seed=5, bits=4, K=64)
     x = np.abs(w.x).astype(np.float32)
