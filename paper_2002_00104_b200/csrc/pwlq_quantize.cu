@@ -44,7 +44,7 @@ struct RowArrays {
 };
 
 // The row a thread is currently in, with its constants in registers, looked up in global memory
-// (long dense rows: the register-only dequantize kernel; and spans without a usable row map).
+// (spans without a usable row map, and the tensor's last, partial span).
 struct RowState {
     int64_t beg = 0, end = 0;
     float m = 0.0f;                                // range width (abs-max, or hi - lo)
@@ -66,27 +66,6 @@ struct RowState {
         end = rows.begin(row + 1);
         load_range(A, row, m, lo);
         P = make_params(m, __ldg(A.p + row), Lf);
-    }
-    // Constants of the row that follows (dense rows), if that row reaches at least to need_end.
-    __device__ __forceinline__ bool next_row(const Rows& rows, const RowArrays& A, float Lf,
-                                             int64_t need_end, float& mB, float& loB,
-                                             PieceParams& PB, int64_t& endB) const {
-        if (rows.offsets || rows.n < need_end - end) return false;
-        const int64_t row = rows.dense_row(end);
-        if (row >= rows.C) return false;
-        endB = end + rows.n;
-        load_range(A, row, mB, loB);
-        PB = make_params(mB, __ldg(A.p + row), Lf);
-        return true;
-    }
-    // Moves on to the row that next_row() returned.
-    __device__ __forceinline__ void advance(float mB, float loB, const PieceParams& PB,
-                                            int64_t endB) {
-        beg = end;
-        end = endB;
-        m = mB;
-        lo = loB;
-        P = PB;
     }
 };
 
@@ -1405,16 +1384,13 @@ static int64_t device_slots(const void* kernel, int threads, size_t smem) {
     return ctas;
 }
 
-// Grid and spans per CTA.  The register-only dequantize kernel for very long dense rows runs a
-// persistent grid, one CTA per slot of the device, that walks the spans with a stride.  The
-// producer / consumer kernels walk consecutive spans, handed out in blocks of at most
-// kSpansPerBlockMax, about two per slot when the input is small: a block should be long enough to
-// pay for the producer's start (finding its first row), and short enough for the hardware
-// scheduler to even out what differs between spans.
+// Grid and spans per CTA.  The producer / consumer kernels walk consecutive spans, handed out in
+// blocks of at most kSpansPerBlockMax, about two per slot when the input is small: a block should
+// be long enough to pay for the producer's start (finding its first row), and short enough for
+// the hardware scheduler to even out what differs between spans.
 struct SpanGrid { unsigned grid; int64_t per_cta; };
-static SpanGrid span_grid(const void* kernel, int threads, size_t smem, int64_t nspans, bool table) {
+static SpanGrid span_grid(const void* kernel, int threads, size_t smem, int64_t nspans) {
     const int64_t slots = device_slots(kernel, threads, smem);
-    if (!table) return SpanGrid{(unsigned)std::min(nspans, slots), 0};
     const int64_t per_cta = std::min<int64_t>(
         std::max<int64_t>((nspans + 2 * slots - 1) / (2 * slots), 1), kSpansPerBlockMax);
     return SpanGrid{(unsigned)((nspans + per_cta - 1) / per_cta), per_cta};
@@ -1466,7 +1442,7 @@ cudaError_t launch_quantize(const float* x, const int64_t* row_offsets, int64_t 
     do {                                                                                          \
         const size_t msmem = sizeof(MapStage<true, FK || UN>) * kMapStages;                       \
         const SpanGrid g = span_grid((const void*)quantize_map_kernel<PK, FK, UN, LG, PR>,        \
-                                     kMapThreads, msmem, nspans, true);                           \
+                                     kMapThreads, msmem, nspans);                                 \
         quantize_map_kernel<PK, FK, UN, LG, PR><<<g.grid, kMapThreads, msmem, stream>>>(          \
             x, rows, total, bits, A, codes, mask, fake, vec_in, vec_fake, vec_codes, g.per_cta,   \
             premap);                                                                              \
@@ -1502,7 +1478,7 @@ cudaError_t launch_dequantize(const uint8_t* codes, const uint8_t* mask,
         const int vc = aligned(codes, PK ? 4 : 8), vo = aligned(y, 16);                           \
         const size_t msmem = sizeof(MapStage<false, UN || BCF>) * kMapStages;                     \
         const SpanGrid g = span_grid((const void*)dequantize_map_kernel<PK, UN, LG, BCF, PR>,     \
-                                     kMapThreads, msmem, nspans, true);                           \
+                                     kMapThreads, msmem, nspans);                                 \
         dequantize_map_kernel<PK, UN, LG, BCF, PR><<<g.grid, kMapThreads, msmem, stream>>>(       \
             codes, mask, rows, total, bits, A, y, vc, vo, g.per_cta, premap);                     \
     } while (0)
@@ -1556,7 +1532,7 @@ cudaError_t launch_quantize2(const float* x, const int64_t* row_offsets, int64_t
 #define PWLQ_LAUNCH_QM(PK, FK, P3)                                                                \
     do {                                                                                          \
         const SpanGrid g = span_grid((const void*)quantize_multi_kernel<PK, FK, P3>, kMapThreads, \
-                                     msmem, nspans, true);                                        \
+                                     msmem, nspans);                                              \
         quantize_multi_kernel<PK, FK, P3><<<g.grid, kMapThreads, msmem, stream>>>(                \
             x, rows, total, bits, m, bp, codes, region2, fake, g.per_cta);                        \
     } while (0)
@@ -1587,7 +1563,7 @@ cudaError_t launch_dequantize2(const uint8_t* codes, const uint8_t* region2,
 #define PWLQ_LAUNCH_DM(PK, P3)                                                                    \
     do {                                                                                          \
         const SpanGrid g = span_grid((const void*)dequantize_multi_kernel<PK, P3>, kMapThreads,   \
-                                     msmem, nspans, true);                                        \
+                                     msmem, nspans);                                              \
         dequantize_multi_kernel<PK, P3><<<g.grid, kMapThreads, msmem, stream>>>(                  \
             codes, region2, rows, total, bits, m, bp, y, g.per_cta);                              \
     } while (0)
